@@ -1,0 +1,419 @@
+"""Pins of the CPU oracle against things other than itself: brute force in
+plain Python loops, closed forms, invariants the paper fixes, and library
+routines for the textbook special cases.  No GPU."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import acache_oracle as orc
+from paper_2608_26140_b200 import workloads as wl
+
+
+def rnd(seed, *shape, std=1.0):
+    return np.random.default_rng(seed).standard_normal(shape) * std
+
+
+# ---------------------------------------------------------------- storage format
+def test_bf16_round_matches_library_cast():
+    a = np.random.default_rng(0).standard_normal(20000).astype(np.float32) * 3
+    # exact ties and specials of the rounding rule
+    ties = np.array([1.00390625, 1.01171875, -1.00390625, 0.0, 2.0 ** -130, 65280.0], np.float32)
+    a = np.concatenate([a, ties])
+    ref = torch.from_numpy(a).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(orc.f64_to_bf16_bits(a.astype(np.float64)), ref)
+    assert np.array_equal(wl.f32_to_bf16_bits(a), ref)
+    back = torch.from_numpy(ref.view(np.int16)).view(torch.bfloat16).double().numpy()
+    assert np.array_equal(orc.bf16_bits_to_f64(ref), back)
+    assert np.array_equal(wl.bf16_bits_to_f32(ref).astype(np.float64), back)
+
+
+# ---------------------------------------------------------------- Eq. 4-5 scoring
+def brute_scores(q, k, group, keep=None, k_ctx=None):
+    """Eq. 4-5 as explicit nested loops with math.exp (fp64 python floats)."""
+    m, H, d = len(q), len(q[0]), len(q[0][0])
+    keys = k if k_ctx is None else k_ctx
+    n_keys = len(keys)
+    lo, L = (0, len(k)) if keep is None else keep
+    s = [0.0] * L
+    for h in range(H):
+        kh = h // group
+        for kq in range(m):
+            z = []
+            for j in range(n_keys):
+                acc = 0.0
+                for i in range(d):
+                    acc += q[kq][h][i] * keys[j][kh][i]
+                z.append(acc / math.sqrt(d))
+            zmax = max(z)
+            e = [math.exp(t - zmax) for t in z]
+            den = sum(e)
+            for j in range(L):
+                s[j] += e[lo + j] / den
+    return s
+
+
+@pytest.mark.parametrize("m,H,Hkv,d,L", [(3, 2, 2, 4, 7), (4, 2, 1, 6, 5), (1, 1, 1, 2, 8), (2, 4, 2, 4, 3)])
+def test_score_brute_force(m, H, Hkv, d, L):
+    q = rnd(1, m, H, d)
+    k = rnd(2, L, Hkv, d)
+    s = orc.score_anchors(q, k)
+    ref = brute_scores(q.tolist(), k.tolist(), H // Hkv)
+    assert np.allclose(s, ref, rtol=1e-12, atol=1e-14)
+
+
+def test_score_full_context_normalisation_brute_force():
+    m, H, Hkv, d, L, T, l = 3, 2, 1, 4, 5, 11, 2
+    q = rnd(3, m, H, d)
+    kc = rnd(4, T, Hkv, d)
+    s = orc.score_anchors(q, kc[l:l + L], kc, l, norm_full=True)
+    ref = brute_scores(q.tolist(), kc[l:l + L].tolist(), H // Hkv, keep=(l, L), k_ctx=kc.tolist())
+    assert np.allclose(s, ref, rtol=1e-12)
+    # the affix columns plus the rest of each row carry all the mass
+    rest = brute_scores(q.tolist(), None, H // Hkv, keep=(0, l), k_ctx=kc.tolist())
+    rest2 = brute_scores(q.tolist(), None, H // Hkv, keep=(l + L, T - l - L), k_ctx=kc.tolist())
+    assert abs(sum(ref) + sum(rest) + sum(rest2) - H * m) < 1e-12
+    assert s.sum() < H * m
+    # affix == whole context: both normalisations coincide
+    s_a = orc.score_anchors(q, kc)
+    s_b = orc.score_anchors(q, kc, kc, 0, norm_full=True)
+    assert np.allclose(s_a, s_b, rtol=1e-13)
+
+
+def test_score_closed_forms_and_invariants():
+    m, H, Hkv, d, L = 5, 4, 2, 8, 13
+    k = rnd(5, L, Hkv, d)
+    # zero queries -> uniform attention -> s_j = H*m/L
+    s0 = orc.score_anchors(np.zeros((m, H, d)), k)
+    assert np.allclose(s0, H * m / L, rtol=1e-13)
+    q = rnd(6, m, H, d)
+    s = orc.score_anchors(q, k)
+    # every softmax row sums to one -> total mass H*m
+    assert abs(s.sum() - H * m) < 1e-10
+    assert np.all(s > 0)
+    # linear in the set of masked positions: duplicating each doubles s
+    s2 = orc.score_anchors(np.concatenate([q, q]), k)
+    assert np.allclose(s2, 2 * s, rtol=1e-13)
+    # additive over disjoint masked sets
+    sa = orc.score_anchors(q[:2], k) + orc.score_anchors(q[2:], k)
+    assert np.allclose(sa, s, rtol=1e-13)
+    # grouped-query == multi-head with each KV head replicated
+    s_mha = orc.score_anchors(q, np.repeat(k, H // Hkv, axis=1))
+    assert np.allclose(s_mha, s, rtol=1e-13)
+    # one key aligned with every query at large norm takes all the mass
+    qa = np.ones((m, H, d))
+    ka = rnd(7, L, Hkv, d) * 0.01
+    ka[4] = 50.0
+    sd = orc.score_anchors(qa, ka)
+    assert abs(sd[4] - H * m) < 1e-6 and sd.argmax() == 4
+    # permuting the affix keys permutes the scores
+    perm = np.random.default_rng(8).permutation(L)
+    assert np.allclose(orc.score_anchors(q, k[perm]), s[perm], rtol=1e-13)
+    # scaling by 1/sqrt(d): doubling d by zero padding must change the logits' scale
+    qp = np.concatenate([q, np.zeros_like(q)], -1)
+    kp = np.concatenate([k, np.zeros_like(k)], -1)
+    s_pad = orc.score_anchors(qp * math.sqrt(math.sqrt(2)), kp * math.sqrt(math.sqrt(2)))
+    assert np.allclose(s_pad, s, rtol=1e-12)
+
+
+# ---------------------------------------------------------------- Eq. 6 selection
+def brute_topk(s, K):
+    L = len(s)
+    sel = []
+    for j in range(L):
+        ahead = 0
+        for i in range(L):
+            if s[i] > s[j] or (s[i] == s[j] and i < j):
+                ahead += 1
+        if ahead < K:
+            sel.append(j)
+    return sel
+
+
+def test_topk_brute_force_and_edges():
+    g = np.random.default_rng(9)
+    for L in (1, 2, 7, 33, 100):
+        s = g.random(L).astype(np.float32)
+        s[g.integers(0, L, size=L // 3)] = s[0]          # ties
+        for K in sorted({0, 1, L // 2, max(L - 1, 0), L}):
+            A, tau, must, may = orc.select_topk(s, K)
+            assert A.tolist() == brute_topk(s.tolist(), K)
+            assert len(A) == K
+            if K:
+                assert tau == np.sort(s)[::-1][K - 1]
+                assert set(must.tolist()) <= set(A.tolist()) <= set(may.tolist())
+    # all equal -> lowest positions
+    A, *_ = orc.select_topk(np.full(10, 0.5, np.float32), 4)
+    assert A.tolist() == [0, 1, 2, 3]
+    # K = L -> identity, K = 0 -> empty
+    s = g.random(9).astype(np.float32)
+    assert orc.select_topk(s, 9)[0].tolist() == list(range(9))
+    assert orc.select_topk(s, 0)[0].size == 0
+    # a permutation of distinct scores permutes the set
+    s = g.permutation(50).astype(np.float32)
+    p = g.permutation(50)
+    A = orc.select_topk(s, 12)[0]
+    Ap = orc.select_topk(s[p], 12)[0]
+    assert sorted(p[Ap].tolist()) == A.tolist()
+    # largest values are the ones taken
+    assert set(A.tolist()) == set(np.argsort(-s)[:12].tolist())
+
+
+def test_k_from_ratio():
+    assert orc.k_from_ratio(512, 0.2) == 103
+    assert orc.k_from_ratio(2048, 0.2) == 410
+    assert orc.k_from_ratio(1024, 0.2) == 205
+    assert orc.k_from_ratio(128, 0.2) == 26
+    assert orc.k_from_ratio(10, 0.3) == 3          # 0.3*10 is not exactly 3 in binary
+    assert orc.k_from_ratio(100, 0.0) == 0
+    assert orc.k_from_ratio(100, 1.0) == 100
+    assert orc.k_from_ratio(100, 1e-4) == 1
+    assert orc.k_from_ratio(100, 1.5) == 100
+    for L in (1, 7, 512, 8192):
+        for r in (0.05, 0.1, 0.2, 0.35, 0.5):
+            K = orc.k_from_ratio(L, r)
+            assert (K - 1) < r * L + 1e-6 and K >= r * L - 1e-6
+
+
+# ---------------------------------------------------------------- layer pieces vs library routines
+def test_rmsnorm_vs_library_and_closed_form():
+    x = rnd(10, 6, 32)
+    g = 1 + 0.1 * rnd(11, 32)
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x), (32,), torch.from_numpy(g), 1e-5).numpy()
+    assert np.allclose(orc.rmsnorm(x, g, 1e-5), ref, rtol=1e-12)
+    c = np.full((1, 16), -3.0)
+    out = orc.rmsnorm(c, g[:16], 1e-5)
+    assert np.allclose(out, -g[:16] / math.sqrt(1 + 1e-5 / 9.0), rtol=1e-13)
+
+
+def test_silu_vs_library():
+    z = rnd(12, 1000) * 4
+    assert np.allclose(orc.silu(z), torch.nn.functional.silu(torch.from_numpy(z)).numpy(), rtol=1e-12, atol=1e-15)
+    assert orc.silu(np.zeros(1))[0] == 0.0
+
+
+def test_rope_properties():
+    d, H, T = 16, 3, 40
+    cos, sin = wl.rope_table(T, d, 1e4)
+    v = rnd(13, 5, H, d)
+    pos = np.array([0, 1, 7, 20, 39])
+    out = orc.rope(v, pos, cos, sin)
+    assert np.allclose(out[0], v[0], atol=1e-7)                                  # position 0: identity
+    assert np.allclose(np.linalg.norm(out, axis=-1), np.linalg.norm(v, axis=-1), rtol=1e-6)
+    q = rnd(14, 1, 1, d); k = rnd(15, 1, 1, d)
+    def dot(p, t):
+        return float((orc.rope(q, np.array([p]), cos, sin) * orc.rope(k, np.array([t]), cos, sin)).sum())
+    assert abs(dot(3, 9) - dot(13, 19)) < 1e-5                                   # relative positions only
+    assert abs(dot(3, 9) - dot(9, 3)) > 1e-3                                     # and their sign matters
+    # explicit 2-d rotation by the tabulated angle of pair (i, i + d/2)
+    i, p = 2, 7
+    ang = p * 1e4 ** (-i / (d / 2))
+    e = np.zeros((1, 1, d)); e[0, 0, i] = 1.0
+    r = orc.rope(e, np.array([p]), cos, sin)[0, 0]
+    assert abs(r[i] - math.cos(ang)) < 1e-6 and abs(r[i + d // 2] - math.sin(ang)) < 1e-6
+    assert np.count_nonzero(np.abs(r) > 1e-12) == 2
+
+
+def test_rope_vs_library_rotary():
+    llama = pytest.importorskip("transformers.models.llama.modeling_llama")
+    d, H, T, n = 8, 2, 16, 5
+    cos, sin = wl.rope_table(T, d, 1e4)
+    v = rnd(16, n, H, d)
+    pos = np.array([0, 3, 4, 9, 15])
+    c = torch.from_numpy(np.concatenate([cos[pos], cos[pos]], -1).astype(np.float64))[None]   # [1, n, d]
+    s = torch.from_numpy(np.concatenate([sin[pos], sin[pos]], -1).astype(np.float64))[None]
+    tv = torch.from_numpy(v).permute(1, 0, 2)[None]                                           # [1, H, n, d]
+    ref, _ = llama.apply_rotary_pos_emb(tv, tv, c, s)
+    assert np.allclose(orc.rope(v, pos, cos, sin), ref[0].permute(1, 0, 2).numpy(), rtol=1e-12, atol=1e-14)
+
+
+# ---------------------------------------------------------------- dense layer vs library ops
+def torch_dense_layer(w, shape, x_bits, cos, sin):
+    """The benchmark layer composed from torch library ops in fp64 (no storage rounding)."""
+    F = torch.nn.functional
+    T = x_bits.shape[0]
+    t = lambda name: torch.from_numpy(orc.bf16_bits_to_f64(w[name]))
+    X = torch.from_numpy(orc.bf16_bits_to_f64(x_bits))
+    xn = F.rms_norm(X, (shape.hidden,), t("attn_norm_g"), shape.rms_eps)
+    bias = (lambda n: t(n)) if w.get("bq") is not None else (lambda n: None)
+    q = F.linear(xn, t("wq"), bias("bq")).view(T, shape.n_heads, shape.head_dim)
+    k = F.linear(xn, t("wk"), bias("bk")).view(T, shape.n_kv_heads, shape.head_dim)
+    v = F.linear(xn, t("wv"), bias("bv")).view(T, shape.n_kv_heads, shape.head_dim)
+    c = torch.from_numpy(np.concatenate([cos[:T], cos[:T]], -1).astype(np.float64))
+    s = torch.from_numpy(np.concatenate([sin[:T], sin[:T]], -1).astype(np.float64))
+    def rot(a):
+        h = a.shape[-1] // 2
+        return torch.cat([-a[..., h:], a[..., :h]], -1)
+    q = q * c[:, None, :] + rot(q) * s[:, None, :]
+    k = k * c[:, None, :] + rot(k) * s[:, None, :]
+    g = shape.n_heads // shape.n_kv_heads
+    o = F.scaled_dot_product_attention(q.permute(1, 0, 2)[None], k.permute(1, 0, 2).repeat_interleave(g, 0)[None],
+                                       v.permute(1, 0, 2).repeat_interleave(g, 0)[None])[0]
+    o = o.permute(1, 0, 2).reshape(T, -1)
+    h1 = X + F.linear(o, t("wo"))
+    xn2 = F.rms_norm(h1, (shape.hidden,), t("mlp_norm_g"), shape.rms_eps)
+    y = h1 + F.linear(F.silu(F.linear(xn2, t("w_gate"))) * F.linear(xn2, t("w_up")), t("w_down"))
+    return y.numpy(), k.numpy(), v.numpy()
+
+
+SMALL = wl.LayerShape(64, 4, 2, 16, 96, 1e-5, True, 1e4, "small")
+
+
+def small_case(shape=SMALL, pre=3, affix=12, post=5, gen=6, n_masked=4, extra="all", ratio=0.25, std=0.2):
+    lay = wl.make_layout(1, pre, affix, post, gen, n_masked, extra)
+    w = wl.layer_weights(shape, 9, 0, std=std)
+    x = wl.hidden_states(shape, lay, 100, 101)
+    xs = wl.hidden_states(shape, lay, 100, 102)
+    cos, sin = wl.rope_table(lay.ctx_len, shape.head_dim, shape.rope_theta)
+    return lay, w, x[0], xs[0], cos, sin
+
+
+def test_dense_layer_vs_library_ops():
+    lay, w, x, _, cos, sin = small_case()
+    y, kb, vb = orc.dense_layer(w, SMALL, x, cos, sin, round_storage=False)
+    yr, kr, vr = torch_dense_layer(w, SMALL, x, cos, sin)
+    assert np.allclose(y, yr, rtol=1e-10, atol=1e-12)
+    assert np.array_equal(kb, orc.f64_to_bf16_bits(kr)) and np.array_equal(vb, orc.f64_to_bf16_bits(vr))
+    # storage rounding alone moves the result by a few bf16 ulps (this small case has large weights)
+    y2, _, _ = orc.dense_layer(w, SMALL, x, cos, sin, round_storage=True)
+    ok, worst = orc.rel_err_gate(y2, yr, 5e-2)
+    assert ok, worst
+
+
+def stale_cache(w, shape, xs, cos, sin, T):
+    """Exact K/V of every row computed from the hidden states ``xs`` (another context)."""
+    X = orc.bf16_bits_to_f64(xs)
+    xn = orc.normed_rows(w, shape, X)
+    k, v = orc.project_kv(w, shape, xn, np.arange(T), cos, sin)
+    return orc.f64_to_bf16_bits(k), orc.f64_to_bf16_bits(v)
+
+
+# ---------------------------------------------------------------- end points of the ratio (Section 5.2)
+@pytest.mark.parametrize("round_storage", [True, False])
+def test_ratio_one_equals_dense_layer(round_storage):
+    lay, w, x, xs, cos, sin = small_case(ratio=1.0)
+    T = lay.ctx_len
+    ck, cv = stale_cache(w, SMALL, xs, cos, sin, T)
+    out = orc.layer_step(w, SMALL, x, ck, cv, T, lay.affix_start, lay.affix_len, lay.masked_pos[0],
+                         lay.extra_rows[0], cos, sin, ratio=1.0, round_storage=round_storage)
+    assert out["anchor_idx"].tolist() == list(range(lay.affix_len))
+    y, kd, vd = orc.dense_layer(w, SMALL, x, cos, sin, round_storage=round_storage)
+    rows = out["rows"]
+    assert sorted(rows.tolist()) == list(range(T))
+    assert np.array_equal(out["cache_k"], kd) and np.array_equal(out["cache_v"], vd)
+    assert np.allclose(out["y"], y[rows], rtol=1e-9, atol=1e-11)
+    assert np.allclose(out["rowsum"], 1.0, atol=1e-12)
+
+
+def test_ratio_zero_is_direct_reuse():
+    lay, w, x, xs, cos, sin = small_case()
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    ck, cv = stale_cache(w, SMALL, xs, cos, sin, T)
+    out = orc.layer_step(w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin, ratio=0.0)
+    assert out["anchor_idx"].size == 0
+    assert np.array_equal(out["cache_k"][l:l + L], ck[l:l + L]) and np.array_equal(out["cache_v"][l:l + L], cv[l:l + L])
+    # request rows attend the stale affix: same as library attention over [stale affix ; fresh request rows]
+    rows = out["rows"]
+    Kc = torch.from_numpy(orc.bf16_bits_to_f64(out["cache_k"]))
+    Vc = torch.from_numpy(orc.bf16_bits_to_f64(out["cache_v"]))
+    g = SMALL.n_heads // SMALL.n_kv_heads
+    q = torch.from_numpy(out["q"])
+    o = torch.nn.functional.scaled_dot_product_attention(
+        q.permute(1, 0, 2)[None], Kc.permute(1, 0, 2).repeat_interleave(g, 0)[None],
+        Vc.permute(1, 0, 2).repeat_interleave(g, 0)[None])[0].permute(1, 0, 2).reshape(len(rows), -1).numpy()
+    assert np.array_equal(orc.f64_to_bf16_bits(o), orc.f64_to_bf16_bits(out["o"])) or \
+        np.max(np.abs(orc.bf16_round(o) - out["o"])) <= 2 ** -7 * np.max(np.abs(o))
+    # with no extra rows either, nothing at all is recomputed
+    out0 = orc.layer_step(w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], np.zeros(0, np.int32), cos, sin, ratio=0.0)
+    assert np.array_equal(out0["cache_k"], ck) and np.array_equal(out0["cache_v"], cv) and out0["y"].shape[0] == 0
+
+
+def test_selective_attention_vs_library_attention():
+    """o of the recomputed rows == library attention of their queries over the working cache."""
+    lay, w, x, xs, cos, sin = small_case(extra="masked")
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    ck, cv = stale_cache(w, SMALL, xs, cos, sin, T)
+    out = orc.layer_step(w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin,
+                         ratio=0.25, round_storage=False)
+    rows = out["rows"]
+    Kc = orc.bf16_bits_to_f64(ck); Vc = orc.bf16_bits_to_f64(cv)
+    # unrounded mode keeps the fresh rows unrounded in the logical view
+    X = orc.bf16_bits_to_f64(x)
+    xn = orc.normed_rows(w, SMALL, X[rows], False)
+    kf, vf = orc.project_kv(w, SMALL, xn, rows, cos, sin, False)
+    Kc[rows] = kf; Vc[rows] = vf
+    g = SMALL.n_heads // SMALL.n_kv_heads
+    tq = torch.from_numpy(out["q"]).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(Kc).permute(1, 0, 2).repeat_interleave(g, 0)[None]
+    tv = torch.from_numpy(Vc).permute(1, 0, 2).repeat_interleave(g, 0)[None]
+    o = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv)[0].permute(1, 0, 2).reshape(len(rows), -1)
+    assert np.allclose(out["o"], o.numpy(), rtol=1e-10, atol=1e-13)
+    assert np.allclose(out["rowsum"], 1.0, atol=1e-12)
+
+
+def test_untouched_rows_byte_identical_and_store_then_attend():
+    lay, w, x, xs, cos, sin = small_case(extra="masked")
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    ck, cv = stale_cache(w, SMALL, xs, cos, sin, T)
+    out = orc.layer_step(w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin, ratio=0.25)
+    rows = out["rows"]
+    K = orc.k_from_ratio(L, 0.25)
+    assert len(out["anchor_idx"]) == K and len(rows) == K + lay.n_extra
+    keep = np.setdiff1d(np.arange(T), rows)
+    assert np.array_equal(out["cache_k"][keep], ck[keep]) and np.array_equal(out["cache_v"][keep], cv[keep])
+    assert np.array_equal(out["cache_k"][rows], out["k_new"]) and np.array_equal(out["cache_v"][rows], out["v_new"])
+    assert not np.array_equal(out["cache_k"][rows], ck[rows])          # the stale rows really were stale
+    # anchors see refreshed K/V: garbage in the stale cache at recomputed rows changes nothing ...
+    ck2, cv2 = ck.copy(), cv.copy()
+    ck2[rows] = 0x4000; cv2[rows] = 0xC000
+    out2 = orc.layer_step(w, SMALL, x, ck2, cv2, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin,
+                          anchor_idx=out["anchor_idx"])
+    assert np.array_equal(out2["y"], out["y"]) and np.array_equal(out2["cache_k"], out["cache_k"])
+    # ... while a change at a reused row does change the recomputed rows' outputs
+    ck3 = ck.copy(); ck3[keep[0]] = 0x4100
+    out3 = orc.layer_step(w, SMALL, x, ck3, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin,
+                          anchor_idx=out["anchor_idx"])
+    assert not np.array_equal(out3["y"], out["y"])
+
+
+def test_idempotent_when_cache_is_current():
+    """If the cached K/V were computed from the very same hidden rows, a refresh rewrites identical bytes."""
+    lay, w, x, _, cos, sin = small_case()
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    ck, cv = stale_cache(w, SMALL, x, cos, sin, T)
+    out = orc.layer_step(w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin, ratio=0.5)
+    assert np.array_equal(out["cache_k"], ck) and np.array_equal(out["cache_v"], cv)
+    y, _, _ = orc.dense_layer(w, SMALL, x, cos, sin)
+    assert np.allclose(out["y"], y[out["rows"]], rtol=1e-9, atol=1e-11)
+
+
+def test_layer_step_scores_use_stale_keys_and_accumulate():
+    lay, w, x, xs, cos, sin = small_case(extra="none")
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    ck, cv = stale_cache(w, SMALL, xs, cos, sin, T)
+    out = orc.layer_step(w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin, ratio=0.25)
+    m, H = lay.n_masked, SMALL.n_heads
+    assert abs(out["scores64"].sum() - H * m) < 1e-9
+    ref = brute_scores(out["q_mask"].tolist(), orc.bf16_bits_to_f64(ck[l:l + L]).tolist(), H // SMALL.n_kv_heads)
+    assert np.allclose(out["scores64"], ref, rtol=1e-12)
+    prev = np.linspace(0, 1, L)
+    out2 = orc.layer_step(w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin,
+                          ratio=0.25, scores_in=prev)
+    assert np.allclose(out2["scores64"], out["scores64"] + prev, rtol=1e-13)
+    # variant with the full-context normaliser carries strictly less mass on the affix
+    out3 = orc.layer_step(w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin,
+                          ratio=0.25, norm_full=True)
+    assert out3["scores64"].sum() < H * m and np.all(out3["scores64"] < out["scores64"])
+
+
+def test_comparators():
+    ok, worst = orc.rel_err_gate(np.array([1.0, 2.0]), np.array([1.0, 2.0]))
+    assert ok and worst == 0
+    assert not orc.rel_err_gate(np.array([1.0, 2.2]), np.array([1.0, 2.0]))[0]
+    must, may = np.array([1, 5]), np.array([1, 3, 5, 7])
+    assert orc.anchor_set_ok(np.array([1, 3, 5]), 3, 10, must, may)[0]
+    assert not orc.anchor_set_ok(np.array([1, 3, 4]), 3, 10, must, may)[0]
+    assert not orc.anchor_set_ok(np.array([3, 5, 7]), 3, 10, must, may)[0]
+    assert not orc.anchor_set_ok(np.array([5, 3, 1]), 3, 10, must, may)[0]
+    assert not orc.anchor_set_ok(np.array([1, 5]), 3, 10, must, may)[0]
