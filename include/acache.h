@@ -1,0 +1,211 @@
+/*
+ * acache.h -- C ABI of the affix-cache refresh path for bidirectional diffusion LLMs
+ *             (ACache: anchor scoring, top-K anchor selection, selective
+ *             recomputation, KV scatter), implemented as CUDA kernels for sm_100a.
+ *
+ * Notation (Section 3.1-3.3 of the paper): the shared affix is the contiguous span
+ * F = {l .. r} of L positions inside a T-token context; M is the set of masked
+ * generation positions (m = |M|); A is the Anchor set (K = |A|), S = F \ A; E is the
+ * set of request-specific positions recomputed together with the anchors (e = |E|);
+ * R = A u E is the recompute set.  The layer is the pre-norm RMSNorm / RoPE / SwiGLU
+ * layer of LLaDA-8B and Dream-7B: D hidden, H query heads, Hkv KV heads, d head dim,
+ * Fm MLP width.
+ *
+ * Conventions that hold for every entry point
+ *  - Pointers marked DEVICE are device addresses on the current CUDA device; pointers
+ *    marked HOST are host addresses.  All device pointers must be 16-byte aligned.
+ *  - bf16 tensors are row-major with the last index contiguous.  Weights are
+ *    [out, in].  The KV cache is token-major [B, ctx_capacity, Hkv, d]; K is stored
+ *    after the rotary embedding.
+ *  - Ownership: the caller owns every buffer (weights, cache, inputs, outputs and the
+ *    workspace).  The library allocates only the small host-side context object in
+ *    acache_create and frees only that in acache_destroy.
+ *  - Asynchrony: every compute entry point only enqueues work on the given stream and
+ *    returns; it never synchronises.  Calls that share one context must be issued on
+ *    one stream (they share the workspace).
+ *  - Errors: every call returns acache_status.  Argument and shape validation happens
+ *    on the host before any launch, so a non-OK status means nothing was enqueued.
+ *    Faults that depend on device data (an index outside its range) never trap: the
+ *    offending row is skipped and a bit is set in a device status word that
+ *    acache_poll_status reads back.
+ *  - Compact row order: every "[B, K+e, ...]" tensor lists, per request, the K anchor
+ *    rows in ascending position followed by the e extra rows in the order given.
+ */
+#ifndef ACACHE_H_
+#define ACACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ACACHE_OK = 0,
+    ACACHE_ERR_INVALID_ARG = 1,       /* NULL / misaligned pointer, negative size, bad range   */
+    ACACHE_ERR_UNSUPPORTED_SHAPE = 2, /* shape outside what the kernels are built for          */
+    ACACHE_ERR_WORKSPACE = 3,         /* workspace missing or smaller than acache_workspace_bytes */
+    ACACHE_ERR_CUDA = 4,              /* a CUDA runtime call failed (see acache_last_error)    */
+    ACACHE_ERR_TIMEOUT = 5            /* a bounded device-side wait expired (status word)      */
+} acache_status;
+
+/* bits of the device status word returned by acache_poll_status */
+#define ACACHE_FLAG_BAD_INDEX   0x1u  /* an anchor / masked / extra index was out of range; row skipped */
+#define ACACHE_FLAG_WAIT_EXPIRED 0x2u /* a bounded wait inside a kernel gave up                          */
+
+/* flags of acache_layer_step */
+#define ACACHE_F_SCORE            0x1u /* form Q for the masked rows from x and run the scoring (Eq. 4-5) */
+#define ACACHE_F_SELECT           0x2u /* run the top-K selection (Eq. 6); otherwise use the given anchor_idx */
+#define ACACHE_F_ACCUMULATE       0x4u /* scores += this layer's scores (Eq. 5 sums over layers)        */
+#define ACACHE_F_SCORE_NORM_FULL  0x8u /* softmax of Eq. 4 over every key of the context, not the affix only */
+#define ACACHE_F_NO_RECOMPUTE    0x10u /* stop after scoring / selection (the selection-time probe)     */
+
+typedef struct CUstream_st *acache_stream_t;   /* a cudaStream_t */
+typedef struct acache_ctx acache_ctx;           /* opaque */
+
+/* Layer shape and the largest problem the context must hold (sizes the workspace). */
+typedef struct {
+    int32_t hidden, n_heads, n_kv_heads, head_dim, ffn;
+    float   rms_eps;
+    int32_t qkv_bias;      /* 0/1: bq, bk, bv present */
+    int32_t max_batch;     /* B                                  */
+    int32_t max_ctx;       /* T (and the cache's ctx_capacity)   */
+    int32_t max_affix;     /* L                                  */
+    int32_t max_rows;      /* K + e per request                  */
+    int32_t max_masked;    /* m per request                      */
+} acache_model_desc;
+
+/* DEVICE bf16 weights, [out, in] row-major.  bq/bk/bv may be NULL when qkv_bias == 0. */
+typedef struct {
+    const void *attn_norm_g;          /* [D]            */
+    const void *wq, *wk, *wv;         /* [H*d, D], [Hkv*d, D], [Hkv*d, D] */
+    const void *bq, *bk, *bv;         /* [H*d], [Hkv*d], [Hkv*d]          */
+    const void *wo;                   /* [D, H*d]       */
+    const void *mlp_norm_g;           /* [D]            */
+    const void *w_gate, *w_up;        /* [Fm, D]        */
+    const void *w_down;               /* [D, Fm]        */
+} acache_layer_weights;
+
+/* One layer's KV cache: DEVICE bf16 [B, ctx_capacity, Hkv, d]; request b starts at
+ * element offset b * batch_stride (normally ctx_capacity * Hkv * d). */
+typedef struct {
+    void   *k, *v;
+    int64_t batch_stride;
+    int32_t ctx_capacity;
+} acache_kv;
+
+/* The request batch: every request shares the layout (ctx_len, affix span, m, e). */
+typedef struct {
+    int32_t batch, ctx_len;
+    int32_t affix_start, affix_len;       /* F = [affix_start, affix_start + affix_len)          */
+    const int32_t *masked_pos;            /* DEVICE [B, n_masked] absolute positions outside F   */
+    int32_t n_masked;
+    const int32_t *extra_rows;            /* DEVICE [B, n_extra] absolute positions outside F; may be NULL when n_extra == 0 */
+    int32_t n_extra;
+    const float *rope_cos, *rope_sin;     /* DEVICE fp32 [>= ctx_len, d/2] rotary table, pairing (i, i + d/2) */
+} acache_request;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Creates the host-side context for one layer shape.  Validates the shape:
+ * head_dim in {64, 128}; n_heads % n_kv_heads == 0; hidden, H*d, Hkv*d and ffn
+ * multiples of 128.  No device memory is allocated. */
+acache_status acache_create(const acache_model_desc *desc, acache_ctx **out);
+
+/* Bytes of device scratch the context needs for the sizes in its descriptor. */
+size_t acache_workspace_bytes(const acache_ctx *ctx);
+
+/* Hands the context its scratch: DEVICE memory, 256-byte aligned, at least
+ * acache_workspace_bytes.  The caller keeps ownership and must keep it alive while
+ * the context is used.  Enqueues a memset of the status word on `stream`. */
+acache_status acache_set_workspace(acache_ctx *ctx, void *dev_ptr, size_t bytes, acache_stream_t stream);
+
+void acache_destroy(acache_ctx *ctx);
+
+/* Text of the last error recorded by this context (HOST string owned by the context). */
+const char *acache_last_error(const acache_ctx *ctx);
+
+/* Copies the device status word to *host_flags (HOST), synchronising `stream`, and
+ * clears it.  Returns ACACHE_ERR_TIMEOUT if ACACHE_FLAG_WAIT_EXPIRED is set. */
+acache_status acache_poll_status(acache_ctx *ctx, acache_stream_t stream, uint32_t *host_flags);
+
+/* Number of kernels this context has launched since creation (for accounting). */
+uint64_t acache_launch_count(const acache_ctx *ctx);
+
+/* ---- the path ------------------------------------------------------------------------ */
+
+/* Eq. 4-5 (Section 3.2), one layer's term:
+ *   a[j,k,h] = Softmax_j( q_mask[k,h,:] . K_affix[j,kv(h),:] / sqrt(d) ),  j in F
+ *   scores[b,j] (+)= sum_h sum_{k in M} a[j,k,h]
+ * q_mask: DEVICE bf16 [B, m, H, d], the post-RoPE queries of the masked positions.
+ * kv: the layer's cache; the affix keys are rows affix_start.. of each request.
+ * scores: DEVICE fp32 [B, L].  accumulate != 0 adds to the existing contents.
+ * norm_full != 0 takes the softmax over all ctx_len keys and keeps the affix columns.
+ * The sum over heads and queries is evaluated in a fixed order (bitwise reproducible). */
+acache_status acache_score_anchors(acache_ctx *ctx, const acache_request *req, const void *q_mask,
+                                   const acache_kv *kv, float *scores, int accumulate, int norm_full,
+                                   acache_stream_t stream);
+
+/* K of Eq. 6 from the recompute ratio: ceil(ratio * L) clipped to [0, L].  HOST, pure. */
+int32_t acache_k_from_ratio(int32_t affix_len, double ratio);
+
+/* Eq. 6 (Section 3.2): A = TopK({s_j}, K).  scores: DEVICE fp32 [B, L].
+ * anchor_idx: DEVICE int32 [B, K], positions relative to affix_start, ascending.
+ * Ties are broken towards the lower position, so the result is unique. */
+acache_status acache_select_topk(acache_ctx *ctx, const float *scores, int32_t batch, int32_t affix_len,
+                                 int32_t k, int32_t *anchor_idx, acache_stream_t stream);
+
+/* Selective recomputation (Section 3.3, Section 4.3) of the rows R = A u E of every
+ * request, WITHOUT touching the cache:
+ *   xn = RMSNorm(x_r) g1; q,k,v = W{q,k,v} xn (+b); RoPE(q,k; position r)
+ *   o  = bidirectional attention of q over all ctx_len keys/values, where positions in
+ *        R read the fresh k/v and all others read the cache (store-then-attend view)
+ *   y  = h1 + Wd (silu(Wg xn2) * (Wu xn2)),  h1 = x_r + Wo o,  xn2 = RMSNorm(h1) g2
+ * x: DEVICE bf16, [B, ctx_len, D] (rows gathered by position) or, if x_is_compact,
+ *    [B, K+e, D] in compact row order.
+ * anchor_idx: DEVICE int32 [B, K] (relative to affix_start); k may be 0.
+ * k_new, v_new: DEVICE bf16 [B, K+e, Hkv, d] out.  y: DEVICE bf16 [B, K+e, D] out. */
+acache_status acache_recompute_anchors(acache_ctx *ctx, const acache_layer_weights *w,
+                                       const acache_request *req, const acache_kv *kv,
+                                       const void *x, int x_is_compact,
+                                       const int32_t *anchor_idx, int32_t k,
+                                       void *k_new, void *v_new, void *y, acache_stream_t stream);
+
+/* Working-cache construction (Section 3.3, Section 4.1): writes the fresh K/V of the
+ * rows R into the cache rows they belong to; every other row is left untouched
+ * (byte-identical).  k_new/v_new as produced by acache_recompute_anchors. */
+acache_status acache_scatter_kv(acache_ctx *ctx, const acache_request *req, acache_kv *kv,
+                                const int32_t *anchor_idx, int32_t k,
+                                const void *k_new, const void *v_new, acache_stream_t stream);
+
+/* One layer-step on one stream: [score -> select ->] recompute -> scatter, with the
+ * scatter fused into the QKV projection and attention reading the updated cache
+ * (store-then-attend, Appendix C.1).  Gives the same cache and (within rounding of
+ * the attention tiling) the same y as the three split calls in sequence.
+ *   flags & ACACHE_F_SCORE : x must be the full [B, ctx_len, D] input; scores is written.
+ *   flags & ACACHE_F_SELECT: anchor_idx [B, K] is written, K = acache_k_from_ratio(L, ratio);
+ *                            otherwise anchor_idx is an input with that K.
+ * scores: DEVICE fp32 [B, L] (may be NULL without F_SCORE/F_SELECT).
+ * y: DEVICE bf16 [B, K+e, D]. */
+acache_status acache_layer_step(acache_ctx *ctx, const acache_layer_weights *w,
+                                const acache_request *req, acache_kv *kv,
+                                const void *x, int x_is_compact, double ratio, uint32_t flags,
+                                float *scores, int32_t *anchor_idx, void *y, acache_stream_t stream);
+
+/* acache_layer_step for a caller whose per-step data lives in HOST memory: copies
+ * x [B, ctx_len, D] (HOST bf16, ideally pinned) to a staging area in the workspace,
+ * runs the layer-step with ACACHE_F_SCORE | ACACHE_F_SELECT | flags, and copies y
+ * [B, K+e, D], anchor_idx [B, K] and scores [B, L] back to the given HOST buffers.
+ * Weights, cache and the request's index arrays stay DEVICE-resident.  All copies are
+ * asynchronous on `stream`; the caller synchronises the stream before reading. */
+acache_status acache_layer_step_host(acache_ctx *ctx, const acache_layer_weights *w,
+                                     const acache_request *req, acache_kv *kv,
+                                     const void *x_host, double ratio, uint32_t flags,
+                                     float *scores_host, int32_t *anchor_idx_host, void *y_host,
+                                     acache_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ACACHE_H_ */

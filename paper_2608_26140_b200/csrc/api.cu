@@ -1,0 +1,413 @@
+// C-ABI entry points (see include/acache.h): argument validation, workspace layout and the
+// kernel sequences of the affix-cache refresh path.  Everything is enqueued on the caller's
+// stream; nothing here allocates device memory or synchronises (except acache_poll_status).
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "../../include/acache.h"
+#include "kernels.h"
+
+using namespace acache;
+
+struct acache_ctx {
+    acache_model_desc d;
+    size_t ws_need = 0;
+    unsigned char* ws = nullptr;
+    size_t ws_have = 0;
+    // workspace offsets (bytes)
+    size_t o_status, o_row_pos, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
+    size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
+    size_t o_xstage, o_ystage, o_sstage, o_astage;
+    std::string err;
+    uint64_t launches = 0;
+};
+
+namespace {
+
+acache_status fail(acache_ctx* c, acache_status s, const char* fmt, ...) {
+    if (c) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        c->err = buf;
+    }
+    return s;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t take(size_t& cur, size_t bytes) {
+    size_t at = cur;
+    cur += (bytes + 255) & ~size_t(255);
+    return at;
+}
+
+template <class T>
+T* wsp(acache_ctx* c, size_t off) { return reinterpret_cast<T*>(c->ws + off); }
+
+acache_status check_cuda(acache_ctx* c, const char* what) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(c, ACACHE_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    return ACACHE_OK;
+}
+
+acache_status check_request(acache_ctx* c, const acache_request* r, const acache_kv* kv, int k, bool need_rope) {
+    const acache_model_desc& d = c->d;
+    if (!c->ws) return fail(c, ACACHE_ERR_WORKSPACE, "workspace not set");
+    if (!r) return fail(c, ACACHE_ERR_INVALID_ARG, "request is NULL");
+    if (r->batch < 0 || r->batch > d.max_batch) return fail(c, ACACHE_ERR_INVALID_ARG, "batch %d outside [0, %d]", r->batch, d.max_batch);
+    if (r->ctx_len <= 0 || r->ctx_len > d.max_ctx) return fail(c, ACACHE_ERR_INVALID_ARG, "ctx_len %d outside (0, %d]", r->ctx_len, d.max_ctx);
+    if (r->affix_len < 0 || r->affix_len > d.max_affix || r->affix_start < 0 ||
+        (int64_t)r->affix_start + r->affix_len > r->ctx_len)
+        return fail(c, ACACHE_ERR_INVALID_ARG, "affix span [%d, +%d) outside the context / max_affix", r->affix_start, r->affix_len);
+    if (r->n_masked < 0 || r->n_masked > d.max_masked) return fail(c, ACACHE_ERR_INVALID_ARG, "n_masked %d outside [0, %d]", r->n_masked, d.max_masked);
+    if (r->n_extra < 0 || k < 0 || k > r->affix_len) return fail(c, ACACHE_ERR_INVALID_ARG, "k %d / n_extra %d out of range", k, r->n_extra);
+    if ((int64_t)k + r->n_extra > d.max_rows) return fail(c, ACACHE_ERR_INVALID_ARG, "k + n_extra = %d exceeds max_rows %d", k + r->n_extra, d.max_rows);
+    if (r->n_masked > 0 && !r->masked_pos) return fail(c, ACACHE_ERR_INVALID_ARG, "masked_pos is NULL");
+    if (r->n_extra > 0 && !r->extra_rows) return fail(c, ACACHE_ERR_INVALID_ARG, "extra_rows is NULL");
+    if (need_rope && (!r->rope_cos || !r->rope_sin || !aligned16(r->rope_cos) || !aligned16(r->rope_sin)))
+        return fail(c, ACACHE_ERR_INVALID_ARG, "rope table NULL or misaligned");
+    if (kv) {
+        if (!kv->k || !kv->v || !aligned16(kv->k) || !aligned16(kv->v)) return fail(c, ACACHE_ERR_INVALID_ARG, "cache pointer NULL or misaligned");
+        if (kv->ctx_capacity < r->ctx_len) return fail(c, ACACHE_ERR_INVALID_ARG, "ctx_capacity %d < ctx_len %d", kv->ctx_capacity, r->ctx_len);
+        if (kv->batch_stride < (int64_t)kv->ctx_capacity * d.n_kv_heads * d.head_dim || (kv->batch_stride & 7))
+            return fail(c, ACACHE_ERR_INVALID_ARG, "batch_stride smaller than one request's cache or not a multiple of 8");
+    }
+    return ACACHE_OK;
+}
+
+acache_status check_weights(acache_ctx* c, const acache_layer_weights* w, bool q_only) {
+    if (!w) return fail(c, ACACHE_ERR_INVALID_ARG, "weights is NULL");
+    const void* need[] = {w->attn_norm_g, w->wq, w->wk, w->wv, w->wo, w->mlp_norm_g, w->w_gate, w->w_up, w->w_down};
+    const int n = q_only ? 2 : 9;
+    for (int i = 0; i < n; ++i)
+        if (!need[i] || !aligned16(need[i])) return fail(c, ACACHE_ERR_INVALID_ARG, "weight pointer %d NULL or misaligned", i);
+    if (c->d.qkv_bias && (!w->bq || (!q_only && (!w->bk || !w->bv))))
+        return fail(c, ACACHE_ERR_INVALID_ARG, "qkv_bias set but a bias pointer is NULL");
+    return ACACHE_OK;
+}
+
+// Q for the masked rows, then Eq. 4-5.
+acache_status run_score(acache_ctx* c, const acache_request* r, const void* q_mask, const acache_kv* kv,
+                        float* scores, int accumulate, int norm_full, cudaStream_t st) {
+    ScoreArgs a{};
+    a.q_mask = q_mask;
+    a.cache_k = kv->k;
+    a.kv_batch_stride = kv->batch_stride;
+    a.batch = r->batch; a.m = r->n_masked;
+    a.n_heads = c->d.n_heads; a.n_kv_heads = c->d.n_kv_heads; a.head_dim = c->d.head_dim;
+    a.affix_start = r->affix_start; a.affix_len = r->affix_len;
+    a.norm_lo = norm_full ? 0 : r->affix_start;
+    a.norm_len = norm_full ? r->ctx_len : r->affix_len;
+    a.row_stats = wsp<float>(c, c->o_stats);
+    a.head_partial = wsp<float>(c, c->o_partial);
+    a.scores = scores;
+    a.accumulate = accumulate;
+    int n = launch_score(a, st);
+    if (n < 0) return fail(c, ACACHE_ERR_UNSUPPORTED_SHAPE, "n_masked %d too large for the scoring kernel", r->n_masked);
+    c->launches += n;
+    return check_cuda(c, "score");
+}
+
+// The recompute of rows R.  fused_cache != null: K/V go straight into the cache and
+// attention reads it; otherwise K/V go to k_new/v_new and attention reads through a slot map.
+acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const acache_request* r,
+                            const acache_kv* kv, bool fuse_scatter, const void* x, int x_is_compact,
+                            const int32_t* anchor_idx, int k, void* k_new, void* v_new, void* y, cudaStream_t st) {
+    const acache_model_desc& d = c->d;
+    const int rows = k + r->n_extra, n = r->batch * rows;
+    if (n == 0) return ACACHE_OK;
+    const int qd = d.n_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim;
+    int32_t* row_pos = wsp<int32_t>(c, c->o_row_pos);
+    int64_t* row_src = wsp<int64_t>(c, c->o_row_src);
+    void* xn = wsp<void>(c, c->o_xn);
+    void* q = wsp<void>(c, c->o_q);
+    void* o = wsp<void>(c, c->o_o);
+    void* h1 = wsp<void>(c, c->o_h1);
+    void* xn2 = wsp<void>(c, c->o_xn2);
+    void* act = wsp<void>(c, c->o_act);
+    uint32_t* status = wsp<uint32_t>(c, c->o_status);
+
+    launch_gather_rmsnorm(x, x_is_compact, (int64_t)r->ctx_len * d.hidden, d.hidden, anchor_idx, k, r->extra_rows,
+                          r->n_extra, r->batch, r->affix_start, r->affix_len, r->ctx_len, w->attn_norm_g, d.rms_eps,
+                          row_pos, row_src, xn, status, st);
+    c->launches += 1;
+
+    GemmArgs g{};
+    g.a = xn; g.M = n; g.K = d.hidden;
+    g.b[0] = w->wq; g.b[1] = w->wk; g.b[2] = w->wv;
+    g.n[0] = qd; g.n[1] = kvd; g.n[2] = kvd;
+    g.epilogue = kEpiQKV;
+    g.bias[0] = d.qkv_bias ? w->bq : nullptr;
+    g.bias[1] = d.qkv_bias ? w->bk : nullptr;
+    g.bias[2] = d.qkv_bias ? w->bv : nullptr;
+    g.row_pos = row_pos; g.rope_cos = r->rope_cos; g.rope_sin = r->rope_sin;
+    g.head_dim = d.head_dim; g.rope_segments = 2;
+    g.out[0] = q; g.out[1] = k_new; g.out[2] = v_new;
+    if (fuse_scatter) { g.cache_k = kv->k; g.cache_v = kv->v; }
+    g.kv_batch_stride = kv->batch_stride; g.rows_per_req = rows;
+    c->launches += launch_gemm(g, st);
+
+    AttnArgs at{};
+    at.q = q; at.cache_k = kv->k; at.cache_v = kv->v; at.kv_batch_stride = kv->batch_stride;
+    if (!fuse_scatter) {
+        int32_t* slot = wsp<int32_t>(c, c->o_slot);
+        launch_build_slot_map(slot, r->ctx_len, row_pos, rows, r->batch, st);
+        c->launches += 1;
+        at.k_new = k_new; at.v_new = v_new; at.slot = slot;
+    }
+    at.batch = r->batch; at.n = rows; at.ctx_len = r->ctx_len;
+    at.n_heads = d.n_heads; at.n_kv_heads = d.n_kv_heads; at.head_dim = d.head_dim;
+    at.o = o;
+    c->launches += launch_attention(at, st);
+
+    GemmArgs go{};
+    go.a = o; go.M = n; go.K = qd; go.b[0] = w->wo; go.n[0] = d.hidden;
+    go.epilogue = kEpiResidual; go.resid = x; go.resid_off = row_src; go.c = h1;
+    c->launches += launch_gemm(go, st);
+
+    launch_rmsnorm(h1, w->mlp_norm_g, d.rms_eps, n, d.hidden, xn2, st);
+    c->launches += 1;
+
+    GemmArgs gu{};
+    gu.a = xn2; gu.M = n; gu.K = d.hidden; gu.b[0] = w->w_gate; gu.b[1] = w->w_up; gu.n[0] = d.ffn; gu.n[1] = d.ffn;
+    gu.epilogue = kEpiSwiGLU; gu.c = act;
+    c->launches += launch_gemm(gu, st);
+
+    GemmArgs gd{};
+    gd.a = act; gd.M = n; gd.K = d.ffn; gd.b[0] = w->w_down; gd.n[0] = d.hidden;
+    gd.epilogue = kEpiResidual; gd.resid = h1; gd.resid_off = nullptr; gd.c = y;
+    c->launches += launch_gemm(gd, st);
+    return check_cuda(c, "recompute");
+}
+
+}  // namespace
+
+extern "C" {
+
+acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
+    if (!desc || !out) return ACACHE_ERR_INVALID_ARG;
+    *out = nullptr;
+    const acache_model_desc& d = *desc;
+    if (d.hidden <= 0 || d.n_heads <= 0 || d.n_kv_heads <= 0 || d.ffn <= 0 || d.max_batch <= 0 || d.max_ctx <= 0 ||
+        d.max_affix < 0 || d.max_rows < 0 || d.max_masked < 0 || !(d.rms_eps >= 0.f))
+        return ACACHE_ERR_INVALID_ARG;
+    if (d.head_dim != 64 && d.head_dim != 128) return ACACHE_ERR_UNSUPPORTED_SHAPE;
+    if (d.n_heads % d.n_kv_heads) return ACACHE_ERR_UNSUPPORTED_SHAPE;
+    const int qd = d.n_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim;
+    if (qd % 128 || kvd % 128 || d.ffn % 128 || d.hidden % 128) return ACACHE_ERR_UNSUPPORTED_SHAPE;
+    acache_ctx* c = new (std::nothrow) acache_ctx();
+    if (!c) return ACACHE_ERR_INVALID_ARG;
+    c->d = d;
+    const size_t nr = (size_t)d.max_batch * d.max_rows, nm = (size_t)d.max_batch * d.max_masked;
+    size_t cur = 0;
+    c->o_status = take(cur, 256);
+    c->o_row_pos = take(cur, nr * 4);
+    c->o_row_src = take(cur, nr * 8);
+    c->o_xn = take(cur, nr * d.hidden * 2);
+    c->o_q = take(cur, nr * qd * 2);
+    c->o_o = take(cur, nr * qd * 2);
+    c->o_h1 = take(cur, nr * d.hidden * 2);
+    c->o_xn2 = take(cur, nr * d.hidden * 2);
+    c->o_act = take(cur, nr * d.ffn * 2);
+    c->o_knew = take(cur, nr * kvd * 2);
+    c->o_vnew = take(cur, nr * kvd * 2);
+    c->o_mrow_pos = take(cur, nm * 4);
+    c->o_mrow_src = take(cur, nm * 8);
+    c->o_xn_mask = take(cur, nm * d.hidden * 2);
+    c->o_qmask = take(cur, nm * qd * 2);
+    c->o_stats = take(cur, (size_t)d.max_batch * d.n_heads * score_num_splits(d.max_ctx) * d.max_masked * 8);
+    c->o_partial = take(cur, (size_t)d.max_batch * d.n_heads * d.max_affix * 4);
+    c->o_slot = take(cur, (size_t)d.max_batch * d.max_ctx * 4);
+    c->o_xstage = take(cur, (size_t)d.max_batch * d.max_ctx * d.hidden * 2);
+    c->o_ystage = take(cur, nr * d.hidden * 2);
+    c->o_sstage = take(cur, (size_t)d.max_batch * d.max_affix * 4);
+    c->o_astage = take(cur, (size_t)d.max_batch * d.max_affix * 4);
+    c->ws_need = cur;
+    *out = c;
+    return ACACHE_OK;
+}
+
+size_t acache_workspace_bytes(const acache_ctx* ctx) { return ctx ? ctx->ws_need : 0; }
+
+acache_status acache_set_workspace(acache_ctx* ctx, void* dev_ptr, size_t bytes, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!dev_ptr || (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return fail(ctx, ACACHE_ERR_INVALID_ARG, "workspace NULL or not 256-byte aligned");
+    if (bytes < ctx->ws_need) return fail(ctx, ACACHE_ERR_WORKSPACE, "workspace %zu < %zu bytes", bytes, ctx->ws_need);
+    ctx->ws = static_cast<unsigned char*>(dev_ptr);
+    ctx->ws_have = bytes;
+    if (cudaMemsetAsync(ctx->ws + ctx->o_status, 0, 256, stream) != cudaSuccess) return check_cuda(ctx, "memset");
+    return ACACHE_OK;
+}
+
+void acache_destroy(acache_ctx* ctx) { delete ctx; }
+
+const char* acache_last_error(const acache_ctx* ctx) { return ctx ? ctx->err.c_str() : "context is NULL"; }
+
+uint64_t acache_launch_count(const acache_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+acache_status acache_poll_status(acache_ctx* ctx, acache_stream_t stream, uint32_t* host_flags) {
+    if (!ctx || !host_flags) return ACACHE_ERR_INVALID_ARG;
+    if (!ctx->ws) return fail(ctx, ACACHE_ERR_WORKSPACE, "workspace not set");
+    uint32_t v = 0;
+    if (cudaMemcpyAsync(&v, ctx->ws + ctx->o_status, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemsetAsync(ctx->ws + ctx->o_status, 0, 4, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return check_cuda(ctx, "poll_status") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "poll_status failed") : ACACHE_ERR_CUDA;
+    *host_flags = v;
+    if (v & ACACHE_FLAG_WAIT_EXPIRED) return fail(ctx, ACACHE_ERR_TIMEOUT, "a bounded device-side wait expired");
+    return ACACHE_OK;
+}
+
+int32_t acache_k_from_ratio(int32_t affix_len, double ratio) {
+    if (affix_len <= 0 || !(ratio > 0.0)) return 0;
+    double k = std::ceil(ratio * (double)affix_len - 1e-9);
+    if (k < 0) k = 0;
+    if (k > affix_len) k = affix_len;
+    return (int32_t)k;
+}
+
+acache_status acache_score_anchors(acache_ctx* ctx, const acache_request* req, const void* q_mask,
+                                   const acache_kv* kv, float* scores, int accumulate, int norm_full,
+                                   acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!kv) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv is NULL");
+    acache_status s = check_request(ctx, req, kv, 0, false);
+    if (s != ACACHE_OK) return s;
+    if (!scores || (req->n_masked > 0 && (!q_mask || !aligned16(q_mask)))) return fail(ctx, ACACHE_ERR_INVALID_ARG, "q_mask / scores NULL or misaligned");
+    return run_score(ctx, req, q_mask, kv, scores, accumulate, norm_full, stream);
+}
+
+acache_status acache_select_topk(acache_ctx* ctx, const float* scores, int32_t batch, int32_t affix_len, int32_t k,
+                                 int32_t* anchor_idx, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (batch < 0 || affix_len < 0 || k < 0 || k > affix_len) return fail(ctx, ACACHE_ERR_INVALID_ARG, "batch %d, affix_len %d, k %d out of range", batch, affix_len, k);
+    if (batch == 0 || k == 0) return ACACHE_OK;
+    if (!scores || !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "scores / anchor_idx is NULL");
+    launch_topk(scores, batch, affix_len, k, anchor_idx, stream);
+    ctx->launches += 1;
+    return check_cuda(ctx, "topk");
+}
+
+acache_status acache_recompute_anchors(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
+                                       const acache_kv* kv, const void* x, int x_is_compact,
+                                       const int32_t* anchor_idx, int32_t k, void* k_new, void* v_new, void* y,
+                                       acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!kv) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv is NULL");
+    acache_status s = check_request(ctx, req, kv, k, true);
+    if (s != ACACHE_OK) return s;
+    if ((s = check_weights(ctx, w, false)) != ACACHE_OK) return s;
+    if (req->batch * (k + req->n_extra) == 0) return ACACHE_OK;
+    if (!x || !k_new || !v_new || !y || !aligned16(x) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(y))
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "x / k_new / v_new / y NULL or misaligned");
+    if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
+    return run_recompute(ctx, w, req, kv, false, x, x_is_compact, anchor_idx, k, k_new, v_new, y, stream);
+}
+
+acache_status acache_scatter_kv(acache_ctx* ctx, const acache_request* req, acache_kv* kv, const int32_t* anchor_idx,
+                                int32_t k, const void* k_new, const void* v_new, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!kv) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv is NULL");
+    acache_status s = check_request(ctx, req, kv, k, false);
+    if (s != ACACHE_OK) return s;
+    if (req->batch * (k + req->n_extra) == 0) return ACACHE_OK;
+    if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return fail(ctx, ACACHE_ERR_INVALID_ARG, "k_new / v_new NULL or misaligned");
+    if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
+    launch_scatter_kv(kv->k, kv->v, kv->batch_stride, req->ctx_len, anchor_idx, k, req->extra_rows, req->n_extra,
+                      req->batch, req->affix_start, req->affix_len, ctx->d.n_kv_heads * ctx->d.head_dim, k_new, v_new,
+                      wsp<uint32_t>(ctx, ctx->o_status), stream);
+    ctx->launches += 1;
+    return check_cuda(ctx, "scatter");
+}
+
+acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
+                                acache_kv* kv, const void* x, int x_is_compact, double ratio, uint32_t flags,
+                                float* scores, int32_t* anchor_idx, void* y, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!kv) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv is NULL");
+    if (!req) return fail(ctx, ACACHE_ERR_INVALID_ARG, "request is NULL");
+    const acache_model_desc& d = ctx->d;
+    const int k = acache_k_from_ratio(req->affix_len, ratio);
+    acache_status s = check_request(ctx, req, kv, k, true);
+    if (s != ACACHE_OK) return s;
+    const bool do_score = flags & ACACHE_F_SCORE, do_select = flags & ACACHE_F_SELECT;
+    const bool do_recompute = !(flags & ACACHE_F_NO_RECOMPUTE);
+    if ((s = check_weights(ctx, w, !do_recompute)) != ACACHE_OK) return s;
+    if (!x || !aligned16(x)) return fail(ctx, ACACHE_ERR_INVALID_ARG, "x NULL or misaligned");
+    if (do_score && x_is_compact) return fail(ctx, ACACHE_ERR_INVALID_ARG, "scoring needs the full [B, ctx_len, D] input");
+    if ((do_score || do_select) && !scores) return fail(ctx, ACACHE_ERR_INVALID_ARG, "scores is NULL");
+    if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
+    if (do_recompute && req->batch * (k + req->n_extra) > 0 && (!y || !aligned16(y))) return fail(ctx, ACACHE_ERR_INVALID_ARG, "y NULL or misaligned");
+
+    if (do_score && req->batch > 0 && req->affix_len > 0) {
+        void* qmask = wsp<void>(ctx, ctx->o_qmask);
+        if (req->n_masked > 0) {
+            int32_t* mpos = wsp<int32_t>(ctx, ctx->o_mrow_pos);
+            void* xnm = wsp<void>(ctx, ctx->o_xn_mask);
+            launch_gather_rmsnorm(x, 0, (int64_t)req->ctx_len * d.hidden, d.hidden, nullptr, 0, req->masked_pos,
+                                  req->n_masked, req->batch, req->affix_start, req->affix_len, req->ctx_len,
+                                  w->attn_norm_g, d.rms_eps, mpos, wsp<int64_t>(ctx, ctx->o_mrow_src), xnm,
+                                  wsp<uint32_t>(ctx, ctx->o_status), stream);
+            ctx->launches += 1;
+            GemmArgs g{};
+            g.a = xnm; g.M = req->batch * req->n_masked; g.K = d.hidden;
+            g.b[0] = w->wq; g.n[0] = d.n_heads * d.head_dim;
+            g.epilogue = kEpiQKV;
+            g.bias[0] = d.qkv_bias ? w->bq : nullptr;
+            g.row_pos = mpos; g.rope_cos = req->rope_cos; g.rope_sin = req->rope_sin;
+            g.head_dim = d.head_dim; g.rope_segments = 1; g.out[0] = qmask; g.rows_per_req = req->n_masked;
+            ctx->launches += launch_gemm(g, stream);
+        }
+        s = run_score(ctx, req, qmask, kv, scores, (flags & ACACHE_F_ACCUMULATE) ? 1 : 0,
+                      (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, stream);
+        if (s != ACACHE_OK) return s;
+    }
+    if (do_select && k > 0 && req->batch > 0) {
+        launch_topk(scores, req->batch, req->affix_len, k, anchor_idx, stream);
+        ctx->launches += 1;
+    }
+    if (do_recompute)
+        return run_recompute(ctx, w, req, kv, true, x, x_is_compact, anchor_idx, k, nullptr, nullptr, y, stream);
+    return check_cuda(ctx, "layer_step");
+}
+
+acache_status acache_layer_step_host(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
+                                     acache_kv* kv, const void* x_host, double ratio, uint32_t flags,
+                                     float* scores_host, int32_t* anchor_idx_host, void* y_host,
+                                     acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!req || !x_host || !scores_host || !y_host) return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL argument");
+    if (!ctx->ws) return fail(ctx, ACACHE_ERR_WORKSPACE, "workspace not set");
+    const acache_model_desc& d = ctx->d;
+    if (req->batch < 0 || req->batch > d.max_batch || req->ctx_len <= 0 || req->ctx_len > d.max_ctx ||
+        req->affix_len < 0 || req->affix_len > d.max_affix)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "batch / ctx_len / affix_len outside the context's limits");
+    const int k = acache_k_from_ratio(req->affix_len, ratio);
+    if (k > 0 && !anchor_idx_host) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx_host is NULL");
+    void* xs = wsp<void>(ctx, ctx->o_xstage);
+    void* ys = wsp<void>(ctx, ctx->o_ystage);
+    float* ss = wsp<float>(ctx, ctx->o_sstage);
+    int32_t* as = wsp<int32_t>(ctx, ctx->o_astage);
+    const size_t xb = (size_t)req->batch * req->ctx_len * d.hidden * 2;
+    if (cudaMemcpyAsync(xs, x_host, xb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return check_cuda(ctx, "H2D x");
+    acache_status s = acache_layer_step(ctx, w, req, kv, xs, 0, ratio, flags | ACACHE_F_SCORE | ACACHE_F_SELECT, ss, as,
+                                        ys, stream);
+    if (s != ACACHE_OK) return s;
+    const size_t rows = (size_t)req->batch * (k + req->n_extra);
+    bool ok = true;
+    if (!(flags & ACACHE_F_NO_RECOMPUTE) && rows)
+        ok &= cudaMemcpyAsync(y_host, ys, rows * d.hidden * 2, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (k) ok &= cudaMemcpyAsync(anchor_idx_host, as, (size_t)req->batch * k * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(scores_host, ss, (size_t)req->batch * req->affix_len * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (!ok) return check_cuda(ctx, "D2H") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "D2H copy failed") : ACACHE_ERR_CUDA;
+    return ACACHE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,208 @@
+// Bidirectional attention of the recomputed rows over the whole logical context
+// (Section 4.3: queries only for R, keys/values for all T positions, no mask).
+// Online-softmax tiles: S = Q K^T and O += P V on bf16 tensor-core tiles with fp32
+// accumulation and fp32 softmax statistics.  Keys/values come from the token-major cache or,
+// where a position -> fresh-row map says so, from the compact fresh K/V (the logical view of
+// the working cache without having written it).
+#include "common.cuh"
+#include "kernels.h"
+
+namespace acache {
+
+template <int D>
+struct AttnTile {
+    static constexpr int BYTES = 64 * D * 2;
+    static constexpr int CPR = D / 8;
+};
+
+template <int D>
+__device__ __forceinline__ void load_q_tile(uint32_t sdst, const __nv_bfloat16* q, int64_t stride, int valid, int tid) {
+    constexpr int CPR = D / 8;
+    for (int c = tid; c < 64 * CPR; c += 128) {
+        int r = c / CPR, cc = c % CPR;
+        int ok = r < valid;
+        cp_async16(sdst + (cc >> 3) * 8192 + swz64(r, cc & 7), q + (int64_t)(ok ? r : 0) * stride + cc * 8, ok ? 16 : 0);
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void load_kv_tile(uint32_t sk, uint32_t sv, const AttnArgs& a, int b, int kvh, int t0,
+                                             int tid) {
+    constexpr int CPR = D / 8;
+    const int64_t kstride = (int64_t)a.n_kv_heads * D;
+    const __nv_bfloat16* ck = static_cast<const __nv_bfloat16*>(a.cache_k) + (int64_t)b * a.kv_batch_stride + kvh * D;
+    const __nv_bfloat16* cv = static_cast<const __nv_bfloat16*>(a.cache_v) + (int64_t)b * a.kv_batch_stride + kvh * D;
+    const __nv_bfloat16* nk = static_cast<const __nv_bfloat16*>(a.k_new) + (int64_t)b * a.n * kstride + kvh * D;
+    const __nv_bfloat16* nv = static_cast<const __nv_bfloat16*>(a.v_new) + (int64_t)b * a.n * kstride + kvh * D;
+    for (int c = tid; c < 64 * CPR; c += 128) {
+        int r = c / CPR, cc = c % CPR;
+        int t = t0 + r;
+        int ok = t < a.ctx_len;
+        const __nv_bfloat16 *pk, *pv;
+        int s = (ok && a.slot) ? a.slot[(int64_t)b * a.ctx_len + t] : -1;
+        if (s >= 0) {
+            pk = nk + (int64_t)s * kstride;
+            pv = nv + (int64_t)s * kstride;
+        } else {
+            pk = ck + (int64_t)(ok ? t : 0) * kstride;
+            pv = cv + (int64_t)(ok ? t : 0) * kstride;
+        }
+        uint32_t off = (cc >> 3) * 8192 + swz64(r, cc & 7);
+        cp_async16(sk + off, pk + cc * 8, ok ? 16 : 0);
+        cp_async16(sv + off, pv + cc * 8, ok ? 16 : 0);
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float scale_log2e) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int TILE = 64 * D * 2;
+    const uint32_t sQ = smem_u32(smem);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int64_t qstride = (int64_t)a.n_heads * D;
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.q) + ((int64_t)b * a.n + qt * 64) * qstride + h * D;
+    const int ntiles = (a.ctx_len + 63) / 64;
+    auto sK = [&](int buf) { return sQ + TILE + buf * 2 * TILE; };
+    auto sV = [&](int buf) { return sQ + 2 * TILE + buf * 2 * TILE; };
+
+    load_q_tile<D>(sQ, q, qstride, min(64, a.n - qt * 64), tid);
+    load_kv_tile<D>(sK(0), sV(0), a, b, kvh, 0, tid);
+    cp_async_commit();
+    cp_async_wait<0>();
+    __syncthreads();
+
+    uint32_t qf[D / 16][4];
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+        int r = warp * 16 + (lane & 15);
+        int chunk = ks * 2 + (lane >> 4);
+        ldmatrix_x4(qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], sQ + (chunk >> 3) * 8192 + swz64(r, chunk & 7));
+    }
+
+    float o[D / 8][4];
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
+    float mx[2] = {-INFINITY, -INFINITY}, den[2] = {0.f, 0.f}, den_bf[2] = {0.f, 0.f};
+
+    for (int t = 0; t < ntiles; ++t) {
+        if (t + 1 < ntiles) {
+            load_kv_tile<D>(sK((t + 1) & 1), sV((t + 1) & 1), a, b, kvh, (t + 1) * 64, tid);
+            cp_async_commit();
+        }
+        const uint32_t sk = sK(t & 1), sv = sV(t & 1);
+        float s[8][4];
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) s[nb][i] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                int n = np * 16 + (lane & 7) + ((lane >> 4) << 3);
+                int chunk = ks * 2 + ((lane >> 3) & 1);
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4(b0, b1, b2, b3, sk + (chunk >> 3) * 8192 + swz64(n, chunk & 7));
+                mma_bf16_16816(s[np * 2], qf[ks], b0, b1);
+                mma_bf16_16816(s[np * 2 + 1], qf[ks], b2, b3);
+            }
+        }
+        const int valid = a.ctx_len - t * 64;
+        float tmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int col = nb * 8 + (lane & 3) * 2 + (i & 1);
+                float v = col < valid ? s[nb][i] * scale_log2e : -INFINITY;
+                s[nb][i] = v;
+                tmax[i >> 1] = fmaxf(tmax[i >> 1], v);
+            }
+        float corr[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 1));
+            tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 2));
+            float nm = fmaxf(mx[r], tmax[r]);
+            corr[r] = exp2f(mx[r] - nm);
+            mx[r] = nm;
+            den[r] *= corr[r];
+            den_bf[r] *= corr[r];
+        }
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) {
+            o[i][0] *= corr[0]; o[i][1] *= corr[0];
+            o[i][2] *= corr[1]; o[i][3] *= corr[1];
+        }
+        uint32_t pf[4][4];
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) {
+            float p0 = exp2f(s[nb][0] - mx[0]), p1 = exp2f(s[nb][1] - mx[0]);
+            float p2 = exp2f(s[nb][2] - mx[1]), p3 = exp2f(s[nb][3] - mx[1]);
+            den[0] += p0 + p1;
+            den[1] += p2 + p3;
+            uint32_t u01 = pack_bf16(p0, p1), u23 = pack_bf16(p2, p3);
+            den_bf[0] += bf16_lo(u01) + bf16_hi(u01);
+            den_bf[1] += bf16_lo(u23) + bf16_hi(u23);
+            pf[nb >> 1][(nb & 1) * 2] = u01;
+            pf[nb >> 1][(nb & 1) * 2 + 1] = u23;
+        }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+            for (int np = 0; np < D / 16; ++np) {
+                int key = kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                int chunk = np * 2 + (lane >> 4);
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(b0, b1, b2, b3, sv + (chunk >> 3) * 8192 + swz64(key, chunk & 7));
+                mma_bf16_16816(o[np * 2], pf[kk], b0, b1);
+                mma_bf16_16816(o[np * 2 + 1], pf[kk], b2, b3);
+            }
+        }
+        if (t + 1 < ntiles) cp_async_wait<0>();
+        __syncthreads();
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 1);
+        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 2);
+        den_bf[r] += __shfl_xor_sync(0xffffffffu, den_bf[r], 1);
+        den_bf[r] += __shfl_xor_sync(0xffffffffu, den_bf[r], 2);
+    }
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int row = qt * 64 + warp * 16 + (lane >> 2) + r * 8;
+        if (row >= a.n) continue;
+        const float inv = 1.f / den[r];
+        __nv_bfloat16* orow = out + ((int64_t)b * a.n + row) * qstride + h * D;
+#pragma unroll
+        for (int nb = 0; nb < D / 8; ++nb) {
+            int col = nb * 8 + (lane & 3) * 2;
+            *reinterpret_cast<uint32_t*>(orow + col) = pack_bf16(o[nb][r * 2] * inv, o[nb][r * 2 + 1] * inv);
+        }
+        if (a.row_sum && (lane & 3) == 0) a.row_sum[((int64_t)b * a.n + row) * a.n_heads + h] = den_bf[r] * inv;
+    }
+}
+
+int launch_attention(const AttnArgs& a, cudaStream_t stream) {
+    if (a.batch == 0 || a.n == 0) return 0;
+    const float scale_log2e = 1.4426950408889634f / sqrtf((float)a.head_dim);
+    dim3 grid((a.n + 63) / 64, a.n_heads, a.batch);
+    if (a.head_dim == 128) {
+        constexpr int SMEM = 5 * 64 * 128 * 2;
+        cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        attention_kernel<128><<<grid, 128, SMEM, stream>>>(a, scale_log2e);
+    } else {
+        constexpr int SMEM = 5 * 64 * 64 * 2;
+        cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        attention_kernel<64><<<grid, 128, SMEM, stream>>>(a, scale_log2e);
+    }
+    return 1;
+}
+
+}  // namespace acache

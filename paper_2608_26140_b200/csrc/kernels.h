@@ -1,0 +1,103 @@
+// Host-side launchers of the CUDA kernels (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace acache {
+
+// ---- rows.cu ----------------------------------------------------------------------------
+// Row plan of the recompute set R and RMSNorm of the gathered rows.
+// Row i of request b (i < k: anchor, else extra) sits at absolute position pos.
+// Writes row_pos[b*(k+e)+i] = pos (or -1 for an out-of-range index, which also sets
+// kFlagBadIndex), row_src = element offset of the row inside x, and
+// xn = bf16(x * rsqrt(mean(x^2)+eps) * g).
+void launch_gather_rmsnorm(const void* x, int x_is_compact, int64_t x_batch_stride, int hidden,
+                           const int32_t* anchor_idx, int k, const int32_t* extra_rows, int e,
+                           int batch, int affix_start, int affix_len, int ctx_len,
+                           const void* gain, float eps, int32_t* row_pos, int64_t* row_src, void* xn,
+                           uint32_t* status, cudaStream_t stream);
+
+// xn = bf16(RMSNorm(x) * g) for compact rows [n, hidden].
+void launch_rmsnorm(const void* x, const void* gain, float eps, int n, int hidden, void* xn,
+                    cudaStream_t stream);
+
+// cache[b, pos_r] = new[b, r] for K and V; rows with an invalid position are skipped.
+void launch_scatter_kv(void* cache_k, void* cache_v, int64_t batch_stride, int ctx_len,
+                       const int32_t* anchor_idx, int k, const int32_t* extra_rows, int e, int batch,
+                       int affix_start, int affix_len, int kv_dim, const void* k_new, const void* v_new,
+                       uint32_t* status, cudaStream_t stream);
+
+// slot[b, t] = compact row index whose fresh K/V replaces position t, or -1.
+void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
+                           cudaStream_t stream);
+
+// ---- score.cu ---------------------------------------------------------------------------
+struct ScoreArgs {
+    const void* q_mask;       // bf16 [B, m, H, d]
+    const void* cache_k;      // bf16 [B, cap, Hkv, d]
+    int64_t kv_batch_stride;  // elements
+    int batch, m, n_heads, n_kv_heads, head_dim;
+    int affix_start, affix_len;
+    int norm_lo, norm_len;    // key range of the softmax normaliser
+    float* row_stats;         // [B, H, n_split, m, 2]
+    float* head_partial;      // [B, H, L]
+    float* scores;            // [B, L]
+    int accumulate;
+};
+int score_num_splits(int norm_len);
+int launch_score(const ScoreArgs& a, cudaStream_t stream);  // returns number of kernels launched
+
+// ---- topk.cu ----------------------------------------------------------------------------
+void launch_topk(const float* scores, int batch, int affix_len, int k, int32_t* anchor_idx,
+                 cudaStream_t stream);
+
+// ---- gemm.cu ----------------------------------------------------------------------------
+enum GemmEpilogue : int {
+    kEpiQKV = 0,     // bias + RoPE on q/k segments, bf16 stores to q / k_new / v_new (+ optional cache scatter)
+    kEpiResidual,    // out = bf16(resid[row] + acc)
+    kEpiSwiGLU,      // out = bf16(silu(gate) * up), B tile = 64 gate rows + 64 up rows
+};
+
+struct GemmArgs {
+    const void* a;            // bf16 [M, K] row-major, lda = K
+    int M, K;
+    // B operand: up to three [N_i, K] row-major weight matrices laid side by side along N
+    const void* b[3];
+    int n[3];
+    int epilogue;
+    // --- kEpiQKV ---
+    const void* bias[3];      // bf16 [N_i] or null
+    const int32_t* row_pos;   // [M] absolute position per row (RoPE angle, scatter target); -1 = invalid
+    const float* rope_cos;    // [T, d/2]
+    const float* rope_sin;
+    int head_dim;
+    int rope_segments;        // number of leading segments that get RoPE (q only: 1, q+k: 2)
+    void* out[3];             // compact bf16 [M, N_i] per segment (may be null)
+    void* cache_k;            // optional fused scatter targets for segments 1 and 2
+    void* cache_v;
+    int64_t kv_batch_stride;
+    int rows_per_req;
+    // --- kEpiResidual ---
+    const void* resid;        // bf16 base pointer
+    const int64_t* resid_off; // [M] element offset of the residual row, or null => row * N
+    // --- kEpiSwiGLU / kEpiResidual output ---
+    void* c;                  // bf16 [M, Nout]
+};
+int launch_gemm(const GemmArgs& g, cudaStream_t stream);
+
+// ---- attn.cu ----------------------------------------------------------------------------
+struct AttnArgs {
+    const void* q;            // bf16 [B, n, H, d] compact
+    const void* cache_k;      // bf16 [B, cap, Hkv, d]
+    const void* cache_v;
+    int64_t kv_batch_stride;
+    const void* k_new;        // bf16 [B, n, Hkv, d] or null
+    const void* v_new;
+    const int32_t* slot;      // [B, ctx_len] or null: >= 0 => read k_new/v_new row slot
+    int batch, n, ctx_len, n_heads, n_kv_heads, head_dim;
+    void* o;                  // bf16 [B, n, H*d]
+    float* row_sum;           // optional [B, n, H]: sum of the normalised weights (debug)
+};
+int launch_attention(const AttnArgs& a, cudaStream_t stream);
+
+}  // namespace acache

@@ -1,0 +1,266 @@
+// Anchor scoring, Eq. 4-5:  a[j,k,h] = Softmax_j(q_mask[k,h] . K_affix[j,kv(h)] / sqrt(d)),
+// s_j (+)= sum_h sum_{k in M} a[j,k,h].
+//
+// Three kernels, no atomics on floats (bitwise reproducible):
+//   1. row statistics: for every masked query row and head, the softmax max and
+//      denominator over the normaliser's key range, split along the keys;
+//   2. column sums: for every affix key and head, sum over the masked queries of
+//      exp2(logit - max) / denominator (logits recomputed, K read a second time);
+//   3. ordered sum over heads into scores.
+// Logits run on the tensor cores (bf16 mma.sync, fp32 accumulate) so that the pass stays
+// bound by the K_affix read, not by ALU work.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace acache {
+
+constexpr int kScoreSplit = 256;      // keys per CTA in the statistics pass
+constexpr int kMaxMaskedSmem = 4096;  // masked rows whose statistics fit in shared memory
+
+int score_num_splits(int norm_len) { return (norm_len + kScoreSplit - 1) / kScoreSplit; }
+
+// Copy a [64 x D] bf16 tile (row stride `stride` elements) into swizzled shared memory:
+// D/64 panels of [64 rows x 64 cols], each row 128 bytes.  Rows >= valid are zero-filled.
+template <int D>
+__device__ __forceinline__ void load_tile64(uint32_t smem_base, const __nv_bfloat16* g, int64_t stride, int valid,
+                                            int tid, int nthreads) {
+    constexpr int CPR = D / 8;   // 16-byte chunks per row
+    for (int c = tid; c < 64 * CPR; c += nthreads) {
+        int r = c / CPR, cc = c % CPR;
+        int ok = r < valid;
+        const __nv_bfloat16* src = g + (int64_t)(ok ? r : 0) * stride + cc * 8;
+        cp_async16(smem_base + (cc >> 3) * 8192 + swz64(r, cc & 7), src, ok ? 16 : 0);
+    }
+}
+
+// A fragments (16 rows x D) of this warp's rows [row0, row0+16) from a swizzled tile.
+template <int D>
+__device__ __forceinline__ void load_a_frags(uint32_t (&a)[D / 16][4], uint32_t smem_base, int row0, int lane) {
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+        int r = row0 + (lane & 15);
+        int chunk = ks * 2 + (lane >> 4);
+        ldmatrix_x4(a[ks][0], a[ks][1], a[ks][2], a[ks][3], smem_base + (chunk >> 3) * 8192 + swz64(r, chunk & 7));
+    }
+}
+
+// acc[nb][4] = A(16 x D) * B^T where B is a swizzled [64 x D] tile (rows = n index).
+template <int D>
+__device__ __forceinline__ void mma_16x64(float (&acc)[8][4], const uint32_t (&a)[D / 16][4], uint32_t smem_b,
+                                          int lane) {
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nb][i] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+        for (int np = 0; np < 4; ++np) {
+            int n = np * 16 + (lane & 7) + ((lane >> 4) << 3);
+            int chunk = ks * 2 + ((lane >> 3) & 1);
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(b0, b1, b2, b3, smem_b + (chunk >> 3) * 8192 + swz64(n, chunk & 7));
+            mma_bf16_16816(acc[np * 2], a[ks], b0, b1);
+            mma_bf16_16816(acc[np * 2 + 1], a[ks], b2, b3);
+        }
+    }
+}
+
+// ---- pass 1: per-row softmax statistics over the normaliser's key range -------------------
+template <int D>
+__global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_split, float scale_log2e) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int TILE = 64 * D * 2;
+    const uint32_t sQ = smem_u32(smem), sK0 = sQ + TILE;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int split = blockIdx.x, h = blockIdx.y;
+    const int mtiles = (a.m + 63) / 64;
+    const int b = blockIdx.z / mtiles, mt = blockIdx.z % mtiles;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int64_t qstride = (int64_t)a.n_heads * D, kstride = (int64_t)a.n_kv_heads * D;
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.q_mask) +
+                             ((int64_t)b * a.m + mt * 64) * qstride + (int64_t)h * D;
+    const int key_lo = split * kScoreSplit;
+    const int key_n = min(kScoreSplit, a.norm_len - key_lo);
+    const __nv_bfloat16* kbase = static_cast<const __nv_bfloat16*>(a.cache_k) + (int64_t)b * a.kv_batch_stride +
+                                 (int64_t)(a.norm_lo + key_lo) * kstride + (int64_t)kvh * D;
+    const int ntiles = (key_n + 63) / 64;
+
+    load_tile64<D>(sQ, q, qstride, min(64, a.m - mt * 64), tid, 128);
+    load_tile64<D>(sK0, kbase, kstride, min(64, key_n), tid, 128);
+    cp_async_commit();
+    cp_async_wait<0>();
+    __syncthreads();
+    uint32_t af[D / 16][4];
+    load_a_frags<D>(af, sQ, warp * 16, lane);
+
+    float mx[2] = {-INFINITY, -INFINITY}, den[2] = {0.f, 0.f};
+    for (int t = 0; t < ntiles; ++t) {
+        const uint32_t sK = sK0 + (t & 1) * TILE;
+        if (t + 1 < ntiles) {
+            load_tile64<D>(sK0 + ((t + 1) & 1) * TILE, kbase + (int64_t)(t + 1) * 64 * kstride, kstride,
+                           min(64, key_n - (t + 1) * 64), tid, 128);
+            cp_async_commit();
+        }
+        float acc[8][4];
+        mma_16x64<D>(acc, af, sK, lane);
+        const int valid = key_n - t * 64;
+        float tmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int col = nb * 8 + (lane & 3) * 2 + (i & 1);
+                float s = col < valid ? acc[nb][i] * scale_log2e : -INFINITY;
+                acc[nb][i] = s;
+                tmax[i >> 1] = fmaxf(tmax[i >> 1], s);
+            }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 1));
+            tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 2));
+            float nm = fmaxf(mx[r], tmax[r]);
+            den[r] *= exp2f(mx[r] - nm);
+            mx[r] = nm;
+        }
+        float part[2] = {0.f, 0.f};
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) part[i >> 1] += exp2f(acc[nb][i] - mx[i >> 1]);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            part[r] += __shfl_xor_sync(0xffffffffu, part[r], 1);
+            part[r] += __shfl_xor_sync(0xffffffffu, part[r], 2);
+            den[r] += part[r];
+        }
+        if (t + 1 < ntiles) cp_async_wait<0>();
+        __syncthreads();
+    }
+    if ((lane & 3) == 0) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            int row = mt * 64 + warp * 16 + (lane >> 2) + r * 8;
+            if (row < a.m) {
+                float* st = a.row_stats + ((((int64_t)b * a.n_heads + h) * n_split + split) * a.m + row) * 2;
+                st[0] = mx[r];
+                st[1] = den[r];
+            }
+        }
+    }
+}
+
+// ---- pass 2: per-key column sums of the normalised weights -------------------------------
+template <int D>
+__global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_split, float scale_log2e) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int TILE = 64 * D * 2;
+    const uint32_t sK = smem_u32(smem), sQ0 = sK + TILE;
+    float* s_max = reinterpret_cast<float*>(smem + 3 * TILE);
+    float* s_inv = s_max + a.m;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int jt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int64_t qstride = (int64_t)a.n_heads * D, kstride = (int64_t)a.n_kv_heads * D;
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.q_mask) + (int64_t)b * a.m * qstride + (int64_t)h * D;
+    const int j0 = jt * 64;
+    const __nv_bfloat16* kbase = static_cast<const __nv_bfloat16*>(a.cache_k) + (int64_t)b * a.kv_batch_stride +
+                                 (int64_t)(a.affix_start + j0) * kstride + (int64_t)kvh * D;
+    const int mtiles = (a.m + 63) / 64;
+
+    load_tile64<D>(sK, kbase, kstride, min(64, a.affix_len - j0), tid, 128);
+    load_tile64<D>(sQ0, q, qstride, min(64, a.m), tid, 128);
+    cp_async_commit();
+
+    // combine the split statistics of every masked row (fixed order)
+    const float* st = a.row_stats + ((int64_t)b * a.n_heads + h) * n_split * a.m * 2;
+    for (int r = tid; r < a.m; r += 128) {
+        float M = -INFINITY;
+        for (int s = 0; s < n_split; ++s) M = fmaxf(M, st[((int64_t)s * a.m + r) * 2]);
+        float Dn = 0.f;
+        for (int s = 0; s < n_split; ++s)
+            Dn += st[((int64_t)s * a.m + r) * 2 + 1] * exp2f(st[((int64_t)s * a.m + r) * 2] - M);
+        s_max[r] = M;
+        s_inv[r] = 1.f / Dn;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    uint32_t af[D / 16][4];
+    load_a_frags<D>(af, sK, warp * 16, lane);
+
+    float colsum[2] = {0.f, 0.f};
+    for (int t = 0; t < mtiles; ++t) {
+        const uint32_t sQ = sQ0 + (t & 1) * TILE;
+        if (t + 1 < mtiles) {
+            load_tile64<D>(sQ0 + ((t + 1) & 1) * TILE, q + (int64_t)(t + 1) * 64 * qstride, qstride,
+                           min(64, a.m - (t + 1) * 64), tid, 128);
+            cp_async_commit();
+        }
+        float acc[8][4];
+        mma_16x64<D>(acc, af, sQ, lane);   // rows = keys, cols = masked queries
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int qrow = t * 64 + nb * 8 + (lane & 3) * 2 + (i & 1);
+                if (qrow < a.m) colsum[i >> 1] += exp2f(acc[nb][i] * scale_log2e - s_max[qrow]) * s_inv[qrow];
+            }
+        if (t + 1 < mtiles) cp_async_wait<0>();
+        __syncthreads();
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        colsum[r] += __shfl_xor_sync(0xffffffffu, colsum[r], 1);
+        colsum[r] += __shfl_xor_sync(0xffffffffu, colsum[r], 2);
+    }
+    if ((lane & 3) == 0) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            int j = j0 + warp * 16 + (lane >> 2) + r * 8;
+            if (j < a.affix_len) a.head_partial[((int64_t)b * a.n_heads + h) * a.affix_len + j] = colsum[r];
+        }
+    }
+}
+
+// ---- pass 3: ordered sum over heads -------------------------------------------------------
+__global__ void __launch_bounds__(256) score_reduce_heads_kernel(const float* __restrict__ head_partial,
+                                                                 float* __restrict__ scores, int n_heads, int L,
+                                                                 int accumulate) {
+    const int b = blockIdx.y;
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= L) return;
+    float s = 0.f;
+    for (int h = 0; h < n_heads; ++h) s += head_partial[((int64_t)b * n_heads + h) * L + j];
+    float* out = scores + (int64_t)b * L + j;
+    *out = accumulate ? *out + s : s;
+}
+
+template <int D>
+static int launch_score_d(const ScoreArgs& a, cudaStream_t stream) {
+    const int n_split = score_num_splits(a.norm_len);
+    const float scale_log2e = 1.4426950408889634f / sqrtf((float)D);
+    constexpr int TILE = 64 * D * 2;
+    const int mtiles = (a.m + 63) / 64;
+    const size_t smem1 = 3 * TILE;
+    const size_t smem2 = 3 * TILE + (size_t)a.m * 8;
+    cudaFuncSetAttribute(score_stats_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
+    cudaFuncSetAttribute(score_colsum_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+    score_stats_kernel<D><<<dim3(n_split, a.n_heads, a.batch * mtiles), 128, smem1, stream>>>(a, n_split, scale_log2e);
+    score_colsum_kernel<D><<<dim3((a.affix_len + 63) / 64, a.n_heads, a.batch), 128, smem2, stream>>>(a, n_split,
+                                                                                                     scale_log2e);
+    score_reduce_heads_kernel<<<dim3((a.affix_len + 255) / 256, a.batch), 256, 0, stream>>>(
+        a.head_partial, a.scores, a.n_heads, a.affix_len, a.accumulate);
+    return 3;
+}
+
+int launch_score(const ScoreArgs& a, cudaStream_t stream) {
+    if (a.batch == 0 || a.affix_len == 0) return 0;
+    if (a.m == 0) {   // no masked rows: this layer contributes nothing
+        if (!a.accumulate) cudaMemsetAsync(a.scores, 0, (size_t)a.batch * a.affix_len * sizeof(float), stream);
+        return 0;
+    }
+    if (a.m > kMaxMaskedSmem) return -1;
+    return a.head_dim == 128 ? launch_score_d<128>(a, stream) : launch_score_d<64>(a, stream);
+}
+
+}  // namespace acache

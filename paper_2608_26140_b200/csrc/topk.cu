@@ -1,0 +1,123 @@
+// Top-K anchor selection, Eq. 6: A = TopK({s_j}, K).  One CTA per request: an exact
+// radix select on the fp32 bit pattern finds the K-th largest score, then one ordered
+// pass over positions emits the anchors ascending, ties going to the lower position.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace acache {
+
+constexpr int kTopkThreads = 1024;
+constexpr int kTopkSmemKeys = 16384;   // keys cached in shared memory up to this L
+
+// Order-preserving map fp32 -> uint32 (larger float <=> larger key).
+__device__ __forceinline__ uint32_t score_key(float f) {
+    uint32_t u = __float_as_uint(f);
+    if (u == 0x80000000u) u = 0u;   // -0 and +0 compare equal
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Exclusive block scan of one int per thread (blockDim.x == kTopkThreads); returns the
+// exclusive prefix and writes the block total to *total.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) warp_tot[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+        int t = warp_tot[lane];
+        int ti = t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int u = __shfl_up_sync(0xffffffffu, ti, o);
+            if (lane >= o) ti += u;
+        }
+        warp_tot[lane] = ti - t;          // exclusive warp offsets
+        if (lane == 31) *total = ti;
+    }
+    __syncthreads();
+    int r = warp_tot[w] + inc - v;
+    __syncthreads();
+    return r;
+}
+
+__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restrict__ scores, int L, int K,
+                                                            int32_t* __restrict__ anchor_idx, int use_smem) {
+    extern __shared__ uint32_t keys_s[];
+    __shared__ int hist[256];
+    __shared__ int warp_tot[32];
+    __shared__ int s_total;
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_want;
+
+    const int b = blockIdx.x;
+    const float* s = scores + (int64_t)b * L;
+    int32_t* out = anchor_idx + (int64_t)b * K;
+    const int tid = threadIdx.x;
+
+    if (use_smem)
+        for (int j = tid; j < L; j += kTopkThreads) keys_s[j] = score_key(s[j]);
+    if (tid == 0) { s_prefix = 0u; s_want = K; }
+    __syncthreads();
+    auto key_at = [&](int j) -> uint32_t { return use_smem ? keys_s[j] : score_key(s[j]); };
+
+    // radix select, most significant byte first: after the loop s_prefix is the key of the
+    // K-th largest element and s_want the number of elements equal to it that are taken.
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const uint32_t mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+        if (tid < 256) hist[tid] = 0;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        for (int j = tid; j < L; j += kTopkThreads) {
+            uint32_t kk = key_at(j);
+            if ((kk & mask) == prefix) atomicAdd(&hist[(kk >> shift) & 0xFF], 1);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int want = s_want, d = 255;
+            for (; d > 0; --d) {           // walk down from the largest digit
+                if (hist[d] >= want) break;
+                want -= hist[d];
+            }
+            s_prefix = prefix | ((uint32_t)d << shift);
+            s_want = want;
+        }
+        __syncthreads();
+    }
+    const uint32_t tau = s_prefix;
+    const int need_eq = s_want;
+
+    // ordered compaction: position ascending, chunk by chunk
+    int base_eq = 0, base_out = 0;
+    for (int j0 = 0; j0 < L; j0 += kTopkThreads) {
+        const int j = j0 + tid;
+        uint32_t kk = j < L ? key_at(j) : 0u;
+        const int is_gt = (j < L) && (kk > tau);
+        const int is_eq = (j < L) && (kk == tau);
+        int eq_rank = base_eq + block_exclusive_scan(is_eq, warp_tot, &s_total);
+        const int eq_total = s_total;
+        const int sel = is_gt || (is_eq && eq_rank < need_eq);
+        int o = base_out + block_exclusive_scan(sel, warp_tot, &s_total);
+        const int sel_total = s_total;
+        if (sel && o < K) out[o] = j;
+        base_eq += eq_total;
+        base_out += sel_total;
+    }
+}
+
+void launch_topk(const float* scores, int batch, int affix_len, int k, int32_t* anchor_idx, cudaStream_t stream) {
+    if (batch == 0 || k == 0) return;
+    const int use_smem = affix_len <= kTopkSmemKeys;
+    const size_t smem = use_smem ? (size_t)affix_len * sizeof(uint32_t) : 0;
+    if (smem > 48 * 1024)
+        cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kTopkSmemKeys * (int)sizeof(uint32_t));
+    topk_kernel<<<batch, kTopkThreads, smem, stream>>>(scores, affix_len, k, anchor_idx, use_smem);
+}
+
+}  // namespace acache

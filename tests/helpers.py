@@ -1,0 +1,86 @@
+"""Shared plumbing of the GPU parity tests: move a seeded host case to the device, run
+the C-ABI calls through the binding, and compare with the CPU oracle."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import acache_oracle as orc
+from paper_2608_26140_b200 import binding as ab
+from paper_2608_26140_b200 import workloads as wl
+
+DEV = "cuda:0"
+TOL = 2e-2     # max relative error of refreshed K/V and layer outputs (bf16 storage, fp32 accumulate)
+
+
+class DeviceCase:
+    """Device copies of a workloads.Case plus a context sized for it."""
+
+    def __init__(self, case: wl.Case, max_rows=None):
+        self.case = case
+        s, lay = case.shape, case.layout
+        self.w_dev = {k: (ab.to_device_bf16(v, DEV) if v is not None else None) for k, v in case.weights.items()}
+        self.lw = ab.Context.weights(self.w_dev)
+        self.x = ab.to_device_bf16(case.x, DEV)
+        self.ck = ab.to_device_bf16(case.cache_k, DEV)
+        self.cv = ab.to_device_bf16(case.cache_v, DEV)
+        self.cos = torch.from_numpy(case.rope_cos).to(DEV)
+        self.sin = torch.from_numpy(case.rope_sin).to(DEV)
+        self.masked = torch.from_numpy(lay.masked_pos).to(DEV)
+        self.extra = torch.from_numpy(lay.extra_rows).to(DEV) if lay.n_extra else None
+        self.req = ab.Context.request(lay.batch, lay.ctx_len, lay.affix_start, lay.affix_len, self.masked,
+                                      self.extra, self.cos, self.sin)
+        rows = max_rows if max_rows is not None else lay.affix_len + lay.n_extra
+        self.ctx = ab.Context.for_shape(s, lay.batch, lay.ctx_len, lay.affix_len, max(rows, 1),
+                                        max(lay.n_masked, 1), DEV)
+
+    def kv(self):
+        return ab.Context.kv(self.ck, self.cv)
+
+    def reset_cache(self):
+        self.ck.copy_(ab.to_device_bf16(self.case.cache_k, DEV))
+        self.cv.copy_(ab.to_device_bf16(self.case.cache_v, DEV))
+
+
+def oracle_step(case: wl.Case, b: int, **kw):
+    lay = case.layout
+    return orc.layer_step(case.weights, case.shape, case.x[b], case.cache_k[b], case.cache_v[b], lay.ctx_len,
+                          lay.affix_start, lay.affix_len, lay.masked_pos[b], lay.extra_rows[b],
+                          case.rope_cos, case.rope_sin, **kw)
+
+
+def assert_close_bf16(gpu_bits: np.ndarray, ref: np.ndarray, what: str, tol: float = TOL):
+    """|a - b| <= tol * max(|b|, rms(b)) elementwise; ``ref`` is fp64 values or bf16 bits."""
+    a = orc.bf16_bits_to_f64(gpu_bits)
+    b = orc.bf16_bits_to_f64(ref) if ref.dtype == np.uint16 else ref
+    assert a.shape == b.shape, (what, a.shape, b.shape)
+    ok, worst = orc.rel_err_gate(a, b, tol)
+    assert ok, f"{what}: worst relative error {worst:.4g} > {tol}"
+    return worst
+
+
+def projected_cache(case: wl.Case, hidden_bits: np.ndarray):
+    """Exact K/V of every position computed by the oracle from the given hidden states
+    (used to build 'the same affix under another suffix' stale caches)."""
+    B, T = hidden_bits.shape[:2]
+    ck = np.empty_like(case.cache_k)
+    cv = np.empty_like(case.cache_v)
+    for b in range(B):
+        xn = orc.normed_rows(case.weights, case.shape, orc.bf16_bits_to_f64(hidden_bits[b]))
+        k, v = orc.project_kv(case.weights, case.shape, xn, np.arange(T), case.rope_cos, case.rope_sin)
+        ck[b, :T] = orc.f64_to_bf16_bits(k)
+        cv[b, :T] = orc.f64_to_bf16_bits(v)
+    return ck, cv
+
+
+def make_projected_case(shape, lay, ratio, cfg_id=0):
+    """Case whose cache holds: affix rows = exact KV of the affix under ANOTHER context
+    (stale), all other rows = exact KV under the current context."""
+    case = wl.make_case(shape, lay, ratio, cfg_id, with_stale_hidden=True)
+    cur_k, cur_v = projected_cache(case, case.x)
+    old_k, old_v = projected_cache(case, case.x_stale)
+    l, L = lay.affix_start, lay.affix_len
+    cur_k[:, l:l + L] = old_k[:, l:l + L]
+    cur_v[:, l:l + L] = old_v[:, l:l + L]
+    case.cache_k, case.cache_v = cur_k, cur_v
+    return case

@@ -1,0 +1,347 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Integer work (anchor indices, untouched cache rows) is compared exactly,
+up to the 1e-3 relative band around the K-th score; bf16 tensors within 2e-2."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import acache_oracle as orc
+from paper_2608_26140_b200 import binding as ab
+from paper_2608_26140_b200 import workloads as wl
+
+from helpers import DEV, TOL, DeviceCase, assert_close_bf16, make_projected_case, oracle_step
+
+pytestmark = pytest.mark.gpu
+
+MID128 = wl.LayerShape(512, 4, 2, 128, 1024, 1e-5, True, 5e5, "mid-d128")
+
+
+def dev_i32(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(DEV)
+
+
+# ------------------------------------------------------------------ Eq. 4-5
+@pytest.mark.parametrize("shape,B,pre,L,post,m,norm_full", [
+    (wl.TINY, 1, 0, 128, 64, 32, False),
+    (wl.TINY, 2, 5, 300, 33, 70, False),       # ragged L and m, affix in the middle
+    (wl.TINY_GQA, 2, 0, 257, 10, 1, True),
+    (MID128, 2, 16, 520, 40, 32, False),
+    (MID128, 1, 0, 1, 64, 3, False),           # one affix token
+    (MID128, 1, 7, 700, 64, 130, True),
+    (wl.LLADA_8B, 1, 0, 512, 256, 32, False),
+])
+def test_score_anchors(shape, B, pre, L, post, m, norm_full):
+    lay = wl.make_layout(B, pre, L, post, max(m, 1), m)
+    T = lay.ctx_len
+    ck, _ = wl.random_kv_cache(shape, lay, 77)
+    q = wl.random_q_mask(shape, lay, 78)
+    ctx = ab.Context.for_shape(shape, B, T, L, 1, max(m, 1), DEV)
+    dk = ab.to_device_bf16(ck, DEV)
+    dq = ab.to_device_bf16(q, DEV)
+    masked = dev_i32(lay.masked_pos)
+    req = ab.Context.request(B, T, lay.affix_start, L, masked, None, None, None)
+    scores = torch.full((B, L), 3.0, dtype=torch.float32, device=DEV)
+    ctx.score_anchors(req, dq, ab.Context.kv(dk, dk), scores, accumulate=False, norm_full=norm_full)
+    ctx.score_anchors(req, dq, ab.Context.kv(dk, dk), scores, accumulate=True, norm_full=norm_full)
+    torch.cuda.synchronize()
+    s_gpu = scores.cpu().numpy().astype(np.float64)
+    for b in range(B):
+        kf = orc.bf16_bits_to_f64(ck[b, :T])
+        ref = 2.0 * orc.score_anchors(orc.bf16_bits_to_f64(q[b]), kf[lay.affix_start:lay.affix_start + L], kf,
+                                      lay.affix_start, norm_full)
+        err = np.abs(s_gpu[b] - ref) / np.maximum(ref, ref.mean())
+        assert err.max() < 1e-3, (b, err.max())
+        if not norm_full:
+            assert abs(s_gpu[b].sum() - 2.0 * shape.n_heads * m) < 1e-3 * shape.n_heads * m
+    assert ctx.poll_status() == 0
+
+
+def test_score_is_bitwise_reproducible():
+    shape, B, L, m = MID128, 2, 1000, 64
+    lay = wl.make_layout(B, 0, L, 8, m, m)
+    ck, _ = wl.random_kv_cache(shape, lay, 5)
+    q = wl.random_q_mask(shape, lay, 6)
+    ctx = ab.Context.for_shape(shape, B, lay.ctx_len, L, 1, m, DEV)
+    dk, dq = ab.to_device_bf16(ck, DEV), ab.to_device_bf16(q, DEV)
+    req = ab.Context.request(B, lay.ctx_len, 0, L, dev_i32(lay.masked_pos), None, None, None)
+    outs = []
+    for _ in range(3):
+        s = torch.empty((B, L), dtype=torch.float32, device=DEV)
+        ctx.score_anchors(req, dq, ab.Context.kv(dk, dk), s)
+        outs.append(s.cpu().numpy())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
+# ------------------------------------------------------------------ Eq. 6
+@pytest.mark.parametrize("B,L", [(1, 1), (3, 7), (2, 1000), (2, 1024), (1, 8192), (2, 16384), (1, 20000)])
+def test_select_topk_exact(B, L):
+    g = np.random.default_rng(L)
+    ctx = ab.Context.for_shape(wl.TINY, B, 256, 128, 1, 1, DEV)
+    for trial, K in enumerate(sorted({0, 1, L // 5, L // 2, L - 1, L})):
+        if K < 0:
+            continue
+        s = g.random((B, L)).astype(np.float32)
+        if trial % 2 == 0 and L > 4:           # heavy ties around the threshold
+            s = np.round(s * 8) / 8
+        s[:, L // 2] = -0.0
+        ds = torch.from_numpy(s).to(DEV)
+        out = torch.full((B, max(K, 1)), -7, dtype=torch.int32, device=DEV)
+        ctx.select_topk(ds, B, L, K, out)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy()
+        for b in range(B):
+            ref = orc.select_topk(s[b], K)[0]
+            assert np.array_equal(got[b, :K], ref), (B, L, K, b)
+    # all-equal scores: lowest positions win
+    ds = torch.full((B, L), 0.25, device=DEV)
+    K = max(1, L // 3)
+    out = torch.empty((B, K), dtype=torch.int32, device=DEV)
+    ctx.select_topk(ds, B, L, K, out)
+    assert np.array_equal(out.cpu().numpy(), np.broadcast_to(np.arange(K, dtype=np.int32), (B, K)))
+
+
+# ------------------------------------------------------------------ selective recompute + scatter
+def run_split_calls(dc: DeviceCase, anchor_idx_dev, K):
+    s, lay = dc.case.shape, dc.case.layout
+    n = K + lay.n_extra
+    B = lay.batch
+    k_new = torch.zeros((B, max(n, 1), s.n_kv_heads, s.head_dim), dtype=torch.bfloat16, device=DEV)
+    v_new = torch.zeros_like(k_new)
+    y = torch.zeros((B, max(n, 1), s.hidden), dtype=torch.bfloat16, device=DEV)
+    dc.ctx.recompute_anchors(dc.lw, dc.req, dc.kv(), dc.x, 0, anchor_idx_dev, K, k_new, v_new, y)
+    return k_new, v_new, y
+
+
+def check_against_oracle(dc, anchors, k_new, v_new, y, cache_k_bits, cache_v_bits, K):
+    """Teacher-forced comparison: the oracle recomputes with the GPU's anchor set."""
+    case, lay = dc.case, dc.case.layout
+    n = K + lay.n_extra
+    worst = 0.0
+    for b in range(lay.batch):
+        ref = oracle_step(case, b, anchor_idx=anchors[b, :K])
+        worst = max(worst, assert_close_bf16(ab.to_host_bits(k_new[b, :n]), ref["k_new"], "k_new"))
+        worst = max(worst, assert_close_bf16(ab.to_host_bits(v_new[b, :n]), ref["v_new"], "v_new"))
+        worst = max(worst, assert_close_bf16(ab.to_host_bits(y[b, :n]), ref["y"], "y"))
+        if cache_k_bits is not None:
+            rows = ref["rows"]
+            keep = np.setdiff1d(np.arange(case.cache_k.shape[1]), rows)
+            assert np.array_equal(cache_k_bits[b][keep], case.cache_k[b][keep]), "untouched K rows changed"
+            assert np.array_equal(cache_v_bits[b][keep], case.cache_v[b][keep]), "untouched V rows changed"
+            assert_close_bf16(cache_k_bits[b][rows], ref["k_new"], "cache K rows")
+            assert_close_bf16(cache_v_bits[b][rows], ref["v_new"], "cache V rows")
+    return worst
+
+
+@pytest.mark.parametrize("shape,B,pre,L,post,gen,m,extra,ratio", [
+    (wl.TINY, 1, 0, 128, 64, 32, 32, "none", 0.2),
+    (wl.TINY, 2, 9, 100, 20, 40, 32, "all", 0.2),       # affix in the middle, ragged tiles
+    (wl.TINY_GQA, 2, 0, 130, 31, 33, 33, "masked", 0.35),
+    (MID128, 2, 4, 200, 30, 32, 32, "all", 0.1),
+    (MID128, 1, 0, 64, 16, 16, 16, "none", 1.0),
+])
+def test_recompute_then_scatter(shape, B, pre, L, post, gen, m, extra, ratio):
+    lay = wl.make_layout(B, pre, L, post, gen, m, extra)
+    case = make_projected_case(shape, lay, ratio, cfg_id=11)
+    dc = DeviceCase(case)
+    K = orc.k_from_ratio(L, ratio)
+    # any valid anchor set will do for the split calls: take a seeded random one
+    g = np.random.default_rng(3)
+    anchors = np.stack([np.sort(g.choice(L, K, replace=False)) for _ in range(B)]).astype(np.int32)
+    da = dev_i32(anchors)
+    k_new, v_new, y = run_split_calls(dc, da, K)
+    torch.cuda.synchronize()
+    # recompute must not have touched the cache
+    assert np.array_equal(ab.to_host_bits(dc.ck), case.cache_k) and np.array_equal(ab.to_host_bits(dc.cv), case.cache_v)
+    dc.ctx.scatter_kv(dc.req, dc.kv(), da, K, k_new, v_new)
+    torch.cuda.synchronize()
+    ckb, cvb = ab.to_host_bits(dc.ck), ab.to_host_bits(dc.cv)
+    check_against_oracle(dc, anchors, k_new, v_new, y, ckb, cvb, K)
+    # the scattered rows are bit-identical to k_new / v_new
+    n = K + lay.n_extra
+    for b in range(B):
+        rows = orc.recompute_set(anchors[b], lay.affix_start, lay.extra_rows[b])
+        assert np.array_equal(ckb[b][rows], ab.to_host_bits(k_new[b, :n]))
+        assert np.array_equal(cvb[b][rows], ab.to_host_bits(v_new[b, :n]))
+    assert dc.ctx.poll_status() == 0
+
+
+# ------------------------------------------------------------------ the chained layer-step
+def run_layer_step(dc: DeviceCase, ratio, flags, anchors_in=None):
+    s, lay = dc.case.shape, dc.case.layout
+    B, L = lay.batch, lay.affix_len
+    K = orc.k_from_ratio(L, ratio)
+    n = K + lay.n_extra
+    scores = torch.zeros((B, L), dtype=torch.float32, device=DEV)
+    anchors = torch.full((B, max(K, 1)), -1, dtype=torch.int32, device=DEV)
+    if anchors_in is not None:
+        anchors[:, :K] = dev_i32(anchors_in)
+    y = torch.zeros((B, max(n, 1), s.hidden), dtype=torch.bfloat16, device=DEV)
+    dc.ctx.layer_step(dc.lw, dc.req, dc.kv(), dc.x, 0, ratio, flags, scores, anchors, y)
+    torch.cuda.synchronize()
+    return K, scores.cpu().numpy(), anchors.cpu().numpy(), y
+
+
+@pytest.mark.parametrize("shape,B,pre,L,post,gen,m,extra", [
+    (wl.TINY, 1, 0, 128, 64, 32, 32, "none"),          # benchmark config 1 (tail rows folded into gen)
+    (wl.TINY, 2, 16, 128, 48, 64, 32, "all"),
+    (wl.TINY_GQA, 2, 0, 200, 24, 32, 32, "all"),
+    (MID128, 2, 8, 260, 30, 34, 32, "masked"),
+])
+@pytest.mark.parametrize("ratio", [0.0, 0.2, 1.0])
+def test_layer_step(shape, B, pre, L, post, gen, m, extra, ratio):
+    lay = wl.make_layout(B, pre, L, post, gen, m, extra)
+    case = make_projected_case(shape, lay, ratio, cfg_id=12)
+    dc = DeviceCase(case)
+    K, s_gpu, a_gpu, y = run_layer_step(dc, ratio, ab.F_SCORE | ab.F_SELECT)
+    n = K + lay.n_extra
+    ckb, cvb = ab.to_host_bits(dc.ck), ab.to_host_bits(dc.cv)
+    for b in range(B):
+        free = oracle_step(case, b, ratio=ratio)                     # the oracle's own selection
+        err = np.abs(s_gpu[b] - free["scores64"]) / np.maximum(free["scores64"], free["scores64"].mean())
+        assert err.max() < 1e-3
+        ok, why = orc.anchor_set_ok(a_gpu[b, :K], K, L, free["must"], free["may"])
+        assert ok, why
+        ref = oracle_step(case, b, anchor_idx=a_gpu[b, :K])          # teacher-forced on the GPU's set
+        rows = ref["rows"]
+        keep = np.setdiff1d(np.arange(lay.ctx_len), rows)
+        assert np.array_equal(ckb[b][keep], case.cache_k[b][keep]) and np.array_equal(cvb[b][keep], case.cache_v[b][keep])
+        if n:
+            assert_close_bf16(ckb[b][rows], ref["k_new"], "K rows")
+            assert_close_bf16(cvb[b][rows], ref["v_new"], "V rows")
+            assert_close_bf16(ab.to_host_bits(y[b, :n]), ref["y"], "y")
+        if ratio == 1.0 and extra == "all":
+            # full recompute == the dense layer written separately in the oracle
+            yd, kd, vd = orc.dense_layer(case.weights, shape, case.x[b], case.rope_cos, case.rope_sin)
+            assert_close_bf16(ckb[b][:lay.ctx_len], kd, "K vs dense")
+            assert_close_bf16(cvb[b][:lay.ctx_len], vd, "V vs dense")
+            assert_close_bf16(ab.to_host_bits(y[b, :n]), yd[rows], "y vs dense")
+        if ratio == 0.0:
+            l = lay.affix_start
+            assert np.array_equal(ckb[b][l:l + L], case.cache_k[b][l:l + L])
+    assert dc.ctx.poll_status() == 0
+
+
+def test_fused_step_equals_split_calls():
+    lay = wl.make_layout(2, 6, 150, 20, 32, 32, "all")
+    case = make_projected_case(MID128, lay, 0.2, cfg_id=13)
+    dc = DeviceCase(case)
+    K, s_gpu, a_gpu, y_fused = run_layer_step(dc, 0.2, ab.F_SCORE | ab.F_SELECT)
+    ck_fused, cv_fused = ab.to_host_bits(dc.ck), ab.to_host_bits(dc.cv)
+    dc.reset_cache()
+    da = dev_i32(a_gpu[:, :K])
+    k_new, v_new, y_split = run_split_calls(dc, da, K)
+    dc.ctx.scatter_kv(dc.req, dc.kv(), da, K, k_new, v_new)
+    torch.cuda.synchronize()
+    assert np.array_equal(ab.to_host_bits(dc.ck), ck_fused) and np.array_equal(ab.to_host_bits(dc.cv), cv_fused)
+    n = K + lay.n_extra
+    assert_close_bf16(ab.to_host_bits(y_split[:, :n]), ab.to_host_bits(y_fused[:, :n]), "split vs fused y")
+    # a second fused step with the anchors given (no scoring) reproduces the first bit for bit
+    dc.reset_cache()
+    _, _, _, y2 = run_layer_step(dc, 0.2, 0, anchors_in=a_gpu[:, :K])
+    assert np.array_equal(ab.to_host_bits(y2), ab.to_host_bits(y_fused))
+    assert np.array_equal(ab.to_host_bits(dc.ck), ck_fused)
+
+
+def test_idempotent_when_cache_is_current():
+    """Cache computed from the very hidden rows being refreshed: refreshed K/V stay within
+    tolerance of the cached ones (the oracle gives identical bytes)."""
+    lay = wl.make_layout(1, 0, 128, 32, 32, 32, "all")
+    case = wl.make_case(wl.TINY, lay, 0.5, cfg_id=14)
+    from helpers import projected_cache
+    case.cache_k, case.cache_v = projected_cache(case, case.x)
+    dc = DeviceCase(case)
+    run_layer_step(dc, 0.5, ab.F_SCORE | ab.F_SELECT)
+    assert_close_bf16(ab.to_host_bits(dc.ck), case.cache_k, "K idempotent")
+    assert_close_bf16(ab.to_host_bits(dc.cv), case.cache_v, "V idempotent")
+
+
+def test_compact_input_matches_gathered_input():
+    lay = wl.make_layout(2, 0, 128, 16, 32, 32, "masked")
+    case = make_projected_case(wl.TINY, lay, 0.25, cfg_id=15)
+    dc = DeviceCase(case)
+    K, _, a_gpu, y_full = run_layer_step(dc, 0.25, ab.F_SCORE | ab.F_SELECT)
+    n = K + lay.n_extra
+    rows = np.stack([orc.recompute_set(a_gpu[b, :K], lay.affix_start, lay.extra_rows[b]) for b in range(2)])
+    xc = torch.stack([dc.x[b, torch.from_numpy(rows[b]).to(DEV)] for b in range(2)]).contiguous()
+    dc.reset_cache()
+    y = torch.zeros((2, n, case.shape.hidden), dtype=torch.bfloat16, device=DEV)
+    anchors = dev_i32(a_gpu[:, :K])
+    dc.ctx.layer_step(dc.lw, dc.req, dc.kv(), xc, 1, 0.25, 0, None, anchors, y)
+    torch.cuda.synchronize()
+    assert np.array_equal(ab.to_host_bits(y), ab.to_host_bits(y_full[:, :n]))
+
+
+def test_out_of_range_index_is_flagged_and_skipped():
+    lay = wl.make_layout(1, 0, 128, 16, 32, 32, "none")
+    case = wl.make_case(wl.TINY, lay, 0.1, cfg_id=16)
+    dc = DeviceCase(case)
+    K = orc.k_from_ratio(128, 0.1)
+    bad = np.arange(K, dtype=np.int32)[None].copy()
+    bad[0, 3] = 100000
+    da = dev_i32(bad)
+    k_new, v_new, y = run_split_calls(dc, da, K)
+    dc.ctx.scatter_kv(dc.req, dc.kv(), da, K, k_new, v_new)
+    torch.cuda.synchronize()
+    assert dc.ctx.poll_status() & ab.FLAG_BAD_INDEX
+    assert dc.ctx.poll_status() == 0                                   # cleared by the poll
+    ckb = ab.to_host_bits(dc.ck)
+    keep = np.setdiff1d(np.arange(lay.ctx_len), np.delete(bad[0], 3))
+    assert np.array_equal(ckb[0][keep], case.cache_k[0][keep])
+
+
+def test_host_buffer_entry_point():
+    lay = wl.make_layout(2, 0, 128, 32, 32, 32, "masked")
+    case = make_projected_case(wl.TINY, lay, 0.2, cfg_id=17)
+    dc = DeviceCase(case)
+    K, s_dev, a_dev, y_dev = run_layer_step(dc, 0.2, ab.F_SCORE | ab.F_SELECT)
+    n = K + lay.n_extra
+    dc.reset_cache()
+    xh = torch.from_numpy(case.x.view(np.int16)).view(torch.bfloat16).pin_memory()
+    sh = torch.zeros((2, 128), dtype=torch.float32).pin_memory()
+    ah = torch.zeros((2, K), dtype=torch.int32).pin_memory()
+    yh = torch.zeros((2, n, case.shape.hidden), dtype=torch.bfloat16).pin_memory()
+    dc.ctx.layer_step_host(dc.lw, dc.req, dc.kv(), xh, 0.2, 0, sh, ah, yh)
+    torch.cuda.synchronize()
+    assert np.array_equal(sh.numpy(), s_dev) and np.array_equal(ah.numpy(), a_dev[:, :K])
+    assert np.array_equal(ab.to_host_bits(yh), ab.to_host_bits(y_dev[:, :n]))
+
+
+def test_invalid_arguments_enqueue_nothing():
+    lay = wl.make_layout(1, 0, 128, 16, 32, 32, "none")
+    case = wl.make_case(wl.TINY, lay, 0.1, cfg_id=18)
+    dc = DeviceCase(case, max_rows=8)
+    before = dc.ctx.launch_count()
+    y = torch.zeros((1, 64, 256), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(ab.AcacheError) as e:      # K = 13 rows > max_rows = 8
+        dc.ctx.layer_step(dc.lw, dc.req, dc.kv(), dc.x, 0, 0.1, 0, None, dev_i32(np.arange(13)[None]), y)
+    assert e.value.status == ab.ERR_INVALID_ARG
+    with pytest.raises(ab.AcacheError):           # misaligned x
+        dc.ctx.layer_step(dc.lw, dc.req, dc.kv(), dc.x.data_ptr() + 2, 0, 0.05, 0, None, dev_i32(np.arange(7)[None]), y)
+    assert dc.ctx.launch_count() == before
+
+
+# ------------------------------------------------------------------ benchmark configuration 2, full size
+@pytest.mark.parametrize("extra", ["none", "all"])
+def test_llada_layer_full_size(extra):
+    """512-token affix + 256 request + 256 generation rows at LLaDA-8B layer shapes, ratio 20 %,
+    in the configuration the benchmark times (random stale cache)."""
+    lay = wl.config_layout(2, extra)
+    case = wl.make_case(wl.LLADA_8B, lay, 0.2, cfg_id=2)
+    dc = DeviceCase(case)
+    K, s_gpu, a_gpu, y = run_layer_step(dc, 0.2, ab.F_SCORE | ab.F_SELECT)
+    assert K == 103
+    n = K + lay.n_extra
+    free = oracle_step(case, 0, ratio=0.2)
+    err = np.abs(s_gpu[0] - free["scores64"]) / np.maximum(free["scores64"], free["scores64"].mean())
+    assert err.max() < 1e-3
+    ok, why = orc.anchor_set_ok(a_gpu[0, :K], K, 512, free["must"], free["may"])
+    assert ok, why
+    ref = free if np.array_equal(free["anchor_idx"], a_gpu[0, :K]) else oracle_step(case, 0, anchor_idx=a_gpu[0, :K])
+    rows = ref["rows"]
+    ckb, cvb = ab.to_host_bits(dc.ck), ab.to_host_bits(dc.cv)
+    keep = np.setdiff1d(np.arange(lay.ctx_len), rows)
+    assert np.array_equal(ckb[0][keep], case.cache_k[0][keep]) and np.array_equal(cvb[0][keep], case.cache_v[0][keep])
+    assert_close_bf16(ckb[0][rows], ref["k_new"], "K rows")
+    assert_close_bf16(cvb[0][rows], ref["v_new"], "V rows")
+    assert_close_bf16(ab.to_host_bits(y[0, :n]), ref["y"], "y")
+    assert dc.ctx.poll_status() == 0
