@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the affix-cache refresh path (one layer-step = anchor scoring, top-K
+selection, selective recomputation, KV scatter) on synthetic LLaDA-8B-shaped inputs.
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA path (C ABI)
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, timed as it stands
+
+Prints ONE JSON line.  ``value`` is affix tokens refreshed per second over all ranks
+(B*K anchors per layer-step / step time, max over ranks), timed with CUDA events on the
+launching stream with the inputs resident in HBM; ``e2e`` is the same through the
+host-buffer entry point with the per-step host<->device copies inside the timed region.
+With N > 1 every rank refreshes its own requests (the path shards by request; weights and
+the affix cache are replicated) and there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_26140_b200 import workloads as wl  # noqa: E402
+
+METRIC = "anchor_refresh_affix_tokens_per_s"
+UNIT = "affix tokens/s"
+RATIO = 0.2
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the gate/up GEMM at this
+# workload, from one ncu capture (summary under profiles/); None until captured.
+NCU_TRAFFIC_BYTES = {"gate_up": None}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), tflops=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops=1400.0, source="fallback")
+
+
+def step_work(shape: wl.LayerShape, lay: wl.Layout, K: int):
+    """Algorithmic bytes and flops of one layer-step (per rank)."""
+    B, T, L, m = lay.batch, lay.ctx_len, lay.affix_len, lay.n_masked
+    D, H, Hkv, d, Fm = shape.hidden, shape.n_heads, shape.n_kv_heads, shape.head_dim, shape.ffn
+    n_r = B * (K + lay.n_extra)
+    n_m = B * m
+    w_bytes = shape.weight_bytes() + 2 * D * 2
+    by = dict(
+        weights=w_bytes,
+        score_k=B * L * Hkv * d * 2,
+        x_rows=(n_r + n_m) * D * 2,
+        attn_kv=B * T * 2 * Hkv * d * 2,
+        scatter=n_r * 2 * Hkv * d * 2,
+        y=n_r * D * 2,
+        scores=B * L * 4 + B * K * 4,
+    )
+    params = D * H * d + 2 * D * Hkv * d + H * d * D + 3 * D * Fm
+    fl = dict(
+        proj=2 * n_r * params + 2 * n_m * D * H * d,
+        score=2 * 2 * n_m * L * H * d,           # logits evaluated twice (statistics + column sums)
+        attn=4 * n_r * T * H * d,
+    )
+    gate_up_bytes = 2 * Fm * D * 2 + n_r * D * 2 + n_r * Fm * 2
+    gate_up_flops = 2 * n_r * D * 2 * Fm
+    return sum(by.values()), sum(fl.values()), gate_up_bytes, gate_up_flops, n_r
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while running."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.sm, self.reasons, self.max_mhz = index, False, [], set(), None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+        while not self.stop_flag:
+            try:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+def build_case(cfg: int, extra: str, batch):
+    shape = {1: wl.TINY, 2: wl.LLADA_8B, 3: wl.LLADA_8B, 4: wl.DREAM_7B}[cfg]
+    lay = wl.config_layout(cfg, extra, n_masked=32, batch=batch)
+    return shape, lay, wl.make_case(shape, lay, RATIO, cfg_id=cfg)
+
+
+# ------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The CPU oracle, unmodified, on the same workload; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import acache_oracle as orc
+    shape, lay, case = build_case(args.config, args.extra, args.batch)
+    L = lay.affix_len
+    K_full = orc.k_from_ratio(L, RATIO)
+    w64 = {k: (orc.bf16_bits_to_f64(v) if v is not None else None) for k, v in case.weights.items()}
+
+    def one_step(K):
+        for b in range(lay.batch):
+            orc.layer_step(w64, shape, case.x[b], case.cache_k[b], case.cache_v[b], lay.ctx_len, lay.affix_start, L,
+                           lay.masked_pos[b], lay.extra_rows[b], case.rope_cos, case.rope_sin, K=K)
+
+    t0 = time.perf_counter()
+    one_step(K_full)                         # calibration (untimed)
+    t_full = time.perf_counter() - t0
+    total = args.steps + args.warmup
+    K = K_full
+    if t_full * total > 150.0:               # bound the run: refresh fewer anchors per step
+        K = max(4, int(K_full * 150.0 / (t_full * total)))
+    for _ in range(args.warmup):
+        one_step(K)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_step(K)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = lay.batch * K / dt
+    cores = _threads_used()
+    sample = f"{K} of {K_full} anchors per request per step (scoring over all {L} affix keys), {lay.batch} request(s)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(shape, lay, args, K),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def _threads_used():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def workload_config(shape, lay, args, K):
+    return {"workload": f"{lay.name}: {shape.name} layer (hidden {shape.hidden}, {shape.n_heads}x{shape.head_dim} heads, "
+                        f"{shape.n_kv_heads} KV heads, MLP {shape.ffn}), batch {lay.batch}/GPU, affix {lay.affix_len} at "
+                        f"{lay.affix_start}, context {lay.ctx_len}, {lay.n_masked} masked rows, ratio {RATIO} (K={K}), "
+                        f"extra rows {lay.n_extra}",
+            "benchmark_config": args.config, "ratio": RATIO, "anchors_per_request": K, "rows_per_request": K + lay.n_extra,
+            "l2": f"per-step weights ({shape.weight_bytes() / 1e6:.0f} MB) exceed L2; {args.instances} weight/cache "
+                  "instances rotated", "parallelism": f"request-sharded x{args.gpus}"}
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    from paper_2608_26140_b200 import binding as ab
+    from paper_2608_26140_b200 import build as abuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        abuild.build()
+    if dist:
+        dist.barrier()
+
+    shape, lay, case = build_case(args.config, args.extra, args.batch)
+    B, T, L = lay.batch, lay.ctx_len, lay.affix_len
+    K = ab.k_from_ratio(L, RATIO)
+    n = K + lay.n_extra
+    inst = []
+    for _ in range(args.instances):
+        w = {k: (ab.to_device_bf16(v, dev) if v is not None else None) for k, v in case.weights.items()}
+        inst.append(dict(w=w, lw=ab.Context.weights(w), x=ab.to_device_bf16(case.x, dev),
+                         ck=ab.to_device_bf16(case.cache_k, dev), cv=ab.to_device_bf16(case.cache_v, dev)))
+    cos, sin = torch.from_numpy(case.rope_cos).to(dev), torch.from_numpy(case.rope_sin).to(dev)
+    masked = torch.from_numpy(lay.masked_pos.copy()).to(dev)
+    extra = torch.from_numpy(lay.extra_rows.copy()).to(dev) if lay.n_extra else None
+    req = ab.Context.request(B, T, lay.affix_start, L, masked, extra, cos, sin)
+    ctx = ab.Context.for_shape(shape, B, T, L, max(n, 1), max(lay.n_masked, 1), dev)
+    scores = torch.zeros((B, L), dtype=torch.float32, device=dev)
+    anchors = torch.zeros((B, max(K, 1)), dtype=torch.int32, device=dev)
+    y = torch.zeros((B, max(n, 1), shape.hidden), dtype=torch.bfloat16, device=dev)
+    flags = ab.F_SCORE | ab.F_SELECT
+
+    def step(i):
+        it = inst[i % len(inst)]
+        ctx.layer_step(it["lw"], req, ab.Context.kv(it["ck"], it["cv"]), it["x"], 0, RATIO, flags, scores, anchors, y)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if not dist:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    sync_all()
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    sync_all()
+    launches = ctx.launch_count() - l0
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_step = ms_total / args.steps
+
+    # second timed pass over the same steps with an event before every stage
+    ctx.stage_timing(True)
+    stage = {s: 0.0 for s in ab.STAGES}
+    for i in range(args.steps):
+        step(i)
+        for s, v in ctx.read_stage_times().items():
+            stage[s] += v / args.steps
+    ctx.stage_timing(False)
+    sampler.stop_flag = True
+    sampler.join()
+    assert ctx.poll_status() == 0, "device status word set during the benchmark"
+
+    # end to end: per-step inputs in pinned host memory, results read back to the host
+    xh = torch.from_numpy(case.x.view(np.int16)).view(torch.bfloat16).pin_memory()
+    sh = torch.zeros((B, L), dtype=torch.float32).pin_memory()
+    ah = torch.zeros((B, max(K, 1)), dtype=torch.int32).pin_memory()
+    yh = torch.zeros((B, max(n, 1), shape.hidden), dtype=torch.bfloat16).pin_memory()
+
+    def step_host(i):
+        it = inst[i % len(inst)]
+        ctx.layer_step_host(it["lw"], req, ab.Context.kv(it["ck"], it["cv"]), xh, RATIO, 0, sh, ah, yh)
+
+    for i in range(3):
+        step_host(i)
+    sync_all()
+    e0.record()
+    for i in range(args.steps):
+        step_host(i)
+    e1.record()
+    sync_all()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    h2d = xh.numel() * 2
+    d2h = n * B * shape.hidden * 2 + B * K * 4 + B * L * 4
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    step_bytes, step_flops, gu_bytes, gu_flops, n_r = step_work(shape, lay, K)
+    t_hbm = step_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_tc = step_flops / (peaks["tflops"] * 1e12)
+    gu_s = stage["gate_up"] * 1e-3
+    gu_hbm_bound = gu_bytes / (peaks["hbm_gbs"] * 1e9) >= gu_flops / (peaks["tflops"] * 1e12)
+    if gu_hbm_bound:
+        ach, peak, unit = gu_bytes / gu_s / 1e9, peaks["hbm_gbs"], "GB/s"
+    else:
+        ach, peak, unit = gu_flops / gu_s / 1e12, peaks["tflops"], "TFLOP/s"
+    roofline = {"kernel": "gate/up projection + SwiGLU (stage gate_up)", "bound": "hbm" if gu_hbm_bound else "tensor",
+                "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "peak_source": peaks["source"],
+                "traffic": NCU_TRAFFIC_BYTES["gate_up"], "algorithmic_bytes": gu_bytes, "algorithmic_flops": gu_flops,
+                "us_per_launch": stage["gate_up"] * 1e3}
+    floor_s = max(t_hbm, t_tc)
+    value = world * B * K / (ms_step * 1e-3)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_step, "us_per_layer_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(shape, lay, args, K),
+        "clocks": sampler.summary(),
+        "e2e": {"value": world * B * K / (ms_e2e * 1e-3), "unit": UNIT, "us_per_layer_step": ms_e2e * 1e3,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "layer_step_roofline": {"bound": "hbm" if t_hbm >= t_tc else "tensor", "algorithmic_bytes": step_bytes,
+                                "algorithmic_flops": step_flops, "floor_us": floor_s * 1e6,
+                                "frac": floor_s / (ms_step * 1e-3), "peak_source": peaks["source"]},
+        "stage_us": {s: v * 1e3 for s, v in stage.items()},
+        "affix_tokens_covered_per_s": world * B * L / (ms_step * 1e-3),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(case, shape, lay)
+    print(json.dumps(out))
+    if dist:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(case, shape, lay):
+    """The oracle as it stands, timed on this machine's host cores on one step of the workload."""
+    from oracle import acache_oracle as orc
+    L = lay.affix_len
+    K = orc.k_from_ratio(L, RATIO)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        for b in range(lay.batch):
+            orc.layer_step(case.weights, shape, case.x[b], case.cache_k[b], case.cache_v[b], lay.ctx_len,
+                           lay.affix_start, L, lay.masked_pos[b], lay.extra_rows[b], case.rope_cos, case.rope_sin,
+                           ratio=RATIO)
+        reps += 1
+        if time.perf_counter() - t0 > 10.0 or reps >= 3:
+            break
+    dt = (time.perf_counter() - t0) / reps
+    return {"value": lay.batch * K / dt, "unit": UNIT, "cores": _threads_used(), "kind": "oracle",
+            "sample": f"{reps} full layer-step(s) of the same workload ({lay.batch} request(s), {K} anchors each), "
+                      f"{dt:.2f} s per step including the oracle's own bf16->fp64 weight conversion"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="benchmark configuration (2 = LLaDA-8B layer, batch 1)")
+    ap.add_argument("--extra", default="none", choices=["none", "all", "masked"],
+                    help="request-specific rows recomputed with the anchors")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--instances", type=int, default=4, help="weight/cache instances rotated between steps")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -133,6 +133,31 @@ acache_status acache_poll_status(acache_ctx *ctx, acache_stream_t stream, uint32
 /* Number of kernels this context has launched since creation (for accounting). */
 uint64_t acache_launch_count(const acache_ctx *ctx);
 
+/* Measurement aid (the paper has no counterpart).  The stages of acache_layer_step, in
+ * launch order; a stage's time runs from its first launch to the next stage's. */
+enum {
+    ACACHE_STAGE_MASK_Q = 0,    /* RMSNorm + Q projection + RoPE of the masked rows  */
+    ACACHE_STAGE_SCORE,         /* Eq. 4-5                                            */
+    ACACHE_STAGE_TOPK,          /* Eq. 6                                              */
+    ACACHE_STAGE_GATHER_NORM,   /* row plan of R, gather, RMSNorm                     */
+    ACACHE_STAGE_QKV,           /* QKV projection + RoPE + KV scatter                 */
+    ACACHE_STAGE_ATTENTION,     /* attention of R over the whole context              */
+    ACACHE_STAGE_OPROJ,         /* output projection + residual                       */
+    ACACHE_STAGE_MLP_NORM,      /* second RMSNorm                                     */
+    ACACHE_STAGE_GATE_UP,       /* gate/up projection + SwiGLU                        */
+    ACACHE_STAGE_DOWN,          /* down projection + residual                         */
+    ACACHE_N_STAGES
+};
+
+/* enable != 0: every following acache_layer_step records a CUDA event on its stream
+ * before each stage (the first call creates the events; they serialise the stages, so a
+ * timed step is slightly slower than an untimed one).  enable == 0 switches it off. */
+acache_status acache_stage_timing(acache_ctx *ctx, int enable);
+
+/* Waits for the last timed acache_layer_step and writes the milliseconds each stage took
+ * to ms[ACACHE_N_STAGES] (HOST); stages that did not run read 0. */
+acache_status acache_read_stage_times(acache_ctx *ctx, float *ms);
+
 /* ---- the path ------------------------------------------------------------------------ */
 
 /* Eq. 4-5 (Section 3.2), one layer's term:

@@ -21,7 +21,9 @@ F_SCORE, F_SELECT, F_ACCUMULATE, F_SCORE_NORM_FULL, F_NO_RECOMPUTE = 0x1, 0x2, 0
 EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "acache_destroy",
            "acache_last_error", "acache_poll_status", "acache_launch_count", "acache_score_anchors",
            "acache_k_from_ratio", "acache_select_topk", "acache_recompute_anchors", "acache_scatter_kv",
-           "acache_layer_step", "acache_layer_step_host"]
+           "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times"]
+
+STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
 
 class ModelDesc(C.Structure):
@@ -98,6 +100,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_layer_step_host.argtypes = [vp, C.POINTER(LayerWeights), C.POINTER(Request), C.POINTER(KV), vp,
                                            C.c_double, u32, vp, vp, vp, vp]
     lib.acache_layer_step_host.restype = C.c_int
+    lib.acache_stage_timing.argtypes = [vp, C.c_int]
+    lib.acache_stage_timing.restype = C.c_int
+    lib.acache_read_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
+    lib.acache_read_stage_times.restype = C.c_int
     if path is None:
         _lib = lib
     return lib
@@ -194,6 +200,15 @@ class Context:
         if st not in (OK, ERR_TIMEOUT):
             self._check(st)
         return int(flags.value)
+
+    def stage_timing(self, enable: bool):
+        self._check(self.lib.acache_stage_timing(self.h, int(enable)))
+
+    def read_stage_times(self) -> Dict[str, float]:
+        """Milliseconds per stage of the last timed layer-step (synchronises)."""
+        ms = (C.c_float * len(STAGES))()
+        self._check(self.lib.acache_read_stage_times(self.h, ms))
+        return {n: float(ms[i]) for i, n in enumerate(STAGES)}
 
     def score_anchors(self, req: Request, q_mask, kv: KV, scores, accumulate=False, norm_full=False):
         self._check(self.lib.acache_score_anchors(self.h, C.byref(req), _ptr(q_mask), C.byref(kv), _ptr(scores),

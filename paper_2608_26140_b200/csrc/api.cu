@@ -24,6 +24,10 @@ struct acache_ctx {
     size_t o_xstage, o_ystage, o_sstage, o_astage;
     std::string err;
     uint64_t launches = 0;
+    // optional per-stage timing (acache_stage_timing)
+    bool timing = false;
+    cudaEvent_t ev[ACACHE_N_STAGES + 1] = {};
+    bool ev_hit[ACACHE_N_STAGES + 1] = {};
 };
 
 namespace {
@@ -50,6 +54,13 @@ size_t take(size_t& cur, size_t bytes) {
 
 template <class T>
 T* wsp(acache_ctx* c, size_t off) { return reinterpret_cast<T*>(c->ws + off); }
+
+// Marks the start of stage `i` (and the end of the stages before it) on the stream.
+void mark(acache_ctx* c, int i, cudaStream_t st) {
+    if (!c->timing) return;
+    cudaEventRecord(c->ev[i], st);
+    c->ev_hit[i] = true;
+}
 
 acache_status check_cuda(acache_ctx* c, const char* what) {
     cudaError_t e = cudaGetLastError();
@@ -122,7 +133,10 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
                             const int32_t* anchor_idx, int k, void* k_new, void* v_new, void* y, cudaStream_t st) {
     const acache_model_desc& d = c->d;
     const int rows = k + r->n_extra, n = r->batch * rows;
-    if (n == 0) return ACACHE_OK;
+    if (n == 0) {
+        mark(c, ACACHE_N_STAGES, st);
+        return ACACHE_OK;
+    }
     const int qd = d.n_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim;
     int32_t* row_pos = wsp<int32_t>(c, c->o_row_pos);
     int64_t* row_src = wsp<int64_t>(c, c->o_row_src);
@@ -134,10 +148,12 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     void* act = wsp<void>(c, c->o_act);
     uint32_t* status = wsp<uint32_t>(c, c->o_status);
 
+    mark(c, ACACHE_STAGE_GATHER_NORM, st);
     launch_gather_rmsnorm(x, x_is_compact, (int64_t)r->ctx_len * d.hidden, d.hidden, anchor_idx, k, r->extra_rows,
                           r->n_extra, r->batch, r->affix_start, r->affix_len, r->ctx_len, w->attn_norm_g, d.rms_eps,
                           row_pos, row_src, xn, status, st);
     c->launches += 1;
+    mark(c, ACACHE_STAGE_QKV, st);
 
     GemmArgs g{};
     g.a = xn; g.M = n; g.K = d.hidden;
@@ -154,6 +170,7 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     g.kv_batch_stride = kv->batch_stride; g.rows_per_req = rows;
     c->launches += launch_gemm(g, st);
 
+    mark(c, ACACHE_STAGE_ATTENTION, st);
     AttnArgs at{};
     at.q = q; at.cache_k = kv->k; at.cache_v = kv->v; at.kv_batch_stride = kv->batch_stride;
     if (!fuse_scatter) {
@@ -167,23 +184,28 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     at.o = o;
     c->launches += launch_attention(at, st);
 
+    mark(c, ACACHE_STAGE_OPROJ, st);
     GemmArgs go{};
     go.a = o; go.M = n; go.K = qd; go.b[0] = w->wo; go.n[0] = d.hidden;
     go.epilogue = kEpiResidual; go.resid = x; go.resid_off = row_src; go.c = h1;
     c->launches += launch_gemm(go, st);
 
+    mark(c, ACACHE_STAGE_MLP_NORM, st);
     launch_rmsnorm(h1, w->mlp_norm_g, d.rms_eps, n, d.hidden, xn2, st);
     c->launches += 1;
+    mark(c, ACACHE_STAGE_GATE_UP, st);
 
     GemmArgs gu{};
     gu.a = xn2; gu.M = n; gu.K = d.hidden; gu.b[0] = w->w_gate; gu.b[1] = w->w_up; gu.n[0] = d.ffn; gu.n[1] = d.ffn;
     gu.epilogue = kEpiSwiGLU; gu.c = act;
     c->launches += launch_gemm(gu, st);
 
+    mark(c, ACACHE_STAGE_DOWN, st);
     GemmArgs gd{};
     gd.a = act; gd.M = n; gd.K = d.ffn; gd.b[0] = w->w_down; gd.n[0] = d.hidden;
     gd.epilogue = kEpiResidual; gd.resid = h1; gd.resid_off = nullptr; gd.c = y;
     c->launches += launch_gemm(gd, st);
+    mark(c, ACACHE_N_STAGES, st);
     return check_cuda(c, "recompute");
 }
 
@@ -246,7 +268,37 @@ acache_status acache_set_workspace(acache_ctx* ctx, void* dev_ptr, size_t bytes,
     return ACACHE_OK;
 }
 
-void acache_destroy(acache_ctx* ctx) { delete ctx; }
+void acache_destroy(acache_ctx* ctx) {
+    if (!ctx) return;
+    for (cudaEvent_t e : ctx->ev)
+        if (e) cudaEventDestroy(e);
+    delete ctx;
+}
+
+acache_status acache_stage_timing(acache_ctx* ctx, int enable) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (enable && !ctx->ev[0]) {
+        for (cudaEvent_t& e : ctx->ev)
+            if (cudaEventCreate(&e) != cudaSuccess) return check_cuda(ctx, "cudaEventCreate");
+    }
+    ctx->timing = enable != 0;
+    for (bool& h : ctx->ev_hit) h = false;
+    return ACACHE_OK;
+}
+
+acache_status acache_read_stage_times(acache_ctx* ctx, float* ms) {
+    if (!ctx || !ms) return ACACHE_ERR_INVALID_ARG;
+    if (!ctx->timing || !ctx->ev_hit[ACACHE_N_STAGES]) return fail(ctx, ACACHE_ERR_INVALID_ARG, "no timed layer-step to read");
+    if (cudaEventSynchronize(ctx->ev[ACACHE_N_STAGES]) != cudaSuccess) return check_cuda(ctx, "cudaEventSynchronize");
+    for (int i = 0; i < ACACHE_N_STAGES; ++i) {
+        ms[i] = 0.f;
+        if (!ctx->ev_hit[i]) continue;
+        int j = i + 1;
+        while (!ctx->ev_hit[j]) ++j;          // the next stage that ran (the end mark always did)
+        if (cudaEventElapsedTime(&ms[i], ctx->ev[i], ctx->ev[j]) != cudaSuccess) return check_cuda(ctx, "cudaEventElapsedTime");
+    }
+    return ACACHE_OK;
+}
 
 const char* acache_last_error(const acache_ctx* ctx) { return ctx ? ctx->err.c_str() : "context is NULL"; }
 
@@ -346,8 +398,10 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
     if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
     if (do_recompute && req->batch * (k + req->n_extra) > 0 && (!y || !aligned16(y))) return fail(ctx, ACACHE_ERR_INVALID_ARG, "y NULL or misaligned");
 
+    if (ctx->timing) for (bool& h : ctx->ev_hit) h = false;
     if (do_score && req->batch > 0 && req->affix_len > 0) {
         void* qmask = wsp<void>(ctx, ctx->o_qmask);
+        mark(ctx, ACACHE_STAGE_MASK_Q, stream);
         if (req->n_masked > 0) {
             int32_t* mpos = wsp<int32_t>(ctx, ctx->o_mrow_pos);
             void* xnm = wsp<void>(ctx, ctx->o_xn_mask);
@@ -365,16 +419,19 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
             g.head_dim = d.head_dim; g.rope_segments = 1; g.out[0] = qmask; g.rows_per_req = req->n_masked;
             ctx->launches += launch_gemm(g, stream);
         }
+        mark(ctx, ACACHE_STAGE_SCORE, stream);
         s = run_score(ctx, req, qmask, kv, scores, (flags & ACACHE_F_ACCUMULATE) ? 1 : 0,
                       (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, stream);
         if (s != ACACHE_OK) return s;
     }
     if (do_select && k > 0 && req->batch > 0) {
+        mark(ctx, ACACHE_STAGE_TOPK, stream);
         launch_topk(scores, req->batch, req->affix_len, k, anchor_idx, stream);
         ctx->launches += 1;
     }
     if (do_recompute)
         return run_recompute(ctx, w, req, kv, true, x, x_is_compact, anchor_idx, k, nullptr, nullptr, y, stream);
+    mark(ctx, ACACHE_N_STAGES, stream);
     return check_cuda(ctx, "layer_step");
 }
 
