@@ -1,6 +1,7 @@
 // C-ABI entry points (see include/acache.h): argument validation, workspace layout and the
 // kernel sequences of the affix-cache refresh path.  Everything is enqueued on the caller's
 // stream; nothing here allocates device memory or synchronises (except acache_poll_status).
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -21,7 +22,7 @@ struct acache_ctx {
     // workspace offsets (bytes)
     size_t o_status, o_row_pos, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
     size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
-    size_t o_xstage, o_ystage, o_sstage, o_astage;
+    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm;
     std::string err;
     uint64_t launches = 0;
     // optional per-stage timing (acache_stage_timing)
@@ -168,6 +169,7 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     g.out[0] = q; g.out[1] = k_new; g.out[2] = v_new;
     if (fuse_scatter) { g.cache_k = kv->k; g.cache_v = kv->v; }
     g.kv_batch_stride = kv->batch_stride; g.rows_per_req = rows;
+    g.partial = wsp<float>(c, c->o_gemm); g.status = status;
     c->launches += launch_gemm(g, st);
 
     mark(c, ACACHE_STAGE_ATTENTION, st);
@@ -188,6 +190,7 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     GemmArgs go{};
     go.a = o; go.M = n; go.K = qd; go.b[0] = w->wo; go.n[0] = d.hidden;
     go.epilogue = kEpiResidual; go.resid = x; go.resid_off = row_src; go.c = h1;
+    go.partial = wsp<float>(c, c->o_gemm); go.status = status;
     c->launches += launch_gemm(go, st);
 
     mark(c, ACACHE_STAGE_MLP_NORM, st);
@@ -198,12 +201,14 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     GemmArgs gu{};
     gu.a = xn2; gu.M = n; gu.K = d.hidden; gu.b[0] = w->w_gate; gu.b[1] = w->w_up; gu.n[0] = d.ffn; gu.n[1] = d.ffn;
     gu.epilogue = kEpiSwiGLU; gu.c = act;
+    gu.partial = wsp<float>(c, c->o_gemm); gu.status = status;
     c->launches += launch_gemm(gu, st);
 
     mark(c, ACACHE_STAGE_DOWN, st);
     GemmArgs gd{};
     gd.a = act; gd.M = n; gd.K = d.ffn; gd.b[0] = w->w_down; gd.n[0] = d.hidden;
     gd.epilogue = kEpiResidual; gd.resid = h1; gd.resid_off = nullptr; gd.c = y;
+    gd.partial = wsp<float>(c, c->o_gemm); gd.status = status;
     c->launches += launch_gemm(gd, st);
     mark(c, ACACHE_N_STAGES, st);
     return check_cuda(c, "recompute");
@@ -251,6 +256,15 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
     c->o_ystage = take(cur, nr * d.hidden * 2);
     c->o_sstage = take(cur, (size_t)d.max_batch * d.max_affix * 4);
     c->o_astage = take(cur, (size_t)d.max_batch * d.max_affix * 4);
+    {
+        const int nri = (int)nr, nmi = (int)nm;
+        size_t pb = gemm_partial_bytes(nri, d.hidden, qd + 2 * kvd, false);
+        pb = std::max(pb, gemm_partial_bytes(nri, qd, d.hidden, false));
+        pb = std::max(pb, gemm_partial_bytes(nri, d.hidden, d.ffn, true));
+        pb = std::max(pb, gemm_partial_bytes(nri, d.ffn, d.hidden, false));
+        pb = std::max(pb, gemm_partial_bytes(nmi, d.hidden, qd, false));
+        c->o_gemm = take(cur, pb);
+    }
     c->ws_need = cur;
     *out = c;
     return ACACHE_OK;
@@ -417,6 +431,7 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
             g.bias[0] = d.qkv_bias ? w->bq : nullptr;
             g.row_pos = mpos; g.rope_cos = req->rope_cos; g.rope_sin = req->rope_sin;
             g.head_dim = d.head_dim; g.rope_segments = 1; g.out[0] = qmask; g.rows_per_req = req->n_masked;
+            g.partial = wsp<float>(ctx, ctx->o_gemm); g.status = wsp<uint32_t>(ctx, ctx->o_status);
             ctx->launches += launch_gemm(g, stream);
         }
         mark(ctx, ACACHE_STAGE_SCORE, stream);

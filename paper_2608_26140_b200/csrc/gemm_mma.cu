@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_mma_kernel(const GemmArgs g
     else epilogue_swiglu(g, stage, m0, nt * 64, g.n[0], tid, GEMM_THREADS);
 }
 
-int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
+int launch_gemm_mma(const GemmArgs& g, cudaStream_t stream) {
     if (g.M == 0) return 0;
     int ntiles;
     if (g.epilogue == kEpiSwiGLU) ntiles = g.n[0] / 64;

@@ -82,8 +82,15 @@ struct GemmArgs {
     const int64_t* resid_off; // [M] element offset of the residual row, or null => row * N
     // --- kEpiSwiGLU / kEpiResidual output ---
     void* c;                  // bf16 [M, Nout]
+    // --- scratch ---
+    float* partial;           // fp32 partial tiles, gemm_partial_bytes() of them
+    uint32_t* status;         // device status word
 };
-int launch_gemm(const GemmArgs& g, cudaStream_t stream);
+// Bytes of fp32 partial-tile scratch a GEMM of M rows, reduction length K and n_total output
+// columns (SwiGLU: the MLP width) needs.
+size_t gemm_partial_bytes(int M, int K, int n_total, bool swiglu);
+int launch_gemm(const GemmArgs& g, cudaStream_t stream);      // tcgen05 main loop + finish kernel
+int launch_gemm_mma(const GemmArgs& g, cudaStream_t stream);  // legacy mma.sync main loop (debug aid)
 
 // ---- attn.cu ----------------------------------------------------------------------------
 struct AttnArgs {
