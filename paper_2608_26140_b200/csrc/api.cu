@@ -22,7 +22,7 @@ struct acache_ctx {
     // workspace offsets (bytes)
     size_t o_status, o_row_pos, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
     size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
-    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm;
+    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn;
     std::string err;
     uint64_t launches = 0;
     // optional per-stage timing (acache_stage_timing)
@@ -184,6 +184,8 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     at.batch = r->batch; at.n = rows; at.ctx_len = r->ctx_len;
     at.n_heads = d.n_heads; at.n_kv_heads = d.n_kv_heads; at.head_dim = d.head_dim;
     at.o = o;
+    at.part_o = wsp<float>(c, c->o_attn);
+    at.part_ml = at.part_o + (size_t)2 * 296 * 64 * d.head_dim;
     c->launches += launch_attention(at, st);
 
     mark(c, ACACHE_STAGE_OPROJ, st);
@@ -265,6 +267,7 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
         pb = std::max(pb, gemm_partial_bytes(nmi, d.hidden, qd, false));
         c->o_gemm = take(cur, pb);
     }
+    c->o_attn = take(cur, attention_scratch_bytes(d.head_dim));
     c->ws_need = cur;
     *out = c;
     return ACACHE_OK;

@@ -9,11 +9,7 @@
 
 namespace acache {
 
-template <int D>
-struct AttnTile {
-    static constexpr int BYTES = 64 * D * 2;
-    static constexpr int CPR = D / 8;
-};
+constexpr int kAttnTargetCtas = 296;   // two CTAs per SM on 148 SMs
 
 template <int D>
 __device__ __forceinline__ void load_q_tile(uint32_t sdst, const __nv_bfloat16* q, int64_t stride, int valid, int tid) {
@@ -53,24 +49,34 @@ __device__ __forceinline__ void load_kv_tile(uint32_t sk, uint32_t sv, const Att
     }
 }
 
+constexpr int ATT_STAGES = 3;
+
+// One CTA: 64 query rows of one head against the key tiles [tile_lo, tile_hi) of its split.
+// With one split the normalised output is written directly; otherwise the unnormalised fp32
+// accumulator and the row statistics go to scratch and attention_combine_kernel merges them.
 template <int D>
-__global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float scale_log2e) {
+__global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float scale_log2e, int n_split,
+                                                        int tiles_per_split) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int TILE = 64 * D * 2;
     const uint32_t sQ = smem_u32(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int qt = blockIdx.x / n_split, split = blockIdx.x % n_split, h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / (a.n_heads / a.n_kv_heads);
     const int64_t qstride = (int64_t)a.n_heads * D;
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.q) + ((int64_t)b * a.n + qt * 64) * qstride + h * D;
-    const int ntiles = (a.ctx_len + 63) / 64;
+    const int all_tiles = (a.ctx_len + 63) / 64;
+    const int tile_lo = split * tiles_per_split;
+    const int ntiles = min(all_tiles, tile_lo + tiles_per_split) - tile_lo;
     auto sK = [&](int buf) { return sQ + TILE + buf * 2 * TILE; };
     auto sV = [&](int buf) { return sQ + 2 * TILE + buf * 2 * TILE; };
 
     load_q_tile<D>(sQ, q, qstride, min(64, a.n - qt * 64), tid);
-    load_kv_tile<D>(sK(0), sV(0), a, b, kvh, 0, tid);
+    load_kv_tile<D>(sK(0), sV(0), a, b, kvh, tile_lo * 64, tid);
     cp_async_commit();
-    cp_async_wait<0>();
+    if (ntiles > 1) load_kv_tile<D>(sK(1), sV(1), a, b, kvh, (tile_lo + 1) * 64, tid);
+    cp_async_commit();
+    cp_async_wait<1>();
     __syncthreads();
 
     uint32_t qf[D / 16][4];
@@ -86,14 +92,14 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
     for (int i = 0; i < D / 8; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
-    float mx[2] = {-INFINITY, -INFINITY}, den[2] = {0.f, 0.f}, den_bf[2] = {0.f, 0.f};
+    float mx[2] = {-INFINITY, -INFINITY}, den[2] = {0.f, 0.f};
 
     for (int t = 0; t < ntiles; ++t) {
-        if (t + 1 < ntiles) {
-            load_kv_tile<D>(sK((t + 1) & 1), sV((t + 1) & 1), a, b, kvh, (t + 1) * 64, tid);
-            cp_async_commit();
-        }
-        const uint32_t sk = sK(t & 1), sv = sV(t & 1);
+        // tile t is resident (waited for below); prefetch tile t + 2 into the buffer tile t - 1 used
+        if (t + 2 < ntiles) load_kv_tile<D>(sK((t + 2) % ATT_STAGES), sV((t + 2) % ATT_STAGES), a, b, kvh,
+                                            (tile_lo + t + 2) * 64, tid);
+        cp_async_commit();
+        const uint32_t sk = sK(t % ATT_STAGES), sv = sV(t % ATT_STAGES);
         float s[8][4];
 #pragma unroll
         for (int nb = 0; nb < 8; ++nb)
@@ -111,7 +117,7 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
                 mma_bf16_16816(s[np * 2 + 1], qf[ks], b2, b3);
             }
         }
-        const int valid = a.ctx_len - t * 64;
+        const int valid = a.ctx_len - (tile_lo + t) * 64;
         float tmax[2] = {-INFINITY, -INFINITY};
 #pragma unroll
         for (int nb = 0; nb < 8; ++nb)
@@ -131,7 +137,6 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
             corr[r] = exp2f(mx[r] - nm);
             mx[r] = nm;
             den[r] *= corr[r];
-            den_bf[r] *= corr[r];
         }
 #pragma unroll
         for (int i = 0; i < D / 8; ++i) {
@@ -145,11 +150,8 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
             float p2 = exp2f(s[nb][2] - mx[1]), p3 = exp2f(s[nb][3] - mx[1]);
             den[0] += p0 + p1;
             den[1] += p2 + p3;
-            uint32_t u01 = pack_bf16(p0, p1), u23 = pack_bf16(p2, p3);
-            den_bf[0] += bf16_lo(u01) + bf16_hi(u01);
-            den_bf[1] += bf16_lo(u23) + bf16_hi(u23);
-            pf[nb >> 1][(nb & 1) * 2] = u01;
-            pf[nb >> 1][(nb & 1) * 2 + 1] = u23;
+            pf[nb >> 1][(nb & 1) * 2] = pack_bf16(p0, p1);
+            pf[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16(p2, p3);
         }
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
@@ -163,46 +165,102 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
                 mma_bf16_16816(o[np * 2 + 1], pf[kk], b2, b3);
             }
         }
-        if (t + 1 < ntiles) cp_async_wait<0>();
+        cp_async_wait<1>();     // everything but the newest group: tile t + 1 has landed
         __syncthreads();
     }
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         den[r] += __shfl_xor_sync(0xffffffffu, den[r], 1);
         den[r] += __shfl_xor_sync(0xffffffffu, den[r], 2);
-        den_bf[r] += __shfl_xor_sync(0xffffffffu, den_bf[r], 1);
-        den_bf[r] += __shfl_xor_sync(0xffffffffu, den_bf[r], 2);
     }
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o);
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         const int row = qt * 64 + warp * 16 + (lane >> 2) + r * 8;
         if (row >= a.n) continue;
-        const float inv = 1.f / den[r];
-        __nv_bfloat16* orow = out + ((int64_t)b * a.n + row) * qstride + h * D;
+        if (n_split == 1) {
+            const float inv = 1.f / den[r];
+            __nv_bfloat16* orow = out + ((int64_t)b * a.n + row) * qstride + h * D;
 #pragma unroll
-        for (int nb = 0; nb < D / 8; ++nb) {
-            int col = nb * 8 + (lane & 3) * 2;
-            *reinterpret_cast<uint32_t*>(orow + col) = pack_bf16(o[nb][r * 2] * inv, o[nb][r * 2 + 1] * inv);
+            for (int nb = 0; nb < D / 8; ++nb) {
+                int col = nb * 8 + (lane & 3) * 2;
+                *reinterpret_cast<uint32_t*>(orow + col) = pack_bf16(o[nb][r * 2] * inv, o[nb][r * 2 + 1] * inv);
+            }
+        } else {
+            const int64_t rh = ((int64_t)b * a.n + row) * a.n_heads + h;
+            float* po = a.part_o + (rh * n_split + split) * D;
+#pragma unroll
+            for (int nb = 0; nb < D / 8; ++nb) {
+                int col = nb * 8 + (lane & 3) * 2;
+                *reinterpret_cast<float2*>(po + col) = make_float2(o[nb][r * 2], o[nb][r * 2 + 1]);
+            }
+            if ((lane & 3) == 0) {
+                a.part_ml[(rh * n_split + split) * 2] = mx[r];
+                a.part_ml[(rh * n_split + split) * 2 + 1] = den[r];
+            }
         }
-        if (a.row_sum && (lane & 3) == 0) a.row_sum[((int64_t)b * a.n + row) * a.n_heads + h] = den_bf[r] * inv;
     }
+}
+
+// Merges the key splits of one (row, head): o = sum_s O_s 2^(m_s - m) / sum_s l_s 2^(m_s - m).
+template <int D>
+__global__ void __launch_bounds__(128) attention_combine_kernel(const AttnArgs a, int n_split, int64_t n_rh) {
+    const int lane = threadIdx.x & 31;
+    const int64_t rh = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (rh >= n_rh) return;
+    float m = -INFINITY;
+    for (int s = 0; s < n_split; ++s) m = fmaxf(m, a.part_ml[(rh * n_split + s) * 2]);
+    float l = 0.f;
+    float acc[D / 32];
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) acc[i] = 0.f;
+    for (int s = 0; s < n_split; ++s) {
+        const float w = exp2f(a.part_ml[(rh * n_split + s) * 2] - m);
+        l += a.part_ml[(rh * n_split + s) * 2 + 1] * w;
+        const float* po = a.part_o + (rh * n_split + s) * D;
+#pragma unroll
+        for (int i = 0; i < D / 32; ++i) acc[i] += po[i * 32 + lane] * w;
+    }
+    const float inv = 1.f / l;
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o) + rh * D;   // [B, n, H, d] is contiguous in (row, head)
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) out[i * 32 + lane] = __float2bfloat16_rn(acc[i] * inv);
+}
+
+// Key splits: enough CTAs to cover the machine about twice when there are few query tiles.
+static int attention_splits(int q_ctas, int key_tiles, int* tiles_per_split) {
+    int want = q_ctas >= kAttnTargetCtas ? 1 : (kAttnTargetCtas + q_ctas - 1) / q_ctas;
+    if (want > key_tiles) want = key_tiles;
+    if (want < 1) want = 1;
+    *tiles_per_split = (key_tiles + want - 1) / want;
+    return (key_tiles + *tiles_per_split - 1) / *tiles_per_split;
+}
+
+size_t attention_scratch_bytes(int head_dim) {
+    // splits are only used below kAttnTargetCtas query CTAs, and n_split * q_ctas < 2 * kAttnTargetCtas
+    return (size_t)2 * kAttnTargetCtas * 64 * (head_dim + 2) * sizeof(float);
 }
 
 int launch_attention(const AttnArgs& a, cudaStream_t stream) {
     if (a.batch == 0 || a.n == 0) return 0;
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)a.head_dim);
-    dim3 grid((a.n + 63) / 64, a.n_heads, a.batch);
+    const int q_tiles = (a.n + 63) / 64;
+    int tps;
+    const int n_split = attention_splits(q_tiles * a.n_heads * a.batch, (a.ctx_len + 63) / 64, &tps);
+    dim3 grid(q_tiles * n_split, a.n_heads, a.batch);
+    const int64_t n_rh = (int64_t)a.batch * a.n * a.n_heads;
     if (a.head_dim == 128) {
-        constexpr int SMEM = 5 * 64 * 128 * 2;
+        constexpr int SMEM = (1 + 2 * ATT_STAGES) * 64 * 128 * 2;
         cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-        attention_kernel<128><<<grid, 128, SMEM, stream>>>(a, scale_log2e);
+        attention_kernel<128><<<grid, 128, SMEM, stream>>>(a, scale_log2e, n_split, tps);
+        if (n_split > 1) attention_combine_kernel<128><<<(unsigned)((n_rh + 3) / 4), 128, 0, stream>>>(a, n_split, n_rh);
     } else {
-        constexpr int SMEM = 5 * 64 * 64 * 2;
+        constexpr int SMEM = (1 + 2 * ATT_STAGES) * 64 * 64 * 2;
         cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-        attention_kernel<64><<<grid, 128, SMEM, stream>>>(a, scale_log2e);
+        attention_kernel<64><<<grid, 128, SMEM, stream>>>(a, scale_log2e, n_split, tps);
+        if (n_split > 1) attention_combine_kernel<64><<<(unsigned)((n_rh + 3) / 4), 128, 0, stream>>>(a, n_split, n_rh);
     }
-    return 1;
+    return n_split > 1 ? 2 : 1;
 }
 
 }  // namespace acache

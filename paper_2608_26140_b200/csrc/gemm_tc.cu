@@ -289,38 +289,116 @@ gemm_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap mapA, const _
 }
 
 // ---- finish: ordered sum of the partial tiles + epilogue --------------------------------------
-__global__ void __launch_bounds__(256) gemm_finish_kernel(const GemmArgs g, const TcPlan p, const float* __restrict__ partial) {
-    extern __shared__ __align__(16) unsigned char fsm[];
-    float* stage = reinterpret_cast<float*>(fsm);
-    const int u = blockIdx.x, mt = blockIdx.y, m0 = mt * TC_BM;
-    const int nt = u >> 1, hh = u & 1;
-    const int t = mt * p.n_tiles + nt;
-    const int c_first = (int)(((int64_t)t * p.KB) / p.U);
-    const int c_last = (int)(((int64_t)(t + 1) * p.KB - 1) / p.U);
-    const float4* src = reinterpret_cast<const float4*>(partial + (int64_t)t * p.smax * TC_SLOT_FLOATS);
-    const int row = threadIdx.x & 127, grp = threadIdx.x >> 7;
-    const bool valid = m0 + row < g.M;
-    const bool swiglu = g.epilogue == kEpiSwiGLU;
-    for (int jc = grp; jc < 32; jc += 2) {
-        const int pc = swiglu ? (jc < 16 ? 16 * hh + jc : 32 + 16 * hh + (jc - 16)) : 32 * hh + jc;
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid) {
-            for (int c = c_first; c <= c_last; ++c) {
-                const float4 v = src[((int64_t)(c - c_first) * (TC_SLOT_FLOATS / 4)) + pc * TC_BM + row];
-                s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+// One thread owns 4 adjacent output columns of one row (plus the 4 columns its epilogue pairs
+// them with: the other rotary half, or the up-projection of a gate column).  A warp covers 32
+// consecutive rows of the same columns, so every partial-tile read is one contiguous 512-byte
+// segment; the slots are summed in ascending CTA order, which makes the result bitwise
+// reproducible.
+constexpr int FIN_ITEMS_PER_SUB = 2;   // items each half-block of 128 threads walks through
+
+__device__ __forceinline__ float4 sum_slots(const float4* __restrict__ src, int nslots, int pc, int row) {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4* q = src + pc * TC_BM + row;
+#pragma unroll 4
+    for (int c = 0; c < nslots; ++c) {
+        const float4 v = __ldcg(q + (int64_t)c * (TC_SLOT_FLOATS / 4));
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    return s;
+}
+
+__device__ __forceinline__ uint2 pack4(float a, float b, float c, float d) {
+    return make_uint2(pack_bf16(a, b), pack_bf16(c, d));
+}
+
+__global__ void __launch_bounds__(256) gemm_finish_kernel(const GemmArgs g, const TcPlan p, const float* __restrict__ partial,
+                                                          int n_items) {
+    const int row = threadIdx.x & 127, sub = threadIdx.x >> 7;
+    const int mt = blockIdx.y, grow = mt * TC_BM + row;
+    if (grow >= g.M) return;
+    for (int k = 0; k < FIN_ITEMS_PER_SUB; ++k) {
+        const int item = (blockIdx.x * 2 + sub) * FIN_ITEMS_PER_SUB + k;
+        if (item >= n_items) return;
+        int nt, pc0, pc1;            // N tile, partial column groups of the two halves
+        int u128 = 0, r = 0;
+        if (g.epilogue == kEpiResidual) {
+            nt = item >> 6; pc0 = item & 63; pc1 = -1;
+        } else if (g.epilogue == kEpiSwiGLU) {
+            nt = item >> 5; pc0 = item & 31; pc1 = 32 + pc0;
+        } else {
+            u128 = item >> 4; r = item & 15;
+            nt = u128 >> 1;
+            const int c4 = g.head_dim == 128 ? r : ((r >> 3) << 4) + (r & 7);
+            pc0 = 32 * (u128 & 1) + c4;
+            pc1 = pc0 + (g.head_dim >> 3);
+        }
+        const int t = mt * p.n_tiles + nt;
+        const int c_first = (int)(((int64_t)t * p.KB) / p.U);
+        const int c_last = (int)(((int64_t)(t + 1) * p.KB - 1) / p.U);
+        const int nslots = c_last - c_first + 1;
+        const float4* src = reinterpret_cast<const float4*>(partial + (int64_t)t * p.smax * TC_SLOT_FLOATS);
+        const float4 v0 = sum_slots(src, nslots, pc0, row);
+        if (g.epilogue == kEpiResidual) {
+            const int N = g.n[0], col = item * 4;
+            const int64_t roff = g.resid_off ? g.resid_off[grow] : (int64_t)grow * N;
+            const uint2 rv = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.resid) + roff + col);
+            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * N + col) =
+                pack4(v0.x + bf16_lo(rv.x), v0.y + bf16_hi(rv.x), v0.z + bf16_lo(rv.y), v0.w + bf16_hi(rv.y));
+            continue;
+        }
+        const float4 v1 = sum_slots(src, nslots, pc1, row);
+        if (g.epilogue == kEpiSwiGLU) {
+            const float gt[4] = {v0.x, v0.y, v0.z, v0.w}, up[4] = {v1.x, v1.y, v1.z, v1.w};
+            float o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[i] = gt[i] / (1.f + __expf(-gt[i])) * up[i];
+            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * g.n[0] + item * 4) =
+                pack4(o[0], o[1], o[2], o[3]);
+            continue;
+        }
+        // q/k/v: bias, rotary embedding with the pairing (i, i + d/2), store (+ fused cache scatter)
+        int seg = 0, c0 = u128 * 128;
+        while (seg < 2 && c0 >= g.n[seg]) { c0 -= g.n[seg]; ++seg; }
+        const int half = g.head_dim >> 1;
+        const int j4 = (g.head_dim == 128 ? r : (r & 7)) * 4;               // index inside the half head
+        const int col = c0 + (g.head_dim == 128 ? r * 4 : ((r >> 3) << 6) + (r & 7) * 4);
+        float lo[4] = {v0.x, v0.y, v0.z, v0.w}, hi[4] = {v1.x, v1.y, v1.z, v1.w};
+        const __nv_bfloat16* bias = static_cast<const __nv_bfloat16*>(g.bias[seg]);
+        if (bias) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                lo[i] += __bfloat162float(bias[col + i]);
+                hi[i] += __bfloat162float(bias[col + half + i]);
             }
         }
-        *reinterpret_cast<float4*>(stage + row * kStagePitch + jc * 4) = s;
-    }
-    __syncthreads();
-    if (g.epilogue == kEpiQKV) {
-        int seg = 0, c0 = u * 128;
-        while (seg < 2 && c0 >= g.n[seg]) { c0 -= g.n[seg]; ++seg; }
-        epilogue_qkv(g, stage, m0, seg, c0, threadIdx.x, 256);
-    } else if (g.epilogue == kEpiResidual) {
-        epilogue_residual(g, stage, m0, u * 128, g.n[0], threadIdx.x, 256);
-    } else {
-        epilogue_swiglu(g, stage, m0, u * 64, g.n[0], threadIdx.x, 256);
+        const int pos = g.row_pos[grow];
+        if (seg < g.rope_segments) {
+            const int pp = pos < 0 ? 0 : pos;
+            const float4 cs = *reinterpret_cast<const float4*>(g.rope_cos + (int64_t)pp * half + j4);
+            const float4 sn = *reinterpret_cast<const float4*>(g.rope_sin + (int64_t)pp * half + j4);
+            const float c[4] = {cs.x, cs.y, cs.z, cs.w}, sv[4] = {sn.x, sn.y, sn.z, sn.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float x = lo[i], y = hi[i];
+                lo[i] = x * c[i] - y * sv[i];
+                hi[i] = y * c[i] + x * sv[i];
+            }
+        }
+        const uint2 plo = pack4(lo[0], lo[1], lo[2], lo[3]), phi = pack4(hi[0], hi[1], hi[2], hi[3]);
+        const int nseg = g.n[seg];
+        if (g.out[seg]) {
+            __nv_bfloat16* o = static_cast<__nv_bfloat16*>(g.out[seg]) + (int64_t)grow * nseg + col;
+            *reinterpret_cast<uint2*>(o) = plo;
+            *reinterpret_cast<uint2*>(o + half) = phi;
+        }
+        __nv_bfloat16* cache = seg == 1 ? static_cast<__nv_bfloat16*>(g.cache_k)
+                             : seg == 2 ? static_cast<__nv_bfloat16*>(g.cache_v) : nullptr;
+        if (cache && pos >= 0) {
+            const int b = grow / g.rows_per_req;
+            __nv_bfloat16* o = cache + (int64_t)b * g.kv_batch_stride + (int64_t)pos * nseg + col;
+            *reinterpret_cast<uint2*>(o) = plo;
+            *reinterpret_cast<uint2*>(o + half) = phi;
+        }
     }
 }
 
@@ -429,12 +507,12 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
     static bool attr = false;
     if (!attr) {
         cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
-        cudaFuncSetAttribute(gemm_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * kStagePitch * 4);
         attr = true;
     }
     gemm_tc_kernel<<<a.p.ctas, TC_THREADS, TC_SMEM, stream>>>(a, *mA, *mB[0], *mB[1], *mB[2]);
-    const int out_units = swiglu ? g.n[0] / 64 : n_total / 128;
-    gemm_finish_kernel<<<dim3(out_units, a.p.m_tiles), 256, 128 * kStagePitch * 4, stream>>>(g, a.p, g.partial);
+    const int n_items = g.epilogue == kEpiQKV ? n_total / 8 : n_total / 4;
+    const int per_cta = 2 * FIN_ITEMS_PER_SUB;
+    gemm_finish_kernel<<<dim3((n_items + per_cta - 1) / per_cta, a.p.m_tiles), 256, 0, stream>>>(g, a.p, g.partial, n_items);
     return 2;
 }
 

@@ -103,8 +103,10 @@ struct AttnArgs {
     const int32_t* slot;      // [B, ctx_len] or null: >= 0 => read k_new/v_new row slot
     int batch, n, ctx_len, n_heads, n_kv_heads, head_dim;
     void* o;                  // bf16 [B, n, H*d]
-    float* row_sum;           // optional [B, n, H]: sum of the normalised weights (debug)
+    float* part_o;            // scratch for key splits: fp32 [B*n*H, n_split, d]
+    float* part_ml;           // scratch for key splits: fp32 [B*n*H, n_split, 2] (max, denominator)
 };
+size_t attention_scratch_bytes(int head_dim);   // bytes for part_o followed by part_ml
 int launch_attention(const AttnArgs& a, cudaStream_t stream);
 
 }  // namespace acache

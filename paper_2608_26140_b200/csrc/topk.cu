@@ -73,9 +73,16 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
         const uint32_t prefix = s_prefix;
-        for (int j = tid; j < L; j += kTopkThreads) {
-            uint32_t kk = key_at(j);
-            if ((kk & mask) == prefix) atomicAdd(&hist[(kk >> shift) & 0xFF], 1);
+        for (int j0 = 0; j0 < L; j0 += kTopkThreads) {
+            // one shared-memory atomic per distinct digit per warp (scores often share their top bytes)
+            const int j = j0 + tid;
+            int digit = -1;
+            if (j < L) {
+                const uint32_t kk = key_at(j);
+                if ((kk & mask) == prefix) digit = (kk >> shift) & 0xFF;
+            }
+            const unsigned peers = __match_any_sync(0xffffffffu, digit);
+            if (digit >= 0 && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
         }
         __syncthreads();
         if (tid == 0) {
