@@ -107,7 +107,7 @@ acache_status check_weights(acache_ctx* c, const acache_layer_weights* w, bool q
 
 // Q for the masked rows, then Eq. 4-5.
 acache_status run_score(acache_ctx* c, const acache_request* r, const void* q_mask, const acache_kv* kv,
-                        float* scores, int accumulate, int norm_full, cudaStream_t st) {
+                        float* scores, int accumulate, int norm_full, int defer_head_sum, cudaStream_t st) {
     ScoreArgs a{};
     a.q_mask = q_mask;
     a.cache_k = kv->k;
@@ -121,6 +121,7 @@ acache_status run_score(acache_ctx* c, const acache_request* r, const void* q_ma
     a.head_partial = wsp<float>(c, c->o_partial);
     a.scores = scores;
     a.accumulate = accumulate;
+    a.defer_head_sum = defer_head_sum;
     int n = launch_score(a, st);
     if (n < 0) return fail(c, ACACHE_ERR_UNSUPPORTED_SHAPE, "n_masked %d too large for the scoring kernel", r->n_masked);
     c->launches += n;
@@ -350,7 +351,7 @@ acache_status acache_score_anchors(acache_ctx* ctx, const acache_request* req, c
     acache_status s = check_request(ctx, req, kv, 0, false);
     if (s != ACACHE_OK) return s;
     if (!scores || (req->n_masked > 0 && (!q_mask || !aligned16(q_mask)))) return fail(ctx, ACACHE_ERR_INVALID_ARG, "q_mask / scores NULL or misaligned");
-    return run_score(ctx, req, q_mask, kv, scores, accumulate, norm_full, stream);
+    return run_score(ctx, req, q_mask, kv, scores, accumulate, norm_full, 0, stream);
 }
 
 acache_status acache_select_topk(acache_ctx* ctx, const float* scores, int32_t batch, int32_t affix_len, int32_t k,
@@ -359,7 +360,7 @@ acache_status acache_select_topk(acache_ctx* ctx, const float* scores, int32_t b
     if (batch < 0 || affix_len < 0 || k < 0 || k > affix_len) return fail(ctx, ACACHE_ERR_INVALID_ARG, "batch %d, affix_len %d, k %d out of range", batch, affix_len, k);
     if (batch == 0 || k == 0) return ACACHE_OK;
     if (!scores || !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "scores / anchor_idx is NULL");
-    launch_topk(scores, batch, affix_len, k, anchor_idx, stream);
+    launch_topk(const_cast<float*>(scores), batch, affix_len, k, anchor_idx, nullptr, 0, 0, stream);
     ctx->launches += 1;
     return check_cuda(ctx, "topk");
 }
@@ -416,6 +417,7 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
     if (do_recompute && req->batch * (k + req->n_extra) > 0 && (!y || !aligned16(y))) return fail(ctx, ACACHE_ERR_INVALID_ARG, "y NULL or misaligned");
 
     if (ctx->timing) for (bool& h : ctx->ev_hit) h = false;
+    bool fused_head_sum = false;
     if (do_score && req->batch > 0 && req->affix_len > 0) {
         void* qmask = wsp<void>(ctx, ctx->o_qmask);
         mark(ctx, ACACHE_STAGE_MASK_Q, stream);
@@ -438,13 +440,17 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
             ctx->launches += launch_gemm(g, stream);
         }
         mark(ctx, ACACHE_STAGE_SCORE, stream);
+        // with a selection to follow, the ordered sum over heads is folded into the selection kernel
+        fused_head_sum = do_select && k > 0 && req->n_masked > 0;
         s = run_score(ctx, req, qmask, kv, scores, (flags & ACACHE_F_ACCUMULATE) ? 1 : 0,
-                      (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, stream);
+                      (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, fused_head_sum ? 1 : 0, stream);
         if (s != ACACHE_OK) return s;
     }
     if (do_select && k > 0 && req->batch > 0) {
         mark(ctx, ACACHE_STAGE_TOPK, stream);
-        launch_topk(scores, req->batch, req->affix_len, k, anchor_idx, stream);
+        launch_topk(scores, req->batch, req->affix_len, k, anchor_idx,
+                    fused_head_sum ? wsp<float>(ctx, ctx->o_partial) : nullptr, d.n_heads,
+                    (flags & ACACHE_F_ACCUMULATE) ? 1 : 0, stream);
         ctx->launches += 1;
     }
     if (do_recompute)

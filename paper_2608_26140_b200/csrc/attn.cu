@@ -6,6 +6,7 @@
 // the working cache without having written it).
 #include "common.cuh"
 #include "kernels.h"
+#include "launch.h"
 
 namespace acache {
 
@@ -60,6 +61,8 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int TILE = 64 * D * 2;
     const uint32_t sQ = smem_u32(smem);
+    pdl_wait();
+    pdl_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int qt = blockIdx.x / n_split, split = blockIdx.x % n_split, h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / (a.n_heads / a.n_kv_heads);
@@ -205,6 +208,8 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
 // Merges the key splits of one (row, head): o = sum_s O_s 2^(m_s - m) / sum_s l_s 2^(m_s - m).
 template <int D>
 __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnArgs a, int n_split, int64_t n_rh) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int64_t rh = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
     if (rh >= n_rh) return;
@@ -252,13 +257,13 @@ int launch_attention(const AttnArgs& a, cudaStream_t stream) {
     if (a.head_dim == 128) {
         constexpr int SMEM = (1 + 2 * ATT_STAGES) * 64 * 128 * 2;
         cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-        attention_kernel<128><<<grid, 128, SMEM, stream>>>(a, scale_log2e, n_split, tps);
-        if (n_split > 1) attention_combine_kernel<128><<<(unsigned)((n_rh + 3) / 4), 128, 0, stream>>>(a, n_split, n_rh);
+        launch_pdl(attention_kernel<128>, grid, 128, SMEM, stream, a, scale_log2e, n_split, tps);
+        if (n_split > 1) launch_pdl(attention_combine_kernel<128>, (unsigned)((n_rh + 3) / 4), 128, 0, stream, a, n_split, n_rh);
     } else {
         constexpr int SMEM = (1 + 2 * ATT_STAGES) * 64 * 64 * 2;
         cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-        attention_kernel<64><<<grid, 128, SMEM, stream>>>(a, scale_log2e, n_split, tps);
-        if (n_split > 1) attention_combine_kernel<64><<<(unsigned)((n_rh + 3) / 4), 128, 0, stream>>>(a, n_split, n_rh);
+        launch_pdl(attention_kernel<64>, grid, 128, SMEM, stream, a, scale_log2e, n_split, tps);
+        if (n_split > 1) launch_pdl(attention_combine_kernel<64>, (unsigned)((n_rh + 3) / 4), 128, 0, stream, a, n_split, n_rh);
     }
     return n_split > 1 ? 2 : 1;
 }

@@ -25,6 +25,7 @@
 #include "common.cuh"
 #include "gemm_epilogue.cuh"
 #include "kernels.h"
+#include "launch.h"
 
 namespace acache {
 
@@ -179,6 +180,9 @@ gemm_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap mapA, const _
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above overlaps the previous kernel's tail; global memory is touched only below
+    pdl_wait();
+    pdl_launch_dependents();
 
     const TcPlan& p = a.p;
     const int it0 = blockIdx.x * p.U;
@@ -313,6 +317,8 @@ __device__ __forceinline__ uint2 pack4(float a, float b, float c, float d) {
 
 __global__ void __launch_bounds__(256) gemm_finish_kernel(const GemmArgs g, const TcPlan p, const float* __restrict__ partial,
                                                           int n_items) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int row = threadIdx.x & 127, sub = threadIdx.x >> 7;
     const int mt = blockIdx.y, grow = mt * TC_BM + row;
     if (grow >= g.M) return;
@@ -509,10 +515,11 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
         cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
         attr = true;
     }
-    gemm_tc_kernel<<<a.p.ctas, TC_THREADS, TC_SMEM, stream>>>(a, *mA, *mB[0], *mB[1], *mB[2]);
+    launch_pdl(gemm_tc_kernel, a.p.ctas, TC_THREADS, TC_SMEM, stream, a, *mA, *mB[0], *mB[1], *mB[2]);
     const int n_items = g.epilogue == kEpiQKV ? n_total / 8 : n_total / 4;
     const int per_cta = 2 * FIN_ITEMS_PER_SUB;
-    gemm_finish_kernel<<<dim3((n_items + per_cta - 1) / per_cta, a.p.m_tiles), 256, 0, stream>>>(g, a.p, g.partial, n_items);
+    launch_pdl(gemm_finish_kernel, dim3((n_items + per_cta - 1) / per_cta, a.p.m_tiles), 256, 0, stream, g, a.p,
+               (const float*)g.partial, n_items);
     return 2;
 }
 

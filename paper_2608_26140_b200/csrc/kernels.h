@@ -43,13 +43,16 @@ struct ScoreArgs {
     float* head_partial;      // [B, H, L]
     float* scores;            // [B, L]
     int accumulate;
+    int defer_head_sum;       // leave head_partial unsummed: launch_topk(.., head_partial) does it
 };
 int score_num_splits(int norm_len);
 int launch_score(const ScoreArgs& a, cudaStream_t stream);  // returns number of kernels launched
 
 // ---- topk.cu ----------------------------------------------------------------------------
-void launch_topk(const float* scores, int batch, int affix_len, int k, int32_t* anchor_idx,
-                 cudaStream_t stream);
+// head_partial != null: first scores[b, j] = (accumulate ? scores[b, j] : 0) + sum_h head_partial[b, h, j]
+// (ordered sum), then the selection runs on the result.
+void launch_topk(float* scores, int batch, int affix_len, int k, int32_t* anchor_idx, const float* head_partial,
+                 int n_heads, int accumulate, cudaStream_t stream);
 
 // ---- gemm.cu ----------------------------------------------------------------------------
 enum GemmEpilogue : int {

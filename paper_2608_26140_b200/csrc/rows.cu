@@ -3,6 +3,7 @@
 // position -> fresh-row map used when the cache must not be mutated.
 #include "common.cuh"
 #include "kernels.h"
+#include "launch.h"
 
 namespace acache {
 
@@ -65,6 +66,8 @@ __global__ void __launch_bounds__(256) gather_rmsnorm_kernel(
     int32_t* __restrict__ row_pos, int64_t* __restrict__ row_src, __nv_bfloat16* __restrict__ xn,
     uint32_t* status) {
     __shared__ float red[8];
+    pdl_wait();
+    pdl_launch_dependents();
     const int rows_per_req = k + e;
     const int row = blockIdx.x;
     const int b = row / rows_per_req, i = row - b * rows_per_req;
@@ -85,6 +88,8 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* __res
                                                       const __nv_bfloat16* __restrict__ gain, float eps,
                                                       int hidden, __nv_bfloat16* __restrict__ xn) {
     __shared__ float red[8];
+    pdl_wait();
+    pdl_launch_dependents();
     const int64_t row = blockIdx.x;
     rmsnorm_row(reinterpret_cast<const uint4*>(x + row * hidden), reinterpret_cast<const uint4*>(gain),
                 reinterpret_cast<uint4*>(xn + row * hidden), hidden, eps, red);
@@ -95,6 +100,8 @@ __global__ void __launch_bounds__(128) scatter_kv_kernel(
     const int32_t* __restrict__ anchor_idx, int k, const int32_t* __restrict__ extra_rows, int e,
     int affix_start, int affix_len, int kv_dim, const __nv_bfloat16* __restrict__ k_new,
     const __nv_bfloat16* __restrict__ v_new, uint32_t* status) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int rows_per_req = k + e;
     const int row = blockIdx.x;
     const int b = row / rows_per_req, i = row - b * rows_per_req;
@@ -116,6 +123,8 @@ __global__ void __launch_bounds__(128) scatter_kv_kernel(
 
 __global__ void __launch_bounds__(1024) slot_map_kernel(int32_t* __restrict__ slot, int ctx_len,
                                                         const int32_t* __restrict__ row_pos, int rows_per_req) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int b = blockIdx.x;
     int32_t* s = slot + (int64_t)b * ctx_len;
     for (int t = threadIdx.x; t < ctx_len; t += blockDim.x) s[t] = -1;
@@ -135,7 +144,7 @@ void launch_gather_rmsnorm(const void* x, int x_is_compact, int64_t x_batch_stri
                            int32_t* row_pos, int64_t* row_src, void* xn, uint32_t* status, cudaStream_t stream) {
     const int n = batch * (k + e);
     if (n == 0) return;
-    gather_rmsnorm_kernel<<<n, 256, 0, stream>>>(
+    launch_pdl(gather_rmsnorm_kernel, n, 256, 0, stream,
         static_cast<const __nv_bfloat16*>(x), x_is_compact, x_batch_stride, hidden, anchor_idx, k, extra_rows, e,
         affix_start, affix_len, ctx_len, static_cast<const __nv_bfloat16*>(gain), eps, row_pos, row_src,
         static_cast<__nv_bfloat16*>(xn), status);
@@ -143,7 +152,7 @@ void launch_gather_rmsnorm(const void* x, int x_is_compact, int64_t x_batch_stri
 
 void launch_rmsnorm(const void* x, const void* gain, float eps, int n, int hidden, void* xn, cudaStream_t stream) {
     if (n == 0) return;
-    rmsnorm_kernel<<<n, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(x),
+    launch_pdl(rmsnorm_kernel, n, 256, 0, stream, static_cast<const __nv_bfloat16*>(x),
                                           static_cast<const __nv_bfloat16*>(gain), eps, hidden,
                                           static_cast<__nv_bfloat16*>(xn));
 }
@@ -153,7 +162,7 @@ void launch_scatter_kv(void* cache_k, void* cache_v, int64_t batch_stride, int c
                        int kv_dim, const void* k_new, const void* v_new, uint32_t* status, cudaStream_t stream) {
     const int n = batch * (k + e);
     if (n == 0) return;
-    scatter_kv_kernel<<<n, 128, 0, stream>>>(static_cast<__nv_bfloat16*>(cache_k),
+    launch_pdl(scatter_kv_kernel, n, 128, 0, stream, static_cast<__nv_bfloat16*>(cache_k),
                                              static_cast<__nv_bfloat16*>(cache_v), batch_stride, ctx_len,
                                              anchor_idx, k, extra_rows, e, affix_start, affix_len, kv_dim,
                                              static_cast<const __nv_bfloat16*>(k_new),
@@ -163,7 +172,7 @@ void launch_scatter_kv(void* cache_k, void* cache_v, int64_t batch_stride, int c
 void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
                            cudaStream_t stream) {
     if (batch == 0) return;
-    slot_map_kernel<<<batch, 1024, 0, stream>>>(slot, ctx_len, row_pos, rows_per_req);
+    launch_pdl(slot_map_kernel, batch, 1024, 0, stream, slot, ctx_len, row_pos, rows_per_req);
 }
 
 }  // namespace acache

@@ -11,6 +11,7 @@
 // bound by the K_affix read, not by ALU work.
 #include "common.cuh"
 #include "kernels.h"
+#include "launch.h"
 
 namespace acache {
 
@@ -72,6 +73,8 @@ __global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_spl
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int TILE = 64 * D * 2;
     const uint32_t sQ = smem_u32(smem), sK0 = sQ + TILE;
+    pdl_wait();
+    pdl_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int split = blockIdx.x, h = blockIdx.y;
     const int mtiles = (a.m + 63) / 64;
@@ -158,6 +161,8 @@ __global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_sp
     const uint32_t sK = smem_u32(smem), sQ0 = sK + TILE;
     float* s_max = reinterpret_cast<float*>(smem + 3 * TILE);
     float* s_inv = s_max + a.m;
+    pdl_wait();
+    pdl_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int jt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / (a.n_heads / a.n_kv_heads);
@@ -226,6 +231,8 @@ __global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_sp
 __global__ void __launch_bounds__(256) score_reduce_heads_kernel(const float* __restrict__ head_partial,
                                                                  float* __restrict__ scores, int n_heads, int L,
                                                                  int accumulate) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int b = blockIdx.y;
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= L) return;
@@ -245,11 +252,13 @@ static int launch_score_d(const ScoreArgs& a, cudaStream_t stream) {
     const size_t smem2 = 3 * TILE + (size_t)a.m * 8;
     cudaFuncSetAttribute(score_stats_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
     cudaFuncSetAttribute(score_colsum_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
-    score_stats_kernel<D><<<dim3(n_split, a.n_heads, a.batch * mtiles), 128, smem1, stream>>>(a, n_split, scale_log2e);
-    score_colsum_kernel<D><<<dim3((a.affix_len + 63) / 64, a.n_heads, a.batch), 128, smem2, stream>>>(a, n_split,
-                                                                                                     scale_log2e);
-    score_reduce_heads_kernel<<<dim3((a.affix_len + 255) / 256, a.batch), 256, 0, stream>>>(
-        a.head_partial, a.scores, a.n_heads, a.affix_len, a.accumulate);
+    launch_pdl(score_stats_kernel<D>, dim3(n_split, a.n_heads, a.batch * mtiles), 128, smem1, stream, a, n_split,
+               scale_log2e);
+    launch_pdl(score_colsum_kernel<D>, dim3((a.affix_len + 63) / 64, a.n_heads, a.batch), 128, smem2, stream, a,
+               n_split, scale_log2e);
+    if (a.defer_head_sum) return 2;   // the selection kernel sums the heads itself
+    launch_pdl(score_reduce_heads_kernel, dim3((a.affix_len + 255) / 256, a.batch), 256, 0, stream, a.head_partial,
+               a.scores, a.n_heads, a.affix_len, a.accumulate);
     return 3;
 }
 

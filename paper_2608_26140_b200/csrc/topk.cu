@@ -3,6 +3,7 @@
 // pass over positions emits the anchors ascending, ties going to the lower position.
 #include "common.cuh"
 #include "kernels.h"
+#include "launch.h"
 
 namespace acache {
 
@@ -45,8 +46,10 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* t
     return r;
 }
 
-__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restrict__ scores, int L, int K,
-                                                            int32_t* __restrict__ anchor_idx, int use_smem) {
+__global__ void __launch_bounds__(kTopkThreads) topk_kernel(float* scores, int L, int K,
+                                                            int32_t* __restrict__ anchor_idx, int use_smem,
+                                                            const float* __restrict__ head_partial, int n_heads,
+                                                            int accumulate) {
     extern __shared__ uint32_t keys_s[];
     __shared__ int hist[256];
     __shared__ int warp_tot[32];
@@ -54,11 +57,21 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
     __shared__ uint32_t s_prefix;
     __shared__ int s_want;
 
+    pdl_wait();
+    pdl_launch_dependents();
     const int b = blockIdx.x;
-    const float* s = scores + (int64_t)b * L;
+    float* s = scores + (int64_t)b * L;
     int32_t* out = anchor_idx + (int64_t)b * K;
     const int tid = threadIdx.x;
 
+    if (head_partial) {   // Eq. 5: ordered sum over heads, fused in front of the selection
+        for (int j = tid; j < L; j += kTopkThreads) {
+            float v = 0.f;
+            for (int h = 0; h < n_heads; ++h) v += head_partial[((int64_t)b * n_heads + h) * L + j];
+            s[j] = accumulate ? s[j] + v : v;
+        }
+        __syncthreads();
+    }
     if (use_smem)
         for (int j = tid; j < L; j += kTopkThreads) keys_s[j] = score_key(s[j]);
     if (tid == 0) { s_prefix = 0u; s_want = K; }
@@ -85,14 +98,30 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
             if (digit >= 0 && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
         }
         __syncthreads();
-        if (tid == 0) {
-            int want = s_want, d = 255;
-            for (; d > 0; --d) {           // walk down from the largest digit
-                if (hist[d] >= want) break;
-                want -= hist[d];
+        if (tid < 32) {
+            // lane l owns digits 255-8l .. 248-8l (descending); find the digit where the running
+            // count from the top reaches the wanted rank
+            int cnt[8], mine = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { cnt[i] = hist[255 - 8 * tid - i]; mine += cnt[i]; }
+            int inc = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int t = __shfl_up_sync(0xffffffffu, inc, o);
+                if (tid >= o) inc += t;
             }
-            s_prefix = prefix | ((uint32_t)d << shift);
-            s_want = want;
+            const int want = s_want;
+            const int before = inc - mine;                 // elements in digits above this lane's
+            if (before < want && want <= inc) {            // exactly one lane
+                int w = want - before, d = 255 - 8 * tid;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (cnt[i] >= w) { d = 255 - 8 * tid - i; break; }
+                    w -= cnt[i];
+                }
+                s_prefix = prefix | ((uint32_t)d << shift);
+                s_want = w;
+            }
         }
         __syncthreads();
     }
@@ -117,14 +146,16 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float* __restr
     }
 }
 
-void launch_topk(const float* scores, int batch, int affix_len, int k, int32_t* anchor_idx, cudaStream_t stream) {
-    if (batch == 0 || k == 0) return;
+void launch_topk(float* scores, int batch, int affix_len, int k, int32_t* anchor_idx, const float* head_partial,
+                 int n_heads, int accumulate, cudaStream_t stream) {
+    if (batch == 0 || (k == 0 && !head_partial)) return;
     const int use_smem = affix_len <= kTopkSmemKeys;
     const size_t smem = use_smem ? (size_t)affix_len * sizeof(uint32_t) : 0;
     if (smem > 48 * 1024)
         cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kTopkSmemKeys * (int)sizeof(uint32_t));
-    topk_kernel<<<batch, kTopkThreads, smem, stream>>>(scores, affix_len, k, anchor_idx, use_smem);
+    launch_pdl(topk_kernel, batch, kTopkThreads, smem, stream, scores, affix_len, k, anchor_idx, use_smem, head_partial,
+               n_heads, accumulate);
 }
 
 }  // namespace acache
