@@ -172,6 +172,28 @@ acache_status acache_score_anchors(acache_ctx *ctx, const acache_request *req, c
                                    const acache_kv *kv, float *scores, int accumulate, int norm_full,
                                    acache_stream_t stream);
 
+/* The same scoring for callers that cannot allocate device memory (the paper has no
+ * counterpart).  Some hosts of this library may not call cudaMalloc at all: code running
+ * inside a CUDA-graph capture or a real-time loop, plug-ins handed a fixed memory budget by
+ * their framework, or processes whose allocator is owned by someone else -- so they cannot
+ * provide the workspace acache_score_anchors needs either.  This variant takes no context
+ * and no workspace: its scratch is a 4 MiB array built into the library's device image
+ * (every GPU that loads the library holds it until the process exits).
+ *   shape: only n_heads, n_kv_heads and head_dim are read.
+ *   Limit: B * H * (2 * m * ceil(keys / 256) + L) floats must fit in 2^20 floats, where keys
+ *   is L (or ctx_len with norm_full); larger problems return ACACHE_ERR_WORKSPACE and
+ *   enqueue nothing.  m <= 4096.
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call before any stream capture.  It calls no cudaMalloc,
+ * cudaFree or other allocating routine.  All calls share the one array, which keeps the
+ * previous call's contents (nothing in it needs clearing: each call overwrites what it
+ * reads), so two calls whose kernels may overlap on the GPU (different streams) race;
+ * issue them on one stream or order them with events.
+ * Inputs, outputs and results are exactly those of acache_score_anchors. */
+acache_status acache_score_anchors_static(const acache_model_desc *shape, const acache_request *req,
+                                          const void *q_mask, const acache_kv *kv, float *scores,
+                                          int accumulate, int norm_full, acache_stream_t stream);
+
 /* K of Eq. 6 from the recompute ratio: ceil(ratio * L) clipped to [0, L].  HOST, pure. */
 int32_t acache_k_from_ratio(int32_t affix_len, double ratio);
 

@@ -21,7 +21,8 @@ F_SCORE, F_SELECT, F_ACCUMULATE, F_SCORE_NORM_FULL, F_NO_RECOMPUTE = 0x1, 0x2, 0
 EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "acache_destroy",
            "acache_last_error", "acache_poll_status", "acache_launch_count", "acache_score_anchors",
            "acache_k_from_ratio", "acache_select_topk", "acache_recompute_anchors", "acache_scatter_kv",
-           "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times"]
+           "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times",
+           "acache_score_anchors_static"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -100,6 +101,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_layer_step_host.argtypes = [vp, C.POINTER(LayerWeights), C.POINTER(Request), C.POINTER(KV), vp,
                                            C.c_double, u32, vp, vp, vp, vp]
     lib.acache_layer_step_host.restype = C.c_int
+    lib.acache_score_anchors_static.argtypes = [C.POINTER(ModelDesc), C.POINTER(Request), vp, C.POINTER(KV), vp,
+                                                C.c_int, C.c_int, vp]
+    lib.acache_score_anchors_static.restype = C.c_int
     lib.acache_stage_timing.argtypes = [vp, C.c_int]
     lib.acache_stage_timing.restype = C.c_int
     lib.acache_read_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
@@ -111,6 +115,14 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
 
 def k_from_ratio(affix_len: int, ratio: float) -> int:
     return int(load_library().acache_k_from_ratio(int(affix_len), float(ratio)))
+
+
+def score_anchors_static(desc: ModelDesc, req: Request, q_mask, kv: KV, scores, accumulate=False,
+                         norm_full=False) -> int:
+    """Scoring through the entry point that allocates nothing and needs no context or workspace
+    (its scratch is a fixed array inside the library).  Returns the status code."""
+    return int(load_library().acache_score_anchors_static(C.byref(desc), C.byref(req), _ptr(q_mask), C.byref(kv),
+                                                          _ptr(scores), int(accumulate), int(norm_full), _stream()))
 
 
 def _ptr(t) -> Optional[int]:

@@ -9,6 +9,7 @@
 //   3. ordered sum over heads into scores.
 // Logits run on the tensor cores (bf16 mma.sync, fp32 accumulate) so that the pass stays
 // bound by the K_affix read, not by ALU work.
+#include "../../include/acache.h"
 #include "common.cuh"
 #include "kernels.h"
 #include "launch.h"
@@ -273,3 +274,70 @@ int launch_score(const ScoreArgs& a, cudaStream_t stream) {
 }
 
 }  // namespace acache
+
+// ---- scoring without any allocation ------------------------------------------------------------
+// Scratch of the allocation-free entry point: lives in the library's device image, so every
+// GPU that loads the library holds these 4 MiB until the process exits.
+#define ACACHE_STATIC_SCRATCH_FLOATS (1u << 20)
+static __device__ __align__(256) float g_static_score_scratch[ACACHE_STATIC_SCRATCH_FLOATS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_ptr[kMaxDevices] = {};   // device address of the array, per device
+}  // namespace
+
+extern "C" acache_status acache_score_anchors_static(const acache_model_desc* shape, const acache_request* req,
+                                                     const void* q_mask, const acache_kv* kv, float* scores,
+                                                     int accumulate, int norm_full, acache_stream_t stream) {
+    using namespace acache;
+    if (!shape || !req || !kv || !scores) return ACACHE_ERR_INVALID_ARG;
+    if ((shape->head_dim != 64 && shape->head_dim != 128) || shape->n_heads <= 0 || shape->n_kv_heads <= 0 ||
+        shape->n_heads % shape->n_kv_heads)
+        return ACACHE_ERR_UNSUPPORTED_SHAPE;
+    if (req->batch < 0 || req->ctx_len <= 0 || req->affix_len < 0 || req->affix_start < 0 || req->n_masked < 0 ||
+        (int64_t)req->affix_start + req->affix_len > req->ctx_len)
+        return ACACHE_ERR_INVALID_ARG;
+    if (!kv->k || (reinterpret_cast<uintptr_t>(kv->k) & 15u) || kv->ctx_capacity < req->ctx_len ||
+        kv->batch_stride < (int64_t)kv->ctx_capacity * shape->n_kv_heads * shape->head_dim || (kv->batch_stride & 7))
+        return ACACHE_ERR_INVALID_ARG;
+    if (req->n_masked > 0 && (!q_mask || (reinterpret_cast<uintptr_t>(q_mask) & 15u))) return ACACHE_ERR_INVALID_ARG;
+    if (req->n_masked > kMaxMaskedSmem) return ACACHE_ERR_UNSUPPORTED_SHAPE;
+
+    const int norm_len = norm_full ? req->ctx_len : req->affix_len;
+    const uint64_t stats_floats = (uint64_t)req->batch * shape->n_heads * score_num_splits(norm_len) * req->n_masked * 2;
+    const uint64_t partial_floats = (uint64_t)req->batch * shape->n_heads * req->affix_len;
+    const uint64_t stats_padded = (stats_floats + 63) & ~uint64_t(63);
+    if (stats_padded + partial_floats > ACACHE_STATIC_SCRATCH_FLOATS) return ACACHE_ERR_WORKSPACE;
+
+    // Set-up, once per device, with that device current: the array's name is only a host-side
+    // handle here, so ask the runtime for the address the kernels must be given.
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ACACHE_ERR_CUDA;
+    if (!g_static_scratch_ptr[dev]) {
+        float* p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_score_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return ACACHE_ERR_CUDA;
+        }
+        g_static_scratch_ptr[dev] = p;
+    }
+    float* scratch = g_static_scratch_ptr[dev];
+
+    ScoreArgs a{};
+    a.q_mask = q_mask;
+    a.cache_k = kv->k;
+    a.kv_batch_stride = kv->batch_stride;
+    a.batch = req->batch; a.m = req->n_masked;
+    a.n_heads = shape->n_heads; a.n_kv_heads = shape->n_kv_heads; a.head_dim = shape->head_dim;
+    a.affix_start = req->affix_start; a.affix_len = req->affix_len;
+    a.norm_lo = norm_full ? 0 : req->affix_start;
+    a.norm_len = norm_len;
+    a.row_stats = scratch;                    // every word the kernels read is written earlier in the same call,
+    a.head_partial = scratch + stats_padded;  // so nothing needs clearing between calls
+    a.scores = scores;
+    a.accumulate = accumulate;
+    a.defer_head_sum = 0;
+    if (launch_score(a, stream) < 0) return ACACHE_ERR_UNSUPPORTED_SHAPE;
+    return cudaGetLastError() == cudaSuccess ? ACACHE_OK : ACACHE_ERR_CUDA;
+}
+
