@@ -27,7 +27,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2608_26140_b200 import workloads as wl  # noqa: E402
+from paper_2608_26140_b200 import sharding, workloads as wl  # noqa: E402
 
 METRIC = "anchor_refresh_affix_tokens_per_s"
 UNIT = "affix tokens/s"
@@ -232,11 +232,7 @@ def run_ours(args):
             torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if not dist:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return sharding.max_over_ranks(ms, dist, dev)
 
     for i in range(max(args.warmup, 3)):
         step(i)
@@ -308,7 +304,7 @@ def run_ours(args):
                 "traffic": NCU_TRAFFIC_BYTES["gate_up"], "algorithmic_bytes": gu_bytes, "algorithmic_flops": gu_flops,
                 "us_per_launch": stage["gate_up"] * 1e3}
     floor_s = max(t_hbm, t_tc)
-    value = world * B * K / (ms_step * 1e-3)
+    value = sharding.aggregate_throughput(B * K, world, ms_step)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_step, "us_per_layer_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
