@@ -22,7 +22,7 @@ struct acache_ctx {
     // workspace offsets (bytes)
     size_t o_status, o_row_pos, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
     size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
-    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn;
+    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar;
     std::string err;
     uint64_t launches = 0;
     // optional per-stage timing (acache_stage_timing)
@@ -150,15 +150,17 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     void* act = wsp<void>(c, c->o_act);
     uint32_t* status = wsp<uint32_t>(c, c->o_status);
 
-    mark(c, ACACHE_STAGE_GATHER_NORM, st);
-    launch_gather_rmsnorm(x, x_is_compact, (int64_t)r->ctx_len * d.hidden, d.hidden, anchor_idx, k, r->extra_rows,
-                          r->n_extra, r->batch, r->affix_start, r->affix_len, r->ctx_len, w->attn_norm_g, d.rms_eps,
-                          row_pos, row_src, xn, status, st);
-    c->launches += 1;
     mark(c, ACACHE_STAGE_QKV, st);
+    unsigned int* grid_bar = wsp<unsigned int>(c, c->o_gridbar);
+    float* partial = wsp<float>(c, c->o_gemm);
 
     GemmArgs g{};
     g.a = xn; g.M = n; g.K = d.hidden;
+    g.prep.enabled = 1; g.prep.x = x; g.prep.x_is_compact = x_is_compact;
+    g.prep.x_batch_stride = (int64_t)r->ctx_len * d.hidden;
+    g.prep.anchor_idx = anchor_idx; g.prep.k = k; g.prep.extra_rows = r->extra_rows; g.prep.e = r->n_extra;
+    g.prep.affix_start = r->affix_start; g.prep.affix_len = r->affix_len; g.prep.ctx_len = r->ctx_len;
+    g.prep.gain = w->attn_norm_g; g.prep.eps = d.rms_eps; g.prep.row_pos = row_pos; g.prep.row_src = row_src;
     g.b[0] = w->wq; g.b[1] = w->wk; g.b[2] = w->wv;
     g.n[0] = qd; g.n[1] = kvd; g.n[2] = kvd;
     g.epilogue = kEpiQKV;
@@ -170,8 +172,9 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     g.out[0] = q; g.out[1] = k_new; g.out[2] = v_new;
     if (fuse_scatter) { g.cache_k = kv->k; g.cache_v = kv->v; }
     g.kv_batch_stride = kv->batch_stride; g.rows_per_req = rows;
-    g.partial = wsp<float>(c, c->o_gemm); g.status = status;
-    c->launches += launch_gemm(g, st);
+    g.partial = partial; g.status = status; g.grid_bar = grid_bar;
+    { int nl = launch_gemm(g, st); if (nl < 0) return check_cuda(c, "qkv projection") == ACACHE_OK ? fail(c, ACACHE_ERR_CUDA, "qkv projection launch failed") : ACACHE_ERR_CUDA;
+    c->launches += nl; }
 
     mark(c, ACACHE_STAGE_ATTENTION, st);
     AttnArgs at{};
@@ -193,26 +196,26 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     GemmArgs go{};
     go.a = o; go.M = n; go.K = qd; go.b[0] = w->wo; go.n[0] = d.hidden;
     go.epilogue = kEpiResidual; go.resid = x; go.resid_off = row_src; go.c = h1;
-    go.partial = wsp<float>(c, c->o_gemm); go.status = status;
-    c->launches += launch_gemm(go, st);
-
-    mark(c, ACACHE_STAGE_MLP_NORM, st);
-    launch_rmsnorm(h1, w->mlp_norm_g, d.rms_eps, n, d.hidden, xn2, st);
-    c->launches += 1;
+    go.partial = partial; go.status = status; go.grid_bar = grid_bar;
+    { int nl = launch_gemm(go, st); if (nl < 0) return check_cuda(c, "output projection") == ACACHE_OK ? fail(c, ACACHE_ERR_CUDA, "output projection launch failed") : ACACHE_ERR_CUDA;
+    c->launches += nl; }
     mark(c, ACACHE_STAGE_GATE_UP, st);
 
     GemmArgs gu{};
+    gu.prep.enabled = 2; gu.prep.x = h1; gu.prep.gain = w->mlp_norm_g; gu.prep.eps = d.rms_eps;   // xn2 = RMSNorm(h1)
     gu.a = xn2; gu.M = n; gu.K = d.hidden; gu.b[0] = w->w_gate; gu.b[1] = w->w_up; gu.n[0] = d.ffn; gu.n[1] = d.ffn;
     gu.epilogue = kEpiSwiGLU; gu.c = act;
-    gu.partial = wsp<float>(c, c->o_gemm); gu.status = status;
-    c->launches += launch_gemm(gu, st);
+    gu.partial = partial; gu.status = status; gu.grid_bar = grid_bar;
+    { int nl = launch_gemm(gu, st); if (nl < 0) return check_cuda(c, "gate/up projection") == ACACHE_OK ? fail(c, ACACHE_ERR_CUDA, "gate/up projection launch failed") : ACACHE_ERR_CUDA;
+    c->launches += nl; }
 
     mark(c, ACACHE_STAGE_DOWN, st);
     GemmArgs gd{};
     gd.a = act; gd.M = n; gd.K = d.ffn; gd.b[0] = w->w_down; gd.n[0] = d.hidden;
     gd.epilogue = kEpiResidual; gd.resid = h1; gd.resid_off = nullptr; gd.c = y;
-    gd.partial = wsp<float>(c, c->o_gemm); gd.status = status;
-    c->launches += launch_gemm(gd, st);
+    gd.partial = partial; gd.status = status; gd.grid_bar = grid_bar;
+    { int nl = launch_gemm(gd, st); if (nl < 0) return check_cuda(c, "down projection") == ACACHE_OK ? fail(c, ACACHE_ERR_CUDA, "down projection launch failed") : ACACHE_ERR_CUDA;
+    c->launches += nl; }
     mark(c, ACACHE_N_STAGES, st);
     return check_cuda(c, "recompute");
 }
@@ -238,6 +241,7 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
     const size_t nr = (size_t)d.max_batch * d.max_rows, nm = (size_t)d.max_batch * d.max_masked;
     size_t cur = 0;
     c->o_status = take(cur, 256);
+    c->o_gridbar = take(cur, 256);
     c->o_row_pos = take(cur, nr * 4);
     c->o_row_src = take(cur, nr * 8);
     c->o_xn = take(cur, nr * d.hidden * 2);
@@ -282,7 +286,8 @@ acache_status acache_set_workspace(acache_ctx* ctx, void* dev_ptr, size_t bytes,
     if (bytes < ctx->ws_need) return fail(ctx, ACACHE_ERR_WORKSPACE, "workspace %zu < %zu bytes", bytes, ctx->ws_need);
     ctx->ws = static_cast<unsigned char*>(dev_ptr);
     ctx->ws_have = bytes;
-    if (cudaMemsetAsync(ctx->ws + ctx->o_status, 0, 256, stream) != cudaSuccess) return check_cuda(ctx, "memset");
+    // status word and grid-barrier words are adjacent: clear both
+    if (cudaMemsetAsync(ctx->ws + ctx->o_status, 0, 512, stream) != cudaSuccess) return check_cuda(ctx, "memset");
     return ACACHE_OK;
 }
 
@@ -331,7 +336,12 @@ acache_status acache_poll_status(acache_ctx* ctx, acache_stream_t stream, uint32
         cudaStreamSynchronize(stream) != cudaSuccess)
         return check_cuda(ctx, "poll_status") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "poll_status failed") : ACACHE_ERR_CUDA;
     *host_flags = v;
-    if (v & ACACHE_FLAG_WAIT_EXPIRED) return fail(ctx, ACACHE_ERR_TIMEOUT, "a bounded device-side wait expired");
+    if (v & ACACHE_FLAG_WAIT_EXPIRED) {
+        // a kernel gave up half way: its grid-barrier words are stale, re-arm them
+        cudaMemsetAsync(ctx->ws + ctx->o_gridbar, 0, 256, stream);
+        cudaStreamSynchronize(stream);
+        return fail(ctx, ACACHE_ERR_TIMEOUT, "a bounded device-side wait expired");
+    }
     return ACACHE_OK;
 }
 
@@ -424,20 +434,23 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
         if (req->n_masked > 0) {
             int32_t* mpos = wsp<int32_t>(ctx, ctx->o_mrow_pos);
             void* xnm = wsp<void>(ctx, ctx->o_xn_mask);
-            launch_gather_rmsnorm(x, 0, (int64_t)req->ctx_len * d.hidden, d.hidden, nullptr, 0, req->masked_pos,
-                                  req->n_masked, req->batch, req->affix_start, req->affix_len, req->ctx_len,
-                                  w->attn_norm_g, d.rms_eps, mpos, wsp<int64_t>(ctx, ctx->o_mrow_src), xnm,
-                                  wsp<uint32_t>(ctx, ctx->o_status), stream);
-            ctx->launches += 1;
             GemmArgs g{};
             g.a = xnm; g.M = req->batch * req->n_masked; g.K = d.hidden;
+            g.prep.enabled = 1; g.prep.x = x; g.prep.x_is_compact = 0;
+            g.prep.x_batch_stride = (int64_t)req->ctx_len * d.hidden;
+            g.prep.anchor_idx = nullptr; g.prep.k = 0; g.prep.extra_rows = req->masked_pos; g.prep.e = req->n_masked;
+            g.prep.affix_start = req->affix_start; g.prep.affix_len = req->affix_len; g.prep.ctx_len = req->ctx_len;
+            g.prep.gain = w->attn_norm_g; g.prep.eps = d.rms_eps; g.prep.row_pos = mpos;
+            g.prep.row_src = wsp<int64_t>(ctx, ctx->o_mrow_src);
             g.b[0] = w->wq; g.n[0] = d.n_heads * d.head_dim;
             g.epilogue = kEpiQKV;
             g.bias[0] = d.qkv_bias ? w->bq : nullptr;
             g.row_pos = mpos; g.rope_cos = req->rope_cos; g.rope_sin = req->rope_sin;
             g.head_dim = d.head_dim; g.rope_segments = 1; g.out[0] = qmask; g.rows_per_req = req->n_masked;
             g.partial = wsp<float>(ctx, ctx->o_gemm); g.status = wsp<uint32_t>(ctx, ctx->o_status);
-            ctx->launches += launch_gemm(g, stream);
+            g.grid_bar = wsp<unsigned int>(ctx, ctx->o_gridbar);
+            { int nl = launch_gemm(g, stream); if (nl < 0) return check_cuda(ctx, "masked-row query projection") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "masked-row query projection launch failed") : ACACHE_ERR_CUDA;
+            ctx->launches += nl; }
         }
         mark(ctx, ACACHE_STAGE_SCORE, stream);
         // with a selection to follow, the ordered sum over heads is folded into the selection kernel

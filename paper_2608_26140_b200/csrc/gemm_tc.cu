@@ -1,20 +1,26 @@
 // C[M, N] = A[M, K] * B[N, K]^T (bf16 in, fp32 accumulate) on the 5th-generation tensor
 // cores for the projections of the selective recomputation (Section 3.3).
 //
-// Design for a weight-streaming GEMM with few rows (M = K anchors + request rows, often
-// <= 128) on 148 SMs:
-//   * work = (output tiles of 128 x 256) x (K blocks of 64); the flat list of
-//     (tile, k-block) iterations is cut into equal contiguous ranges, one per CTA, so every
-//     SM streams the same number of weight bytes whatever N and K are;
-//   * per CTA: one thread issues TMA loads of the A tile and the two 128-row halves of the
-//     B tile into a 4-stage shared-memory ring (128-byte swizzle), one thread issues
-//     tcgen05.mma (128 x 256 x 16) into a TMEM accumulator (two accumulators of 256 columns,
-//     so the next segment's MMAs overlap the previous segment's drain), four warps drain
-//     TMEM with tcgen05.ld and write fp32 partial tiles;
-//   * a second kernel sums the partial tiles of each output tile in a fixed order
-//     (bitwise reproducible) and applies the epilogue (gemm_epilogue.cuh).
-// Every mbarrier wait is bounded: on expiry the CTA raises kFlagWaitExpired in the status
-// word, stops issuing work, frees its TMEM and returns.
+// gemm_tc_kernel (at most one CTA per SM):
+//   phase 0 (optional)  gather the rows of R (or take compact rows) and RMSNorm them into the
+//                       A operand, then a grid-wide barrier
+//   phase 1             the contraction: work = (output tiles of 128 x 256) x (K blocks of 64),
+//                       the flat list of (tile, k-block) iterations cut into equal contiguous
+//                       ranges, one per CTA, so every SM streams the same number of weight
+//                       bytes whatever N and K are.  One thread issues TMA loads into a 4-stage
+//                       128-byte-swizzled ring (weights evict-first, activations evict-last in
+//                       L2), one thread issues tcgen05.mma (128 x 256 x 16) into one of two TMEM
+//                       accumulators, four warps drain TMEM with tcgen05.ld and write fp32
+//                       partial tiles
+// gemm_finish_kernel: sums the partial tiles of every output element in ascending CTA order
+//   (bitwise reproducible) and applies the epilogue: bias + RoPE + KV scatter, residual add,
+//   or SwiGLU.  It is a kernel of its own because it is bound by L2 latency and wants far
+//   more threads in flight than one CTA per SM provides (measured: fused into the contraction
+//   kernel behind a second grid barrier it was ~10 us slower per projection).
+//
+// Every wait (mbarrier or grid barrier) is bounded: on expiry the CTA raises kFlagWaitExpired
+// in the status word, stops issuing work, lets its in-flight copies land, frees its TMEM and
+// returns.  The grid never exceeds the SM count, so all CTAs are resident for the barrier.
 #include <cuda.h>
 
 #include <cstdio>
@@ -23,9 +29,9 @@
 #include <mutex>
 
 #include "common.cuh"
-#include "gemm_epilogue.cuh"
 #include "kernels.h"
 #include "launch.h"
+#include "rows.cuh"
 
 namespace acache {
 
@@ -33,23 +39,15 @@ constexpr int TC_BM = 128, TC_BN = 256, TC_BK = 64, TC_STAGES = 4;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;          // 16 KB
 constexpr int TC_HALF_BYTES = 128 * TC_BK * 2;         // 16 KB: one 128-row half of the B tile
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + 2 * TC_HALF_BYTES;
-constexpr int TC_THREADS = 192;                        // warp 0: TMA, warp 1: MMA, warps 2-5: drain
+constexpr int TC_THREADS = 384;                        // warp 0: TMA, warp 1: MMA, warps 2-5: drain; all 12 warps do phase 0
 constexpr int TC_SMEM = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int TC_SLOT_FLOATS = TC_BM * TC_BN;          // one fp32 partial tile
 constexpr uint32_t TC_WAIT_LIMIT = 1u << 22;
+constexpr uint32_t GRID_WAIT_LIMIT = 1u << 21;
 
 struct TcPlan {
     int m_tiles, n_tiles, KB, tiles, U, ctas, smax;
     int units;            // 128-row B halves over all segments (non-SwiGLU) or ffn/128 (SwiGLU)
-};
-
-struct TcArgs {
-    int M;
-    int swiglu;
-    int n[3];             // segment widths (non-SwiGLU)
-    TcPlan p;
-    float* partial;
-    uint32_t* status;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -85,11 +83,30 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+// L2 eviction policies: the weights stream through once (evict first); the activation rows
+// every CTA re-reads and the partial tiles the finish phase reads back should stay (evict last).
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                            uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
         : "memory");
+}
+__device__ __forceinline__ void st_hint_f4(float4* p, float4 v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
+                 ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy)
+                 : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -137,23 +154,191 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n) {
 }
 
 // Which weight matrix and row the 128-row half `h` of N tile `nt` starts at; -1 if past the end.
-__device__ __forceinline__ int half_source(const TcArgs& a, int nt, int h, int& row) {
-    if (a.swiglu) {
+__device__ __forceinline__ int half_source(const GemmArgs& g, const TcPlan& p, int nt, int h, int& row) {
+    if (g.epilogue == kEpiSwiGLU) {
         row = nt * 128;
         return h;                      // half 0: gate rows, half 1: up rows
     }
     int u = nt * 2 + h;
-    if (u >= a.p.units) return -1;
+    if (u >= p.units) return -1;
     int r = u * 128, seg = 0;
-    while (seg < 2 && r >= a.n[seg]) { r -= a.n[seg]; ++seg; }
+    while (seg < 2 && r >= g.n[seg]) { r -= g.n[seg]; ++seg; }
     row = r;
     return seg;
 }
 
+// Grid-wide barrier number `k` (1, 2, ...) of this launch on a pair of counters in global
+// memory: arrivals only ever add to bar[0], so barrier k is passed at k * gridDim.x.  Bounded;
+// returns false (and raises the CTA's abort flag) if the others do not arrive.
+__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int k, volatile int* abort_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0 && !*abort_flag) {
+        __threadfence();
+        atomicAdd(&bar[0], 1u);
+        const unsigned int target = k * gridDim.x;
+        bool ok = false;
+        for (uint32_t i = 0; i < GRID_WAIT_LIMIT; ++i) {
+            unsigned int v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
+            if (v >= target) { ok = true; break; }
+            __nanosleep(i < 64 ? 20 : 100);
+        }
+        if (!ok) *abort_flag = 1;
+        __threadfence();
+    }
+    __syncthreads();
+    return !*abort_flag;
+}
+
+__device__ __forceinline__ uint4 pack8(const float* v) {
+    return make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+
+// Ordered sums over the partial-tile slots of one row for 16 adjacent columns starting at column
+// group pc0 and, if pc1 >= 0, 16 more starting at pc1.  Loads are issued two slots at a time
+// for all eight column groups (16 independent 16-byte loads in flight per thread) and added in
+// slot order, which keeps the result bitwise reproducible.
+__device__ __forceinline__ void sum_slots16(const float4* __restrict__ src, int nslots, int pc0, int pc1, int row,
+                                            float (&lo)[16], float (&hi)[16]) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { lo[i] = 0.f; hi[i] = 0.f; }
+    const float4* q0 = src + pc0 * TC_BM + row;
+    const float4* q1 = src + (pc1 < 0 ? pc0 : pc1) * TC_BM + row;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c0 = 0; c0 < nslots; c0 += 2) {
+        float4 a[2][4], b[2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const bool in = c0 + i < nslots;
+            const int64_t so = (int64_t)(c0 + i) * (TC_SLOT_FLOATS / 4);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                a[i][j] = in ? __ldcg(q0 + so + j * TC_BM) : zero;
+                b[i][j] = (in && pc1 >= 0) ? __ldcg(q1 + so + j * TC_BM) : zero;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            if (c0 + i < nslots) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    lo[4 * j] += a[i][j].x; lo[4 * j + 1] += a[i][j].y; lo[4 * j + 2] += a[i][j].z; lo[4 * j + 3] += a[i][j].w;
+                    hi[4 * j] += b[i][j].x; hi[4 * j + 1] += b[i][j].y; hi[4 * j + 2] += b[i][j].z; hi[4 * j + 3] += b[i][j].w;
+                }
+            }
+        }
+    }
+}
+
+// Output columns per work item: 16 (a full 32-byte sector of bf16 per row, so no store is a
+// partial-sector write).  q/k/v items carry 16 columns of each rotary half.
+__host__ __device__ __forceinline__ int finish_items(int epilogue, int n_total) {
+    return epilogue == kEpiQKV ? n_total / 32 : n_total / 16;
+}
+
+// Epilogue of one work item of row `grow`.
+__device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, int item, int mt, int row) {
+    const int grow = mt * TC_BM + row;
+    int nt, pc0, pc1;            // N tile, first partial column group of each half
+    int u128 = 0, lo_col = 0;
+    const int half = g.head_dim >> 1;
+    if (g.epilogue == kEpiResidual) {
+        nt = item >> 4; pc0 = (item & 15) * 4; pc1 = -1;
+    } else if (g.epilogue == kEpiSwiGLU) {
+        nt = item >> 3; pc0 = (item & 7) * 4; pc1 = 32 + pc0;
+    } else {
+        u128 = item >> 2;
+        const int r = item & 3;
+        nt = u128 >> 1;
+        lo_col = g.head_dim == 128 ? 16 * r : 64 * (r >> 1) + 16 * (r & 1);   // column inside the 128-wide unit
+        pc0 = 32 * (u128 & 1) + (lo_col >> 2);
+        pc1 = pc0 + (half >> 2);
+    }
+    const int t = mt * p.n_tiles + nt;
+    const int c_first = (int)(((int64_t)t * p.KB) / p.U);
+    const int c_last = (int)(((int64_t)(t + 1) * p.KB - 1) / p.U);
+    const int nslots = c_last - c_first + 1;
+    const float4* src = reinterpret_cast<const float4*>(g.partial + (int64_t)t * p.smax * TC_SLOT_FLOATS);
+    // loads that do not depend on the sums go first so that they overlap the partial-tile reads
+    int pos = 0;
+    int64_t roff = 0;
+    if (g.epilogue == kEpiQKV) pos = __ldcg(g.row_pos + grow);
+    if (g.epilogue == kEpiResidual) roff = g.resid_off ? __ldcg(g.resid_off + grow) : (int64_t)grow * g.n[0];
+    float lo[16], hi[16];
+    sum_slots16(src, nslots, pc0, pc1, row, lo, hi);
+
+    if (g.epilogue == kEpiResidual) {
+        const int N = g.n[0], col = item * 16;
+        const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(g.resid) + roff + col);
+        const uint4 r0 = __ldcg(rp), r1 = __ldcg(rp + 1);
+        const uint32_t rw[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { lo[2 * i] += bf16_lo(rw[i]); lo[2 * i + 1] += bf16_hi(rw[i]); }
+        uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * N + col);
+        o[0] = pack8(lo);
+        o[1] = pack8(lo + 8);
+        return;
+    }
+    if (g.epilogue == kEpiSwiGLU) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) lo[i] = lo[i] / (1.f + __expf(-lo[i])) * hi[i];
+        uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * g.n[0] + item * 16);
+        o[0] = pack8(lo);
+        o[1] = pack8(lo + 8);
+        return;
+    }
+    // q/k/v: bias, rotary embedding with the pairing (i, i + d/2), store (+ fused cache scatter)
+    int seg = 0, c0 = u128 * 128;
+    while (seg < 2 && c0 >= g.n[seg]) { c0 -= g.n[seg]; ++seg; }
+    const int col = c0 + lo_col;                          // column inside the segment
+    const int j0 = lo_col & (half - 1);                   // index inside the half head
+    const __nv_bfloat16* bias = static_cast<const __nv_bfloat16*>(g.bias[seg]);
+    if (bias) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            lo[i] += __bfloat162float(bias[col + i]);
+            hi[i] += __bfloat162float(bias[col + half + i]);
+        }
+    }
+    if (seg < g.rope_segments) {
+        const int pp = pos < 0 ? 0 : pos;
+        const float4* cs = reinterpret_cast<const float4*>(g.rope_cos + (int64_t)pp * half + j0);
+        const float4* sn = reinterpret_cast<const float4*>(g.rope_sin + (int64_t)pp * half + j0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float4 c4 = cs[j], s4 = sn[j];
+            const float c[4] = {c4.x, c4.y, c4.z, c4.w}, sv[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float x = lo[4 * j + i], y = hi[4 * j + i];
+                lo[4 * j + i] = x * c[i] - y * sv[i];
+                hi[4 * j + i] = y * c[i] + x * sv[i];
+            }
+        }
+    }
+    const uint4 l0 = pack8(lo), l1 = pack8(lo + 8), h0 = pack8(hi), h1 = pack8(hi + 8);
+    const int nseg = g.n[seg];
+    if (g.out[seg]) {
+        __nv_bfloat16* o = static_cast<__nv_bfloat16*>(g.out[seg]) + (int64_t)grow * nseg + col;
+        reinterpret_cast<uint4*>(o)[0] = l0; reinterpret_cast<uint4*>(o)[1] = l1;
+        reinterpret_cast<uint4*>(o + half)[0] = h0; reinterpret_cast<uint4*>(o + half)[1] = h1;
+    }
+    __nv_bfloat16* cache = seg == 1 ? static_cast<__nv_bfloat16*>(g.cache_k)
+                         : seg == 2 ? static_cast<__nv_bfloat16*>(g.cache_v) : nullptr;
+    if (cache && pos >= 0) {
+        const int b = grow / g.rows_per_req;
+        __nv_bfloat16* o = cache + (int64_t)b * g.kv_batch_stride + (int64_t)pos * nseg + col;
+        reinterpret_cast<uint4*>(o)[0] = l0; reinterpret_cast<uint4*>(o)[1] = l1;
+        reinterpret_cast<uint4*>(o + half)[0] = h0; reinterpret_cast<uint4*>(o + half)[1] = h1;
+    }
+}
+
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB0,
-               const __grid_constant__ CUtensorMap mapB1, const __grid_constant__ CUtensorMap mapB2) {
+gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtensorMap mapA,
+               const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
+               const __grid_constant__ CUtensorMap mapB2) {
     extern __shared__ unsigned char smem_raw[];
+    __shared__ float red[TC_THREADS / 32];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bars = base + TC_STAGES * TC_STAGE_BYTES;
@@ -164,6 +349,7 @@ gemm_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap mapA, const _
     auto tfull_bar = [&](int i) { return bars + 8 * (2 * TC_STAGES + i); };
     auto tempty_bar = [&](int i) { return bars + 8 * (2 * TC_STAGES + 2 + i); };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    unsigned int nbar = 0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -184,45 +370,73 @@ gemm_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap mapA, const _
     pdl_wait();
     pdl_launch_dependents();
 
-    const TcPlan& p = a.p;
+    // ---------------- phase 0: gather the rows of R and RMSNorm them into A ----------------
+    if (g.prep.enabled) {
+        const RowPrep& rp = g.prep;
+        const int rows_per_req = rp.k + rp.e;
+        for (int row = blockIdx.x; row < g.M; row += gridDim.x) {
+            int64_t src = (int64_t)row * g.K;
+            if (rp.enabled == 1) {       // rows of R: position from the anchor / extra-row lists
+                const int b = row / rows_per_req, i = row - b * rows_per_req;
+                const int pos = row_position(rp.anchor_idx, rp.k, rp.extra_rows, rp.e, b, i, rp.affix_start,
+                                             rp.affix_len, rp.ctx_len);
+                if (!rp.x_is_compact) src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
+                if (threadIdx.x == 0) {
+                    rp.row_pos[row] = pos;
+                    rp.row_src[row] = src;
+                    if (pos < 0) atomicOr(g.status, kFlagBadIndex);
+                }
+            }
+            rmsnorm_row(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(rp.x) + src),
+                        reinterpret_cast<const uint4*>(rp.gain),
+                        reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(const_cast<void*>(g.a)) + (int64_t)row * g.K),
+                        g.K, rp.eps, red);
+        }
+        asm volatile("fence.proxy.async;" ::: "memory");   // the rows are read back through TMA
+        grid_barrier(g.grid_bar, ++nbar, abort_flag);
+        asm volatile("fence.proxy.async;" ::: "memory");
+    }
+
+    // ---------------- phase 1: the contraction ----------------
     const int it0 = blockIdx.x * p.U;
     const int it1 = min(it0 + p.U, p.tiles * p.KB);
 
     if (warp == 0 && lane == 0) {
-        // ---------------- TMA producer ----------------
+        // TMA producer
         const CUtensorMap* maps[3] = {&mapB0, &mapB1, &mapB2};
         int stage = 0;
         uint32_t phase = 0;
-        bool ok = true;
+        bool ok = !*abort_flag;
+        const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
         for (int it = it0; it < it1 && ok;) {
             const int t = it / p.KB, kb0 = it - t * p.KB;
             const int kb1 = min(p.KB, kb0 + (it1 - it));
             const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
             int row0, row1;
-            const int s0 = half_source(a, nt, 0, row0), s1 = half_source(a, nt, 1, row1);
+            const int s0 = half_source(g, p, nt, 0, row0), s1 = half_source(g, p, nt, 1, row1);
             const uint32_t bytes = TC_A_BYTES + TC_HALF_BYTES * (1 + (s1 >= 0));
             for (int kb = kb0; kb < kb1; ++kb) {
                 if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag))) break;
                 const uint32_t sA = base + stage * TC_STAGE_BYTES, sB = sA + TC_A_BYTES;
                 mbar_expect_tx(full_bar(stage), bytes);
-                tma_load_2d(sA, &mapA, kb * TC_BK, mt * TC_BM, full_bar(stage));
-                tma_load_2d(sB, maps[s0], kb * TC_BK, row0, full_bar(stage));
-                if (s1 >= 0) tma_load_2d(sB + TC_HALF_BYTES, maps[s1], kb * TC_BK, row1, full_bar(stage));
+                tma_load_2d(sA, &mapA, kb * TC_BK, mt * TC_BM, full_bar(stage), pol_a);
+                tma_load_2d(sB, maps[s0], kb * TC_BK, row0, full_bar(stage), pol_w);
+                if (s1 >= 0) tma_load_2d(sB + TC_HALF_BYTES, maps[s1], kb * TC_BK, row1, full_bar(stage), pol_w);
                 if (++stage == TC_STAGES) { stage = 0; phase ^= 1; }
             }
             it += kb1 - kb0;
         }
     } else if (warp == 1 && lane == 0) {
-        // ---------------- MMA issuer ----------------
+        // MMA issuer
         int stage = 0, acc = 0;
         uint32_t phase = 0, acc_phase = 0;
-        bool ok = true;
+        bool ok = !*abort_flag;
         for (int it = it0; it < it1 && ok;) {
             const int t = it / p.KB, kb0 = it - t * p.KB;
             const int kb1 = min(p.KB, kb0 + (it1 - it));
             const int nt = t % p.n_tiles;
             int row1;
-            const uint32_t idesc = idesc_bf16(half_source(a, nt, 1, row1) >= 0 ? 256 : 128);
+            const uint32_t idesc = idesc_bf16(half_source(g, p, nt, 1, row1) >= 0 ? 256 : 128);
             if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag))) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * TC_BN;
@@ -242,31 +456,32 @@ gemm_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap mapA, const _
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             it += kb1 - kb0;
         }
-    } else if (warp >= 2) {
-        // ---------------- drain: TMEM -> fp32 partial tile ----------------
+    } else if (warp >= 2 && warp < 6) {
+        // drain: TMEM -> fp32 partial tile, layout [column / 4][row][4]
         const int q = warp & 3;                   // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
         int acc = 0;
         uint32_t acc_phase = 0;
-        bool ok = true;
+        bool ok = !*abort_flag;
+        const uint64_t pol_p = policy_evict_last();
         for (int it = it0; it < it1 && ok;) {
             const int t = it / p.KB, kb0 = it - t * p.KB;
             const int kb1 = min(p.KB, kb0 + (it1 - it));
             const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
             int row1;
-            const int nchunks = half_source(a, nt, 1, row1) >= 0 ? 8 : 4;
+            const int nchunks = half_source(g, p, nt, 1, row1) >= 0 ? 8 : 4;
             const int slot = blockIdx.x - (int)(((int64_t)t * p.KB) / p.U);
-            float4* dst = reinterpret_cast<float4*>(a.partial + ((int64_t)t * p.smax + slot) * TC_SLOT_FLOATS);
+            float4* dst = reinterpret_cast<float4*>(g.partial + ((int64_t)t * p.smax + slot) * TC_SLOT_FLOATS);
             if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) break;
             tc_fence_after();
-            const bool valid = mt * TC_BM + row < a.M;
+            const bool valid = mt * TC_BM + row < g.M;
             for (int c = 0; c < nchunks; ++c) {
                 float v[32];
                 tc_ld32(tmem_base + acc * TC_BN + c * 32 + ((uint32_t)(q * 32) << 16), v);
                 if (valid) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        dst[(c * 8 + i) * TC_BM + row] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        st_hint_f4(&dst[(c * 8 + i) * TC_BM + row], make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]), pol_p);
                 }
             }
             tc_fence_before();
@@ -276,15 +491,24 @@ gemm_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap mapA, const _
             it += kb1 - kb0;
         }
     }
-    // ---------------- teardown ----------------
     tc_fence_before();
+    __syncthreads();
+    // ---------------- teardown ----------------
     __syncthreads();
     if (*abort_flag) {
         if (threadIdx.x == 0) {
-            atomicOr(a.status, kFlagWaitExpired);
+            atomicOr(g.status, kFlagWaitExpired);
             for (int i = 0; i < 4096; ++i) __nanosleep(64);   // let copies already in flight land
         }
         __syncthreads();
+    } else if (threadIdx.x == 0 && nbar > 0) {
+        // the last CTA to leave re-arms the barrier words for the next launch
+        __threadfence();
+        if (atomicAdd(&g.grid_bar[1], 1u) == gridDim.x - 1) {
+            g.grid_bar[0] = 0u;
+            __threadfence();
+            g.grid_bar[1] = 0u;
+        }
     }
     if (warp == 1) {
         tc_fence_after();
@@ -292,120 +516,17 @@ gemm_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap mapA, const _
     }
 }
 
-// ---- finish: ordered sum of the partial tiles + epilogue --------------------------------------
-// One thread owns 4 adjacent output columns of one row (plus the 4 columns its epilogue pairs
-// them with: the other rotary half, or the up-projection of a gate column).  A warp covers 32
-// consecutive rows of the same columns, so every partial-tile read is one contiguous 512-byte
-// segment; the slots are summed in ascending CTA order, which makes the result bitwise
-// reproducible.
-constexpr int FIN_ITEMS_PER_SUB = 2;   // items each half-block of 128 threads walks through
-
-__device__ __forceinline__ float4 sum_slots(const float4* __restrict__ src, int nslots, int pc, int row) {
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    const float4* q = src + pc * TC_BM + row;
-#pragma unroll 4
-    for (int c = 0; c < nslots; ++c) {
-        const float4 v = __ldcg(q + (int64_t)c * (TC_SLOT_FLOATS / 4));
-        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-    }
-    return s;
-}
-
-__device__ __forceinline__ uint2 pack4(float a, float b, float c, float d) {
-    return make_uint2(pack_bf16(a, b), pack_bf16(c, d));
-}
-
-__global__ void __launch_bounds__(256) gemm_finish_kernel(const GemmArgs g, const TcPlan p, const float* __restrict__ partial,
-                                                          int n_items) {
+__global__ void __launch_bounds__(256) gemm_finish_kernel(const GemmArgs g, const TcPlan p, int n_items) {
     pdl_wait();
     pdl_launch_dependents();
-    const int row = threadIdx.x & 127, sub = threadIdx.x >> 7;
-    const int mt = blockIdx.y, grow = mt * TC_BM + row;
-    if (grow >= g.M) return;
-    for (int k = 0; k < FIN_ITEMS_PER_SUB; ++k) {
-        const int item = (blockIdx.x * 2 + sub) * FIN_ITEMS_PER_SUB + k;
-        if (item >= n_items) return;
-        int nt, pc0, pc1;            // N tile, partial column groups of the two halves
-        int u128 = 0, r = 0;
-        if (g.epilogue == kEpiResidual) {
-            nt = item >> 6; pc0 = item & 63; pc1 = -1;
-        } else if (g.epilogue == kEpiSwiGLU) {
-            nt = item >> 5; pc0 = item & 31; pc1 = 32 + pc0;
-        } else {
-            u128 = item >> 4; r = item & 15;
-            nt = u128 >> 1;
-            const int c4 = g.head_dim == 128 ? r : ((r >> 3) << 4) + (r & 7);
-            pc0 = 32 * (u128 & 1) + c4;
-            pc1 = pc0 + (g.head_dim >> 3);
-        }
-        const int t = mt * p.n_tiles + nt;
-        const int c_first = (int)(((int64_t)t * p.KB) / p.U);
-        const int c_last = (int)(((int64_t)(t + 1) * p.KB - 1) / p.U);
-        const int nslots = c_last - c_first + 1;
-        const float4* src = reinterpret_cast<const float4*>(partial + (int64_t)t * p.smax * TC_SLOT_FLOATS);
-        const float4 v0 = sum_slots(src, nslots, pc0, row);
-        if (g.epilogue == kEpiResidual) {
-            const int N = g.n[0], col = item * 4;
-            const int64_t roff = g.resid_off ? g.resid_off[grow] : (int64_t)grow * N;
-            const uint2 rv = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(g.resid) + roff + col);
-            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * N + col) =
-                pack4(v0.x + bf16_lo(rv.x), v0.y + bf16_hi(rv.x), v0.z + bf16_lo(rv.y), v0.w + bf16_hi(rv.y));
-            continue;
-        }
-        const float4 v1 = sum_slots(src, nslots, pc1, row);
-        if (g.epilogue == kEpiSwiGLU) {
-            const float gt[4] = {v0.x, v0.y, v0.z, v0.w}, up[4] = {v1.x, v1.y, v1.z, v1.w};
-            float o[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) o[i] = gt[i] / (1.f + __expf(-gt[i])) * up[i];
-            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * g.n[0] + item * 4) =
-                pack4(o[0], o[1], o[2], o[3]);
-            continue;
-        }
-        // q/k/v: bias, rotary embedding with the pairing (i, i + d/2), store (+ fused cache scatter)
-        int seg = 0, c0 = u128 * 128;
-        while (seg < 2 && c0 >= g.n[seg]) { c0 -= g.n[seg]; ++seg; }
-        const int half = g.head_dim >> 1;
-        const int j4 = (g.head_dim == 128 ? r : (r & 7)) * 4;               // index inside the half head
-        const int col = c0 + (g.head_dim == 128 ? r * 4 : ((r >> 3) << 6) + (r & 7) * 4);
-        float lo[4] = {v0.x, v0.y, v0.z, v0.w}, hi[4] = {v1.x, v1.y, v1.z, v1.w};
-        const __nv_bfloat16* bias = static_cast<const __nv_bfloat16*>(g.bias[seg]);
-        if (bias) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                lo[i] += __bfloat162float(bias[col + i]);
-                hi[i] += __bfloat162float(bias[col + half + i]);
-            }
-        }
-        const int pos = g.row_pos[grow];
-        if (seg < g.rope_segments) {
-            const int pp = pos < 0 ? 0 : pos;
-            const float4 cs = *reinterpret_cast<const float4*>(g.rope_cos + (int64_t)pp * half + j4);
-            const float4 sn = *reinterpret_cast<const float4*>(g.rope_sin + (int64_t)pp * half + j4);
-            const float c[4] = {cs.x, cs.y, cs.z, cs.w}, sv[4] = {sn.x, sn.y, sn.z, sn.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float x = lo[i], y = hi[i];
-                lo[i] = x * c[i] - y * sv[i];
-                hi[i] = y * c[i] + x * sv[i];
-            }
-        }
-        const uint2 plo = pack4(lo[0], lo[1], lo[2], lo[3]), phi = pack4(hi[0], hi[1], hi[2], hi[3]);
-        const int nseg = g.n[seg];
-        if (g.out[seg]) {
-            __nv_bfloat16* o = static_cast<__nv_bfloat16*>(g.out[seg]) + (int64_t)grow * nseg + col;
-            *reinterpret_cast<uint2*>(o) = plo;
-            *reinterpret_cast<uint2*>(o + half) = phi;
-        }
-        __nv_bfloat16* cache = seg == 1 ? static_cast<__nv_bfloat16*>(g.cache_k)
-                             : seg == 2 ? static_cast<__nv_bfloat16*>(g.cache_v) : nullptr;
-        if (cache && pos >= 0) {
-            const int b = grow / g.rows_per_req;
-            __nv_bfloat16* o = cache + (int64_t)b * g.kv_batch_stride + (int64_t)pos * nseg + col;
-            *reinterpret_cast<uint2*>(o) = plo;
-            *reinterpret_cast<uint2*>(o + half) = phi;
-        }
-    }
+    const int rows_per = p.m_tiles == 1 ? ((g.M + 31) & ~31) : TC_BM;
+    const int64_t work = (int64_t)n_items * p.m_tiles * rows_per;
+    const int64_t w = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (w >= work) return;
+    const int row = (int)(w % rows_per);
+    const int64_t s = w / rows_per;
+    const int item = (int)(s % n_items), mt = (int)(s / n_items);
+    if (mt * TC_BM + row < g.M) finish_item(g, p, item, mt, row);
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -485,24 +606,16 @@ TcPlan make_plan(int M, int K, int units, bool swiglu) {
 
 size_t gemm_partial_bytes(int M, int K, int n_total, bool swiglu) {
     if (M <= 0) return 0;
-    TcPlan p = make_plan(M, K, swiglu ? n_total / 128 : n_total / 128, swiglu);
+    TcPlan p = make_plan(M, K, n_total / 128, swiglu);
     return (size_t)p.tiles * p.smax * TC_SLOT_FLOATS * sizeof(float);
 }
 
 int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
     if (g.M == 0) return 0;
-    static const bool use_mma = [] { const char* e = getenv("ACACHE_GEMM_IMPL"); return e && !strcmp(e, "mma"); }();
-    if (use_mma) return launch_gemm_mma(g, stream);
-    std::lock_guard<std::mutex> lock(g_map_mutex);
     const bool swiglu = g.epilogue == kEpiSwiGLU;
     const int n_total = swiglu ? g.n[0] : g.n[0] + g.n[1] + g.n[2];
-    TcArgs a{};
-    a.M = g.M;
-    a.swiglu = swiglu;
-    a.n[0] = g.n[0]; a.n[1] = g.n[1]; a.n[2] = g.n[2];
-    a.p = make_plan(g.M, g.K, n_total / 128, swiglu);
-    a.partial = g.partial;
-    a.status = g.status;
+    const TcPlan p = make_plan(g.M, g.K, n_total / 128, swiglu);
+    std::lock_guard<std::mutex> lock(g_map_mutex);
     const CUtensorMap* mA = get_map(g.a, g.M, g.K);
     const CUtensorMap* mB[3] = {nullptr, nullptr, nullptr};
     for (int i = 0; i < 3; ++i)
@@ -515,11 +628,17 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
         cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
         attr = true;
     }
-    launch_pdl(gemm_tc_kernel, a.p.ctas, TC_THREADS, TC_SMEM, stream, a, *mA, *mB[0], *mB[1], *mB[2]);
-    const int n_items = g.epilogue == kEpiQKV ? n_total / 8 : n_total / 4;
-    const int per_cta = 2 * FIN_ITEMS_PER_SUB;
-    launch_pdl(gemm_finish_kernel, dim3((n_items + per_cta - 1) / per_cta, a.p.m_tiles), 256, 0, stream, g, a.p,
-               (const float*)g.partial, n_items);
+    // a plain launch: a cooperative one measured ~2.5 us slower and cannot overlap the previous
+    // kernel's tail; the grid never exceeds the SM count at one CTA per SM and the barrier is bounded
+    if (launch_pdl(gemm_tc_kernel, dim3(p.ctas), dim3(TC_THREADS), TC_SMEM, stream, g, p, *mA, *mB[0], *mB[1], *mB[2]) !=
+        cudaSuccess)
+        return -1;
+    const int n_items = finish_items(g.epilogue, n_total);
+    const int rows_per = p.m_tiles == 1 ? ((g.M + 31) & ~31) : TC_BM;
+    const int64_t work = (int64_t)n_items * p.m_tiles * rows_per;
+    if (launch_pdl(gemm_finish_kernel, dim3((unsigned)((work + 255) / 256)), dim3(256), 0, stream, g, p, n_items) !=
+        cudaSuccess)
+        return -1;
     return 2;
 }
 

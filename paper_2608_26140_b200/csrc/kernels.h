@@ -6,21 +6,6 @@
 namespace acache {
 
 // ---- rows.cu ----------------------------------------------------------------------------
-// Row plan of the recompute set R and RMSNorm of the gathered rows.
-// Row i of request b (i < k: anchor, else extra) sits at absolute position pos.
-// Writes row_pos[b*(k+e)+i] = pos (or -1 for an out-of-range index, which also sets
-// kFlagBadIndex), row_src = element offset of the row inside x, and
-// xn = bf16(x * rsqrt(mean(x^2)+eps) * g).
-void launch_gather_rmsnorm(const void* x, int x_is_compact, int64_t x_batch_stride, int hidden,
-                           const int32_t* anchor_idx, int k, const int32_t* extra_rows, int e,
-                           int batch, int affix_start, int affix_len, int ctx_len,
-                           const void* gain, float eps, int32_t* row_pos, int64_t* row_src, void* xn,
-                           uint32_t* status, cudaStream_t stream);
-
-// xn = bf16(RMSNorm(x) * g) for compact rows [n, hidden].
-void launch_rmsnorm(const void* x, const void* gain, float eps, int n, int hidden, void* xn,
-                    cudaStream_t stream);
-
 // cache[b, pos_r] = new[b, r] for K and V; rows with an invalid position are skipped.
 void launch_scatter_kv(void* cache_k, void* cache_v, int64_t batch_stride, int ctx_len,
                        const int32_t* anchor_idx, int k, const int32_t* extra_rows, int e, int batch,
@@ -61,6 +46,26 @@ enum GemmEpilogue : int {
     kEpiSwiGLU,      // out = bf16(silu(gate) * up), B tile = 64 gate rows + 64 up rows
 };
 
+// Row plan of the recompute set R and RMSNorm of the gathered rows, run in front of a GEMM:
+// row i of request b (i < k: anchor, else extra) sits at absolute position pos; writes
+// row_pos[b*(k+e)+i] = pos (-1 for an out-of-range index, which also raises kFlagBadIndex),
+// row_src = element offset of the row inside x, and the GEMM's A rows
+// xn = bf16(x * rsqrt(mean(x^2) + eps) * g).
+struct RowPrep {
+    int enabled;              // 0: off, 1: gather the rows of R, 2: the rows of x as they are (compact)
+    const void* x;            // bf16 [B, ctx_len, hidden] or compact [B, k+e, hidden]
+    int x_is_compact;
+    int64_t x_batch_stride;
+    const int32_t* anchor_idx;
+    int k;
+    const int32_t* extra_rows;
+    int e;
+    int affix_start, affix_len, ctx_len;
+    const void* gain;
+    float eps;
+    int32_t* row_pos;
+    int64_t* row_src;
+};
 struct GemmArgs {
     const void* a;            // bf16 [M, K] row-major, lda = K
     int M, K;
@@ -85,15 +90,17 @@ struct GemmArgs {
     const int64_t* resid_off; // [M] element offset of the residual row, or null => row * N
     // --- kEpiSwiGLU / kEpiResidual output ---
     void* c;                  // bf16 [M, Nout]
+    // --- row work fused in front of the contraction ---
+    RowPrep prep;             // writes the A rows (a) before the contraction
     // --- scratch ---
     float* partial;           // fp32 partial tiles, gemm_partial_bytes() of them
     uint32_t* status;         // device status word
+    unsigned int* grid_bar;   // two zero-initialised words for the kernel's grid barriers
 };
 // Bytes of fp32 partial-tile scratch a GEMM of M rows, reduction length K and n_total output
 // columns (SwiGLU: the MLP width) needs.
 size_t gemm_partial_bytes(int M, int K, int n_total, bool swiglu);
-int launch_gemm(const GemmArgs& g, cudaStream_t stream);      // tcgen05 main loop + finish kernel
-int launch_gemm_mma(const GemmArgs& g, cudaStream_t stream);  // legacy mma.sync main loop (debug aid)
+int launch_gemm(const GemmArgs& g, cudaStream_t stream);      // kernels launched, or -1 if a launch failed
 
 // ---- attn.cu ----------------------------------------------------------------------------
 struct AttnArgs {

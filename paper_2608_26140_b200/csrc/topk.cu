@@ -67,7 +67,16 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(float* scores, int L
     if (head_partial) {   // Eq. 5: ordered sum over heads, fused in front of the selection
         for (int j = tid; j < L; j += kTopkThreads) {
             float v = 0.f;
-            for (int h = 0; h < n_heads; ++h) v += head_partial[((int64_t)b * n_heads + h) * L + j];
+            const float* hp = head_partial + (int64_t)b * n_heads * L + j;
+            int h = 0;
+            for (; h + 8 <= n_heads; h += 8) {      // 8 loads in flight, added in head order
+                float t[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) t[i] = __ldcg(hp + (int64_t)(h + i) * L);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v += t[i];
+            }
+            for (; h < n_heads; ++h) v += __ldcg(hp + (int64_t)h * L);
             s[j] = accumulate ? s[j] + v : v;
         }
         __syncthreads();
