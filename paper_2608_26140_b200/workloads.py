@@ -293,10 +293,12 @@ class Case:
 
 
 def make_case(shape: LayerShape, lay: Layout, ratio: float, cfg_id: int = 0, layer: int = 0,
-              with_stale_hidden: bool = False, hot_frac: float = 0.0) -> Case:
-    """One single-layer case with a randomly drawn (stale) cache."""
+              with_stale_hidden: bool = False, hot_frac: float = 0.0,
+              weights: Optional[Dict[str, Optional[np.ndarray]]] = None) -> Case:
+    """One single-layer case with a randomly drawn (stale) cache.  ``weights`` reuses an
+    earlier ``layer_weights`` draw (they depend only on shape, cfg_id and layer)."""
     base = SEED_BASE + 4096 * cfg_id + 64 * layer
-    w = layer_weights(shape, cfg_id, layer)
+    w = weights if weights is not None else layer_weights(shape, cfg_id, layer)
     x = hidden_states(shape, lay, base + 20, base + 21)
     xs = hidden_states(shape, lay, base + 20, base + 22) if with_stale_hidden else None
     ck, cv = random_kv_cache(shape, lay, base + 30, hot_frac=hot_frac)

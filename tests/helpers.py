@@ -2,6 +2,8 @@
 the C-ABI calls through the binding, and compare with the CPU oracle."""
 from __future__ import annotations
 
+import functools
+
 import numpy as np
 import torch
 
@@ -11,6 +13,12 @@ from paper_2608_26140_b200 import workloads as wl
 
 DEV = "cuda:0"
 TOL = 2e-2     # max relative error of refreshed K/V and layer outputs (bf16 storage, fp32 accumulate)
+
+
+@functools.lru_cache(maxsize=2)
+def cached_weights(shape, cfg_id):
+    """Layer weights of (shape, cfg_id), drawn once per test session (read-only)."""
+    return wl.layer_weights(shape, cfg_id, 0)
 
 
 class DeviceCase:
