@@ -230,7 +230,9 @@ acache_status acache_scatter_kv(acache_ctx *ctx, const acache_request *req, acac
  * scatter fused into the QKV projection and attention reading the updated cache
  * (store-then-attend, Appendix C.1).  Gives the same cache and (within rounding of
  * the attention tiling) the same y as the three split calls in sequence.
- *   flags & ACACHE_F_SCORE : x must be the full [B, ctx_len, D] input; scores is written.
+ *   flags & ACACHE_F_SCORE : scores is written.  With a compact x the masked positions must be
+ *                            among extra_rows (their rows are looked up there); a masked position
+ *                            that is not raises ACACHE_FLAG_BAD_INDEX.
  *   flags & ACACHE_F_SELECT: anchor_idx [B, K] is written, K = acache_k_from_ratio(L, ratio);
  *                            otherwise anchor_idx is an input with that K.
  * scores: DEVICE fp32 [B, L] (may be NULL without F_SCORE/F_SELECT).

@@ -351,6 +351,63 @@ def dense_layer(weights, shape, x: np.ndarray, cos, sin, round_storage: bool = T
 
 
 # --------------------------------------------------------------------------
+# N layers: the one-shot probe of Section 3.2 and the refresh pass of Section 3.3
+# --------------------------------------------------------------------------
+def probe_forward(layers, shape, x0: np.ndarray, caches, ctx_len: int, affix_start: int, affix_len: int,
+                  masked_pos: np.ndarray, probe_rows: np.ndarray, cos, sin, norm_full: bool = False,
+                  round_storage: bool = True):
+    """One-shot probe (Section 3.2): forward only the non-affix rows P through all N layers with the
+    precomputed affix cache as fixed past KV; at every layer score the affix keys by the attention
+    they receive from the masked rows and sum over layers (Eq. 5).
+
+    layers: list of weight dicts; x0 [T, D] bf16 bits (layer-0 input); caches: list of
+    (cache_k, cache_v) bf16 bits per layer; probe_rows: absolute positions P (must contain masked_pos).
+    The scores of layer n use that layer's cache as it is before the probe writes its own rows.
+    Returns (scores fp64 [L], list of working caches, list of per-layer outputs y [|P|, D]).
+    """
+    rows = np.asarray(probe_rows, dtype=np.int64)
+    where = {int(p): i for i, p in enumerate(rows)}
+    mask_idx = np.array([where[int(p)] for p in masked_pos], dtype=np.int64)
+    x_rows = bf16_bits_to_f64(x0)[rows]
+    s = np.zeros(affix_len, F64)
+    out_caches, ys = [], []
+    for W, (ck, cv) in zip(layers, caches):
+        r = recompute_rows(W, shape, x_rows, rows, ck, cv, ctx_len, cos, sin, round_storage)
+        Kall = bf16_bits_to_f64(ck[:ctx_len])
+        s += score_anchors(r["q"][mask_idx], Kall[affix_start:affix_start + affix_len], Kall, affix_start, norm_full)
+        x_rows = r["y"]
+        out_caches.append((r["cache_k"], r["cache_v"]))
+        ys.append(r["y"])
+    return s, out_caches, ys
+
+
+def refresh_forward(layers, shape, x0: np.ndarray, caches, ctx_len: int, affix_start: int,
+                    anchor_idx: np.ndarray, extra_rows: np.ndarray, cos, sin, round_storage: bool = True):
+    """Refresh pass (Section 3.3): recompute the anchors and the request rows through all N layers;
+    layer n+1's input rows are layer n's output rows.  Returns (rows, working caches, per-layer y)."""
+    rows = recompute_set(anchor_idx, affix_start, extra_rows)
+    x_rows = bf16_bits_to_f64(x0)[rows]
+    out_caches, ys = [], []
+    for W, (ck, cv) in zip(layers, caches):
+        r = recompute_rows(W, shape, x_rows, rows, ck, cv, ctx_len, cos, sin, round_storage)
+        x_rows = r["y"]
+        out_caches.append((r["cache_k"], r["cache_v"]))
+        ys.append(r["y"])
+    return rows, out_caches, ys
+
+
+def dense_forward(layers, shape, x0: np.ndarray, cos, sin, round_storage: bool = True):
+    """All positions through all N layers (the full-recompute end point); returns per-layer (y, K, V)."""
+    x = x0
+    outs = []
+    for W in layers:
+        y, kb, vb = dense_layer(W, shape, x, cos, sin, round_storage)
+        outs.append((y, kb, vb))
+        x = f64_to_bf16_bits(y)
+    return outs
+
+
+# --------------------------------------------------------------------------
 # comparison helpers used by the parity tests
 # --------------------------------------------------------------------------
 def rel_err_gate(a: np.ndarray, b: np.ndarray, tol: float = 2e-2) -> Tuple[bool, float]:

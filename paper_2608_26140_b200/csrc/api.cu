@@ -22,7 +22,7 @@ struct acache_ctx {
     // workspace offsets (bytes)
     size_t o_status, o_row_pos, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
     size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
-    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar;
+    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar, o_mcidx;
     std::string err;
     uint64_t launches = 0;
     // optional per-stage timing (acache_stage_timing)
@@ -254,6 +254,7 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
     c->o_vnew = take(cur, nr * kvd * 2);
     c->o_mrow_pos = take(cur, nm * 4);
     c->o_mrow_src = take(cur, nm * 8);
+    c->o_mcidx = take(cur, nm * 4);
     c->o_xn_mask = take(cur, nm * d.hidden * 2);
     c->o_qmask = take(cur, nm * qd * 2);
     c->o_stats = take(cur, (size_t)d.max_batch * d.n_heads * score_num_splits(d.max_ctx) * d.max_masked * 8);
@@ -421,7 +422,6 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
     const bool do_recompute = !(flags & ACACHE_F_NO_RECOMPUTE);
     if ((s = check_weights(ctx, w, !do_recompute)) != ACACHE_OK) return s;
     if (!x || !aligned16(x)) return fail(ctx, ACACHE_ERR_INVALID_ARG, "x NULL or misaligned");
-    if (do_score && x_is_compact) return fail(ctx, ACACHE_ERR_INVALID_ARG, "scoring needs the full [B, ctx_len, D] input");
     if ((do_score || do_select) && !scores) return fail(ctx, ACACHE_ERR_INVALID_ARG, "scores is NULL");
     if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
     if (do_recompute && req->batch * (k + req->n_extra) > 0 && (!y || !aligned16(y))) return fail(ctx, ACACHE_ERR_INVALID_ARG, "y NULL or misaligned");
@@ -436,7 +436,16 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
             void* xnm = wsp<void>(ctx, ctx->o_xn_mask);
             GemmArgs g{};
             g.a = xnm; g.M = req->batch * req->n_masked; g.K = d.hidden;
-            g.prep.enabled = 1; g.prep.x = x; g.prep.x_is_compact = 0;
+            g.prep.enabled = 1; g.prep.x = x; g.prep.x_is_compact = x_is_compact;
+            if (x_is_compact) {
+                // the masked rows are among the extra rows of the compact input: find where
+                int32_t* cidx = wsp<int32_t>(ctx, ctx->o_mcidx);
+                launch_match_rows(req->masked_pos, req->n_masked, req->extra_rows, req->n_extra, k, req->batch, cidx,
+                                  wsp<uint32_t>(ctx, ctx->o_status), stream);
+                ctx->launches += 1;
+                g.prep.compact_idx = cidx;
+                g.prep.compact_rows = k + req->n_extra;
+            }
             g.prep.x_batch_stride = (int64_t)req->ctx_len * d.hidden;
             g.prep.anchor_idx = nullptr; g.prep.k = 0; g.prep.extra_rows = req->masked_pos; g.prep.e = req->n_masked;
             g.prep.affix_start = req->affix_start; g.prep.affix_len = req->affix_len; g.prep.ctx_len = req->ctx_len;

@@ -380,7 +380,12 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
                 const int b = row / rows_per_req, i = row - b * rows_per_req;
                 const int pos = row_position(rp.anchor_idx, rp.k, rp.extra_rows, rp.e, b, i, rp.affix_start,
                                              rp.affix_len, rp.ctx_len);
-                if (!rp.x_is_compact) src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
+                if (!rp.x_is_compact) {
+                    src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
+                } else if (rp.compact_idx) {
+                    const int ci = rp.compact_idx[row];
+                    src = ((int64_t)b * rp.compact_rows + (ci < 0 ? 0 : ci)) * g.K;
+                }
                 if (threadIdx.x == 0) {
                     rp.row_pos[row] = pos;
                     rp.row_src[row] = src;

@@ -12,6 +12,10 @@ void launch_scatter_kv(void* cache_k, void* cache_v, int64_t batch_stride, int c
                        int affix_start, int affix_len, int kv_dim, const void* k_new, const void* v_new,
                        uint32_t* status, cudaStream_t stream);
 
+// idx[b, i] = compact row (k + j) whose position extra_rows[b, j] equals masked_pos[b, i], or -1.
+void launch_match_rows(const int32_t* masked_pos, int m, const int32_t* extra_rows, int e, int k, int batch,
+                       int32_t* idx, uint32_t* status, cudaStream_t stream);
+
 // slot[b, t] = compact row index whose fresh K/V replaces position t, or -1.
 void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
                            cudaStream_t stream);
@@ -56,6 +60,8 @@ struct RowPrep {
     const void* x;            // bf16 [B, ctx_len, hidden] or compact [B, k+e, hidden]
     int x_is_compact;
     int64_t x_batch_stride;
+    const int32_t* compact_idx;  // optional [B, k+e]: row i reads compact row compact_idx[..] of its request
+    int compact_rows;            // rows per request of the compact x that compact_idx points into
     const int32_t* anchor_idx;
     int k;
     const int32_t* extra_rows;

@@ -51,6 +51,32 @@ __global__ void __launch_bounds__(1024) slot_map_kernel(int32_t* __restrict__ sl
     }
 }
 
+// idx[b, i] = k + j where extra_rows[b, j] == masked_pos[b, i]: the compact row that holds a
+// masked position when the layer input is given in compact row order; -1 (and kFlagBadIndex)
+// if the position is not among the extra rows.
+__global__ void __launch_bounds__(256) match_rows_kernel(const int32_t* __restrict__ masked_pos, int m,
+                                                         const int32_t* __restrict__ extra_rows, int e, int k,
+                                                         int32_t* __restrict__ idx, uint32_t* status) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int b = blockIdx.y;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= m) return;
+    const int want = masked_pos[(int64_t)b * m + i];
+    int found = -1;
+    for (int j = 0; j < e; ++j)
+        if (extra_rows[(int64_t)b * e + j] == want) { found = k + j; break; }
+    idx[(int64_t)b * m + i] = found;
+    if (found < 0) atomicOr(status, kFlagBadIndex);
+}
+
+void launch_match_rows(const int32_t* masked_pos, int m, const int32_t* extra_rows, int e, int k, int batch,
+                       int32_t* idx, uint32_t* status, cudaStream_t stream) {
+    if (batch == 0 || m == 0) return;
+    launch_pdl(match_rows_kernel, dim3((m + 255) / 256, batch), dim3(256), 0, stream, masked_pos, m, extra_rows, e, k, idx,
+               status);
+}
+
 void launch_scatter_kv(void* cache_k, void* cache_v, int64_t batch_stride, int ctx_len, const int32_t* anchor_idx,
                        int k, const int32_t* extra_rows, int e, int batch, int affix_start, int affix_len,
                        int kv_dim, const void* k_new, const void* v_new, uint32_t* status, cudaStream_t stream) {

@@ -407,6 +407,52 @@ def test_layer_step_scores_use_stale_keys_and_accumulate():
     assert out3["scores64"].sum() < H * m and np.all(out3["scores64"] < out["scores64"])
 
 
+def two_layer_case(extra="all"):
+    lay = wl.make_layout(1, 3, 12, 5, 6, 4, extra)
+    layers = [wl.layer_weights(SMALL, 9, n, std=0.2) for n in range(2)]
+    x = wl.hidden_states(SMALL, lay, 100, 101)[0]
+    xs = wl.hidden_states(SMALL, lay, 100, 102)[0]
+    cos, sin = wl.rope_table(lay.ctx_len, SMALL.head_dim, SMALL.rope_theta)
+    # stale caches: exact K/V of every layer of a dense forward under ANOTHER context
+    caches = [(kb, vb) for (_, kb, vb) in orc.dense_forward(layers, SMALL, xs, cos, sin)]
+    return lay, layers, x, caches, cos, sin
+
+
+def test_multilayer_refresh_at_ratio_one_equals_dense_forward():
+    round_storage = True      # between layers the hidden rows are a stored bf16 tensor
+    lay, layers, x, caches, cos, sin = two_layer_case()
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    rows, out_caches, ys = orc.refresh_forward(layers, SMALL, x, caches, T, l, np.arange(L), lay.extra_rows[0], cos, sin,
+                                               round_storage)
+    dense = orc.dense_forward(layers, SMALL, x, cos, sin, round_storage)
+    assert sorted(rows.tolist()) == list(range(T))
+    for n in range(2):
+        y, kd, vd = dense[n]
+        assert np.array_equal(out_caches[n][0], kd) and np.array_equal(out_caches[n][1], vd)
+        assert np.allclose(ys[n], y[rows], rtol=1e-9, atol=1e-10)
+
+
+def test_multilayer_probe_scores_and_ratio_zero_refresh():
+    lay, layers, x, caches, cos, sin = two_layer_case()
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    P, M = lay.extra_rows[0], lay.masked_pos[0]
+    s, pc, pys = orc.probe_forward(layers, SMALL, x, caches, T, l, L, M, P, cos, sin)
+    N, H, m = 2, SMALL.n_heads, len(M)
+    assert abs(s.sum() - N * H * m) < 1e-9 and np.all(s > 0)            # Eq. 5 sums over layers
+    # layer 0's share is the single-layer score
+    one = orc.layer_step(layers[0], SMALL, x, caches[0][0], caches[0][1], T, l, L, M, P, cos, sin, ratio=0.0)
+    s1, _, _ = orc.probe_forward(layers[:1], SMALL, x, caches[:1], T, l, L, M, P, cos, sin)
+    assert np.allclose(s1, one["scores64"], rtol=1e-13)
+    assert np.all(s > s1)
+    # the probe is the refresh pass with no anchors: same rows, same outputs, affix rows untouched
+    rows, rc, rys = orc.refresh_forward(layers, SMALL, x, caches, T, l, np.zeros(0, np.int64), P, cos, sin)
+    for n in range(2):
+        assert np.array_equal(rys[n], pys[n]) and np.array_equal(rc[n][0], pc[n][0])
+        assert np.array_equal(pc[n][0][l:l + L], caches[n][0][l:l + L])
+    # layer 1's scores use layer 1's queries: they differ from scoring layer 0's queries on layer 1's keys
+    assert not np.allclose(s - s1, s1)
+
+
 def test_comparators():
     ok, worst = orc.rel_err_gate(np.array([1.0, 2.0]), np.array([1.0, 2.0]))
     assert ok and worst == 0
