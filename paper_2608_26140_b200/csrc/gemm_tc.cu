@@ -39,7 +39,7 @@ constexpr int TC_BM = 128, TC_BN = 256, TC_BK = 64, TC_STAGES = 4;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;          // 16 KB
 constexpr int TC_HALF_BYTES = 128 * TC_BK * 2;         // 16 KB: one 128-row half of the B tile
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + 2 * TC_HALF_BYTES;
-constexpr int TC_THREADS = 384;                        // warp 0: TMA, warp 1: MMA, warps 2-5: drain; all 12 warps do phase 0
+constexpr int TC_THREADS = 192;                        // warp 0: TMA, warp 1: MMA, warps 2-5: drain; all six warps do phase 0
 constexpr int TC_SMEM = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int TC_SLOT_FLOATS = TC_BM * TC_BN;          // one fp32 partial tile
 constexpr uint32_t TC_WAIT_LIMIT = 1u << 22;
@@ -194,108 +194,48 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
     return make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
 }
 
-// Ordered sums over the partial-tile slots of one row for 16 adjacent columns starting at column
-// group pc0 and, if pc1 >= 0, 16 more starting at pc1.  Loads are issued two slots at a time
-// for all eight column groups (16 independent 16-byte loads in flight per thread) and added in
-// slot order, which keeps the result bitwise reproducible.
-__device__ __forceinline__ void sum_slots16(const float4* __restrict__ src, int nslots, int pc0, int pc1, int row,
-                                            float (&lo)[16], float (&hi)[16]) {
+// ---- epilogues on W adjacent fp32 accumulator columns of one row (W = 16 or 32) ----------------
+// Every store is W*2 bytes of one row: whole 32-byte sectors, no partial-sector writes.
+
+// out[grow, col..col+W) = bf16(resid[grow] + acc)
+template <int W>
+__device__ __forceinline__ void out_residual(const GemmArgs& g, int grow, int col, float (&v)[W]) {
+    const int N = g.n[0];
+    const int64_t roff = g.resid_off ? __ldcg(g.resid_off + grow) : (int64_t)grow * N;
+    const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(g.resid) + roff + col);
+    uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * N + col);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) { lo[i] = 0.f; hi[i] = 0.f; }
-    const float4* q0 = src + pc0 * TC_BM + row;
-    const float4* q1 = src + (pc1 < 0 ? pc0 : pc1) * TC_BM + row;
-    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c0 = 0; c0 < nslots; c0 += 2) {
-        float4 a[2][4], b[2][4];
+    for (int j = 0; j < W / 8; ++j) {
+        const uint4 r = __ldcg(rp + j);
+        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const bool in = c0 + i < nslots;
-            const int64_t so = (int64_t)(c0 + i) * (TC_SLOT_FLOATS / 4);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                a[i][j] = in ? __ldcg(q0 + so + j * TC_BM) : zero;
-                b[i][j] = (in && pc1 >= 0) ? __ldcg(q1 + so + j * TC_BM) : zero;
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            if (c0 + i < nslots) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    lo[4 * j] += a[i][j].x; lo[4 * j + 1] += a[i][j].y; lo[4 * j + 2] += a[i][j].z; lo[4 * j + 3] += a[i][j].w;
-                    hi[4 * j] += b[i][j].x; hi[4 * j + 1] += b[i][j].y; hi[4 * j + 2] += b[i][j].z; hi[4 * j + 3] += b[i][j].w;
-                }
-            }
-        }
+        for (int i = 0; i < 4; ++i) { v[8 * j + 2 * i] += bf16_lo(rw[i]); v[8 * j + 2 * i + 1] += bf16_hi(rw[i]); }
+        o[j] = pack8(v + 8 * j);
     }
 }
 
-// Output columns per work item: 16 (a full 32-byte sector of bf16 per row, so no store is a
-// partial-sector write).  q/k/v items carry 16 columns of each rotary half.
-__host__ __device__ __forceinline__ int finish_items(int epilogue, int n_total) {
-    return epilogue == kEpiQKV ? n_total / 32 : n_total / 16;
+// out[grow, col..col+W) = bf16(silu(gate) * up)
+template <int W>
+__device__ __forceinline__ void out_swiglu(const GemmArgs& g, int grow, int col, float (&gate)[W], const float (&up)[W]) {
+    uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * g.n[0] + col);
+#pragma unroll
+    for (int i = 0; i < W; ++i) gate[i] = gate[i] / (1.f + __expf(-gate[i])) * up[i];
+#pragma unroll
+    for (int j = 0; j < W / 8; ++j) o[j] = pack8(gate + 8 * j);
 }
 
-// Epilogue of one work item of row `grow`.
-__device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, int item, int mt, int row) {
-    const int grow = mt * TC_BM + row;
-    int nt, pc0, pc1;            // N tile, first partial column group of each half
-    int u128 = 0, lo_col = 0;
+// q/k/v: bias, rotary embedding with the pairing (i, i + d/2) at the row's position, bf16 store
+// to the compact output and, for k/v, straight into the cache row (scatter fused).
+// lo/hi: W columns of each rotary half; col: column of lo[0] inside segment seg; j0: its index
+// inside the half head.
+template <int W>
+__device__ __forceinline__ void out_qkv(const GemmArgs& g, int grow, int pos, int seg, int col, int j0, float (&lo)[W],
+                                        float (&hi)[W]) {
     const int half = g.head_dim >> 1;
-    if (g.epilogue == kEpiResidual) {
-        nt = item >> 4; pc0 = (item & 15) * 4; pc1 = -1;
-    } else if (g.epilogue == kEpiSwiGLU) {
-        nt = item >> 3; pc0 = (item & 7) * 4; pc1 = 32 + pc0;
-    } else {
-        u128 = item >> 2;
-        const int r = item & 3;
-        nt = u128 >> 1;
-        lo_col = g.head_dim == 128 ? 16 * r : 64 * (r >> 1) + 16 * (r & 1);   // column inside the 128-wide unit
-        pc0 = 32 * (u128 & 1) + (lo_col >> 2);
-        pc1 = pc0 + (half >> 2);
-    }
-    const int t = mt * p.n_tiles + nt;
-    const int c_first = (int)(((int64_t)t * p.KB) / p.U);
-    const int c_last = (int)(((int64_t)(t + 1) * p.KB - 1) / p.U);
-    const int nslots = c_last - c_first + 1;
-    const float4* src = reinterpret_cast<const float4*>(g.partial + (int64_t)t * p.smax * TC_SLOT_FLOATS);
-    // loads that do not depend on the sums go first so that they overlap the partial-tile reads
-    int pos = 0;
-    int64_t roff = 0;
-    if (g.epilogue == kEpiQKV) pos = __ldcg(g.row_pos + grow);
-    if (g.epilogue == kEpiResidual) roff = g.resid_off ? __ldcg(g.resid_off + grow) : (int64_t)grow * g.n[0];
-    float lo[16], hi[16];
-    sum_slots16(src, nslots, pc0, pc1, row, lo, hi);
-
-    if (g.epilogue == kEpiResidual) {
-        const int N = g.n[0], col = item * 16;
-        const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(g.resid) + roff + col);
-        const uint4 r0 = __ldcg(rp), r1 = __ldcg(rp + 1);
-        const uint32_t rw[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { lo[2 * i] += bf16_lo(rw[i]); lo[2 * i + 1] += bf16_hi(rw[i]); }
-        uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * N + col);
-        o[0] = pack8(lo);
-        o[1] = pack8(lo + 8);
-        return;
-    }
-    if (g.epilogue == kEpiSwiGLU) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) lo[i] = lo[i] / (1.f + __expf(-lo[i])) * hi[i];
-        uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * g.n[0] + item * 16);
-        o[0] = pack8(lo);
-        o[1] = pack8(lo + 8);
-        return;
-    }
-    // q/k/v: bias, rotary embedding with the pairing (i, i + d/2), store (+ fused cache scatter)
-    int seg = 0, c0 = u128 * 128;
-    while (seg < 2 && c0 >= g.n[seg]) { c0 -= g.n[seg]; ++seg; }
-    const int col = c0 + lo_col;                          // column inside the segment
-    const int j0 = lo_col & (half - 1);                   // index inside the half head
     const __nv_bfloat16* bias = static_cast<const __nv_bfloat16*>(g.bias[seg]);
     if (bias) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < W; ++i) {
             lo[i] += __bfloat162float(bias[col + i]);
             hi[i] += __bfloat162float(bias[col + half + i]);
         }
@@ -305,7 +245,7 @@ __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, 
         const float4* cs = reinterpret_cast<const float4*>(g.rope_cos + (int64_t)pp * half + j0);
         const float4* sn = reinterpret_cast<const float4*>(g.rope_sin + (int64_t)pp * half + j0);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < W / 4; ++j) {
             const float4 c4 = cs[j], s4 = sn[j];
             const float c[4] = {c4.x, c4.y, c4.z, c4.w}, sv[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
@@ -316,20 +256,145 @@ __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, 
             }
         }
     }
-    const uint4 l0 = pack8(lo), l1 = pack8(lo + 8), h0 = pack8(hi), h1 = pack8(hi + 8);
     const int nseg = g.n[seg];
-    if (g.out[seg]) {
-        __nv_bfloat16* o = static_cast<__nv_bfloat16*>(g.out[seg]) + (int64_t)grow * nseg + col;
-        reinterpret_cast<uint4*>(o)[0] = l0; reinterpret_cast<uint4*>(o)[1] = l1;
-        reinterpret_cast<uint4*>(o + half)[0] = h0; reinterpret_cast<uint4*>(o + half)[1] = h1;
-    }
     __nv_bfloat16* cache = seg == 1 ? static_cast<__nv_bfloat16*>(g.cache_k)
                          : seg == 2 ? static_cast<__nv_bfloat16*>(g.cache_v) : nullptr;
-    if (cache && pos >= 0) {
-        const int b = grow / g.rows_per_req;
-        __nv_bfloat16* o = cache + (int64_t)b * g.kv_batch_stride + (int64_t)pos * nseg + col;
-        reinterpret_cast<uint4*>(o)[0] = l0; reinterpret_cast<uint4*>(o)[1] = l1;
-        reinterpret_cast<uint4*>(o + half)[0] = h0; reinterpret_cast<uint4*>(o + half)[1] = h1;
+    __nv_bfloat16* o1 = g.out[seg] ? static_cast<__nv_bfloat16*>(g.out[seg]) + (int64_t)grow * nseg + col : nullptr;
+    __nv_bfloat16* o2 = (cache && pos >= 0)
+                            ? cache + (int64_t)(grow / g.rows_per_req) * g.kv_batch_stride + (int64_t)pos * nseg + col
+                            : nullptr;
+#pragma unroll
+    for (int j = 0; j < W / 8; ++j) {
+        const uint4 l = pack8(lo + 8 * j), h = pack8(hi + 8 * j);
+        if (o1) { reinterpret_cast<uint4*>(o1)[j] = l; reinterpret_cast<uint4*>(o1 + half)[j] = h; }
+        if (o2) { reinterpret_cast<uint4*>(o2)[j] = l; reinterpret_cast<uint4*>(o2 + half)[j] = h; }
+    }
+}
+
+// Segment and in-segment column of the 128-wide column unit u128 of a q/k/v projection.
+__device__ __forceinline__ void qkv_unit(const GemmArgs& g, int u128, int& seg, int& c0) {
+    seg = 0; c0 = u128 * 128;
+    while (seg < 2 && c0 >= g.n[seg]) { c0 -= g.n[seg]; ++seg; }
+}
+
+// ---- split tiles: partial slots and their ordered sum -------------------------------------------
+// A tile whose K range is cut between CTAs is accumulated through fp32 partial tiles.  Each CTA owns
+// two slots: slot 0 for its first segment, slot 1 for its last (segments in between are whole tiles
+// and never need one).  Tile t's contributors are CTAs c_first..c_last; CTA c's part of it is that
+// CTA's first segment exactly when the CTA starts inside the tile.
+__device__ __forceinline__ void tile_cover(const TcPlan& p, int t, int& c_first, int& c_last) {
+    c_first = (int)(((int64_t)t * p.KB) / p.U);
+    c_last = (int)(((int64_t)(t + 1) * p.KB - 1) / p.U);
+}
+__device__ __forceinline__ int64_t slot_of(const TcPlan& p, int t, int c) {
+    return (int64_t)c * 2 + ((int64_t)c * p.U >= (int64_t)t * p.KB ? 0 : 1);
+}
+
+// Ordered sums over the contributing CTAs' partial tiles of one row for 16 adjacent columns
+// starting at column group pc0 and, if pc1 >= 0, 16 more starting at pc1.  Loads are issued two
+// CTAs at a time for all eight column groups (16 independent 16-byte loads in flight per thread)
+// and added in ascending CTA order, which keeps the result bitwise reproducible.
+__device__ __forceinline__ void sum_slots16(const float* __restrict__ partial, const TcPlan& p, int t, int c_first,
+                                            int c_last, int pc0, int pc1, int row, float (&lo)[16], float (&hi)[16]) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { lo[i] = 0.f; hi[i] = 0.f; }
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int o0 = pc0 * TC_BM + row, o1 = (pc1 < 0 ? pc0 : pc1) * TC_BM + row;
+    for (int c = c_first; c <= c_last; c += 2) {
+        float4 a[2][4], b[2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const bool in = c + i <= c_last;
+            const float4* src = reinterpret_cast<const float4*>(partial) + slot_of(p, t, in ? c + i : c) * (TC_SLOT_FLOATS / 4);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                a[i][j] = in ? __ldcg(src + o0 + j * TC_BM) : zero;
+                b[i][j] = (in && pc1 >= 0) ? __ldcg(src + o1 + j * TC_BM) : zero;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            if (c + i <= c_last) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    lo[4 * j] += a[i][j].x; lo[4 * j + 1] += a[i][j].y; lo[4 * j + 2] += a[i][j].z; lo[4 * j + 3] += a[i][j].w;
+                    hi[4 * j] += b[i][j].x; hi[4 * j + 1] += b[i][j].y; hi[4 * j + 2] += b[i][j].z; hi[4 * j + 3] += b[i][j].w;
+                }
+            }
+        }
+    }
+}
+
+// Work items of the finish per output tile: 16 output columns each (q/k/v: 16 of each rotary half).
+__host__ __device__ __forceinline__ int finish_items_per_tile(int epilogue) { return epilogue == kEpiResidual ? 16 : 8; }
+
+// Finish of one work item of split tile t = nt * m_tiles + mt for tile row `row`.
+__device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, int t, int item, int row) {
+    const int nt = t / p.m_tiles, mt = t - nt * p.m_tiles;
+    const int grow = mt * TC_BM + row;
+    int c_first, c_last;
+    tile_cover(p, t, c_first, c_last);
+    const int half = g.head_dim >> 1;
+    int pc0, pc1 = -1, u128 = 0, lo_col = 0;
+    if (g.epilogue == kEpiResidual) {
+        pc0 = item * 4;
+    } else if (g.epilogue == kEpiSwiGLU) {
+        pc0 = item * 4; pc1 = 32 + pc0;
+    } else {
+        const int h = item >> 2, r = item & 3;
+        u128 = nt * 2 + h;
+        if (u128 >= p.units) return;                                      // the tile's second half is past the end
+        lo_col = g.head_dim == 128 ? 16 * r : 64 * (r >> 1) + 16 * (r & 1);   // column inside the 128-wide unit
+        pc0 = 32 * h + (lo_col >> 2);
+        pc1 = pc0 + (half >> 2);
+    }
+    int pos = 0;
+    if (g.epilogue == kEpiQKV) pos = __ldcg(g.row_pos + grow);     // independent of the sums: overlaps their loads
+    float lo[16], hi[16];
+    sum_slots16(g.partial, p, t, c_first, c_last, pc0, pc1, row, lo, hi);
+    if (g.epilogue == kEpiResidual) {
+        out_residual<16>(g, grow, nt * TC_BN + item * 16, lo);
+    } else if (g.epilogue == kEpiSwiGLU) {
+        out_swiglu<16>(g, grow, nt * 128 + item * 16, lo, hi);
+    } else {
+        int seg, c0;
+        qkv_unit(g, u128, seg, c0);
+        out_qkv<16>(g, grow, pos, seg, c0 + lo_col, lo_col & (half - 1), lo, hi);
+    }
+}
+
+// Epilogue of a whole tile straight from TMEM (the CTA covered the tile's entire K range):
+// thread = one row of the tile, 32 accumulator columns per tcgen05.ld.
+__device__ __forceinline__ void direct_epilogue(const GemmArgs& g, const TcPlan& p, uint32_t taddr, int nt, int grow,
+                                                bool valid, int nchunks) {
+    if (g.epilogue == kEpiResidual) {
+        for (int c = 0; c < nchunks; ++c) {
+            float v[32];
+            tc_ld32(taddr + c * 32, v);
+            if (valid) out_residual<32>(g, grow, nt * TC_BN + c * 32, v);
+        }
+    } else if (g.epilogue == kEpiSwiGLU) {
+        for (int c = 0; c < 4; ++c) {
+            float gate[32], up[32];
+            tc_ld32(taddr + c * 32, gate);
+            tc_ld32(taddr + 128 + c * 32, up);
+            if (valid) out_swiglu<32>(g, grow, nt * 128 + c * 32, gate, up);
+        }
+    } else {
+        const int half = g.head_dim >> 1;
+        const int pos = valid ? __ldcg(g.row_pos + grow) : 0;
+        for (int h = 0; h < nchunks / 4; ++h) {
+            int seg, c0;
+            qkv_unit(g, nt * 2 + h, seg, c0);
+            for (int r = 0; r < 2; ++r) {
+                // d = 128: chunks (r, r + 2) of the unit; d = 64: chunks (2r, 2r + 1)
+                const int cl = g.head_dim == 128 ? r : 2 * r, ch = g.head_dim == 128 ? r + 2 : 2 * r + 1;
+                float lo[32], hi[32];
+                tc_ld32(taddr + h * 128 + cl * 32, lo);
+                tc_ld32(taddr + h * 128 + ch * 32, hi);
+                if (valid) out_qkv<32>(g, grow, pos, seg, c0 + cl * 32, (cl * 32) & (half - 1), lo, hi);
+            }
+        }
     }
 }
 
@@ -416,7 +481,7 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
         for (int it = it0; it < it1 && ok;) {
             const int t = it / p.KB, kb0 = it - t * p.KB;
             const int kb1 = min(p.KB, kb0 + (it1 - it));
-            const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
+            const int nt = t / p.m_tiles, mt = t - nt * p.m_tiles;
             int row0, row1;
             const int s0 = half_source(g, p, nt, 0, row0), s1 = half_source(g, p, nt, 1, row1);
             const uint32_t bytes = TC_A_BYTES + TC_HALF_BYTES * (1 + (s1 >= 0));
@@ -439,7 +504,7 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
         for (int it = it0; it < it1 && ok;) {
             const int t = it / p.KB, kb0 = it - t * p.KB;
             const int kb1 = min(p.KB, kb0 + (it1 - it));
-            const int nt = t % p.n_tiles;
+            const int nt = t / p.m_tiles;
             int row1;
             const uint32_t idesc = idesc_bf16(half_source(g, p, nt, 1, row1) >= 0 ? 256 : 128);
             if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag))) break;
@@ -462,7 +527,8 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
             it += kb1 - kb0;
         }
     } else if (warp >= 2 && warp < 6) {
-        // drain: TMEM -> fp32 partial tile, layout [column / 4][row][4]
+        // drain: whole tiles get their epilogue straight from TMEM; a tile whose K range is split
+        // between CTAs goes to this CTA's fp32 partial slot, layout [column / 4][row][4]
         const int q = warp & 3;                   // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
         int acc = 0;
@@ -472,21 +538,26 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
         for (int it = it0; it < it1 && ok;) {
             const int t = it / p.KB, kb0 = it - t * p.KB;
             const int kb1 = min(p.KB, kb0 + (it1 - it));
-            const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
+            const int nt = t / p.m_tiles, mt = t - nt * p.m_tiles;
             int row1;
             const int nchunks = half_source(g, p, nt, 1, row1) >= 0 ? 8 : 4;
-            const int slot = blockIdx.x - (int)(((int64_t)t * p.KB) / p.U);
-            float4* dst = reinterpret_cast<float4*>(g.partial + ((int64_t)t * p.smax + slot) * TC_SLOT_FLOATS);
             if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) break;
             tc_fence_after();
             const bool valid = mt * TC_BM + row < g.M;
-            for (int c = 0; c < nchunks; ++c) {
-                float v[32];
-                tc_ld32(tmem_base + acc * TC_BN + c * 32 + ((uint32_t)(q * 32) << 16), v);
-                if (valid) {
+            const uint32_t taddr = tmem_base + acc * TC_BN + ((uint32_t)(q * 32) << 16);
+            if (kb0 == 0 && kb1 == p.KB) {
+                direct_epilogue(g, p, taddr, nt, mt * TC_BM + row, valid, nchunks);
+            } else {
+                float4* dst = reinterpret_cast<float4*>(g.partial) +
+                              ((int64_t)blockIdx.x * 2 + (it == it0 ? 0 : 1)) * (TC_SLOT_FLOATS / 4);
+                for (int c = 0; c < nchunks; ++c) {
+                    float v[32];
+                    tc_ld32(taddr + c * 32, v);
+                    if (valid) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        st_hint_f4(&dst[(c * 8 + i) * TC_BM + row], make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]), pol_p);
+                        for (int i = 0; i < 8; ++i)
+                            st_hint_f4(&dst[(c * 8 + i) * TC_BM + row], make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]), pol_p);
+                    }
                 }
             }
             tc_fence_before();
@@ -521,17 +592,23 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     }
 }
 
-__global__ void __launch_bounds__(256) gemm_finish_kernel(const GemmArgs g, const TcPlan p, int n_items) {
+// Finish of the split tiles: grid row y finishes tile split.tile[y]; blockIdx.x * 256 +
+// threadIdx.x -> (item, row).
+struct SplitTiles {
+    int n;
+    int tile[160];     // one per CTA boundary that cuts a tile (at most SM count - 1)
+};
+
+__global__ void __launch_bounds__(256, 2) gemm_finish_kernel(const GemmArgs g, const TcPlan p, const SplitTiles split) {
     pdl_wait();
     pdl_launch_dependents();
+    const int t = split.tile[blockIdx.y];
+    const int mt = t % p.m_tiles;
     const int rows_per = p.m_tiles == 1 ? ((g.M + 31) & ~31) : TC_BM;
-    const int64_t work = (int64_t)n_items * p.m_tiles * rows_per;
-    const int64_t w = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (w >= work) return;
-    const int row = (int)(w % rows_per);
-    const int64_t s = w / rows_per;
-    const int item = (int)(s % n_items), mt = (int)(s / n_items);
-    if (mt * TC_BM + row < g.M) finish_item(g, p, item, mt, row);
+    const int w = blockIdx.x * 256 + threadIdx.x;
+    const int row = w % rows_per, item = w / rows_per;
+    if (item >= finish_items_per_tile(g.epilogue) || mt * TC_BM + row >= g.M) return;
+    finish_item(g, p, t, item, row);
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -603,16 +680,16 @@ TcPlan make_plan(int M, int K, int units, bool swiglu) {
     const int g = (int)(total < sm_count() ? total : sm_count());
     p.U = (int)((total + g - 1) / g);
     p.ctas = (int)((total + p.U - 1) / p.U);
-    p.smax = (p.KB + p.U - 1) / p.U + 1;
+    p.smax = 2;   // partial slots per CTA
     return p;
 }
 
 }  // namespace
 
 size_t gemm_partial_bytes(int M, int K, int n_total, bool swiglu) {
-    if (M <= 0) return 0;
-    TcPlan p = make_plan(M, K, n_total / 128, swiglu);
-    return (size_t)p.tiles * p.smax * TC_SLOT_FLOATS * sizeof(float);
+    (void)M; (void)K; (void)n_total; (void)swiglu;
+    // two fp32 partial tiles per CTA, at most one CTA per SM, whatever the problem size
+    return (size_t)sm_count() * 2 * TC_SLOT_FLOATS * sizeof(float);
 }
 
 int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
@@ -638,10 +715,18 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
     if (launch_pdl(gemm_tc_kernel, dim3(p.ctas), dim3(TC_THREADS), TC_SMEM, stream, g, p, *mA, *mB[0], *mB[1], *mB[2]) !=
         cudaSuccess)
         return -1;
-    const int n_items = finish_items(g.epilogue, n_total);
+    // tiles whose K range is cut by a boundary between two CTAs, each listed once
+    SplitTiles split{};
+    for (int c = 1; c < p.ctas && split.n < 160; ++c) {
+        const int64_t cut = (int64_t)c * p.U;
+        if (cut % p.KB == 0) continue;
+        const int t = (int)(cut / p.KB);
+        if (split.n == 0 || split.tile[split.n - 1] != t) split.tile[split.n++] = t;
+    }
+    if (split.n == 0) return 1;
     const int rows_per = p.m_tiles == 1 ? ((g.M + 31) & ~31) : TC_BM;
-    const int64_t work = (int64_t)n_items * p.m_tiles * rows_per;
-    if (launch_pdl(gemm_finish_kernel, dim3((unsigned)((work + 255) / 256)), dim3(256), 0, stream, g, p, n_items) !=
+    const int per_tile = finish_items_per_tile(g.epilogue) * rows_per;
+    if (launch_pdl(gemm_finish_kernel, dim3((per_tile + 255) / 256, split.n), dim3(256), 0, stream, g, p, split) !=
         cudaSuccess)
         return -1;
     return 2;
