@@ -457,6 +457,17 @@ def test_comparators():
     ok, worst = orc.rel_err_gate(np.array([1.0, 2.0]), np.array([1.0, 2.0]))
     assert ok and worst == 0
     assert not orc.rel_err_gate(np.array([1.0, 2.2]), np.array([1.0, 2.0]))[0]
+    g = np.random.default_rng(3)
+    b = g.standard_normal(400000)
+    assert orc.rel_err_gate(b * (1 + 2e-3 * g.standard_normal(b.size)), b)[0]          # bf16-ulp sized noise
+    one = b.copy(); one[7] += 0.03                                                    # one element at 3 % of rms:
+    assert orc.rel_err_gate(one, b)[0]                                                # inside the rounding tail
+    one[7] += 0.03
+    assert not orc.rel_err_gate(one, b)[0]                                            # 6 %: a wrong element
+    few = b.copy(); few[:40] += 0.03
+    assert not orc.rel_err_gate(few, b)[0]                                            # too many elements over 2 %
+    assert not orc.rel_err_gate(b * 1.02, b)[0]                                       # systematic 2 % error
+    assert not orc.rel_err_gate(b + 0.02, b)[0]                                       # a dropped bias-like term
     must, may = np.array([1, 5]), np.array([1, 3, 5, 7])
     assert orc.anchor_set_ok(np.array([1, 3, 5]), 3, 10, must, may)[0]
     assert not orc.anchor_set_ok(np.array([1, 3, 4]), 3, 10, must, may)[0]
