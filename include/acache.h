@@ -74,6 +74,8 @@ typedef struct {
     int32_t max_affix;     /* L                                  */
     int32_t max_rows;      /* K + e per request                  */
     int32_t max_masked;    /* m per request                      */
+    int32_t max_vocab;     /* V of acache_predict_commit, 0 if unused          */
+    int32_t max_block;     /* rows per request of acache_predict_commit, 0 if unused */
 } acache_model_desc;
 
 /* DEVICE bf16 weights, [out, in] row-major.  bq/bk/bv may be NULL when qkv_bias == 0. */
@@ -241,6 +243,21 @@ acache_status acache_layer_step(acache_ctx *ctx, const acache_layer_weights *w,
                                 const acache_request *req, acache_kv *kv,
                                 const void *x, int x_is_compact, double ratio, uint32_t flags,
                                 float *scores, int32_t *anchor_idx, void *y, acache_stream_t stream);
+
+/* Predict-then-commit on the current block (Section 3.1, Eq. 2-3, with the confidence-threshold
+ * commit rule the paper's set-up uses, threshold 0.9 in Section 5):
+ *   z = W_lm (RMSNorm(h_i) g);  token_i = argmax_v z_v;  conf_i = softmax(z)[token_i]
+ *   commit_i = conf_i > threshold; a request none of whose rows qualifies commits its single most
+ *   confident row (lowest index on ties).
+ * h: DEVICE bf16 [B, h_rows, D], the last layer's compact output; block_rows: DEVICE int32
+ * [B, n_blk], the compact row (0 <= . < h_rows) of each masked position of the current block.
+ * final_norm_g: DEVICE bf16 [D]; w_lm: DEVICE bf16 [V, D], V a multiple of 128.
+ * token, commit: DEVICE int32 [B, n_blk]; confidence: DEVICE fp32 [B, n_blk].
+ * Needs batch * n_blk <= max_batch * max_block, V <= max_vocab of the descriptor. */
+acache_status acache_predict_commit(acache_ctx *ctx, const void *h, int32_t h_rows, const int32_t *block_rows,
+                                    int32_t batch, int32_t n_blk, const void *final_norm_g, const void *w_lm,
+                                    int32_t vocab, float threshold, int32_t *token, float *confidence,
+                                    int32_t *commit, acache_stream_t stream);
 
 /* acache_layer_step for a caller whose per-step data lives in HOST memory: copies
  * x [B, ctx_len, D] (HOST bf16, ideally pinned) to a staging area in the workspace,

@@ -408,6 +408,32 @@ def dense_forward(layers, shape, x0: np.ndarray, cos, sin, round_storage: bool =
 
 
 # --------------------------------------------------------------------------
+# Eq. 2-3: predict the masked positions of the current block, commit the confident ones
+# --------------------------------------------------------------------------
+def predict_commit(h_rows: np.ndarray, final_norm_g: np.ndarray, w_lm: np.ndarray, eps: float, threshold: float,
+                   round_storage: bool = True):
+    """One request's block: z = W_lm (RMSNorm(h) g); token = argmax_v z (lowest index on ties);
+    confidence = softmax(z)[token]; commit = confidence > threshold, or, if no row qualifies, the
+    single most confident row (lowest index on ties) -- the threshold rule of the decoding
+    schedule the paper builds on (Section 3.1; threshold 0.9 in Section 5).
+
+    h_rows [n, D] fp64 (bf16 values); final_norm_g [D] and w_lm [V, D] bf16 bits or floats.
+    Returns (token int32 [n], confidence fp64 [n], commit bool [n], logits fp64 [n, V]).
+    """
+    g = bf16_bits_to_f64(final_norm_g) if final_norm_g.dtype == np.uint16 else np.asarray(final_norm_g, F64)
+    W = bf16_bits_to_f64(w_lm) if w_lm.dtype == np.uint16 else np.asarray(w_lm, F64)
+    hn = _store(rmsnorm(h_rows, g, eps), round_storage)
+    z = hn @ W.T
+    token = np.argmax(z, axis=1).astype(np.int32)
+    zmax = z.max(axis=1, keepdims=True)
+    conf = 1.0 / np.exp(z - zmax).sum(axis=1)
+    commit = conf > threshold
+    if z.shape[0] and not commit.any():
+        commit[int(np.argmax(conf))] = True
+    return token, conf, commit, z
+
+
+# --------------------------------------------------------------------------
 # comparison helpers used by the parity tests
 # --------------------------------------------------------------------------
 def rel_err_gate(a: np.ndarray, b: np.ndarray, tol: float = 2e-2) -> Tuple[bool, float]:

@@ -22,7 +22,7 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_last_error", "acache_poll_status", "acache_launch_count", "acache_score_anchors",
            "acache_k_from_ratio", "acache_select_topk", "acache_recompute_anchors", "acache_scatter_kv",
            "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times",
-           "acache_score_anchors_static"]
+           "acache_score_anchors_static", "acache_predict_commit"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -31,7 +31,8 @@ class ModelDesc(C.Structure):
     _fields_ = [("hidden", C.c_int32), ("n_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("ffn", C.c_int32), ("rms_eps", C.c_float),
                 ("qkv_bias", C.c_int32), ("max_batch", C.c_int32), ("max_ctx", C.c_int32),
-                ("max_affix", C.c_int32), ("max_rows", C.c_int32), ("max_masked", C.c_int32)]
+                ("max_affix", C.c_int32), ("max_rows", C.c_int32), ("max_masked", C.c_int32),
+                ("max_vocab", C.c_int32), ("max_block", C.c_int32)]
 
 
 class LayerWeights(C.Structure):
@@ -104,6 +105,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_score_anchors_static.argtypes = [C.POINTER(ModelDesc), C.POINTER(Request), vp, C.POINTER(KV), vp,
                                                 C.c_int, C.c_int, vp]
     lib.acache_score_anchors_static.restype = C.c_int
+    lib.acache_predict_commit.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, i32, C.c_float, vp, vp, vp, vp]
+    lib.acache_predict_commit.restype = C.c_int
     lib.acache_stage_timing.argtypes = [vp, C.c_int]
     lib.acache_stage_timing.restype = C.c_int
     lib.acache_read_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
@@ -143,11 +146,11 @@ class Context:
     """One layer shape + workspace.  Mirrors the C entry points one to one."""
 
     def __init__(self, hidden, n_heads, n_kv_heads, head_dim, ffn, rms_eps, qkv_bias,
-                 max_batch, max_ctx, max_affix, max_rows, max_masked, device="cuda:0"):
+                 max_batch, max_ctx, max_affix, max_rows, max_masked, device="cuda:0", max_vocab=0, max_block=0):
         import torch
         self.lib = load_library()
         self.desc = ModelDesc(hidden, n_heads, n_kv_heads, head_dim, ffn, rms_eps, int(bool(qkv_bias)),
-                              max_batch, max_ctx, max_affix, max_rows, max_masked)
+                              max_batch, max_ctx, max_affix, max_rows, max_masked, max_vocab, max_block)
         h = C.c_void_p()
         st = self.lib.acache_create(C.byref(self.desc), C.byref(h))
         if st != OK:
@@ -163,9 +166,10 @@ class Context:
         self.workspace_bytes = nbytes
 
     @classmethod
-    def for_shape(cls, shape, max_batch, max_ctx, max_affix, max_rows, max_masked, device="cuda:0"):
+    def for_shape(cls, shape, max_batch, max_ctx, max_affix, max_rows, max_masked, device="cuda:0", max_vocab=0,
+                  max_block=0):
         return cls(shape.hidden, shape.n_heads, shape.n_kv_heads, shape.head_dim, shape.ffn, shape.rms_eps,
-                   shape.qkv_bias, max_batch, max_ctx, max_affix, max_rows, max_masked, device)
+                   shape.qkv_bias, max_batch, max_ctx, max_affix, max_rows, max_masked, device, max_vocab, max_block)
 
     def close(self):
         if getattr(self, "h", None):
@@ -244,6 +248,12 @@ class Context:
         self._check(self.lib.acache_layer_step(self.h, C.byref(w), C.byref(req), C.byref(kv), _ptr(x),
                                                int(x_is_compact), float(ratio), int(flags), _ptr(scores),
                                                _ptr(anchor_idx), _ptr(y), _stream()))
+
+    def predict_commit(self, h, h_rows, block_rows, batch, n_blk, final_norm_g, w_lm, vocab, threshold, token,
+                       confidence, commit):
+        self._check(self.lib.acache_predict_commit(self.h, _ptr(h), h_rows, _ptr(block_rows), batch, n_blk,
+                                                   _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold), _ptr(token),
+                                                   _ptr(confidence), _ptr(commit), _stream()))
 
     def layer_step_host(self, w: LayerWeights, req: Request, kv: KV, x_host, ratio, flags, scores_host,
                         anchor_idx_host, y_host):

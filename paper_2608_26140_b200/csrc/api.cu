@@ -22,7 +22,7 @@ struct acache_ctx {
     // workspace offsets (bytes)
     size_t o_status, o_row_pos, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
     size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
-    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar, o_mcidx;
+    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar, o_mcidx, o_lstats, o_lxn;
     std::string err;
     uint64_t launches = 0;
     // optional per-stage timing (acache_stage_timing)
@@ -229,7 +229,8 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
     *out = nullptr;
     const acache_model_desc& d = *desc;
     if (d.hidden <= 0 || d.n_heads <= 0 || d.n_kv_heads <= 0 || d.ffn <= 0 || d.max_batch <= 0 || d.max_ctx <= 0 ||
-        d.max_affix < 0 || d.max_rows < 0 || d.max_masked < 0 || !(d.rms_eps >= 0.f))
+        d.max_affix < 0 || d.max_rows < 0 || d.max_masked < 0 || d.max_vocab < 0 || d.max_block < 0 ||
+        !(d.rms_eps >= 0.f))
         return ACACHE_ERR_INVALID_ARG;
     if (d.head_dim != 64 && d.head_dim != 128) return ACACHE_ERR_UNSUPPORTED_SHAPE;
     if (d.n_heads % d.n_kv_heads) return ACACHE_ERR_UNSUPPORTED_SHAPE;
@@ -274,6 +275,12 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
         c->o_gemm = take(cur, pb);
     }
     c->o_attn = take(cur, attention_scratch_bytes(d.head_dim));
+    {
+        const size_t lrows = (size_t)d.max_batch * (d.max_block > 0 ? d.max_block : 0);
+        const size_t ltiles = d.max_vocab > 0 ? (size_t)(d.max_vocab + 255) / 256 : 0;
+        c->o_lstats = take(cur, lrows * ltiles * 16 * 16);
+        c->o_lxn = take(cur, lrows * d.hidden * 2);
+    }
     c->ws_need = cur;
     *out = c;
     return ACACHE_OK;
@@ -479,6 +486,40 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
         return run_recompute(ctx, w, req, kv, true, x, x_is_compact, anchor_idx, k, nullptr, nullptr, y, stream);
     mark(ctx, ACACHE_N_STAGES, stream);
     return check_cuda(ctx, "layer_step");
+}
+
+acache_status acache_predict_commit(acache_ctx* ctx, const void* h, int32_t h_rows, const int32_t* block_rows,
+                                    int32_t batch, int32_t n_blk, const void* final_norm_g, const void* w_lm,
+                                    int32_t vocab, float threshold, int32_t* token, float* confidence,
+                                    int32_t* commit, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!ctx->ws) return fail(ctx, ACACHE_ERR_WORKSPACE, "workspace not set");
+    const acache_model_desc& d = ctx->d;
+    if (batch < 0 || n_blk < 0 || h_rows <= 0 || vocab <= 0) return fail(ctx, ACACHE_ERR_INVALID_ARG, "negative size");
+    if ((int64_t)batch * n_blk > (int64_t)d.max_batch * d.max_block || vocab > d.max_vocab)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "batch * n_blk = %lld / vocab = %d exceed the context's limits (%lld, %d)",
+                    (long long)batch * n_blk, vocab, (long long)d.max_batch * d.max_block, d.max_vocab);
+    if (vocab % 128) return fail(ctx, ACACHE_ERR_UNSUPPORTED_SHAPE, "vocab %d is not a multiple of 128", vocab);
+    if (batch * n_blk == 0) return ACACHE_OK;
+    if (!h || !block_rows || !final_norm_g || !w_lm || !token || !confidence || !commit || !aligned16(h) ||
+        !aligned16(final_norm_g) || !aligned16(w_lm))
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL or misaligned pointer");
+    GemmArgs g{};
+    g.a = wsp<void>(ctx, ctx->o_lxn); g.M = batch * n_blk; g.K = d.hidden;
+    g.b[0] = w_lm; g.n[0] = vocab;
+    g.epilogue = kEpiLogits;
+    g.prep.enabled = 3; g.prep.x = h; g.prep.x_is_compact = 1; g.prep.compact_idx = block_rows; g.prep.compact_rows = h_rows;
+    g.prep.k = 0; g.prep.e = n_blk; g.prep.gain = final_norm_g; g.prep.eps = d.rms_eps;
+    g.logit_stats = wsp<float4>(ctx, ctx->o_lstats);
+    g.partial = wsp<float>(ctx, ctx->o_gemm); g.status = wsp<uint32_t>(ctx, ctx->o_status);
+    g.grid_bar = wsp<unsigned int>(ctx, ctx->o_gridbar);
+    int nl = launch_gemm(g, stream);
+    if (nl < 0) return check_cuda(ctx, "LM head") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "LM head launch failed") : ACACHE_ERR_CUDA;
+    ctx->launches += nl;
+    nl = launch_predict_commit(g, batch, n_blk, threshold, token, confidence, commit, stream);
+    if (nl < 0) return check_cuda(ctx, "predict/commit") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "predict/commit launch failed") : ACACHE_ERR_CUDA;
+    ctx->launches += nl;
+    return check_cuda(ctx, "predict_commit");
 }
 
 acache_status acache_layer_step_host(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,

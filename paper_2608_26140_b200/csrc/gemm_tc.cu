@@ -325,8 +325,28 @@ __device__ __forceinline__ void sum_slots16(const float* __restrict__ partial, c
     }
 }
 
+// Softmax statistics of W logits starting at vocabulary index col: running (max, sum exp(z - max),
+// arg max with the lowest index on ties).
+template <int W>
+__device__ __forceinline__ void logit_stats_update(const float (&v)[W], int col, float& m, float& s, int& arg) {
+    float cm = v[0];
+    int ca = 0;
+#pragma unroll
+    for (int i = 1; i < W; ++i)
+        if (v[i] > cm) { cm = v[i]; ca = i; }
+    if (cm > m) {
+        s *= __expf(m - cm);
+        m = cm;
+        arg = col + ca;
+    }
+#pragma unroll
+    for (int i = 0; i < W; ++i) s += __expf(v[i] - m);
+}
+
 // Work items of the finish per output tile: 16 output columns each (q/k/v: 16 of each rotary half).
-__host__ __device__ __forceinline__ int finish_items_per_tile(int epilogue) { return epilogue == kEpiResidual ? 16 : 8; }
+__host__ __device__ __forceinline__ int finish_items_per_tile(int epilogue) {
+    return (epilogue == kEpiResidual || epilogue == kEpiLogits) ? 16 : 8;
+}
 
 // Finish of one work item of split tile t = nt * m_tiles + mt for tile row `row`.
 __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, int t, int item, int row) {
@@ -336,8 +356,9 @@ __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, 
     tile_cover(p, t, c_first, c_last);
     const int half = g.head_dim >> 1;
     int pc0, pc1 = -1, u128 = 0, lo_col = 0;
-    if (g.epilogue == kEpiResidual) {
+    if (g.epilogue == kEpiResidual || g.epilogue == kEpiLogits) {
         pc0 = item * 4;
+        if (g.epilogue == kEpiLogits && nt * 2 + (item >> 3) >= p.units) return;   // past the vocabulary's end
     } else if (g.epilogue == kEpiSwiGLU) {
         pc0 = item * 4; pc1 = 32 + pc0;
     } else {
@@ -354,6 +375,11 @@ __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, 
     sum_slots16(g.partial, p, t, c_first, c_last, pc0, pc1, row, lo, hi);
     if (g.epilogue == kEpiResidual) {
         out_residual<16>(g, grow, nt * TC_BN + item * 16, lo);
+    } else if (g.epilogue == kEpiLogits) {
+        float m = -INFINITY, sm = 0.f;
+        int arg = 0;
+        logit_stats_update<16>(lo, nt * TC_BN + item * 16, m, sm, arg);
+        g.logit_stats[((int64_t)grow * p.n_tiles + nt) * 16 + item] = make_float4(m, sm, __int_as_float(arg), 0.f);
     } else if (g.epilogue == kEpiSwiGLU) {
         out_swiglu<16>(g, grow, nt * 128 + item * 16, lo, hi);
     } else {
@@ -373,6 +399,15 @@ __device__ __forceinline__ void direct_epilogue(const GemmArgs& g, const TcPlan&
             tc_ld32(taddr + c * 32, v);
             if (valid) out_residual<32>(g, grow, nt * TC_BN + c * 32, v);
         }
+    } else if (g.epilogue == kEpiLogits) {
+        float m = -INFINITY, sm = 0.f;
+        int arg = 0;
+        for (int c = 0; c < nchunks; ++c) {
+            float v[32];
+            tc_ld32(taddr + c * 32, v);
+            logit_stats_update<32>(v, nt * TC_BN + c * 32, m, sm, arg);
+        }
+        if (valid) g.logit_stats[((int64_t)grow * p.n_tiles + nt) * 16] = make_float4(m, sm, __int_as_float(arg), 0.f);
     } else if (g.epilogue == kEpiSwiGLU) {
         for (int c = 0; c < 4; ++c) {
             float gate[32], up[32];
@@ -441,6 +476,14 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
         const int rows_per_req = rp.k + rp.e;
         for (int row = blockIdx.x; row < g.M; row += gridDim.x) {
             int64_t src = (int64_t)row * g.K;
+            if (rp.enabled == 3) {       // compact rows picked by index
+                const int b = row / rows_per_req;
+                const int ci = rp.compact_idx[row];
+                if (ci < 0 || ci >= rp.compact_rows) {
+                    if (threadIdx.x == 0) atomicOr(g.status, kFlagBadIndex);
+                }
+                src = ((int64_t)b * rp.compact_rows + (ci < 0 || ci >= rp.compact_rows ? 0 : ci)) * g.K;
+            }
             if (rp.enabled == 1) {       // rows of R: position from the anchor / extra-row lists
                 const int b = row / rows_per_req, i = row - b * rows_per_req;
                 const int pos = row_position(rp.anchor_idx, rp.k, rp.extra_rows, rp.e, b, i, rp.affix_start,
@@ -611,6 +654,84 @@ __global__ void __launch_bounds__(256, 2) gemm_finish_kernel(const GemmArgs g, c
     finish_item(g, p, t, item, row);
 }
 
+// ---- predict and commit (Eq. 2-3): confidence and arg max per row, commit rule per request ------
+struct LogitAcc { float m, s; int arg; };
+__device__ __forceinline__ void logit_merge(LogitAcc& a, float m, float s, int arg) {
+    if (s == 0.f) return;            // an empty entry
+    if (m > a.m || (m == a.m && arg < a.arg && s > 0.f)) {
+        a.s = a.s * __expf(a.m - m) + s;
+        a.m = m;
+        a.arg = arg;
+    } else {
+        a.s += s * __expf(m - a.m);
+    }
+}
+
+// One CTA per row: merges the per-tile statistics (16 entries for a tile whose K range was split
+// between CTAs, one otherwise) in a fixed order.
+__global__ void __launch_bounds__(256) logit_reduce_kernel(const GemmArgs g, const TcPlan p, int32_t* __restrict__ token,
+                                                           float* __restrict__ confidence) {
+    __shared__ float sm_m[256], sm_s[256];
+    __shared__ int sm_a[256];
+    pdl_wait();
+    pdl_launch_dependents();
+    const int row = blockIdx.x, mt = row / TC_BM;
+    LogitAcc a{-INFINITY, 0.f, 0x7fffffff};
+    for (int nt = threadIdx.x; nt < p.n_tiles; nt += 256) {
+        int c_first, c_last;
+        tile_cover(p, nt * p.m_tiles + mt, c_first, c_last);
+        const int n_entries = c_first == c_last ? 1 : 16;
+        const float4* e = g.logit_stats + ((int64_t)row * p.n_tiles + nt) * 16;
+        for (int i = 0; i < n_entries; ++i) {
+            if (n_entries == 16 && nt * 2 + (i >> 3) >= p.units) break;
+            const float4 v = __ldcg(e + i);
+            logit_merge(a, v.x, v.y, __float_as_int(v.z));
+        }
+    }
+    sm_m[threadIdx.x] = a.m; sm_s[threadIdx.x] = a.s; sm_a[threadIdx.x] = a.arg;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) {
+            LogitAcc x{sm_m[threadIdx.x], sm_s[threadIdx.x], sm_a[threadIdx.x]};
+            logit_merge(x, sm_m[threadIdx.x + o], sm_s[threadIdx.x + o], sm_a[threadIdx.x + o]);
+            sm_m[threadIdx.x] = x.m; sm_s[threadIdx.x] = x.s; sm_a[threadIdx.x] = x.arg;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        token[row] = sm_a[0];
+        confidence[row] = 1.f / sm_s[0];       // softmax probability of the arg max
+    }
+}
+
+// One warp per request: commit the rows above the threshold, or the single most confident row
+// (lowest index on ties) if there is none.
+__global__ void __launch_bounds__(32) commit_kernel(const float* __restrict__ confidence, int n_blk, float threshold,
+                                                    int32_t* __restrict__ commit) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const float* c = confidence + (int64_t)b * n_blk;
+    int32_t* out = commit + (int64_t)b * n_blk;
+    int any = 0, best = 0x7fffffff;
+    float bestc = -INFINITY;
+    for (int i = lane; i < n_blk; i += 32) {
+        const float v = __ldcg(c + i);
+        const int f = v > threshold;
+        out[i] = f;
+        any |= f;
+        if (v > bestc) { bestc = v; best = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        any |= __shfl_xor_sync(0xffffffffu, any, o);
+        const float oc = __shfl_xor_sync(0xffffffffu, bestc, o);
+        const int ob = __shfl_xor_sync(0xffffffffu, best, o);
+        if (oc > bestc || (oc == bestc && ob < best)) { bestc = oc; best = ob; }
+    }
+    if (!any && lane == 0 && best < n_blk) out[best] = 1;
+}
+
 // ---- host side ------------------------------------------------------------------------------
 namespace {
 
@@ -690,6 +811,17 @@ size_t gemm_partial_bytes(int M, int K, int n_total, bool swiglu) {
     (void)M; (void)K; (void)n_total; (void)swiglu;
     // two fp32 partial tiles per CTA, at most one CTA per SM, whatever the problem size
     return (size_t)sm_count() * 2 * TC_SLOT_FLOATS * sizeof(float);
+}
+
+int launch_predict_commit(const GemmArgs& g, int batch, int n_blk, float threshold, int32_t* token, float* confidence,
+                          int32_t* commit, cudaStream_t stream) {
+    if (g.M == 0) return 0;
+    const TcPlan p = make_plan(g.M, g.K, g.n[0] / 128, false);
+    if (launch_pdl(logit_reduce_kernel, dim3(g.M), dim3(256), 0, stream, g, p, token, confidence) != cudaSuccess) return -1;
+    if (launch_pdl(commit_kernel, dim3(batch), dim3(32), 0, stream, (const float*)confidence, n_blk, threshold, commit) !=
+        cudaSuccess)
+        return -1;
+    return 2;
 }
 
 int launch_gemm(const GemmArgs& g, cudaStream_t stream) {

@@ -47,7 +47,8 @@ void launch_topk(float* scores, int batch, int affix_len, int k, int32_t* anchor
 enum GemmEpilogue : int {
     kEpiQKV = 0,     // bias + RoPE on q/k segments, bf16 stores to q / k_new / v_new (+ optional cache scatter)
     kEpiResidual,    // out = bf16(resid[row] + acc)
-    kEpiSwiGLU,      // out = bf16(silu(gate) * up), B tile = 64 gate rows + 64 up rows
+    kEpiSwiGLU,      // out = bf16(silu(gate) * up); B tile = 128 gate rows + 128 up rows
+    kEpiLogits,      // no tensor out: per (row, tile[, 16-column item]) softmax statistics (max, sum exp, argmax)
 };
 
 // Row plan of the recompute set R and RMSNorm of the gathered rows, run in front of a GEMM:
@@ -56,7 +57,8 @@ enum GemmEpilogue : int {
 // row_src = element offset of the row inside x, and the GEMM's A rows
 // xn = bf16(x * rsqrt(mean(x^2) + eps) * g).
 struct RowPrep {
-    int enabled;              // 0: off, 1: gather the rows of R, 2: the rows of x as they are (compact)
+    int enabled;              // 0: off, 1: gather the rows of R, 2: the rows of x as they are (compact),
+                              // 3: compact rows picked by compact_idx (no positions)
     const void* x;            // bf16 [B, ctx_len, hidden] or compact [B, k+e, hidden]
     int x_is_compact;
     int64_t x_batch_stride;
@@ -96,6 +98,8 @@ struct GemmArgs {
     const int64_t* resid_off; // [M] element offset of the residual row, or null => row * N
     // --- kEpiSwiGLU / kEpiResidual output ---
     void* c;                  // bf16 [M, Nout]
+    // --- kEpiLogits ---
+    float4* logit_stats;      // [M, n_tiles, 16] of (max, sum exp(z - max), argmax as int bits, -)
     // --- row work fused in front of the contraction ---
     RowPrep prep;             // writes the A rows (a) before the contraction
     // --- scratch ---
@@ -107,6 +111,12 @@ struct GemmArgs {
 // columns (SwiGLU: the MLP width) needs.
 size_t gemm_partial_bytes(int M, int K, int n_total, bool swiglu);
 int launch_gemm(const GemmArgs& g, cudaStream_t stream);      // kernels launched, or -1 if a launch failed
+
+// Softmax confidence and arg max of every row from the statistics a kEpiLogits GEMM left
+// (launch_gemm must have run with the same M, K, n_total), then the commit rule per request:
+// commit[b, i] = conf > threshold, and if no row of request b qualifies, its most confident row.
+int launch_predict_commit(const GemmArgs& g, int batch, int n_blk, float threshold, int32_t* token, float* confidence,
+                          int32_t* commit, cudaStream_t stream);
 
 // ---- attn.cu ----------------------------------------------------------------------------
 struct AttnArgs {

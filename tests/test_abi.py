@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def desc(**kw):
     d = dict(hidden=256, n_heads=4, n_kv_heads=4, head_dim=64, ffn=1024, rms_eps=1e-5, qkv_bias=0,
-             max_batch=2, max_ctx=256, max_affix=128, max_rows=64, max_masked=32)
+             max_batch=2, max_ctx=256, max_affix=128, max_rows=64, max_masked=32, max_vocab=0, max_block=0)
     d.update(kw)
     return ab.ModelDesc(*[d[f] for f, _ in ab.ModelDesc._fields_])
 

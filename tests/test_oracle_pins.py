@@ -453,6 +453,28 @@ def test_multilayer_probe_scores_and_ratio_zero_refresh():
     assert not np.allclose(s - s1, s1)
 
 
+def test_predict_commit_vs_library_softmax_and_rule():
+    g = np.random.default_rng(21)
+    n, D, V = 9, 32, 50
+    h = g.standard_normal((n, D))
+    gain = 1 + 0.1 * g.standard_normal(D)
+    W = g.standard_normal((V, D)) * 0.3
+    W[7] *= 6.0                                                 # one token some rows are sure about
+    h[2] = 4.0 * W[7] / np.linalg.norm(W[7]); h[5] = 5.0 * W[7] / np.linalg.norm(W[7])
+    tok, conf, commit, z = orc.predict_commit(h, gain, W, 1e-5, 0.9, round_storage=False)
+    hn = torch.nn.functional.rms_norm(torch.from_numpy(h), (D,), torch.from_numpy(gain), 1e-5)
+    p = torch.softmax(hn @ torch.from_numpy(W).T, dim=-1)
+    assert np.array_equal(tok, p.argmax(-1).numpy()) and np.allclose(conf, p.max(-1).values.numpy(), rtol=1e-12)
+    assert tok[2] == 7 and tok[5] == 7 and conf[5] > 0.9
+    assert np.array_equal(commit, conf > 0.9) and commit.any()
+    # nobody above the threshold: exactly the single most confident row commits
+    tok2, conf2, commit2, _ = orc.predict_commit(h, gain, W, 1e-5, 1.1, round_storage=False)
+    assert commit2.sum() == 1 and commit2[np.argmax(conf2)]
+    # closed forms: equal logits -> confidence 1/V and the lowest index; ties go to the lower row too
+    tok3, conf3, commit3, _ = orc.predict_commit(np.ones((3, D)), np.ones(D), np.zeros((V, D)), 1e-5, 0.9)
+    assert np.all(tok3 == 0) and np.allclose(conf3, 1.0 / V) and commit3.tolist() == [True, False, False]
+
+
 def test_comparators():
     ok, worst = orc.rel_err_gate(np.array([1.0, 2.0]), np.array([1.0, 2.0]))
     assert ok and worst == 0

@@ -50,7 +50,7 @@ def test_static_scratch_scoring_matches_workspace_scoring_twice_in_a_row():
 def test_static_scratch_rejects_oversized_problems_without_launching():
     shape = wl.LLADA_8B
     desc = ab.ModelDesc(shape.hidden, shape.n_heads, shape.n_kv_heads, shape.head_dim, shape.ffn, shape.rms_eps, 0,
-                        64, 40000, 40000, 1, 32)
+                        64, 40000, 40000, 1, 32, 0, 0)
     dummy = torch.zeros(1024, dtype=torch.bfloat16, device=DEV)
     masked = torch.zeros((64, 32), dtype=torch.int32, device=DEV)
     req = ab.Context.request(64, 40000, 0, 32768, masked, None, None, None)     # 64 * 32 * 32768 floats >> 2^20
