@@ -106,6 +106,10 @@ typedef struct {
     const int32_t *extra_rows;            /* DEVICE [B, n_extra] absolute positions outside F; may be NULL when n_extra == 0 */
     int32_t n_extra;
     const float *rope_cos, *rope_sin;     /* DEVICE fp32 [>= ctx_len, d/2] rotary table, pairing (i, i + d/2) */
+    const int32_t *token_ids;             /* optional DEVICE [B, ctx_len]: when set, the non-compact `x` of a call is an
+                                             embedding table bf16 [n_embed, D] and position t of request b reads row
+                                             token_ids[b, t] (an id outside [0, n_embed) raises ACACHE_FLAG_BAD_INDEX) */
+    int32_t n_embed;
 } acache_request;
 
 /* ---- context ------------------------------------------------------------------------ */
@@ -258,6 +262,22 @@ acache_status acache_predict_commit(acache_ctx *ctx, const void *h, int32_t h_ro
                                     int32_t batch, int32_t n_blk, const void *final_norm_g, const void *w_lm,
                                     int32_t vocab, float threshold, int32_t *token, float *confidence,
                                     int32_t *commit, acache_stream_t stream);
+
+/* One denoising step's model pass for a batch of requests (the "recompute forward" of Section 4.3
+ * followed by Eq. 2-3): the rows R = A u E of every request go through n_layers layers, each layer
+ * refreshing its cache rows exactly as acache_layer_step(flags = 0) does with the fixed anchor set;
+ * the last layer's rows named by block_rows then go through acache_predict_commit.
+ *   layers, kvs: HOST arrays of n_layers weight structs / cache descriptors (DEVICE pointers inside).
+ *   x0: DEVICE bf16 layer-0 input, [B, ctx_len, D], or the embedding table when req->token_ids is set.
+ *   y_a, y_b: DEVICE bf16 [B, K+e, D] each; layer outputs alternate between them, the last layer's
+ *             output is in *y_last (HOST pointer to a DEVICE pointer, may be NULL).
+ *   block_rows: DEVICE int32 [B, n_blk] compact rows (in [0, K+e)) of the current block's masked positions. */
+acache_status acache_denoise_step(acache_ctx *ctx, int32_t n_layers, const acache_layer_weights *layers,
+                                  acache_kv *kvs, const acache_request *req, const void *x0,
+                                  const int32_t *anchor_idx, int32_t k, void *y_a, void *y_b, void **y_last,
+                                  const int32_t *block_rows, int32_t n_blk, const void *final_norm_g,
+                                  const void *w_lm, int32_t vocab, float threshold, int32_t *token,
+                                  float *confidence, int32_t *commit, acache_stream_t stream);
 
 /* acache_layer_step for a caller whose per-step data lives in HOST memory: copies
  * x [B, ctx_len, D] (HOST bf16, ideally pinned) to a staging area in the workspace,

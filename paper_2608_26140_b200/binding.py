@@ -22,7 +22,7 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_last_error", "acache_poll_status", "acache_launch_count", "acache_score_anchors",
            "acache_k_from_ratio", "acache_select_topk", "acache_recompute_anchors", "acache_scatter_kv",
            "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times",
-           "acache_score_anchors_static", "acache_predict_commit"]
+           "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -48,7 +48,7 @@ class Request(C.Structure):
     _fields_ = [("batch", C.c_int32), ("ctx_len", C.c_int32), ("affix_start", C.c_int32),
                 ("affix_len", C.c_int32), ("masked_pos", C.c_void_p), ("n_masked", C.c_int32),
                 ("extra_rows", C.c_void_p), ("n_extra", C.c_int32), ("rope_cos", C.c_void_p),
-                ("rope_sin", C.c_void_p)]
+                ("rope_sin", C.c_void_p), ("token_ids", C.c_void_p), ("n_embed", C.c_int32)]
 
 
 class AcacheError(RuntimeError):
@@ -107,6 +107,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_score_anchors_static.restype = C.c_int
     lib.acache_predict_commit.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, i32, C.c_float, vp, vp, vp, vp]
     lib.acache_predict_commit.restype = C.c_int
+    lib.acache_denoise_step.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request), vp, vp, i32,
+                                        vp, vp, C.POINTER(vp), vp, i32, vp, vp, i32, C.c_float, vp, vp, vp, vp]
+    lib.acache_denoise_step.restype = C.c_int
     lib.acache_stage_timing.argtypes = [vp, C.c_int]
     lib.acache_stage_timing.restype = C.c_int
     lib.acache_read_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
@@ -200,11 +203,12 @@ class Context:
         return KV(cache_k.data_ptr(), cache_v.data_ptr(), cap * hkv * d, cap)
 
     @staticmethod
-    def request(batch, ctx_len, affix_start, affix_len, masked_pos, extra_rows, rope_cos, rope_sin) -> Request:
+    def request(batch, ctx_len, affix_start, affix_len, masked_pos, extra_rows, rope_cos, rope_sin,
+                token_ids=None, n_embed=0) -> Request:
         nm = 0 if masked_pos is None else int(masked_pos.shape[1])
         ne = 0 if extra_rows is None else int(extra_rows.shape[1])
         return Request(batch, ctx_len, affix_start, affix_len, _ptr(masked_pos) if nm else None, nm,
-                       _ptr(extra_rows) if ne else None, ne, _ptr(rope_cos), _ptr(rope_sin))
+                       _ptr(extra_rows) if ne else None, ne, _ptr(rope_cos), _ptr(rope_sin), _ptr(token_ids), n_embed)
 
     # ---- entry points ----
     def launch_count(self) -> int:
@@ -254,6 +258,19 @@ class Context:
         self._check(self.lib.acache_predict_commit(self.h, _ptr(h), h_rows, _ptr(block_rows), batch, n_blk,
                                                    _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold), _ptr(token),
                                                    _ptr(confidence), _ptr(commit), _stream()))
+
+    def denoise_step(self, layers, kvs, req: Request, x0, anchor_idx, k, y_a, y_b, block_rows, n_blk, final_norm_g,
+                     w_lm, vocab, threshold, token, confidence, commit) -> int:
+        """layers: list of LayerWeights, kvs: list of KV.  Returns the device address of the last layer's output."""
+        n = len(layers)
+        la = (LayerWeights * n)(*layers)
+        ka = (KV * n)(*kvs)
+        last = C.c_void_p()
+        self._check(self.lib.acache_denoise_step(self.h, n, la, ka, C.byref(req), _ptr(x0), _ptr(anchor_idx), k,
+                                                 _ptr(y_a), _ptr(y_b), C.byref(last), _ptr(block_rows), n_blk,
+                                                 _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold), _ptr(token),
+                                                 _ptr(confidence), _ptr(commit), _stream()))
+        return last.value
 
     def layer_step_host(self, w: LayerWeights, req: Request, kv: KV, x_host, ratio, flags, scores_host,
                         anchor_idx_host, y_host):

@@ -161,6 +161,7 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     g.prep.anchor_idx = anchor_idx; g.prep.k = k; g.prep.extra_rows = r->extra_rows; g.prep.e = r->n_extra;
     g.prep.affix_start = r->affix_start; g.prep.affix_len = r->affix_len; g.prep.ctx_len = r->ctx_len;
     g.prep.gain = w->attn_norm_g; g.prep.eps = d.rms_eps; g.prep.row_pos = row_pos; g.prep.row_src = row_src;
+    if (!x_is_compact && r->token_ids) { g.prep.token_ids = r->token_ids; g.prep.table_rows = r->n_embed; }
     g.b[0] = w->wq; g.b[1] = w->wk; g.b[2] = w->wv;
     g.n[0] = qd; g.n[1] = kvd; g.n[2] = kvd;
     g.epilogue = kEpiQKV;
@@ -458,6 +459,7 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
             g.prep.affix_start = req->affix_start; g.prep.affix_len = req->affix_len; g.prep.ctx_len = req->ctx_len;
             g.prep.gain = w->attn_norm_g; g.prep.eps = d.rms_eps; g.prep.row_pos = mpos;
             g.prep.row_src = wsp<int64_t>(ctx, ctx->o_mrow_src);
+            if (!x_is_compact && req->token_ids) { g.prep.token_ids = req->token_ids; g.prep.table_rows = req->n_embed; }
             g.b[0] = w->wq; g.n[0] = d.n_heads * d.head_dim;
             g.epilogue = kEpiQKV;
             g.bias[0] = d.qkv_bias ? w->bq : nullptr;
@@ -520,6 +522,36 @@ acache_status acache_predict_commit(acache_ctx* ctx, const void* h, int32_t h_ro
     if (nl < 0) return check_cuda(ctx, "predict/commit") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "predict/commit launch failed") : ACACHE_ERR_CUDA;
     ctx->launches += nl;
     return check_cuda(ctx, "predict_commit");
+}
+
+acache_status acache_denoise_step(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers,
+                                  acache_kv* kvs, const acache_request* req, const void* x0,
+                                  const int32_t* anchor_idx, int32_t k, void* y_a, void* y_b, void** y_last,
+                                  const int32_t* block_rows, int32_t n_blk, const void* final_norm_g,
+                                  const void* w_lm, int32_t vocab, float threshold, int32_t* token,
+                                  float* confidence, int32_t* commit, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (n_layers <= 0 || !layers || !kvs || !req || !x0 || !y_a || !y_b)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL argument or n_layers <= 0");
+    if (k < 0 || k > req->affix_len) return fail(ctx, ACACHE_ERR_INVALID_ARG, "k %d outside [0, affix_len]", k);
+    // the ratio that maps back to exactly k anchors
+    const double ratio = req->affix_len > 0 ? ((double)k - 0.5) / (double)req->affix_len : 0.0;
+    if (acache_k_from_ratio(req->affix_len, k > 0 ? ratio : 0.0) != k) return fail(ctx, ACACHE_ERR_INVALID_ARG, "k not representable");
+    const void* x = x0;
+    void* y = y_a;
+    for (int n = 0; n < n_layers; ++n) {
+        y = (n & 1) ? y_b : y_a;
+        acache_status s = acache_layer_step(ctx, &layers[n], req, &kvs[n], x, n > 0, k > 0 ? ratio : 0.0, 0u, nullptr,
+                                            const_cast<int32_t*>(anchor_idx), y, stream);
+        if (s != ACACHE_OK) return s;
+        x = y;
+    }
+    if (y_last) *y_last = y;
+    const int rows = k + req->n_extra;
+    if (n_blk == 0 || req->batch == 0) return ACACHE_OK;
+    if (rows == 0) return fail(ctx, ACACHE_ERR_INVALID_ARG, "no rows were recomputed: nothing to predict from");
+    return acache_predict_commit(ctx, y, rows, block_rows, req->batch, n_blk, final_norm_g, w_lm, vocab, threshold, token,
+                                 confidence, commit, stream);
 }
 
 acache_status acache_layer_step_host(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,

@@ -489,7 +489,16 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
                 const int pos = row_position(rp.anchor_idx, rp.k, rp.extra_rows, rp.e, b, i, rp.affix_start,
                                              rp.affix_len, rp.ctx_len);
                 if (!rp.x_is_compact) {
-                    src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
+                    if (rp.token_ids) {       // x is an embedding table: the row of the token at that position
+                        int id = rp.token_ids[(int64_t)b * rp.ctx_len + (pos < 0 ? 0 : pos)];
+                        if (id < 0 || id >= rp.table_rows) {
+                            if (threadIdx.x == 0) atomicOr(g.status, kFlagBadIndex);
+                            id = 0;
+                        }
+                        src = (int64_t)id * g.K;
+                    } else {
+                        src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
+                    }
                 } else if (rp.compact_idx) {
                     const int ci = rp.compact_idx[row];
                     src = ((int64_t)b * rp.compact_rows + (ci < 0 ? 0 : ci)) * g.K;

@@ -62,6 +62,8 @@ struct RowPrep {
     const void* x;            // bf16 [B, ctx_len, hidden] or compact [B, k+e, hidden]
     int x_is_compact;
     int64_t x_batch_stride;
+    const int32_t* token_ids;    // optional [B, ctx_len]: x is an embedding table [table_rows, hidden] indexed by token id
+    int table_rows;
     const int32_t* compact_idx;  // optional [B, k+e]: row i reads compact row compact_idx[..] of its request
     int compact_rows;            // rows per request of the compact x that compact_idx points into
     const int32_t* anchor_idx;

@@ -66,7 +66,7 @@ def test_workspace_grows_with_problem_size(lib):
 def test_calls_without_workspace_are_rejected_before_any_launch(lib):
     h = C.c_void_p()
     lib.acache_create(C.byref(desc()), C.byref(h))
-    req = ab.Request(1, 256, 0, 128, None, 0, None, 0, None, None)
+    req = ab.Request(1, 256, 0, 128, None, 0, None, 0, None, None, None, 0)
     kv = ab.KV(None, None, 0, 256)
     st = lib.acache_score_anchors(h, C.byref(req), None, C.byref(kv), None, 0, 0, None)
     assert st == ab.ERR_WORKSPACE

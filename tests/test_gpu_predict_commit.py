@@ -65,3 +65,68 @@ def test_predict_commit(shape, V, B, h_rows, n_blk):
     if B > 1:
         assert commit[B - 1].sum().item() == 1                  # the fallback path was exercised
     assert (commit[0] != 0).sum().item() >= 1
+
+
+def test_denoise_step_two_layers_with_embedding_lookup():
+    """acache_denoise_step: token ids -> embedding rows -> two refresh layers with a fixed anchor set ->
+    LM head + commit, against the oracle's refresh_forward + predict_commit."""
+    shape, n_layers, B, V = wl.TINY_GQA, 2, 2, 640
+    lay = wl.make_layout(B, 4, 64, 12, 32, 32, "all")
+    T, l, L, P = lay.ctx_len, lay.affix_start, lay.affix_len, lay.n_extra
+    K = 16
+    g = np.random.default_rng(5)
+    layers = [wl.layer_weights(shape, 41, n) for n in range(n_layers)]
+    embed = wl.normal_bf16(7101, (V, shape.hidden), 1.0)
+    w_lm = wl.normal_bf16(7102, (V, shape.hidden), 0.02)
+    gain = wl.normal_bf16(7103, (shape.hidden,), 0.05, 1.0)
+    ids = g.integers(0, V, size=(B, T)).astype(np.int32)
+    ids[:, l:l + L] = ids[0, l:l + L]                               # the affix text is shared
+    x0 = embed[ids]                                                 # [B, T, D] bf16 bits
+    cos, sin = wl.rope_table(T, shape.head_dim, shape.rope_theta)
+    caches = [[wl.random_kv_cache(shape, wl.make_layout(1, 4, 64, 12, 32, 32, "all"), 900 + 10 * n + b) for n in range(n_layers)]
+              for b in range(B)]
+    caches = [[(ck[0], cv[0]) for (ck, cv) in per_b] for per_b in caches]
+    anchors = np.stack([np.sort(g.choice(L, K, replace=False)) for _ in range(B)]).astype(np.int32)
+    # current block = the masked rows; their compact rows: anchors first, then extras in order
+    where = {int(p): i for i, p in enumerate(lay.extra_rows[0])}
+    block_rows = np.stack([[K + where[int(p)] for p in lay.masked_pos[b]] for b in range(B)]).astype(np.int32)
+    n_blk = block_rows.shape[1]
+
+    ctx = ab.Context.for_shape(shape, B, T, L, K + P, lay.n_masked, DEV, max_vocab=V, max_block=n_blk)
+    dl = [{k: (ab.to_device_bf16(v, DEV) if v is not None else None) for k, v in w.items()} for w in layers]
+    lws = [ab.Context.weights(w) for w in dl]
+    dk = [ab.to_device_bf16(np.stack([caches[b][n][0] for b in range(B)]), DEV) for n in range(n_layers)]
+    dv = [ab.to_device_bf16(np.stack([caches[b][n][1] for b in range(B)]), DEV) for n in range(n_layers)]
+    kvs = [ab.Context.kv(dk[n], dv[n]) for n in range(n_layers)]
+    dcos, dsin = torch.from_numpy(cos).to(DEV), torch.from_numpy(sin).to(DEV)
+    masked = torch.from_numpy(lay.masked_pos.copy()).to(DEV)
+    extra = torch.from_numpy(lay.extra_rows.copy()).to(DEV)
+    dids = torch.from_numpy(ids).to(DEV)
+    req = ab.Context.request(B, T, l, L, masked, extra, dcos, dsin, token_ids=dids, n_embed=V)
+    de, dw, dg = ab.to_device_bf16(embed, DEV), ab.to_device_bf16(w_lm, DEV), ab.to_device_bf16(gain, DEV)
+    ya = torch.zeros((B, K + P, shape.hidden), dtype=torch.bfloat16, device=DEV)
+    yb = torch.zeros_like(ya)
+    da, dbr = torch.from_numpy(anchors).to(DEV), torch.from_numpy(block_rows).to(DEV)
+    token = torch.full((B, n_blk), -1, dtype=torch.int32, device=DEV)
+    conf = torch.zeros((B, n_blk), dtype=torch.float32, device=DEV)
+    commit = torch.full((B, n_blk), -1, dtype=torch.int32, device=DEV)
+    last = ctx.denoise_step(lws, kvs, req, de, da, K, ya, yb, dbr, n_blk, dg, dw, V, 0.9, token, conf, commit)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    assert last == yb.data_ptr()                                    # two layers: a then b
+    from helpers import TOL, assert_close_bf16
+    for b in range(B):
+        rows, ref_caches, ys = orc.refresh_forward(layers, shape, x0[b], caches[b], T, l, anchors[b], lay.extra_rows[b],
+                                                   cos, sin)
+        assert_close_bf16(ab.to_host_bits(yb[b]), ys[-1], "last layer output", 2 * TOL)
+        for n in range(n_layers):
+            assert_close_bf16(ab.to_host_bits(dk[n][b])[rows], ref_caches[n][0][rows], f"layer {n} K", 2 * TOL)
+        # teacher-forced head: the oracle's head on the GPU's own last-layer rows
+        hrows = orc.bf16_bits_to_f64(ab.to_host_bits(yb[b]))[block_rows[b]]
+        tok, cf, cm, z = orc.predict_commit(hrows, gain, w_lm, shape.rms_eps, 0.9)
+        zs = np.sort(z, axis=1)
+        clear = (zs[:, -1] - zs[:, -2]) > 1e-3 * np.abs(zs[:, -1]).clip(1e-3)
+        assert np.array_equal(token.cpu().numpy()[b][clear], tok[clear]) and clear.mean() > 0.8
+        assert np.allclose(conf.cpu().numpy()[b], cf, rtol=2e-3)
+        assert commit[b].sum().item() == cm.sum() == 1              # random weights: nobody is confident
+        assert cf[int(np.argmax(commit.cpu().numpy()[b]))] >= cf.max() * (1 - 2e-3)
