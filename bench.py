@@ -328,6 +328,159 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------
+def run_denoise(args):
+    """Benchmark configuration 3: one denoising step's model pass = 32 LLaDA-8B layers refreshing
+    R = anchors + all request rows of 16 requests that share a 2048-token affix, then final norm,
+    LM head and the commit rule on the current 32-token block (acache_denoise_step)."""
+    import torch
+    from paper_2608_26140_b200 import binding as ab
+    from paper_2608_26140_b200 import build as abuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        abuild.build()
+    if dist:
+        dist.barrier()
+    shape, n_layers, V, n_blk = wl.LLADA_8B, args.layers, 126464, 32
+    lay = wl.config_layout(3, "all", n_masked=32, batch=args.batch)
+    B, T, L, P = lay.batch, lay.ctx_len, lay.affix_len, lay.n_extra
+    K = ab.k_from_ratio(L, RATIO)
+    n = K + P
+    # 4 seeded weight sets tiled over the layers, one seeded cache replicated per layer (distinct
+    # device buffers, so nothing is shared or cached between layers)
+    host_sets = [wl.layer_weights(shape, 3, i) for i in range(min(4, n_layers))]
+    dev_sets = [{k: (ab.to_device_bf16(v, dev) if v is not None else None) for k, v in w.items()} for w in host_sets]
+    layers_dev, lws = [], []
+    for i in range(n_layers):
+        w = {k: (v.clone() if v is not None else None) for k, v in dev_sets[i % len(dev_sets)].items()} if i >= len(dev_sets) \
+            else dev_sets[i]
+        layers_dev.append(w)
+        lws.append(ab.Context.weights(w))
+    ck, cv = wl.random_kv_cache(shape, lay, wl.SEED_BASE + 4096 * 3 + 30)
+    ck0, cv0 = ab.to_device_bf16(ck, dev), ab.to_device_bf16(cv, dev)
+    dk = [ck0] + [ck0.clone() for _ in range(n_layers - 1)]
+    dv = [cv0] + [cv0.clone() for _ in range(n_layers - 1)]
+    kvs = [ab.Context.kv(dk[i], dv[i]) for i in range(n_layers)]
+    embed = ab.to_device_bf16(wl.normal_bf16(wl.SEED_BASE + 4096 * 3 + 40, (V, shape.hidden), 1.0), dev)
+    w_lm = ab.to_device_bf16(wl.normal_bf16(wl.SEED_BASE + 4096 * 3 + 41, (V, shape.hidden), 0.02), dev)
+    gain = ab.to_device_bf16(wl.normal_bf16(wl.SEED_BASE + 4096 * 3 + 42, (shape.hidden,), 0.05, 1.0), dev)
+    g = np.random.Generator(np.random.Philox(wl.SEED_BASE + 4096 * 3 + 43))
+    ids = g.integers(0, V - 1, size=(B, T)).astype(np.int32)
+    ids[:, lay.affix_start:lay.affix_start + L] = ids[0, lay.affix_start:lay.affix_start + L]
+    ids[:, lay.masked_pos[0]] = V - 1                              # mask id
+    anchors = np.stack([np.sort(g.choice(L, K, replace=False)) for _ in range(B)]).astype(np.int32)
+    where = {int(p): i for i, p in enumerate(lay.extra_rows[0])}
+    block_rows = np.stack([[K + where[int(p)] for p in lay.masked_pos[b][:n_blk]] for b in range(B)]).astype(np.int32)
+    cos_h, sin_h = wl.rope_table(T, shape.head_dim, shape.rope_theta)
+    cos, sin = torch.from_numpy(cos_h).to(dev), torch.from_numpy(sin_h).to(dev)
+    masked = torch.from_numpy(lay.masked_pos.copy()).to(dev)
+    extra = torch.from_numpy(lay.extra_rows.copy()).to(dev)
+    dids = torch.from_numpy(ids).to(dev)
+    req = ab.Context.request(B, T, lay.affix_start, L, masked, extra, cos, sin, token_ids=dids, n_embed=V)
+    ctx = ab.Context.for_shape(shape, B, T, L, n, lay.n_masked, dev, max_vocab=V, max_block=n_blk)
+    ya = torch.zeros((B, n, shape.hidden), dtype=torch.bfloat16, device=dev)
+    yb = torch.zeros_like(ya)
+    da, dbr = torch.from_numpy(anchors).to(dev), torch.from_numpy(block_rows).to(dev)
+    token = torch.zeros((B, n_blk), dtype=torch.int32, device=dev)
+    conf = torch.zeros((B, n_blk), dtype=torch.float32, device=dev)
+    commit = torch.zeros((B, n_blk), dtype=torch.int32, device=dev)
+
+    def step():
+        ctx.denoise_step(lws, kvs, req, embed, da, K, ya, yb, dbr, n_blk, gain, w_lm, V, 0.9, token, conf, commit)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sync_all()
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    sync_all()
+    sampler.stop_flag = True
+    sampler.join()
+    launches = ctx.launch_count() - l0
+    ms_step = sharding.max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    assert ctx.poll_status() == 0
+    # end to end: token ids come from the host every step, tokens / confidence / commit flags go back
+    ids_h = torch.from_numpy(ids).pin_memory()
+    tok_h, conf_h, com_h = (torch.zeros((B, n_blk), dtype=torch.int32).pin_memory(),
+                            torch.zeros((B, n_blk), dtype=torch.float32).pin_memory(),
+                            torch.zeros((B, n_blk), dtype=torch.int32).pin_memory())
+
+    def step_host():
+        dids.copy_(ids_h, non_blocking=True)
+        step()
+        tok_h.copy_(token, non_blocking=True); conf_h.copy_(conf, non_blocking=True); com_h.copy_(commit, non_blocking=True)
+
+    for _ in range(2):
+        step_host()
+    sync_all()
+    e0.record()
+    for _ in range(args.steps):
+        step_host()
+    e1.record()
+    sync_all()
+    ms_e2e = sharding.max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    peaks = load_peaks()
+    lay1 = lay
+    step_bytes, step_flops, gu_bytes, gu_flops, n_r = step_work(shape, lay1, K)
+    # no scoring in a refresh step: drop the masked-row projection and the score pass
+    D, H, d = shape.hidden, shape.n_heads, shape.head_dim
+    layer_flops = step_flops - 2 * B * lay.n_masked * D * H * d - 4 * B * lay.n_masked * L * H * d
+    head_flops = 2 * B * n_blk * D * V
+    flops = n_layers * layer_flops + head_flops
+    bytes_ = n_layers * step_bytes + 2 * V * D
+    floor_s = max(flops / (peaks["tflops"] * 1e12), bytes_ / (peaks["hbm_gbs"] * 1e9))
+    out = {
+        "metric": "denoise_steps_per_s", "value": world / (ms_step * 1e-3), "unit": "denoising steps/s (model pass + commit)",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic; 4 seeded layer weight sets tiled over the layers, one seeded cache replicated per layer",
+        "config": {"workload": f"cfg3: LLaDA-8B shapes, {n_layers} layers, vocab {V}, batch {B}/GPU sharing a {L}-token prefix "
+                               f"affix, {P} request rows each, ratio {RATIO} (K={K}), {n} rows recomputed per request, "
+                               f"{n_blk}-token block", "benchmark_config": 3, "layers": n_layers,
+                   "l2": "per-layer weights (436 MB) exceed L2; every layer has its own weight and cache buffers",
+                   "parallelism": f"request-sharded x{world}"},
+        "clocks": sampler.summary(),
+        "e2e": {"value": world / (ms_e2e * 1e-3), "unit": "denoising steps/s", "h2d_bytes_per_step": int(ids_h.numel() * 4),
+                "d2h_bytes_per_step": int(3 * B * n_blk * 4)},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "whole step (tensor-bound)", "bound": "tensor", "achieved": flops / (ms_step * 1e-3) / 1e12,
+                     "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": floor_s / (ms_step * 1e-3),
+                     "peak_source": peaks["source"], "traffic": None, "algorithmic_flops": flops, "algorithmic_bytes": bytes_},
+        "affix_tokens_refreshed_per_s": world * B * K * n_layers / (ms_step * 1e-3),
+        "ms_per_layer": (ms_step) / n_layers,
+    }
+    print(json.dumps(out))
+    if dist:
+        dist.destroy_process_group()
+
+
 def cpu_baseline(case, shape, lay):
     """The oracle as it stands, timed on this machine's host cores on one step of the workload."""
     from oracle import acache_oracle as orc
@@ -361,9 +514,12 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--instances", type=int, default=4, help="weight/cache instances rotated between steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=32, help="layers of the --config 3 denoising step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.config == 3:
+        run_denoise(args)
     else:
         run_ours(args)
 
