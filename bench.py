@@ -33,9 +33,10 @@ METRIC = "anchor_refresh_affix_tokens_per_s"
 UNIT = "affix tokens/s"
 RATIO = 0.2
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the gate/up GEMM at this
-# workload, from one ncu capture (summary under profiles/); None until captured.
-NCU_TRAFFIC_BYTES = {"gate_up": None}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the gate/up GEMM at the default
+# workload (configuration 2, anchors only), from one ncu capture: 202.36 MB read + 5.98 MB written
+# (profiles/layer_step_cfg2_tcgen05.md).  Not captured for other workloads.
+NCU_TRAFFIC_BYTES = {"gate_up": 208334848}
 
 
 def load_peaks():
@@ -301,7 +302,8 @@ def run_ours(args):
         ach, peak, unit = gu_flops / gu_s / 1e12, peaks["tflops"], "TFLOP/s"
     roofline = {"kernel": "gate/up projection + SwiGLU (stage gate_up)", "bound": "hbm" if gu_hbm_bound else "tensor",
                 "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "peak_source": peaks["source"],
-                "traffic": NCU_TRAFFIC_BYTES["gate_up"], "algorithmic_bytes": gu_bytes, "algorithmic_flops": gu_flops,
+                "traffic": NCU_TRAFFIC_BYTES["gate_up"] if (args.config == 2 and lay.n_extra == 0 and B == 1) else None,
+                "algorithmic_bytes": gu_bytes, "algorithmic_flops": gu_flops,
                 "us_per_launch": stage["gate_up"] * 1e3}
     floor_s = max(t_hbm, t_tc)
     value = sharding.aggregate_throughput(B * K, world, ms_step)
