@@ -103,6 +103,9 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
         : "memory");
 }
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
+}
 __device__ __forceinline__ void st_hint_f4(float4* p, float4 v, uint64_t policy) {
     asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
                  ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy)
@@ -466,7 +469,33 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    // everything above overlaps the previous kernel's tail; global memory is touched only below
+    const int it0 = blockIdx.x * p.U;
+    const int it1 = min(it0 + p.U, p.tiles * p.KB);
+    // The weights are constant inputs (no earlier kernel writes them), so their loads may start
+    // before the previous kernel has finished: fill the ring's weight halves now and ask L2 for the
+    // k-blocks after that.  The activation halves follow once the producer kernel is done.
+    constexpr int kPrefetchL2 = 12;
+    int prefilled = 0;
+    if (warp == 0 && lane == 0) {
+        const CUtensorMap* maps[3] = {&mapB0, &mapB1, &mapB2};
+        const uint64_t pol_w = policy_evict_first();
+        for (int i = 0; i < TC_STAGES + kPrefetchL2 && it0 + i < it1; ++i) {
+            const int it = it0 + i, t = it / p.KB, kb = it - t * p.KB, nt = t / p.m_tiles;
+            int row0, row1;
+            const int s0 = half_source(g, p, nt, 0, row0), s1 = half_source(g, p, nt, 1, row1);
+            if (i < TC_STAGES) {
+                const uint32_t sB = base + i * TC_STAGE_BYTES + TC_A_BYTES;
+                mbar_expect_tx(full_bar(i), TC_A_BYTES + TC_HALF_BYTES * (1 + (s1 >= 0)));
+                tma_load_2d(sB, maps[s0], kb * TC_BK, row0, full_bar(i), pol_w);
+                if (s1 >= 0) tma_load_2d(sB + TC_HALF_BYTES, maps[s1], kb * TC_BK, row1, full_bar(i), pol_w);
+                prefilled = i + 1;
+            } else {
+                tma_prefetch_2d(maps[s0], kb * TC_BK, row0);
+                if (s1 >= 0) tma_prefetch_2d(maps[s1], kb * TC_BK, row1);
+            }
+        }
+    }
+    // everything above overlaps the previous kernel's tail; its outputs are touched only below
     pdl_wait();
     pdl_launch_dependents();
 
@@ -520,8 +549,6 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     }
 
     // ---------------- phase 1: the contraction ----------------
-    const int it0 = blockIdx.x * p.U;
-    const int it1 = min(it0 + p.U, p.tiles * p.KB);
 
     if (warp == 0 && lane == 0) {
         // TMA producer
@@ -538,12 +565,17 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
             const int s0 = half_source(g, p, nt, 0, row0), s1 = half_source(g, p, nt, 1, row1);
             const uint32_t bytes = TC_A_BYTES + TC_HALF_BYTES * (1 + (s1 >= 0));
             for (int kb = kb0; kb < kb1; ++kb) {
-                if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag))) break;
                 const uint32_t sA = base + stage * TC_STAGE_BYTES, sB = sA + TC_A_BYTES;
-                mbar_expect_tx(full_bar(stage), bytes);
-                tma_load_2d(sA, &mapA, kb * TC_BK, mt * TC_BM, full_bar(stage), pol_a);
-                tma_load_2d(sB, maps[s0], kb * TC_BK, row0, full_bar(stage), pol_w);
-                if (s1 >= 0) tma_load_2d(sB + TC_HALF_BYTES, maps[s1], kb * TC_BK, row1, full_bar(stage), pol_w);
+                if (prefilled > 0) {          // this stage's weight halves are already on their way
+                    --prefilled;
+                    tma_load_2d(sA, &mapA, kb * TC_BK, mt * TC_BM, full_bar(stage), pol_a);
+                } else {
+                    if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag))) break;
+                    mbar_expect_tx(full_bar(stage), bytes);
+                    tma_load_2d(sA, &mapA, kb * TC_BK, mt * TC_BM, full_bar(stage), pol_a);
+                    tma_load_2d(sB, maps[s0], kb * TC_BK, row0, full_bar(stage), pol_w);
+                    if (s1 >= 0) tma_load_2d(sB + TC_HALF_BYTES, maps[s1], kb * TC_BK, row1, full_bar(stage), pol_w);
+                }
                 if (++stage == TC_STAGES) { stage = 0; phase ^= 1; }
             }
             it += kb1 - kb0;
