@@ -23,6 +23,7 @@
 // returns.  The grid never exceeds the SM count, so all CTAs are resident for the barrier.
 #include <cuda.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -436,6 +437,56 @@ __device__ __forceinline__ void direct_epilogue(const GemmArgs& g, const TcPlan&
     }
 }
 
+// Phase 0 of the projection kernels: the rows of R (or compact rows) -> RMSNorm -> the A operand,
+// one row per CTA at a time, then a grid-wide barrier; the rows are read back through TMA.
+__device__ __forceinline__ void prep_phase(const GemmArgs& g, float* red, volatile int* abort_flag, unsigned int& nbar) {
+    const RowPrep& rp = g.prep;
+    const int rows_per_req = rp.k + rp.e;
+    for (int row = blockIdx.x; row < g.M; row += gridDim.x) {
+        int64_t src = (int64_t)row * g.K;
+        if (rp.enabled == 3) {       // compact rows picked by index
+            const int b = row / rows_per_req;
+            const int ci = rp.compact_idx[row];
+            if (ci < 0 || ci >= rp.compact_rows) {
+                if (threadIdx.x == 0) atomicOr(g.status, kFlagBadIndex);
+            }
+            src = ((int64_t)b * rp.compact_rows + (ci < 0 || ci >= rp.compact_rows ? 0 : ci)) * g.K;
+        }
+        if (rp.enabled == 1) {       // rows of R: position from the anchor / extra-row lists
+            const int b = row / rows_per_req, i = row - b * rows_per_req;
+            const int pos = row_position(rp.anchor_idx, rp.k, rp.extra_rows, rp.e, b, i, rp.affix_start,
+                                         rp.affix_len, rp.ctx_len);
+            if (!rp.x_is_compact) {
+                if (rp.token_ids) {       // x is an embedding table: the row of the token at that position
+                    int id = rp.token_ids[(int64_t)b * rp.ctx_len + (pos < 0 ? 0 : pos)];
+                    if (id < 0 || id >= rp.table_rows) {
+                        if (threadIdx.x == 0) atomicOr(g.status, kFlagBadIndex);
+                        id = 0;
+                    }
+                    src = (int64_t)id * g.K;
+                } else {
+                    src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
+                }
+            } else if (rp.compact_idx) {
+                const int ci = rp.compact_idx[row];
+                src = ((int64_t)b * rp.compact_rows + (ci < 0 ? 0 : ci)) * g.K;
+            }
+            if (threadIdx.x == 0) {
+                rp.row_pos[row] = pos;
+                rp.row_src[row] = src;
+                if (pos < 0) atomicOr(g.status, kFlagBadIndex);
+            }
+        }
+        rmsnorm_row(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(rp.x) + src),
+                    reinterpret_cast<const uint4*>(rp.gain),
+                    reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(const_cast<void*>(g.a)) + (int64_t)row * g.K),
+                    g.K, rp.eps, red);
+    }
+    asm volatile("fence.proxy.async;" ::: "memory");   // the rows are read back through TMA
+    grid_barrier(g.grid_bar, ++nbar, abort_flag);
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtensorMap mapA,
                const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
@@ -500,53 +551,7 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     pdl_launch_dependents();
 
     // ---------------- phase 0: gather the rows of R and RMSNorm them into A ----------------
-    if (g.prep.enabled) {
-        const RowPrep& rp = g.prep;
-        const int rows_per_req = rp.k + rp.e;
-        for (int row = blockIdx.x; row < g.M; row += gridDim.x) {
-            int64_t src = (int64_t)row * g.K;
-            if (rp.enabled == 3) {       // compact rows picked by index
-                const int b = row / rows_per_req;
-                const int ci = rp.compact_idx[row];
-                if (ci < 0 || ci >= rp.compact_rows) {
-                    if (threadIdx.x == 0) atomicOr(g.status, kFlagBadIndex);
-                }
-                src = ((int64_t)b * rp.compact_rows + (ci < 0 || ci >= rp.compact_rows ? 0 : ci)) * g.K;
-            }
-            if (rp.enabled == 1) {       // rows of R: position from the anchor / extra-row lists
-                const int b = row / rows_per_req, i = row - b * rows_per_req;
-                const int pos = row_position(rp.anchor_idx, rp.k, rp.extra_rows, rp.e, b, i, rp.affix_start,
-                                             rp.affix_len, rp.ctx_len);
-                if (!rp.x_is_compact) {
-                    if (rp.token_ids) {       // x is an embedding table: the row of the token at that position
-                        int id = rp.token_ids[(int64_t)b * rp.ctx_len + (pos < 0 ? 0 : pos)];
-                        if (id < 0 || id >= rp.table_rows) {
-                            if (threadIdx.x == 0) atomicOr(g.status, kFlagBadIndex);
-                            id = 0;
-                        }
-                        src = (int64_t)id * g.K;
-                    } else {
-                        src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
-                    }
-                } else if (rp.compact_idx) {
-                    const int ci = rp.compact_idx[row];
-                    src = ((int64_t)b * rp.compact_rows + (ci < 0 ? 0 : ci)) * g.K;
-                }
-                if (threadIdx.x == 0) {
-                    rp.row_pos[row] = pos;
-                    rp.row_src[row] = src;
-                    if (pos < 0) atomicOr(g.status, kFlagBadIndex);
-                }
-            }
-            rmsnorm_row(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(rp.x) + src),
-                        reinterpret_cast<const uint4*>(rp.gain),
-                        reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(const_cast<void*>(g.a)) + (int64_t)row * g.K),
-                        g.K, rp.eps, red);
-        }
-        asm volatile("fence.proxy.async;" ::: "memory");   // the rows are read back through TMA
-        grid_barrier(g.grid_bar, ++nbar, abort_flag);
-        asm volatile("fence.proxy.async;" ::: "memory");
-    }
+    if (g.prep.enabled) prep_phase(g, red, abort_flag, nbar);
 
     // ---------------- phase 1: the contraction ----------------
 
@@ -673,6 +678,246 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
+// ---- cta_group::2: two SMs on one 256 x 256 output tile (many-row problems) -----------------------
+// A cluster of two CTAs owns a tile: CTA r holds rows [128 r, 128 r + 128) of A and the r-th
+// 128-row half of the weight tile in its own shared memory, so each SM moves half of the weight
+// bytes per flop that the one-CTA kernel moves; the leader CTA's MMA thread issues
+// tcgen05.mma.cta_group::2 (M = 256) and each CTA's TMEM receives its 128 rows of the result.
+// Tiles are whole (no K split): clusters walk the tile list round-robin, weight-tile-major.
+// Barriers: the leader's full[s] counts both CTAs' TMA bytes (announced by the leader's producer); empty[s] and tmem_full[a] live in
+// each CTA and are signalled by a tcgen05.commit multicast to both; the leader's tmem_empty[a]
+// collects the drain warps of both CTAs.
+constexpr int TC2_STAGES = 6;
+constexpr int TC2_STAGE_BYTES = TC_A_BYTES + TC_HALF_BYTES;     // 32 KB per CTA and stage
+constexpr int TC2_SMEM = TC2_STAGES * TC2_STAGE_BYTES + 1024 + 256;
+
+// Tile order of the two-SM kernel: groups of kTileGroupN weight tiles; inside a group the row
+// pairs are walked with the group's weight tiles innermost.  The ~74 clusters running at any
+// moment then cover about 9 row pairs x 8 weight tiles, whose A and B blocks (tens of MB) stay in
+// L2 while they are reused, instead of streaming the whole A matrix from HBM once per weight tile.
+constexpr int kTileGroupN = 8;
+__device__ __forceinline__ void tile_coords(int t, int m_pairs, int n_tiles, int& nt, int& mp) {
+    const int full = n_tiles / kTileGroupN, per_group = kTileGroupN * m_pairs;
+    if (t < full * per_group) {
+        const int grp = t / per_group, r = t - grp * per_group;
+        mp = r / kTileGroupN;
+        nt = grp * kTileGroupN + (r - mp * kTileGroupN);
+    } else {
+        const int r = t - full * per_group, gn = n_tiles - full * kTileGroupN;
+        mp = r / gn;
+        nt = full * kTileGroupN + (r - mp * gn);
+    }
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < TC_WAIT_LIMIT; ++i) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (i > 128) {
+            __nanosleep(40);
+            if (*abort_flag) return false;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+// TMA load into this CTA's shared memory that completes on a barrier of the CTA pair's leader
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cluster,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tc2_commit_both(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3)
+                 : "memory");
+}
+__device__ __forceinline__ void tc2_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __grid_constant__ CUtensorMap mapA,
+                const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
+                const __grid_constant__ CUtensorMap mapB2) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ float red[TC_THREADS / 32];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + TC2_STAGES * TC2_STAGE_BYTES;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + TC2_STAGES * TC2_STAGE_BYTES + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + TC2_STAGES * TC2_STAGE_BYTES + 200);
+    auto full_bar = [&](int s) { return bars + 8 * s; };
+    auto empty_bar = [&](int s) { return bars + 8 * (TC2_STAGES + s); };
+    auto tfull_bar = [&](int i) { return bars + 8 * (2 * TC2_STAGES + i); };
+    auto tempty_bar = [&](int i) { return bars + 8 * (2 * TC2_STAGES + 2 + i); };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int cluster_id = blockIdx.x >> 1;
+    unsigned int nbar = 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TC2_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();          // the peer's barriers are initialised before anyone signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();
+    pdl_launch_dependents();
+
+    if (g.prep.enabled) prep_phase(g, red, abort_flag, nbar);
+
+    const int m_pairs = (p.m_tiles + 1) >> 1;
+    const int tiles = m_pairs * p.n_tiles;
+
+    if (warp == 0 && lane == 0) {
+        // TMA producer of this CTA: its 128 rows of A and its half of the weight tile
+        const CUtensorMap* maps[3] = {&mapB0, &mapB1, &mapB2};
+        int stage = 0, issued = 0;
+        uint32_t phase = 0;
+        bool ok = !*abort_flag;
+        const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
+        for (int t = cluster_id; t < tiles && ok; t += clusters) {
+            int nt, mp;
+            tile_coords(t, m_pairs, p.n_tiles, nt, mp);
+            int brow;
+            const int bs = half_source(g, p, nt, (int)rank, brow);
+            const int arow = (mp * 2 + (int)rank) * TC_BM;
+            for (int kb = 0; kb < p.KB; ++kb) {
+                if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag))) break;
+                const uint32_t sA = base + stage * TC2_STAGE_BYTES, sB = sA + TC_A_BYTES;
+                const uint32_t lead_full = mapa_u32(full_bar(stage), 0);
+                // the leader announces the bytes of both CTAs; the peer's copies only report completion
+                if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * TC2_STAGE_BYTES);
+                tma_load_2d_pair(sA, &mapA, kb * TC_BK, arow, lead_full, pol_a);
+                tma_load_2d_pair(sB, maps[bs], kb * TC_BK, brow, lead_full, pol_w);
+                ++issued;
+                if (++stage == TC2_STAGES) { stage = 0; phase ^= 1; }
+            }
+        }
+        // wait until the MMAs have consumed everything this CTA loaded, so that no signal from the
+        // leader can arrive after this CTA has left
+        for (int i = 0; i < min(issued, TC2_STAGES) && ok; ++i) {
+            ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag);
+            if (++stage == TC2_STAGES) { stage = 0; phase ^= 1; }
+        }
+    } else if (warp == 1 && lane == 0 && rank == 0) {
+        // MMA issuer (leader CTA only)
+        int stage = 0, acc = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        bool ok = !*abort_flag;
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+        for (int t = cluster_id; t < tiles && ok; t += clusters) {
+            if (!(ok = mbar_wait_cluster(tempty_bar(acc), acc_phase ^ 1, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * TC_BN;
+            for (int kb = 0; kb < p.KB; ++kb) {
+                if (!(ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t sA = base + stage * TC2_STAGE_BYTES, sB = sA + TC_A_BYTES;
+                const uint64_t da = smem_desc_sw128(sA), db = smem_desc_sw128(sB);
+#pragma unroll
+                for (int k = 0; k < TC_BK / 16; ++k)
+                    tc2_mma(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                tc2_commit_both(empty_bar(stage));
+                if (++stage == TC2_STAGES) { stage = 0; phase ^= 1; }
+            }
+            if (!ok) break;
+            tc2_commit_both(tfull_bar(acc));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    } else if (warp >= 2 && warp < 6) {
+        // drain: this CTA's 128 rows of the tile, epilogue straight from TMEM
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = !*abort_flag;
+        for (int t = cluster_id; t < tiles && ok; t += clusters) {
+            int nt, mp;
+            tile_coords(t, m_pairs, p.n_tiles, nt, mp);
+            const int grow = (mp * 2 + (int)rank) * TC_BM + row;
+            if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + acc * TC_BN + ((uint32_t)(q * 32) << 16);
+            direct_epilogue(g, p, taddr, nt, grow, grow < g.M, 8);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_u32(tempty_bar(acc), 0));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) {
+            atomicOr(g.status, kFlagWaitExpired);
+            for (int i = 0; i < 4096; ++i) __nanosleep(64);
+        }
+        __syncthreads();
+    } else if (threadIdx.x == 0 && nbar > 0) {
+        __threadfence();
+        if (atomicAdd(&g.grid_bar[1], 1u) == gridDim.x - 1) {
+            g.grid_bar[0] = 0u;
+            __threadfence();
+            g.grid_bar[1] = 0u;
+        }
+    }
+    cluster_sync_all();          // neither CTA leaves while its peer may still signal it
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
     }
 }
 
@@ -881,8 +1126,43 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
     static bool attr = false;
     if (!attr) {
         cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
+        cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC2_SMEM);
         attr = true;
     }
+    // Many rows: two SMs per 256 x 256 tile (no K split, every tile whole).
+    static const int pair_min_tiles = [] { const char* e = getenv("ACACHE_GEMM_PAIR_MIN_MTILES"); return e ? atoi(e) : 4; }();
+    if (p.m_tiles >= pair_min_tiles && g.epilogue != kEpiLogits && (p.units % 2 == 0 || swiglu) && sm_count() >= 2) {
+        const int m_pairs = (p.m_tiles + 1) / 2;
+        const int tiles = m_pairs * p.n_tiles;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(sm_count() / 2 * 2);
+        cfg.blockDim = dim3(TC_THREADS);
+        cfg.dynamicSmemBytes = TC2_SMEM;
+        cfg.stream = stream;
+        cudaLaunchAttribute at[2];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 2;
+        // all clusters must be resident at once (phase 0 ends in a grid-wide barrier)
+        static int max_clusters = 0;
+        if (!max_clusters) {
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, gemm_tc2_kernel, &cfg) != cudaSuccess || n <= 0) {
+                (void)cudaGetLastError();
+                n = -1;
+            }
+            max_clusters = n;
+        }
+        if (max_clusters < 1) goto single_cta;
+        const int clusters = std::min(std::min(max_clusters, sm_count() / 2), tiles);
+        cfg.gridDim = dim3(clusters * 2);
+        if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, g, p, clusters, *mA, *mB[0], *mB[1], *mB[2]) != cudaSuccess) return -1;
+        return 1;
+    }
+single_cta:
     // a plain launch: a cooperative one measured ~2.5 us slower and cannot overlap the previous
     // kernel's tail; the grid never exceeds the SM count at one CTA per SM and the barrier is bounded
     if (launch_pdl(gemm_tc_kernel, dim3(p.ctas), dim3(TC_THREADS), TC_SMEM, stream, g, p, *mA, *mB[0], *mB[1], *mB[2]) !=
