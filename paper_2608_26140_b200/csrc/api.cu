@@ -189,6 +189,7 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     at.batch = r->batch; at.n = rows; at.ctx_len = r->ctx_len;
     at.n_heads = d.n_heads; at.n_kv_heads = d.n_kv_heads; at.head_dim = d.head_dim;
     at.o = o;
+    at.status = status;
     at.part_o = wsp<float>(c, c->o_attn);
     at.part_ml = at.part_o + (size_t)2 * 296 * 64 * d.head_dim;
     c->launches += launch_attention(at, st);

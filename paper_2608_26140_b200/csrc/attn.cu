@@ -4,6 +4,8 @@
 // accumulation and fp32 softmax statistics.  Keys/values come from the token-major cache or,
 // where a position -> fresh-row map says so, from the compact fresh K/V (the logical view of
 // the working cache without having written it).
+#include <cstdlib>
+
 #include "common.cuh"
 #include "kernels.h"
 #include "launch.h"
@@ -248,6 +250,11 @@ size_t attention_scratch_bytes(int head_dim) {
 
 int launch_attention(const AttnArgs& a, cudaStream_t stream) {
     if (a.batch == 0 || a.n == 0) return 0;
+    static const bool no_tc = [] { const char* e = getenv("ACACHE_ATTN_TC"); return e && e[0] == '0'; }();
+    if (!no_tc) {
+        const int r = launch_attention_tc(a, a.status, stream);
+        if (r != 0) return r;
+    }
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)a.head_dim);
     const int q_tiles = (a.n + 63) / 64;
     int tps;

@@ -1,0 +1,366 @@
+// Bidirectional attention of many recomputed rows over the whole context (Section 4.3) on the
+// 5th-generation tensor cores.  One CTA = 128 query rows of one head; key/value tiles of 128
+// keys stream through shared memory by TMA (3-d tensor maps: positions past the context end and
+// rows past the request's row count read as zero).
+//
+//   S = Q K^T    tcgen05.mma 128 x 128 x 16, both operands K-major, into one of two TMEM buffers
+//   softmax      four warps, thread = query row: scaled max, exp2, running denominator; P is
+//                written as bf16 into a 128-byte-swizzled shared tile
+//   O += P V     tcgen05.mma 128 x 128 x 16, A = P (K-major over keys), B = V read in place as an
+//                MN-major operand (token-major V rows are contiguous along the head dimension)
+//
+// The S of tile j+1 is issued before the softmax of tile j is consumed, so tensor work overlaps the
+// exponentials.  The running maximum used for the exponent is only raised (and O rescaled in
+// TMEM) when the true maximum has grown by more than 2^8, which keeps P within bf16 range and
+// makes rescales rare.  Every mbarrier wait is bounded (status flag kFlagWaitExpired on expiry).
+#include <cuda.h>
+
+#include <mutex>
+
+#include "common.cuh"
+#include "kernels.h"
+#include "launch.h"
+#include "tc_ptx.cuh"
+
+namespace acache {
+
+constexpr int AT_THREADS = 192;                  // warp 0: TMA, warp 1: MMA, warps 2-5: softmax (thread = row)
+constexpr int AT_TILE = 128 * 128 * 2;           // 32 KB: a [128 x 128] bf16 tile as two 64-column panels
+constexpr int AT_PANEL = 128 * 64 * 2;           // 16 KB
+constexpr int AT_SMEM = 6 * AT_TILE + 1024 + 256;   // Q, K x2, V x2, P
+constexpr float kRescaleGap = 8.f;               // log2 units
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar,
+                                            uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]),
+          "f"(v[9]), "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "f"(v[16]), "f"(v[17]),
+          "f"(v[18]), "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]),
+          "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// MN-major bf16 operand with the 128-byte swizzle: rows of the K index are 128 bytes (64 elements
+// of the MN index), 8-row groups 1024 bytes apart (stride byte offset), and the next 64 elements
+// of the MN index start one 16 KB panel further (leading byte offset).
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t saddr) {
+    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(AT_PANEL >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+struct AttnTcArgs {
+    void* o;                  // bf16 [B, n, H*d]
+    int n, ctx_len, n_heads, n_kv_heads;
+    float scale_log2e;
+    uint32_t* status;
+};
+
+__global__ void __launch_bounds__(AT_THREADS, 1)
+attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                    const __grid_constant__ CUtensorMap mapV) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t sQ = base, sK0 = base + AT_TILE, sV0 = base + 3 * AT_TILE, sP = base + 5 * AT_TILE;
+    const uint32_t bars = base + 6 * AT_TILE;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + 6 * AT_TILE + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + 6 * AT_TILE + 200);
+    // barriers: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 v_full | 7,8 v_empty | 9,10 s_full | 11,12 s_empty |
+    //           13 p_full | 14 p_empty
+    auto bar = [&](int i) { return bars + 8 * i; };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int n_tiles = (a.ctx_len + 127) / 128;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(11), 4); mbar_init(bar(12), 4);      // s_empty: the four softmax warps
+        mbar_init(bar(13), 4);                             // p_full
+        mbar_init(bar(14), 1);                             // p_empty
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tS0 = tmem_base, tO = tmem_base + 256;
+    pdl_wait();
+    pdl_launch_dependents();
+
+    if (warp == 0 && lane == 0) {
+        // ---------------- TMA producer ----------------
+        const uint64_t pol_q = policy_evict_first(), pol_kv = policy_evict_last();
+        mbar_expect_tx(bar(0), AT_TILE);
+        tma_load_3d(sQ, &mapQ, h * 128, qt * 128, b, bar(0), pol_q);
+        tma_load_3d(sQ + AT_PANEL, &mapQ, h * 128 + 64, qt * 128, b, bar(0), pol_q);
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int s = j & 1;
+            const uint32_t par = ((j >> 1) & 1) ^ 1;
+            if (!(ok = mbar_wait(bar(3 + s), par, abort_flag))) break;
+            mbar_expect_tx(bar(1 + s), AT_TILE);
+            tma_load_3d(sK0 + s * AT_TILE, &mapK, kvh * 128, j * 128, b, bar(1 + s), pol_kv);
+            tma_load_3d(sK0 + s * AT_TILE + AT_PANEL, &mapK, kvh * 128 + 64, j * 128, b, bar(1 + s), pol_kv);
+            if (!(ok = mbar_wait(bar(7 + s), par, abort_flag))) break;
+            mbar_expect_tx(bar(5 + s), AT_TILE);
+            tma_load_3d(sV0 + s * AT_TILE, &mapV, kvh * 128, j * 128, b, bar(5 + s), pol_kv);
+            tma_load_3d(sV0 + s * AT_TILE + AT_PANEL, &mapV, kvh * 128 + 64, j * 128, b, bar(5 + s), pol_kv);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer ----------------
+        // S = Q K^T: M 128, N 128, both K-major.  O += P V: M 128, N 128, A K-major, B MN-major.
+        const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        const uint32_t idesc_o = idesc_s | (1u << 16);
+        auto issue_s = [&](int j) {
+            const int s = j & 1;
+            const uint32_t k = sK0 + s * AT_TILE;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t da = smem_desc_sw128(sQ + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
+                const uint64_t db = smem_desc_sw128(k + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
+                tc_mma(tS0 + s * 128, da, db, idesc_s, ks > 0 ? 1u : 0u);
+            }
+            tc_commit(bar(9 + s));     // s_full
+            tc_commit(bar(3 + s));     // k_empty
+        };
+        bool ok = mbar_wait(bar(0), 0, abort_flag) && mbar_wait(bar(1), 0, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            issue_s(0);
+        }
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            if (j + 1 < n_tiles) {
+                const int s = (j + 1) & 1;
+                const uint32_t par = ((j + 1) >> 1) & 1;
+                if (!(ok = mbar_wait(bar(1 + s), par, abort_flag))) break;          // K of tile j+1 landed
+                if (!(ok = mbar_wait(bar(11 + s), par ^ 1, abort_flag))) break;     // its S buffer has been read
+                tc_fence_after();
+                issue_s(j + 1);
+            }
+            const int s = j & 1;
+            if (!(ok = mbar_wait(bar(13), j & 1, abort_flag))) break;               // P of tile j written, O rescaled
+            if (!(ok = mbar_wait(bar(5 + s), (j >> 1) & 1, abort_flag))) break;     // V of tile j landed
+            tc_fence_after();
+            const uint32_t v = sV0 + s * AT_TILE;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t da = smem_desc_sw128(sP + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
+                const uint64_t db = smem_desc_mn_sw128(v + ks * 2048);
+                tc_mma(tO, da, db, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+            }
+            tc_commit(bar(14));        // p_empty: P free, O updated
+            tc_commit(bar(7 + s));     // v_empty
+        }
+    } else if (warp >= 2) {
+        // ---------------- softmax: thread = query row ----------------
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+        float m_use = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int s = j & 1;
+            if (!(ok = mbar_wait(bar(9 + s), (j >> 1) & 1, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t tS = tS0 + s * 128 + lane_off;
+            const int valid = a.ctx_len - j * 128;
+            // pass 1: the tile's row maximum
+            float mt = -INFINITY;
+            for (int c = 0; c < 4; ++c) {
+                float v[32];
+                tc_ld32(tS + c * 32, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (c * 32 + i < valid) mt = fmaxf(mt, v[i]);
+            }
+            mt *= a.scale_log2e;
+            bool raise = false;
+            if (j == 0) {
+                m_use = mt;
+            } else if (mt - m_use > kRescaleGap) {
+                raise = true;
+            }
+            // O and P belong to the previous tile's P V until it has completed
+            if (j > 0 && !(ok = mbar_wait(bar(14), (j - 1) & 1, abort_flag))) break;
+            tc_fence_after();
+            if (__any_sync(0xffffffffu, raise)) {
+                const float f = raise ? exp2f(m_use - mt) : 1.f;
+                for (int c = 0; c < 4; ++c) {
+                    float v[32];
+                    tc_ld32(tO + lane_off + c * 32, v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] *= f;
+                    tc_st32(tO + lane_off + c * 32, v);
+                }
+                tc_wait_st();
+                l *= f;
+                if (raise) m_use = mt;
+            }
+            // pass 2: exponentials, denominator, P as bf16 into the swizzled tile
+            for (int c = 0; c < 4; ++c) {
+                float v[32];
+                tc_ld32(tS + c * 32, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float p = c * 32 + i < valid ? exp2f(v[i] * a.scale_log2e - m_use) : 0.f;
+                    l += p;
+                    v[i] = p;
+                }
+#pragma unroll
+                for (int k8 = 0; k8 < 4; ++k8) {
+                    const int chunk = c * 4 + k8;                 // 16-byte chunk of the row: 8 keys
+                    const uint32_t addr = sP + (chunk >> 3) * AT_PANEL + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
+                    const float* pv = v + k8 * 8;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(pv[0], pv[1])),
+                                 "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])), "r"(pack_bf16(pv[6], pv[7]))
+                                 : "memory");
+                }
+            }
+            tc_fence_before();
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core's async proxy
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(bar(11 + s));   // s_empty
+                mbar_arrive(bar(13));       // p_full
+            }
+        }
+        // epilogue: O / l once the last P V has completed
+        if (ok && n_tiles > 0) ok = mbar_wait(bar(14), (n_tiles - 1) & 1, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            const int grow = qt * 128 + row;
+            const float inv = 1.f / l;
+            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o) + (((int64_t)b * a.n + grow) * a.n_heads + h) * 128;
+            for (int c = 0; c < 4; ++c) {
+                float v[32];
+                tc_ld32(tO + lane_off + c * 32, v);
+                if (grow < a.n) {
+#pragma unroll
+                    for (int k8 = 0; k8 < 4; ++k8) {
+                        const float* pv = v + k8 * 8;
+                        *reinterpret_cast<uint4*>(out + c * 32 + k8 * 8) =
+                            make_uint4(pack_bf16(pv[0] * inv, pv[1] * inv), pack_bf16(pv[2] * inv, pv[3] * inv),
+                                       pack_bf16(pv[4] * inv, pv[5] * inv), pack_bf16(pv[6] * inv, pv[7] * inv));
+                    }
+                }
+            }
+        }
+    }
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) {
+            atomicOr(a.status, kFlagWaitExpired);
+            for (int i = 0; i < 4096; ++i) __nanosleep(64);   // let copies already in flight land
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn3() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 [batch, rows, cols] with row stride = cols and the given batch stride (elements);
+// box = 64 cols x 128 rows x 1, 128-byte swizzle, zero fill out of bounds.
+struct Map3Key { const void* ptr; int rows, cols, batch; int64_t bstride; };
+struct Map3Entry { Map3Key key; CUtensorMap map; };
+constexpr int kMap3Cache = 64;
+std::mutex g_map3_mutex;
+Map3Entry g_maps3[kMap3Cache];
+int g_map3_count = 0, g_map3_next = 0;
+
+const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int64_t bstride) {
+    for (int i = 0; i < g_map3_count; ++i) {
+        const Map3Key& k = g_maps3[i].key;
+        if (k.ptr == ptr && k.rows == rows && k.cols == cols && k.batch == batch && k.bstride == bstride) return &g_maps3[i].map;
+    }
+    EncodeTiledFn fn = encode_fn3();
+    if (!fn) return nullptr;
+    Map3Entry& e = g_maps3[g_map3_next];
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)bstride * 2};
+    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return nullptr;
+    e.key = Map3Key{ptr, rows, cols, batch, bstride};
+    g_map3_next = (g_map3_next + 1) % kMap3Cache;
+    if (g_map3_count < kMap3Cache) ++g_map3_count;
+    return &e.map;
+}
+
+}  // namespace
+
+// Returns the number of kernels launched, 0 if this problem is not for the tensor-core kernel
+// (the caller then uses the mma.sync kernel), -1 if a launch failed.
+int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream) {
+    if (a.head_dim != 128 || a.slot || a.batch == 0 || a.n == 0) return 0;
+    const int q_tiles = (a.n + 127) / 128;
+    if ((int64_t)q_tiles * a.n_heads * a.batch < 148) return 0;       // few rows: the key-split kernel fills the machine better
+    if ((a.kv_batch_stride * 2) % 16) return 0;
+    std::lock_guard<std::mutex> lock(g_map3_mutex);
+    const CUtensorMap* mq = get_map3(a.q, a.n, a.n_heads * 128, a.batch, (int64_t)a.n * a.n_heads * 128);
+    const CUtensorMap* mk = get_map3(a.cache_k, a.ctx_len, a.n_kv_heads * 128, a.batch, a.kv_batch_stride);
+    const CUtensorMap* mv = get_map3(a.cache_v, a.ctx_len, a.n_kv_heads * 128, a.batch, a.kv_batch_stride);
+    if (!mq || !mk || !mv) return 0;
+    static bool attr = false;
+    if (!attr) {
+        cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM);
+        attr = true;
+    }
+    AttnTcArgs t{};
+    t.o = a.o; t.n = a.n; t.ctx_len = a.ctx_len; t.n_heads = a.n_heads; t.n_kv_heads = a.n_kv_heads;
+    t.scale_log2e = 1.4426950408889634f / sqrtf(128.f);
+    t.status = status;
+    if (launch_pdl(attention_tc_kernel, dim3(q_tiles, a.n_heads, a.batch), dim3(AT_THREADS), AT_SMEM, stream, t, *mq, *mk, *mv) !=
+        cudaSuccess)
+        return -1;
+    return 1;
+}
+
+}  // namespace acache
