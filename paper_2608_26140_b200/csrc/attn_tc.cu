@@ -27,7 +27,7 @@ namespace acache {
 constexpr int AT_THREADS = 192;                  // warp 0: TMA, warp 1: MMA, warps 2-5: softmax (thread = row)
 constexpr int AT_TILE = 128 * 128 * 2;           // 32 KB: a [128 x 128] bf16 tile as two 64-column panels
 constexpr int AT_PANEL = 128 * 64 * 2;           // 16 KB
-constexpr int AT_SMEM = 6 * AT_TILE + 1024 + 256;   // Q, K x2, V x2, P
+constexpr int AT_SMEM = 7 * AT_TILE + 1024 + 256;   // Q, K x2, V x2, P x2
 constexpr float kRescaleGap = 8.f;               // log2 units
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar,
@@ -48,6 +48,11 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const float (&v)[32]) {
           "f"(v[18]), "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]),
           "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
         : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -76,12 +81,12 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t sQ = base, sK0 = base + AT_TILE, sV0 = base + 3 * AT_TILE, sP = base + 5 * AT_TILE;
-    const uint32_t bars = base + 6 * AT_TILE;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + 6 * AT_TILE + 192);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + 6 * AT_TILE + 200);
+    const uint32_t sQ = base, sK0 = base + AT_TILE, sV0 = base + 3 * AT_TILE, sP0 = base + 5 * AT_TILE;
+    const uint32_t bars = base + 7 * AT_TILE;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + 7 * AT_TILE + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + 7 * AT_TILE + 200);
     // barriers: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 v_full | 7,8 v_empty | 9,10 s_full | 11,12 s_empty |
-    //           13 p_full | 14 p_empty
+    //           13,14 p_full | 15,16 p_empty
     auto bar = [&](int i) { return bars + 8 * i; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -91,8 +96,8 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
         mbar_init(bar(11), 4); mbar_init(bar(12), 4);      // s_empty: the four softmax warps
-        mbar_init(bar(13), 4);                             // p_full
-        mbar_init(bar(14), 1);                             // p_empty
+        mbar_init(bar(13), 4); mbar_init(bar(14), 4);      // p_full
+        mbar_init(bar(15), 1); mbar_init(bar(16), 1);      // p_empty
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -160,17 +165,17 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
                 issue_s(j + 1);
             }
             const int s = j & 1;
-            if (!(ok = mbar_wait(bar(13), j & 1, abort_flag))) break;               // P of tile j written, O rescaled
+            if (!(ok = mbar_wait(bar(13 + s), (j >> 1) & 1, abort_flag))) break;    // P of tile j written, O rescaled
             if (!(ok = mbar_wait(bar(5 + s), (j >> 1) & 1, abort_flag))) break;     // V of tile j landed
             tc_fence_after();
             const uint32_t v = sV0 + s * AT_TILE;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                const uint64_t da = smem_desc_sw128(sP + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
+                const uint64_t da = smem_desc_sw128(sP0 + s * AT_TILE + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
                 const uint64_t db = smem_desc_mn_sw128(v + ks * 2048);
                 tc_mma(tO, da, db, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
             }
-            tc_commit(bar(14));        // p_empty: P free, O updated
+            tc_commit(bar(15 + s));    // p_empty: this P buffer is free, O holds tiles 0..j
             tc_commit(bar(7 + s));     // v_empty
         }
     } else if (warp >= 2) {
@@ -186,15 +191,19 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             tc_fence_after();
             const uint32_t tS = tS0 + s * 128 + lane_off;
             const int valid = a.ctx_len - j * 128;
-            // pass 1: the tile's row maximum
+            // the whole row of S into registers, then the S buffer is free for tile j + 2
+            float sv[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tc_ld32(tS + c * 32, sv[c]);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(11 + s));   // s_empty
             float mt = -INFINITY;
-            for (int c = 0; c < 4; ++c) {
-                float v[32];
-                tc_ld32(tS + c * 32, v);
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
-                    if (c * 32 + i < valid) mt = fmaxf(mt, v[i]);
-            }
+                    if (c * 32 + i < valid) mt = fmaxf(mt, sv[c][i]);
             mt *= a.scale_log2e;
             bool raise = false;
             if (j == 0) {
@@ -202,11 +211,11 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             } else if (mt - m_use > kRescaleGap) {
                 raise = true;
             }
-            // O and P belong to the previous tile's P V until it has completed
-            if (j > 0 && !(ok = mbar_wait(bar(14), (j - 1) & 1, abort_flag))) break;
-            tc_fence_after();
             if (__any_sync(0xffffffffu, raise)) {
-                const float f = raise ? exp2f(m_use - mt) : 1.f;
+                // O may only be touched once the P V of tile j - 1 has completed
+                if (!(ok = mbar_wait(bar(15 + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag))) break;
+                tc_fence_after();
+                const float f = raise ? fast_exp2(m_use - mt) : 1.f;
                 for (int c = 0; c < 4; ++c) {
                     float v[32];
                     tc_ld32(tO + lane_off + c * 32, v);
@@ -218,21 +227,22 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
                 l *= f;
                 if (raise) m_use = mt;
             }
-            // pass 2: exponentials, denominator, P as bf16 into the swizzled tile
+            // this P buffer was last read by the P V of tile j - 2
+            if (j >= 2 && !(ok = mbar_wait(bar(15 + s), ((j - 2) >> 1) & 1, abort_flag))) break;
+            const uint32_t sP = sP0 + s * AT_TILE;
+#pragma unroll
             for (int c = 0; c < 4; ++c) {
-                float v[32];
-                tc_ld32(tS + c * 32, v);
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    const float p = c * 32 + i < valid ? exp2f(v[i] * a.scale_log2e - m_use) : 0.f;
+                    const float p = c * 32 + i < valid ? fast_exp2(sv[c][i] * a.scale_log2e - m_use) : 0.f;
                     l += p;
-                    v[i] = p;
+                    sv[c][i] = p;
                 }
 #pragma unroll
                 for (int k8 = 0; k8 < 4; ++k8) {
                     const int chunk = c * 4 + k8;                 // 16-byte chunk of the row: 8 keys
                     const uint32_t addr = sP + (chunk >> 3) * AT_PANEL + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
-                    const float* pv = v + k8 * 8;
+                    const float* pv = sv[c] + k8 * 8;
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(pv[0], pv[1])),
                                  "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])), "r"(pack_bf16(pv[6], pv[7]))
                                  : "memory");
@@ -241,13 +251,10 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             tc_fence_before();
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core's async proxy
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar(11 + s));   // s_empty
-                mbar_arrive(bar(13));       // p_full
-            }
+            if (lane == 0) mbar_arrive(bar(13 + s));   // p_full
         }
         // epilogue: O / l once the last P V has completed
-        if (ok && n_tiles > 0) ok = mbar_wait(bar(14), (n_tiles - 1) & 1, abort_flag);
+        if (ok && n_tiles > 0) ok = mbar_wait(bar(15 + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, abort_flag);
         if (ok) {
             tc_fence_after();
             const int grow = qt * 128 + row;
