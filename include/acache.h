@@ -90,7 +90,12 @@ typedef struct {
 } acache_layer_weights;
 
 /* One layer's KV cache: DEVICE bf16 [B, ctx_capacity, Hkv, d]; request b starts at
- * element offset b * batch_stride (normally ctx_capacity * Hkv * d). */
+ * element offset b * batch_stride (normally ctx_capacity * Hkv * d).
+ * batch_stride == 0: ONE cache [ctx_capacity, Hkv, d] shared by every request of the batch (the
+ * shared-affix storage of Section 4.1).  Accepted by the calls that only read the cache:
+ * acache_score_anchors, and acache_recompute_anchors, whose k_new / v_new are then the requests'
+ * private slots (anchors + request rows) and whose attention reads every other position from
+ * the shared copy.  Calls that write the cache reject it. */
 typedef struct {
     void   *k, *v;
     int64_t batch_stride;

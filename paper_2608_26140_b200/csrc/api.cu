@@ -69,7 +69,9 @@ acache_status check_cuda(acache_ctx* c, const char* what) {
     return ACACHE_OK;
 }
 
-acache_status check_request(acache_ctx* c, const acache_request* r, const acache_kv* kv, int k, bool need_rope) {
+// shared_ok: the call only reads the cache, so one copy may serve the whole batch (batch_stride 0)
+acache_status check_request(acache_ctx* c, const acache_request* r, const acache_kv* kv, int k, bool need_rope,
+                            bool shared_ok = false) {
     const acache_model_desc& d = c->d;
     if (!c->ws) return fail(c, ACACHE_ERR_WORKSPACE, "workspace not set");
     if (!r) return fail(c, ACACHE_ERR_INVALID_ARG, "request is NULL");
@@ -88,7 +90,10 @@ acache_status check_request(acache_ctx* c, const acache_request* r, const acache
     if (kv) {
         if (!kv->k || !kv->v || !aligned16(kv->k) || !aligned16(kv->v)) return fail(c, ACACHE_ERR_INVALID_ARG, "cache pointer NULL or misaligned");
         if (kv->ctx_capacity < r->ctx_len) return fail(c, ACACHE_ERR_INVALID_ARG, "ctx_capacity %d < ctx_len %d", kv->ctx_capacity, r->ctx_len);
-        if (kv->batch_stride < (int64_t)kv->ctx_capacity * d.n_kv_heads * d.head_dim || (kv->batch_stride & 7))
+        const bool shared = kv->batch_stride == 0;
+        if (shared && !shared_ok)
+            return fail(c, ACACHE_ERR_INVALID_ARG, "batch_stride 0 (one cache shared by the batch) is only valid for calls that do not write the cache");
+        if (!shared && (kv->batch_stride < (int64_t)kv->ctx_capacity * d.n_kv_heads * d.head_dim || (kv->batch_stride & 7)))
             return fail(c, ACACHE_ERR_INVALID_ARG, "batch_stride smaller than one request's cache or not a multiple of 8");
     }
     return ACACHE_OK;
@@ -368,7 +373,7 @@ acache_status acache_score_anchors(acache_ctx* ctx, const acache_request* req, c
                                    acache_stream_t stream) {
     if (!ctx) return ACACHE_ERR_INVALID_ARG;
     if (!kv) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv is NULL");
-    acache_status s = check_request(ctx, req, kv, 0, false);
+    acache_status s = check_request(ctx, req, kv, 0, false, true);
     if (s != ACACHE_OK) return s;
     if (!scores || (req->n_masked > 0 && (!q_mask || !aligned16(q_mask)))) return fail(ctx, ACACHE_ERR_INVALID_ARG, "q_mask / scores NULL or misaligned");
     return run_score(ctx, req, q_mask, kv, scores, accumulate, norm_full, 0, stream);
@@ -391,7 +396,7 @@ acache_status acache_recompute_anchors(acache_ctx* ctx, const acache_layer_weigh
                                        acache_stream_t stream) {
     if (!ctx) return ACACHE_ERR_INVALID_ARG;
     if (!kv) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv is NULL");
-    acache_status s = check_request(ctx, req, kv, k, true);
+    acache_status s = check_request(ctx, req, kv, k, true, true);
     if (s != ACACHE_OK) return s;
     if ((s = check_weights(ctx, w, false)) != ACACHE_OK) return s;
     if (req->batch * (k + req->n_extra) == 0) return ACACHE_OK;

@@ -345,3 +345,53 @@ def test_llada_layer_full_size(extra):
     assert_close_bf16(cvb[0][rows], ref["v_new"], "V rows")
     assert_close_bf16(ab.to_host_bits(y[0, :n]), ref["y"], "y")
     assert dc.ctx.poll_status() == 0
+
+
+# ------------------------------------------------------------------ shared affix storage (Section 4.1)
+def test_shared_affix_cache_with_private_rows():
+    """One copy of the affix K/V (batch_stride = 0) serves three requests: scoring reads it, the
+    refresh writes each request's anchors and request rows to its private k_new / v_new and its
+    attention reads all other positions from the shared copy, which stays untouched."""
+    shape, B = MID128, 3
+    lay = wl.make_layout(B, 0, 160, 24, 32, 32, "all")
+    case = wl.make_case(shape, lay, 0.2, cfg_id=19)
+    T, L = lay.ctx_len, lay.affix_len
+    shared_k, shared_v = case.cache_k[0].copy(), case.cache_v[0].copy()      # [T, Hkv, d]; only affix rows matter
+    dc = DeviceCase(case)
+    dsk, dsv = ab.to_device_bf16(shared_k[None], DEV), ab.to_device_bf16(shared_v[None], DEV)
+    kv = ab.KV(dsk.data_ptr(), dsv.data_ptr(), 0, T)
+    K = orc.k_from_ratio(L, 0.2)
+    n = K + lay.n_extra
+    # scores from masked-row queries computed by the oracle (any queries would do)
+    q = wl.random_q_mask(shape, lay, 91)
+    dq = ab.to_device_bf16(q, DEV)
+    scores = torch.zeros((B, L), dtype=torch.float32, device=DEV)
+    dc.ctx.score_anchors(dc.req, dq, kv, scores)
+    anchors = torch.zeros((B, K), dtype=torch.int32, device=DEV)
+    dc.ctx.select_topk(scores, B, L, K, anchors)
+    k_new = torch.zeros((B, n, shape.n_kv_heads, shape.head_dim), dtype=torch.bfloat16, device=DEV)
+    v_new = torch.zeros_like(k_new)
+    y = torch.zeros((B, n, shape.hidden), dtype=torch.bfloat16, device=DEV)
+    dc.ctx.recompute_anchors(dc.lw, dc.req, kv, dc.x, 0, anchors, K, k_new, v_new, y)
+    torch.cuda.synchronize()
+    assert dc.ctx.poll_status() == 0
+    assert np.array_equal(ab.to_host_bits(dsk[0]), shared_k) and np.array_equal(ab.to_host_bits(dsv[0]), shared_v)
+    s_gpu, a_gpu = scores.cpu().numpy(), anchors.cpu().numpy()
+    for b in range(B):
+        kf = orc.bf16_bits_to_f64(shared_k[:T])
+        s_ref = orc.score_anchors(orc.bf16_bits_to_f64(q[b]), kf[lay.affix_start:lay.affix_start + L])
+        assert (np.abs(s_gpu[b] - s_ref) / np.maximum(s_ref, s_ref.mean())).max() < 1e-3
+        _, _, must, may = orc.select_topk(s_ref.astype(np.float32), K)
+        ok, why = orc.anchor_set_ok(a_gpu[b], K, L, must, may)
+        assert ok, why
+        # the oracle with a private copy of the shared cache for this request
+        ref = orc.layer_step(case.weights, shape, case.x[b], shared_k, shared_v, T, lay.affix_start, L,
+                             lay.masked_pos[b], lay.extra_rows[b], case.rope_cos, case.rope_sin, anchor_idx=a_gpu[b])
+        assert_close_bf16(ab.to_host_bits(k_new[b]), ref["k_new"], "private K")
+        assert_close_bf16(ab.to_host_bits(v_new[b]), ref["v_new"], "private V")
+        assert_close_bf16(ab.to_host_bits(y[b]), ref["y"], "y")
+    # calls that write the cache refuse a shared one
+    with pytest.raises(ab.AcacheError):
+        dc.ctx.scatter_kv(dc.req, kv, anchors, K, k_new, v_new)
+    with pytest.raises(ab.AcacheError):
+        dc.ctx.layer_step(dc.lw, dc.req, kv, dc.x, 0, 0.2, 0, None, anchors, y)
