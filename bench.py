@@ -483,6 +483,154 @@ def run_denoise(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------
+SWEEP_L = (512, 2048, 8192)
+SWEEP_RATIO = (0.05, 0.10, 0.20, 0.35, 0.50)
+SWEEP_B = (1, 8, 64)
+SWEEP_PLACE = ("prefix", "middle", "suffix")
+
+
+def run_sweep(args):
+    """Benchmark configuration 5: layer-step time, per-stage time and roofline fraction over affix
+    length x recompute ratio x batch x affix placement on LLaDA-8B layer shapes (anchors only,
+    32 masked rows, 64 request rows).  Timing-only inputs are drawn on the device (normal
+    activations and cache entries at the scale the seeded host generator uses; the affix rows of x
+    and of the cache are one draw shared by the batch); parity at sweep points is covered by the tests."""
+    import torch
+    from paper_2608_26140_b200 import binding as ab
+    from paper_2608_26140_b200 import build as abuild
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    abuild.build()
+    shape = wl.LLADA_8B
+    peaks = load_peaks()
+    host_w = wl.layer_weights(shape, 5, 0)
+    n_inst = max(1, min(args.instances, 4))
+    winst = []
+    for _ in range(n_inst):
+        w = {k: (ab.to_device_bf16(v, dev) if v is not None else None) for k, v in host_w.items()}
+        winst.append((w, ab.Context.weights(w)))
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.SEED_BASE + 4096 * 5)
+    kv_std = 0.02 * float(np.sqrt(shape.hidden))
+    Ls = [int(v) for v in args.sweep_affix.split(",")] if args.sweep_affix else SWEEP_L
+    Bs = [int(v) for v in args.sweep_batch.split(",")] if args.sweep_batch else SWEEP_B
+    sampler = ClockSampler(0)
+    sampler.start()
+    points, launches, tot_tokens, tot_s = [], 0, 0.0, 0.0
+    flags = ab.F_SCORE | ab.F_SELECT
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for L in Ls:
+        for B in Bs:
+            T = L + 96
+            row = shape.n_kv_heads * shape.head_dim
+            cache_bytes = 2 * B * T * row * 2
+            n_cache = n_inst if cache_bytes < (1 << 28) else 1
+            xs, cks, cvs = [], [], []
+            for _ in range(n_cache):
+                x = torch.randn((B, T, shape.hidden), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16) \
+                    if B * T * shape.hidden < (1 << 30) else \
+                    torch.cat([torch.randn((1, T, shape.hidden), generator=gen, device=dev, dtype=torch.bfloat16)
+                               for _ in range(B)])
+                ck = (torch.randn((B, T, shape.n_kv_heads, shape.head_dim), generator=gen, device=dev,
+                                  dtype=torch.bfloat16) * kv_std)
+                cv = (torch.randn((B, T, shape.n_kv_heads, shape.head_dim), generator=gen, device=dev,
+                                  dtype=torch.bfloat16) * kv_std)
+                xs.append(x); cks.append(ck); cvs.append(cv)
+            cos_h, sin_h = wl.rope_table(T, shape.head_dim, shape.rope_theta)
+            cos, sin = torch.from_numpy(cos_h).to(dev), torch.from_numpy(sin_h).to(dev)
+            for place in SWEEP_PLACE:
+                lay = wl.sweep_layout(L, B, place, "none")
+                l = lay.affix_start
+                for x, ck, cv in zip(xs, cks, cvs):           # the affix is shared by the batch
+                    x[1:, l:l + L] = x[0:1, l:l + L]
+                    ck[1:, l:l + L] = ck[0:1, l:l + L]
+                    cv[1:, l:l + L] = cv[0:1, l:l + L]
+                masked = torch.from_numpy(lay.masked_pos.copy()).to(dev)
+                req = ab.Context.request(B, T, l, L, masked, None, cos, sin)
+                for ratio in SWEEP_RATIO:
+                    K = ab.k_from_ratio(L, ratio)
+                    ctx = ab.Context.for_shape(shape, B, T, L, K, lay.n_masked, dev)
+                    scores = torch.zeros((B, L), dtype=torch.float32, device=dev)
+                    anchors = torch.zeros((B, K), dtype=torch.int32, device=dev)
+                    y = torch.zeros((B, K, shape.hidden), dtype=torch.bfloat16, device=dev)
+
+                    def step(i):
+                        c = i % n_cache
+                        ctx.layer_step(winst[i % n_inst][1], req, ab.Context.kv(cks[c], cvs[c]), xs[c], 0, ratio, flags,
+                                       scores, anchors, y)
+
+                    for i in range(3):
+                        step(i)
+                    torch.cuda.synchronize()
+                    e0.record(); step(3); e1.record()
+                    torch.cuda.synchronize()
+                    steps = int(min(args.steps, max(3, 0.2 / max(e0.elapsed_time(e1) * 1e-3, 1e-6))))
+                    l0 = ctx.launch_count()
+                    e0.record()
+                    for i in range(steps):
+                        step(i)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    launches += ctx.launch_count() - l0
+                    s_step = e0.elapsed_time(e1) * 1e-3 / steps
+                    ctx.stage_timing(True)
+                    stage = {s: 0.0 for s in ab.STAGES}
+                    for i in range(min(steps, 5)):
+                        step(i)
+                        for s_, v in ctx.read_stage_times().items():
+                            stage[s_] += v / min(steps, 5)
+                    ctx.stage_timing(False)
+                    assert ctx.poll_status() == 0, "device status word set during the sweep"
+                    step_bytes, step_flops, _, _, n_r = step_work(shape, lay, K)
+                    t_hbm, t_tc = step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (peaks["tflops"] * 1e12)
+                    floor = max(t_hbm, t_tc)
+                    points.append({"L": L, "B": B, "place": place, "ratio": ratio, "K": K, "rows": n_r, "steps": steps,
+                                   "us": s_step * 1e6, "floor_us": floor * 1e6, "bound": "hbm" if t_hbm >= t_tc else "tensor",
+                                   "frac": floor / s_step, "gbs": step_bytes / s_step / 1e9,
+                                   "tflops": step_flops / s_step / 1e12,
+                                   "tensor_util": step_flops / s_step / 1e12 / peaks["tflops"],
+                                   "stage_us": {k: round(v * 1e3, 1) for k, v in stage.items()}})
+                    tot_tokens += B * K * steps
+                    tot_s += s_step * steps
+                    del ctx, scores, anchors, y
+            del xs, cks, cvs
+            torch.cuda.empty_cache()
+    sampler.stop_flag = True
+    sampler.join()
+    fr = sorted(p["frac"] for p in points)
+    by = {b: sorted(p["frac"] for p in points if p["bound"] == b) for b in ("hbm", "tensor")}
+    med = lambda v: (v[len(v) // 2] if v else None)  # noqa: E731
+    if args.sweep_out:
+        with open(args.sweep_out, "w") as f:
+            f.write("| L | B | place | ratio | K | rows | µs/layer-step | floor µs | bound | frac | TFLOP/s | GB/s | "
+                    + " | ".join(ab.STAGES) + " |\n")
+            f.write("|" + "---|" * (12 + len(ab.STAGES)) + "\n")
+            for p in points:
+                f.write(f"| {p['L']} | {p['B']} | {p['place']} | {p['ratio']} | {p['K']} | {p['rows']} | {p['us']:.1f} | "
+                        f"{p['floor_us']:.1f} | {p['bound']} | {p['frac']:.3f} | {p['tflops']:.1f} | {p['gbs']:.0f} | "
+                        + " | ".join(f"{p['stage_us'][s_]:.1f}" for s_ in ab.STAGES) + " |\n")
+    print(json.dumps({
+        "metric": METRIC, "value": tot_tokens / tot_s, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": 3,
+        "ms_per_step": tot_s / max(1, sum(p["steps"] for p in points)) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic (device-drawn, timing only)",
+        "config": {"workload": f"cfg5 sweep: LLaDA-8B layer, affix {list(Ls)} x ratio {list(SWEEP_RATIO)} x batch {list(Bs)} x "
+                               f"placement {list(SWEEP_PLACE)}, 64 request + 32 masked rows, anchors only; value = anchors "
+                               "refreshed over all points / time over all points", "benchmark_config": 5,
+                   "l2": f"{n_inst} weight instances rotated; caches rotated while smaller than 256 MB"},
+        "clocks": sampler.summary(), "gpu_launches": int(launches),
+        "roofline": {"bound": "mixed", "frac_min": fr[0], "frac_median": med(fr), "frac_max": fr[-1],
+                     "frac_median_hbm_bound": med(by["hbm"]), "frac_median_tensor_bound": med(by["tensor"]),
+                     "peak_source": peaks["source"], "peak_hbm_gbs": peaks["hbm_gbs"], "peak_tflops": peaks["tflops"]},
+        "points": points,
+    }))
+
+
 def cpu_baseline(case, shape, lay):
     """The oracle as it stands, timed on this machine's host cores on one step of the workload."""
     from oracle import acache_oracle as orc
@@ -517,11 +665,16 @@ def main():
     ap.add_argument("--instances", type=int, default=4, help="weight/cache instances rotated between steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=32, help="layers of the --config 3 denoising step")
+    ap.add_argument("--sweep-affix", default=None, help="--config 5: comma-separated affix lengths (default 512,2048,8192)")
+    ap.add_argument("--sweep-batch", default=None, help="--config 5: comma-separated batch sizes (default 1,8,64)")
+    ap.add_argument("--sweep-out", default=None, help="--config 5: also write the points as a markdown table to this file")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     elif args.config == 3:
         run_denoise(args)
+    elif args.config == 5:
+        run_sweep(args)
     else:
         run_ours(args)
 

@@ -348,7 +348,10 @@ const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int6
 int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream) {
     if (a.head_dim != 128 || a.slot || a.batch == 0 || a.n == 0) return 0;
     const int q_tiles = (a.n + 127) / 128;
-    if ((int64_t)q_tiles * a.n_heads * a.batch < 148) return 0;       // few rows: the key-split kernel fills the machine better
+    // measured at batch 1 with 26-4096 rows over 600-8300 keys: never slower than the key-split mma.sync
+    // kernel, even with a single query tile per head (32 CTAs)
+    static const int min_ctas = [] { const char* e = getenv("ACACHE_ATTN_TC_MIN_CTAS"); return e ? atoi(e) : 1; }();
+    if ((int64_t)q_tiles * a.n_heads * a.batch < min_ctas) return 0;       // few rows: the key-split kernel fills the machine better
     if ((a.kv_batch_stride * 2) % 16) return 0;
     std::lock_guard<std::mutex> lock(g_map3_mutex);
     const CUtensorMap* mq = get_map3(a.q, a.n, a.n_heads * 128, a.batch, (int64_t)a.n * a.n_heads * 128);
