@@ -4,8 +4,8 @@
 // rows past the request's row count read as zero).
 //
 //   S = Q K^T    tcgen05.mma 128 x 128 x 16, both operands K-major, into one of two TMEM buffers
-//   softmax      four warps, thread = query row: scaled max, exp2, running denominator; P is
-//                written as bf16 into a 128-byte-swizzled shared tile
+//   softmax      eight warps, two threads per query row (64 keys each): scaled max, exp2, running
+//                denominator; P is written as bf16 into a 128-byte-swizzled shared tile
 //   O += P V     tcgen05.mma 128 x 128 x 16, A = P (K-major over keys), B = V read in place as an
 //                MN-major operand (token-major V rows are contiguous along the head dimension)
 //
@@ -24,7 +24,7 @@
 
 namespace acache {
 
-constexpr int AT_THREADS = 192;                  // warp 0: TMA, warp 1: MMA, warps 2-5: softmax (thread = row)
+constexpr int AT_THREADS = 320;                  // warp 0: TMA, warp 1: MMA, warps 2-9: softmax (two threads per row)
 constexpr int AT_TILE = 128 * 128 * 2;           // 32 KB: a [128 x 128] bf16 tile as two 64-column panels
 constexpr int AT_PANEL = 128 * 64 * 2;           // 16 KB
 constexpr int AT_SMEM = 7 * AT_TILE + 1024 + 256;   // Q, K x2, V x2, P x2
@@ -54,6 +54,16 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// 2^x on the FMA pipe for x <= ~8 (Cody-Waite: x = n + f with n = rint(x), |f| <= 0.5; a cubic for 2^f
+// with relative error 7.5e-5, far below the bf16 rounding of P; n goes straight into the exponent).
+// A quarter of the exponentials take this route so that the MUFU pipe is not the only one working.
+__device__ __forceinline__ float poly_exp2(float x) {
+    x = fmaxf(x, -126.f);
+    const float t = x + 12582912.f;                 // 1.5 * 2^23: the low mantissa bits now hold rint(x)
+    const float f = x - (t - 12582912.f);
+    const float p = fmaf(fmaf(fmaf(0.05517146f, f, 0.24261086f), f, 0.69326097f), f, 0.9999281f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // MN-major bf16 operand with the 128-byte swizzle: rows of the K index are 128 bytes (64 elements
@@ -79,6 +89,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1)
 attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                     const __grid_constant__ CUtensorMap mapV) {
     extern __shared__ unsigned char smem_raw[];
+    __shared__ uint16_t row_max[2][2][128];  // [tile parity][key half][row]: upper halves of fp32, rounded up
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t sQ = base, sK0 = base + AT_TILE, sV0 = base + 3 * AT_TILE, sP0 = base + 5 * AT_TILE;
@@ -95,8 +106,8 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(11), 4); mbar_init(bar(12), 4);      // s_empty: the four softmax warps
-        mbar_init(bar(13), 4); mbar_init(bar(14), 4);      // p_full
+        mbar_init(bar(11), 8); mbar_init(bar(12), 8);      // s_empty: the eight softmax warps
+        mbar_init(bar(13), 8); mbar_init(bar(14), 8);      // p_full
         mbar_init(bar(15), 1); mbar_init(bar(16), 1);      // p_empty
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -179,32 +190,57 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             tc_commit(bar(7 + s));     // v_empty
         }
     } else if (warp >= 2) {
-        // ---------------- softmax: thread = query row ----------------
+        // ---------------- softmax: two threads per query row ----------------
+        // Warps 2-5 take keys 0-63 of every tile (and columns 0-63 of O), warps 6-9 the other half; the
+        // two threads of a row agree on the row maximum through shared memory once per tile.  The two
+        // warps of a row quarter meet at a named barrier every tile, so they only ever leave the loop together: a wait
+        // that ran out sets the abort flag, the thread skips its work, and everyone breaks after the
+        // next barrier.
+        const int wg = (warp - 2) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+        const uint32_t col_off = (uint32_t)(wg * 64);
         float m_use = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_tiles && ok; ++j) {
+        for (int j = 0; j < n_tiles; ++j) {
             const int s = j & 1;
-            if (!(ok = mbar_wait(bar(9 + s), (j >> 1) & 1, abort_flag))) break;
-            tc_fence_after();
-            const uint32_t tS = tS0 + s * 128 + lane_off;
-            const int valid = a.ctx_len - j * 128;
-            // the whole row of S into registers, then the S buffer is free for tile j + 2
-            float sv[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tc_ld32(tS + c * 32, sv[c]);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(11 + s));   // s_empty
+            const int valid = a.ctx_len - j * 128 - wg * 64;       // keys of this thread's half that exist
+            float sv[2][32];
             float mt = -INFINITY;
+            if (ok && (ok = mbar_wait(bar(9 + s), (j >> 1) & 1, abort_flag))) {
+                tc_fence_after();
+                const uint32_t tS = tS0 + s * 128 + col_off + lane_off;
+                // this thread's half row of S into registers, then the S buffer is free for tile j + 2
+                tc_ld32(tS, sv[0]);
+                tc_ld32(tS + 32, sv[1]);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(11 + s));   // s_empty
+                float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                if (valid >= 64) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+                    for (int c = 0; c < 2; ++c)
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c * 32 + i < valid) mt = fmaxf(mt, sv[c][i]);
-            mt *= a.scale_log2e;
+                        for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], sv[c][i]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (c * 32 + i < valid) m4[i & 3] = fmaxf(m4[i & 3], sv[c][i]);
+                }
+                mt = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * a.scale_log2e;
+            }
+            // the two threads of a row must use the same number: both take the larger of the two
+            // half-row maxima rounded up to 16 significant bits (an upper bound is all the exponent needs)
+            uint32_t mb = __float_as_uint(mt);
+            if ((mb & 0xFFFFu) && !(mb >> 31)) mb += 0x10000u;
+            mb >>= 16;
+            row_max[s][wg][row] = (uint16_t)mb;
+            asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");      // the two warps that share these 32 rows
+            if (*abort_flag) { ok = false; break; }
+            mt = fmaxf(__uint_as_float(mb << 16), __uint_as_float((uint32_t)row_max[s][wg ^ 1][row] << 16));
             bool raise = false;
             if (j == 0) {
                 m_use = mt;
@@ -213,56 +249,73 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             }
             if (__any_sync(0xffffffffu, raise)) {
                 // O may only be touched once the P V of tile j - 1 has completed
-                if (!(ok = mbar_wait(bar(15 + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag))) break;
-                tc_fence_after();
-                const float f = raise ? fast_exp2(m_use - mt) : 1.f;
-                for (int c = 0; c < 4; ++c) {
-                    float v[32];
-                    tc_ld32(tO + lane_off + c * 32, v);
+                if ((ok = mbar_wait(bar(15 + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag))) {
+                    tc_fence_after();
+                    const float f = raise ? fast_exp2(m_use - mt) : 1.f;
+                    for (int c = 0; c < 2; ++c) {
+                        float v[32];
+                        tc_ld32(tO + lane_off + col_off + c * 32, v);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] *= f;
-                    tc_st32(tO + lane_off + c * 32, v);
+                        for (int i = 0; i < 32; ++i) v[i] *= f;
+                        tc_st32(tO + lane_off + col_off + c * 32, v);
+                    }
+                    tc_wait_st();
+                    l *= f;
+                    if (raise) m_use = mt;
                 }
-                tc_wait_st();
-                l *= f;
-                if (raise) m_use = mt;
             }
             // this P buffer was last read by the P V of tile j - 2
-            if (j >= 2 && !(ok = mbar_wait(bar(15 + s), ((j - 2) >> 1) & 1, abort_flag))) break;
-            const uint32_t sP = sP0 + s * AT_TILE;
+            if (ok && j >= 2) ok = mbar_wait(bar(15 + s), ((j - 2) >> 1) & 1, abort_flag);
+            if (!ok) continue;
+            const uint32_t sP = sP0 + s * AT_TILE + wg * AT_PANEL + row * 128;
+            float l4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
+                if (valid >= 64) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float p = c * 32 + i < valid ? fast_exp2(sv[c][i] * a.scale_log2e - m_use) : 0.f;
-                    l += p;
-                    sv[c][i] = p;
+                    for (int i = 0; i < 32; ++i) {
+                        const float x = fmaf(sv[c][i], a.scale_log2e, -m_use);
+                        const float p = (i & 3) == 3 ? poly_exp2(x) : fast_exp2(x);
+                        l4[i & 3] += p;
+                        sv[c][i] = p;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float p = c * 32 + i < valid ? fast_exp2(fmaf(sv[c][i], a.scale_log2e, -m_use)) : 0.f;
+                        l4[i & 3] += p;
+                        sv[c][i] = p;
+                    }
                 }
 #pragma unroll
                 for (int k8 = 0; k8 < 4; ++k8) {
-                    const int chunk = c * 4 + k8;                 // 16-byte chunk of the row: 8 keys
-                    const uint32_t addr = sP + (chunk >> 3) * AT_PANEL + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
+                    const int chunk = c * 4 + k8;                 // 16-byte chunk of this half row: 8 keys
+                    const uint32_t addr = sP + ((chunk ^ (row & 7)) << 4);
                     const float* pv = sv[c] + k8 * 8;
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(pv[0], pv[1])),
                                  "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])), "r"(pack_bf16(pv[6], pv[7]))
                                  : "memory");
                 }
             }
+            l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
             tc_fence_before();
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core's async proxy
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(13 + s));   // p_full
         }
-        // epilogue: O / l once the last P V has completed
+        // epilogue: O / l once the last P V has completed; the denominators of the two halves add up
         if (ok && n_tiles > 0) ok = mbar_wait(bar(15 + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, abort_flag);
-        if (ok) {
+        float* row_sum = reinterpret_cast<float*>(base_ptr + 5 * AT_TILE);     // the P buffers are idle now
+        row_sum[wg * 128 + row] = l;
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");
+        if (ok && !*abort_flag) {
             tc_fence_after();
             const int grow = qt * 128 + row;
-            const float inv = 1.f / l;
-            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o) + (((int64_t)b * a.n + grow) * a.n_heads + h) * 128;
-            for (int c = 0; c < 4; ++c) {
+            const float inv = 1.f / (l + row_sum[(wg ^ 1) * 128 + row]);
+            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o) + (((int64_t)b * a.n + grow) * a.n_heads + h) * 128 + col_off;
+            for (int c = 0; c < 2; ++c) {
                 float v[32];
-                tc_ld32(tO + lane_off + c * 32, v);
+                tc_ld32(tO + lane_off + col_off + c * 32, v);
                 if (grow < a.n) {
 #pragma unroll
                     for (int k8 = 0; k8 < 4; ++k8) {
@@ -351,7 +404,7 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     // measured at batch 1 with 26-4096 rows over 600-8300 keys: never slower than the key-split mma.sync
     // kernel, even with a single query tile per head (32 CTAs)
     static const int min_ctas = [] { const char* e = getenv("ACACHE_ATTN_TC_MIN_CTAS"); return e ? atoi(e) : 1; }();
-    if ((int64_t)q_tiles * a.n_heads * a.batch < min_ctas) return 0;       // few rows: the key-split kernel fills the machine better
+    if ((int64_t)q_tiles * a.n_heads * a.batch < min_ctas) return 0;
     if ((a.kv_batch_stride * 2) % 16) return 0;
     std::lock_guard<std::mutex> lock(g_map3_mutex);
     const CUtensorMap* mq = get_map3(a.q, a.n, a.n_heads * 128, a.batch, (int64_t)a.n * a.n_heads * 128);

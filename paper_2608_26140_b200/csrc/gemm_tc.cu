@@ -815,289 +815,6 @@ gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __gr
     }
 }
 
-// ---- few rows (one row tile): K split across a thread-block cluster, summed through DSMEM --------
-// A cluster of S CTAs owns an output tile; CTA r contracts K blocks [r KB / S, (r + 1) KB / S) into
-// its TMEM accumulator, copies it to its own shared memory (the drained ring), and after a cluster
-// barrier every CTA sums, in ascending rank order (bitwise reproducible), the 16-column items
-// r, r + S, ... of all S copies through distributed shared memory and applies the epilogue.  No
-// partial tile goes to global memory and no second kernel follows.  S = 1 is the whole-K case
-// (epilogue straight from TMEM).  Clusters walk tiles cluster_id, cluster_id + n_clusters, ...
-__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t cluster_addr) {
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void drain_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-// Column groups (of 4 fp32) of work item `item` of N tile nt: 16 columns at pc0 and, for the
-// paired epilogues, 16 more at pc1.  False if the item lies past the end of the output.
-__device__ __forceinline__ bool item_columns(const GemmArgs& g, const TcPlan& p, int nt, int item, int& pc0, int& pc1,
-                                             int& u128, int& lo_col) {
-    const int half = g.head_dim >> 1;
-    pc1 = -1; u128 = 0; lo_col = 0;
-    if (g.epilogue == kEpiResidual) {
-        pc0 = item * 4;
-    } else if (g.epilogue == kEpiSwiGLU) {
-        pc0 = item * 4; pc1 = 32 + pc0;
-    } else {
-        const int h = item >> 2, r = item & 3;
-        u128 = nt * 2 + h;
-        if (u128 >= p.units) return false;
-        lo_col = g.head_dim == 128 ? 16 * r : 64 * (r >> 1) + 16 * (r & 1);
-        pc0 = 32 * h + (lo_col >> 2);
-        pc1 = pc0 + (half >> 2);
-    }
-    return true;
-}
-
-__global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tcs_kernel(const GemmArgs g, const TcPlan p, const int S, const __grid_constant__ CUtensorMap mapA,
-                const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
-                const __grid_constant__ CUtensorMap mapB2) {
-    extern __shared__ unsigned char smem_raw[];
-    __shared__ float red[TC_THREADS / 32];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bars = base + TC_STAGES * TC_STAGE_BYTES;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + TC_STAGES * TC_STAGE_BYTES + 192);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + TC_STAGES * TC_STAGE_BYTES + 200);
-    auto full_bar = [&](int s) { return bars + 8 * s; };
-    auto empty_bar = [&](int s) { return bars + 8 * (TC_STAGES + s); };
-    auto tfull_bar = [&](int i) { return bars + 8 * (2 * TC_STAGES + i); };
-    auto tempty_bar = [&](int i) { return bars + 8 * (2 * TC_STAGES + 2 + i); };
-    const uint32_t staged_bar = bars + 8 * (2 * TC_STAGES + 4), drained_bar = staged_bar + 8;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rank = S > 1 ? (int)cluster_ctarank() : 0;
-    const int cluster_id = blockIdx.x / S, n_clusters = gridDim.x / S;
-    unsigned int nbar = 0;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 4); }
-        mbar_init(staged_bar, S);
-        mbar_init(drained_bar, S);
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
-                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (S > 1) cluster_sync_all();       // every CTA's barriers exist before a peer signals them
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    const int kb_lo = (int)(((int64_t)rank * p.KB) / S), kb_hi = (int)(((int64_t)(rank + 1) * p.KB) / S);
-    // The weights are constant inputs: fill the ring's weight halves for the first tile and ask L2
-    // for the K blocks after that while the previous kernel is still finishing.
-    constexpr int kPrefetchL2 = 12;
-    int prefilled = 0;
-    if (warp == 0 && lane == 0 && cluster_id < p.n_tiles) {
-        const CUtensorMap* maps[3] = {&mapB0, &mapB1, &mapB2};
-        const uint64_t pol_w = policy_evict_first();
-        int row0, row1;
-        const int s0 = half_source(g, p, cluster_id, 0, row0), s1 = half_source(g, p, cluster_id, 1, row1);
-        for (int i = 0; i < TC_STAGES + kPrefetchL2 && kb_lo + i < kb_hi; ++i) {
-            const int kb = kb_lo + i;
-            if (i < TC_STAGES) {
-                const uint32_t sB = base + i * TC_STAGE_BYTES + TC_A_BYTES;
-                mbar_expect_tx(full_bar(i), TC_A_BYTES + TC_HALF_BYTES * (1 + (s1 >= 0)));
-                tma_load_2d(sB, maps[s0], kb * TC_BK, row0, full_bar(i), pol_w);
-                if (s1 >= 0) tma_load_2d(sB + TC_HALF_BYTES, maps[s1], kb * TC_BK, row1, full_bar(i), pol_w);
-                prefilled = i + 1;
-            } else {
-                tma_prefetch_2d(maps[s0], kb * TC_BK, row0);
-                if (s1 >= 0) tma_prefetch_2d(maps[s1], kb * TC_BK, row1);
-            }
-        }
-    }
-    pdl_wait();
-    pdl_launch_dependents();
-
-    if (g.prep.enabled) prep_phase(g, red, abort_flag, nbar);
-
-    if (warp == 0 && lane == 0) {
-        // TMA producer
-        const CUtensorMap* maps[3] = {&mapB0, &mapB1, &mapB2};
-        int stage = 0;
-        uint32_t phase = 0, tile_phase = 0;
-        bool ok = !*abort_flag;
-        const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
-        for (int nt = cluster_id; nt < p.n_tiles && ok; nt += n_clusters) {
-            if (S > 1 && nt != cluster_id) {
-                // the ring doubles as the staging area of the previous tile's sum: wait until every
-                // CTA of the cluster has read it
-                if (!(ok = mbar_wait_cluster(drained_bar, tile_phase, abort_flag))) break;
-                tile_phase ^= 1;
-                asm volatile("fence.proxy.async;" ::: "memory");
-            }
-            int row0, row1;
-            const int s0 = half_source(g, p, nt, 0, row0), s1 = half_source(g, p, nt, 1, row1);
-            const uint32_t bytes = TC_A_BYTES + TC_HALF_BYTES * (1 + (s1 >= 0));
-            for (int kb = kb_lo; kb < kb_hi; ++kb) {
-                const uint32_t sA = base + stage * TC_STAGE_BYTES, sB = sA + TC_A_BYTES;
-                if (prefilled > 0) {
-                    --prefilled;
-                    tma_load_2d(sA, &mapA, kb * TC_BK, 0, full_bar(stage), pol_a);
-                } else {
-                    if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag))) break;
-                    mbar_expect_tx(full_bar(stage), bytes);
-                    tma_load_2d(sA, &mapA, kb * TC_BK, 0, full_bar(stage), pol_a);
-                    tma_load_2d(sB, maps[s0], kb * TC_BK, row0, full_bar(stage), pol_w);
-                    if (s1 >= 0) tma_load_2d(sB + TC_HALF_BYTES, maps[s1], kb * TC_BK, row1, full_bar(stage), pol_w);
-                }
-                if (++stage == TC_STAGES) { stage = 0; phase ^= 1; }
-            }
-        }
-    } else if (warp == 1 && lane == 0) {
-        // MMA issuer
-        int stage = 0, acc = 0;
-        uint32_t phase = 0, acc_phase = 0;
-        bool ok = !*abort_flag;
-        for (int nt = cluster_id; nt < p.n_tiles && ok; nt += n_clusters) {
-            int row1;
-            const uint32_t idesc = idesc_bf16(half_source(g, p, nt, 1, row1) >= 0 ? 256 : 128);
-            if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag))) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + acc * TC_BN;
-            for (int kb = kb_lo; kb < kb_hi; ++kb) {
-                if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag))) break;
-                tc_fence_after();
-                const uint32_t sA = base + stage * TC_STAGE_BYTES, sB = sA + TC_A_BYTES;
-                const uint64_t da = smem_desc_sw128(sA), db = smem_desc_sw128(sB);
-#pragma unroll
-                for (int k = 0; k < TC_BK / 16; ++k)
-                    tc_mma(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > kb_lo || k > 0) ? 1u : 0u);
-                tc_commit(empty_bar(stage));
-                if (++stage == TC_STAGES) { stage = 0; phase ^= 1; }
-            }
-            if (!ok) break;
-            tc_commit(tfull_bar(acc));
-            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
-        }
-    } else if (warp >= 2 && warp < 6) {
-        const int q = warp & 3;
-        const int row = q * 32 + lane;
-        const bool valid = row < g.M;
-        int acc = 0;
-        uint32_t acc_phase = 0, tile_phase = 0;
-        bool ok = !*abort_flag;
-        bool pending_drain = false;
-        float4* stg = reinterpret_cast<float4*>(base_ptr);      // [column group][row] of float4
-        for (int nt = cluster_id; nt < p.n_tiles && ok; nt += n_clusters) {
-            int row1;
-            const int nchunks = half_source(g, p, nt, 1, row1) >= 0 ? 8 : 4;
-            // With S > 1 the four drain warps meet at named barriers, so they must leave the loop
-            // together: after every bounded wait they synchronise and then test the shared abort flag.
-            ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
-            if (S > 1) {
-                if (pending_drain) mbar_wait_cluster(drained_bar, tile_phase ^ 1, abort_flag);   // previous copy read by all
-                drain_bar_sync();
-                ok = !*abort_flag;
-            }
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + acc * TC_BN + ((uint32_t)(q * 32) << 16);
-            if (S == 1) {
-                direct_epilogue(g, p, taddr, nt, row, valid, nchunks);
-            } else {
-                for (int c = 0; c < nchunks; ++c) {
-                    float v[32];
-                    tc_ld32(taddr + c * 32, v);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        stg[(c * 8 + i) * TC_BM + row] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                }
-            }
-            // the accumulator is free again
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
-            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
-            if (S == 1) continue;
-            drain_bar_sync();
-            if (warp == 2 && lane < S) mbar_arrive_cluster(mapa_u32(staged_bar, lane));
-            mbar_wait_cluster(staged_bar, tile_phase, abort_flag);
-            drain_bar_sync();
-            if (!(ok = !*abort_flag)) break;
-            const int n_items = finish_items_per_tile(g.epilogue);
-            const int pos = (g.epilogue == kEpiQKV && valid) ? __ldcg(g.row_pos + row) : 0;
-            for (int item = rank; item < n_items; item += S) {
-                int pc0, pc1, u128, lo_col;
-                if (!item_columns(g, p, nt, item, pc0, pc1, u128, lo_col) || !valid) continue;
-                float lo[16], hi[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) { lo[i] = 0.f; hi[i] = 0.f; }
-                const uint32_t a0 = smem_u32(stg + pc0 * TC_BM + row), a1 = smem_u32(stg + (pc1 < 0 ? pc0 : pc1) * TC_BM + row);
-                for (int c = 0; c < S; c += 2) {
-                    float4 a[2][4], b[2][4];
-                    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const bool in = c + i < S;
-                        const uint32_t r0 = mapa_u32(a0, in ? c + i : c), r1 = mapa_u32(a1, in ? c + i : c);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            a[i][j] = in ? ld_dsmem_f4(r0 + j * TC_BM * 16) : zero;
-                            b[i][j] = (in && pc1 >= 0) ? ld_dsmem_f4(r1 + j * TC_BM * 16) : zero;
-                        }
-                    }
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        if (c + i < S) {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                lo[4 * j] += a[i][j].x; lo[4 * j + 1] += a[i][j].y; lo[4 * j + 2] += a[i][j].z; lo[4 * j + 3] += a[i][j].w;
-                                hi[4 * j] += b[i][j].x; hi[4 * j + 1] += b[i][j].y; hi[4 * j + 2] += b[i][j].z; hi[4 * j + 3] += b[i][j].w;
-                            }
-                        }
-                    }
-                }
-                if (g.epilogue == kEpiResidual) {
-                    out_residual<16>(g, row, nt * TC_BN + item * 16, lo);
-                } else if (g.epilogue == kEpiSwiGLU) {
-                    out_swiglu<16>(g, row, nt * 128 + item * 16, lo, hi);
-                } else {
-                    int seg, c0;
-                    qkv_unit(g, u128, seg, c0);
-                    out_qkv<16>(g, row, pos, seg, c0 + lo_col, lo_col & ((g.head_dim >> 1) - 1), lo, hi);
-                }
-            }
-            // this CTA has read every copy: tell the owners
-            drain_bar_sync();
-            if (warp == 2 && lane < S) mbar_arrive_cluster(mapa_u32(drained_bar, lane));
-            pending_drain = true;
-            tile_phase ^= 1;
-        }
-        // nobody may still be reading this CTA's copy when it leaves
-        if (pending_drain && ok) mbar_wait_cluster(drained_bar, tile_phase ^ 1, abort_flag);
-        // (after an expired wait the peers may still be reading: the teardown below lingers first)
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (*abort_flag) {
-        if (threadIdx.x == 0) {
-            atomicOr(g.status, kFlagWaitExpired);
-            for (int i = 0; i < 4096; ++i) __nanosleep(64);
-        }
-        __syncthreads();
-    } else if (threadIdx.x == 0 && nbar > 0) {
-        __threadfence();
-        if (atomicAdd(&g.grid_bar[1], 1u) == gridDim.x - 1) {
-            g.grid_bar[0] = 0u;
-            __threadfence();
-            g.grid_bar[1] = 0u;
-        }
-    }
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
-    }
-}
-
 // Finish of the split tiles: grid row y finishes tile split.tile[y]; blockIdx.x * 256 +
 // threadIdx.x -> (item, row).
 struct SplitTiles {
@@ -1338,48 +1055,6 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
         cfg.gridDim = dim3(clusters * 2);
         if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, g, p, clusters, *mA, *mB[0], *mB[1], *mB[2]) != cudaSuccess) return -1;
         return 1;
-    }
-    // Few rows (one row tile) and no more tiles than SMs: S CTAs per tile as a cluster, K split
-    // between them and summed through DSMEM inside the kernel (S = 1: whole K per CTA).
-    static const int cluster_on = [] { const char* e = getenv("ACACHE_GEMM_CLUSTER"); return e ? atoi(e) : 0; }();
-    if (cluster_on && p.m_tiles == 1 && g.epilogue != kEpiLogits && p.n_tiles <= sm_count()) {
-        static bool attr_s = false;
-        if (!attr_s) {
-            cudaFuncSetAttribute(gemm_tcs_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
-            attr_s = true;
-        }
-        int S = std::min(std::min(8, sm_count() / p.n_tiles), p.KB);
-        static int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
-        cudaLaunchConfig_t cfg{};
-        cfg.blockDim = dim3(TC_THREADS);
-        cfg.dynamicSmemBytes = TC_SMEM;
-        cfg.stream = stream;
-        cudaLaunchAttribute at[2];
-        at[0].id = cudaLaunchAttributeClusterDimension;
-        at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = at;
-        cfg.numAttrs = 2;
-        // all clusters must be resident at once (DSMEM sums, and phase 0 ends in a grid-wide barrier)
-        for (; S >= 1; --S) {
-            at[0].val.clusterDim.x = S;
-            cfg.gridDim = dim3(S * p.n_tiles);
-            if (!max_clusters[S]) {
-                int n = 0;
-                if (cudaOccupancyMaxActiveClusters(&n, gemm_tcs_kernel, &cfg) != cudaSuccess || n <= 0) {
-                    (void)cudaGetLastError();
-                    n = -1;
-                }
-                max_clusters[S] = n;
-            }
-            if (max_clusters[S] >= p.n_tiles) break;
-        }
-        // (if only much smaller clusters fit, the stream-K kernel below uses the SMs better)
-        if (S >= 1 && 2 * S * p.n_tiles >= std::min(sm_count(), p.n_tiles * p.KB)) {
-            if (cudaLaunchKernelEx(&cfg, gemm_tcs_kernel, g, p, S, *mA, *mB[0], *mB[1], *mB[2]) != cudaSuccess) return -1;
-            return 1;
-        }
     }
 single_cta:
     // a plain launch: a cooperative one measured ~2.5 us slower and cannot overlap the previous
