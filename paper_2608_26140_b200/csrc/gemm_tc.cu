@@ -331,50 +331,116 @@ __device__ __forceinline__ void direct_epilogue(const GemmArgs& g, const TcPlan&
     }
 }
 
-// Phase 0 of the projection kernels: the rows of R (or compact rows) -> RMSNorm -> the A operand,
-// one row per CTA at a time, then a grid-wide barrier; the rows are read back through TMA.
-__device__ __forceinline__ void prep_phase(const GemmArgs& g, float* red, volatile int* abort_flag, unsigned int& nbar) {
+// Where row `row` of the A operand comes from (element offset inside rp.x); `writer` (one thread per
+// row) records the row's position and source for the later kernels and raises the bad-index flag.
+__device__ __forceinline__ int64_t prep_row_source(const GemmArgs& g, int row, bool writer) {
     const RowPrep& rp = g.prep;
     const int rows_per_req = rp.k + rp.e;
-    for (int row = blockIdx.x; row < g.M; row += gridDim.x) {
-        int64_t src = (int64_t)row * g.K;
-        if (rp.enabled == 3) {       // compact rows picked by index
-            const int b = row / rows_per_req;
-            const int ci = rp.compact_idx[row];
-            if (ci < 0 || ci >= rp.compact_rows) {
-                if (threadIdx.x == 0) atomicOr(g.status, kFlagBadIndex);
-            }
-            src = ((int64_t)b * rp.compact_rows + (ci < 0 || ci >= rp.compact_rows ? 0 : ci)) * g.K;
+    int64_t src = (int64_t)row * g.K;
+    if (rp.enabled == 3) {       // compact rows picked by index
+        const int b = row / rows_per_req;
+        const int ci = rp.compact_idx[row];
+        if (ci < 0 || ci >= rp.compact_rows) {
+            if (writer) atomicOr(g.status, kFlagBadIndex);
         }
-        if (rp.enabled == 1) {       // rows of R: position from the anchor / extra-row lists
-            const int b = row / rows_per_req, i = row - b * rows_per_req;
-            const int pos = row_position(rp.anchor_idx, rp.k, rp.extra_rows, rp.e, b, i, rp.affix_start,
-                                         rp.affix_len, rp.ctx_len);
-            if (!rp.x_is_compact) {
-                if (rp.token_ids) {       // x is an embedding table: the row of the token at that position
-                    int id = rp.token_ids[(int64_t)b * rp.ctx_len + (pos < 0 ? 0 : pos)];
-                    if (id < 0 || id >= rp.table_rows) {
-                        if (threadIdx.x == 0) atomicOr(g.status, kFlagBadIndex);
-                        id = 0;
-                    }
-                    src = (int64_t)id * g.K;
-                } else {
-                    src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
+        src = ((int64_t)b * rp.compact_rows + (ci < 0 || ci >= rp.compact_rows ? 0 : ci)) * g.K;
+    }
+    if (rp.enabled == 1) {       // rows of R: position from the anchor / extra-row lists
+        const int b = row / rows_per_req, i = row - b * rows_per_req;
+        const int pos = row_position(rp.anchor_idx, rp.k, rp.extra_rows, rp.e, b, i, rp.affix_start,
+                                     rp.affix_len, rp.ctx_len);
+        if (!rp.x_is_compact) {
+            if (rp.token_ids) {       // x is an embedding table: the row of the token at that position
+                int id = rp.token_ids[(int64_t)b * rp.ctx_len + (pos < 0 ? 0 : pos)];
+                if (id < 0 || id >= rp.table_rows) {
+                    if (writer) atomicOr(g.status, kFlagBadIndex);
+                    id = 0;
                 }
-            } else if (rp.compact_idx) {
-                const int ci = rp.compact_idx[row];
-                src = ((int64_t)b * rp.compact_rows + (ci < 0 ? 0 : ci)) * g.K;
+                src = (int64_t)id * g.K;
+            } else {
+                src = (int64_t)b * rp.x_batch_stride + (int64_t)(pos < 0 ? 0 : pos) * g.K;
             }
-            if (threadIdx.x == 0) {
-                rp.row_pos[row] = pos;
-                rp.row_src[row] = src;
-                if (pos < 0) atomicOr(g.status, kFlagBadIndex);
+        } else if (rp.compact_idx) {
+            const int ci = rp.compact_idx[row];
+            src = ((int64_t)b * rp.compact_rows + (ci < 0 ? 0 : ci)) * g.K;
+        }
+        if (writer) {
+            rp.row_pos[row] = pos;
+            rp.row_src[row] = src;
+            if (pos < 0) atomicOr(g.status, kFlagBadIndex);
+        }
+    }
+    return src;
+}
+
+// out = bf16(x * rsqrt(mean(x^2) + eps) * g) for one row, by one warp: two passes over the row with
+// eight independent 16-byte loads in flight per lane (the second pass hits L1 / L2).
+__device__ __forceinline__ void rmsnorm_row_warp(const uint4* __restrict__ xr, const uint4* __restrict__ gn,
+                                                 uint4* __restrict__ out, int hidden, float eps, int lane) {
+    const int nchunk = hidden >> 3;
+    float ss = 0.f;
+    for (int c0 = 0; c0 < nchunk; c0 += 256) {
+        uint4 u[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int c = c0 + i * 32 + lane;
+            u[i] = c < nchunk ? __ldcg(xr + c) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { const float a = bf16_lo(w[e]), b = bf16_hi(w[e]); ss += a * a + b * b; }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const float rstd = rsqrtf(ss / (float)hidden + eps);
+    for (int c0 = 0; c0 < nchunk; c0 += 256) {
+        uint4 u[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int c = c0 + i * 32 + lane;
+            u[i] = c < nchunk ? __ldcg(xr + c) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int c = c0 + i * 32 + lane;
+            if (c < nchunk) {
+                const uint4 gg = __ldg(gn + c);
+                const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+                const uint32_t gw[4] = {gg.x, gg.y, gg.z, gg.w};
+                uint32_t r[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    r[e] = pack_bf16(bf16_lo(w[e]) * rstd * bf16_lo(gw[e]), bf16_hi(w[e]) * rstd * bf16_hi(gw[e]));
+                out[c] = make_uint4(r[0], r[1], r[2], r[3]);
             }
         }
-        rmsnorm_row(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(rp.x) + src),
-                    reinterpret_cast<const uint4*>(rp.gain),
-                    reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(const_cast<void*>(g.a)) + (int64_t)row * g.K),
-                    g.K, rp.eps, red);
+    }
+}
+
+// Phase 0 of the projection kernels: the rows of R (or compact rows) -> RMSNorm -> the A operand,
+// then a grid-wide barrier; the rows are read back through TMA.  With no more rows than CTAs a
+// whole CTA takes a row (shortest latency); with many rows every warp takes rows of its own, which
+// keeps six rows in flight per SM instead of one.
+__device__ __forceinline__ void prep_phase(const GemmArgs& g, float* red, volatile int* abort_flag, unsigned int& nbar) {
+    const RowPrep& rp = g.prep;
+    const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(rp.x);
+    __nv_bfloat16* a_out = static_cast<__nv_bfloat16*>(const_cast<void*>(g.a));
+    if (g.M <= (int)gridDim.x) {
+        for (int row = blockIdx.x; row < g.M; row += gridDim.x) {
+            const int64_t src = prep_row_source(g, row, threadIdx.x == 0);
+            rmsnorm_row(reinterpret_cast<const uint4*>(x + src), reinterpret_cast<const uint4*>(rp.gain),
+                        reinterpret_cast<uint4*>(a_out + (int64_t)row * g.K), g.K, rp.eps, red);
+        }
+    } else {
+        const int nw = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int row = blockIdx.x * nw + warp; row < g.M; row += gridDim.x * nw) {
+            const int64_t src = prep_row_source(g, row, lane == 0);
+            rmsnorm_row_warp(reinterpret_cast<const uint4*>(x + src), reinterpret_cast<const uint4*>(rp.gain),
+                             reinterpret_cast<uint4*>(a_out + (int64_t)row * g.K), g.K, rp.eps, lane);
+        }
     }
     asm volatile("fence.proxy.async;" ::: "memory");   // the rows are read back through TMA
     grid_barrier(g.grid_bar, ++nbar, abort_flag);
