@@ -572,11 +572,13 @@ def run_sweep(args):
                     torch.cuda.synchronize()
                     steps = int(min(args.steps, max(3, 0.2 / max(e0.elapsed_time(e1) * 1e-3, 1e-6))))
                     l0 = ctx.launch_count()
+                    c0 = len(sampler.sm)
                     e0.record()
                     for i in range(steps):
                         step(i)
                     e1.record()
                     torch.cuda.synchronize()
+                    clk = sampler.sm[c0:] or sampler.sm[-1:]
                     launches += ctx.launch_count() - l0
                     s_step = e0.elapsed_time(e1) * 1e-3 / steps
                     ctx.stage_timing(True)
@@ -591,7 +593,7 @@ def run_sweep(args):
                     t_hbm, t_tc = step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (peaks["tflops"] * 1e12)
                     floor = max(t_hbm, t_tc)
                     points.append({"L": L, "B": B, "place": place, "ratio": ratio, "K": K, "rows": n_r, "steps": steps,
-                                   "us": s_step * 1e6, "floor_us": floor * 1e6, "bound": "hbm" if t_hbm >= t_tc else "tensor",
+                                   "us": s_step * 1e6, "sm_mhz": float(np.median(clk)) if clk else None, "floor_us": floor * 1e6, "bound": "hbm" if t_hbm >= t_tc else "tensor",
                                    "frac": floor / s_step, "gbs": step_bytes / s_step / 1e9,
                                    "tflops": step_flops / s_step / 1e12,
                                    "tensor_util": step_flops / s_step / 1e12 / peaks["tflops"],
@@ -608,12 +610,12 @@ def run_sweep(args):
     med = lambda v: (v[len(v) // 2] if v else None)  # noqa: E731
     if args.sweep_out:
         with open(args.sweep_out, "w") as f:
-            f.write("| L | B | place | ratio | K | rows | µs/layer-step | floor µs | bound | frac | TFLOP/s | GB/s | "
+            f.write("| L | B | place | ratio | K | rows | µs/layer-step | SM MHz | floor µs | bound | frac | TFLOP/s | GB/s | "
                     + " | ".join(ab.STAGES) + " |\n")
-            f.write("|" + "---|" * (12 + len(ab.STAGES)) + "\n")
+            f.write("|" + "---|" * (13 + len(ab.STAGES)) + "\n")
             for p in points:
                 f.write(f"| {p['L']} | {p['B']} | {p['place']} | {p['ratio']} | {p['K']} | {p['rows']} | {p['us']:.1f} | "
-                        f"{p['floor_us']:.1f} | {p['bound']} | {p['frac']:.3f} | {p['tflops']:.1f} | {p['gbs']:.0f} | "
+                        f"{p['sm_mhz'] or 0:.0f} | {p['floor_us']:.1f} | {p['bound']} | {p['frac']:.3f} | {p['tflops']:.1f} | {p['gbs']:.0f} | "
                         + " | ".join(f"{p['stage_us'][s_]:.1f}" for s_ in ab.STAGES) + " |\n")
     print(json.dumps({
         "metric": METRIC, "value": tot_tokens / tot_s, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": 3,
