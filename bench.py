@@ -401,6 +401,9 @@ def run_denoise(args):
     def step():
         ctx.denoise_step(lws, kvs, req, embed, da, K, ya, yb, dbr, n_blk, gain, w_lm, V, 0.9, token, conf, commit)
 
+    if args.generate:
+        return run_generate(args, locals())
+
     def sync_all():
         torch.cuda.synchronize()
         if dist:
@@ -633,6 +636,79 @@ def run_sweep(args):
     }))
 
 
+def run_generate(args, e):
+    """Benchmark configuration 3, one whole block decoded with the refresh-then-decode schedule
+    (acache_generate_block): one refresh pass over R = anchors + all request rows, then decode passes
+    over the block's 32 rows until every request has committed its block (random-init weights never
+    reach the 0.9 threshold, so every pass commits exactly one token per request: the longest schedule)."""
+    import torch
+    from paper_2608_26140_b200 import binding as ab
+    ctx, dist, dev, world, rank = e["ctx"], e["dist"], e["dev"], e["world"], e["rank"]
+    lay, B, T, L, K, n, V, n_blk, shape, n_layers = (e["lay"], e["B"], e["T"], e["L"], e["K"], e["n"], e["V"], e["n_blk"],
+                                                   e["shape"], e["n_layers"])
+    ids0 = torch.from_numpy(e["ids"]).to(dev)
+    dids = e["dids"]
+    block_pos = torch.from_numpy(np.ascontiguousarray(lay.masked_pos[:, :n_blk])).to(dev)
+    req_d = ab.Context.request(B, T, lay.affix_start, L, e["masked"], block_pos, e["cos"], e["sin"], token_ids=dids, n_embed=V)
+    rows_d = torch.arange(n_blk, dtype=torch.int32, device=dev).repeat(B, 1).contiguous()
+    left = torch.zeros((B,), dtype=torch.int32, device=dev)
+
+    def block():
+        dids.copy_(ids0)
+        return ctx.generate_block(e["lws"], e["kvs"], e["req"], req_d, e["embed"], e["da"], K, e["ya"], e["yb"], e["dbr"], rows_d,
+                                  n_blk, e["gain"], e["w_lm"], V, 0.9, V - 1, n_blk + 1, e["token"], e["conf"], e["commit"], left)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    block()                                   # warm-up: one whole block (33 model passes at most)
+    sync_all()
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    l0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_blocks = max(1, min(args.steps, 3))
+    e0.record()
+    passes = 0
+    for _ in range(n_blocks):
+        passes += block()
+    e1.record()
+    sync_all()
+    sampler.stop_flag = True
+    sampler.join()
+    launches = ctx.launch_count() - l0
+    ms_block = sharding.max_over_ranks(e0.elapsed_time(e1), dist, dev) / n_blocks
+    assert ctx.poll_status() == 0
+    assert int(left.sum().item()) == 0, "the block was not fully decoded"
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    peaks = load_peaks()
+    tokens = world * B * n_blk
+    print(json.dumps({
+        "metric": "generated_tokens_per_s", "value": tokens / (ms_block * 1e-3), "unit": "generated tokens/s",
+        "n_gpus": world, "steps": n_blocks, "warmup": 1, "ms_per_step": ms_block, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic; random-init weights: no confidence reaches the threshold, so each pass commits one token per request",
+        "config": {"workload": f"cfg3 block decode: LLaDA-8B shapes, {n_layers} layers, vocab {V}, batch {B}/GPU sharing a {L}-token "
+                               f"prefix affix, one {n_blk}-token block per request: 1 refresh pass ({n} rows per request, K={K}) + "
+                               f"decode passes over the block's {n_blk} rows", "benchmark_config": 3, "layers": n_layers,
+                   "model_passes_per_block": passes / n_blocks, "parallelism": f"request-sharded x{world}"},
+        "clocks": sampler.summary(), "gpu_launches": int(launches), "ms_per_block": ms_block,
+        "ms_per_model_pass": ms_block / (passes / n_blocks),
+        "e2e": {"value": tokens / (ms_block * 1e-3), "unit": "generated tokens/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": int(4 * B * passes / n_blocks),
+                "note": "the schedule reads 4 bytes per request back after every model pass (inside the timed region)"},
+        "roofline": {"bound": "mixed", "peak_source": peaks["source"], "note": "refresh pass tensor-bound, decode passes (512 rows) near the weight-streaming floor"},
+    }))
+    if dist:
+        dist.destroy_process_group()
+
+
 def cpu_baseline(case, shape, lay):
     """The oracle as it stands, timed on this machine's host cores on one step of the workload."""
     from oracle import acache_oracle as orc
@@ -667,6 +743,8 @@ def main():
     ap.add_argument("--instances", type=int, default=4, help="weight/cache instances rotated between steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=32, help="layers of the --config 3 denoising step")
+    ap.add_argument("--generate", action="store_true",
+                    help="--config 3: decode one whole 32-token block per request (refresh + decode passes)")
     ap.add_argument("--sweep-affix", default=None, help="--config 5: comma-separated affix lengths (default 512,2048,8192)")
     ap.add_argument("--sweep-batch", default=None, help="--config 5: comma-separated batch sizes (default 1,8,64)")
     ap.add_argument("--sweep-out", default=None, help="--config 5: also write the points as a markdown table to this file")

@@ -284,6 +284,57 @@ acache_status acache_denoise_step(acache_ctx *ctx, int32_t n_layers, const acach
                                   const void *w_lm, int32_t vocab, float threshold, int32_t *token,
                                   float *confidence, int32_t *commit, acache_stream_t stream);
 
+/* The one-shot probe and the selection it feeds (Section 3.2): every request's request-specific rows
+ * (req->extra_rows = all non-affix positions, which must include the masked ones) go through the
+ * n_layers layers with the affix K/V as cached; at every layer the masked rows' queries are scored
+ * against the cached affix keys (Eq. 4) and the scores accumulate over the layers (Eq. 5); then
+ * Eq. 6 picks K = acache_k_from_ratio(affix_len, ratio) anchors once for all layers.  Equivalent to
+ * n_layers calls of acache_layer_step(ratio 0, ACACHE_F_SCORE [| ACACHE_F_ACCUMULATE]) followed by
+ * acache_select_topk; like them it writes the fresh K/V of the request-specific rows into kvs.
+ *   flags: 0 or ACACHE_F_SCORE_NORM_FULL.  layers, kvs: HOST arrays (DEVICE pointers inside).
+ *   x0: DEVICE bf16 [B, ctx_len, D], or the embedding table when req->token_ids is set.
+ *   y_a, y_b: DEVICE bf16 [B, e, D] each (layer outputs alternate between them).
+ *   scores: DEVICE fp32 [B, L] (overwritten); anchor_idx: DEVICE int32 [B, K] ascending. */
+acache_status acache_probe_select(acache_ctx *ctx, int32_t n_layers, const acache_layer_weights *layers,
+                                  acache_kv *kvs, const acache_request *req, const void *x0, double ratio,
+                                  uint32_t flags, void *y_a, void *y_b, float *scores, int32_t *anchor_idx,
+                                  acache_stream_t stream);
+
+/* Eq. 3 applied to the sequence: among the block's positions block_pos[b, i] whose token id is still
+ * mask_id, those with confidence[b, i] > threshold receive token[b, i]; if a request has masked
+ * positions but none qualifies, its single most confident masked position does (lowest i on ties).
+ * Positions already decoded are left alone whatever their confidence.
+ *   token_ids: DEVICE int32 [B, ctx_len], updated in place; block_pos: DEVICE int32 [B, n_blk] absolute
+ *   positions; token, confidence: DEVICE [B, n_blk] as written by acache_predict_commit for those rows;
+ *   remaining: DEVICE int32 [B], masked positions left in the block after the update.
+ * A position outside [0, ctx_len) raises ACACHE_FLAG_BAD_INDEX and is skipped. */
+acache_status acache_commit_update(acache_ctx *ctx, int32_t *token_ids, int32_t ctx_len, const int32_t *block_pos,
+                                   int32_t batch, int32_t n_blk, const int32_t *token, const float *confidence,
+                                   int32_t mask_id, float threshold, int32_t *remaining, acache_stream_t stream);
+
+/* Decoding of one block with the refresh-then-decode schedule of Section 4.3 / Section 5: step 0 is
+ * acache_denoise_step over R = A u E (req_refresh: anchors + all request-specific rows), which brings
+ * the caches up to date; every later step recomputes only the block's rows (req_decode: k = 0,
+ * extra_rows = the block's positions) over the same caches.  After each step acache_commit_update
+ * writes the committed tokens into token_ids; the loop ends when no request has a masked position
+ * left in the block or after max_steps steps.
+ *   Both requests must name the same token_ids (DEVICE int32 [B, ctx_len], updated in place); embed is
+ *   the embedding table [n_embed, D].  block_rows_refresh / block_rows_decode: DEVICE int32 [B, n_blk],
+ *   the compact row of each block position inside the rows of the refresh / decode pass (the latter
+ *   normally 0 .. n_blk-1).  y_a, y_b: DEVICE bf16 [B, K+e, D] sized for the refresh pass.
+ *   token, confidence, commit: DEVICE [B, n_blk] (the last step's predictions); remaining: DEVICE [B].
+ *   steps_done: HOST, number of model passes run.
+ * THIS CALL SYNCHRONISES the stream once per step (it reads `remaining` back, 4 bytes per request). */
+acache_status acache_generate_block(acache_ctx *ctx, int32_t n_layers, const acache_layer_weights *layers,
+                                    acache_kv *kvs, const acache_request *req_refresh,
+                                    const acache_request *req_decode, const void *embed,
+                                    const int32_t *anchor_idx, int32_t k, void *y_a, void *y_b,
+                                    const int32_t *block_rows_refresh, const int32_t *block_rows_decode,
+                                    int32_t n_blk, const void *final_norm_g, const void *w_lm, int32_t vocab,
+                                    float threshold, int32_t mask_id, int32_t max_steps, int32_t *token,
+                                    float *confidence, int32_t *commit, int32_t *remaining, int32_t *steps_done,
+                                    acache_stream_t stream);
+
 /* acache_layer_step for a caller whose per-step data lives in HOST memory: copies
  * x [B, ctx_len, D] (HOST bf16, ideally pinned) to a staging area in the workspace,
  * runs the layer-step with ACACHE_F_SCORE | ACACHE_F_SELECT | flags, and copies y

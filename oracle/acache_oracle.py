@@ -433,6 +433,60 @@ def predict_commit(h_rows: np.ndarray, final_norm_g: np.ndarray, w_lm: np.ndarra
     return token, conf, commit, z
 
 
+def commit_update(token_ids: np.ndarray, block_pos: np.ndarray, token: np.ndarray, confidence: np.ndarray,
+                  mask_id: int, threshold: float) -> int:
+    """Eq. 3 on one request's sequence: the block positions that still hold ``mask_id`` and whose
+    confidence exceeds the threshold receive their predicted token; if there are masked positions
+    but none qualifies, the single most confident masked one does (lowest index on ties).
+    Already decoded positions are left alone.  ``token_ids`` [T] is updated in place; returns the
+    number of masked positions left in the block."""
+    masked = [i for i, p in enumerate(block_pos) if token_ids[p] == mask_id]
+    if not masked:
+        return 0
+    hits = [i for i in masked if confidence[i] > threshold]
+    if not hits:
+        best = masked[0]
+        for i in masked[1:]:
+            if confidence[i] > confidence[best]:
+                best = i
+        hits = [best]
+    for i in hits:
+        token_ids[block_pos[i]] = token[i]
+    return len(masked) - len(hits)
+
+
+def generate_block(layers, shape, embed: np.ndarray, final_norm_g: np.ndarray, w_lm: np.ndarray,
+                   token_ids: np.ndarray, caches, ctx_len: int, affix_start: int, anchor_idx: np.ndarray,
+                   request_rows: np.ndarray, block_pos: np.ndarray, cos, sin, mask_id: int, threshold: float,
+                   max_steps: int, round_storage: bool = True):
+    """One request, one block, refresh-then-decode (Section 4.3 with the threshold schedule of
+    Section 5): step 0 recomputes R = A u E (anchors + all request-specific rows) through all layers
+    from the token embeddings, later steps only the block's rows over the caches the earlier steps
+    left; after every step the block rows are predicted (Eq. 2) and Eq. 3 commits into ``token_ids``.
+
+    embed [V, D] bf16 bits; token_ids [T] int (updated in place); caches: list of (K, V) bf16 bits.
+    Returns (steps, working caches, history) where history[s] = (token, confidence, token_ids copy)."""
+    history = []
+    steps = 0
+    for step in range(max_steps):
+        if step == 0:
+            a_idx, extra = np.asarray(anchor_idx), np.asarray(request_rows)
+        else:
+            a_idx, extra = np.zeros((0,), np.int64), np.asarray(block_pos)
+        x0 = embed[np.asarray(token_ids[:ctx_len], dtype=np.int64)]
+        rows, caches, ys = refresh_forward(layers, shape, x0, caches, ctx_len, affix_start, a_idx, extra, cos, sin,
+                                           round_storage)
+        where = {int(p): i for i, p in enumerate(rows)}
+        h = ys[-1][[where[int(p)] for p in block_pos]]
+        token, conf, _, _ = predict_commit(h, final_norm_g, w_lm, shape.rms_eps, threshold, round_storage)
+        left = commit_update(token_ids, block_pos, token, conf, mask_id, threshold)
+        history.append((token.copy(), conf.copy(), np.array(token_ids).copy()))
+        steps = step + 1
+        if left == 0:
+            break
+    return steps, caches, history
+
+
 # --------------------------------------------------------------------------
 # comparison helpers used by the parity tests
 # --------------------------------------------------------------------------

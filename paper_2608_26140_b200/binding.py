@@ -22,7 +22,8 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_last_error", "acache_poll_status", "acache_launch_count", "acache_score_anchors",
            "acache_k_from_ratio", "acache_select_topk", "acache_recompute_anchors", "acache_scatter_kv",
            "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times",
-           "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step"]
+           "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step", "acache_probe_select",
+           "acache_commit_update", "acache_generate_block"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -110,6 +111,15 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_denoise_step.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request), vp, vp, i32,
                                         vp, vp, C.POINTER(vp), vp, i32, vp, vp, i32, C.c_float, vp, vp, vp, vp]
     lib.acache_denoise_step.restype = C.c_int
+    lib.acache_probe_select.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request), vp,
+                                        C.c_double, u32, vp, vp, vp, vp, vp]
+    lib.acache_probe_select.restype = C.c_int
+    lib.acache_commit_update.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, i32, C.c_float, vp, vp]
+    lib.acache_commit_update.restype = C.c_int
+    lib.acache_generate_block.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request),
+                                          C.POINTER(Request), vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, i32, C.c_float,
+                                          i32, i32, vp, vp, vp, vp, C.POINTER(i32), vp]
+    lib.acache_generate_block.restype = C.c_int
     lib.acache_stage_timing.argtypes = [vp, C.c_int]
     lib.acache_stage_timing.restype = C.c_int
     lib.acache_read_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
@@ -271,6 +281,34 @@ class Context:
                                                  _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold), _ptr(token),
                                                  _ptr(confidence), _ptr(commit), _stream()))
         return last.value
+
+    def probe_select(self, layers, kvs, req: Request, x0, ratio, flags, y_a, y_b, scores, anchor_idx):
+        n = len(layers)
+        la = (LayerWeights * n)(*layers)
+        ka = (KV * n)(*kvs)
+        self._check(self.lib.acache_probe_select(self.h, n, la, ka, C.byref(req), _ptr(x0), float(ratio), int(flags),
+                                                 _ptr(y_a), _ptr(y_b), _ptr(scores), _ptr(anchor_idx), _stream()))
+
+    def commit_update(self, token_ids, ctx_len, block_pos, batch, n_blk, token, confidence, mask_id, threshold, remaining):
+        self._check(self.lib.acache_commit_update(self.h, _ptr(token_ids), ctx_len, _ptr(block_pos), batch, n_blk,
+                                                  _ptr(token), _ptr(confidence), int(mask_id), float(threshold),
+                                                  _ptr(remaining), _stream()))
+
+    def generate_block(self, layers, kvs, req_refresh: Request, req_decode: Request, embed, anchor_idx, k, y_a, y_b,
+                       block_rows_refresh, block_rows_decode, n_blk, final_norm_g, w_lm, vocab, threshold, mask_id,
+                       max_steps, token, confidence, commit, remaining) -> int:
+        """Returns the number of model passes run (synchronises the stream once per pass)."""
+        n = len(layers)
+        la = (LayerWeights * n)(*layers)
+        ka = (KV * n)(*kvs)
+        steps = C.c_int32(0)
+        self._check(self.lib.acache_generate_block(self.h, n, la, ka, C.byref(req_refresh), C.byref(req_decode), _ptr(embed),
+                                                   _ptr(anchor_idx), k, _ptr(y_a), _ptr(y_b), _ptr(block_rows_refresh),
+                                                   _ptr(block_rows_decode), n_blk, _ptr(final_norm_g), _ptr(w_lm), vocab,
+                                                   float(threshold), int(mask_id), int(max_steps), _ptr(token),
+                                                   _ptr(confidence), _ptr(commit), _ptr(remaining), C.byref(steps),
+                                                   _stream()))
+        return int(steps.value)
 
     def layer_step_host(self, w: LayerWeights, req: Request, kv: KV, x_host, ratio, flags, scores_host,
                         anchor_idx_host, y_host):

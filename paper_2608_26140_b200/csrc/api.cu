@@ -560,6 +560,85 @@ acache_status acache_denoise_step(acache_ctx* ctx, int32_t n_layers, const acach
                                  confidence, commit, stream);
 }
 
+acache_status acache_probe_select(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers, acache_kv* kvs,
+                                  const acache_request* req, const void* x0, double ratio, uint32_t flags, void* y_a,
+                                  void* y_b, float* scores, int32_t* anchor_idx, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (n_layers <= 0 || !layers || !kvs || !req || !x0 || !y_a || !y_b || !scores)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL argument or n_layers <= 0");
+    if (flags & ~(uint32_t)ACACHE_F_SCORE_NORM_FULL) return fail(ctx, ACACHE_ERR_INVALID_ARG, "only ACACHE_F_SCORE_NORM_FULL is accepted here");
+    const int k = acache_k_from_ratio(req->affix_len, ratio);
+    if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
+    const void* x = x0;
+    for (int n = 0; n < n_layers; ++n) {
+        void* y = (n & 1) ? y_b : y_a;
+        // K = 0 anchors: the rows are the request-specific ones; the affix keys stay as cached (stale)
+        acache_status s = acache_layer_step(ctx, &layers[n], req, &kvs[n], x, n > 0, 0.0,
+                                            flags | ACACHE_F_SCORE | (n > 0 ? ACACHE_F_ACCUMULATE : 0u), scores, nullptr, y, stream);
+        if (s != ACACHE_OK) return s;
+        x = y;
+    }
+    return acache_select_topk(ctx, scores, req->batch, req->affix_len, k, anchor_idx, stream);
+}
+
+acache_status acache_commit_update(acache_ctx* ctx, int32_t* token_ids, int32_t ctx_len, const int32_t* block_pos,
+                                   int32_t batch, int32_t n_blk, const int32_t* token, const float* confidence,
+                                   int32_t mask_id, float threshold, int32_t* remaining, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!ctx->ws) return fail(ctx, ACACHE_ERR_WORKSPACE, "workspace not set");
+    if (batch < 0 || n_blk < 0 || ctx_len <= 0) return fail(ctx, ACACHE_ERR_INVALID_ARG, "negative size");
+    if (batch == 0) return ACACHE_OK;
+    if (!token_ids || !remaining || (n_blk > 0 && (!block_pos || !token || !confidence)))
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL pointer");
+    launch_commit_update(token_ids, ctx_len, block_pos, batch, n_blk, token, confidence, mask_id, threshold, remaining,
+                         wsp<uint32_t>(ctx, ctx->o_status), stream);
+    ctx->launches += 1;
+    return check_cuda(ctx, "commit_update");
+}
+
+acache_status acache_generate_block(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers, acache_kv* kvs,
+                                    const acache_request* req_refresh, const acache_request* req_decode,
+                                    const void* embed, const int32_t* anchor_idx, int32_t k, void* y_a, void* y_b,
+                                    const int32_t* block_rows_refresh, const int32_t* block_rows_decode, int32_t n_blk,
+                                    const void* final_norm_g, const void* w_lm, int32_t vocab, float threshold,
+                                    int32_t mask_id, int32_t max_steps, int32_t* token, float* confidence,
+                                    int32_t* commit, int32_t* remaining, int32_t* steps_done, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!req_refresh || !req_decode || !steps_done || !remaining)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL argument");
+    if (!req_refresh->token_ids || req_refresh->token_ids != req_decode->token_ids)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "both requests must name the same token_ids array");
+    if (req_decode->n_extra != n_blk || req_decode->batch != req_refresh->batch || req_decode->ctx_len != req_refresh->ctx_len)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "req_decode must recompute exactly the block's n_blk rows of the same batch");
+    if (req_refresh->batch > 4096) return fail(ctx, ACACHE_ERR_INVALID_ARG, "batch too large for the step loop");
+    *steps_done = 0;
+    if (req_refresh->batch == 0 || n_blk == 0 || max_steps <= 0) return ACACHE_OK;
+    int32_t* ids = const_cast<int32_t*>(req_refresh->token_ids);
+    int32_t left[4096];
+    for (int step = 0; step < max_steps; ++step) {
+        // step 0 refreshes the anchors and every request-specific row; later steps only the block's rows
+        const bool refresh = step == 0;
+        const acache_request* r = refresh ? req_refresh : req_decode;
+        acache_status s = acache_denoise_step(ctx, n_layers, layers, kvs, r, embed, refresh ? anchor_idx : nullptr,
+                                              refresh ? k : 0, y_a, y_b, nullptr,
+                                              refresh ? block_rows_refresh : block_rows_decode, n_blk, final_norm_g, w_lm,
+                                              vocab, threshold, token, confidence, commit, stream);
+        if (s != ACACHE_OK) return s;
+        s = acache_commit_update(ctx, ids, r->ctx_len, req_decode->extra_rows, r->batch, n_blk, token, confidence, mask_id,
+                                 threshold, remaining, stream);
+        if (s != ACACHE_OK) return s;
+        *steps_done = step + 1;
+        // the schedule ends when no request has a masked position left in the block: one small read-back per step
+        if (cudaMemcpyAsync(left, remaining, sizeof(int32_t) * r->batch, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess)
+            return check_cuda(ctx, "generate_block read-back") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "read-back failed") : ACACHE_ERR_CUDA;
+        int total = 0;
+        for (int b = 0; b < r->batch; ++b) total += left[b];
+        if (total == 0) break;
+    }
+    return ACACHE_OK;
+}
+
 acache_status acache_layer_step_host(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
                                      acache_kv* kv, const void* x_host, double ratio, uint32_t flags,
                                      float* scores_host, int32_t* anchor_idx_host, void* y_host,

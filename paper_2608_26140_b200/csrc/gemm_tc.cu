@@ -48,6 +48,7 @@ constexpr uint32_t GRID_WAIT_LIMIT = 1u << 21;
 
 struct TcPlan {
     int m_tiles, n_tiles, KB, tiles, U, ctas, smax;
+    int prefetch;         // K blocks past the ring whose weight tiles are requested into L2 before the dependency wait
     int units;            // 128-row B halves over all segments (non-SwiGLU) or ffn/128 (SwiGLU)
 };
 
@@ -485,7 +486,7 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     // The weights are constant inputs (no earlier kernel writes them), so their loads may start
     // before the previous kernel has finished: fill the ring's weight halves now and ask L2 for the
     // k-blocks after that.  The activation halves follow once the producer kernel is done.
-    constexpr int kPrefetchL2 = 12;
+    const int kPrefetchL2 = p.prefetch;
     int prefilled = 0;
     if (warp == 0 && lane == 0) {
         const CUtensorMap* maps[3] = {&mapB0, &mapB1, &mapB2};
@@ -1048,6 +1049,8 @@ TcPlan make_plan(int M, int K, int units, bool swiglu) {
     p.U = (int)((total + g - 1) / g);
     p.ctas = (int)((total + p.U - 1) / p.U);
     p.smax = 2;   // partial slots per CTA
+    static const int prefetch = [] { const char* e = getenv("ACACHE_GEMM_PREFETCH"); return e ? atoi(e) : 12; }();
+    p.prefetch = prefetch;
     return p;
 }
 

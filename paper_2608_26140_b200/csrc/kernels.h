@@ -16,6 +16,12 @@ void launch_scatter_kv(void* cache_k, void* cache_v, int64_t batch_stride, int c
 void launch_match_rows(const int32_t* masked_pos, int m, const int32_t* extra_rows, int e, int k, int batch,
                        int32_t* idx, uint32_t* status, cudaStream_t stream);
 
+// Eq. 3 on the sequence state: the block's still-masked positions whose confidence exceeds the threshold
+// (else the single most confident one) receive their predicted token; remaining[b] = masked positions left.
+void launch_commit_update(int32_t* token_ids, int ctx_len, const int32_t* block_pos, int batch, int n_blk,
+                          const int32_t* token, const float* confidence, int mask_id, float threshold,
+                          int32_t* remaining, uint32_t* status, cudaStream_t stream);
+
 // slot[b, t] = compact row index whose fresh K/V replaces position t, or -1.
 void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
                            cudaStream_t stream);

@@ -70,6 +70,65 @@ __global__ void __launch_bounds__(256) match_rows_kernel(const int32_t* __restri
     if (found < 0) atomicOr(status, kFlagBadIndex);
 }
 
+// Eq. 3 on the sequence state: among the block's positions that still hold the mask id, those whose
+// confidence exceeds the threshold receive their predicted token; if none does, the single most
+// confident one (lowest index on ties).  One warp per request; remaining[b] = masked positions left.
+__global__ void __launch_bounds__(32) commit_update_kernel(int32_t* __restrict__ token_ids, int ctx_len,
+                                                           const int32_t* __restrict__ block_pos, int n_blk,
+                                                           const int32_t* __restrict__ token,
+                                                           const float* __restrict__ confidence, int mask_id,
+                                                           float threshold, int32_t* __restrict__ remaining,
+                                                           uint32_t* __restrict__ status) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int b = blockIdx.x, lane = threadIdx.x;
+    int32_t* ids = token_ids + (int64_t)b * ctx_len;
+    int n_masked = 0, n_commit = 0, best_i = -1;
+    float best_c = -INFINITY;
+    for (int i0 = 0; i0 < n_blk; i0 += 32) {
+        const int i = i0 + lane;
+        bool masked = false, hit = false;
+        float c = -INFINITY;
+        int pos = 0;
+        if (i < n_blk) {
+            pos = block_pos[(int64_t)b * n_blk + i];
+            if (pos < 0 || pos >= ctx_len) {
+                atomicOr(status, kFlagBadIndex);
+            } else {
+                masked = ids[pos] == mask_id;
+                c = confidence[(int64_t)b * n_blk + i];
+                hit = masked && c > threshold;
+                if (hit) ids[pos] = token[(int64_t)b * n_blk + i];
+            }
+        }
+        n_masked += __popc(__ballot_sync(0xffffffffu, masked));
+        n_commit += __popc(__ballot_sync(0xffffffffu, hit));
+        // most confident masked row of this chunk, lowest index on ties
+        float cc = masked ? c : -INFINITY;
+        int ci = masked ? i : 0x7fffffff;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float oc = __shfl_xor_sync(0xffffffffu, cc, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, ci, o);
+            if (oc > cc || (oc == cc && oi < ci)) { cc = oc; ci = oi; }
+        }
+        if (ci != 0x7fffffff && (cc > best_c || best_i < 0)) { best_c = cc; best_i = ci; }
+    }
+    if (n_commit == 0 && n_masked > 0 && best_i >= 0) {
+        if (lane == 0) ids[block_pos[(int64_t)b * n_blk + best_i]] = token[(int64_t)b * n_blk + best_i];
+        n_commit = 1;
+    }
+    if (lane == 0) remaining[b] = n_masked - n_commit;
+}
+
+void launch_commit_update(int32_t* token_ids, int ctx_len, const int32_t* block_pos, int batch, int n_blk,
+                          const int32_t* token, const float* confidence, int mask_id, float threshold,
+                          int32_t* remaining, uint32_t* status, cudaStream_t stream) {
+    if (batch == 0) return;
+    launch_pdl(commit_update_kernel, dim3(batch), dim3(32), 0, stream, token_ids, ctx_len, block_pos, n_blk, token, confidence,
+               mask_id, threshold, remaining, status);
+}
+
 void launch_match_rows(const int32_t* masked_pos, int m, const int32_t* extra_rows, int e, int k, int batch,
                        int32_t* idx, uint32_t* status, cudaStream_t stream) {
     if (batch == 0 || m == 0) return;

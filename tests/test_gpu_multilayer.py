@@ -58,6 +58,19 @@ def test_probe_select_refresh(shape, n_layers, norm_full):
     torch.cuda.synchronize()
     s_gpu, a_gpu = scores.cpu().numpy(), anchors.cpu().numpy()
 
+    # ---- the same through the single entry point, on fresh copies of the caches: identical bits
+    dk2 = [ab.to_device_bf16(np.stack([caches[b][n][0] for b in range(B)]), DEV) for n in range(n_layers)]
+    dv2 = [ab.to_device_bf16(np.stack([caches[b][n][1] for b in range(B)]), DEV) for n in range(n_layers)]
+    scores2 = torch.full((B, L), 7.0, dtype=torch.float32, device=DEV)
+    anchors2 = torch.zeros((B, K), dtype=torch.int32, device=DEV)
+    ya, yb = torch.zeros_like(y[0]), torch.zeros_like(y[0])
+    ctx.probe_select(lws, [ab.Context.kv(dk2[n], dv2[n]) for n in range(n_layers)], req, dx, ratio, nf, ya, yb, scores2, anchors2)
+    torch.cuda.synchronize()
+    assert np.array_equal(scores2.cpu().numpy(), s_gpu) and np.array_equal(anchors2.cpu().numpy(), a_gpu)
+    for n in range(n_layers):
+        assert torch.equal(dk2[n], dk[n]) and torch.equal(dv2[n], dv[n])
+    assert torch.equal(yb if n_layers % 2 == 0 else ya, y[-1])
+
     # ---- refresh with the fixed anchor set
     yr = [torch.zeros((B, K + P, shape.hidden), dtype=torch.bfloat16, device=DEV) for _ in range(n_layers)]
     for n in range(n_layers):

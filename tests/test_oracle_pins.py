@@ -475,6 +475,62 @@ def test_predict_commit_vs_library_softmax_and_rule():
     assert np.all(tok3 == 0) and np.allclose(conf3, 1.0 / V) and commit3.tolist() == [True, False, False]
 
 
+def test_commit_update_rule_by_hand():
+    MASK = 99
+    ids = np.array([5, MASK, MASK, 7, MASK, MASK], dtype=np.int32)
+    pos = np.array([1, 2, 3, 4, 5])                       # the block: positions 1..5 (position 3 already decoded)
+    tok = np.array([11, 12, 13, 14, 15], dtype=np.int32)
+    conf = np.array([0.95, 0.2, 0.99, 0.91, 0.3])
+    left = orc.commit_update(ids, pos, tok, conf, MASK, 0.9)
+    assert ids.tolist() == [5, 11, MASK, 7, 14, MASK] and left == 2      # 0.99 at the decoded position is ignored
+    # nobody above the threshold: only the most confident masked position, lowest index on ties
+    conf2 = np.array([0.0, 0.4, 0.8, 0.0, 0.4])
+    left = orc.commit_update(ids, pos, tok, conf2, MASK, 0.9)
+    assert ids.tolist() == [5, 11, 12, 7, 14, MASK] and left == 1
+    left = orc.commit_update(ids, pos, tok, conf2, MASK, 0.9)
+    assert ids.tolist() == [5, 11, 12, 7, 14, 15] and left == 0
+    assert orc.commit_update(ids, pos, tok, conf, MASK, 0.9) == 0 and ids.tolist() == [5, 11, 12, 7, 14, 15]
+
+
+def test_generate_block_schedule_properties():
+    """Refresh-then-decode: end points of the threshold and the structure of the steps."""
+    lay, layers, x, caches, cos, sin = two_layer_case()
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    g = np.random.default_rng(77)
+    V, MASK = 128, 127
+    embed = wl.normal_bf16(901, (V, SMALL.hidden), 1.0)
+    w_lm = wl.normal_bf16(902, (V, SMALL.hidden), 0.5)
+    gain = wl.normal_bf16(903, (SMALL.hidden,), 0.05, 1.0)
+    ids0 = g.integers(0, V - 1, size=T).astype(np.int32)
+    block = lay.masked_pos[0][:8]
+    ids0[lay.masked_pos[0]] = MASK
+    anchors = np.sort(g.choice(L, orc.k_from_ratio(L, 0.25), replace=False))
+    run = lambda thr, steps: orc.generate_block(layers, SMALL, embed, gain, w_lm, ids0.copy(), caches, T, l, anchors,
+                                                lay.extra_rows[0], block, cos, sin, MASK, thr, steps)
+    # threshold below every confidence: everything commits after the refresh step alone
+    steps, c_all, hist = run(-1.0, 20)
+    assert steps == 1 and np.array_equal(hist[0][2][block], hist[0][0])
+    # threshold above 1: exactly one position per step, the most confident masked one each time
+    steps, c_one, hist = run(1.5, 20)
+    assert steps == len(block)
+    prev = ids0
+    for tok, conf, ids in hist:
+        changed = np.flatnonzero(ids != prev)
+        assert changed.size == 1 and prev[changed[0]] == MASK
+        i = int(np.flatnonzero(block == changed[0])[0])
+        still = np.array([prev[p] == MASK for p in block])
+        assert conf[i] == conf[still].max() and ids[changed[0]] == tok[i]
+        prev = ids
+    # step 0 is the refresh pass: its caches are those of refresh_forward from the embedded tokens
+    rows, rc, _ = orc.refresh_forward(layers, SMALL, embed[ids0], caches, T, l, anchors, lay.extra_rows[0], cos, sin)
+    assert np.array_equal(c_all[0][0], rc[0][0]) and np.array_equal(c_all[1][1], rc[1][1])
+    # decode steps touch only the block's cache rows
+    keep = np.setdiff1d(np.arange(T), block)
+    assert np.array_equal(c_one[1][0][keep], rc[1][0][keep]) and not np.array_equal(c_one[1][0][block], rc[1][0][block])
+    # max_steps cuts the schedule short
+    assert run(1.5, 3)[0] == 3
+
+
 def test_comparators():
     ok, worst = orc.rel_err_gate(np.array([1.0, 2.0]), np.array([1.0, 2.0]))
     assert ok and worst == 0
