@@ -528,8 +528,10 @@ def run_sweep(args):
     points, launches, tot_tokens, tot_s = [], 0, 0.0, 0.0
     flags = ab.F_SCORE | ab.F_SELECT
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for L in Ls:
-        for B in Bs:
+    # light points first: after a point that draws the full power budget the SM clock stays low for a while,
+    # which would be charged to the small points that follow it
+    for B in Bs:
+        for L in Ls:
             T = L + 96
             row = shape.n_kv_heads * shape.head_dim
             cache_bytes = 2 * B * T * row * 2

@@ -49,6 +49,8 @@ constexpr uint32_t GRID_WAIT_LIMIT = 1u << 21;
 struct TcPlan {
     int m_tiles, n_tiles, KB, tiles, U, ctas, smax;
     int prefetch;         // K blocks past the ring whose weight tiles are requested into L2 before the dependency wait
+    int pair_u;           // two-SM kernel, stream-K mode: (pair tile, K block) iterations per cluster (0: whole tiles)
+    int m_pairs;          // 256-row tile rows of the two-SM kernel
     int units;            // 128-row B halves over all segments (non-SwiGLU) or ffn/128 (SwiGLU)
 };
 
@@ -181,11 +183,24 @@ __device__ __forceinline__ void qkv_unit(const GemmArgs& g, int u128, int& seg, 
 // two slots: slot 0 for its first segment, slot 1 for its last (segments in between are whole tiles
 // and never need one).  Tile t's contributors are CTAs c_first..c_last; CTA c's part of it is that
 // CTA's first segment exactly when the CTA starts inside the tile.
+// In the two-SM kernel's stream-K mode the contributors are clusters, the tile that is cut is the
+// 256-row pair tile tp = nt * m_pairs + mt / 2, and each CTA of a cluster (rank = mt & 1) has its own
+// pair of slots: slot = (cluster * 2 + segment) * 2 + rank.
 __device__ __forceinline__ void tile_cover(const TcPlan& p, int t, int& c_first, int& c_last) {
-    c_first = (int)(((int64_t)t * p.KB) / p.U);
-    c_last = (int)(((int64_t)(t + 1) * p.KB - 1) / p.U);
+    if (p.pair_u) {
+        const int nt = t / p.m_tiles, mt = t - nt * p.m_tiles;
+        t = nt * p.m_pairs + (mt >> 1);
+    }
+    const int U = p.pair_u ? p.pair_u : p.U;
+    c_first = (int)(((int64_t)t * p.KB) / U);
+    c_last = (int)(((int64_t)(t + 1) * p.KB - 1) / U);
 }
 __device__ __forceinline__ int64_t slot_of(const TcPlan& p, int t, int c) {
+    if (p.pair_u) {
+        const int nt = t / p.m_tiles, mt = t - nt * p.m_tiles;
+        const int tp = nt * p.m_pairs + (mt >> 1);
+        return ((int64_t)c * 2 + ((int64_t)c * p.pair_u >= (int64_t)tp * p.KB ? 0 : 1)) * 2 + (mt & 1);
+    }
     return (int64_t)c * 2 + ((int64_t)c * p.U >= (int64_t)t * p.KB ? 0 : 1);
 }
 
@@ -789,13 +804,19 @@ gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __gr
         uint32_t phase = 0;
         bool ok = !*abort_flag;
         const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
-        for (int t = cluster_id; t < tiles && ok; t += clusters) {
+        // work list: whole tiles round-robin (pair_u == 0), or this cluster's contiguous range of
+        // (tile, K block) iterations, tiles in weight-tile-major order (stream-K)
+        const long long it_end = p.pair_u ? min((long long)(cluster_id + 1) * p.pair_u, (long long)tiles * p.KB) : 0;
+        long long it = p.pair_u ? (long long)cluster_id * p.pair_u : 0;
+        for (int t = p.pair_u ? (int)(it / p.KB) : cluster_id; ok && (p.pair_u ? it < it_end : t < tiles);) {
             int nt, mp;
-            tile_coords(t, m_pairs, p.n_tiles, nt, mp);
+            if (p.pair_u) { nt = t / m_pairs; mp = t - nt * m_pairs; } else tile_coords(t, m_pairs, p.n_tiles, nt, mp);
+            const int kb0 = p.pair_u ? (int)(it - (long long)t * p.KB) : 0;
+            const int kb1 = p.pair_u ? (int)min((long long)p.KB, (long long)(kb0 + (it_end - it))) : p.KB;
             int brow;
             const int bs = half_source(g, p, nt, (int)rank, brow);
             const int arow = (mp * 2 + (int)rank) * TC_BM;
-            for (int kb = 0; kb < p.KB; ++kb) {
+            for (int kb = kb0; kb < kb1; ++kb) {
                 if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag))) break;
                 const uint32_t sA = base + stage * TC2_STAGE_BYTES, sB = sA + TC_A_BYTES;
                 const uint32_t lead_full = mapa_u32(full_bar(stage), 0);
@@ -806,6 +827,7 @@ gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __gr
                 ++issued;
                 if (++stage == TC2_STAGES) { stage = 0; phase ^= 1; }
             }
+            if (p.pair_u) { it += kb1 - kb0; ++t; } else t += clusters;
         }
         // wait until the MMAs have consumed everything this CTA loaded, so that no signal from the
         // leader can arrive after this CTA has left
@@ -819,24 +841,29 @@ gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __gr
         uint32_t phase = 0, acc_phase = 0;
         bool ok = !*abort_flag;
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-        for (int t = cluster_id; t < tiles && ok; t += clusters) {
+        const long long it_end = p.pair_u ? min((long long)(cluster_id + 1) * p.pair_u, (long long)tiles * p.KB) : 0;
+        long long it = p.pair_u ? (long long)cluster_id * p.pair_u : 0;
+        for (int t = p.pair_u ? (int)(it / p.KB) : cluster_id; ok && (p.pair_u ? it < it_end : t < tiles);) {
+            const int kb0 = p.pair_u ? (int)(it - (long long)t * p.KB) : 0;
+            const int kb1 = p.pair_u ? (int)min((long long)p.KB, (long long)(kb0 + (it_end - it))) : p.KB;
             if (!(ok = mbar_wait_cluster(tempty_bar(acc), acc_phase ^ 1, abort_flag))) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * TC_BN;
-            for (int kb = 0; kb < p.KB; ++kb) {
+            for (int kb = kb0; kb < kb1; ++kb) {
                 if (!(ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t sA = base + stage * TC2_STAGE_BYTES, sB = sA + TC_A_BYTES;
                 const uint64_t da = smem_desc_sw128(sA), db = smem_desc_sw128(sB);
 #pragma unroll
                 for (int k = 0; k < TC_BK / 16; ++k)
-                    tc2_mma(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    tc2_mma(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
                 tc2_commit_both(empty_bar(stage));
                 if (++stage == TC2_STAGES) { stage = 0; phase ^= 1; }
             }
             if (!ok) break;
             tc2_commit_both(tfull_bar(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            if (p.pair_u) { it += kb1 - kb0; ++t; } else t += clusters;
         }
     } else if (warp >= 2 && warp < 6) {
         // drain: this CTA's 128 rows of the tile, epilogue straight from TMEM
@@ -845,18 +872,40 @@ gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __gr
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = !*abort_flag;
-        for (int t = cluster_id; t < tiles && ok; t += clusters) {
+        const long long it_end = p.pair_u ? min((long long)(cluster_id + 1) * p.pair_u, (long long)tiles * p.KB) : 0;
+        long long it = p.pair_u ? (long long)cluster_id * p.pair_u : 0;
+        const long long it_first = it;
+        const uint64_t pol_p = policy_evict_last();
+        for (int t = p.pair_u ? (int)(it / p.KB) : cluster_id; ok && (p.pair_u ? it < it_end : t < tiles);) {
             int nt, mp;
-            tile_coords(t, m_pairs, p.n_tiles, nt, mp);
+            if (p.pair_u) { nt = t / m_pairs; mp = t - nt * m_pairs; } else tile_coords(t, m_pairs, p.n_tiles, nt, mp);
+            const int kb0 = p.pair_u ? (int)(it - (long long)t * p.KB) : 0;
+            const int kb1 = p.pair_u ? (int)min((long long)p.KB, (long long)(kb0 + (it_end - it))) : p.KB;
             const int grow = (mp * 2 + (int)rank) * TC_BM + row;
             if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag))) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + acc * TC_BN + ((uint32_t)(q * 32) << 16);
-            direct_epilogue(g, p, taddr, nt, grow, grow < g.M, 8);
+            if (kb0 == 0 && kb1 == p.KB) {
+                direct_epilogue(g, p, taddr, nt, grow, grow < g.M, 8);
+            } else {
+                // a tile whose K range is cut between clusters: this CTA's 128 rows to its fp32 partial slot
+                float4* dst = reinterpret_cast<float4*>(g.partial) +
+                              (((int64_t)cluster_id * 2 + (it == it_first ? 0 : 1)) * 2 + rank) * (TC_SLOT_FLOATS / 4);
+                for (int c = 0; c < 8; ++c) {
+                    float v[32];
+                    tc_ld32(taddr + c * 32, v);
+                    if (grow < g.M) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            st_hint_f4(&dst[(c * 8 + i) * TC_BM + row], make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]), pol_p);
+                    }
+                }
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_u32(tempty_bar(acc), 0));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            if (p.pair_u) { it += kb1 - kb0; ++t; } else t += clusters;
         }
     }
     tc_fence_before();
@@ -1092,8 +1141,10 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
         cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC2_SMEM);
         attr = true;
     }
-    // Many rows: two SMs per 256 x 256 tile (no K split, every tile whole).
-    static const int pair_min_tiles = [] { const char* e = getenv("ACACHE_GEMM_PAIR_MIN_MTILES"); return e ? atoi(e) : 4; }();
+    // Two or more row tiles: two SMs per 256 x 256 tile.  With many tiles per cluster every tile is whole
+    // and the clusters walk them round-robin; with few, the (tile, K block) iterations are cut into equal
+    // contiguous ranges, one per cluster (stream-K), and the cut tiles go through the finish kernel.
+    static const int pair_min_tiles = [] { const char* e = getenv("ACACHE_GEMM_PAIR_MIN_MTILES"); return e ? atoi(e) : 2; }();
     if (p.m_tiles >= pair_min_tiles && g.epilogue != kEpiLogits && (p.units % 2 == 0 || swiglu) && sm_count() >= 2) {
         const int m_pairs = (p.m_tiles + 1) / 2;
         const int tiles = m_pairs * p.n_tiles;
@@ -1120,10 +1171,38 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
             max_clusters = n;
         }
         if (max_clusters < 1) goto single_cta;
-        const int clusters = std::min(std::min(max_clusters, sm_count() / 2), tiles);
+        TcPlan pp = p;
+        pp.m_pairs = m_pairs;
+        int clusters = std::min(std::min(max_clusters, sm_count() / 2), tiles);
+        // measured: cutting tiles pays (partial tiles + finish kernel included) up to about two thirds of a wave
+        static const int stream_k_pct = [] { const char* e = getenv("ACACHE_GEMM_PAIR_STREAMK_PCT"); return e ? atoi(e) : 66; }();
+        SplitTiles split{};
+        if (tiles * 100 <= stream_k_pct * std::min(max_clusters, sm_count() / 2)) {
+            const int64_t total = (int64_t)tiles * p.KB;
+            clusters = (int)std::min<int64_t>(std::min(max_clusters, sm_count() / 2), total);
+            pp.pair_u = (int)((total + clusters - 1) / clusters);
+            clusters = (int)((total + pp.pair_u - 1) / pp.pair_u);
+            // pair tiles cut by a boundary between two clusters: both of their 128-row tiles go to the finish
+            int last = -1;
+            for (int c = 1; c < clusters; ++c) {
+                const int64_t cut = (int64_t)c * pp.pair_u;
+                if (cut % p.KB == 0) continue;
+                const int tp = (int)(cut / p.KB);
+                if (tp == last) continue;
+                last = tp;
+                const int nt = tp / m_pairs, mp = tp - nt * m_pairs;
+                for (int r = 0; r < 2; ++r)
+                    if (mp * 2 + r < p.m_tiles && split.n < 160) split.tile[split.n++] = nt * p.m_tiles + mp * 2 + r;
+            }
+            if (split.n >= 159) { pp.pair_u = 0; split.n = 0; clusters = std::min(std::min(max_clusters, sm_count() / 2), tiles); }
+        }
         cfg.gridDim = dim3(clusters * 2);
-        if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, g, p, clusters, *mA, *mB[0], *mB[1], *mB[2]) != cudaSuccess) return -1;
-        return 1;
+        if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, g, pp, clusters, *mA, *mB[0], *mB[1], *mB[2]) != cudaSuccess) return -1;
+        if (split.n == 0) return 1;
+        const int per_tile = finish_items_per_tile(g.epilogue) * TC_BM;
+        if (launch_pdl(gemm_finish_kernel, dim3((per_tile + 255) / 256, split.n), dim3(256), 0, stream, g, pp, split) != cudaSuccess)
+            return -1;
+        return 2;
     }
 single_cta:
     // a plain launch: a cooperative one measured ~2.5 us slower and cannot overlap the previous
