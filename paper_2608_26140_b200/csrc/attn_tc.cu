@@ -4,7 +4,7 @@
 // rows past the request's row count read as zero).
 //
 //   S = Q K^T    tcgen05.mma 128 x 128 x 16, both operands K-major, into one of two TMEM buffers
-//   softmax      eight warps, two threads per query row (64 keys each): scaled max, exp2, running
+//   softmax      sixteen warps, four threads per query row (32 keys each): scaled max, exp2, running
 //                denominator; P is written as bf16 into a 128-byte-swizzled shared tile
 //   O += P V     tcgen05.mma 128 x 128 x 16, A = P (K-major over keys), B = V read in place as an
 //                MN-major operand (token-major V rows are contiguous along the head dimension)
@@ -24,10 +24,11 @@
 
 namespace acache {
 
-constexpr int AT_THREADS = 320;                  // warp 0: TMA, warp 1: MMA, warps 2-9: softmax (two threads per row)
+constexpr int AT_THREADS = 608;                  // warp 0: TMA, warp 1: S MMAs, warps 2-17: softmax (four threads per row), warp 18: PV MMAs
 constexpr int AT_TILE = 128 * 128 * 2;           // 32 KB: a [128 x 128] bf16 tile as two 64-column panels
 constexpr int AT_PANEL = 128 * 64 * 2;           // 16 KB
-constexpr int AT_SMEM = 7 * AT_TILE + 1024 + 256;   // Q, K x2, V x2, P x2
+constexpr int AT_SLACK = 256;                    // the dynamic window starts 1024-aligned in practice; checked at run time
+constexpr int AT_SMEM = 7 * AT_TILE + AT_SLACK + 256;   // Q, K x2, V x2, P x2
 constexpr float kRescaleGap = 8.f;               // log2 units
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar,
@@ -89,9 +90,13 @@ __global__ void __launch_bounds__(AT_THREADS, 1)
 attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                     const __grid_constant__ CUtensorMap mapV) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ uint16_t row_max[2][2][128];  // [tile parity][key half][row]: upper halves of fp32, rounded up
+    __shared__ uint16_t row_max[2][4][128];  // [tile parity][key quarter][row]: upper halves of fp32, rounded up
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    if (base - smem_u32(smem_raw) > (uint32_t)AT_SLACK) {      // the tiles would not fit: report, touch nothing
+        if (threadIdx.x == 0) atomicOr(a.status, kFlagWaitExpired);
+        return;
+    }
     const uint32_t sQ = base, sK0 = base + AT_TILE, sV0 = base + 3 * AT_TILE, sP0 = base + 5 * AT_TILE;
     const uint32_t bars = base + 7 * AT_TILE;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + 7 * AT_TILE + 192);
@@ -106,8 +111,8 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(11), 8); mbar_init(bar(12), 8);      // s_empty: the eight softmax warps
-        mbar_init(bar(13), 8); mbar_init(bar(14), 8);      // p_full
+        mbar_init(bar(11), 16); mbar_init(bar(12), 16);    // s_empty: the sixteen softmax warps
+        mbar_init(bar(13), 16); mbar_init(bar(14), 16);    // p_full
         mbar_init(bar(15), 1); mbar_init(bar(16), 1);      // p_empty
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -145,12 +150,20 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             tma_load_3d(sV0 + s * AT_TILE + AT_PANEL, &mapV, kvh * 128 + 64, j * 128, b, bar(5 + s), pol_kv);
         }
     } else if (warp == 1 && lane == 0) {
-        // ---------------- MMA issuer ----------------
-        // S = Q K^T: M 128, N 128, both K-major.  O += P V: M 128, N 128, A K-major, B MN-major.
+        // ---------------- MMA issuer 1: S = Q K^T (M 128, N 128, both operands K-major) ----------------
+        // The two products are issued by two threads of different warps: one thread doing both spends
+        // more time in its four barrier waits and sixteen issues per tile than the tensor pipe needs
+        // for the work.  Every tcgen05.commit tracks the issuing thread's own MMAs, and the cross
+        // dependencies (P of tile j after S of tile j, S buffer reuse, O in tile order) all go through
+        // mbarriers, so no ordering between the two threads is assumed.
         const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        const uint32_t idesc_o = idesc_s | (1u << 16);
-        auto issue_s = [&](int j) {
+        bool ok = mbar_wait(bar(0), 0, abort_flag);
+        for (int j = 0; j < n_tiles && ok; ++j) {
             const int s = j & 1;
+            const uint32_t par = (j >> 1) & 1;
+            if (!(ok = mbar_wait(bar(1 + s), par, abort_flag))) break;          // K of tile j landed
+            if (!(ok = mbar_wait(bar(11 + s), par ^ 1, abort_flag))) break;     // its S buffer has been read (tile j - 2)
+            tc_fence_after();
             const uint32_t k = sK0 + s * AT_TILE;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
@@ -160,21 +173,12 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             }
             tc_commit(bar(9 + s));     // s_full
             tc_commit(bar(3 + s));     // k_empty
-        };
-        bool ok = mbar_wait(bar(0), 0, abort_flag) && mbar_wait(bar(1), 0, abort_flag);
-        if (ok) {
-            tc_fence_after();
-            issue_s(0);
         }
+    } else if (warp == AT_THREADS / 32 - 1 && lane == 0) {
+        // ---------------- MMA issuer 2: O += P V (A = P K-major, B = V MN-major) ----------------
+        const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
-            if (j + 1 < n_tiles) {
-                const int s = (j + 1) & 1;
-                const uint32_t par = ((j + 1) >> 1) & 1;
-                if (!(ok = mbar_wait(bar(1 + s), par, abort_flag))) break;          // K of tile j+1 landed
-                if (!(ok = mbar_wait(bar(11 + s), par ^ 1, abort_flag))) break;     // its S buffer has been read
-                tc_fence_after();
-                issue_s(j + 1);
-            }
             const int s = j & 1;
             if (!(ok = mbar_wait(bar(13 + s), (j >> 1) & 1, abort_flag))) break;    // P of tile j written, O rescaled
             if (!(ok = mbar_wait(bar(5 + s), (j >> 1) & 1, abort_flag))) break;     // V of tile j landed
@@ -189,58 +193,55 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             tc_commit(bar(15 + s));    // p_empty: this P buffer is free, O holds tiles 0..j
             tc_commit(bar(7 + s));     // v_empty
         }
-    } else if (warp >= 2) {
-        // ---------------- softmax: two threads per query row ----------------
-        // Warps 2-5 take keys 0-63 of every tile (and columns 0-63 of O), warps 6-9 the other half; the
-        // two threads of a row agree on the row maximum through shared memory once per tile.  The two
-        // warps of a row quarter meet at a named barrier every tile, so they only ever leave the loop together: a wait
-        // that ran out sets the abort flag, the thread skips its work, and everyone breaks after the
-        // next barrier.
-        const int wg = (warp - 2) >> 2;
+    } else if (warp >= 2 && warp < 18) {
+        // ---------------- softmax: four threads per query row ----------------
+        // Warp 2 + 4 c + q' (q = warp & 3 is its TMEM lane quarter) takes keys [32 c, 32 c + 32) of every
+        // tile for the 32 rows of quarter q, and columns [32 c, 32 c + 32) of O.  Sixteen warps (four per
+        // scheduler) keep the exponential, conversion and TMEM-load latencies of one warp hidden behind
+        // the others.  The four threads of a row agree on the row maximum through shared memory once per
+        // tile.  The four warps of a row quarter meet at a named barrier every tile, so they only ever
+        // leave the loop together: a wait that ran out sets the abort flag, the thread skips its work,
+        // and everyone breaks after the next barrier.
+        const int c4 = (warp - 2) >> 2;
         const int q = warp & 3;
         const int row = q * 32 + lane;
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-        const uint32_t col_off = (uint32_t)(wg * 64);
+        const uint32_t col_off = (uint32_t)(c4 * 32);
         float m_use = -INFINITY, l = 0.f;
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j & 1;
-            const int valid = a.ctx_len - j * 128 - wg * 64;       // keys of this thread's half that exist
-            float sv[2][32];
+            const int valid = a.ctx_len - j * 128 - c4 * 32;       // keys of this thread's quarter that exist
+            float sv[32];
             float mt = -INFINITY;
             if (ok && (ok = mbar_wait(bar(9 + s), (j >> 1) & 1, abort_flag))) {
                 tc_fence_after();
-                const uint32_t tS = tS0 + s * 128 + col_off + lane_off;
-                // this thread's half row of S into registers, then the S buffer is free for tile j + 2
-                tc_ld32(tS, sv[0]);
-                tc_ld32(tS + 32, sv[1]);
+                // this thread's quarter row of S into registers, then the S buffer is free for tile j + 2
+                tc_ld32(tS0 + s * 128 + col_off + lane_off, sv);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(11 + s));   // s_empty
                 float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                if (valid >= 64) {
+                if (valid >= 32) {
 #pragma unroll
-                    for (int c = 0; c < 2; ++c)
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], sv[c][i]);
+                    for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], sv[i]);
                 } else {
 #pragma unroll
-                    for (int c = 0; c < 2; ++c)
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (c * 32 + i < valid) m4[i & 3] = fmaxf(m4[i & 3], sv[c][i]);
+                    for (int i = 0; i < 32; ++i)
+                        if (i < valid) m4[i & 3] = fmaxf(m4[i & 3], sv[i]);
                 }
                 mt = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * a.scale_log2e;
             }
-            // the two threads of a row must use the same number: both take the larger of the two
-            // half-row maxima rounded up to 16 significant bits (an upper bound is all the exponent needs)
+            // the four threads of a row must use the same number: all take the largest of the four
+            // quarter-row maxima rounded up to 16 significant bits (an upper bound is all the exponent needs)
             uint32_t mb = __float_as_uint(mt);
             if ((mb & 0xFFFFu) && !(mb >> 31)) mb += 0x10000u;
             mb >>= 16;
-            row_max[s][wg][row] = (uint16_t)mb;
-            asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");      // the two warps that share these 32 rows
+            row_max[s][c4][row] = (uint16_t)mb;
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");     // the four warps that share these 32 rows
             if (*abort_flag) { ok = false; break; }
-            mt = fmaxf(__uint_as_float(mb << 16), __uint_as_float((uint32_t)row_max[s][wg ^ 1][row] << 16));
+            mt = fmaxf(fmaxf(__uint_as_float((uint32_t)row_max[s][0][row] << 16), __uint_as_float((uint32_t)row_max[s][1][row] << 16)),
+                       fmaxf(__uint_as_float((uint32_t)row_max[s][2][row] << 16), __uint_as_float((uint32_t)row_max[s][3][row] << 16)));
             bool raise = false;
             if (j == 0) {
                 m_use = mt;
@@ -252,13 +253,11 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
                 if ((ok = mbar_wait(bar(15 + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag))) {
                     tc_fence_after();
                     const float f = raise ? fast_exp2(m_use - mt) : 1.f;
-                    for (int c = 0; c < 2; ++c) {
-                        float v[32];
-                        tc_ld32(tO + lane_off + col_off + c * 32, v);
+                    float v[32];
+                    tc_ld32(tO + lane_off + col_off, v);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] *= f;
-                        tc_st32(tO + lane_off + col_off + c * 32, v);
-                    }
+                    for (int i = 0; i < 32; ++i) v[i] *= f;
+                    tc_st32(tO + lane_off + col_off, v);
                     tc_wait_st();
                     l *= f;
                     if (raise) m_use = mt;
@@ -267,35 +266,33 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             // this P buffer was last read by the P V of tile j - 2
             if (ok && j >= 2) ok = mbar_wait(bar(15 + s), ((j - 2) >> 1) & 1, abort_flag);
             if (!ok) continue;
-            const uint32_t sP = sP0 + s * AT_TILE + wg * AT_PANEL + row * 128;
+            // 32 keys = four 16-byte chunks of the row, chunks 4 c4 .. 4 c4 + 3 of the 16 in a 128-key tile
+            const uint32_t sP = sP0 + s * AT_TILE + (c4 >> 1) * AT_PANEL + row * 128;
             float l4[4] = {0.f, 0.f, 0.f, 0.f};
+            if (valid >= 32) {
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                if (valid >= 64) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float x = fmaf(sv[c][i], a.scale_log2e, -m_use);
-                        const float p = (i & 3) == 3 ? poly_exp2(x) : fast_exp2(x);
-                        l4[i & 3] += p;
-                        sv[c][i] = p;
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float p = c * 32 + i < valid ? fast_exp2(fmaf(sv[c][i], a.scale_log2e, -m_use)) : 0.f;
-                        l4[i & 3] += p;
-                        sv[c][i] = p;
-                    }
+                for (int i = 0; i < 32; ++i) {
+                    const float x = fmaf(sv[i], a.scale_log2e, -m_use);
+                    const float p = (i & 3) == 3 ? poly_exp2(x) : fast_exp2(x);
+                    l4[i & 3] += p;
+                    sv[i] = p;
                 }
+            } else {
 #pragma unroll
-                for (int k8 = 0; k8 < 4; ++k8) {
-                    const int chunk = c * 4 + k8;                 // 16-byte chunk of this half row: 8 keys
-                    const uint32_t addr = sP + ((chunk ^ (row & 7)) << 4);
-                    const float* pv = sv[c] + k8 * 8;
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(pv[0], pv[1])),
-                                 "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])), "r"(pack_bf16(pv[6], pv[7]))
-                                 : "memory");
+                for (int i = 0; i < 32; ++i) {
+                    const float p = i < valid ? fast_exp2(fmaf(sv[i], a.scale_log2e, -m_use)) : 0.f;
+                    l4[i & 3] += p;
+                    sv[i] = p;
                 }
+            }
+#pragma unroll
+            for (int k8 = 0; k8 < 4; ++k8) {
+                const int chunk = (c4 & 1) * 4 + k8;              // chunk inside the 64-key panel
+                const uint32_t addr = sP + ((chunk ^ (row & 7)) << 4);
+                const float* pv = sv + k8 * 8;
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(pv[0], pv[1])),
+                             "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])), "r"(pack_bf16(pv[6], pv[7]))
+                             : "memory");
             }
             l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
             tc_fence_before();
@@ -303,27 +300,25 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(13 + s));   // p_full
         }
-        // epilogue: O / l once the last P V has completed; the denominators of the two halves add up
+        // epilogue: O / l once the last P V has completed; the denominators of the four quarters add up
         if (ok && n_tiles > 0) ok = mbar_wait(bar(15 + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, abort_flag);
         float* row_sum = reinterpret_cast<float*>(base_ptr + 5 * AT_TILE);     // the P buffers are idle now
-        row_sum[wg * 128 + row] = l;
-        asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");
+        row_sum[c4 * 128 + row] = l;
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
         if (ok && !*abort_flag) {
             tc_fence_after();
             const int grow = qt * 128 + row;
-            const float inv = 1.f / (l + row_sum[(wg ^ 1) * 128 + row]);
+            const float inv = 1.f / ((row_sum[row] + row_sum[128 + row]) + (row_sum[256 + row] + row_sum[384 + row]));
             __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o) + (((int64_t)b * a.n + grow) * a.n_heads + h) * 128 + col_off;
-            for (int c = 0; c < 2; ++c) {
-                float v[32];
-                tc_ld32(tO + lane_off + col_off + c * 32, v);
-                if (grow < a.n) {
+            float v[32];
+            tc_ld32(tO + lane_off + col_off, v);
+            if (grow < a.n) {
 #pragma unroll
-                    for (int k8 = 0; k8 < 4; ++k8) {
-                        const float* pv = v + k8 * 8;
-                        *reinterpret_cast<uint4*>(out + c * 32 + k8 * 8) =
-                            make_uint4(pack_bf16(pv[0] * inv, pv[1] * inv), pack_bf16(pv[2] * inv, pv[3] * inv),
-                                       pack_bf16(pv[4] * inv, pv[5] * inv), pack_bf16(pv[6] * inv, pv[7] * inv));
-                    }
+                for (int k8 = 0; k8 < 4; ++k8) {
+                    const float* pv = v + k8 * 8;
+                    *reinterpret_cast<uint4*>(out + k8 * 8) =
+                        make_uint4(pack_bf16(pv[0] * inv, pv[1] * inv), pack_bf16(pv[2] * inv, pv[3] * inv),
+                                   pack_bf16(pv[4] * inv, pv[5] * inv), pack_bf16(pv[6] * inv, pv[7] * inv));
                 }
             }
         }
