@@ -711,6 +711,92 @@ def run_generate(args, e):
         dist.destroy_process_group()
 
 
+def run_shared(args):
+    """Shared affix storage (Section 4.1) against one working cache per request, one layer of benchmark
+    configuration 3 or 4: the same refresh (scores, selection, R = anchors + all request rows) once through
+    acache_layer_step on B private caches [B, T, Hkv, d], once through acache_score_anchors /
+    acache_select_topk / acache_recompute_anchors on ONE cache [T, Hkv, d] (batch_stride 0) with every
+    request's fresh rows in its private k_new / v_new [B, K+e, Hkv, d]."""
+    import torch
+    from paper_2608_26140_b200 import binding as ab
+    from paper_2608_26140_b200 import build as abuild
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    abuild.build()
+    cfg = args.config
+    shape = wl.LLADA_8B if cfg == 3 else wl.DREAM_7B
+    lay = wl.config_layout(cfg, "all", n_masked=32, batch=args.batch)
+    B, T, L, P = lay.batch, lay.ctx_len, lay.affix_len, lay.n_extra
+    K = ab.k_from_ratio(L, RATIO)
+    n = K + P
+    w = wl.layer_weights(shape, cfg, 0)
+    wd = {k: (ab.to_device_bf16(v, dev) if v is not None else None) for k, v in w.items()}
+    lw = ab.Context.weights(wd)
+    ck, cv = wl.random_kv_cache(shape, lay, wl.SEED_BASE + 4096 * cfg + 30)
+    dk, dv = ab.to_device_bf16(ck, dev), ab.to_device_bf16(cv, dev)
+    sk, sv = dk[0:1].clone(), dv[0:1].clone()                       # the shared copy
+    gen = torch.Generator(device=dev); gen.manual_seed(wl.SEED_BASE + 4096 * cfg + 31)
+    x = torch.randn((B, T, shape.hidden), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    x[1:, lay.affix_start:lay.affix_start + L] = x[0:1, lay.affix_start:lay.affix_start + L]
+    cos_h, sin_h = wl.rope_table(T, shape.head_dim, shape.rope_theta)
+    cos, sin = torch.from_numpy(cos_h).to(dev), torch.from_numpy(sin_h).to(dev)
+    masked = torch.from_numpy(lay.masked_pos.copy()).to(dev)
+    extra = torch.from_numpy(lay.extra_rows.copy()).to(dev)
+    req = ab.Context.request(B, T, lay.affix_start, L, masked, extra, cos, sin)
+    ctx = ab.Context.for_shape(shape, B, T, L, n, lay.n_masked, dev)
+    scores = torch.zeros((B, L), dtype=torch.float32, device=dev)
+    anchors = torch.zeros((B, K), dtype=torch.int32, device=dev)
+    y = torch.zeros((B, n, shape.hidden), dtype=torch.bfloat16, device=dev)
+    k_new = torch.zeros((B, n, shape.n_kv_heads, shape.head_dim), dtype=torch.bfloat16, device=dev)
+    v_new = torch.zeros_like(k_new)
+    q_mask = torch.randn((B, lay.n_masked, shape.n_heads, shape.head_dim), generator=gen, device=dev,
+                         dtype=torch.float32).mul_(0.02 * float(np.sqrt(shape.hidden))).to(torch.bfloat16)
+    kv_priv = ab.Context.kv(dk, dv)
+    kv_shared = ab.KV(sk.data_ptr(), sv.data_ptr(), 0, T)
+
+    def private_step():
+        ctx.layer_step(lw, req, kv_priv, x, 0, RATIO, ab.F_SCORE | ab.F_SELECT, scores, anchors, y)
+
+    def shared_step():
+        ctx.score_anchors(req, q_mask, kv_shared, scores)
+        ctx.select_topk(scores, B, L, K, anchors)
+        ctx.recompute_anchors(lw, req, kv_shared, x, 0, anchors, K, k_new, v_new, y)
+
+    res = {}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for name, fn in (("private", private_step), ("shared", shared_step)):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        res[name] = e0.elapsed_time(e1) / args.steps
+        ctx.stage_timing(True)
+        fn()
+        res[name + "_stage_us"] = {k_: round(v * 1e3, 1) for k_, v in ctx.read_stage_times().items() if v}
+        ctx.stage_timing(False)
+    assert ctx.poll_status() == 0
+    row = shape.n_kv_heads * shape.head_dim * 2 * 2            # K and V bytes of one position
+    kv_private, kv_shared_b = B * T * row, T * row + B * n * row
+    print(json.dumps({
+        "metric": METRIC, "value": B * K / (res["shared"] * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": 3,
+        "ms_per_step": res["shared"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"cfg{cfg} one layer, shared affix storage: {shape.name}, batch {B} sharing a {L}-token affix, "
+                               f"K={K} anchors + {P} request rows per request ({B * n} rows)", "benchmark_config": cfg},
+        "shared_storage": {"ms_per_layer": res["shared"], "kv_bytes_per_layer": kv_shared_b, "stage_us": res["shared_stage_us"],
+                           "note": "the masked-row queries are given (acache_score_anchors); the split calls do not write the cache"},
+        "private_caches": {"ms_per_layer": res["private"], "kv_bytes_per_layer": kv_private, "stage_us": res["private_stage_us"],
+                           "note": "acache_layer_step including the masked-row query projection"},
+        "kv_bytes_ratio": kv_shared_b / kv_private,
+    }))
+
+
 def cpu_baseline(case, shape, lay):
     """The oracle as it stands, timed on this machine's host cores on one step of the workload."""
     from oracle import acache_oracle as orc
@@ -745,6 +831,8 @@ def main():
     ap.add_argument("--instances", type=int, default=4, help="weight/cache instances rotated between steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=32, help="layers of the --config 3 denoising step")
+    ap.add_argument("--shared", action="store_true",
+                    help="--config 3 or 4: one layer with shared affix storage (batch_stride 0) against private caches")
     ap.add_argument("--generate", action="store_true",
                     help="--config 3: decode one whole 32-token block per request (refresh + decode passes)")
     ap.add_argument("--sweep-affix", default=None, help="--config 5: comma-separated affix lengths (default 512,2048,8192)")
@@ -753,6 +841,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.shared and args.config in (3, 4):
+        run_shared(args)
     elif args.config == 3:
         run_denoise(args)
     elif args.config == 5:

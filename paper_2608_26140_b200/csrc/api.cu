@@ -22,7 +22,7 @@ struct acache_ctx {
     // workspace offsets (bytes)
     size_t o_status, o_row_pos, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
     size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
-    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar, o_mcidx, o_lstats, o_lxn;
+    size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar, o_mcidx, o_lstats, o_lxn, o_keymask;
     std::string err;
     uint64_t launches = 0;
     // optional per-stage timing (acache_stage_timing)
@@ -190,6 +190,13 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
         launch_build_slot_map(slot, r->ctx_len, row_pos, rows, r->batch, st);
         c->launches += 1;
         at.k_new = k_new; at.v_new = v_new; at.slot = slot;
+        // key masks of the same map, for the kernel that reads cache and fresh rows as two sources
+        at.excl_words = (r->ctx_len + 31) / 32; at.keep_words = (rows + 31) / 32;
+        uint32_t* km = wsp<uint32_t>(c, c->o_keymask);
+        at.pos_excl = km; at.row_keep = km + (size_t)r->batch * at.excl_words;
+        launch_key_masks(slot, r->ctx_len, row_pos, rows, r->batch, km, at.excl_words, km + (size_t)r->batch * at.excl_words,
+                         at.keep_words, st);
+        c->launches += 1;
     }
     at.batch = r->batch; at.n = rows; at.ctx_len = r->ctx_len;
     at.n_heads = d.n_heads; at.n_kv_heads = d.n_kv_heads; at.head_dim = d.head_dim;
@@ -268,6 +275,7 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
     c->o_stats = take(cur, (size_t)d.max_batch * d.n_heads * score_num_splits(d.max_ctx) * d.max_masked * 8);
     c->o_partial = take(cur, (size_t)d.max_batch * d.n_heads * d.max_affix * 4);
     c->o_slot = take(cur, (size_t)d.max_batch * d.max_ctx * 4);
+    c->o_keymask = take(cur, (size_t)d.max_batch * ((d.max_ctx + 31) / 32 + (d.max_rows + 31) / 32 + 2) * 4);
     c->o_xstage = take(cur, (size_t)d.max_batch * d.max_ctx * d.hidden * 2);
     c->o_ystage = take(cur, nr * d.hidden * 2);
     c->o_sstage = take(cur, (size_t)d.max_batch * d.max_affix * 4);

@@ -84,11 +84,18 @@ struct AttnTcArgs {
     int n, ctx_len, n_heads, n_kv_heads;
     float scale_log2e;
     uint32_t* status;
+    // two key sources (shared storage + private rows, Section 4.1): after the cache's tiles come the tiles of
+    // the fresh rows [B, n, Hkv, d]; pos_excl masks the cache positions those rows serve, row_keep the fresh
+    // rows that do not serve their position (duplicates).  n_fresh_tiles = 0: the cache alone.
+    int n_fresh_tiles, excl_words, keep_words, cache_shared;
+    const uint32_t* pos_excl;
+    const uint32_t* row_keep;
 };
 
 __global__ void __launch_bounds__(AT_THREADS, 1)
 attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-                    const __grid_constant__ CUtensorMap mapV) {
+                    const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapKn,
+                    const __grid_constant__ CUtensorMap mapVn) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ uint16_t row_max[2][4][128];  // [tile parity][key quarter][row]: upper halves of fp32, rounded up
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -107,7 +114,9 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / (a.n_heads / a.n_kv_heads);
-    const int n_tiles = (a.ctx_len + 127) / 128;
+    const int n_cache_tiles = (a.ctx_len + 127) / 128;
+    const int n_tiles = n_cache_tiles + a.n_fresh_tiles;
+    const int kb = a.cache_shared ? 0 : b;          // one cache for the whole batch, or one per request
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
@@ -141,13 +150,17 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             const int s = j & 1;
             const uint32_t par = ((j >> 1) & 1) ^ 1;
             if (!(ok = mbar_wait(bar(3 + s), par, abort_flag))) break;
+            const bool fresh = j >= n_cache_tiles;
+            const CUtensorMap* mk = fresh ? &mapKn : &mapK;
+            const CUtensorMap* mv = fresh ? &mapVn : &mapV;
+            const int r0 = (fresh ? j - n_cache_tiles : j) * 128, bz = fresh ? b : kb;
             mbar_expect_tx(bar(1 + s), AT_TILE);
-            tma_load_3d(sK0 + s * AT_TILE, &mapK, kvh * 128, j * 128, b, bar(1 + s), pol_kv);
-            tma_load_3d(sK0 + s * AT_TILE + AT_PANEL, &mapK, kvh * 128 + 64, j * 128, b, bar(1 + s), pol_kv);
+            tma_load_3d(sK0 + s * AT_TILE, mk, kvh * 128, r0, bz, bar(1 + s), pol_kv);
+            tma_load_3d(sK0 + s * AT_TILE + AT_PANEL, mk, kvh * 128 + 64, r0, bz, bar(1 + s), pol_kv);
             if (!(ok = mbar_wait(bar(7 + s), par, abort_flag))) break;
             mbar_expect_tx(bar(5 + s), AT_TILE);
-            tma_load_3d(sV0 + s * AT_TILE, &mapV, kvh * 128, j * 128, b, bar(5 + s), pol_kv);
-            tma_load_3d(sV0 + s * AT_TILE + AT_PANEL, &mapV, kvh * 128 + 64, j * 128, b, bar(5 + s), pol_kv);
+            tma_load_3d(sV0 + s * AT_TILE, mv, kvh * 128, r0, bz, bar(5 + s), pol_kv);
+            tma_load_3d(sV0 + s * AT_TILE + AT_PANEL, mv, kvh * 128 + 64, r0, bz, bar(5 + s), pol_kv);
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------- MMA issuer 1: S = Q K^T (M 128, N 128, both operands K-major) ----------------
@@ -211,7 +224,17 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j & 1;
-            const int valid = a.ctx_len - j * 128 - c4 * 32;       // keys of this thread's quarter that exist
+            // which of this thread's 32 keys count: the cache's positions up to the context end, minus those a
+            // fresh row serves; of the fresh rows, those that serve their position
+            uint32_t keep;
+            if (j < n_cache_tiles) {
+                const int valid = a.ctx_len - j * 128 - c4 * 32;
+                keep = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
+                if (a.n_fresh_tiles && j * 4 + c4 < a.excl_words) keep &= ~__ldg(a.pos_excl + (int64_t)b * a.excl_words + j * 4 + c4);
+            } else {
+                const int w = (j - n_cache_tiles) * 4 + c4;
+                keep = w < a.keep_words ? __ldg(a.row_keep + (int64_t)b * a.keep_words + w) : 0u;
+            }
             float sv[32];
             float mt = -INFINITY;
             if (ok && (ok = mbar_wait(bar(9 + s), (j >> 1) & 1, abort_flag))) {
@@ -222,13 +245,13 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(11 + s));   // s_empty
                 float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                if (valid >= 32) {
+                if (keep == 0xffffffffu) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], sv[i]);
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (i < valid) m4[i & 3] = fmaxf(m4[i & 3], sv[i]);
+                        if ((keep >> i) & 1u) m4[i & 3] = fmaxf(m4[i & 3], sv[i]);
                 }
                 mt = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * a.scale_log2e;
             }
@@ -269,7 +292,7 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             // 32 keys = four 16-byte chunks of the row, chunks 4 c4 .. 4 c4 + 3 of the 16 in a 128-key tile
             const uint32_t sP = sP0 + s * AT_TILE + (c4 >> 1) * AT_PANEL + row * 128;
             float l4[4] = {0.f, 0.f, 0.f, 0.f};
-            if (valid >= 32) {
+            if (keep == 0xffffffffu) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     const float x = fmaf(sv[i], a.scale_log2e, -m_use);
@@ -280,7 +303,7 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    const float p = i < valid ? fast_exp2(fmaf(sv[i], a.scale_log2e, -m_use)) : 0.f;
+                    const float p = ((keep >> i) & 1u) ? fast_exp2(fmaf(sv[i], a.scale_log2e, -m_use)) : 0.f;
                     l4[i & 3] += p;
                     sv[i] = p;
                 }
@@ -394,18 +417,27 @@ const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int6
 // Returns the number of kernels launched, 0 if this problem is not for the tensor-core kernel
 // (the caller then uses the mma.sync kernel), -1 if a launch failed.
 int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream) {
-    if (a.head_dim != 128 || a.slot || a.batch == 0 || a.n == 0) return 0;
+    if (a.head_dim != 128 || a.batch == 0 || a.n == 0) return 0;
+    // reads through the position -> row map become two key sources when the key masks came with it
+    const bool two_src = a.slot && a.pos_excl && a.row_keep && a.k_new && a.v_new;
+    if (a.slot && !two_src) return 0;
     const int q_tiles = (a.n + 127) / 128;
     // measured at batch 1 with 26-4096 rows over 600-8300 keys: never slower than the key-split mma.sync
     // kernel, even with a single query tile per head (32 CTAs)
     static const int min_ctas = [] { const char* e = getenv("ACACHE_ATTN_TC_MIN_CTAS"); return e ? atoi(e) : 1; }();
     if ((int64_t)q_tiles * a.n_heads * a.batch < min_ctas) return 0;
     if ((a.kv_batch_stride * 2) % 16) return 0;
+    const bool shared = a.kv_batch_stride == 0;           // one cache for the whole batch
+    const int kv_cols = a.n_kv_heads * 128;
     std::lock_guard<std::mutex> lock(g_map3_mutex);
     const CUtensorMap* mq = get_map3(a.q, a.n, a.n_heads * 128, a.batch, (int64_t)a.n * a.n_heads * 128);
-    const CUtensorMap* mk = get_map3(a.cache_k, a.ctx_len, a.n_kv_heads * 128, a.batch, a.kv_batch_stride);
-    const CUtensorMap* mv = get_map3(a.cache_v, a.ctx_len, a.n_kv_heads * 128, a.batch, a.kv_batch_stride);
-    if (!mq || !mk || !mv) return 0;
+    const CUtensorMap* mk = get_map3(a.cache_k, a.ctx_len, kv_cols, shared ? 1 : a.batch,
+                                     shared ? (int64_t)a.ctx_len * kv_cols : a.kv_batch_stride);
+    const CUtensorMap* mv = get_map3(a.cache_v, a.ctx_len, kv_cols, shared ? 1 : a.batch,
+                                     shared ? (int64_t)a.ctx_len * kv_cols : a.kv_batch_stride);
+    const CUtensorMap* mkn = two_src ? get_map3(a.k_new, a.n, kv_cols, a.batch, (int64_t)a.n * kv_cols) : mk;
+    const CUtensorMap* mvn = two_src ? get_map3(a.v_new, a.n, kv_cols, a.batch, (int64_t)a.n * kv_cols) : mv;
+    if (!mq || !mk || !mv || !mkn || !mvn) return 0;
     static bool attr = false;
     if (!attr) {
         cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM);
@@ -415,8 +447,13 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     t.o = a.o; t.n = a.n; t.ctx_len = a.ctx_len; t.n_heads = a.n_heads; t.n_kv_heads = a.n_kv_heads;
     t.scale_log2e = 1.4426950408889634f / sqrtf(128.f);
     t.status = status;
-    if (launch_pdl(attention_tc_kernel, dim3(q_tiles, a.n_heads, a.batch), dim3(AT_THREADS), AT_SMEM, stream, t, *mq, *mk, *mv) !=
-        cudaSuccess)
+    t.cache_shared = shared ? 1 : 0;
+    if (two_src) {
+        t.n_fresh_tiles = q_tiles; t.excl_words = a.excl_words; t.keep_words = a.keep_words;
+        t.pos_excl = a.pos_excl; t.row_keep = a.row_keep;
+    }
+    if (launch_pdl(attention_tc_kernel, dim3(q_tiles, a.n_heads, a.batch), dim3(AT_THREADS), AT_SMEM, stream, t, *mq, *mk, *mv,
+                   *mkn, *mvn) != cudaSuccess)
         return -1;
     return 1;
 }

@@ -26,6 +26,11 @@ void launch_commit_update(int32_t* token_ids, int ctx_len, const int32_t* block_
 void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
                            cudaStream_t stream);
 
+// pos_excl[b, t / 32] bit t % 32 = position t is served by a fresh row; row_keep[b, i / 32] bit i % 32 = fresh
+// row i serves its position (built from the position -> row map, so duplicates resolve the same way).
+void launch_key_masks(const int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
+                      uint32_t* pos_excl, int excl_words, uint32_t* row_keep, int keep_words, cudaStream_t stream);
+
 // ---- score.cu ---------------------------------------------------------------------------
 struct ScoreArgs {
     const void* q_mask;       // bf16 [B, m, H, d]
@@ -135,6 +140,9 @@ struct AttnArgs {
     const void* k_new;        // bf16 [B, n, Hkv, d] or null
     const void* v_new;
     const int32_t* slot;      // [B, ctx_len] or null: >= 0 => read k_new/v_new row slot
+    const uint32_t* pos_excl; // optional key masks of the same map (launch_key_masks): with them the tensor-core
+    const uint32_t* row_keep; //   kernel reads the cache and k_new / v_new as two key sources instead of gathering
+    int excl_words, keep_words;
     int batch, n, ctx_len, n_heads, n_kv_heads, head_dim;
     void* o;                  // bf16 [B, n, H*d]
     float* part_o;            // scratch for key splits: fp32 [B*n*H, n_split, d]

@@ -51,6 +51,42 @@ __global__ void __launch_bounds__(1024) slot_map_kernel(int32_t* __restrict__ sl
     }
 }
 
+// Bit masks over keys for the attention that reads the cache and the fresh rows as two sources
+// (Section 4.1: shared storage + private slots): pos_excl[b] bit t = position t is served by a fresh
+// row (skip it in the cache); row_keep[b] bit i = fresh row i is the one that serves its position
+// (the last one wins if two rows name the same position, as in the position -> row map).
+__global__ void __launch_bounds__(1024) key_mask_kernel(const int32_t* __restrict__ slot, int ctx_len,
+                                                        const int32_t* __restrict__ row_pos, int rows_per_req,
+                                                        uint32_t* __restrict__ pos_excl, int excl_words,
+                                                        uint32_t* __restrict__ row_keep, int keep_words) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    const int32_t* s = slot + (int64_t)b * ctx_len;
+    for (int w = warp; w < excl_words; w += nw) {
+        const int t = w * 32 + lane;
+        const uint32_t bits = __ballot_sync(0xffffffffu, t < ctx_len && s[t] >= 0);
+        if (lane == 0) pos_excl[(int64_t)b * excl_words + w] = bits;
+    }
+    for (int w = warp; w < keep_words; w += nw) {
+        const int i = w * 32 + lane;
+        bool ok = false;
+        if (i < rows_per_req) {
+            const int p = row_pos[(int64_t)b * rows_per_req + i];
+            ok = p >= 0 && p < ctx_len && s[p] == i;
+        }
+        const uint32_t bits = __ballot_sync(0xffffffffu, ok);
+        if (lane == 0) row_keep[(int64_t)b * keep_words + w] = bits;
+    }
+}
+
+void launch_key_masks(const int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
+                      uint32_t* pos_excl, int excl_words, uint32_t* row_keep, int keep_words, cudaStream_t stream) {
+    if (batch == 0) return;
+    launch_pdl(key_mask_kernel, batch, 1024, 0, stream, slot, ctx_len, row_pos, rows_per_req, pos_excl, excl_words, row_keep,
+               keep_words);
+}
+
 // idx[b, i] = k + j where extra_rows[b, j] == masked_pos[b, i]: the compact row that holds a
 // masked position when the layer input is given in compact row order; -1 (and kFlagBadIndex)
 // if the position is not among the extra rows.

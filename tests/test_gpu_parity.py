@@ -395,3 +395,23 @@ def test_shared_affix_cache_with_private_rows():
         dc.ctx.scatter_kv(dc.req, kv, anchors, K, k_new, v_new)
     with pytest.raises(ab.AcacheError):
         dc.ctx.layer_step(dc.lw, dc.req, kv, dc.x, 0, 0.2, 0, None, anchors, y)
+
+
+def test_duplicate_row_is_served_once_in_the_split_calls():
+    """Two fresh rows naming the same position: the position -> row map lets the later one serve it, and the
+    attention that reads cache and fresh rows as two key sources must not count the position twice."""
+    shape, B = MID128, 1
+    lay = wl.make_layout(B, 0, 140, 20, 32, 32, "all")
+    dup = np.concatenate([lay.extra_rows, lay.extra_rows[:, 3:4]], axis=1)          # one position twice
+    lay2 = wl.Layout(lay.batch, lay.ctx_len, lay.affix_start, lay.affix_len, lay.masked_pos, np.ascontiguousarray(dup), "dup")
+    case = wl.make_case(shape, lay2, 0.25, cfg_id=23)
+    dc = DeviceCase(case)
+    K = orc.k_from_ratio(lay.affix_len, 0.25)
+    g = np.random.default_rng(4)
+    anchors = np.sort(g.choice(lay.affix_len, K, replace=False))[None].astype(np.int32)
+    k_new, v_new, y = run_split_calls(dc, dev_i32(anchors), K)
+    torch.cuda.synchronize()
+    assert dc.ctx.poll_status() == 0
+    ref = oracle_step(case, 0, anchor_idx=anchors[0])
+    assert_close_bf16(ab.to_host_bits(y[0]), ref["y"], "y with a duplicated row")
+    assert_close_bf16(ab.to_host_bits(k_new[0]), ref["k_new"], "k_new with a duplicated row")
