@@ -284,6 +284,21 @@ acache_status acache_denoise_step(acache_ctx *ctx, int32_t n_layers, const acach
                                   const void *w_lm, int32_t vocab, float threshold, int32_t *token,
                                   float *confidence, int32_t *commit, acache_stream_t stream);
 
+/* acache_denoise_step over shared affix storage (Section 4.1): the same N-layer refresh of R = A u E and the
+ * same predict-then-commit, but no cache is written.  kvs[n] may have batch_stride 0 (one cache per layer
+ * for the whole batch); layer n's fresh K/V go to the requests' private slots k_new[n] / v_new[n] (HOST
+ * arrays of n_layers DEVICE pointers, each bf16 [B, K+e, Hkv, d]), and layer n's attention reads the
+ * positions of R from them and every other position from kvs[n], exactly as acache_recompute_anchors.
+ * A later step over the same R can leave the shared caches as they are and keep these slots.
+ * Other arguments as acache_denoise_step. */
+acache_status acache_denoise_step_shared(acache_ctx *ctx, int32_t n_layers, const acache_layer_weights *layers,
+                                         const acache_kv *kvs, const acache_request *req, const void *x0,
+                                         const int32_t *anchor_idx, int32_t k, void *const *k_new,
+                                         void *const *v_new, void *y_a, void *y_b, void **y_last,
+                                         const int32_t *block_rows, int32_t n_blk, const void *final_norm_g,
+                                         const void *w_lm, int32_t vocab, float threshold, int32_t *token,
+                                         float *confidence, int32_t *commit, acache_stream_t stream);
+
 /* The one-shot probe and the selection it feeds (Section 3.2): every request's request-specific rows
  * (req->extra_rows = all non-affix positions, which must include the masked ones) go through the
  * n_layers layers with the affix K/V as cached; at every layer the masked rows' queries are scored

@@ -23,7 +23,7 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_k_from_ratio", "acache_select_topk", "acache_recompute_anchors", "acache_scatter_kv",
            "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times",
            "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step", "acache_probe_select",
-           "acache_commit_update", "acache_generate_block"]
+           "acache_commit_update", "acache_generate_block", "acache_denoise_step_shared"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -111,6 +111,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_denoise_step.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request), vp, vp, i32,
                                         vp, vp, C.POINTER(vp), vp, i32, vp, vp, i32, C.c_float, vp, vp, vp, vp]
     lib.acache_denoise_step.restype = C.c_int
+    lib.acache_denoise_step_shared.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request), vp, vp, i32,
+                                               C.POINTER(vp), C.POINTER(vp), vp, vp, C.POINTER(vp), vp, i32, vp, vp, i32,
+                                               C.c_float, vp, vp, vp, vp]
+    lib.acache_denoise_step_shared.restype = C.c_int
     lib.acache_probe_select.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request), vp,
                                         C.c_double, u32, vp, vp, vp, vp, vp]
     lib.acache_probe_select.restype = C.c_int
@@ -280,6 +284,21 @@ class Context:
                                                  _ptr(y_a), _ptr(y_b), C.byref(last), _ptr(block_rows), n_blk,
                                                  _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold), _ptr(token),
                                                  _ptr(confidence), _ptr(commit), _stream()))
+        return last.value
+
+    def denoise_step_shared(self, layers, kvs, req: Request, x0, anchor_idx, k, k_new, v_new, y_a, y_b, block_rows, n_blk,
+                            final_norm_g, w_lm, vocab, threshold, token, confidence, commit) -> int:
+        """k_new, v_new: lists of per-layer tensors [B, K+e, Hkv, d].  Returns the device address of the last output."""
+        n = len(layers)
+        la = (LayerWeights * n)(*layers)
+        ka = (KV * n)(*kvs)
+        kn = (C.c_void_p * n)(*[_ptr(t) for t in k_new])
+        vn = (C.c_void_p * n)(*[_ptr(t) for t in v_new])
+        last = C.c_void_p()
+        self._check(self.lib.acache_denoise_step_shared(self.h, n, la, ka, C.byref(req), _ptr(x0), _ptr(anchor_idx), k, kn, vn,
+                                                        _ptr(y_a), _ptr(y_b), C.byref(last), _ptr(block_rows), n_blk,
+                                                        _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold), _ptr(token),
+                                                        _ptr(confidence), _ptr(commit), _stream()))
         return last.value
 
     def probe_select(self, layers, kvs, req: Request, x0, ratio, flags, y_a, y_b, scores, anchor_idx):

@@ -568,6 +568,32 @@ acache_status acache_denoise_step(acache_ctx* ctx, int32_t n_layers, const acach
                                  confidence, commit, stream);
 }
 
+acache_status acache_denoise_step_shared(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers,
+                                         const acache_kv* kvs, const acache_request* req, const void* x0,
+                                         const int32_t* anchor_idx, int32_t k, void* const* k_new, void* const* v_new,
+                                         void* y_a, void* y_b, void** y_last, const int32_t* block_rows, int32_t n_blk,
+                                         const void* final_norm_g, const void* w_lm, int32_t vocab, float threshold,
+                                         int32_t* token, float* confidence, int32_t* commit, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (n_layers <= 0 || !layers || !kvs || !req || !x0 || !y_a || !y_b || !k_new || !v_new)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL argument or n_layers <= 0");
+    const void* x = x0;
+    void* y = y_a;
+    for (int n = 0; n < n_layers; ++n) {
+        y = (n & 1) ? y_b : y_a;
+        acache_status s = acache_recompute_anchors(ctx, &layers[n], req, &kvs[n], x, n > 0, anchor_idx, k, k_new[n], v_new[n], y,
+                                                   stream);
+        if (s != ACACHE_OK) return s;
+        x = y;
+    }
+    if (y_last) *y_last = y;
+    const int rows = k + req->n_extra;
+    if (n_blk == 0 || req->batch == 0) return ACACHE_OK;
+    if (rows == 0) return fail(ctx, ACACHE_ERR_INVALID_ARG, "no rows were recomputed: nothing to predict from");
+    return acache_predict_commit(ctx, y, rows, block_rows, req->batch, n_blk, final_norm_g, w_lm, vocab, threshold, token,
+                                 confidence, commit, stream);
+}
+
 acache_status acache_probe_select(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers, acache_kv* kvs,
                                   const acache_request* req, const void* x0, double ratio, uint32_t flags, void* y_a,
                                   void* y_b, float* scores, int32_t* anchor_idx, acache_stream_t stream) {
