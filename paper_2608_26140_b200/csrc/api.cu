@@ -486,7 +486,9 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
         }
         mark(ctx, ACACHE_STAGE_SCORE, stream);
         // with a selection to follow, the ordered sum over heads is folded into the selection kernel
-        fused_head_sum = do_select && k > 0 && req->n_masked > 0;
+        // (only while one CTA per request can read all heads' partial sums quickly: at L = 8192 the separate,
+        // grid-wide head sum takes 4 us where the folded one took 28)
+        fused_head_sum = do_select && k > 0 && req->n_masked > 0 && (int64_t)req->affix_len * d.n_heads <= 65536;
         s = run_score(ctx, req, qmask, kv, scores, (flags & ACACHE_F_ACCUMULATE) ? 1 : 0,
                       (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, fused_head_sum ? 1 : 0, stream);
         if (s != ACACHE_OK) return s;

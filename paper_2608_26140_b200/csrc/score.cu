@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_spl
     pdl_wait();
     pdl_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int split = blockIdx.x, h = blockIdx.y;
+    const int split = blockIdx.y, h = blockIdx.x;     // heads fastest: CTAs running together read whole K rows
     const int mtiles = (a.m + 63) / 64;
     const int b = blockIdx.z / mtiles, mt = blockIdx.z % mtiles;
     const int kvh = h / (a.n_heads / a.n_kv_heads);
@@ -155,26 +155,31 @@ __global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_spl
 }
 
 // ---- pass 2: per-key column sums of the normalised weights -------------------------------
+// One CTA = `kt_per_cta` consecutive tiles of 64 affix keys of one head (four when the masked rows fit
+// one 64-row tile, so that the combination of the split statistics and the Q tile load are paid once
+// per 256 keys; one otherwise, with the Q tiles streaming through a double buffer).
 template <int D>
-__global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_split, float scale_log2e) {
+__global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_split, float scale_log2e, int kt_per_cta) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int TILE = 64 * D * 2;
-    const uint32_t sK = smem_u32(smem), sQ0 = sK + TILE;
-    float* s_max = reinterpret_cast<float*>(smem + 3 * TILE);
+    const uint32_t sK0 = smem_u32(smem), sQ0 = sK0 + 2 * TILE;
+    float* s_max = reinterpret_cast<float*>(smem + 4 * TILE);
     float* s_inv = s_max + a.m;
     pdl_wait();
     pdl_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int jt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int h = blockIdx.x, b = blockIdx.z;                     // heads fastest (see the statistics pass)
     const int kvh = h / (a.n_heads / a.n_kv_heads);
     const int64_t qstride = (int64_t)a.n_heads * D, kstride = (int64_t)a.n_kv_heads * D;
     const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.q_mask) + (int64_t)b * a.m * qstride + (int64_t)h * D;
-    const int j0 = jt * 64;
+    const int key_tiles = (a.affix_len + 63) / 64;
+    const int jt_first = blockIdx.y * kt_per_cta;
+    const int n_my = min(kt_per_cta, key_tiles - jt_first);
     const __nv_bfloat16* kbase = static_cast<const __nv_bfloat16*>(a.cache_k) + (int64_t)b * a.kv_batch_stride +
-                                 (int64_t)(a.affix_start + j0) * kstride + (int64_t)kvh * D;
+                                 (int64_t)a.affix_start * kstride + (int64_t)kvh * D;
     const int mtiles = (a.m + 63) / 64;
 
-    load_tile64<D>(sK, kbase, kstride, min(64, a.affix_len - j0), tid, 128);
+    load_tile64<D>(sK0, kbase + (int64_t)jt_first * 64 * kstride, kstride, min(64, a.affix_len - jt_first * 64), tid, 128);
     load_tile64<D>(sQ0, q, qstride, min(64, a.m), tid, 128);
     cp_async_commit();
 
@@ -189,41 +194,51 @@ __global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_sp
         s_max[r] = M;
         s_inv[r] = 1.f / Dn;
     }
-    cp_async_wait<0>();
-    __syncthreads();
-    uint32_t af[D / 16][4];
-    load_a_frags<D>(af, sK, warp * 16, lane);
-
-    float colsum[2] = {0.f, 0.f};
-    for (int t = 0; t < mtiles; ++t) {
-        const uint32_t sQ = sQ0 + (t & 1) * TILE;
-        if (t + 1 < mtiles) {
-            load_tile64<D>(sQ0 + ((t + 1) & 1) * TILE, q + (int64_t)(t + 1) * 64 * qstride, qstride,
-                           min(64, a.m - (t + 1) * 64), tid, 128);
+    for (int kt = 0; kt < n_my; ++kt) {
+        const int j0 = (jt_first + kt) * 64;
+        cp_async_wait<0>();
+        __syncthreads();
+        if (kt + 1 < n_my) {
+            load_tile64<D>(sK0 + ((kt + 1) & 1) * TILE, kbase + (int64_t)(j0 + 64) * kstride, kstride,
+                           min(64, a.affix_len - (j0 + 64)), tid, 128);
             cp_async_commit();
         }
-        float acc[8][4];
-        mma_16x64<D>(acc, af, sQ, lane);   // rows = keys, cols = masked queries
-#pragma unroll
-        for (int nb = 0; nb < 8; ++nb)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                int qrow = t * 64 + nb * 8 + (lane & 3) * 2 + (i & 1);
-                if (qrow < a.m) colsum[i >> 1] += exp2f(acc[nb][i] * scale_log2e - s_max[qrow]) * s_inv[qrow];
+        uint32_t af[D / 16][4];
+        load_a_frags<D>(af, sK0 + (kt & 1) * TILE, warp * 16, lane);
+
+        float colsum[2] = {0.f, 0.f};
+        for (int t = 0; t < mtiles; ++t) {
+            const uint32_t sQ = sQ0 + (t & 1) * TILE;
+            if (t + 1 < mtiles) {          // only with one key tile per CTA: nothing else is in flight
+                load_tile64<D>(sQ0 + ((t + 1) & 1) * TILE, q + (int64_t)(t + 1) * 64 * qstride, qstride,
+                               min(64, a.m - (t + 1) * 64), tid, 128);
+                cp_async_commit();
             }
-        if (t + 1 < mtiles) cp_async_wait<0>();
-        __syncthreads();
-    }
+            float acc[8][4];
+            mma_16x64<D>(acc, af, sQ, lane);   // rows = keys, cols = masked queries
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        colsum[r] += __shfl_xor_sync(0xffffffffu, colsum[r], 1);
-        colsum[r] += __shfl_xor_sync(0xffffffffu, colsum[r], 2);
-    }
-    if ((lane & 3) == 0) {
+            for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    int qrow = t * 64 + nb * 8 + (lane & 3) * 2 + (i & 1);
+                    if (qrow < a.m) colsum[i >> 1] += exp2f(acc[nb][i] * scale_log2e - s_max[qrow]) * s_inv[qrow];
+                }
+            if (t + 1 < mtiles) {
+                cp_async_wait<0>();
+                __syncthreads();
+            }
+        }
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-            int j = j0 + warp * 16 + (lane >> 2) + r * 8;
-            if (j < a.affix_len) a.head_partial[((int64_t)b * a.n_heads + h) * a.affix_len + j] = colsum[r];
+            colsum[r] += __shfl_xor_sync(0xffffffffu, colsum[r], 1);
+            colsum[r] += __shfl_xor_sync(0xffffffffu, colsum[r], 2);
+        }
+        if ((lane & 3) == 0) {
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                int j = j0 + warp * 16 + (lane >> 2) + r * 8;
+                if (j < a.affix_len) a.head_partial[((int64_t)b * a.n_heads + h) * a.affix_len + j] = colsum[r];
+            }
         }
     }
 }
@@ -250,13 +265,18 @@ static int launch_score_d(const ScoreArgs& a, cudaStream_t stream) {
     constexpr int TILE = 64 * D * 2;
     const int mtiles = (a.m + 63) / 64;
     const size_t smem1 = 3 * TILE;
-    const size_t smem2 = 3 * TILE + (size_t)a.m * 8;
+    const size_t smem2 = 4 * TILE + (size_t)a.m * 8;
+    const int key_tiles = (a.affix_len + 63) / 64;
+    // several key tiles per CTA only while that still leaves a few waves of CTAs (measured: L = 512, B = 1 is
+    // faster with one tile per CTA, L = 8192 with four)
+    const int64_t ctas1 = (int64_t)a.n_heads * key_tiles * a.batch;
+    const int kt_per_cta = mtiles > 1 ? 1 : ctas1 >= 2400 ? 4 : ctas1 >= 1200 ? 2 : 1;
     cudaFuncSetAttribute(score_stats_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
     cudaFuncSetAttribute(score_colsum_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
-    launch_pdl(score_stats_kernel<D>, dim3(n_split, a.n_heads, a.batch * mtiles), 128, smem1, stream, a, n_split,
+    launch_pdl(score_stats_kernel<D>, dim3(a.n_heads, n_split, a.batch * mtiles), 128, smem1, stream, a, n_split,
                scale_log2e);
-    launch_pdl(score_colsum_kernel<D>, dim3((a.affix_len + 63) / 64, a.n_heads, a.batch), 128, smem2, stream, a,
-               n_split, scale_log2e);
+    launch_pdl(score_colsum_kernel<D>, dim3(a.n_heads, (key_tiles + kt_per_cta - 1) / kt_per_cta, a.batch), 128, smem2, stream, a,
+               n_split, scale_log2e, kt_per_cta);
     if (a.defer_head_sum) return 2;   // the selection kernel sums the heads itself
     launch_pdl(score_reduce_heads_kernel, dim3((a.affix_len + 255) / 256, a.batch), 256, 0, stream, a.head_partial,
                a.scores, a.n_heads, a.affix_len, a.accumulate);
