@@ -127,6 +127,7 @@ acache_status run_score(acache_ctx* c, const acache_request* r, const void* q_ma
     a.scores = scores;
     a.accumulate = accumulate;
     a.defer_head_sum = defer_head_sum;
+    a.status = wsp<uint32_t>(c, c->o_status);
     int n = launch_score(a, st);
     if (n < 0) return fail(c, ACACHE_ERR_UNSUPPORTED_SHAPE, "n_masked %d too large for the scoring kernel", r->n_masked);
     c->launches += n;

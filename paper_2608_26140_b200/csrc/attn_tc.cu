@@ -381,12 +381,14 @@ EncodeTiledFn encode_fn3() {
     return fn;
 }
 
+}  // namespace
+
 // bf16 [batch, rows, cols] with row stride = cols and the given batch stride (elements);
 // box = 64 cols x 128 rows x 1, 128-byte swizzle, zero fill out of bounds.
 struct Map3Key { const void* ptr; int rows, cols, batch; int64_t bstride; };
 struct Map3Entry { Map3Key key; CUtensorMap map; };
 constexpr int kMap3Cache = 64;
-std::mutex g_map3_mutex;
+std::mutex g_map3_mutex;   // guards the cache below; held from the lookups to the launch that uses them
 Map3Entry g_maps3[kMap3Cache];
 int g_map3_count = 0, g_map3_next = 0;
 
@@ -412,6 +414,8 @@ const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int6
     return &e.map;
 }
 
+
+namespace {
 }  // namespace
 
 // Returns the number of kernels launched, 0 if this problem is not for the tensor-core kernel

@@ -44,7 +44,12 @@ struct ScoreArgs {
     float* scores;            // [B, L]
     int accumulate;
     int defer_head_sum;       // leave head_partial unsummed: launch_topk(.., head_partial) does it
+    uint32_t* status;         // device status word (bounded waits of the tensor-core kernels); may be null
 };
+// tcgen05 kernels for head dimension 128 and up to 256 masked rows (two passes into row_stats / head_partial);
+// 0 = not applicable, -1 = launch failed.  Their statistics use one entry per score_tc_splits() keys.
+int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream);
+int score_tc_splits(int norm_len);
 int score_num_splits(int norm_len);
 int launch_score(const ScoreArgs& a, cudaStream_t stream);  // returns number of kernels launched
 

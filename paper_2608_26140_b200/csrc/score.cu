@@ -290,6 +290,14 @@ int launch_score(const ScoreArgs& a, cudaStream_t stream) {
         return 0;
     }
     if (a.m > kMaxMaskedSmem) return -1;
+    const int tc = launch_score_tc(a, a.status, stream);
+    if (tc < 0) return -1;
+    if (tc > 0) {
+        if (a.defer_head_sum) return tc;
+        launch_pdl(score_reduce_heads_kernel, dim3((a.affix_len + 255) / 256, a.batch), 256, 0, stream, a.head_partial,
+                   a.scores, a.n_heads, a.affix_len, a.accumulate);
+        return tc + 1;
+    }
     return a.head_dim == 128 ? launch_score_d<128>(a, stream) : launch_score_d<64>(a, stream);
 }
 

@@ -1,0 +1,374 @@
+// Anchor scoring (Eq. 4-5) for head dimension 128 on the 5th-generation tensor cores.  Both passes stream
+// the cached affix keys through shared memory by TMA and are bound by that read:
+//
+//   pass 1, row statistics   S = Q_mask K^T  (M = 128 masked rows of one head, N = 256 keys per stage);
+//                            thread = masked row: running maximum and denominator over the normaliser's
+//                            key range, one entry per CTA (key split);
+//   pass 2, column sums      D = K Q_mask^T  (M = 128 keys, N = the masked rows rounded up to 32);
+//                            thread = key: sum over the masked rows of exp2(logit - max_q) / den_q,
+//                            a sum over the accumulator's columns, so no thread exchanges anything.
+//
+// The orientation is swapped between the passes so that each reduction runs along the TMEM columns a
+// thread holds.  Rows of the query tile past the last masked row and keys past the range read as zero
+// through the tensor maps and are masked out.  No float atomics: results are bitwise reproducible.
+// Every mbarrier wait is bounded (status flag kFlagWaitExpired on expiry).
+#include <cuda.h>
+
+#include <mutex>
+
+#include "common.cuh"
+#include "kernels.h"
+#include "launch.h"
+#include "tc_ptx.cuh"
+
+namespace acache {
+
+namespace {
+
+constexpr int ST_THREADS = 192;                 // warp 0: TMA, warp 1: MMA, warps 2-5: one thread per accumulator row
+constexpr int ST_PANEL128 = 128 * 64 * 2;       // 16 KB: 128 rows x 64 columns
+constexpr int ST_PANEL256 = 256 * 64 * 2;       // 32 KB
+constexpr int ST_Q_BYTES = 2 * ST_PANEL128;     // pass 1: the query tile, 128 rows x 128
+constexpr int ST_K_BYTES = 2 * ST_PANEL256;     // pass 1: 256 keys x 128 per stage
+constexpr int ST_SMEM1 = ST_Q_BYTES + 2 * ST_K_BYTES + 1024 + 256;
+constexpr int CS_Q_BYTES = 2 * ST_PANEL256;     // pass 2: up to 256 masked rows x 128
+constexpr int CS_K_BYTES = 2 * ST_PANEL128;     // pass 2: 128 keys x 128 per stage
+constexpr int CS_STAGES = 3;
+constexpr int CS_SMEM = CS_Q_BYTES + CS_STAGES * CS_K_BYTES + 2048 + 1024 + 256;
+constexpr int kKeysPerCta1 = 1024;              // pass 1: keys per CTA = one statistics entry
+constexpr int kTilesPerCta2 = 4;                // pass 2: 128-key tiles per CTA
+
+__device__ __forceinline__ void tma3(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(pol)
+        : "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+struct ScoreTcArgs {
+    float* row_stats;        // [B, H, n_split, m, 2]
+    float* head_partial;     // [B, H, L]
+    int m, n_heads, n_kv_heads;
+    int norm_lo, norm_len, affix_start, affix_len;
+    int n_split, cache_shared;
+    float scale_log2e;
+    uint32_t* status;
+};
+
+// ---- pass 1 -------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ST_THREADS, 1)
+score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t sQ = base, sK0 = base + ST_Q_BYTES;
+    const uint32_t bars = base + ST_Q_BYTES + 2 * ST_K_BYTES;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + ST_Q_BYTES + 2 * ST_K_BYTES + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + ST_Q_BYTES + 2 * ST_K_BYTES + 200);
+    // barriers: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 s_full | 7,8 s_empty
+    auto bar = [&](int i) { return bars + 8 * i; };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.x, split = blockIdx.y;
+    const int mtiles = (a.m + 127) / 128;
+    const int b = blockIdx.z / mtiles, mt = blockIdx.z - b * mtiles;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int kb = a.cache_shared ? 0 : b;
+    const int key0 = split * kKeysPerCta1;
+    const int n_keys = min(kKeysPerCta1, a.norm_len - key0);
+    const int n_stage = (n_keys + 255) / 256;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i <= 6; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(7), 4); mbar_init(bar(8), 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();
+    pdl_launch_dependents();
+
+    if (warp == 0 && lane == 0) {
+        const uint64_t pol_q = policy_evict_last(), pol_k = policy_evict_last();   // the second pass reads the keys again
+        mbar_expect_tx(bar(0), ST_Q_BYTES);
+        tma3(sQ, &mapQ, h * 128, mt * 128, b, bar(0), pol_q);
+        tma3(sQ + ST_PANEL128, &mapQ, h * 128 + 64, mt * 128, b, bar(0), pol_q);
+        bool ok = true;
+        for (int st = 0; st < n_stage && ok; ++st) {
+            const int s = st & 1;
+            if (!(ok = mbar_wait(bar(3 + s), ((st >> 1) & 1) ^ 1, abort_flag))) break;
+            mbar_expect_tx(bar(1 + s), ST_K_BYTES);
+            const uint32_t dst = sK0 + s * ST_K_BYTES;
+            const int row = a.norm_lo + key0 + st * 256;
+#pragma unroll
+            for (int p = 0; p < 2; ++p)
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+                    tma3(dst + p * ST_PANEL256 + r * ST_PANEL128, &mapK, kvh * 128 + p * 64, row + r * 128, kb, bar(1 + s), pol_k);
+        }
+    } else if (warp == 1 && lane == 0) {
+        const uint32_t idesc = idesc_bf16(256);
+        bool ok = mbar_wait(bar(0), 0, abort_flag);
+        for (int st = 0; st < n_stage && ok; ++st) {
+            const int s = st & 1;
+            const uint32_t par = (st >> 1) & 1;
+            if (!(ok = mbar_wait(bar(1 + s), par, abort_flag))) break;
+            if (!(ok = mbar_wait(bar(7 + s), par ^ 1, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t k = sK0 + s * ST_K_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t da = smem_desc_sw128(sQ + (ks >> 2) * ST_PANEL128) + (uint64_t)((ks & 3) * 2);
+                const uint64_t db = smem_desc_sw128(k + (ks >> 2) * ST_PANEL256) + (uint64_t)((ks & 3) * 2);
+                tc_mma(tmem_base + s * 256, da, db, idesc, ks > 0 ? 1u : 0u);
+            }
+            tc_commit(bar(5 + s));     // s_full
+            tc_commit(bar(3 + s));     // k_empty
+        }
+    } else if (warp >= 2) {
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const int grow = mt * 128 + row;
+        const bool live = (mt * 128 + q * 32) < a.m;        // whole warps past the last masked row only keep the barriers moving
+        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+        float mx = -INFINITY, den = 0.f;
+        bool ok = true;
+        for (int st = 0; st < n_stage && ok; ++st) {
+            const int s = st & 1;
+            if (!(ok = mbar_wait(bar(5 + s), (st >> 1) & 1, abort_flag))) break;
+            tc_fence_after();
+            if (live) {
+                const int valid = n_keys - st * 256;
+                for (int c = 0; c < 8 && c * 32 < valid; ++c) {
+                    float v[32];
+                    tc_ld32(tmem_base + s * 256 + lane_off + c * 32, v);
+                    const int nv = valid - c * 32;
+                    float tm = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        v[i] = i < nv ? v[i] * a.scale_log2e : -INFINITY;
+                        tm = fmaxf(tm, v[i]);
+                    }
+                    const float nm = fmaxf(mx, tm);
+                    float part = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) part += ex2(v[i] - nm);
+                    den = den * ex2(mx - nm) + part;
+                    mx = nm;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(7 + s));   // s_empty
+        }
+        if (ok && live && grow < a.m) {
+            float* stp = a.row_stats + ((((int64_t)b * a.n_heads + h) * a.n_split + split) * a.m + grow) * 2;
+            stp[0] = mx;
+            stp[1] = den;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) {
+            atomicOr(a.status, kFlagWaitExpired);
+            for (int i = 0; i < 4096; ++i) __nanosleep(64);
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
+// ---- pass 2 -------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ST_THREADS, 1)
+score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_constant__ CUtensorMap mapQ,
+                       const __grid_constant__ CUtensorMap mapK) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t sQ = base, sK0 = base + CS_Q_BYTES;
+    float* s_max = reinterpret_cast<float*>(base_ptr + CS_Q_BYTES + CS_STAGES * CS_K_BYTES);     // [256]
+    float* s_inv = s_max + 256;
+    const uint32_t bars = base + CS_Q_BYTES + CS_STAGES * CS_K_BYTES + 2048;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + CS_Q_BYTES + CS_STAGES * CS_K_BYTES + 2048 + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + CS_Q_BYTES + CS_STAGES * CS_K_BYTES + 2048 + 200);
+    // barriers: 0 q_full | 1..3 k_full | 4..6 k_empty | 7,8 d_full | 9,10 d_empty
+    auto bar = [&](int i) { return bars + 8 * i; };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.x, chunk = blockIdx.y, b = blockIdx.z;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int kb = a.cache_shared ? 0 : b;
+    const int key_tiles = (a.affix_len + 127) / 128;
+    const int t0 = chunk * kTilesPerCta2;
+    const int n_tiles = min(kTilesPerCta2, key_tiles - t0);
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i <= 8; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(9), 4); mbar_init(bar(10), 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();
+    pdl_launch_dependents();
+
+    // combine the split statistics of every masked row (fixed order)
+    if (threadIdx.x >= 64) {
+        const float* st = a.row_stats + ((int64_t)b * a.n_heads + h) * a.n_split * a.m * 2;
+        for (int r = threadIdx.x - 64; r < 256; r += 128) {
+            float M = -INFINITY, Dn = 0.f;
+            if (r < a.m) {
+                for (int s = 0; s < a.n_split; ++s) M = fmaxf(M, st[((int64_t)s * a.m + r) * 2]);
+                for (int s = 0; s < a.n_split; ++s)
+                    Dn += st[((int64_t)s * a.m + r) * 2 + 1] * ex2(st[((int64_t)s * a.m + r) * 2] - M);
+            }
+            s_max[r] = r < a.m ? M : 0.f;           // padding rows: logit 0, weight 0
+            s_inv[r] = r < a.m ? 1.f / Dn : 0.f;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
+
+    if (warp == 0 && lane == 0) {
+        const uint64_t pol = policy_evict_first();
+        const uint64_t pol_q = policy_evict_last();
+        mbar_expect_tx(bar(0), 2u * (uint32_t)((n_pad + 127) / 128) * ST_PANEL128);   // whole boxes, zero fill included
+        for (int p = 0; p < 2; ++p)
+            for (int r = 0; r * 128 < n_pad; ++r)      // a box is 128 rows: rows past n_pad are loaded too but never read
+                tma3(sQ + p * ST_PANEL256 + r * ST_PANEL128, &mapQ, h * 128 + p * 64, r * 128, b, bar(0), pol_q);
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int s = t % CS_STAGES;
+            if (!(ok = mbar_wait(bar(4 + s), ((t / CS_STAGES) & 1) ^ 1, abort_flag))) break;
+            mbar_expect_tx(bar(1 + s), CS_K_BYTES);
+            const uint32_t dst = sK0 + s * CS_K_BYTES;
+            const int row = a.affix_start + (t0 + t) * 128;
+            tma3(dst, &mapK, kvh * 128, row, kb, bar(1 + s), pol);
+            tma3(dst + ST_PANEL128, &mapK, kvh * 128 + 64, row, kb, bar(1 + s), pol);
+        }
+    } else if (warp == 1 && lane == 0) {
+        const uint32_t idesc = idesc_bf16(n_pad);
+        bool ok = mbar_wait(bar(0), 0, abort_flag);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int s = t % CS_STAGES, d = t & 1;
+            if (!(ok = mbar_wait(bar(1 + s), (t / CS_STAGES) & 1, abort_flag))) break;
+            if (!(ok = mbar_wait(bar(9 + d), ((t >> 1) & 1) ^ 1, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t k = sK0 + s * CS_K_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t da = smem_desc_sw128(k + (ks >> 2) * ST_PANEL128) + (uint64_t)((ks & 3) * 2);
+                const uint64_t db = smem_desc_sw128(sQ + (ks >> 2) * ST_PANEL256) + (uint64_t)((ks & 3) * 2);
+                tc_mma(tmem_base + d * 256, da, db, idesc, ks > 0 ? 1u : 0u);
+            }
+            tc_commit(bar(7 + d));     // d_full
+            tc_commit(bar(4 + s));     // k_empty
+        }
+    } else if (warp >= 2) {
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int d = t & 1;
+            if (!(ok = mbar_wait(bar(7 + d), (t >> 1) & 1, abort_flag))) break;
+            tc_fence_after();
+            float sum = 0.f;
+            for (int c = 0; c * 32 < n_pad; ++c) {
+                float v[32];
+                tc_ld32(tmem_base + d * 256 + lane_off + c * 32, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) sum += ex2(fmaf(v[i], a.scale_log2e, -s_max[c * 32 + i])) * s_inv[c * 32 + i];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(9 + d));   // d_empty
+            const int j = (t0 + t) * 128 + row;
+            if (j < a.affix_len) a.head_partial[((int64_t)b * a.n_heads + h) * a.affix_len + j] = sum;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) {
+            atomicOr(a.status, kFlagWaitExpired);
+            for (int i = 0; i < 4096; ++i) __nanosleep(64);
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
+}  // namespace
+
+int score_tc_splits(int norm_len) { return (norm_len + kKeysPerCta1 - 1) / kKeysPerCta1; }
+
+// Launches the two passes; 0 if the problem is not for these kernels (the caller uses the mma.sync ones).
+int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
+    if (a.head_dim != 128 || a.m > 256 || a.m <= 0 || !status) return 0;
+    if ((a.kv_batch_stride * 2) % 16) return 0;
+    static const bool off = [] { const char* e = getenv("ACACHE_SCORE_TC"); return e && e[0] == '0'; }();
+    if (off) return 0;
+    // measured (m = 32): the mma.sync kernels win while there is little to read (L = 512, B = 1: 16.5 against 22 us),
+    // these from a few thousand keys up (L = 8192: 58 against 74 us; B = 8, L = 2048: 100 against 131 us)
+    if ((int64_t)a.batch * a.norm_len < 4096) return 0;
+    const bool shared = a.kv_batch_stride == 0;
+    const int kv_cols = a.n_kv_heads * 128;
+    const int ctx_rows = a.norm_lo + a.norm_len > a.affix_start + a.affix_len ? a.norm_lo + a.norm_len : a.affix_start + a.affix_len;
+    std::lock_guard<std::mutex> lock(g_map3_mutex);
+    const CUtensorMap* mq = get_map3(a.q_mask, a.m, a.n_heads * 128, a.batch, (int64_t)a.m * a.n_heads * 128);
+    const CUtensorMap* mk = get_map3(a.cache_k, ctx_rows, kv_cols, shared ? 1 : a.batch,
+                                     shared ? (int64_t)ctx_rows * kv_cols : a.kv_batch_stride);
+    if (!mq || !mk) return 0;
+    static bool attr = false;
+    if (!attr) {
+        cudaFuncSetAttribute(score_stats_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM1);
+        cudaFuncSetAttribute(score_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CS_SMEM);
+        attr = true;
+    }
+    ScoreTcArgs t{};
+    t.row_stats = a.row_stats; t.head_partial = a.head_partial;
+    t.m = a.m; t.n_heads = a.n_heads; t.n_kv_heads = a.n_kv_heads;
+    t.norm_lo = a.norm_lo; t.norm_len = a.norm_len; t.affix_start = a.affix_start; t.affix_len = a.affix_len;
+    t.n_split = score_tc_splits(a.norm_len); t.cache_shared = shared ? 1 : 0;
+    t.scale_log2e = 1.4426950408889634f / sqrtf(128.f);
+    t.status = status;
+    const int mtiles = (a.m + 127) / 128;
+    if (launch_pdl(score_stats_tc_kernel, dim3(a.n_heads, t.n_split, a.batch * mtiles), dim3(ST_THREADS), ST_SMEM1, stream, t, *mq,
+                   *mk) != cudaSuccess)
+        return -1;
+    const int n_pad = (a.m + 31) & ~31;
+    const int key_tiles = (a.affix_len + 127) / 128;
+    if (launch_pdl(score_colsum_tc_kernel, dim3(a.n_heads, (key_tiles + kTilesPerCta2 - 1) / kTilesPerCta2, a.batch),
+                   dim3(ST_THREADS), CS_SMEM, stream, t, n_pad, *mq, *mk) != cudaSuccess)
+        return -1;
+    return 2;
+}
+
+}  // namespace acache

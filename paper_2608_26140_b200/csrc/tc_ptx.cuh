@@ -4,6 +4,8 @@
 #pragma once
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace acache {
@@ -115,5 +117,11 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+
+// 3-d tensor maps over bf16 [batch, rows, cols] (row stride = cols, batch stride in elements), box 64 cols x
+// 128 rows x 1, 128-byte swizzle, zero fill out of bounds; cached by (pointer, shape).  Host side, defined in
+// attn_tc.cu; the returned pointer stays valid while g_map3_mutex is held.
+const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int64_t bstride);
+extern std::mutex g_map3_mutex;
 
 }  // namespace acache
