@@ -26,6 +26,7 @@ namespace acache {
 namespace {
 
 constexpr int ST_THREADS = 192;                 // warp 0: TMA, warp 1: MMA, warps 2-5: one thread per accumulator row
+constexpr int ST_THREADS1 = 576;                // pass 1: sixteen statistics warps, four per row quarter (64 of a stage's 256 keys each)
 constexpr int ST_PANEL128 = 128 * 64 * 2;       // 16 KB: 128 rows x 64 columns
 constexpr int ST_PANEL256 = 256 * 64 * 2;       // 32 KB
 constexpr int ST_Q_BYTES = 2 * ST_PANEL128;     // pass 1: the query tile, 128 rows x 128
@@ -62,7 +63,7 @@ struct ScoreTcArgs {
 };
 
 // ---- pass 1 -------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(ST_THREADS, 1)
+__global__ void __launch_bounds__(ST_THREADS1, 1)
 score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -85,7 +86,7 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 6; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(7), 4); mbar_init(bar(8), 4);
+        mbar_init(bar(7), 16); mbar_init(bar(8), 16);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -139,7 +140,9 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
             tc_commit(bar(3 + s));     // k_empty
         }
     } else if (warp >= 2) {
-        const int q = warp & 3;
+        // thread = (masked row, quarter of the stage's keys): with few masked rows only the warps of the first
+        // row quarter(s) have work, so each row's 256 keys per stage are split over four warps
+        const int q = warp & 3, cw = (warp - 2) >> 2;
         const int row = q * 32 + lane;
         const int grow = mt * 128 + row;
         const bool live = (mt * 128 + q * 32) < a.m;        // whole warps past the last masked row only keep the barriers moving
@@ -151,10 +154,10 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
             if (!(ok = mbar_wait(bar(5 + s), (st >> 1) & 1, abort_flag))) break;
             tc_fence_after();
             if (live) {
-                const int valid = n_keys - st * 256;
-                for (int c = 0; c < 8 && c * 32 < valid; ++c) {
+                const int valid = n_keys - st * 256 - cw * 64;     // keys of this thread's quarter that exist
+                for (int c = 0; c < 2 && c * 32 < valid; ++c) {
                     float v[32];
-                    tc_ld32(tmem_base + s * 256 + lane_off + c * 32, v);
+                    tc_ld32(tmem_base + s * 256 + lane_off + cw * 64 + c * 32, v);
                     const int nv = valid - c * 32;
                     float tm = -INFINITY;
 #pragma unroll
@@ -174,10 +177,17 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(7 + s));   // s_empty
         }
-        if (ok && live && grow < a.m) {
+        // merge the four key quarters of every row in a fixed order (the K stages are idle by now)
+        float2* ex = reinterpret_cast<float2*>(base_ptr + ST_Q_BYTES);
+        ex[cw * 128 + row] = make_float2(mx, den);
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+        if (ok && !*abort_flag && cw == 0 && live && grow < a.m) {
+            float M = -INFINITY, Dn = 0.f;
+            for (int c = 0; c < 4; ++c) M = fmaxf(M, ex[c * 128 + row].x);
+            for (int c = 0; c < 4; ++c) Dn += ex[c * 128 + row].y * ex2(ex[c * 128 + row].x - M);
             float* stp = a.row_stats + ((((int64_t)b * a.n_heads + h) * a.n_split + split) * a.m + grow) * 2;
-            stp[0] = mx;
-            stp[1] = den;
+            stp[0] = M;
+            stp[1] = Dn;
         }
     }
     tc_fence_before();
@@ -360,7 +370,7 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
     t.scale_log2e = 1.4426950408889634f / sqrtf(128.f);
     t.status = status;
     const int mtiles = (a.m + 127) / 128;
-    if (launch_pdl(score_stats_tc_kernel, dim3(a.n_heads, t.n_split, a.batch * mtiles), dim3(ST_THREADS), ST_SMEM1, stream, t, *mq,
+    if (launch_pdl(score_stats_tc_kernel, dim3(a.n_heads, t.n_split, a.batch * mtiles), dim3(ST_THREADS1), ST_SMEM1, stream, t, *mq,
                    *mk) != cudaSuccess)
         return -1;
     const int n_pad = (a.m + 31) & ~31;
