@@ -415,3 +415,47 @@ def test_duplicate_row_is_served_once_in_the_split_calls():
     ref = oracle_step(case, 0, anchor_idx=anchors[0])
     assert_close_bf16(ab.to_host_bits(y[0]), ref["y"], "y with a duplicated row")
     assert_close_bf16(ab.to_host_bits(k_new[0]), ref["k_new"], "k_new with a duplicated row")
+
+
+def test_degenerate_inputs():
+    """Empty batch, no masked rows, a one-token affix: nothing faults, the defined results come out."""
+    shape = MID128
+    lay = wl.make_layout(2, 3, 40, 9, 32, 32, "all")
+    case = wl.make_case(shape, lay, 0.25, cfg_id=27)
+    dc = DeviceCase(case)
+    B, L, T = lay.batch, lay.affix_len, lay.ctx_len
+    K = orc.k_from_ratio(L, 0.25)
+    n = K + lay.n_extra
+    scores = torch.full((B, L), 5.0, dtype=torch.float32, device=DEV)
+    anchors = torch.full((B, K), -1, dtype=torch.int32, device=DEV)
+    y = torch.zeros((B, n, shape.hidden), dtype=torch.bfloat16, device=DEV)
+    # an empty batch launches nothing
+    req0 = ab.Context.request(0, T, lay.affix_start, L, dc.masked, dc.extra, dc.cos, dc.sin)
+    l0 = dc.ctx.launch_count()
+    dc.ctx.layer_step(dc.lw, req0, dc.kv(), dc.x, 0, 0.25, ab.F_SCORE | ab.F_SELECT, scores, anchors, y)
+    assert dc.ctx.launch_count() == l0
+    # no masked rows: this layer adds nothing to the scores (they are zeroed unless accumulating), Eq. 6 on
+    # all-equal scores takes the K lowest positions, and the refresh of those rows is the oracle's
+    req1 = ab.Context.request(B, T, lay.affix_start, L, None, dc.extra, dc.cos, dc.sin)
+    dc.ctx.layer_step(dc.lw, req1, dc.kv(), dc.x, 0, 0.25, ab.F_SCORE | ab.F_SELECT, scores, anchors, y)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(scores).item() == 0
+    assert np.array_equal(anchors.cpu().numpy(), np.broadcast_to(np.arange(K, dtype=np.int32), (B, K)))
+    for b in range(B):
+        ref = oracle_step(case, b, anchor_idx=np.arange(K))
+        assert_close_bf16(ab.to_host_bits(y[b]), ref["y"], "y with the K lowest positions as anchors")
+    scores.fill_(2.0)
+    dc.ctx.layer_step(dc.lw, req1, dc.kv(), dc.x, 0, 0.0, ab.F_SCORE | ab.F_ACCUMULATE | ab.F_NO_RECOMPUTE, scores, None, None)
+    torch.cuda.synchronize()
+    assert torch.all(scores == 2.0).item()
+    assert dc.ctx.poll_status() == 0
+    # a one-token affix at ratio 1: K = 1, the single affix row is refreshed
+    lay1 = wl.make_layout(1, 5, 1, 6, 32, 32, "none")
+    case1 = wl.make_case(shape, lay1, 1.0, cfg_id=28)
+    dc1 = DeviceCase(case1)
+    K1, s1, a1, y1 = run_layer_step(dc1, 1.0, ab.F_SCORE | ab.F_SELECT)
+    assert K1 == 1 and a1[0, 0] == 0
+    assert abs(s1[0, 0] - shape.n_heads * lay1.n_masked) < 1e-3 * shape.n_heads * lay1.n_masked     # softmax over one key
+    ref = oracle_step(case1, 0, anchor_idx=np.array([0]))
+    assert_close_bf16(ab.to_host_bits(y1[0, :1]), ref["y"], "y of the single affix row")
+    assert dc1.ctx.poll_status() == 0
