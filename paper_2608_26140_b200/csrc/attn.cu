@@ -3,7 +3,9 @@
 // Online-softmax tiles: S = Q K^T and O += P V on bf16 tensor-core tiles with fp32
 // accumulation and fp32 softmax statistics.  Keys/values come from the token-major cache or,
 // where a position -> fresh-row map says so, from the compact fresh K/V (the logical view of
-// the working cache without having written it).
+// the working cache without having written it).  This file holds the mma.sync kernels (head
+// dimension 64, and the fallback when the tcgen05 kernel of attn_tc.cu is switched off) and
+// the dispatch between the two.
 #include <cstdlib>
 
 #include "common.cuh"

@@ -12,6 +12,9 @@
 //                       L2), one thread issues tcgen05.mma (128 x 256 x 16) into one of two TMEM
 //                       accumulators, four warps drain TMEM with tcgen05.ld and write fp32
 //                       partial tiles
+// gemm_tc2_kernel (two or more 128-row tiles): a cluster of two CTAs per 256 x 256 tile,
+//   tcgen05.mma.cta_group::2; whole tiles walked round-robin, or, when the tiles fill less than
+//   two thirds of a wave, equal contiguous (tile, k-block) ranges per cluster like the kernel above.
 // gemm_finish_kernel: sums the partial tiles of every output element in ascending CTA order
 //   (bitwise reproducible) and applies the epilogue: bias + RoPE + KV scatter, residual add,
 //   or SwiGLU.  It is a kernel of its own because it is bound by L2 latency and wants far

@@ -154,7 +154,8 @@ struct AttnArgs {
     float* part_ml;           // scratch for key splits: fp32 [B*n*H, n_split, 2] (max, denominator)
     uint32_t* status;         // device status word
 };
-// tcgen05 kernel for many rows (head_dim 128, cache read in place); 0 = not applicable.
+// tcgen05 kernel (head_dim 128; the cache read in place, or cache + fresh rows as two key sources when the
+// key masks are given); 0 = not applicable.
 int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream);
 size_t attention_scratch_bytes(int head_dim);   // bytes for part_o followed by part_ml
 int launch_attention(const AttnArgs& a, cudaStream_t stream);
