@@ -25,17 +25,16 @@ namespace acache {
 
 namespace {
 
-constexpr int ST_THREADS = 192;                 // warp 0: TMA, warp 1: MMA, warps 2-5: one thread per accumulator row
-constexpr int ST_THREADS1 = 576;                // pass 1: sixteen statistics warps, four per row quarter (64 of a stage's 256 keys each)
+constexpr int ST_THREADS = 192;                 // pass 2: warp 0 TMA, warp 1 MMA, warps 2-5 one thread per key
+constexpr int ST_THREADS1 = 320;                // pass 1: eight statistics warps, two per row quarter (64 of a stage's 128 keys each)
 constexpr int ST_PANEL128 = 128 * 64 * 2;       // 16 KB: 128 rows x 64 columns
-constexpr int ST_PANEL256 = 256 * 64 * 2;       // 32 KB
 constexpr int ST_Q_BYTES = 2 * ST_PANEL128;     // pass 1: the query tile, 128 rows x 128
-constexpr int ST_K_BYTES = 2 * ST_PANEL256;     // pass 1: 256 keys x 128 per stage
+constexpr int ST_K_BYTES = 2 * ST_PANEL128;     // 128 keys x 128 per stage (both passes)
+// Both kernels are sized so that two CTAs share an SM (about 100 KB of shared memory and 256 TMEM columns
+// each): a CTA streams only a few stages, and the second CTA's stream hides the first one's start-up.
 constexpr int ST_SMEM1 = ST_Q_BYTES + 2 * ST_K_BYTES + 1024 + 256;
-constexpr int CS_Q_BYTES = 2 * ST_PANEL256;     // pass 2: up to 256 masked rows x 128
-constexpr int CS_K_BYTES = 2 * ST_PANEL128;     // pass 2: 128 keys x 128 per stage
-constexpr int CS_STAGES = 3;
-constexpr int CS_SMEM = CS_Q_BYTES + CS_STAGES * CS_K_BYTES + 2048 + 1024 + 256;
+constexpr int CS_STAGES = 2;
+constexpr int CS_TABLES = 2048;                 // max and 1 / denominator of up to 256 masked rows
 constexpr int kKeysPerCta1 = 1024;              // pass 1: keys per CTA = one statistics entry
 constexpr int kTilesPerCta2 = 4;                // pass 2: 128-key tiles per CTA
 
@@ -63,7 +62,7 @@ struct ScoreTcArgs {
 };
 
 // ---- pass 1 -------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(ST_THREADS1, 1)
+__global__ void __launch_bounds__(ST_THREADS1, 2)
 score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -82,16 +81,16 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
     const int kb = a.cache_shared ? 0 : b;
     const int key0 = split * kKeysPerCta1;
     const int n_keys = min(kKeysPerCta1, a.norm_len - key0);
-    const int n_stage = (n_keys + 255) / 256;
+    const int n_stage = (n_keys + 127) / 128;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 6; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(7), 16); mbar_init(bar(8), 16);
+        mbar_init(bar(7), 8); mbar_init(bar(8), 8);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;"
                      ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -113,15 +112,12 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
             if (!(ok = mbar_wait(bar(3 + s), ((st >> 1) & 1) ^ 1, abort_flag))) break;
             mbar_expect_tx(bar(1 + s), ST_K_BYTES);
             const uint32_t dst = sK0 + s * ST_K_BYTES;
-            const int row = a.norm_lo + key0 + st * 256;
-#pragma unroll
-            for (int p = 0; p < 2; ++p)
-#pragma unroll
-                for (int r = 0; r < 2; ++r)
-                    tma3(dst + p * ST_PANEL256 + r * ST_PANEL128, &mapK, kvh * 128 + p * 64, row + r * 128, kb, bar(1 + s), pol_k);
+            const int row = a.norm_lo + key0 + st * 128;
+            tma3(dst, &mapK, kvh * 128, row, kb, bar(1 + s), pol_k);
+            tma3(dst + ST_PANEL128, &mapK, kvh * 128 + 64, row, kb, bar(1 + s), pol_k);
         }
     } else if (warp == 1 && lane == 0) {
-        const uint32_t idesc = idesc_bf16(256);
+        const uint32_t idesc = idesc_bf16(128);
         bool ok = mbar_wait(bar(0), 0, abort_flag);
         for (int st = 0; st < n_stage && ok; ++st) {
             const int s = st & 1;
@@ -133,15 +129,15 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const uint64_t da = smem_desc_sw128(sQ + (ks >> 2) * ST_PANEL128) + (uint64_t)((ks & 3) * 2);
-                const uint64_t db = smem_desc_sw128(k + (ks >> 2) * ST_PANEL256) + (uint64_t)((ks & 3) * 2);
-                tc_mma(tmem_base + s * 256, da, db, idesc, ks > 0 ? 1u : 0u);
+                const uint64_t db = smem_desc_sw128(k + (ks >> 2) * ST_PANEL128) + (uint64_t)((ks & 3) * 2);
+                tc_mma(tmem_base + s * 128, da, db, idesc, ks > 0 ? 1u : 0u);
             }
             tc_commit(bar(5 + s));     // s_full
             tc_commit(bar(3 + s));     // k_empty
         }
     } else if (warp >= 2) {
-        // thread = (masked row, quarter of the stage's keys): with few masked rows only the warps of the first
-        // row quarter(s) have work, so each row's 256 keys per stage are split over four warps
+        // thread = (masked row, half of the stage's keys): with few masked rows only the warps of the first
+        // row quarter(s) have work, so each row's 128 keys per stage are split over two warps
         const int q = warp & 3, cw = (warp - 2) >> 2;
         const int row = q * 32 + lane;
         const int grow = mt * 128 + row;
@@ -154,10 +150,10 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
             if (!(ok = mbar_wait(bar(5 + s), (st >> 1) & 1, abort_flag))) break;
             tc_fence_after();
             if (live) {
-                const int valid = n_keys - st * 256 - cw * 64;     // keys of this thread's quarter that exist
+                const int valid = n_keys - st * 128 - cw * 64;     // keys of this thread's half that exist
                 for (int c = 0; c < 2 && c * 32 < valid; ++c) {
                     float v[32];
-                    tc_ld32(tmem_base + s * 256 + lane_off + cw * 64 + c * 32, v);
+                    tc_ld32(tmem_base + s * 128 + lane_off + cw * 64 + c * 32, v);
                     const int nv = valid - c * 32;
                     float tm = -INFINITY;
 #pragma unroll
@@ -177,14 +173,14 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(7 + s));   // s_empty
         }
-        // merge the four key quarters of every row in a fixed order (the K stages are idle by now)
+        // merge the two key halves of every row in a fixed order (the K stages are idle by now)
         float2* ex = reinterpret_cast<float2*>(base_ptr + ST_Q_BYTES);
         ex[cw * 128 + row] = make_float2(mx, den);
-        asm volatile("bar.sync 1, 512;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (ok && !*abort_flag && cw == 0 && live && grow < a.m) {
             float M = -INFINITY, Dn = 0.f;
-            for (int c = 0; c < 4; ++c) M = fmaxf(M, ex[c * 128 + row].x);
-            for (int c = 0; c < 4; ++c) Dn += ex[c * 128 + row].y * ex2(ex[c * 128 + row].x - M);
+            for (int c = 0; c < 2; ++c) M = fmaxf(M, ex[c * 128 + row].x);
+            for (int c = 0; c < 2; ++c) Dn += ex[c * 128 + row].y * ex2(ex[c * 128 + row].x - M);
             float* stp = a.row_stats + ((((int64_t)b * a.n_heads + h) * a.n_split + split) * a.m + grow) * 2;
             stp[0] = M;
             stp[1] = Dn;
@@ -201,24 +197,28 @@ score_stats_tc_kernel(const ScoreTcArgs a, const __grid_constant__ CUtensorMap m
     }
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem_base) : "memory");
     }
 }
 
 // ---- pass 2 -------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(ST_THREADS, 1)
+__global__ void __launch_bounds__(ST_THREADS, 2)
 score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_constant__ CUtensorMap mapQ,
                        const __grid_constant__ CUtensorMap mapK) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t sQ = base, sK0 = base + CS_Q_BYTES;
-    float* s_max = reinterpret_cast<float*>(base_ptr + CS_Q_BYTES + CS_STAGES * CS_K_BYTES);     // [256]
+    // the query tile: two 64-column panels of q_rows (128 or 256) rows each
+    const int q_rows = n_pad <= 128 ? 128 : 256;
+    const uint32_t q_panel = (uint32_t)q_rows * 128u, q_bytes = 2u * q_panel;
+    const uint32_t tmem_cols = n_pad <= 128 ? 256u : 512u;        // two accumulators of n_pad columns
+    const uint32_t sQ = base, sK0 = base + q_bytes;
+    float* s_max = reinterpret_cast<float*>(base_ptr + q_bytes + CS_STAGES * ST_K_BYTES);     // [256]
     float* s_inv = s_max + 256;
-    const uint32_t bars = base + CS_Q_BYTES + CS_STAGES * CS_K_BYTES + 2048;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + CS_Q_BYTES + CS_STAGES * CS_K_BYTES + 2048 + 192);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + CS_Q_BYTES + CS_STAGES * CS_K_BYTES + 2048 + 200);
-    // barriers: 0 q_full | 1..3 k_full | 4..6 k_empty | 7,8 d_full | 9,10 d_empty
+    const uint32_t bars = base + q_bytes + CS_STAGES * ST_K_BYTES + CS_TABLES;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + q_bytes + CS_STAGES * ST_K_BYTES + CS_TABLES + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + q_bytes + CS_STAGES * ST_K_BYTES + CS_TABLES + 200);
+    // barriers: 0 q_full | 1,2 k_full | 4,5 k_empty | 7,8 d_full | 9,10 d_empty
     auto bar = [&](int i) { return bars + 8 * i; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.x, chunk = blockIdx.y, b = blockIdx.z;
@@ -235,8 +235,8 @@ score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_consta
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
-                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -265,16 +265,16 @@ score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_consta
     if (warp == 0 && lane == 0) {
         const uint64_t pol = policy_evict_first();
         const uint64_t pol_q = policy_evict_last();
-        mbar_expect_tx(bar(0), 2u * (uint32_t)((n_pad + 127) / 128) * ST_PANEL128);   // whole boxes, zero fill included
+        mbar_expect_tx(bar(0), q_bytes);               // whole boxes of 128 rows, zero fill included
         for (int p = 0; p < 2; ++p)
-            for (int r = 0; r * 128 < n_pad; ++r)      // a box is 128 rows: rows past n_pad are loaded too but never read
-                tma3(sQ + p * ST_PANEL256 + r * ST_PANEL128, &mapQ, h * 128 + p * 64, r * 128, b, bar(0), pol_q);
+            for (int r = 0; r * 128 < q_rows; ++r)
+                tma3(sQ + p * q_panel + r * ST_PANEL128, &mapQ, h * 128 + p * 64, r * 128, b, bar(0), pol_q);
         bool ok = true;
         for (int t = 0; t < n_tiles && ok; ++t) {
             const int s = t % CS_STAGES;
             if (!(ok = mbar_wait(bar(4 + s), ((t / CS_STAGES) & 1) ^ 1, abort_flag))) break;
-            mbar_expect_tx(bar(1 + s), CS_K_BYTES);
-            const uint32_t dst = sK0 + s * CS_K_BYTES;
+            mbar_expect_tx(bar(1 + s), ST_K_BYTES);
+            const uint32_t dst = sK0 + s * ST_K_BYTES;
             const int row = a.affix_start + (t0 + t) * 128;
             tma3(dst, &mapK, kvh * 128, row, kb, bar(1 + s), pol);
             tma3(dst + ST_PANEL128, &mapK, kvh * 128 + 64, row, kb, bar(1 + s), pol);
@@ -287,12 +287,12 @@ score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_consta
             if (!(ok = mbar_wait(bar(1 + s), (t / CS_STAGES) & 1, abort_flag))) break;
             if (!(ok = mbar_wait(bar(9 + d), ((t >> 1) & 1) ^ 1, abort_flag))) break;
             tc_fence_after();
-            const uint32_t k = sK0 + s * CS_K_BYTES;
+            const uint32_t k = sK0 + s * ST_K_BYTES;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const uint64_t da = smem_desc_sw128(k + (ks >> 2) * ST_PANEL128) + (uint64_t)((ks & 3) * 2);
-                const uint64_t db = smem_desc_sw128(sQ + (ks >> 2) * ST_PANEL256) + (uint64_t)((ks & 3) * 2);
-                tc_mma(tmem_base + d * 256, da, db, idesc, ks > 0 ? 1u : 0u);
+                const uint64_t db = smem_desc_sw128(sQ + (ks >> 2) * q_panel) + (uint64_t)((ks & 3) * 2);
+                tc_mma(tmem_base + d * (tmem_cols >> 1), da, db, idesc, ks > 0 ? 1u : 0u);
             }
             tc_commit(bar(7 + d));     // d_full
             tc_commit(bar(4 + s));     // k_empty
@@ -309,7 +309,7 @@ score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_consta
             float sum = 0.f;
             for (int c = 0; c * 32 < n_pad; ++c) {
                 float v[32];
-                tc_ld32(tmem_base + d * 256 + lane_off + c * 32, v);
+                tc_ld32(tmem_base + d * (tmem_cols >> 1) + lane_off + c * 32, v);
 #pragma unroll
                 for (int i = 0; i < 32; ++i) sum += ex2(fmaf(v[i], a.scale_log2e, -s_max[c * 32 + i])) * s_inv[c * 32 + i];
             }
@@ -331,7 +331,7 @@ score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_consta
     }
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
 }
 
@@ -345,9 +345,10 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
     if ((a.kv_batch_stride * 2) % 16) return 0;
     static const bool off = [] { const char* e = getenv("ACACHE_SCORE_TC"); return e && e[0] == '0'; }();
     if (off) return 0;
-    // measured (m = 32): the mma.sync kernels win while there is little to read (L = 512, B = 1: 16.5 against 22 us),
-    // these from a few thousand keys up (L = 8192: 58 against 74 us; B = 8, L = 2048: 100 against 131 us)
-    if ((int64_t)a.batch * a.norm_len < 4096) return 0;
+    // measured (m = 32): the mma.sync kernels win while there is little to read (L = 512, B = 1: 16 against 20 us),
+    // these from about two thousand keys up (L = 2048: 23 against 28 us; L = 8192: 38 against 74 us)
+    static const int min_keys = [] { const char* e = getenv("ACACHE_SCORE_TC_MIN_KEYS"); return e ? atoi(e) : 2048; }();
+    if ((int64_t)a.batch * a.norm_len < min_keys) return 0;
     const bool shared = a.kv_batch_stride == 0;
     const int kv_cols = a.n_kv_heads * 128;
     const int ctx_rows = a.norm_lo + a.norm_len > a.affix_start + a.affix_len ? a.norm_lo + a.norm_len : a.affix_start + a.affix_len;
@@ -359,7 +360,8 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
     static bool attr = false;
     if (!attr) {
         cudaFuncSetAttribute(score_stats_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM1);
-        cudaFuncSetAttribute(score_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CS_SMEM);
+        cudaFuncSetAttribute(score_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             2 * 256 * 128 + CS_STAGES * ST_K_BYTES + CS_TABLES + 1024 + 256);
         attr = true;
     }
     ScoreTcArgs t{};
@@ -375,8 +377,9 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
         return -1;
     const int n_pad = (a.m + 31) & ~31;
     const int key_tiles = (a.affix_len + 127) / 128;
+    const int cs_smem = 2 * (n_pad <= 128 ? 128 : 256) * 128 + CS_STAGES * ST_K_BYTES + CS_TABLES + 1024 + 256;
     if (launch_pdl(score_colsum_tc_kernel, dim3(a.n_heads, (key_tiles + kTilesPerCta2 - 1) / kTilesPerCta2, a.batch),
-                   dim3(ST_THREADS), CS_SMEM, stream, t, n_pad, *mq, *mk) != cudaSuccess)
+                   dim3(ST_THREADS), cs_smem, stream, t, n_pad, *mq, *mk) != cudaSuccess)
         return -1;
     return 2;
 }
