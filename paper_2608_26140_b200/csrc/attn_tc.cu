@@ -5,8 +5,8 @@
 //
 //   S = Q K^T    tcgen05.mma 128 x 128 x 16, both operands K-major, into one of two TMEM buffers
 //   softmax      sixteen warps, four threads per query row (32 keys each): scaled max, exp2, running
-//                denominator; P is written as bf16 into a 128-byte-swizzled shared tile
-//   O += P V     tcgen05.mma 128 x 128 x 16, A = P (K-major over keys), B = V read in place as an
+//                denominator; P is written as packed bf16 over the first 64 columns of its S buffer
+//   O += P V     tcgen05.mma 128 x 128 x 16, A = P read from tensor memory, B = V read in place as an
 //                MN-major operand (token-major V rows are contiguous along the head dimension)
 //
 // The S of tile j+1 is issued before the softmax of tile j is consumed, so tensor work overlaps the
@@ -28,7 +28,7 @@ constexpr int AT_THREADS = 608;                  // warp 0: TMA, warp 1: S MMAs,
 constexpr int AT_TILE = 128 * 128 * 2;           // 32 KB: a [128 x 128] bf16 tile as two 64-column panels
 constexpr int AT_PANEL = 128 * 64 * 2;           // 16 KB
 constexpr int AT_SLACK = 256;                    // the dynamic window starts 1024-aligned in practice; checked at run time
-constexpr int AT_SMEM = 7 * AT_TILE + AT_SLACK + 256;   // Q, K x2, V x2, P x2
+constexpr int AT_SMEM = 5 * AT_TILE + AT_SLACK + 256;   // Q, K x2, V x2 (P lives in tensor memory)
 constexpr float kRescaleGap = 8.f;               // log2 units
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar,
@@ -64,6 +64,23 @@ __device__ __forceinline__ float poly_exp2(float x) {
     const float f = x - (t - 12582912.f);
     const float p = fmaf(fmaf(fmaf(0.05517146f, f, 0.24261086f), f, 0.69326097f), f, 0.9999281f);
     return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+// D += A B with A read from tensor memory (rows = TMEM lanes, two bf16 of consecutive K per 32-bit column)
+__device__ __forceinline__ void tc_mma_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -104,12 +121,12 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
         if (threadIdx.x == 0) atomicOr(a.status, kFlagWaitExpired);
         return;
     }
-    const uint32_t sQ = base, sK0 = base + AT_TILE, sV0 = base + 3 * AT_TILE, sP0 = base + 5 * AT_TILE;
-    const uint32_t bars = base + 7 * AT_TILE;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + 7 * AT_TILE + 192);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + 7 * AT_TILE + 200);
-    // barriers: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 v_full | 7,8 v_empty | 9,10 s_full | 11,12 s_empty |
-    //           13,14 p_full | 15,16 p_empty
+    const uint32_t sQ = base, sK0 = base + AT_TILE, sV0 = base + 3 * AT_TILE;
+    const uint32_t bars = base + 5 * AT_TILE;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + 5 * AT_TILE + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + 5 * AT_TILE + 200);
+    // barriers: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 v_full | 7,8 v_empty | 9,10 s_full | 11,12 unused |
+    //           13,14 p_full | 15,16 pv_done (P V of the tile completed: O holds it, its S/P buffer is free)
     auto bar = [&](int i) { return bars + 8 * i; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -120,9 +137,8 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(11), 16); mbar_init(bar(12), 16);    // s_empty: the sixteen softmax warps
-        mbar_init(bar(13), 16); mbar_init(bar(14), 16);    // p_full
-        mbar_init(bar(15), 1); mbar_init(bar(16), 1);      // p_empty
+        mbar_init(bar(13), 16); mbar_init(bar(14), 16);    // p_full: the sixteen softmax warps
+        mbar_init(bar(15), 1); mbar_init(bar(16), 1);      // pv_done
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -175,7 +191,8 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             const int s = j & 1;
             const uint32_t par = (j >> 1) & 1;
             if (!(ok = mbar_wait(bar(1 + s), par, abort_flag))) break;          // K of tile j landed
-            if (!(ok = mbar_wait(bar(11 + s), par ^ 1, abort_flag))) break;     // its S buffer has been read (tile j - 2)
+            // its S buffer also holds the P of tile j - 2: free once that tile's P V has completed
+            if (j >= 2 && !(ok = mbar_wait(bar(15 + s), ((j - 2) >> 1) & 1, abort_flag))) break;
             tc_fence_after();
             const uint32_t k = sK0 + s * AT_TILE;
 #pragma unroll
@@ -199,11 +216,10 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             const uint32_t v = sV0 + s * AT_TILE;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                const uint64_t da = smem_desc_sw128(sP0 + s * AT_TILE + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
                 const uint64_t db = smem_desc_mn_sw128(v + ks * 2048);
-                tc_mma(tO, da, db, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+                tc_mma_ta(tO, tS0 + s * 128 + ks * 8, db, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);   // 16 keys = 8 columns of P
             }
-            tc_commit(bar(15 + s));    // p_empty: this P buffer is free, O holds tiles 0..j
+            tc_commit(bar(15 + s));    // pv_done: O holds tiles 0..j, the S/P buffer is free
             tc_commit(bar(7 + s));     // v_empty
         }
     } else if (warp >= 2 && warp < 18) {
@@ -241,9 +257,6 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
                 tc_fence_after();
                 // this thread's quarter row of S into registers, then the S buffer is free for tile j + 2
                 tc_ld32(tS0 + s * 128 + col_off + lane_off, sv);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(11 + s));   // s_empty
                 float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 if (keep == 0xffffffffu) {
 #pragma unroll
@@ -286,11 +299,9 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
                     if (raise) m_use = mt;
                 }
             }
-            // this P buffer was last read by the P V of tile j - 2
-            if (ok && j >= 2) ok = mbar_wait(bar(15 + s), ((j - 2) >> 1) & 1, abort_flag);
             if (!ok) continue;
-            // 32 keys = four 16-byte chunks of the row, chunks 4 c4 .. 4 c4 + 3 of the 16 in a 128-key tile
-            const uint32_t sP = sP0 + s * AT_TILE + (c4 >> 1) * AT_PANEL + row * 128;
+            // P overwrites the S buffer in tensor memory: 32 keys = 16 columns of two bf16 at column 16 c4
+            // (every thread of the row has read its S columns: they all passed the barrier above)
             float l4[4] = {0.f, 0.f, 0.f, 0.f};
             if (keep == 0xffffffffu) {
 #pragma unroll
@@ -308,24 +319,19 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
                     sv[i] = p;
                 }
             }
+            uint32_t pk[16];
 #pragma unroll
-            for (int k8 = 0; k8 < 4; ++k8) {
-                const int chunk = (c4 & 1) * 4 + k8;              // chunk inside the 64-key panel
-                const uint32_t addr = sP + ((chunk ^ (row & 7)) << 4);
-                const float* pv = sv + k8 * 8;
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(pv[0], pv[1])),
-                             "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])), "r"(pack_bf16(pv[6], pv[7]))
-                             : "memory");
-            }
+            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(sv[2 * i], sv[2 * i + 1]);
+            tc_st16(tS0 + s * 128 + c4 * 16 + lane_off, pk);
+            tc_wait_st();
             l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
             tc_fence_before();
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core's async proxy
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(13 + s));   // p_full
         }
         // epilogue: O / l once the last P V has completed; the denominators of the four quarters add up
         if (ok && n_tiles > 0) ok = mbar_wait(bar(15 + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, abort_flag);
-        float* row_sum = reinterpret_cast<float*>(base_ptr + 5 * AT_TILE);     // the P buffers are idle now
+        float* row_sum = reinterpret_cast<float*>(base_ptr + AT_TILE);         // the K stages are idle now
         row_sum[c4 * 128 + row] = l;
         asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
         if (ok && !*abort_flag) {
@@ -385,30 +391,31 @@ EncodeTiledFn encode_fn3() {
 
 // bf16 [batch, rows, cols] with row stride = cols and the given batch stride (elements);
 // box = 64 cols x 128 rows x 1, 128-byte swizzle, zero fill out of bounds.
-struct Map3Key { const void* ptr; int rows, cols, batch; int64_t bstride; };
+struct Map3Key { const void* ptr; int rows, cols, batch; int64_t bstride; int box_rows; };
 struct Map3Entry { Map3Key key; CUtensorMap map; };
 constexpr int kMap3Cache = 64;
 std::mutex g_map3_mutex;   // guards the cache below; held from the lookups to the launch that uses them
 Map3Entry g_maps3[kMap3Cache];
 int g_map3_count = 0, g_map3_next = 0;
 
-const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int64_t bstride) {
+const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int64_t bstride, int box_rows) {
     for (int i = 0; i < g_map3_count; ++i) {
         const Map3Key& k = g_maps3[i].key;
-        if (k.ptr == ptr && k.rows == rows && k.cols == cols && k.batch == batch && k.bstride == bstride) return &g_maps3[i].map;
+        if (k.ptr == ptr && k.rows == rows && k.cols == cols && k.batch == batch && k.bstride == bstride && k.box_rows == box_rows)
+            return &g_maps3[i].map;
     }
     EncodeTiledFn fn = encode_fn3();
     if (!fn) return nullptr;
     Map3Entry& e = g_maps3[g_map3_next];
     cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
     cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)bstride * 2};
-    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     if (fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return nullptr;
-    e.key = Map3Key{ptr, rows, cols, batch, bstride};
+    e.key = Map3Key{ptr, rows, cols, batch, bstride, box_rows};
     g_map3_next = (g_map3_next + 1) % kMap3Cache;
     if (g_map3_count < kMap3Cache) ++g_map3_count;
     return &e.map;

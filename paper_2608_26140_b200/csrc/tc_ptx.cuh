@@ -119,9 +119,9 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n) {
 
 
 // 3-d tensor maps over bf16 [batch, rows, cols] (row stride = cols, batch stride in elements), box 64 cols x
-// 128 rows x 1, 128-byte swizzle, zero fill out of bounds; cached by (pointer, shape).  Host side, defined in
+// box_rows rows x 1, 128-byte swizzle, zero fill out of bounds; cached by (pointer, shape, box).  Host side, defined in
 // attn_tc.cu; the returned pointer stays valid while g_map3_mutex is held.
-const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int64_t bstride);
+const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int64_t bstride, int box_rows = 128);
 extern std::mutex g_map3_mutex;
 
 }  // namespace acache
