@@ -368,6 +368,304 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
     }
 }
 
+// ---- two query tiles per CTA ------------------------------------------------------------------
+// 256 query rows of one head share every K/V tile that lands in shared memory.  Each 128-row tile has
+// its own S buffer, O accumulator and softmax warps (one thread per row, all 128 keys of the tile in
+// registers: the row maximum needs no exchange).  One thread issues all four products; the P of a tile
+// lives in its S buffer, so a tile's next S is issued right after its P V (the tensor pipe executes one
+// thread's instructions in order) and the two tiles' chains S -> softmax -> P V interleave: while one
+// tile's softmax runs, the tensor pipe works on the other's.
+constexpr int AT2_THREADS = 320;                 // warp 0: TMA, warp 1: MMA issuer, warps 2-5 / 6-9: softmax of tile 0 / 1
+constexpr int AT2_SMEM = 6 * AT_TILE + AT_SLACK + 256;   // Q x2, K x2, V x2
+
+__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, float (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]),
+          "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]), "=f"(v[16]),
+          "=f"(v[17]), "=f"(v[18]), "=f"(v[19]), "=f"(v[20]), "=f"(v[21]), "=f"(v[22]), "=f"(v[23]), "=f"(v[24]),
+          "=f"(v[25]), "=f"(v[26]), "=f"(v[27]), "=f"(v[28]), "=f"(v[29]), "=f"(v[30]), "=f"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+// The loads above are complete after this; the values pass through it so that no use can move ahead of it.
+__device__ __forceinline__ void tc_wait_ld32(float (&v)[32]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]), "+f"(v[8]),
+          "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15]), "+f"(v[16]),
+          "+f"(v[17]), "+f"(v[18]), "+f"(v[19]), "+f"(v[20]), "+f"(v[21]), "+f"(v[22]), "+f"(v[23]), "+f"(v[24]),
+          "+f"(v[25]), "+f"(v[26]), "+f"(v[27]), "+f"(v[28]), "+f"(v[29]), "+f"(v[30]), "+f"(v[31])
+        :
+        : "memory");
+}
+__device__ __forceinline__ void tc_st32u(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+          "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+          "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+
+__global__ void __launch_bounds__(AT2_THREADS, 1)
+attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                      const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapKn,
+                      const __grid_constant__ CUtensorMap mapVn) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    if (base - smem_u32(smem_raw) > (uint32_t)AT_SLACK) {      // the tiles would not fit: report, touch nothing
+        if (threadIdx.x == 0) atomicOr(a.status, kFlagWaitExpired);
+        return;
+    }
+    const uint32_t sQ = base, sK0 = base + 2 * AT_TILE, sV0 = base + 4 * AT_TILE;
+    const uint32_t bars = base + 6 * AT_TILE;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + 6 * AT_TILE + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + 6 * AT_TILE + 200);
+    // barriers: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 v_full | 7,8 v_empty | 9,10 s_full (tile 0, 1) |
+    //           11,12 p_full (tile 0, 1) | 13,14 pv_done (tile 0, 1)
+    auto bar = [&](int i) { return bars + 8 * i; };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int n_cache_tiles = (a.ctx_len + 127) / 128;
+    const int n_tiles = n_cache_tiles + a.n_fresh_tiles;
+    const int kb = a.cache_shared ? 0 : b;
+    const int n_sets = (qt * 256 + 128 < a.n) ? 2 : 1;      // the last CTA of an odd tile count has one tile
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(11), 4); mbar_init(bar(12), 4);      // p_full: the four softmax warps of the tile
+        mbar_init(bar(13), 1); mbar_init(bar(14), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    // columns: S of tile 0 | S of tile 1 | O of tile 0 | O of tile 1, 128 each
+    pdl_wait();
+    pdl_launch_dependents();
+
+    if (warp == 0 && lane == 0) {
+        // ---------------- TMA producer ----------------
+        const uint64_t pol_q = policy_evict_first(), pol_kv = policy_evict_last();
+        mbar_expect_tx(bar(0), n_sets * AT_TILE);
+        for (int t = 0; t < n_sets; ++t) {
+            tma_load_3d(sQ + t * AT_TILE, &mapQ, h * 128, qt * 256 + t * 128, b, bar(0), pol_q);
+            tma_load_3d(sQ + t * AT_TILE + AT_PANEL, &mapQ, h * 128 + 64, qt * 256 + t * 128, b, bar(0), pol_q);
+        }
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int s = j & 1;
+            const uint32_t par = ((j >> 1) & 1) ^ 1;
+            if (!(ok = mbar_wait(bar(3 + s), par, abort_flag))) break;
+            const bool fresh = j >= n_cache_tiles;
+            const CUtensorMap* mk = fresh ? &mapKn : &mapK;
+            const CUtensorMap* mv = fresh ? &mapVn : &mapV;
+            const int r0 = (fresh ? j - n_cache_tiles : j) * 128, bz = fresh ? b : kb;
+            mbar_expect_tx(bar(1 + s), AT_TILE);
+            tma_load_3d(sK0 + s * AT_TILE, mk, kvh * 128, r0, bz, bar(1 + s), pol_kv);
+            tma_load_3d(sK0 + s * AT_TILE + AT_PANEL, mk, kvh * 128 + 64, r0, bz, bar(1 + s), pol_kv);
+            if (!(ok = mbar_wait(bar(7 + s), par, abort_flag))) break;
+            mbar_expect_tx(bar(5 + s), AT_TILE);
+            tma_load_3d(sV0 + s * AT_TILE, mv, kvh * 128, r0, bz, bar(5 + s), pol_kv);
+            tma_load_3d(sV0 + s * AT_TILE + AT_PANEL, mv, kvh * 128 + 64, r0, bz, bar(5 + s), pol_kv);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer ----------------
+        const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        const uint32_t idesc_o = idesc_s | (1u << 16);       // B = V is MN-major
+        auto issue_s = [&](int t, int j) {                   // S_t = Q_t K_j^T, then s_full of tile t
+            const uint32_t k = sK0 + (j & 1) * AT_TILE;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t da = smem_desc_sw128(sQ + t * AT_TILE + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
+                const uint64_t db = smem_desc_sw128(k + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
+                tc_mma(tmem_base + t * 128, da, db, idesc_s, ks > 0 ? 1u : 0u);
+            }
+            tc_commit(bar(9 + t));
+        };
+        bool ok = mbar_wait(bar(0), 0, abort_flag);
+        if (ok && n_tiles > 0 && (ok = mbar_wait(bar(1), 0, abort_flag))) {
+            tc_fence_after();
+            for (int t = 0; t < n_sets; ++t) issue_s(t, 0);
+            tc_commit(bar(3));                               // k_empty of stage 0
+        }
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int s = j & 1;
+            const bool more = j + 1 < n_tiles;
+            if (!(ok = mbar_wait(bar(5 + s), (j >> 1) & 1, abort_flag))) break;             // V of tile j landed
+            if (more && !(ok = mbar_wait(bar(1 + (s ^ 1)), ((j + 1) >> 1) & 1, abort_flag))) break;   // K of tile j + 1 landed
+            const uint32_t v = sV0 + s * AT_TILE;
+            for (int t = 0; t < n_sets && ok; ++t) {
+                if (!(ok = mbar_wait(bar(11 + t), j & 1, abort_flag))) break;               // P_t of tile j written, O_t rescaled
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    tc_mma_ta(tmem_base + 256 + t * 128, tmem_base + t * 128 + ks * 8, smem_desc_mn_sw128(v + ks * 2048), idesc_o,
+                              (j > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(bar(13 + t));                      // pv_done: O_t holds tiles 0..j
+                if (more) issue_s(t, j + 1);                 // overwrites P_t: executes after the P V just issued
+            }
+            tc_commit(bar(7 + s));                           // v_empty
+            if (more) tc_commit(bar(3 + (s ^ 1)));           // k_empty of tile j + 1
+        }
+    } else if (warp >= 2 && warp < 2 + 4 * n_sets) {
+        // ---------------- softmax: one thread per query row ----------------
+        const int t = (warp - 2) >> 2;
+        const int q = warp & 3;                              // the warp's TMEM lane quarter
+        const int row = q * 32 + lane;
+        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+        const uint32_t tS = tmem_base + t * 128 + lane_off, tO = tmem_base + 256 + t * 128 + lane_off;
+        float m_use = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            // which of the tile's 128 keys count: the cache's positions up to the context end, minus those a
+            // fresh row serves; of the fresh rows, those that serve their position
+            uint32_t keep[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (j < n_cache_tiles) {
+                    const int valid = a.ctx_len - j * 128 - c * 32;
+                    keep[c] = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
+                    if (a.n_fresh_tiles && j * 4 + c < a.excl_words) keep[c] &= ~__ldg(a.pos_excl + (int64_t)b * a.excl_words + j * 4 + c);
+                } else {
+                    const int w = (j - n_cache_tiles) * 4 + c;
+                    keep[c] = w < a.keep_words ? __ldg(a.row_keep + (int64_t)b * a.keep_words + w) : 0u;
+                }
+            }
+            const bool all = (keep[0] & keep[1] & keep[2] & keep[3]) == 0xffffffffu;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(9 + t), j & 1, abort_flag)))) break;   // warp-uniform: the TMEM accesses below are collective
+            tc_fence_after();
+            float sv[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tc_ld32_nowait(tS + c * 32, sv[c]);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tc_wait_ld32(sv[c]);
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (all) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], sv[c][i]);
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if ((keep[c] >> i) & 1u) m4[i & 3] = fmaxf(m4[i & 3], sv[c][i]);
+            }
+            const float mt = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * a.scale_log2e;
+            bool raise = false;
+            if (j == 0) {
+                m_use = mt;
+            } else if (mt - m_use > kRescaleGap) {
+                raise = true;
+            }
+            if (__any_sync(0xffffffffu, raise)) {
+                // O may only be touched once the P V of tile j - 1 has completed
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(13 + t), (j - 1) & 1, abort_flag)))) break;
+                tc_fence_after();
+                const float f = raise ? fast_exp2(m_use - mt) : 1.f;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    float v[32];
+                    tc_ld32(tO + c * 32, v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] *= f;
+                    tc_st32(tO + c * 32, v);
+                }
+                tc_wait_st();
+                l *= f;
+                if (raise) m_use = mt;
+            }
+            // P as packed bf16 over the first 64 columns of the S buffer (this thread's own row: all of it is in registers)
+            float l4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t pk[32];
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int c = hf * 2 + cc;
+                    if (all) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float x = fmaf(sv[c][i], a.scale_log2e, -m_use);
+                            const float p = (i & 3) == 3 ? poly_exp2(x) : fast_exp2(x);
+                            l4[i & 3] += p;
+                            sv[c][i] = p;
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float p = ((keep[c] >> i) & 1u) ? fast_exp2(fmaf(sv[c][i], a.scale_log2e, -m_use)) : 0.f;
+                            l4[i & 3] += p;
+                            sv[c][i] = p;
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk[cc * 16 + i] = pack_bf16(sv[c][2 * i], sv[c][2 * i + 1]);
+                }
+                tc_st32u(tS + hf * 32, pk);
+            }
+            tc_wait_st();
+            l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(11 + t));   // p_full
+        }
+        // epilogue: O / l once the last P V has completed
+        if (ok && n_tiles > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(13 + t), (n_tiles - 1) & 1, abort_flag));
+        if (ok) {
+            tc_fence_after();
+            const int grow = qt * 256 + t * 128 + row;
+            const float inv = 1.f / l;
+            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o) + (((int64_t)b * a.n + grow) * a.n_heads + h) * 128;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                float v[32];
+                tc_ld32(tO + c * 32, v);
+                if (grow < a.n) {
+#pragma unroll
+                    for (int k8 = 0; k8 < 4; ++k8) {
+                        const float* pv = v + k8 * 8;
+                        *reinterpret_cast<uint4*>(out + c * 32 + k8 * 8) =
+                            make_uint4(pack_bf16(pv[0] * inv, pv[1] * inv), pack_bf16(pv[2] * inv, pv[3] * inv),
+                                       pack_bf16(pv[4] * inv, pv[5] * inv), pack_bf16(pv[6] * inv, pv[7] * inv));
+                    }
+                }
+            }
+        }
+    }
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) {
+            atomicOr(a.status, kFlagWaitExpired);
+            for (int i = 0; i < 4096; ++i) __nanosleep(64);   // let copies already in flight land
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
 // ---- host side ------------------------------------------------------------------------------
 namespace {
 
@@ -452,6 +750,7 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     static bool attr = false;
     if (!attr) {
         cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM);
+        cudaFuncSetAttribute(attention_tc2q_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT2_SMEM);
         attr = true;
     }
     AttnTcArgs t{};
@@ -463,10 +762,15 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
         t.n_fresh_tiles = q_tiles; t.excl_words = a.excl_words; t.keep_words = a.keep_words;
         t.pos_excl = a.pos_excl; t.row_keep = a.row_keep;
     }
-    if (launch_pdl(attention_tc_kernel, dim3(q_tiles, a.n_heads, a.batch), dim3(AT_THREADS), AT_SMEM, stream, t, *mq, *mk, *mv,
-                   *mkn, *mvn) != cudaSuccess)
-        return -1;
-    return 1;
+    static const bool use_2q = [] { const char* e = getenv("ACACHE_ATTN_TC2Q"); return !e || atoi(e) != 0; }();
+    cudaError_t err;
+    if (use_2q && q_tiles >= 2)
+        err = launch_pdl(attention_tc2q_kernel, dim3((q_tiles + 1) / 2, a.n_heads, a.batch), dim3(AT2_THREADS), AT2_SMEM, stream, t,
+                         *mq, *mk, *mv, *mkn, *mvn);
+    else
+        err = launch_pdl(attention_tc_kernel, dim3(q_tiles, a.n_heads, a.batch), dim3(AT_THREADS), AT_SMEM, stream, t, *mq, *mk,
+                         *mv, *mkn, *mvn);
+    return err == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace acache
