@@ -39,6 +39,9 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy)
         : "memory");
 }
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
 __device__ __forceinline__ void tc_st32(uint32_t taddr, const float (&v)[32]) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -105,6 +108,7 @@ struct AttnTcArgs {
     // the fresh rows [B, n, Hkv, d]; pos_excl masks the cache positions those rows serve, row_keep the fresh
     // rows that do not serve their position (duplicates).  n_fresh_tiles = 0: the cache alone.
     int n_fresh_tiles, excl_words, keep_words, cache_shared;
+    int kv_prefetch;          // two-query-tile kernel: K/V tiles requested into L2 ahead of the rings
     const uint32_t* pos_excl;
     const uint32_t* row_keep;
 };
@@ -369,13 +373,21 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
 }
 
 // ---- two query tiles per CTA ------------------------------------------------------------------
-// 256 query rows of one head share every K/V tile that lands in shared memory.  Each 128-row tile has
-// its own S buffer, O accumulator and softmax warps (one thread per row, all 128 keys of the tile in
-// registers: the row maximum needs no exchange).  One thread issues all four products; the P of a tile
-// lives in its S buffer, so a tile's next S is issued right after its P V (the tensor pipe executes one
-// thread's instructions in order) and the two tiles' chains S -> softmax -> P V interleave: while one
-// tile's softmax runs, the tensor pipe works on the other's.
-constexpr int AT2_THREADS = 320;                 // warp 0: TMA, warp 1: MMA issuer, warps 2-5 / 6-9: softmax of tile 0 / 1
+// 256 query rows of one head share every K/V tile that lands in shared memory.  Each 128-row query tile
+// has its own S buffer, O accumulator and softmax warps (one thread per row: the row maximum needs no
+// exchange).  The softmax works through a tile's 128 keys in two halves of 64 (so that a row's values
+// fit in registers without spilling) and writes each half's P over the low columns of the S buffer; one
+// thread issues everything: the P V of a half as soon as that half's P is there, and after the second
+// half the tile's next S into the same buffer (the tensor pipe executes one thread's instructions in
+// order).  While one query tile's softmax runs, the tensor pipe works on the other's.  Measured and not
+// kept: S as two 64-key products into two buffers per query tile (a 128 x 64 x 16 product holds the
+// issuing thread as long as a 128 x 128 x 16 one: 74 against 66 cycles), and one issuing thread per query
+// tile (their interleaved instructions ran slower than one thread's fixed order).
+//
+// The exponent reference of a row only moves when a half's maximum exceeds it by more than 2^8 (then O
+// and the denominator are rescaled), so the common path is: x = s * scale - reference (two per FFMA2),
+// maximum, exp2 (a quarter of them on the FMA pipe), bf16 pack, store to tensor memory.
+constexpr int AT2_THREADS = 320;                 // warp 0: TMA, warp 1: MMA issuer, warps 2-5 / 6-9: softmax of query tile 0 / 1
 constexpr int AT2_SMEM = 6 * AT_TILE + AT_SLACK + 256;   // Q x2, K x2, V x2
 
 __device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, float (&v)[32]) {
@@ -428,8 +440,8 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
     const uint32_t bars = base + 6 * AT_TILE;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + 6 * AT_TILE + 192);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + 6 * AT_TILE + 200);
-    // barriers: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 v_full | 7,8 v_empty | 9,10 s_full (tile 0, 1) |
-    //           11,12 p_full (tile 0, 1) | 13,14 pv_done (tile 0, 1)
+    // barriers: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 v_full | 7,8 v_empty | 9 + t: s_full |
+    //           11 + 2 t + hb: p_full | 15 + 2 t + hb: pv_done   (query tile t, key half hb)
     auto bar = [&](int i) { return bars + 8 * i; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -441,8 +453,8 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(11), 4); mbar_init(bar(12), 4);      // p_full: the four softmax warps of the tile
-        mbar_init(bar(13), 1); mbar_init(bar(14), 1);
+        for (int i = 11; i <= 14; ++i) mbar_init(bar(i), 4);   // p_full: the four softmax warps of the query tile
+        for (int i = 15; i <= 18; ++i) mbar_init(bar(i), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -455,7 +467,7 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    // columns: S of tile 0 | S of tile 1 | O of tile 0 | O of tile 1, 128 each
+    // columns: S of query tile 0 | S of query tile 1 | O of query tile 0 | O of query tile 1, 128 each
     pdl_wait();
     pdl_launch_dependents();
 
@@ -467,10 +479,23 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
             tma_load_3d(sQ + t * AT_TILE, &mapQ, h * 128, qt * 256 + t * 128, b, bar(0), pol_q);
             tma_load_3d(sQ + t * AT_TILE + AT_PANEL, &mapQ, h * 128 + 64, qt * 256 + t * 128, b, bar(0), pol_q);
         }
+        // K/V tiles a few iterations ahead are requested into L2, so that the loads into the two-stage rings
+        // (issued one iteration before use) do not wait on HBM
+        auto prefetch_tile = [&](int j) {
+            if (j >= n_tiles) return;
+            const bool fresh = j >= n_cache_tiles;
+            const int r0 = (fresh ? j - n_cache_tiles : j) * 128, bz = fresh ? b : kb;
+            tma_prefetch_3d(fresh ? &mapKn : &mapK, kvh * 128, r0, bz);
+            tma_prefetch_3d(fresh ? &mapKn : &mapK, kvh * 128 + 64, r0, bz);
+            tma_prefetch_3d(fresh ? &mapVn : &mapV, kvh * 128, r0, bz);
+            tma_prefetch_3d(fresh ? &mapVn : &mapV, kvh * 128 + 64, r0, bz);
+        };
+        for (int j = 2; j < 2 + a.kv_prefetch; ++j) prefetch_tile(j);
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
             const int s = j & 1;
             const uint32_t par = ((j >> 1) & 1) ^ 1;
+            if (a.kv_prefetch) prefetch_tile(j + 2 + a.kv_prefetch);
             if (!(ok = mbar_wait(bar(3 + s), par, abort_flag))) break;
             const bool fresh = j >= n_cache_tiles;
             const CUtensorMap* mk = fresh ? &mapKn : &mapK;
@@ -488,7 +513,7 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
         // ---------------- MMA issuer ----------------
         const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         const uint32_t idesc_o = idesc_s | (1u << 16);       // B = V is MN-major
-        auto issue_s = [&](int t, int j) {                   // S_t = Q_t K_j^T, then s_full of tile t
+        auto issue_s = [&](int t, int j) {                   // S_t = Q_t K_j^T, then s_full of query tile t
             const uint32_t k = sK0 + (j & 1) * AT_TILE;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
@@ -507,18 +532,22 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
         for (int j = 0; j < n_tiles && ok; ++j) {
             const int s = j & 1;
             const bool more = j + 1 < n_tiles;
-            if (!(ok = mbar_wait(bar(5 + s), (j >> 1) & 1, abort_flag))) break;             // V of tile j landed
+            if (!(ok = mbar_wait(bar(5 + s), (j >> 1) & 1, abort_flag))) break;                       // V of tile j landed
             if (more && !(ok = mbar_wait(bar(1 + (s ^ 1)), ((j + 1) >> 1) & 1, abort_flag))) break;   // K of tile j + 1 landed
             const uint32_t v = sV0 + s * AT_TILE;
             for (int t = 0; t < n_sets && ok; ++t) {
-                if (!(ok = mbar_wait(bar(11 + t), j & 1, abort_flag))) break;               // P_t of tile j written, O_t rescaled
-                tc_fence_after();
+                for (int hb = 0; hb < 2 && ok; ++hb) {
+                    if (!(ok = mbar_wait(bar(11 + 2 * t + hb), j & 1, abort_flag))) break;  // P of this half written, O rescaled
+                    tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    tc_mma_ta(tmem_base + 256 + t * 128, tmem_base + t * 128 + ks * 8, smem_desc_mn_sw128(v + ks * 2048), idesc_o,
-                              (j > 0 || ks > 0) ? 1u : 0u);
-                tc_commit(bar(13 + t));                      // pv_done: O_t holds tiles 0..j
-                if (more) issue_s(t, j + 1);                 // overwrites P_t: executes after the P V just issued
+                    for (int k4 = 0; k4 < 4; ++k4) {
+                        const int ks = hb * 4 + k4;          // 16 keys = 8 columns of P
+                        tc_mma_ta(tmem_base + 256 + t * 128, tmem_base + t * 128 + ks * 8, smem_desc_mn_sw128(v + ks * 2048), idesc_o,
+                                  (j > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    tc_commit(bar(15 + 2 * t + hb));         // pv_done: O holds everything up to this half
+                }
+                if (ok && more) issue_s(t, j + 1);           // overwrites P: executes after the P V just issued
             }
             tc_commit(bar(7 + s));                           // v_empty
             if (more) tc_commit(bar(3 + (s ^ 1)));           // k_empty of tile j + 1
@@ -530,105 +559,124 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
         const int row = q * 32 + lane;
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const uint32_t tS = tmem_base + t * 128 + lane_off, tO = tmem_base + 256 + t * 128 + lane_off;
+        const float2 sc2 = make_float2(a.scale_log2e, a.scale_log2e);
         float m_use = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            // which of the tile's 128 keys count: the cache's positions up to the context end, minus those a
+        for (int i = 0; i < 2 * n_tiles && ok; ++i) {
+            const int hb = i & 1, j = i >> 1;
+            // which of the half's 64 keys count: the cache's positions up to the context end, minus those a
             // fresh row serves; of the fresh rows, those that serve their position
-            uint32_t keep[4];
+            uint32_t keep[2];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
+                const int w = hb * 2 + c;
                 if (j < n_cache_tiles) {
-                    const int valid = a.ctx_len - j * 128 - c * 32;
+                    const int valid = a.ctx_len - j * 128 - w * 32;
                     keep[c] = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
-                    if (a.n_fresh_tiles && j * 4 + c < a.excl_words) keep[c] &= ~__ldg(a.pos_excl + (int64_t)b * a.excl_words + j * 4 + c);
+                    if (a.n_fresh_tiles && j * 4 + w < a.excl_words) keep[c] &= ~__ldg(a.pos_excl + (int64_t)b * a.excl_words + j * 4 + w);
                 } else {
-                    const int w = (j - n_cache_tiles) * 4 + c;
-                    keep[c] = w < a.keep_words ? __ldg(a.row_keep + (int64_t)b * a.keep_words + w) : 0u;
+                    const int fw = (j - n_cache_tiles) * 4 + w;
+                    keep[c] = fw < a.keep_words ? __ldg(a.row_keep + (int64_t)b * a.keep_words + fw) : 0u;
                 }
             }
-            const bool all = (keep[0] & keep[1] & keep[2] & keep[3]) == 0xffffffffu;
-            if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(9 + t), j & 1, abort_flag)))) break;   // warp-uniform: the TMEM accesses below are collective
-            tc_fence_after();
-            float sv[4][32];
+            const bool all = (keep[0] & keep[1]) == 0xffffffffu;
+            // warp-uniform: the tensor-memory accesses below are collective
+            if (hb == 0) {
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(9 + t), j & 1, abort_flag)))) break;
+                tc_fence_after();
+            }
+            float sv[2][32];
+            tc_ld32_nowait(tS + hb * 64, sv[0]);
+            tc_ld32_nowait(tS + hb * 64 + 32, sv[1]);
+            tc_wait_ld32(sv[0]);
+            tc_wait_ld32(sv[1]);
+            // x = s * scale - reference, in place; the reference is 0 until a half with a key that counts
+            const bool first = m_use == -INFINITY;
+            const float m_ref = first ? 0.f : m_use;
+            const float2 mr2 = make_float2(-m_ref, -m_ref);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tc_ld32_nowait(tS + c * 32, sv[c]);
+            for (int c = 0; c < 2; ++c)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tc_wait_ld32(sv[c]);
+                for (int e = 0; e < 16; ++e) {
+                    const float2 r = __ffma2_rn(make_float2(sv[c][2 * e], sv[c][2 * e + 1]), sc2, mr2);
+                    sv[c][2 * e] = r.x;
+                    sv[c][2 * e + 1] = r.y;
+                }
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             if (all) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], sv[c][i]);
+                    for (int e = 0; e < 32; ++e) m4[e & 3] = fmaxf(m4[e & 3], sv[c][e]);
             } else {
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if ((keep[c] >> i) & 1u) m4[i & 3] = fmaxf(m4[i & 3], sv[c][i]);
+                    for (int e = 0; e < 32; ++e)
+                        if ((keep[c] >> e) & 1u) m4[e & 3] = fmaxf(m4[e & 3], sv[c][e]);
             }
-            const float mt = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * a.scale_log2e;
-            bool raise = false;
-            if (j == 0) {
-                m_use = mt;
-            } else if (mt - m_use > kRescaleGap) {
-                raise = true;
-            }
+            const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+            const bool raise = mx > kRescaleGap || (first && mx > -INFINITY);
             if (__any_sync(0xffffffffu, raise)) {
-                // O may only be touched once the P V of tile j - 1 has completed
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(13 + t), (j - 1) & 1, abort_flag)))) break;
-                tc_fence_after();
-                const float f = raise ? fast_exp2(m_use - mt) : 1.f;
+                const float f = raise ? (first ? 0.f : fast_exp2(-mx)) : 1.f;
+                if (i > 0) {
+                    // O may only be touched once the P V of half i - 1 (and with it every earlier one) has completed
+                    if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(15 + 2 * t + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abort_flag)))) break;
+                    tc_fence_after();
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    float v[32];
-                    tc_ld32(tO + c * 32, v);
+                    for (int c = 0; c < 4; ++c) {
+                        float v[32];
+                        tc_ld32(tO + c * 32, v);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] *= f;
-                    tc_st32(tO + c * 32, v);
-                }
-                tc_wait_st();
-                l *= f;
-                if (raise) m_use = mt;
-            }
-            // P as packed bf16 over the first 64 columns of the S buffer (this thread's own row: all of it is in registers)
-            float l4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                uint32_t pk[32];
-#pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    const int c = hf * 2 + cc;
-                    if (all) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const float x = fmaf(sv[c][i], a.scale_log2e, -m_use);
-                            const float p = (i & 3) == 3 ? poly_exp2(x) : fast_exp2(x);
-                            l4[i & 3] += p;
-                            sv[c][i] = p;
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const float p = ((keep[c] >> i) & 1u) ? fast_exp2(fmaf(sv[c][i], a.scale_log2e, -m_use)) : 0.f;
-                            l4[i & 3] += p;
-                            sv[c][i] = p;
-                        }
+                        for (int e = 0; e < 32; ++e) v[e] *= f;
+                        tc_st32(tO + c * 32, v);
                     }
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) pk[cc * 16 + i] = pack_bf16(sv[c][2 * i], sv[c][2 * i + 1]);
+                    tc_wait_st();
                 }
-                tc_st32u(tS + hf * 32, pk);
+                l *= f;
+                if (raise) {
+                    m_use = m_ref + mx;
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) sv[c][e] -= mx;
+                }
             }
+            // P as packed bf16: the half's 64 keys go to columns 32 hb .. 32 hb + 31 of the S buffer, over S values of
+            // keys below 64 that this thread read in the first half
+            float2 l2a = make_float2(0.f, 0.f), l2b = make_float2(0.f, 0.f);
+            uint32_t pk[32];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                if (all) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        const float2 pa = make_float2(fast_exp2(sv[c][e]), fast_exp2(sv[c][e + 1]));
+                        const float2 pb = make_float2(fast_exp2(sv[c][e + 2]), poly_exp2(sv[c][e + 3]));
+                        l2a = __fadd2_rn(l2a, pa);
+                        l2b = __fadd2_rn(l2b, pb);
+                        pk[c * 16 + (e >> 1)] = pack_bf16(pa.x, pa.y);
+                        pk[c * 16 + (e >> 1) + 1] = pack_bf16(pb.x, pb.y);
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const float p0 = ((keep[c] >> e) & 1u) ? fast_exp2(sv[c][e]) : 0.f;
+                        const float p1 = ((keep[c] >> (e + 1)) & 1u) ? fast_exp2(sv[c][e + 1]) : 0.f;
+                        l2a = __fadd2_rn(l2a, make_float2(p0, p1));
+                        pk[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
+                    }
+                }
+            }
+            tc_st32u(tS + hb * 32, pk);
             tc_wait_st();
-            l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+            l += (l2a.x + l2a.y) + (l2b.x + l2b.y);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(11 + t));   // p_full
+            if (lane == 0) mbar_arrive(bar(11 + 2 * t + hb));   // p_full
         }
         // epilogue: O / l once the last P V has completed
-        if (ok && n_tiles > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(13 + t), (n_tiles - 1) & 1, abort_flag));
+        if (ok && n_tiles > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(15 + 2 * t + 1), (n_tiles - 1) & 1, abort_flag));
         if (ok) {
             tc_fence_after();
             const int grow = qt * 256 + t * 128 + row;
@@ -762,6 +810,8 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
         t.n_fresh_tiles = q_tiles; t.excl_words = a.excl_words; t.keep_words = a.keep_words;
         t.pos_excl = a.pos_excl; t.row_keep = a.row_keep;
     }
+    static const int kv_prefetch = [] { const char* e = getenv("ACACHE_ATTN_KV_PREFETCH"); return e ? atoi(e) : 2; }();
+    t.kv_prefetch = kv_prefetch;
     static const bool use_2q = [] { const char* e = getenv("ACACHE_ATTN_TC2Q"); return !e || atoi(e) != 0; }();
     cudaError_t err;
     if (use_2q && q_tiles >= 2)
