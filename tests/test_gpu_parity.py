@@ -348,19 +348,20 @@ def test_llada_layer_full_size(extra):
 
 
 # ------------------------------------------------------------------ shared affix storage (Section 4.1)
-def test_shared_affix_cache_with_private_rows():
+@pytest.mark.parametrize("L,ratio", [(160, 0.2), (400, 0.7)])    # 88 rows: one query tile; 336 rows: three (two per CTA + one)
+def test_shared_affix_cache_with_private_rows(L, ratio):
     """One copy of the affix K/V (batch_stride = 0) serves three requests: scoring reads it, the
     refresh writes each request's anchors and request rows to its private k_new / v_new and its
     attention reads all other positions from the shared copy, which stays untouched."""
     shape, B = MID128, 3
-    lay = wl.make_layout(B, 0, 160, 24, 32, 32, "all")
-    case = wl.make_case(shape, lay, 0.2, cfg_id=19)
+    lay = wl.make_layout(B, 0, L, 24, 32, 32, "all")
+    case = wl.make_case(shape, lay, ratio, cfg_id=19)
     T, L = lay.ctx_len, lay.affix_len
     shared_k, shared_v = case.cache_k[0].copy(), case.cache_v[0].copy()      # [T, Hkv, d]; only affix rows matter
     dc = DeviceCase(case)
     dsk, dsv = ab.to_device_bf16(shared_k[None], DEV), ab.to_device_bf16(shared_v[None], DEV)
     kv = ab.KV(dsk.data_ptr(), dsv.data_ptr(), 0, T)
-    K = orc.k_from_ratio(L, 0.2)
+    K = orc.k_from_ratio(L, ratio)
     n = K + lay.n_extra
     # scores from masked-row queries computed by the oracle (any queries would do)
     q = wl.random_q_mask(shape, lay, 91)
@@ -394,7 +395,7 @@ def test_shared_affix_cache_with_private_rows():
     with pytest.raises(ab.AcacheError):
         dc.ctx.scatter_kv(dc.req, kv, anchors, K, k_new, v_new)
     with pytest.raises(ab.AcacheError):
-        dc.ctx.layer_step(dc.lw, dc.req, kv, dc.x, 0, 0.2, 0, None, anchors, y)
+        dc.ctx.layer_step(dc.lw, dc.req, kv, dc.x, 0, ratio, 0, None, anchors, y)
 
 
 def test_duplicate_row_is_served_once_in_the_split_calls():
