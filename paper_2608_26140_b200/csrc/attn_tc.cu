@@ -1,15 +1,18 @@
 // Bidirectional attention of many recomputed rows over the whole context (Section 4.3) on the
-// 5th-generation tensor cores.  One CTA = 128 query rows of one head; key/value tiles of 128
-// keys stream through shared memory by TMA (3-d tensor maps: positions past the context end and
-// rows past the request's row count read as zero).
+// 5th-generation tensor cores.  Two kernels share the scheme below: attention_tc_kernel (one CTA = 128
+// query rows of one head; used when a request has at most 128 rows) and attention_tc2q_kernel (one CTA
+// = 256 query rows, described where it is defined).  Key/value tiles of 128 keys stream through shared
+// memory by TMA (3-d tensor maps: positions past the context end and rows past the request's row count
+// read as zero).
 //
-//   S = Q K^T    tcgen05.mma 128 x 128 x 16, both operands K-major, into one of two TMEM buffers
-//   softmax      sixteen warps, four threads per query row (32 keys each): scaled max, exp2, running
-//                denominator; P is written as packed bf16 over the first 64 columns of its S buffer
+//   S = Q K^T    tcgen05.mma 128 x 128 x 16, both operands K-major, into a TMEM buffer
+//   softmax      scaled max, exp2, running denominator; P is written as packed bf16 over the low
+//                columns of its S buffer, so it never passes through shared memory
 //   O += P V     tcgen05.mma 128 x 128 x 16, A = P read from tensor memory, B = V read in place as an
 //                MN-major operand (token-major V rows are contiguous along the head dimension)
 //
-// The S of tile j+1 is issued before the softmax of tile j is consumed, so tensor work overlaps the
+// One-tile kernel: sixteen softmax warps, four threads per query row (32 keys each), two S buffers: the
+// S of tile j+1 is issued before the softmax of tile j is consumed, so tensor work overlaps the
 // exponentials.  The running maximum used for the exponent is only raised (and O rescaled in
 // TMEM) when the true maximum has grown by more than 2^8, which keeps P within bf16 range and
 // makes rescales rare.  Every mbarrier wait is bounded (status flag kFlagWaitExpired on expiry).
@@ -138,10 +141,13 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
     const int n_cache_tiles = (a.ctx_len + 127) / 128;
     const int n_tiles = n_cache_tiles + a.n_fresh_tiles;
     const int kb = a.cache_shared ? 0 : b;          // one cache for the whole batch, or one per request
+    // 32-row quarters of the tile that hold rows of the request: the softmax warps of the others have nothing
+    // to do (their rows of S, P and O are never read), which matters when a decode pass brings 32 rows
+    const int live_q = min(4, (a.n - qt * 128 + 31) / 32);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(13), 16); mbar_init(bar(14), 16);    // p_full: the sixteen softmax warps
+        mbar_init(bar(13), 4 * live_q); mbar_init(bar(14), 4 * live_q);    // p_full: the softmax warps that have rows
         mbar_init(bar(15), 1); mbar_init(bar(16), 1);      // pv_done
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -226,7 +232,7 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             tc_commit(bar(15 + s));    // pv_done: O holds tiles 0..j, the S/P buffer is free
             tc_commit(bar(7 + s));     // v_empty
         }
-    } else if (warp >= 2 && warp < 18) {
+    } else if (warp >= 2 && warp < 18 && (warp & 3) < live_q) {
         // ---------------- softmax: four threads per query row ----------------
         // Warp 2 + 4 c + q' (q = warp & 3 is its TMEM lane quarter) takes keys [32 c, 32 c + 32) of every
         // tile for the 32 rows of quarter q, and columns [32 c, 32 c + 32) of O.  Sixteen warps (four per
@@ -453,7 +459,8 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
-        for (int i = 11; i <= 14; ++i) mbar_init(bar(i), 4);   // p_full: the four softmax warps of the query tile
+        for (int i = 11; i <= 14; ++i)                         // p_full: the softmax warps of the query tile that have rows
+            mbar_init(bar(i), max(1, min(4, (a.n - qt * 256 - (i >= 13 ? 128 : 0) + 31) / 32)));
         for (int i = 15; i <= 18; ++i) mbar_init(bar(i), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -552,7 +559,7 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
             tc_commit(bar(7 + s));                           // v_empty
             if (more) tc_commit(bar(3 + (s ^ 1)));           // k_empty of tile j + 1
         }
-    } else if (warp >= 2 && warp < 2 + 4 * n_sets) {
+    } else if (warp >= 2 && warp < 2 + 4 * n_sets && (warp & 3) * 32 < a.n - qt * 256 - ((warp - 2) >> 2) * 128) {
         // ---------------- softmax: one thread per query row ----------------
         const int t = (warp - 2) >> 2;
         const int q = warp & 3;                              // the warp's TMEM lane quarter
@@ -812,7 +819,13 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     }
     static const int kv_prefetch = [] { const char* e = getenv("ACACHE_ATTN_KV_PREFETCH"); return e ? atoi(e) : 2; }();
     t.kv_prefetch = kv_prefetch;
-    static const bool use_2q = [] { const char* e = getenv("ACACHE_ATTN_TC2Q"); return !e || atoi(e) != 0; }();
+    // Two query tiles per CTA pay off when the halved grid still fills the SMs and the context is short enough
+    // for the per-CTA prologue and epilogue to matter (measured, one against the other: 2048-2560 keys with
+    // 1000+ rows, 8-15 % faster; 8192 keys, 5-10 % slower; fewer CTAs than SMs, up to 1.8x slower).
+    // ACACHE_ATTN_TC2Q = 0: never, 2: whenever there are two tiles.
+    static const int mode_2q = [] { const char* e = getenv("ACACHE_ATTN_TC2Q"); return e ? atoi(e) : 1; }();
+    const bool use_2q = mode_2q == 2 || (mode_2q == 1 && a.ctx_len + (two_src ? a.n : 0) <= 4096 &&
+                                         (int64_t)((q_tiles + 1) / 2) * a.n_heads * a.batch >= 148);
     cudaError_t err;
     if (use_2q && q_tiles >= 2)
         err = launch_pdl(attention_tc2q_kernel, dim3((q_tiles + 1) / 2, a.n_heads, a.batch), dim3(AT2_THREADS), AT2_SMEM, stream, t,
