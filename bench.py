@@ -655,8 +655,20 @@ def run_generate(args, e):
     rows_d = torch.arange(n_blk, dtype=torch.int32, device=dev).repeat(B, 1).contiguous()
     left = torch.zeros((B,), dtype=torch.int32, device=dev)
 
+    shared = bool(args.shared)
+    if shared:
+        # one copy of every layer's cache serves the batch (batch_stride 0); what a request changes lives in its
+        # private slots [B, K + e, Hkv, d] per layer
+        kvs_sh = [ab.KV(e["dk"][i][0:1].data_ptr(), e["dv"][i][0:1].data_ptr(), 0, T) for i in range(n_layers)]
+        ks = [torch.zeros((B, n, shape.n_kv_heads, shape.head_dim), dtype=torch.bfloat16, device=dev) for _ in range(n_layers)]
+        vs = [torch.zeros_like(t) for t in ks]
+
     def block():
         dids.copy_(ids0)
+        if shared:
+            return ctx.generate_block_shared(e["lws"], kvs_sh, e["req"], req_d, e["embed"], e["da"], K, ks, vs, e["ya"], e["yb"],
+                                             e["dbr"], rows_d, n_blk, e["gain"], e["w_lm"], V, 0.9, V - 1, n_blk + 1,
+                                             e["token"], e["conf"], e["commit"], left)
         return ctx.generate_block(e["lws"], e["kvs"], e["req"], req_d, e["embed"], e["da"], K, e["ya"], e["yb"], e["dbr"], rows_d,
                                   n_blk, e["gain"], e["w_lm"], V, 0.9, V - 1, n_blk + 1, e["token"], e["conf"], e["commit"], left)
 
@@ -698,7 +710,10 @@ def run_generate(args, e):
         "data": "synthetic; random-init weights: no confidence reaches the threshold, so each pass commits one token per request",
         "config": {"workload": f"cfg3 block decode: LLaDA-8B shapes, {n_layers} layers, vocab {V}, batch {B}/GPU sharing a {L}-token "
                                f"prefix affix, one {n_blk}-token block per request: 1 refresh pass ({n} rows per request, K={K}) + "
-                               f"decode passes over the block's {n_blk} rows", "benchmark_config": 3, "layers": n_layers,
+                               f"decode passes over the block's {n_blk} rows; "
+                               + ("shared affix storage: one cache per layer for the batch + private slots"
+                                  if shared else "one working cache per request and layer"),
+                   "benchmark_config": 3, "layers": n_layers, "storage": "shared" if shared else "private",
                    "model_passes_per_block": passes / n_blocks, "parallelism": f"request-sharded x{world}"},
         "clocks": sampler.summary(), "gpu_launches": int(launches), "ms_per_block": ms_block,
         "ms_per_model_pass": ms_block / (passes / n_blocks),
@@ -834,14 +849,15 @@ def main():
     ap.add_argument("--shared", action="store_true",
                     help="--config 3 or 4: one layer with shared affix storage (batch_stride 0) against private caches")
     ap.add_argument("--generate", action="store_true",
-                    help="--config 3: decode one whole 32-token block per request (refresh + decode passes)")
+                    help="--config 3: decode one whole 32-token block per request (refresh + decode passes); "
+                         "with --shared over shared affix storage")
     ap.add_argument("--sweep-affix", default=None, help="--config 5: comma-separated affix lengths (default 512,2048,8192)")
     ap.add_argument("--sweep-batch", default=None, help="--config 5: comma-separated batch sizes (default 1,8,64)")
     ap.add_argument("--sweep-out", default=None, help="--config 5: also write the points as a markdown table to this file")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    elif args.shared and args.config in (3, 4):
+    elif args.shared and args.config in (3, 4) and not args.generate:
         run_shared(args)
     elif args.config == 3:
         run_denoise(args)

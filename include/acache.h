@@ -299,6 +299,56 @@ acache_status acache_denoise_step_shared(acache_ctx *ctx, int32_t n_layers, cons
                                          const void *w_lm, int32_t vocab, float threshold, int32_t *token,
                                          float *confidence, int32_t *commit, acache_stream_t stream);
 
+/* A decode pass over shared affix storage (Section 4.1 storage under the Section 4.3 schedule): after a
+ * refresh pass (acache_recompute_anchors / acache_denoise_step_shared with kv->batch_stride = 0) has
+ * filled the private slot arrays k_slots / v_slots [B, k + e_slots, Hkv, d] with the anchors and the
+ * request-specific rows of req_slots, this call recomputes only the rows req_rows->extra_rows (n_extra
+ * per request: the block being decoded) through one layer.  Their fresh K/V overwrite slot rows
+ * slot_rows[b, i] (the index of row i's position inside the slot array: k + its index in
+ * req_slots->extra_rows); their attention reads every other position from the shared cache, except
+ * those a slot row serves, which come from the slots (the read-slot map of Section 4.1).
+ *   req_rows, req_slots: same batch, ctx_len, affix span and rope tables; req_slots, anchor_idx and k as
+ *   given to the refresh pass.  x, x_is_compact: as acache_recompute_anchors, for the rows of req_rows.
+ *   slot_rows: DEVICE int32 [B, n_extra]; a value outside [0, k + e_slots) raises
+ *   ACACHE_FLAG_BAD_INDEX and that row's K/V is not stored.  A position that appears twice in the slot
+ *   array is served by its last row; slot_rows must name that one.
+ *   k_slots, v_slots: DEVICE bf16, updated in place.  y: DEVICE bf16 [B, n_extra, D].
+ * The shared cache is not written. */
+acache_status acache_recompute_rows_shared(acache_ctx *ctx, const acache_layer_weights *w,
+                                           const acache_request *req_rows, const acache_request *req_slots,
+                                           const acache_kv *kv, const void *x, int x_is_compact,
+                                           const int32_t *anchor_idx, int32_t k, const int32_t *slot_rows,
+                                           void *k_slots, void *v_slots, void *y, acache_stream_t stream);
+
+/* n_layers of acache_recompute_rows_shared chained (layer n reads kvs[n], k_slots[n], v_slots[n]; HOST
+ * arrays of DEVICE pointers), then Eq. 2-3 on the rows block_rows of the last layer's output, as
+ * acache_denoise_step_shared does for the refresh pass.  y_a, y_b: DEVICE bf16 [B, n_extra, D]. */
+acache_status acache_decode_step_shared(acache_ctx *ctx, int32_t n_layers, const acache_layer_weights *layers,
+                                        const acache_kv *kvs, const acache_request *req_rows,
+                                        const acache_request *req_slots, const void *x0,
+                                        const int32_t *anchor_idx, int32_t k, const int32_t *slot_rows,
+                                        void *const *k_slots, void *const *v_slots, void *y_a, void *y_b,
+                                        void **y_last, const int32_t *block_rows, int32_t n_blk,
+                                        const void *final_norm_g, const void *w_lm, int32_t vocab, float threshold,
+                                        int32_t *token, float *confidence, int32_t *commit, acache_stream_t stream);
+
+/* acache_generate_block over shared affix storage: step 0 is acache_denoise_step_shared over
+ * R = A u E (req_refresh), which fills the private slots; every later step is
+ * acache_decode_step_shared over the block's rows (req_decode) with slot_rows = block_rows_refresh.
+ * The shared caches kvs[n] (batch_stride 0) are never written; everything a request changes lives in
+ * its slots.  Other arguments, the commit rule and the one synchronisation per step as
+ * acache_generate_block. */
+acache_status acache_generate_block_shared(acache_ctx *ctx, int32_t n_layers, const acache_layer_weights *layers,
+                                           const acache_kv *kvs, const acache_request *req_refresh,
+                                           const acache_request *req_decode, const void *embed,
+                                           const int32_t *anchor_idx, int32_t k, void *const *k_slots,
+                                           void *const *v_slots, void *y_a, void *y_b,
+                                           const int32_t *block_rows_refresh, const int32_t *block_rows_decode,
+                                           int32_t n_blk, const void *final_norm_g, const void *w_lm, int32_t vocab,
+                                           float threshold, int32_t mask_id, int32_t max_steps, int32_t *token,
+                                           float *confidence, int32_t *commit, int32_t *remaining,
+                                           int32_t *steps_done, acache_stream_t stream);
+
 /* The one-shot probe and the selection it feeds (Section 3.2): every request's request-specific rows
  * (req->extra_rows = all non-affix positions, which must include the masked ones) go through the
  * n_layers layers with the affix K/V as cached; at every layer the masked rows' queries are scored

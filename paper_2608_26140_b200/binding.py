@@ -23,7 +23,8 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_k_from_ratio", "acache_select_topk", "acache_recompute_anchors", "acache_scatter_kv",
            "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times",
            "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step", "acache_probe_select",
-           "acache_commit_update", "acache_generate_block", "acache_denoise_step_shared"]
+           "acache_commit_update", "acache_generate_block", "acache_denoise_step_shared", "acache_recompute_rows_shared",
+           "acache_decode_step_shared", "acache_generate_block_shared"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -124,6 +125,17 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
                                           C.POINTER(Request), vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, i32, C.c_float,
                                           i32, i32, vp, vp, vp, vp, C.POINTER(i32), vp]
     lib.acache_generate_block.restype = C.c_int
+    lib.acache_recompute_rows_shared.argtypes = [vp, C.POINTER(LayerWeights), C.POINTER(Request), C.POINTER(Request),
+                                                 C.POINTER(KV), vp, C.c_int, vp, i32, vp, vp, vp, vp, vp]
+    lib.acache_recompute_rows_shared.restype = C.c_int
+    lib.acache_decode_step_shared.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request),
+                                              C.POINTER(Request), vp, vp, i32, vp, C.POINTER(vp), C.POINTER(vp), vp, vp,
+                                              C.POINTER(vp), vp, i32, vp, vp, i32, C.c_float, vp, vp, vp, vp]
+    lib.acache_decode_step_shared.restype = C.c_int
+    lib.acache_generate_block_shared.argtypes = [vp, i32, C.POINTER(LayerWeights), C.POINTER(KV), C.POINTER(Request),
+                                                 C.POINTER(Request), vp, vp, i32, C.POINTER(vp), C.POINTER(vp), vp, vp, vp, vp,
+                                                 i32, vp, vp, i32, C.c_float, i32, i32, vp, vp, vp, vp, C.POINTER(i32), vp]
+    lib.acache_generate_block_shared.restype = C.c_int
     lib.acache_stage_timing.argtypes = [vp, C.c_int]
     lib.acache_stage_timing.restype = C.c_int
     lib.acache_read_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
@@ -300,6 +312,47 @@ class Context:
                                                         _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold), _ptr(token),
                                                         _ptr(confidence), _ptr(commit), _stream()))
         return last.value
+
+    def recompute_rows_shared(self, w: LayerWeights, req_rows: Request, req_slots: Request, kv: KV, x, x_is_compact,
+                              anchor_idx, k, slot_rows, k_slots, v_slots, y):
+        self._check(self.lib.acache_recompute_rows_shared(self.h, C.byref(w), C.byref(req_rows), C.byref(req_slots),
+                                                          C.byref(kv), _ptr(x), int(x_is_compact), _ptr(anchor_idx), k,
+                                                          _ptr(slot_rows), _ptr(k_slots), _ptr(v_slots), _ptr(y), _stream()))
+
+    def decode_step_shared(self, layers, kvs, req_rows: Request, req_slots: Request, x0, anchor_idx, k, slot_rows, k_slots,
+                           v_slots, y_a, y_b, block_rows, n_blk, final_norm_g, w_lm, vocab, threshold, token, confidence,
+                           commit) -> int:
+        """k_slots, v_slots: lists of per-layer tensors [B, K+e, Hkv, d] as the refresh pass left them."""
+        n = len(layers)
+        la = (LayerWeights * n)(*layers)
+        ka = (KV * n)(*kvs)
+        kn = (C.c_void_p * n)(*[_ptr(t) for t in k_slots])
+        vn = (C.c_void_p * n)(*[_ptr(t) for t in v_slots])
+        last = C.c_void_p()
+        self._check(self.lib.acache_decode_step_shared(self.h, n, la, ka, C.byref(req_rows), C.byref(req_slots), _ptr(x0),
+                                                       _ptr(anchor_idx), k, _ptr(slot_rows), kn, vn, _ptr(y_a), _ptr(y_b),
+                                                       C.byref(last), _ptr(block_rows), n_blk, _ptr(final_norm_g), _ptr(w_lm),
+                                                       vocab, float(threshold), _ptr(token), _ptr(confidence), _ptr(commit),
+                                                       _stream()))
+        return last.value
+
+    def generate_block_shared(self, layers, kvs, req_refresh: Request, req_decode: Request, embed, anchor_idx, k, k_slots,
+                              v_slots, y_a, y_b, block_rows_refresh, block_rows_decode, n_blk, final_norm_g, w_lm, vocab,
+                              threshold, mask_id, max_steps, token, confidence, commit, remaining) -> int:
+        """acache_generate_block over shared affix storage; returns the number of model passes run."""
+        n = len(layers)
+        la = (LayerWeights * n)(*layers)
+        ka = (KV * n)(*kvs)
+        kn = (C.c_void_p * n)(*[_ptr(t) for t in k_slots])
+        vn = (C.c_void_p * n)(*[_ptr(t) for t in v_slots])
+        steps = C.c_int32(0)
+        self._check(self.lib.acache_generate_block_shared(self.h, n, la, ka, C.byref(req_refresh), C.byref(req_decode),
+                                                          _ptr(embed), _ptr(anchor_idx), k, kn, vn, _ptr(y_a), _ptr(y_b),
+                                                          _ptr(block_rows_refresh), _ptr(block_rows_decode), n_blk,
+                                                          _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold),
+                                                          int(mask_id), int(max_steps), _ptr(token), _ptr(confidence),
+                                                          _ptr(commit), _ptr(remaining), C.byref(steps), _stream()))
+        return int(steps.value)
 
     def probe_select(self, layers, kvs, req: Request, x0, ratio, flags, y_a, y_b, scores, anchor_idx):
         n = len(layers)

@@ -20,7 +20,7 @@ struct acache_ctx {
     unsigned char* ws = nullptr;
     size_t ws_have = 0;
     // workspace offsets (bytes)
-    size_t o_status, o_row_pos, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
+    size_t o_status, o_row_pos, o_row_pos2, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
     size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
     size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar, o_mcidx, o_lstats, o_lxn, o_keymask;
     std::string err;
@@ -136,9 +136,21 @@ acache_status run_score(acache_ctx* c, const acache_request* r, const void* q_ma
 
 // The recompute of rows R.  fused_cache != null: K/V go straight into the cache and
 // attention reads it; otherwise K/V go to k_new/v_new and attention reads through a slot map.
+// The private slot array a decode pass over shared storage works against: k anchors and e extra rows per
+// request as an earlier refresh pass over the same storage wrote them; out_rows[b, i] = the slot row that
+// holds row i of the rows recomputed now.
+struct PrivateRows {
+    const int32_t* anchor_idx;
+    int k;
+    const int32_t* extra_rows;
+    int e;
+    const int32_t* out_rows;
+};
+
 acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const acache_request* r,
                             const acache_kv* kv, bool fuse_scatter, const void* x, int x_is_compact,
-                            const int32_t* anchor_idx, int k, void* k_new, void* v_new, void* y, cudaStream_t st) {
+                            const int32_t* anchor_idx, int k, void* k_new, void* v_new, void* y, cudaStream_t st,
+                            const PrivateRows* priv = nullptr) {
     const acache_model_desc& d = c->d;
     const int rows = k + r->n_extra, n = r->batch * rows;
     if (n == 0) {
@@ -179,6 +191,7 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     g.out[0] = q; g.out[1] = k_new; g.out[2] = v_new;
     if (fuse_scatter) { g.cache_k = kv->k; g.cache_v = kv->v; }
     g.kv_batch_stride = kv->batch_stride; g.rows_per_req = rows;
+    if (priv) { g.kv_out_rows = priv->out_rows; g.kv_out_stride = priv->k + priv->e; }
     g.partial = partial; g.status = status; g.grid_bar = grid_bar;
     { int nl = launch_gemm(g, st); if (nl < 0) return check_cuda(c, "qkv projection") == ACACHE_OK ? fail(c, ACACHE_ERR_CUDA, "qkv projection launch failed") : ACACHE_ERR_CUDA;
     c->launches += nl; }
@@ -187,15 +200,27 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     AttnArgs at{};
     at.q = q; at.cache_k = kv->k; at.cache_v = kv->v; at.kv_batch_stride = kv->batch_stride;
     if (!fuse_scatter) {
+        // the rows that serve their positions from k_new / v_new: the rows recomputed now, or the whole private
+        // slot array of which they refreshed a part
+        const int fresh = priv ? priv->k + priv->e : rows;
+        const int32_t* fresh_pos = row_pos;
+        if (priv) {
+            int32_t* rp2 = wsp<int32_t>(c, c->o_row_pos2);
+            launch_row_positions(priv->anchor_idx, priv->k, priv->extra_rows, priv->e, r->affix_start, r->affix_len, r->ctx_len,
+                                 r->batch, rp2, status, st);
+            c->launches += 1;
+            fresh_pos = rp2;
+            at.n_fresh = fresh;
+        }
         int32_t* slot = wsp<int32_t>(c, c->o_slot);
-        launch_build_slot_map(slot, r->ctx_len, row_pos, rows, r->batch, st);
+        launch_build_slot_map(slot, r->ctx_len, fresh_pos, fresh, r->batch, st);
         c->launches += 1;
         at.k_new = k_new; at.v_new = v_new; at.slot = slot;
         // key masks of the same map, for the kernel that reads cache and fresh rows as two sources
-        at.excl_words = (r->ctx_len + 31) / 32; at.keep_words = (rows + 31) / 32;
+        at.excl_words = (r->ctx_len + 31) / 32; at.keep_words = (fresh + 31) / 32;
         uint32_t* km = wsp<uint32_t>(c, c->o_keymask);
         at.pos_excl = km; at.row_keep = km + (size_t)r->batch * at.excl_words;
-        launch_key_masks(slot, r->ctx_len, row_pos, rows, r->batch, km, at.excl_words, km + (size_t)r->batch * at.excl_words,
+        launch_key_masks(slot, r->ctx_len, fresh_pos, fresh, r->batch, km, at.excl_words, km + (size_t)r->batch * at.excl_words,
                          at.keep_words, st);
         c->launches += 1;
     }
@@ -259,6 +284,7 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
     c->o_status = take(cur, 256);
     c->o_gridbar = take(cur, 256);
     c->o_row_pos = take(cur, nr * 4);
+    c->o_row_pos2 = take(cur, nr * 4);
     c->o_row_src = take(cur, nr * 8);
     c->o_xn = take(cur, nr * d.hidden * 2);
     c->o_q = take(cur, nr * qd * 2);
@@ -595,6 +621,104 @@ acache_status acache_denoise_step_shared(acache_ctx* ctx, int32_t n_layers, cons
     if (rows == 0) return fail(ctx, ACACHE_ERR_INVALID_ARG, "no rows were recomputed: nothing to predict from");
     return acache_predict_commit(ctx, y, rows, block_rows, req->batch, n_blk, final_norm_g, w_lm, vocab, threshold, token,
                                  confidence, commit, stream);
+}
+
+acache_status acache_recompute_rows_shared(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req_rows,
+                                           const acache_request* req_slots, const acache_kv* kv, const void* x,
+                                           int x_is_compact, const int32_t* anchor_idx, int32_t k, const int32_t* slot_rows,
+                                           void* k_slots, void* v_slots, void* y, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!kv || !req_slots) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv / req_slots is NULL");
+    acache_status s = check_request(ctx, req_rows, kv, 0, true, true);
+    if (s != ACACHE_OK) return s;
+    if ((s = check_request(ctx, req_slots, kv, k, true, true)) != ACACHE_OK) return s;
+    if ((s = check_weights(ctx, w, false)) != ACACHE_OK) return s;
+    if (req_rows->batch != req_slots->batch || req_rows->ctx_len != req_slots->ctx_len ||
+        req_rows->affix_start != req_slots->affix_start || req_rows->affix_len != req_slots->affix_len)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "req_rows and req_slots describe different contexts");
+    if (req_rows->batch * req_rows->n_extra == 0) return ACACHE_OK;
+    if (k + req_slots->n_extra == 0) return fail(ctx, ACACHE_ERR_INVALID_ARG, "the private slot array is empty");
+    if (!x || !k_slots || !v_slots || !y || !slot_rows || !aligned16(x) || !aligned16(k_slots) || !aligned16(v_slots) ||
+        !aligned16(y))
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "x / k_slots / v_slots / y / slot_rows NULL or misaligned");
+    if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
+    const PrivateRows priv{anchor_idx, k, req_slots->extra_rows, req_slots->n_extra, slot_rows};
+    return run_recompute(ctx, w, req_rows, kv, false, x, x_is_compact, nullptr, 0, k_slots, v_slots, y, stream, &priv);
+}
+
+acache_status acache_decode_step_shared(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers,
+                                        const acache_kv* kvs, const acache_request* req_rows,
+                                        const acache_request* req_slots, const void* x0, const int32_t* anchor_idx,
+                                        int32_t k, const int32_t* slot_rows, void* const* k_slots, void* const* v_slots,
+                                        void* y_a, void* y_b, void** y_last, const int32_t* block_rows, int32_t n_blk,
+                                        const void* final_norm_g, const void* w_lm, int32_t vocab, float threshold,
+                                        int32_t* token, float* confidence, int32_t* commit, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (n_layers <= 0 || !layers || !kvs || !req_rows || !req_slots || !x0 || !y_a || !y_b || !k_slots || !v_slots)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL argument or n_layers <= 0");
+    const void* x = x0;
+    void* y = y_a;
+    for (int n = 0; n < n_layers; ++n) {
+        y = (n & 1) ? y_b : y_a;
+        acache_status s = acache_recompute_rows_shared(ctx, &layers[n], req_rows, req_slots, &kvs[n], x, n > 0, anchor_idx, k,
+                                                       slot_rows, k_slots[n], v_slots[n], y, stream);
+        if (s != ACACHE_OK) return s;
+        x = y;
+    }
+    if (y_last) *y_last = y;
+    if (n_blk == 0 || req_rows->batch == 0) return ACACHE_OK;
+    if (req_rows->n_extra == 0) return fail(ctx, ACACHE_ERR_INVALID_ARG, "no rows were recomputed: nothing to predict from");
+    return acache_predict_commit(ctx, y, req_rows->n_extra, block_rows, req_rows->batch, n_blk, final_norm_g, w_lm, vocab,
+                                 threshold, token, confidence, commit, stream);
+}
+
+acache_status acache_generate_block_shared(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers,
+                                           const acache_kv* kvs, const acache_request* req_refresh,
+                                           const acache_request* req_decode, const void* embed, const int32_t* anchor_idx,
+                                           int32_t k, void* const* k_slots, void* const* v_slots, void* y_a, void* y_b,
+                                           const int32_t* block_rows_refresh, const int32_t* block_rows_decode,
+                                           int32_t n_blk, const void* final_norm_g, const void* w_lm, int32_t vocab,
+                                           float threshold, int32_t mask_id, int32_t max_steps, int32_t* token,
+                                           float* confidence, int32_t* commit, int32_t* remaining, int32_t* steps_done,
+                                           acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!req_refresh || !req_decode || !steps_done || !remaining)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "NULL argument");
+    if (!req_refresh->token_ids || req_refresh->token_ids != req_decode->token_ids)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "both requests must name the same token_ids array");
+    if (req_decode->n_extra != n_blk || req_decode->batch != req_refresh->batch || req_decode->ctx_len != req_refresh->ctx_len)
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "req_decode must recompute exactly the block's n_blk rows of the same batch");
+    if (req_refresh->batch > 4096) return fail(ctx, ACACHE_ERR_INVALID_ARG, "batch too large for the step loop");
+    *steps_done = 0;
+    if (req_refresh->batch == 0 || n_blk == 0 || max_steps <= 0) return ACACHE_OK;
+    int32_t* ids = const_cast<int32_t*>(req_refresh->token_ids);
+    int32_t left[4096];
+    for (int step = 0; step < max_steps; ++step) {
+        // step 0 fills the private slots with the anchors and every request-specific row; later steps refresh
+        // the block's rows inside those slots
+        acache_status s;
+        if (step == 0)
+            s = acache_denoise_step_shared(ctx, n_layers, layers, kvs, req_refresh, embed, anchor_idx, k, k_slots, v_slots, y_a, y_b,
+                                           nullptr, block_rows_refresh, n_blk, final_norm_g, w_lm, vocab, threshold, token,
+                                           confidence, commit, stream);
+        else
+            s = acache_decode_step_shared(ctx, n_layers, layers, kvs, req_decode, req_refresh, embed, anchor_idx, k,
+                                          block_rows_refresh, k_slots, v_slots, y_a, y_b, nullptr, block_rows_decode, n_blk,
+                                          final_norm_g, w_lm, vocab, threshold, token, confidence, commit, stream);
+        if (s != ACACHE_OK) return s;
+        s = acache_commit_update(ctx, ids, req_refresh->ctx_len, req_decode->extra_rows, req_refresh->batch, n_blk, token,
+                                 confidence, mask_id, threshold, remaining, stream);
+        if (s != ACACHE_OK) return s;
+        *steps_done = step + 1;
+        if (cudaMemcpyAsync(left, remaining, sizeof(int32_t) * req_refresh->batch, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess)
+            return check_cuda(ctx, "generate_block_shared read-back") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "read-back failed")
+                                                                                   : ACACHE_ERR_CUDA;
+        int total = 0;
+        for (int b = 0; b < req_refresh->batch; ++b) total += left[b];
+        if (total == 0) break;
+    }
+    return ACACHE_OK;
 }
 
 acache_status acache_probe_select(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers, acache_kv* kvs,

@@ -33,8 +33,9 @@ __device__ __forceinline__ void load_kv_tile(uint32_t sk, uint32_t sv, const Att
     const int64_t kstride = (int64_t)a.n_kv_heads * D;
     const __nv_bfloat16* ck = static_cast<const __nv_bfloat16*>(a.cache_k) + (int64_t)b * a.kv_batch_stride + kvh * D;
     const __nv_bfloat16* cv = static_cast<const __nv_bfloat16*>(a.cache_v) + (int64_t)b * a.kv_batch_stride + kvh * D;
-    const __nv_bfloat16* nk = static_cast<const __nv_bfloat16*>(a.k_new) + (int64_t)b * a.n * kstride + kvh * D;
-    const __nv_bfloat16* nv = static_cast<const __nv_bfloat16*>(a.v_new) + (int64_t)b * a.n * kstride + kvh * D;
+    const int n_fresh = a.n_fresh ? a.n_fresh : a.n;
+    const __nv_bfloat16* nk = static_cast<const __nv_bfloat16*>(a.k_new) + (int64_t)b * n_fresh * kstride + kvh * D;
+    const __nv_bfloat16* nv = static_cast<const __nv_bfloat16*>(a.v_new) + (int64_t)b * n_fresh * kstride + kvh * D;
     for (int c = tid; c < 64 * CPR; c += 128) {
         int r = c / CPR, cc = c % CPR;
         int t = t0 + r;

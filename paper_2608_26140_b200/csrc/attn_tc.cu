@@ -799,8 +799,9 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
                                      shared ? (int64_t)a.ctx_len * kv_cols : a.kv_batch_stride);
     const CUtensorMap* mv = get_map3(a.cache_v, a.ctx_len, kv_cols, shared ? 1 : a.batch,
                                      shared ? (int64_t)a.ctx_len * kv_cols : a.kv_batch_stride);
-    const CUtensorMap* mkn = two_src ? get_map3(a.k_new, a.n, kv_cols, a.batch, (int64_t)a.n * kv_cols) : mk;
-    const CUtensorMap* mvn = two_src ? get_map3(a.v_new, a.n, kv_cols, a.batch, (int64_t)a.n * kv_cols) : mv;
+    const int n_fresh = a.n_fresh ? a.n_fresh : a.n;
+    const CUtensorMap* mkn = two_src ? get_map3(a.k_new, n_fresh, kv_cols, a.batch, (int64_t)n_fresh * kv_cols) : mk;
+    const CUtensorMap* mvn = two_src ? get_map3(a.v_new, n_fresh, kv_cols, a.batch, (int64_t)n_fresh * kv_cols) : mv;
     if (!mq || !mk || !mv || !mkn || !mvn) return 0;
     static bool attr = false;
     if (!attr) {
@@ -814,7 +815,7 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     t.status = status;
     t.cache_shared = shared ? 1 : 0;
     if (two_src) {
-        t.n_fresh_tiles = q_tiles; t.excl_words = a.excl_words; t.keep_words = a.keep_words;
+        t.n_fresh_tiles = (n_fresh + 127) / 128; t.excl_words = a.excl_words; t.keep_words = a.keep_words;
         t.pos_excl = a.pos_excl; t.row_keep = a.row_keep;
     }
     static const int kv_prefetch = [] { const char* e = getenv("ACACHE_ATTN_KV_PREFETCH"); return e ? atoi(e) : 2; }();
@@ -824,7 +825,7 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     // 1000+ rows, 8-15 % faster; 8192 keys, 5-10 % slower; fewer CTAs than SMs, up to 1.8x slower).
     // ACACHE_ATTN_TC2Q = 0: never, 2: whenever there are two tiles.
     static const int mode_2q = [] { const char* e = getenv("ACACHE_ATTN_TC2Q"); return e ? atoi(e) : 1; }();
-    const bool use_2q = mode_2q == 2 || (mode_2q == 1 && a.ctx_len + (two_src ? a.n : 0) <= 4096 &&
+    const bool use_2q = mode_2q == 2 || (mode_2q == 1 && a.ctx_len + (two_src ? n_fresh : 0) <= 4096 &&
                                          (int64_t)((q_tiles + 1) / 2) * a.n_heads * a.batch >= 148);
     cudaError_t err;
     if (use_2q && q_tiles >= 2)

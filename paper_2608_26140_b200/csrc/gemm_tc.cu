@@ -163,7 +163,17 @@ __device__ __forceinline__ void out_qkv(const GemmArgs& g, int grow, int pos, in
     const int nseg = g.n[seg];
     __nv_bfloat16* cache = seg == 1 ? static_cast<__nv_bfloat16*>(g.cache_k)
                          : seg == 2 ? static_cast<__nv_bfloat16*>(g.cache_v) : nullptr;
-    __nv_bfloat16* o1 = g.out[seg] ? static_cast<__nv_bfloat16*>(g.out[seg]) + (int64_t)grow * nseg + col : nullptr;
+    int64_t orow = grow;
+    bool o1_ok = g.out[seg] != nullptr;
+    if (seg >= 1 && g.kv_out_rows && o1_ok) {          // the row's place in its request's private slot array
+        const int r = __ldg(g.kv_out_rows + grow);
+        if ((unsigned)r >= (unsigned)g.kv_out_stride) {
+            atomicOr(g.status, kFlagBadIndex);
+            o1_ok = false;
+        }
+        orow = (int64_t)(grow / g.rows_per_req) * g.kv_out_stride + r;
+    }
+    __nv_bfloat16* o1 = o1_ok ? static_cast<__nv_bfloat16*>(g.out[seg]) + orow * nseg + col : nullptr;
     __nv_bfloat16* o2 = (cache && pos >= 0)
                             ? cache + (int64_t)(grow / g.rows_per_req) * g.kv_batch_stride + (int64_t)pos * nseg + col
                             : nullptr;

@@ -23,6 +23,9 @@ void launch_commit_update(int32_t* token_ids, int ctx_len, const int32_t* block_
                           int32_t* remaining, uint32_t* status, cudaStream_t stream);
 
 // slot[b, t] = compact row index whose fresh K/V replaces position t, or -1.
+// Positions of the rows of a private slot array (k anchors, then e extra rows per request).
+void launch_row_positions(const int32_t* anchor_idx, int k, const int32_t* extra_rows, int e, int affix_start, int affix_len,
+                          int ctx_len, int batch, int32_t* row_pos, uint32_t* status, cudaStream_t stream);
 void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
                            cudaStream_t stream);
 
@@ -111,6 +114,10 @@ struct GemmArgs {
     void* cache_v;
     int64_t kv_batch_stride;
     int rows_per_req;
+    // optional: row i of the k/v segments goes to row kv_out_rows[i] of its request's kv_out_stride rows of
+    // out[1] / out[2] (a decode pass refreshing some rows of a larger private slot array) instead of row i
+    const int32_t* kv_out_rows;
+    int kv_out_stride;
     // --- kEpiResidual ---
     const void* resid;        // bf16 base pointer
     const int64_t* resid_off; // [M] element offset of the residual row, or null => row * N
@@ -142,8 +149,9 @@ struct AttnArgs {
     const void* cache_k;      // bf16 [B, cap, Hkv, d]
     const void* cache_v;
     int64_t kv_batch_stride;
-    const void* k_new;        // bf16 [B, n, Hkv, d] or null
+    const void* k_new;        // bf16 [B, n_fresh, Hkv, d] or null
     const void* v_new;
+    int n_fresh;              // rows per request in k_new / v_new; 0 = n (the rows being recomputed are the fresh rows)
     const int32_t* slot;      // [B, ctx_len] or null: >= 0 => read k_new/v_new row slot
     const uint32_t* pos_excl; // optional key masks of the same map (launch_key_masks): with them the tensor-core
     const uint32_t* row_keep; //   kernel reads the cache and k_new / v_new as two key sources instead of gathering

@@ -184,6 +184,28 @@ void launch_scatter_kv(void* cache_k, void* cache_v, int64_t batch_stride, int c
                                              static_cast<const __nv_bfloat16*>(v_new), status);
 }
 
+// row_pos[b, i] = position of private row i of request b (anchors first, then the extra rows); -1 and
+// kFlagBadIndex for an index out of range.
+__global__ void __launch_bounds__(256) row_pos_kernel(const int32_t* __restrict__ anchor_idx, int k,
+                                                      const int32_t* __restrict__ extra_rows, int e, int affix_start,
+                                                      int affix_len, int ctx_len, int32_t* __restrict__ row_pos,
+                                                      uint32_t* status) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int b = blockIdx.y, i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= k + e) return;
+    const int pos = row_position(anchor_idx, k, extra_rows, e, b, i, affix_start, affix_len, ctx_len);
+    if (pos < 0) atomicOr(status, kFlagBadIndex);
+    row_pos[(int64_t)b * (k + e) + i] = pos;
+}
+
+void launch_row_positions(const int32_t* anchor_idx, int k, const int32_t* extra_rows, int e, int affix_start, int affix_len,
+                          int ctx_len, int batch, int32_t* row_pos, uint32_t* status, cudaStream_t stream) {
+    if (batch == 0 || k + e == 0) return;
+    launch_pdl(row_pos_kernel, dim3((k + e + 255) / 256, batch), dim3(256), 0, stream, anchor_idx, k, extra_rows, e, affix_start,
+               affix_len, ctx_len, row_pos, status);
+}
+
 void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
                            cudaStream_t stream) {
     if (batch == 0) return;

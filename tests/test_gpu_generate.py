@@ -61,14 +61,25 @@ def test_commit_update_bitwise():
     assert ctx.poll_status() == 0
 
 
-@pytest.mark.parametrize("shape,n_layers,threshold", [(wl.TINY, 2, 0.9), (wl.TINY_GQA, 2, 0.35)])
-def test_generate_block_vs_oracle(shape, n_layers, threshold):
+MID128 = wl.LayerShape(512, 4, 2, 128, 1024, 1e-5, True, 5e5, "mid-d128")
+
+
+@pytest.mark.parametrize("shape,n_layers,threshold,storage", [
+    (wl.TINY, 2, 0.9, "private"), (wl.TINY_GQA, 2, 0.35, "private"),
+    (wl.TINY_GQA, 2, 0.35, "shared"), (MID128, 2, 0.5, "shared")])
+def test_generate_block_vs_oracle(shape, n_layers, threshold, storage):
     """Step by step with teacher forcing: before every step the oracle takes the GPU's token state
     (the masked rows of this small random model have nearly equal confidences, so which one the
     fallback commits is not unique); per step the predictions must agree and the GPU's commits must
-    be valid under the oracle's confidences.  The C loop must then reproduce the stepwise run exactly."""
+    be valid under the oracle's confidences.  The C loop must then reproduce the stepwise run exactly.
+    storage = "shared": one stale cache per layer serves both requests (batch_stride 0), the refresh
+    pass fills private slots and the decode passes refresh the block's rows inside them; the oracle
+    runs the same schedule on a private copy of that cache per request."""
     B, n_blk, ratio, band = 2, 8, 0.25, 0.03
+    shared = storage == "shared"
     lay, layers, embed, w_lm, gain, ids, caches, cos, sin = small_model(shape, n_layers, B, 4242)
+    if shared:
+        caches = [caches[0] for _ in range(B)]
     T, l, L, P = lay.ctx_len, lay.affix_start, lay.affix_len, lay.n_extra
     K = orc.k_from_ratio(L, ratio)
     g = np.random.default_rng(9)
@@ -95,22 +106,44 @@ def test_generate_block_vs_oracle(shape, n_layers, threshold):
     left = torch.zeros((B,), dtype=torch.int32, device=DEV)
 
     def device_state():
-        dk = [ab.to_device_bf16(np.stack([caches[b][n][0] for b in range(B)]), DEV) for n in range(n_layers)]
-        dv = [ab.to_device_bf16(np.stack([caches[b][n][1] for b in range(B)]), DEV) for n in range(n_layers)]
+        nb = 1 if shared else B
+        dk = [ab.to_device_bf16(np.stack([caches[b][n][0] for b in range(nb)]), DEV) for n in range(n_layers)]
+        dv = [ab.to_device_bf16(np.stack([caches[b][n][1] for b in range(nb)]), DEV) for n in range(n_layers)]
         d_ids = torch.from_numpy(ids.copy()).to(DEV)
         req_r = ab.Context.request(B, T, l, L, masked, extra, dcos, dsin, token_ids=d_ids, n_embed=V)
         req_d = ab.Context.request(B, T, l, L, masked, d_block, dcos, dsin, token_ids=d_ids, n_embed=V)
-        return dk, dv, [ab.Context.kv(dk[n], dv[n]) for n in range(n_layers)], d_ids, req_r, req_d
+        if shared:
+            kvs = [ab.KV(dk[n].data_ptr(), dv[n].data_ptr(), 0, T) for n in range(n_layers)]
+        else:
+            kvs = [ab.Context.kv(dk[n], dv[n]) for n in range(n_layers)]
+        return dk, dv, kvs, d_ids, req_r, req_d
+
+    def slots():
+        z = lambda: [torch.zeros((B, K + P, shape.n_kv_heads, shape.head_dim), dtype=torch.bfloat16, device=DEV)
+                     for _ in range(n_layers)]
+        return z(), z()
+
+    def one_step(refresh, kvs, req_r, req_d, ks, vs):
+        if not shared:
+            ctx.denoise_step(lws, kvs, req_r if refresh else req_d, d_embed, d_anchors if refresh else None,
+                             K if refresh else 0, ya, yb, rows_r if refresh else rows_d, n_blk, d_gain, d_wlm, V, threshold,
+                             token, conf, commit)
+        elif refresh:
+            ctx.denoise_step_shared(lws, kvs, req_r, d_embed, d_anchors, K, ks, vs, ya, yb, rows_r, n_blk, d_gain, d_wlm, V,
+                                    threshold, token, conf, commit)
+        else:
+            ctx.decode_step_shared(lws, kvs, req_d, req_r, d_embed, d_anchors, K, rows_r, ks, vs, ya, yb, rows_d, n_blk,
+                                   d_gain, d_wlm, V, threshold, token, conf, commit)
 
     # ---- stepwise on the GPU, the oracle teacher-forced with the GPU's token state
     dk, dv, kvs, d_ids, req_r, req_d = device_state()
+    ks, vs = slots()
     ref_ids = ids.copy()
     ref_caches = [list(caches[b]) for b in range(B)]
     steps_gpu = 0
     for step in range(2 * n_blk):
         refresh = step == 0
-        ctx.denoise_step(lws, kvs, req_r if refresh else req_d, d_embed, d_anchors if refresh else None, K if refresh else 0,
-                         ya, yb, rows_r if refresh else rows_d, n_blk, d_gain, d_wlm, V, threshold, token, conf, commit)
+        one_step(refresh, kvs, req_r, req_d, ks, vs)
         ctx.commit_update(d_ids, T, d_block, B, n_blk, token, conf, MASK, threshold, left)
         torch.cuda.synchronize()
         steps_gpu += 1
@@ -143,21 +176,37 @@ def test_generate_block_vs_oracle(shape, n_layers, threshold):
         if int(left.sum().item()) == 0:
             break
     assert not np.any(ref_ids[:, block] == MASK) or steps_gpu == 2 * n_blk
-    final_ids, final_k = d_ids.cpu().numpy().copy(), [ab.to_host_bits(t) for t in dk]
     from helpers import TOL, assert_close_bf16
-    for b in range(B):
+    final_ids = d_ids.cpu().numpy().copy()
+    if shared:
+        # the shared caches are untouched; every private slot row holds what the oracle's cache holds at its position
+        final_k = [ab.to_host_bits(t) for t in ks]
         for n in range(n_layers):
-            assert_close_bf16(final_k[n][b], ref_caches[b][n][0], f"layer {n} K cache after the block", 2 * TOL)
+            assert np.array_equal(ab.to_host_bits(dk[n])[0], caches[0][n][0]) and np.array_equal(ab.to_host_bits(dv[n])[0], caches[0][n][1])
+            for b in range(B):
+                pos = np.concatenate([l + anchors[b], lay.extra_rows[b]])
+                assert_close_bf16(final_k[n][b], ref_caches[b][n][0][pos], f"layer {n} private K slots after the block", 2 * TOL)
+                assert_close_bf16(ab.to_host_bits(vs[n])[b], ref_caches[b][n][1][pos], f"layer {n} private V slots after the block", 2 * TOL)
+    else:
+        final_k = [ab.to_host_bits(t) for t in dk]
+        for b in range(B):
+            for n in range(n_layers):
+                assert_close_bf16(final_k[n][b], ref_caches[b][n][0], f"layer {n} K cache after the block", 2 * TOL)
     assert ctx.poll_status() == 0
 
     # ---- the C loop reproduces the stepwise run bit for bit
     dk, dv, kvs, d_ids, req_r, req_d = device_state()
-    steps = ctx.generate_block(lws, kvs, req_r, req_d, d_embed, d_anchors, K, ya, yb, rows_r, rows_d, n_blk, d_gain, d_wlm, V,
-                               threshold, MASK, 2 * n_blk, token, conf, commit, left)
+    ks, vs = slots()
+    if shared:
+        steps = ctx.generate_block_shared(lws, kvs, req_r, req_d, d_embed, d_anchors, K, ks, vs, ya, yb, rows_r, rows_d, n_blk,
+                                          d_gain, d_wlm, V, threshold, MASK, 2 * n_blk, token, conf, commit, left)
+    else:
+        steps = ctx.generate_block(lws, kvs, req_r, req_d, d_embed, d_anchors, K, ya, yb, rows_r, rows_d, n_blk, d_gain, d_wlm, V,
+                                   threshold, MASK, 2 * n_blk, token, conf, commit, left)
     torch.cuda.synchronize()
     assert steps == steps_gpu
     assert np.array_equal(d_ids.cpu().numpy(), final_ids)
     assert left.cpu().numpy().tolist() == [0] * B
     for n in range(n_layers):
-        assert np.array_equal(ab.to_host_bits(dk[n]), final_k[n])
+        assert np.array_equal(ab.to_host_bits(ks[n] if shared else dk[n]), final_k[n])
     assert ctx.poll_status() == 0
