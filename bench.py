@@ -695,7 +695,8 @@ def run_generate(args, e):
     sampler.join()
     launches = ctx.launch_count() - l0
     ms_block = sharding.max_over_ranks(e0.elapsed_time(e1), dist, dev) / n_blocks
-    assert ctx.poll_status() == 0
+    flags = ctx.poll_status()
+    assert flags == 0, f"device status flags {flags:#x}"
     assert int(left.sum().item()) == 0, "the block was not fully decoded"
     if rank != 0:
         if dist:

@@ -146,11 +146,14 @@ struct PrivateRows {
     int e;
     const int32_t* out_rows;
 };
+// Slot map and key masks of the fresh rows are the same for every layer of a pass: the first layer of a
+// multi-layer call builds them in the workspace, the later ones reuse them.
+struct MapReuse { bool reuse; };
 
 acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const acache_request* r,
                             const acache_kv* kv, bool fuse_scatter, const void* x, int x_is_compact,
                             const int32_t* anchor_idx, int k, void* k_new, void* v_new, void* y, cudaStream_t st,
-                            const PrivateRows* priv = nullptr) {
+                            const PrivateRows* priv = nullptr, MapReuse maps = MapReuse{false}) {
     const acache_model_desc& d = c->d;
     const int rows = k + r->n_extra, n = r->batch * rows;
     if (n == 0) {
@@ -206,23 +209,26 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
         const int32_t* fresh_pos = row_pos;
         if (priv) {
             int32_t* rp2 = wsp<int32_t>(c, c->o_row_pos2);
-            launch_row_positions(priv->anchor_idx, priv->k, priv->extra_rows, priv->e, r->affix_start, r->affix_len, r->ctx_len,
-                                 r->batch, rp2, status, st);
-            c->launches += 1;
+            if (!maps.reuse) {
+                launch_row_positions(priv->anchor_idx, priv->k, priv->extra_rows, priv->e, r->affix_start, r->affix_len,
+                                     r->ctx_len, r->batch, rp2, status, st);
+                c->launches += 1;
+            }
             fresh_pos = rp2;
             at.n_fresh = fresh;
         }
         int32_t* slot = wsp<int32_t>(c, c->o_slot);
-        launch_build_slot_map(slot, r->ctx_len, fresh_pos, fresh, r->batch, st);
-        c->launches += 1;
         at.k_new = k_new; at.v_new = v_new; at.slot = slot;
         // key masks of the same map, for the kernel that reads cache and fresh rows as two sources
         at.excl_words = (r->ctx_len + 31) / 32; at.keep_words = (fresh + 31) / 32;
         uint32_t* km = wsp<uint32_t>(c, c->o_keymask);
         at.pos_excl = km; at.row_keep = km + (size_t)r->batch * at.excl_words;
-        launch_key_masks(slot, r->ctx_len, fresh_pos, fresh, r->batch, km, at.excl_words, km + (size_t)r->batch * at.excl_words,
-                         at.keep_words, st);
-        c->launches += 1;
+        if (!maps.reuse) {
+            launch_build_slot_map(slot, r->ctx_len, fresh_pos, fresh, r->batch, st);
+            launch_key_masks(slot, r->ctx_len, fresh_pos, fresh, r->batch, km, at.excl_words,
+                             km + (size_t)r->batch * at.excl_words, at.keep_words, st);
+            c->launches += 2;
+        }
     }
     at.batch = r->batch; at.n = rows; at.ctx_len = r->ctx_len;
     at.n_heads = d.n_heads; at.n_kv_heads = d.n_kv_heads; at.head_dim = d.head_dim;
@@ -261,6 +267,10 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
 }
 
 }  // namespace
+
+// Set by the multi-layer entry points around their layers after the first (same rows, same maps); the
+// single-layer entry points read it.  Thread-local: a context is used from one thread at a time.
+static thread_local bool g_reuse_maps = false;
 
 extern "C" {
 
@@ -438,7 +448,8 @@ acache_status acache_recompute_anchors(acache_ctx* ctx, const acache_layer_weigh
     if (!x || !k_new || !v_new || !y || !aligned16(x) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(y))
         return fail(ctx, ACACHE_ERR_INVALID_ARG, "x / k_new / v_new / y NULL or misaligned");
     if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
-    return run_recompute(ctx, w, req, kv, false, x, x_is_compact, anchor_idx, k, k_new, v_new, y, stream);
+    return run_recompute(ctx, w, req, kv, false, x, x_is_compact, anchor_idx, k, k_new, v_new, y, stream, nullptr,
+                         MapReuse{g_reuse_maps});
 }
 
 acache_status acache_scatter_kv(acache_ctx* ctx, const acache_request* req, acache_kv* kv, const int32_t* anchor_idx,
@@ -610,8 +621,10 @@ acache_status acache_denoise_step_shared(acache_ctx* ctx, int32_t n_layers, cons
     void* y = y_a;
     for (int n = 0; n < n_layers; ++n) {
         y = (n & 1) ? y_b : y_a;
+        g_reuse_maps = n > 0;
         acache_status s = acache_recompute_anchors(ctx, &layers[n], req, &kvs[n], x, n > 0, anchor_idx, k, k_new[n], v_new[n], y,
                                                    stream);
+        g_reuse_maps = false;
         if (s != ACACHE_OK) return s;
         x = y;
     }
@@ -643,7 +656,8 @@ acache_status acache_recompute_rows_shared(acache_ctx* ctx, const acache_layer_w
         return fail(ctx, ACACHE_ERR_INVALID_ARG, "x / k_slots / v_slots / y / slot_rows NULL or misaligned");
     if (k > 0 && !anchor_idx) return fail(ctx, ACACHE_ERR_INVALID_ARG, "anchor_idx is NULL");
     const PrivateRows priv{anchor_idx, k, req_slots->extra_rows, req_slots->n_extra, slot_rows};
-    return run_recompute(ctx, w, req_rows, kv, false, x, x_is_compact, nullptr, 0, k_slots, v_slots, y, stream, &priv);
+    return run_recompute(ctx, w, req_rows, kv, false, x, x_is_compact, nullptr, 0, k_slots, v_slots, y, stream, &priv,
+                         MapReuse{g_reuse_maps});
 }
 
 acache_status acache_decode_step_shared(acache_ctx* ctx, int32_t n_layers, const acache_layer_weights* layers,
@@ -660,8 +674,10 @@ acache_status acache_decode_step_shared(acache_ctx* ctx, int32_t n_layers, const
     void* y = y_a;
     for (int n = 0; n < n_layers; ++n) {
         y = (n & 1) ? y_b : y_a;
+        g_reuse_maps = n > 0;
         acache_status s = acache_recompute_rows_shared(ctx, &layers[n], req_rows, req_slots, &kvs[n], x, n > 0, anchor_idx, k,
                                                        slot_rows, k_slots[n], v_slots[n], y, stream);
+        g_reuse_maps = false;
         if (s != ACACHE_OK) return s;
         x = y;
     }

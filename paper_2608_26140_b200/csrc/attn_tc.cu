@@ -112,6 +112,10 @@ struct AttnTcArgs {
     // rows that do not serve their position (duplicates).  n_fresh_tiles = 0: the cache alone.
     int n_fresh_tiles, excl_words, keep_words, cache_shared;
     int kv_prefetch;          // two-query-tile kernel: K/V tiles requested into L2 ahead of the rings
+    // one-tile kernel over a shared cache with at most 32 rows per request (decode passes): group = 4 puts the rows
+    // of four requests into the four 32-row quarters of one tile, so that the shared cache's key tiles are read
+    // once per four requests; each request's fresh tiles follow, visible to its own quarter only.  Else 1.
+    int group, batch;
     const uint32_t* pos_excl;
     const uint32_t* row_keep;
 };
@@ -139,11 +143,14 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
     const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / (a.n_heads / a.n_kv_heads);
     const int n_cache_tiles = (a.ctx_len + 127) / 128;
-    const int n_tiles = n_cache_tiles + a.n_fresh_tiles;
+    const int n_tiles = n_cache_tiles + a.n_fresh_tiles * min(a.group, a.batch - (int)blockIdx.z * a.group);
     const int kb = a.cache_shared ? 0 : b;          // one cache for the whole batch, or one per request
-    // 32-row quarters of the tile that hold rows of the request: the softmax warps of the others have nothing
-    // to do (their rows of S, P and O are never read), which matters when a decode pass brings 32 rows
-    const int live_q = min(4, (a.n - qt * 128 + 31) / 32);
+    const int G = a.group;                          // requests per tile (4: blockIdx.z counts groups of four)
+    const int b0 = b * G;                           // first request of the tile
+    const int n_req = min(G, a.batch - b0);
+    // 32-row quarters of the tile that hold rows: the softmax warps of the others have nothing to do (their
+    // rows of S, P and O are never read), which matters when a decode pass brings 32 rows per request
+    const int live_q = G > 1 ? n_req : min(4, (a.n - qt * 128 + 31) / 32);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
@@ -168,9 +175,18 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
     if (warp == 0 && lane == 0) {
         // ---------------- TMA producer ----------------
         const uint64_t pol_q = policy_evict_first(), pol_kv = policy_evict_last();
-        mbar_expect_tx(bar(0), AT_TILE);
-        tma_load_3d(sQ, &mapQ, h * 128, qt * 128, b, bar(0), pol_q);
-        tma_load_3d(sQ + AT_PANEL, &mapQ, h * 128 + 64, qt * 128, b, bar(0), pol_q);
+        if (G > 1) {
+            // 32-row boxes: request b0 + r fills rows [32 r, 32 r + 32) of both panels (rows past its n read as zero)
+            mbar_expect_tx(bar(0), n_req * 8192);
+            for (int r = 0; r < n_req; ++r) {
+                tma_load_3d(sQ + r * 4096, &mapQ, h * 128, 0, b0 + r, bar(0), pol_q);
+                tma_load_3d(sQ + AT_PANEL + r * 4096, &mapQ, h * 128 + 64, 0, b0 + r, bar(0), pol_q);
+            }
+        } else {
+            mbar_expect_tx(bar(0), AT_TILE);
+            tma_load_3d(sQ, &mapQ, h * 128, qt * 128, b, bar(0), pol_q);
+            tma_load_3d(sQ + AT_PANEL, &mapQ, h * 128 + 64, qt * 128, b, bar(0), pol_q);
+        }
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
             const int s = j & 1;
@@ -179,7 +195,8 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             const bool fresh = j >= n_cache_tiles;
             const CUtensorMap* mk = fresh ? &mapKn : &mapK;
             const CUtensorMap* mv = fresh ? &mapVn : &mapV;
-            const int r0 = (fresh ? j - n_cache_tiles : j) * 128, bz = fresh ? b : kb;
+            const int f = j - n_cache_tiles;                          // fresh tiles: request by request
+            const int r0 = (fresh ? f % a.n_fresh_tiles : j) * 128, bz = fresh ? b0 + f / a.n_fresh_tiles : kb;
             mbar_expect_tx(bar(1 + s), AT_TILE);
             tma_load_3d(sK0 + s * AT_TILE, mk, kvh * 128, r0, bz, bar(1 + s), pol_kv);
             tma_load_3d(sK0 + s * AT_TILE + AT_PANEL, mk, kvh * 128 + 64, r0, bz, bar(1 + s), pol_kv);
@@ -246,6 +263,7 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
         const int row = q * 32 + lane;
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const uint32_t col_off = (uint32_t)(c4 * 32);
+        const int bq = G > 1 ? b0 + q : b;          // the request whose rows this quarter holds
         float m_use = -INFINITY, l = 0.f;
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
@@ -256,10 +274,27 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             if (j < n_cache_tiles) {
                 const int valid = a.ctx_len - j * 128 - c4 * 32;
                 keep = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
-                if (a.n_fresh_tiles && j * 4 + c4 < a.excl_words) keep &= ~__ldg(a.pos_excl + (int64_t)b * a.excl_words + j * 4 + c4);
+                if (a.n_fresh_tiles && j * 4 + c4 < a.excl_words) keep &= ~__ldg(a.pos_excl + (int64_t)bq * a.excl_words + j * 4 + c4);
             } else {
-                const int w = (j - n_cache_tiles) * 4 + c4;
-                keep = w < a.keep_words ? __ldg(a.row_keep + (int64_t)b * a.keep_words + w) : 0u;
+                const int f = j - n_cache_tiles;
+                if (G > 1 && f / a.n_fresh_tiles != q) {
+                    // another request's fresh rows: none of them is a key of this quarter's rows.  All four warps
+                    // of the quarter come here, so none of them goes to the quarter's barrier for this tile.
+                    if (ok && (ok = mbar_wait(bar(9 + s), (j >> 1) & 1, abort_flag))) {
+                        tc_fence_after();
+                        uint32_t pz[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) pz[i] = 0u;
+                        tc_st16(tS0 + s * 128 + c4 * 16 + lane_off, pz);
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(13 + s));
+                    }
+                    continue;
+                }
+                const int w = (f % a.n_fresh_tiles) * 4 + c4;
+                keep = w < a.keep_words ? __ldg(a.row_keep + (int64_t)bq * a.keep_words + w) : 0u;
             }
             float sv[32];
             float mt = -INFINITY;
@@ -346,9 +381,9 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
         asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
         if (ok && !*abort_flag) {
             tc_fence_after();
-            const int grow = qt * 128 + row;
+            const int grow = G > 1 ? lane : qt * 128 + row;     // the row inside its request
             const float inv = 1.f / ((row_sum[row] + row_sum[128 + row]) + (row_sum[256 + row] + row_sum[384 + row]));
-            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o) + (((int64_t)b * a.n + grow) * a.n_heads + h) * 128 + col_off;
+            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.o) + (((int64_t)bq * a.n + grow) * a.n_heads + h) * 128 + col_off;
             float v[32];
             tc_ld32(tO + lane_off + col_off, v);
             if (grow < a.n) {
@@ -746,8 +781,8 @@ EncodeTiledFn encode_fn3() {
 // box = 64 cols x 128 rows x 1, 128-byte swizzle, zero fill out of bounds.
 struct Map3Key { const void* ptr; int rows, cols, batch; int64_t bstride; int box_rows; };
 struct Map3Entry { Map3Key key; CUtensorMap map; };
-constexpr int kMap3Cache = 64;
-std::mutex g_map3_mutex;   // guards the cache below; held from the lookups to the launch that uses them
+constexpr int kMap3Cache = 1024;
+std::mutex g_map3_mutex;   // guards the cache below; a returned pointer is only good until the next lookup: callers copy the map
 Map3Entry g_maps3[kMap3Cache];
 int g_map3_count = 0, g_map3_next = 0;
 
@@ -794,14 +829,24 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     const bool shared = a.kv_batch_stride == 0;           // one cache for the whole batch
     const int kv_cols = a.n_kv_heads * 128;
     std::lock_guard<std::mutex> lock(g_map3_mutex);
-    const CUtensorMap* mq = get_map3(a.q, a.n, a.n_heads * 128, a.batch, (int64_t)a.n * a.n_heads * 128);
-    const CUtensorMap* mk = get_map3(a.cache_k, a.ctx_len, kv_cols, shared ? 1 : a.batch,
-                                     shared ? (int64_t)a.ctx_len * kv_cols : a.kv_batch_stride);
-    const CUtensorMap* mv = get_map3(a.cache_v, a.ctx_len, kv_cols, shared ? 1 : a.batch,
-                                     shared ? (int64_t)a.ctx_len * kv_cols : a.kv_batch_stride);
+    // decode passes over a shared cache: the rows of four requests share one tile (see AttnTcArgs::group)
+    static const bool group_on = [] { const char* e = getenv("ACACHE_ATTN_GROUP"); return !e || atoi(e) != 0; }();
+    const int group = (group_on && two_src && shared && a.n <= 32 && a.batch >= 2) ? 4 : 1;
+    CUtensorMap maps[5];
+    const CUtensorMap* found[5];
+    found[0] = get_map3(a.q, a.n, a.n_heads * 128, a.batch, (int64_t)a.n * a.n_heads * 128, group > 1 ? 32 : 128);
+    if (found[0]) maps[0] = *found[0];
+    found[1] = get_map3(a.cache_k, a.ctx_len, kv_cols, shared ? 1 : a.batch, shared ? (int64_t)a.ctx_len * kv_cols : a.kv_batch_stride);
+    if (found[1]) maps[1] = *found[1];
+    found[2] = get_map3(a.cache_v, a.ctx_len, kv_cols, shared ? 1 : a.batch, shared ? (int64_t)a.ctx_len * kv_cols : a.kv_batch_stride);
+    if (found[2]) maps[2] = *found[2];
     const int n_fresh = a.n_fresh ? a.n_fresh : a.n;
-    const CUtensorMap* mkn = two_src ? get_map3(a.k_new, n_fresh, kv_cols, a.batch, (int64_t)n_fresh * kv_cols) : mk;
-    const CUtensorMap* mvn = two_src ? get_map3(a.v_new, n_fresh, kv_cols, a.batch, (int64_t)n_fresh * kv_cols) : mv;
+    found[3] = two_src ? get_map3(a.k_new, n_fresh, kv_cols, a.batch, (int64_t)n_fresh * kv_cols) : found[1];
+    if (found[3]) maps[3] = two_src ? *found[3] : maps[1];
+    found[4] = two_src ? get_map3(a.v_new, n_fresh, kv_cols, a.batch, (int64_t)n_fresh * kv_cols) : found[2];
+    if (found[4]) maps[4] = two_src ? *found[4] : maps[2];
+    const CUtensorMap *mq = found[0] ? &maps[0] : nullptr, *mk = found[1] ? &maps[1] : nullptr, *mv = found[2] ? &maps[2] : nullptr,
+                      *mkn = found[3] ? &maps[3] : nullptr, *mvn = found[4] ? &maps[4] : nullptr;
     if (!mq || !mk || !mv || !mkn || !mvn) return 0;
     static bool attr = false;
     if (!attr) {
@@ -814,6 +859,7 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     t.scale_log2e = 1.4426950408889634f / sqrtf(128.f);
     t.status = status;
     t.cache_shared = shared ? 1 : 0;
+    t.group = group; t.batch = a.batch;
     if (two_src) {
         t.n_fresh_tiles = (n_fresh + 127) / 128; t.excl_words = a.excl_words; t.keep_words = a.keep_words;
         t.pos_excl = a.pos_excl; t.row_keep = a.row_keep;
@@ -832,8 +878,8 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
         err = launch_pdl(attention_tc2q_kernel, dim3((q_tiles + 1) / 2, a.n_heads, a.batch), dim3(AT2_THREADS), AT2_SMEM, stream, t,
                          *mq, *mk, *mv, *mkn, *mvn);
     else
-        err = launch_pdl(attention_tc_kernel, dim3(q_tiles, a.n_heads, a.batch), dim3(AT_THREADS), AT_SMEM, stream, t, *mq, *mk,
-                         *mv, *mkn, *mvn);
+        err = launch_pdl(attention_tc_kernel, dim3(q_tiles, a.n_heads, (a.batch + group - 1) / group), dim3(AT_THREADS), AT_SMEM,
+                         stream, t, *mq, *mk, *mv, *mkn, *mvn);
     return err == cudaSuccess ? 1 : -1;
 }
 

@@ -1063,11 +1063,12 @@ EncodeTiledFn encode_fn() {
 // bf16 [rows, cols] row-major, box = 128 rows x 64 cols, 128-byte swizzle, zero fill out of bounds.
 struct MapKey { const void* ptr; int rows, cols; };
 struct MapEntry { MapKey key; CUtensorMap map; };
-constexpr int kMapCache = 64;
+constexpr int kMapCache = 1024;   // a 32-layer model has over 200 weight matrices
 std::mutex g_map_mutex;
 MapEntry g_maps[kMapCache];
 int g_map_count = 0, g_map_next = 0;
 
+// The pointer is only good until the next call (a miss may replace any entry): callers copy the map.
 const CUtensorMap* get_map(const void* ptr, int rows, int cols) {
     for (int i = 0; i < g_map_count; ++i)
         if (g_maps[i].key.ptr == ptr && g_maps[i].key.rows == rows && g_maps[i].key.cols == cols) return &g_maps[i].map;
@@ -1141,13 +1142,21 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
     const int n_total = swiglu ? g.n[0] : g.n[0] + g.n[1] + g.n[2];
     const TcPlan p = make_plan(g.M, g.K, n_total / 128, swiglu);
     std::lock_guard<std::mutex> lock(g_map_mutex);
-    const CUtensorMap* mA = get_map(g.a, g.M, g.K);
-    const CUtensorMap* mB[3] = {nullptr, nullptr, nullptr};
+    CUtensorMap map_a, map_b[3];
+    {
+        const CUtensorMap* m = get_map(g.a, g.M, g.K);
+        if (!m) return -1;
+        map_a = *m;
+    }
+    bool have_b[3] = {false, false, false};
     for (int i = 0; i < 3; ++i)
-        if (g.b[i]) mB[i] = get_map(g.b[i], swiglu ? g.n[0] : g.n[i], g.K);
-    if (!mA || !mB[0]) return -1;
-    for (int i = 1; i < 3; ++i)
-        if (!mB[i]) mB[i] = mB[0];
+        if (g.b[i]) {
+            const CUtensorMap* m = get_map(g.b[i], swiglu ? g.n[0] : g.n[i], g.K);
+            if (m) { map_b[i] = *m; have_b[i] = true; }
+        }
+    if (!have_b[0]) return -1;
+    const CUtensorMap* mA = &map_a;
+    const CUtensorMap* mB[3] = {&map_b[0], have_b[1] ? &map_b[1] : &map_b[0], have_b[2] ? &map_b[2] : &map_b[0]};
     static bool attr = false;
     if (!attr) {
         cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);

@@ -353,10 +353,14 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
     const int kv_cols = a.n_kv_heads * 128;
     const int ctx_rows = a.norm_lo + a.norm_len > a.affix_start + a.affix_len ? a.norm_lo + a.norm_len : a.affix_start + a.affix_len;
     std::lock_guard<std::mutex> lock(g_map3_mutex);
+    CUtensorMap map_q, map_k;
     const CUtensorMap* mq = get_map3(a.q_mask, a.m, a.n_heads * 128, a.batch, (int64_t)a.m * a.n_heads * 128);
+    if (!mq) return 0;
+    map_q = *mq; mq = &map_q;        // the cache may replace the entry at the next lookup
     const CUtensorMap* mk = get_map3(a.cache_k, ctx_rows, kv_cols, shared ? 1 : a.batch,
                                      shared ? (int64_t)ctx_rows * kv_cols : a.kv_batch_stride);
-    if (!mq || !mk) return 0;
+    if (!mk) return 0;
+    map_k = *mk; mk = &map_k;
     static bool attr = false;
     if (!attr) {
         cudaFuncSetAttribute(score_stats_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM1);

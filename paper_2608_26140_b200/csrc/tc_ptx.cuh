@@ -120,7 +120,7 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n) {
 
 // 3-d tensor maps over bf16 [batch, rows, cols] (row stride = cols, batch stride in elements), box 64 cols x
 // box_rows rows x 1, 128-byte swizzle, zero fill out of bounds; cached by (pointer, shape, box).  Host side, defined in
-// attn_tc.cu; the returned pointer stays valid while g_map3_mutex is held.
+// attn_tc.cu; the returned pointer is good until the next lookup (copy the map), under g_map3_mutex.
 const CUtensorMap* get_map3(const void* ptr, int rows, int cols, int batch, int64_t bstride, int box_rows = 128);
 extern std::mutex g_map3_mutex;
 

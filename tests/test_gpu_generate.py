@@ -64,10 +64,11 @@ def test_commit_update_bitwise():
 MID128 = wl.LayerShape(512, 4, 2, 128, 1024, 1e-5, True, 5e5, "mid-d128")
 
 
-@pytest.mark.parametrize("shape,n_layers,threshold,storage", [
-    (wl.TINY, 2, 0.9, "private"), (wl.TINY_GQA, 2, 0.35, "private"),
-    (wl.TINY_GQA, 2, 0.35, "shared"), (MID128, 2, 0.5, "shared")])
-def test_generate_block_vs_oracle(shape, n_layers, threshold, storage):
+@pytest.mark.parametrize("shape,n_layers,threshold,storage,B", [
+    (wl.TINY, 2, 0.9, "private", 2), (wl.TINY_GQA, 2, 0.35, "private", 2),
+    (wl.TINY_GQA, 2, 0.35, "shared", 2), (MID128, 2, 0.5, "shared", 2),
+    (MID128, 2, 0.5, "shared", 5)])       # five requests: one full group of four in a decode-pass attention tile + one
+def test_generate_block_vs_oracle(shape, n_layers, threshold, storage, B):
     """Step by step with teacher forcing: before every step the oracle takes the GPU's token state
     (the masked rows of this small random model have nearly equal confidences, so which one the
     fallback commits is not unique); per step the predictions must agree and the GPU's commits must
@@ -75,7 +76,7 @@ def test_generate_block_vs_oracle(shape, n_layers, threshold, storage):
     storage = "shared": one stale cache per layer serves both requests (batch_stride 0), the refresh
     pass fills private slots and the decode passes refresh the block's rows inside them; the oracle
     runs the same schedule on a private copy of that cache per request."""
-    B, n_blk, ratio, band = 2, 8, 0.25, 0.03
+    n_blk, ratio, band = 8, 0.25, 0.03
     shared = storage == "shared"
     lay, layers, embed, w_lm, gain, ids, caches, cos, sin = small_model(shape, n_layers, B, 4242)
     if shared:
