@@ -16,6 +16,10 @@
 // exponentials.  The running maximum used for the exponent is only raised (and O rescaled in
 // TMEM) when the true maximum has grown by more than 2^8, which keeps P within bf16 range and
 // makes rescales rare.  Every mbarrier wait is bounded (status flag kFlagWaitExpired on expiry).
+// With two key sources (a cache shared by the batch + each request's private rows, Section 4.1) the
+// private rows' tiles follow the cache's, and key masks tell which of the two serves a position; when
+// every request brings at most 32 rows (decode passes), four requests share one tile, one per 32-row
+// quarter, so that the shared cache's tiles are read once per four requests.
 #include <cuda.h>
 
 #include <mutex>

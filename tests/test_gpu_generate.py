@@ -211,3 +211,53 @@ def test_generate_block_vs_oracle(shape, n_layers, threshold, storage, B):
     for n in range(n_layers):
         assert np.array_equal(ab.to_host_bits(ks[n] if shared else dk[n]), final_k[n])
     assert ctx.poll_status() == 0
+
+
+def test_decode_over_shared_storage_flags_a_bad_slot_row_and_rejects_mismatched_requests():
+    """A slot row outside the slot array raises the bad-index flag and that row's K/V is not stored (the
+    other rows are); requests that describe different contexts are refused before anything is enqueued."""
+    shape, n_layers, B, n_blk, ratio = MID128, 1, 2, 8, 0.25
+    lay, layers, embed, w_lm, gain, ids, caches, cos, sin = small_model(shape, n_layers, B, 77)
+    T, l, L, P = lay.ctx_len, lay.affix_start, lay.affix_len, lay.n_extra
+    K = orc.k_from_ratio(L, ratio)
+    g = np.random.default_rng(2)
+    anchors = torch.from_numpy(np.stack([np.sort(g.choice(L, K, replace=False)) for _ in range(B)]).astype(np.int32)).to(DEV)
+    block = np.stack([lay.masked_pos[b][:n_blk] for b in range(B)]).astype(np.int32)
+    where = {int(p): i for i, p in enumerate(lay.extra_rows[0])}
+    rows_r = np.stack([[K + where[int(p)] for p in block[b]] for b in range(B)]).astype(np.int32)
+    bad_rows = rows_r.copy()
+    bad_rows[1, 2] = K + P                     # one past the end of the slot array
+    w = {k: (ab.to_device_bf16(v, DEV) if v is not None else None) for k, v in layers[0].items()}
+    lw = ab.Context.weights(w)
+    dcos, dsin = torch.from_numpy(cos).to(DEV), torch.from_numpy(sin).to(DEV)
+    masked, extra = torch.from_numpy(lay.masked_pos.copy()).to(DEV), torch.from_numpy(lay.extra_rows.copy()).to(DEV)
+    d_block = torch.from_numpy(block).to(DEV)
+    dk, dv = ab.to_device_bf16(caches[0][0][0][None], DEV), ab.to_device_bf16(caches[0][0][1][None], DEV)
+    kv = ab.KV(dk.data_ptr(), dv.data_ptr(), 0, T)
+    req_s = ab.Context.request(B, T, l, L, masked, extra, dcos, dsin)
+    req_r = ab.Context.request(B, T, l, L, masked, d_block, dcos, dsin)
+    ctx = ab.Context.for_shape(shape, B, T, L, K + P, lay.n_masked, DEV)
+    ks = torch.zeros((B, K + P, shape.n_kv_heads, shape.head_dim), dtype=torch.bfloat16, device=DEV)
+    vs = torch.zeros_like(ks)
+    x = ab.to_device_bf16(wl.normal_bf16(3, (B, n_blk, shape.hidden), 1.0), DEV)
+    y = torch.zeros((B, n_blk, shape.hidden), dtype=torch.bfloat16, device=DEV)
+    ctx.recompute_rows_shared(lw, req_r, req_s, kv, x, 1, anchors, K, torch.from_numpy(bad_rows).to(DEV), ks, vs, y)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() & ab.FLAG_BAD_INDEX
+    kb = ab.to_host_bits(ks)
+    written = np.zeros((B, K + P), dtype=bool)
+    for b in range(B):
+        for i in range(n_blk):
+            if not (b == 1 and i == 2):
+                written[b, rows_r[b, i]] = True
+    assert np.all(kb[~written] == 0), "a row outside the block's slots was written"
+    assert all(np.any(kb[b, r] != 0) for b in range(B) for r in np.flatnonzero(written[b])), "a block row was not stored"
+    # a request pair that disagrees on the context is refused
+    req_other = ab.Context.request(B, T, l, L - 1, masked, d_block, dcos, dsin)
+    with pytest.raises(ab.AcacheError):
+        ctx.recompute_rows_shared(lw, req_other, req_s, kv, x, 1, anchors, K, torch.from_numpy(rows_r).to(DEV), ks, vs, y)
+    # and so is a cache with one copy per request where the call wants nothing written: allowed (reads only) -- but a
+    # NULL slot_rows is not
+    with pytest.raises(ab.AcacheError):
+        ctx.recompute_rows_shared(lw, req_r, req_s, kv, x, 1, anchors, K, None, ks, vs, y)
+    assert ctx.poll_status() == 0
