@@ -299,6 +299,18 @@ acache_status acache_denoise_step_shared(acache_ctx *ctx, int32_t n_layers, cons
                                          const void *w_lm, int32_t vocab, float threshold, int32_t *token,
                                          float *confidence, int32_t *commit, acache_stream_t stream);
 
+/* acache_layer_step on storage that is not written (Section 4.1): the cache may be one copy for the
+ * whole batch (kv->batch_stride = 0) or one per request; scores and selection read it, and the refreshed
+ * K/V of the rows of R go to k_new / v_new (DEVICE bf16 [B, K + e, Hkv, d], the request's private slots)
+ * instead of into the cache; their attention reads every other position from the cache.  Equivalent to the
+ * masked rows' query projection + acache_score_anchors + acache_select_topk + acache_recompute_anchors.
+ * Flags, x, scores, anchor_idx and y as acache_layer_step; k_new / v_new may be NULL only with
+ * ACACHE_F_NO_RECOMPUTE. */
+acache_status acache_layer_step_shared(acache_ctx *ctx, const acache_layer_weights *w, const acache_request *req,
+                                       const acache_kv *kv, const void *x, int x_is_compact, double ratio,
+                                       uint32_t flags, float *scores, int32_t *anchor_idx, void *k_new,
+                                       void *v_new, void *y, acache_stream_t stream);
+
 /* A decode pass over shared affix storage (Section 4.1 storage under the Section 4.3 schedule): after a
  * refresh pass (acache_recompute_anchors / acache_denoise_step_shared with kv->batch_stride = 0) has
  * filled the private slot arrays k_slots / v_slots [B, k + e_slots, Hkv, d] with the anchors and the

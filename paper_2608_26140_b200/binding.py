@@ -24,7 +24,7 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times",
            "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step", "acache_probe_select",
            "acache_commit_update", "acache_generate_block", "acache_denoise_step_shared", "acache_recompute_rows_shared",
-           "acache_decode_step_shared", "acache_generate_block_shared"]
+           "acache_decode_step_shared", "acache_generate_block_shared", "acache_layer_step_shared"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -125,6 +125,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
                                           C.POINTER(Request), vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, i32, C.c_float,
                                           i32, i32, vp, vp, vp, vp, C.POINTER(i32), vp]
     lib.acache_generate_block.restype = C.c_int
+    lib.acache_layer_step_shared.argtypes = [vp, C.POINTER(LayerWeights), C.POINTER(Request), C.POINTER(KV), vp, C.c_int,
+                                             C.c_double, u32, vp, vp, vp, vp, vp, vp]
+    lib.acache_layer_step_shared.restype = C.c_int
     lib.acache_recompute_rows_shared.argtypes = [vp, C.POINTER(LayerWeights), C.POINTER(Request), C.POINTER(Request),
                                                  C.POINTER(KV), vp, C.c_int, vp, i32, vp, vp, vp, vp, vp]
     lib.acache_recompute_rows_shared.restype = C.c_int
@@ -312,6 +315,13 @@ class Context:
                                                         _ptr(final_norm_g), _ptr(w_lm), vocab, float(threshold), _ptr(token),
                                                         _ptr(confidence), _ptr(commit), _stream()))
         return last.value
+
+    def layer_step_shared(self, w: LayerWeights, req: Request, kv: KV, x, x_is_compact, ratio, flags, scores, anchor_idx,
+                          k_new, v_new, y):
+        """The fused layer-step over storage that is not written (the cache may be shared by the batch)."""
+        self._check(self.lib.acache_layer_step_shared(self.h, C.byref(w), C.byref(req), C.byref(kv), _ptr(x), int(x_is_compact),
+                                                      float(ratio), int(flags), _ptr(scores), _ptr(anchor_idx), _ptr(k_new),
+                                                      _ptr(v_new), _ptr(y), _stream()))
 
     def recompute_rows_shared(self, w: LayerWeights, req_rows: Request, req_slots: Request, kv: KV, x, x_is_compact,
                               anchor_idx, k, slot_rows, k_slots, v_slots, y):

@@ -468,15 +468,22 @@ acache_status acache_scatter_kv(acache_ctx* ctx, const acache_request* req, acac
     return check_cuda(ctx, "scatter");
 }
 
-acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
-                                acache_kv* kv, const void* x, int x_is_compact, double ratio, uint32_t flags,
-                                float* scores, int32_t* anchor_idx, void* y, acache_stream_t stream) {
+}  // extern "C"
+
+namespace {
+// The layer-step on one working cache per request (k_new = v_new = NULL: fresh K/V go straight into the cache) or
+// on storage that is not written (fresh K/V to k_new / v_new [B, K + e, Hkv, d]; the cache may be shared).
+acache_status layer_step_impl(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
+                              const acache_kv* kv, const void* x, int x_is_compact, double ratio, uint32_t flags,
+                              float* scores, int32_t* anchor_idx, void* k_new, void* v_new, void* y,
+                              acache_stream_t stream) {
     if (!ctx) return ACACHE_ERR_INVALID_ARG;
     if (!kv) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv is NULL");
     if (!req) return fail(ctx, ACACHE_ERR_INVALID_ARG, "request is NULL");
     const acache_model_desc& d = ctx->d;
     const int k = acache_k_from_ratio(req->affix_len, ratio);
-    acache_status s = check_request(ctx, req, kv, k, true);
+    const bool to_slots = k_new != nullptr;
+    acache_status s = check_request(ctx, req, kv, k, true, to_slots);
     if (s != ACACHE_OK) return s;
     const bool do_score = flags & ACACHE_F_SCORE, do_select = flags & ACACHE_F_SELECT;
     const bool do_recompute = !(flags & ACACHE_F_NO_RECOMPUTE);
@@ -539,9 +546,30 @@ acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, 
         ctx->launches += 1;
     }
     if (do_recompute)
-        return run_recompute(ctx, w, req, kv, true, x, x_is_compact, anchor_idx, k, nullptr, nullptr, y, stream);
+        return run_recompute(ctx, w, req, kv, !to_slots, x, x_is_compact, anchor_idx, k, k_new, v_new, y, stream);
     mark(ctx, ACACHE_N_STAGES, stream);
     return check_cuda(ctx, "layer_step");
+}
+}  // namespace
+
+extern "C" {
+
+acache_status acache_layer_step(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
+                                acache_kv* kv, const void* x, int x_is_compact, double ratio, uint32_t flags,
+                                float* scores, int32_t* anchor_idx, void* y, acache_stream_t stream) {
+    return layer_step_impl(ctx, w, req, kv, x, x_is_compact, ratio, flags, scores, anchor_idx, nullptr, nullptr, y, stream);
+}
+
+acache_status acache_layer_step_shared(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
+                                       const acache_kv* kv, const void* x, int x_is_compact, double ratio,
+                                       uint32_t flags, float* scores, int32_t* anchor_idx, void* k_new, void* v_new,
+                                       void* y, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!(flags & ACACHE_F_NO_RECOMPUTE) && (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)))
+        return fail(ctx, ACACHE_ERR_INVALID_ARG, "k_new / v_new NULL or misaligned");
+    static char dummy;        // a scoring-only call stores no K/V: any non-NULL value selects the read-only path
+    return layer_step_impl(ctx, w, req, kv, x, x_is_compact, ratio, flags, scores, anchor_idx, k_new ? k_new : &dummy,
+                           v_new ? v_new : &dummy, y, stream);
 }
 
 acache_status acache_predict_commit(acache_ctx* ctx, const void* h, int32_t h_rows, const int32_t* block_rows,

@@ -391,6 +391,26 @@ def test_shared_affix_cache_with_private_rows(L, ratio):
         assert_close_bf16(ab.to_host_bits(k_new[b]), ref["k_new"], "private K")
         assert_close_bf16(ab.to_host_bits(v_new[b]), ref["v_new"], "private V")
         assert_close_bf16(ab.to_host_bits(y[b]), ref["y"], "y")
+    # the fused call over the same storage: the masked rows' queries now come from its own projection of x
+    k2, v2, y2 = torch.zeros_like(k_new), torch.zeros_like(v_new), torch.zeros_like(y)
+    scores2, anchors2 = torch.zeros_like(scores), torch.zeros_like(anchors)
+    dc.ctx.layer_step_shared(dc.lw, dc.req, kv, dc.x, 0, ratio, ab.F_SCORE | ab.F_SELECT, scores2, anchors2, k2, v2, y2)
+    torch.cuda.synchronize()
+    assert dc.ctx.poll_status() == 0
+    assert np.array_equal(ab.to_host_bits(dsk[0]), shared_k) and np.array_equal(ab.to_host_bits(dsv[0]), shared_v)
+    s2, a2 = scores2.cpu().numpy(), anchors2.cpu().numpy()
+    for b in range(B):
+        free = orc.layer_step(case.weights, shape, case.x[b], shared_k, shared_v, T, lay.affix_start, L,
+                              lay.masked_pos[b], lay.extra_rows[b], case.rope_cos, case.rope_sin, ratio=ratio)
+        assert (np.abs(s2[b] - free["scores64"]) / np.maximum(free["scores64"], free["scores64"].mean())).max() < 1e-3
+        ok, why = orc.anchor_set_ok(a2[b], K, L, free["must"], free["may"])
+        assert ok, why
+        ref = free if np.array_equal(free["anchor_idx"], a2[b]) else orc.layer_step(
+            case.weights, shape, case.x[b], shared_k, shared_v, T, lay.affix_start, L, lay.masked_pos[b], lay.extra_rows[b],
+            case.rope_cos, case.rope_sin, anchor_idx=a2[b])
+        assert_close_bf16(ab.to_host_bits(k2[b]), ref["k_new"], "private K (fused call)")
+        assert_close_bf16(ab.to_host_bits(v2[b]), ref["v_new"], "private V (fused call)")
+        assert_close_bf16(ab.to_host_bits(y2[b]), ref["y"], "y (fused call)")
     # calls that write the cache refuse a shared one
     with pytest.raises(ab.AcacheError):
         dc.ctx.scatter_kv(dc.req, kv, anchors, K, k_new, v_new)
