@@ -1,7 +1,7 @@
 """The attention kernel is chosen by problem size (one or two query tiles per CTA on the tcgen05
 path, mma.sync for head dimension 64), so the small parity cases never reach some of the kernels
 that the full-size runs use, e.g. the two-query-tile kernel reading two key sources (shared affix
-storage).  The choice is read from the environment once per process; each case below runs the
+storage), and switches such as the grouping of four requests per decode-pass tile have a second path.  The choice is read from the environment once per process; each case below runs the
 attention-heavy parity tests in a child process with one kernel forced."""
 import os
 import subprocess
@@ -12,14 +12,15 @@ import pytest
 pytestmark = pytest.mark.gpu
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-SELECT = "shared or layer_step or recompute_then_scatter or duplicate_row or full_size or idempotent"
+SELECT = ("shared or layer_step or recompute_then_scatter or duplicate_row or full_size or idempotent or "
+          "generate_block or decode_over_shared")
 
 
-@pytest.mark.parametrize("switch", ["ACACHE_ATTN_TC2Q=2", "ACACHE_ATTN_TC2Q=0", "ACACHE_ATTN_TC=0"])
+@pytest.mark.parametrize("switch", ["ACACHE_ATTN_TC2Q=2", "ACACHE_ATTN_TC2Q=0", "ACACHE_ATTN_TC=0", "ACACHE_ATTN_GROUP=0"])
 def test_parity_with_one_attention_kernel_forced(switch):
     name, value = switch.split("=")
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
-           "tests/test_gpu_parity.py", "tests/test_gpu_predict_commit.py", "-k", SELECT]
+           "tests/test_gpu_parity.py", "tests/test_gpu_predict_commit.py", "tests/test_gpu_generate.py", "-k", SELECT]
     r = subprocess.run(cmd, cwd=ROOT, env={**os.environ, name: value}, capture_output=True, text=True, timeout=1200)
     assert r.returncode == 0, (r.stdout[-3000:], r.stderr[-1000:])
     assert " passed" in r.stdout and "no tests ran" not in r.stdout
