@@ -780,6 +780,27 @@ def run_shared(args):
         ctx.select_topk(scores, B, L, K, anchors)
         ctx.recompute_anchors(lw, req, kv_shared, x, 0, anchors, K, k_new, v_new, y)
 
+    if args.decode:
+        # one layer of a decode pass: only the first 32 masked rows of every request are recomputed.  Private caches:
+        # acache_layer_step with ratio 0 on those rows; shared storage: the slots as a refresh left them
+        # (shared_step above), then acache_recompute_rows_shared for the block's rows.
+        n_blk = 32
+        blk = np.ascontiguousarray(lay.masked_pos[:, :n_blk])
+        dblk = torch.from_numpy(blk.copy()).to(dev)
+        req_blk = ab.Context.request(B, T, lay.affix_start, L, masked, dblk, cos, sin)
+        where = {int(p_): i for i, p_ in enumerate(lay.extra_rows[0])}
+        slot_rows = torch.from_numpy(np.stack([[K + where[int(p_)] for p_ in blk[b]] for b in range(B)]).astype(np.int32)).to(dev)
+        xb = torch.randn((B, n_blk, shape.hidden), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        yb = torch.zeros((B, n_blk, shape.hidden), dtype=torch.bfloat16, device=dev)
+        shared_step()                                   # fills k_new / v_new and the anchors
+        torch.cuda.synchronize()
+
+        def private_step():                             # noqa: F811
+            ctx.layer_step(lw, req_blk, kv_priv, xb, 1, 0.0, 0, None, None, yb)
+
+        def shared_step():                              # noqa: F811
+            ctx.recompute_rows_shared(lw, req_blk, req, kv_shared, xb, 1, anchors, K, slot_rows, k_new, v_new, yb)
+
     res = {}
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for name, fn in (("private", private_step), ("shared", shared_step)):
@@ -804,7 +825,9 @@ def run_shared(args):
         "ms_per_step": res["shared"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": f"cfg{cfg} one layer, shared affix storage: {shape.name}, batch {B} sharing a {L}-token affix, "
-                               f"K={K} anchors + {P} request rows per request ({B * n} rows)", "benchmark_config": cfg},
+                               + (f"decode pass: the block's 32 rows per request ({B * 32} rows) against {n} slot rows per request"
+                                  if args.decode else f"K={K} anchors + {P} request rows per request ({B * n} rows)"),
+                   "benchmark_config": cfg, "pass": "decode" if args.decode else "refresh"},
         "shared_storage": {"ms_per_layer": res["shared"], "kv_bytes_per_layer": kv_shared_b, "stage_us": res["shared_stage_us"],
                            "note": "the masked-row queries are given (acache_score_anchors); the split calls do not write the cache"},
         "private_caches": {"ms_per_layer": res["private"], "kv_bytes_per_layer": kv_private, "stage_us": res["private_stage_us"],
@@ -849,6 +872,8 @@ def main():
     ap.add_argument("--layers", type=int, default=32, help="layers of the --config 3 denoising step")
     ap.add_argument("--shared", action="store_true",
                     help="--config 3 or 4: one layer with shared affix storage (batch_stride 0) against private caches")
+    ap.add_argument("--decode", action="store_true",
+                    help="with --shared: time one layer of a decode pass (32 rows per request) instead of the refresh")
     ap.add_argument("--generate", action="store_true",
                     help="--config 3: decode one whole 32-token block per request (refresh + decode passes); "
                          "with --shared over shared affix storage")
