@@ -270,6 +270,36 @@ __device__ __forceinline__ void logit_stats_update(const float (&v)[W], int col,
     for (int i = 0; i < W; ++i) s += __expf(v[i] - m);
 }
 
+// The same for one group of 16 columns, four CTAs at a time (the registers the second group would take hold
+// two more CTAs' loads): epilogues without a second group (residual, logits) have nine or ten contributors per
+// tile on the narrow projections, and every round of loads is a trip to L2.
+__device__ __forceinline__ void sum_slots16_single(const float* __restrict__ partial, const TcPlan& p, int t, int c_first,
+                                                   int c_last, int pc0, int row, float (&lo)[16]) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) lo[i] = 0.f;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int o0 = pc0 * TC_BM + row;
+    for (int c = c_first; c <= c_last; c += 4) {
+        float4 a[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const bool in = c + i <= c_last;
+            const float4* src = reinterpret_cast<const float4*>(partial) + slot_of(p, t, in ? c + i : c) * (TC_SLOT_FLOATS / 4);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) a[i][j] = in ? __ldcg(src + o0 + j * TC_BM) : zero;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (c + i <= c_last) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    lo[4 * j] += a[i][j].x; lo[4 * j + 1] += a[i][j].y; lo[4 * j + 2] += a[i][j].z; lo[4 * j + 3] += a[i][j].w;
+                }
+            }
+        }
+    }
+}
+
 // Work items of the finish per output tile: 16 output columns each (q/k/v: 16 of each rotary half).
 __host__ __device__ __forceinline__ int finish_items_per_tile(int epilogue) {
     return (epilogue == kEpiResidual || epilogue == kEpiLogits) ? 16 : 8;
@@ -299,7 +329,8 @@ __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, 
     int pos = 0;
     if (g.epilogue == kEpiQKV) pos = __ldcg(g.row_pos + grow);     // independent of the sums: overlaps their loads
     float lo[16], hi[16];
-    sum_slots16(g.partial, p, t, c_first, c_last, pc0, pc1, row, lo, hi);
+    if (pc1 < 0) sum_slots16_single(g.partial, p, t, c_first, c_last, pc0, row, lo);
+    else sum_slots16(g.partial, p, t, c_first, c_last, pc0, pc1, row, lo, hi);
     if (g.epilogue == kEpiResidual) {
         out_residual<16>(g, grow, nt * TC_BN + item * 16, lo);
     } else if (g.epilogue == kEpiLogits) {
