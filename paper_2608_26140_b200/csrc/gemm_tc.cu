@@ -328,11 +328,21 @@ __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, 
     }
     int pos = 0;
     if (g.epilogue == kEpiQKV) pos = __ldcg(g.row_pos + grow);     // independent of the sums: overlaps their loads
+    uint4 res[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+    if (g.epilogue == kEpiResidual) {                              // so is the residual row (its offset first)
+        const int64_t roff = g.resid_off ? __ldcg(g.resid_off + grow) : (int64_t)grow * g.n[0];
+        const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(g.resid) + roff + nt * TC_BN + item * 16);
+        res[0] = __ldcg(rp); res[1] = __ldcg(rp + 1);
+    }
     float lo[16], hi[16];
     if (pc1 < 0) sum_slots16_single(g.partial, p, t, c_first, c_last, pc0, row, lo);
     else sum_slots16(g.partial, p, t, c_first, c_last, pc0, pc1, row, lo, hi);
     if (g.epilogue == kEpiResidual) {
-        out_residual<16>(g, grow, nt * TC_BN + item * 16, lo);
+        const uint32_t rw[8] = {res[0].x, res[0].y, res[0].z, res[0].w, res[1].x, res[1].y, res[1].z, res[1].w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { lo[2 * i] += bf16_lo(rw[i]); lo[2 * i + 1] += bf16_hi(rw[i]); }
+        uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(g.c) + (int64_t)grow * g.n[0] + nt * TC_BN + item * 16);
+        o[0] = pack8(lo); o[1] = pack8(lo + 8);
     } else if (g.epilogue == kEpiLogits) {
         float m = -INFINITY, sm = 0.f;
         int arg = 0;
