@@ -112,8 +112,9 @@ acache_status check_weights(acache_ctx* c, const acache_layer_weights* w, bool q
 
 // Q for the masked rows, then Eq. 4-5.
 acache_status run_score(acache_ctx* c, const acache_request* r, const void* q_mask, const acache_kv* kv,
-                        float* scores, int accumulate, int norm_full, int defer_head_sum, cudaStream_t st) {
+                        float* scores, int accumulate, int norm_full, int defer_head_sum, cudaStream_t st, int early_k = 0) {
     ScoreArgs a{};
+    a.early_k = early_k;
     a.q_mask = q_mask;
     a.cache_k = kv->k;
     a.kv_batch_stride = kv->batch_stride;
@@ -534,8 +535,10 @@ acache_status layer_step_impl(acache_ctx* ctx, const acache_layer_weights* w, co
         // (only while one CTA per request can read all heads' partial sums quickly: at L = 8192 the separate,
         // grid-wide head sum takes 4 us where the folded one took 28)
         fused_head_sum = do_select && k > 0 && req->n_masked > 0 && (int64_t)req->affix_len * d.n_heads <= 65536;
+        // the masked rows' projection was launched just above: nothing that writes the cache is the scoring kernels'
+        // direct predecessor, so they may request their first key tiles early
         s = run_score(ctx, req, qmask, kv, scores, (flags & ACACHE_F_ACCUMULATE) ? 1 : 0,
-                      (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, fused_head_sum ? 1 : 0, stream);
+                      (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, fused_head_sum ? 1 : 0, stream, req->n_masked > 0 ? 1 : 0);
         if (s != ACACHE_OK) return s;
     }
     if (do_select && k > 0 && req->batch > 0) {

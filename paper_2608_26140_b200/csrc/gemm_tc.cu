@@ -306,34 +306,50 @@ __host__ __device__ __forceinline__ int finish_items_per_tile(int epilogue) {
 }
 
 // Finish of one work item of split tile t = nt * m_tiles + mt for tile row `row`.
-__device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, int t, int item, int row) {
-    const int nt = t / p.m_tiles, mt = t - nt * p.m_tiles;
-    const int grow = mt * TC_BM + row;
-    int c_first, c_last;
-    tile_cover(p, t, c_first, c_last);
+// The row's 32 bytes of residual under an item's 16 columns (kEpiResidual).
+__device__ __forceinline__ void load_residual16(const GemmArgs& g, int grow, int col, uint4 (&res)[2]) {
+    const int64_t roff = g.resid_off ? __ldcg(g.resid_off + grow) : (int64_t)grow * g.n[0];
+    const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(g.resid) + roff + col);
+    res[0] = __ldcg(rp); res[1] = __ldcg(rp + 1);
+}
+
+// Where an item of the finish lives: everything that can be worked out before the projection has finished.
+struct FinishItem {
+    int nt, grow, c_first, c_last, pc0, pc1, u128, lo_col;
+    bool skip;
+};
+__device__ __forceinline__ FinishItem finish_plan(const GemmArgs& g, const TcPlan& p, int t, int item, int row) {
+    FinishItem f;
+    f.nt = t / p.m_tiles;
+    f.grow = (t - f.nt * p.m_tiles) * TC_BM + row;
+    tile_cover(p, t, f.c_first, f.c_last);
     const int half = g.head_dim >> 1;
-    int pc0, pc1 = -1, u128 = 0, lo_col = 0;
+    f.pc1 = -1; f.u128 = 0; f.lo_col = 0; f.skip = false;
     if (g.epilogue == kEpiResidual || g.epilogue == kEpiLogits) {
-        pc0 = item * 4;
-        if (g.epilogue == kEpiLogits && nt * 2 + (item >> 3) >= p.units) return;   // past the vocabulary's end
+        f.pc0 = item * 4;
+        if (g.epilogue == kEpiLogits && f.nt * 2 + (item >> 3) >= p.units) f.skip = true;   // past the vocabulary's end
     } else if (g.epilogue == kEpiSwiGLU) {
-        pc0 = item * 4; pc1 = 32 + pc0;
+        f.pc0 = item * 4; f.pc1 = 32 + f.pc0;
     } else {
         const int h = item >> 2, r = item & 3;
-        u128 = nt * 2 + h;
-        if (u128 >= p.units) return;                                      // the tile's second half is past the end
-        lo_col = g.head_dim == 128 ? 16 * r : 64 * (r >> 1) + 16 * (r & 1);   // column inside the 128-wide unit
-        pc0 = 32 * h + (lo_col >> 2);
-        pc1 = pc0 + (half >> 2);
+        f.u128 = f.nt * 2 + h;
+        if (f.u128 >= p.units) f.skip = true;                                 // the tile's second half is past the end
+        f.lo_col = g.head_dim == 128 ? 16 * r : 64 * (r >> 1) + 16 * (r & 1);   // column inside the 128-wide unit
+        f.pc0 = 32 * h + (f.lo_col >> 2);
+        f.pc1 = f.pc0 + (half >> 2);
     }
+    return f;
+}
+
+// res: the residual, loaded by the caller (kEpiResidual only).
+__device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, int t, int item, int row, const FinishItem& f,
+                                            const uint4 (&res)[2]) {
+    if (f.skip) return;
+    const int nt = f.nt, grow = f.grow, c_first = f.c_first, c_last = f.c_last, pc0 = f.pc0, pc1 = f.pc1, u128 = f.u128,
+              lo_col = f.lo_col;
+    const int half = g.head_dim >> 1;
     int pos = 0;
     if (g.epilogue == kEpiQKV) pos = __ldcg(g.row_pos + grow);     // independent of the sums: overlaps their loads
-    uint4 res[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
-    if (g.epilogue == kEpiResidual) {                              // so is the residual row (its offset first)
-        const int64_t roff = g.resid_off ? __ldcg(g.resid_off + grow) : (int64_t)grow * g.n[0];
-        const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(g.resid) + roff + nt * TC_BN + item * 16);
-        res[0] = __ldcg(rp); res[1] = __ldcg(rp + 1);
-    }
     float lo[16], hi[16];
     if (pc1 < 0) sum_slots16_single(g.partial, p, t, c_first, c_last, pc0, row, lo);
     else sum_slots16(g.partial, p, t, c_first, c_last, pc0, pc1, row, lo, hi);
@@ -993,15 +1009,25 @@ struct SplitTiles {
 };
 
 __global__ void __launch_bounds__(256, 2) gemm_finish_kernel(const GemmArgs g, const TcPlan p, const SplitTiles split) {
-    pdl_wait();
-    pdl_launch_dependents();
     const int t = split.tile[blockIdx.y];
     const int mt = t % p.m_tiles;
     const int rows_per = p.m_tiles == 1 ? ((g.M + 31) & ~31) : TC_BM;
     const int w = blockIdx.x * 256 + threadIdx.x;
     const int row = w % rows_per, item = w / rows_per;
-    if (item >= finish_items_per_tile(g.epilogue) || mt * TC_BM + row >= g.M) return;
-    finish_item(g, p, t, item, row);
+    const bool active = item < finish_items_per_tile(g.epilogue) && mt * TC_BM + row < g.M;
+    // The residual rows and their offsets are outputs of kernels that had completed before the projection
+    // whose tiles are finished here passed its own dependency wait, and this kernel starts after that: they can
+    // be requested while the projection is still running.
+    uint4 res[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+    FinishItem f{};
+    if (active) {
+        f = finish_plan(g, p, t, item, row);
+        if (g.epilogue == kEpiResidual) load_residual16(g, f.grow, f.nt * TC_BN + item * 16, res);
+    }
+    pdl_wait();
+    pdl_launch_dependents();
+    if (!active) return;
+    finish_item(g, p, t, item, row, f, res);
 }
 
 // ---- predict and commit (Eq. 2-3): confidence and arg max per row, commit rule per request ------

@@ -48,6 +48,8 @@ struct ScoreArgs {
     int accumulate;
     int defer_head_sum;       // leave head_partial unsummed: launch_topk(.., head_partial) does it
     uint32_t* status;         // device status word (bounded waits of the tensor-core kernels); may be null
+    int early_k;              // the cache was last written at least two kernels back on this stream: its first
+                              // key tiles may be requested before the wait for the producer of q_mask
 };
 // tcgen05 kernels for head dimension 128 and up to 256 masked rows (two passes into row_stats / head_partial);
 // 0 = not applicable, -1 = launch failed.  Their statistics use one entry per score_tc_splits() keys.

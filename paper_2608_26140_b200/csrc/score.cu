@@ -74,8 +74,6 @@ __global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_spl
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int TILE = 64 * D * 2;
     const uint32_t sQ = smem_u32(smem), sK0 = sQ + TILE;
-    pdl_wait();
-    pdl_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int split = blockIdx.y, h = blockIdx.x;     // heads fastest: CTAs running together read whole K rows
     const int mtiles = (a.m + 63) / 64;
@@ -90,8 +88,13 @@ __global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_spl
                                  (int64_t)(a.norm_lo + key_lo) * kstride + (int64_t)kvh * D;
     const int ntiles = (key_n + 63) / 64;
 
+    // early_k: the cache was last written at least two kernels back (the layer-step: the masked rows' projection
+    // sits in between), so the first key tile can be requested while the producer of Q is still running
+    if (a.early_k) load_tile64<D>(sK0, kbase, kstride, min(64, key_n), tid, 128);
+    pdl_wait();
+    pdl_launch_dependents();
     load_tile64<D>(sQ, q, qstride, min(64, a.m - mt * 64), tid, 128);
-    load_tile64<D>(sK0, kbase, kstride, min(64, key_n), tid, 128);
+    if (!a.early_k) load_tile64<D>(sK0, kbase, kstride, min(64, key_n), tid, 128);
     cp_async_commit();
     cp_async_wait<0>();
     __syncthreads();
@@ -165,8 +168,6 @@ __global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_sp
     const uint32_t sK0 = smem_u32(smem), sQ0 = sK0 + 2 * TILE;
     float* s_max = reinterpret_cast<float*>(smem + 4 * TILE);
     float* s_inv = s_max + a.m;
-    pdl_wait();
-    pdl_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = blockIdx.x, b = blockIdx.z;                     // heads fastest (see the statistics pass)
     const int kvh = h / (a.n_heads / a.n_kv_heads);
@@ -179,7 +180,12 @@ __global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_sp
                                  (int64_t)a.affix_start * kstride + (int64_t)kvh * D;
     const int mtiles = (a.m + 63) / 64;
 
-    load_tile64<D>(sK0, kbase + (int64_t)jt_first * 64 * kstride, kstride, min(64, a.affix_len - jt_first * 64), tid, 128);
+    if (a.early_k)
+        load_tile64<D>(sK0, kbase + (int64_t)jt_first * 64 * kstride, kstride, min(64, a.affix_len - jt_first * 64), tid, 128);
+    pdl_wait();
+    pdl_launch_dependents();
+    if (!a.early_k)
+        load_tile64<D>(sK0, kbase + (int64_t)jt_first * 64 * kstride, kstride, min(64, a.affix_len - jt_first * 64), tid, 128);
     load_tile64<D>(sQ0, q, qstride, min(64, a.m), tid, 128);
     cp_async_commit();
 
