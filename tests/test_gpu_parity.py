@@ -138,6 +138,12 @@ def check_against_oracle(dc, anchors, k_new, v_new, y, cache_k_bits, cache_v_bit
     (wl.TINY_GQA, 2, 0, 130, 31, 33, 33, "masked", 0.35),
     (MID128, 2, 4, 200, 30, 32, 32, "all", 0.1),
     (MID128, 1, 0, 64, 16, 16, 16, "none", 1.0),
+    # row counts at the edges of the attention kernels' 128-row query tiles (128, 129, 256, 257, 384 rows)
+    (MID128, 2, 0, 400, 8, 32, 32, "none", 0.32),
+    (MID128, 2, 0, 400, 8, 32, 32, "none", 0.3225),
+    (MID128, 2, 0, 400, 8, 32, 32, "none", 0.64),
+    (MID128, 2, 0, 400, 8, 32, 32, "none", 0.6425),
+    (MID128, 2, 0, 400, 8, 32, 32, "none", 0.96),
 ])
 def test_recompute_then_scatter(shape, B, pre, L, post, gen, m, extra, ratio):
     lay = wl.make_layout(B, pre, L, post, gen, m, extra)
