@@ -37,6 +37,43 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 __device__ __forceinline__ void rmsnorm_row(const uint4* __restrict__ xr, const uint4* __restrict__ g,
                                             uint4* __restrict__ out, int hidden, float eps, float* red) {
     const int nchunk = hidden >> 3;
+    if (nchunk <= 3 * (int)blockDim.x) {
+        // the row fits in three 16-byte pieces per thread: one pass, the row stays in registers, and the gain is
+        // requested before the block-wide sum so that it arrives meanwhile
+        uint4 u[3], gg[3];
+        float ss1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const int c = threadIdx.x + i * blockDim.x;
+            u[i] = c < nchunk ? __ldcg(xr + c) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const int c = threadIdx.x + i * blockDim.x;
+            gg[i] = c < nchunk ? g[c] : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { const float a = bf16_lo(w[e]), b = bf16_hi(w[e]); ss1 += a * a + b * b; }
+        }
+        const float rstd1 = rsqrtf(block_sum(ss1, red) / (float)hidden + eps);
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const int c = threadIdx.x + i * blockDim.x;
+            if (c < nchunk) {
+                const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+                const uint32_t gw[4] = {gg[i].x, gg[i].y, gg[i].z, gg[i].w};
+                uint32_t r[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    r[e] = pack_bf16(bf16_lo(w[e]) * rstd1 * bf16_lo(gw[e]), bf16_hi(w[e]) * rstd1 * bf16_hi(gw[e]));
+                out[c] = make_uint4(r[0], r[1], r[2], r[3]);
+            }
+        }
+        return;
+    }
     float ss = 0.f;
     for (int c = threadIdx.x; c < nchunk; c += blockDim.x) {
         uint4 u = __ldcg(xr + c);
