@@ -69,7 +69,14 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(float* scores, int L
             float v = 0.f;
             const float* hp = head_partial + (int64_t)b * n_heads * L + j;
             int h = 0;
-            for (; h + 8 <= n_heads; h += 8) {      // 8 loads in flight, added in head order
+            for (; h + 32 <= n_heads; h += 32) {    // 32 loads in flight (one trip to L2), added in head order
+                float t[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) t[i] = __ldcg(hp + (int64_t)(h + i) * L);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v += t[i];
+            }
+            for (; h + 8 <= n_heads; h += 8) {
                 float t[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) t[i] = __ldcg(hp + (int64_t)(h + i) * L);
@@ -77,12 +84,14 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(float* scores, int L
                 for (int i = 0; i < 8; ++i) v += t[i];
             }
             for (; h < n_heads; ++h) v += __ldcg(hp + (int64_t)h * L);
-            s[j] = accumulate ? s[j] + v : v;
+            const float f = accumulate ? s[j] + v : v;
+            s[j] = f;
+            if (use_smem) keys_s[j] = score_key(f);          // the selection reads the keys from shared memory
         }
         __syncthreads();
-    }
-    if (use_smem)
+    } else if (use_smem) {
         for (int j = tid; j < L; j += kTopkThreads) keys_s[j] = score_key(s[j]);
+    }
     if (tid == 0) { s_prefix = 0u; s_want = K; }
     __syncthreads();
     auto key_at = [&](int j) -> uint32_t { return use_smem ? keys_s[j] : score_key(s[j]); };
