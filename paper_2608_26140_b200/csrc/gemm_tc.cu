@@ -221,16 +221,17 @@ __device__ __forceinline__ int64_t slot_of(const TcPlan& p, int t, int c) {
 // starting at column group pc0 and, if pc1 >= 0, 16 more starting at pc1.  Loads are issued two
 // CTAs at a time for all eight column groups (16 independent 16-byte loads in flight per thread)
 // and added in ascending CTA order, which keeps the result bitwise reproducible.
+template <int NC>      // contributing CTAs per round of loads: 2, or 4 where the kernel may use 255 registers
 __device__ __forceinline__ void sum_slots16(const float* __restrict__ partial, const TcPlan& p, int t, int c_first,
                                             int c_last, int pc0, int pc1, int row, float (&lo)[16], float (&hi)[16]) {
 #pragma unroll
     for (int i = 0; i < 16; ++i) { lo[i] = 0.f; hi[i] = 0.f; }
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
     const int o0 = pc0 * TC_BM + row, o1 = (pc1 < 0 ? pc0 : pc1) * TC_BM + row;
-    for (int c = c_first; c <= c_last; c += 2) {
-        float4 a[2][4], b[2][4];
+    for (int c = c_first; c <= c_last; c += NC) {
+        float4 a[NC][4], b[NC][4];
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < NC; ++i) {
             const bool in = c + i <= c_last;
             const float4* src = reinterpret_cast<const float4*>(partial) + slot_of(p, t, in ? c + i : c) * (TC_SLOT_FLOATS / 4);
 #pragma unroll
@@ -240,7 +241,7 @@ __device__ __forceinline__ void sum_slots16(const float* __restrict__ partial, c
             }
         }
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < NC; ++i) {
             if (c + i <= c_last) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -342,6 +343,7 @@ __device__ __forceinline__ FinishItem finish_plan(const GemmArgs& g, const TcPla
 }
 
 // res: the residual, loaded by the caller (kEpiResidual only).
+template <int NC>
 __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, int t, int item, int row, const FinishItem& f,
                                             const uint4 (&res)[2]) {
     if (f.skip) return;
@@ -352,7 +354,7 @@ __device__ __forceinline__ void finish_item(const GemmArgs& g, const TcPlan& p, 
     if (g.epilogue == kEpiQKV) pos = __ldcg(g.row_pos + grow);     // independent of the sums: overlaps their loads
     float lo[16], hi[16];
     if (pc1 < 0) sum_slots16_single(g.partial, p, t, c_first, c_last, pc0, row, lo);
-    else sum_slots16(g.partial, p, t, c_first, c_last, pc0, pc1, row, lo, hi);
+    else sum_slots16<NC>(g.partial, p, t, c_first, c_last, pc0, pc1, row, lo, hi);
     if (g.epilogue == kEpiResidual) {
         const uint32_t rw[8] = {res[0].x, res[0].y, res[0].z, res[0].w, res[1].x, res[1].y, res[1].z, res[1].w};
 #pragma unroll
@@ -1008,7 +1010,10 @@ struct SplitTiles {
     int tile[160];     // one per CTA boundary that cuts a tile (at most SM count - 1)
 };
 
-__global__ void __launch_bounds__(256, 2) gemm_finish_kernel(const GemmArgs g, const TcPlan p, const SplitTiles split) {
+// NC = 4 (255 registers, one block per SM) serves finishes of at most one block per SM with two column groups per
+// item: the masked rows' query projection has nine or ten contributors per tile and every round is a trip to L2.
+template <int NC>
+__global__ void __launch_bounds__(256, NC == 2 ? 2 : 1) gemm_finish_kernel(const GemmArgs g, const TcPlan p, const SplitTiles split) {
     const int t = split.tile[blockIdx.y];
     const int mt = t % p.m_tiles;
     const int rows_per = p.m_tiles == 1 ? ((g.M + 31) & ~31) : TC_BM;
@@ -1027,7 +1032,7 @@ __global__ void __launch_bounds__(256, 2) gemm_finish_kernel(const GemmArgs g, c
     pdl_wait();
     pdl_launch_dependents();
     if (!active) return;
-    finish_item(g, p, t, item, row, f, res);
+    finish_item<NC>(g, p, t, item, row, f, res);
 }
 
 // ---- predict and commit (Eq. 2-3): confidence and arg max per row, commit rule per request ------
@@ -1289,7 +1294,7 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
         if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, g, pp, clusters, *mA, *mB[0], *mB[1], *mB[2]) != cudaSuccess) return -1;
         if (split.n == 0) return 1;
         const int per_tile = finish_items_per_tile(g.epilogue) * TC_BM;
-        if (launch_pdl(gemm_finish_kernel, dim3((per_tile + 255) / 256, split.n), dim3(256), 0, stream, g, pp, split) != cudaSuccess)
+        if (launch_pdl(gemm_finish_kernel<2>, dim3((per_tile + 255) / 256, split.n), dim3(256), 0, stream, g, pp, split) != cudaSuccess)
             return -1;
         return 2;
     }
@@ -1310,8 +1315,10 @@ single_cta:
     if (split.n == 0) return 1;
     const int rows_per = p.m_tiles == 1 ? ((g.M + 31) & ~31) : TC_BM;
     const int per_tile = finish_items_per_tile(g.epilogue) * rows_per;
-    if (launch_pdl(gemm_finish_kernel, dim3((per_tile + 255) / 256, split.n), dim3(256), 0, stream, g, p, split) !=
-        cudaSuccess)
+    const dim3 fgrid((per_tile + 255) / 256, split.n);
+    const bool wide = g.epilogue == kEpiQKV && (int)(fgrid.x * fgrid.y) <= sm_count();
+    if ((wide ? launch_pdl(gemm_finish_kernel<4>, fgrid, dim3(256), 0, stream, g, p, split)
+              : launch_pdl(gemm_finish_kernel<2>, fgrid, dim3(256), 0, stream, g, p, split)) != cudaSuccess)
         return -1;
     return 2;
 }
