@@ -90,11 +90,17 @@ __global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_spl
 
     // early_k: the cache was last written at least two kernels back (the layer-step: the masked rows' projection
     // sits in between), so the first key tile can be requested while the producer of Q is still running
-    if (a.early_k) load_tile64<D>(sK0, kbase, kstride, min(64, key_n), tid, 128);
+    // all of the CTA's key tiles (at most kScoreSplit / 64 = 4) are requested at once: one trip to memory instead
+    // of one per tile; with early_k (see ScoreArgs) before the wait for the producer of Q
+    auto load_keys = [&]() {
+        for (int t = 0; t < ntiles; ++t)
+            load_tile64<D>(sK0 + t * TILE, kbase + (int64_t)t * 64 * kstride, kstride, min(64, key_n - t * 64), tid, 128);
+    };
+    if (a.early_k) load_keys();
     pdl_wait();
     pdl_launch_dependents();
     load_tile64<D>(sQ, q, qstride, min(64, a.m - mt * 64), tid, 128);
-    if (!a.early_k) load_tile64<D>(sK0, kbase, kstride, min(64, key_n), tid, 128);
+    if (!a.early_k) load_keys();
     cp_async_commit();
     cp_async_wait<0>();
     __syncthreads();
@@ -103,12 +109,7 @@ __global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_spl
 
     float mx[2] = {-INFINITY, -INFINITY}, den[2] = {0.f, 0.f};
     for (int t = 0; t < ntiles; ++t) {
-        const uint32_t sK = sK0 + (t & 1) * TILE;
-        if (t + 1 < ntiles) {
-            load_tile64<D>(sK0 + ((t + 1) & 1) * TILE, kbase + (int64_t)(t + 1) * 64 * kstride, kstride,
-                           min(64, key_n - (t + 1) * 64), tid, 128);
-            cp_async_commit();
-        }
+        const uint32_t sK = sK0 + t * TILE;
         float acc[8][4];
         mma_16x64<D>(acc, af, sK, lane);
         const int valid = key_n - t * 64;
@@ -141,8 +142,6 @@ __global__ void __launch_bounds__(128) score_stats_kernel(ScoreArgs a, int n_spl
             part[r] += __shfl_xor_sync(0xffffffffu, part[r], 2);
             den[r] += part[r];
         }
-        if (t + 1 < ntiles) cp_async_wait<0>();
-        __syncthreads();
     }
     if ((lane & 3) == 0) {
 #pragma unroll
@@ -270,7 +269,7 @@ static int launch_score_d(const ScoreArgs& a, cudaStream_t stream) {
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)D);
     constexpr int TILE = 64 * D * 2;
     const int mtiles = (a.m + 63) / 64;
-    const size_t smem1 = 3 * TILE;
+    const size_t smem1 = (1 + kScoreSplit / 64) * TILE;      // the Q tile and all of a split's key tiles
     const size_t smem2 = 4 * TILE + (size_t)a.m * 8;
     const int key_tiles = (a.affix_len + 63) / 64;
     // several key tiles per CTA only while that still leaves a few waves of CTAs (measured: L = 512, B = 1 is
