@@ -9,6 +9,7 @@
 //   3. ordered sum over heads into scores.
 // Logits run on the tensor cores (bf16 mma.sync, fp32 accumulate) so that the pass stays
 // bound by the K_affix read, not by ALU work.
+#include <cooperative_groups.h>
 #include "../../include/acache.h"
 #include "common.cuh"
 #include "kernels.h"
@@ -248,6 +249,147 @@ __global__ void __launch_bounds__(128) score_colsum_kernel(ScoreArgs a, int n_sp
     }
 }
 
+// ---- both passes in one launch: short affixes, one request or a few ----------------------------------
+// With at most 1024 affix keys a head's work is cut over a cluster of eight CTAs, 64 or 128 keys each: every CTA takes
+// the softmax statistics of all masked rows over its own keys, the four parts meet through distributed shared
+// memory, and each CTA then takes the column sums of its own keys from the tiles it already holds.  One launch
+// instead of two, and the statistics never leave the cluster.  Only when the normaliser runs over the affix
+// keys themselves and the grid fits the SMs in one wave.
+constexpr int kSmallCluster = 8;
+
+template <int D, int kSmallTiles>          // key tiles per CTA: 1 (up to 512 affix keys) or 2 (up to 1024)
+__global__ void __cluster_dims__(kSmallCluster, 1, 1) __launch_bounds__(128) score_small_kernel(ScoreArgs a, float scale_log2e) {
+    namespace cg = cooperative_groups;
+    extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int TILE = 64 * D * 2;
+    const uint32_t sQ = smem_u32(smem), sK0 = sQ + TILE;
+    float* s_stat = reinterpret_cast<float*>(smem + (1 + kSmallTiles) * TILE);     // [tile][64 rows][max, den]
+    float* s_max = s_stat + kSmallTiles * 128;
+    float* s_inv = s_max + 64;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rank = blockIdx.x % kSmallCluster, h = blockIdx.x / kSmallCluster, b = blockIdx.y;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int64_t qstride = (int64_t)a.n_heads * D, kstride = (int64_t)a.n_kv_heads * D;
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.q_mask) + (int64_t)b * a.m * qstride + (int64_t)h * D;
+    const int key0 = rank * kSmallTiles * 64;                                      // first affix key of this CTA
+    const __nv_bfloat16* kbase = static_cast<const __nv_bfloat16*>(a.cache_k) + (int64_t)b * a.kv_batch_stride +
+                                 (int64_t)(a.affix_start + key0) * kstride + (int64_t)kvh * D;
+    const int nkeys = max(0, min(kSmallTiles * 64, a.affix_len - key0));
+    const int ntiles = (nkeys + 63) / 64;
+    auto load_keys = [&]() {
+        for (int t = 0; t < ntiles; ++t)
+            load_tile64<D>(sK0 + t * TILE, kbase + (int64_t)t * 64 * kstride, kstride, min(64, nkeys - t * 64), tid, 128);
+    };
+    if (a.early_k) load_keys();          // see ScoreArgs::early_k
+    pdl_wait();
+    pdl_launch_dependents();
+    load_tile64<D>(sQ, q, qstride, min(64, a.m), tid, 128);
+    if (!a.early_k) load_keys();
+    cp_async_commit();
+    cp_async_wait<0>();
+    __syncthreads();
+
+    // pass 1: warp w takes the 16-row group (w & 1) [+ 2 in a second round] over key tile w >> 1
+    const int groups = (a.m + 15) / 16;
+    constexpr int WPT = 4 / kSmallTiles;      // warps per key tile
+    for (int g0 = 0; g0 < groups; g0 += WPT) {
+        const int rg = g0 + warp % WPT, t = warp / WPT;
+        if (rg >= groups) continue;
+        float mx[2] = {-INFINITY, -INFINITY}, den[2] = {0.f, 0.f};
+        if (t < ntiles) {
+            uint32_t af[D / 16][4];
+            load_a_frags<D>(af, sQ, rg * 16, lane);
+            float acc[8][4];
+            mma_16x64<D>(acc, af, sK0 + t * TILE, lane);
+            const int valid = nkeys - t * 64;
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int col = nb * 8 + (lane & 3) * 2 + (i & 1);
+                    const float sc = col < valid ? acc[nb][i] * scale_log2e : -INFINITY;
+                    acc[nb][i] = sc;
+                    mx[i >> 1] = fmaxf(mx[i >> 1], sc);
+                }
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+            }
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) den[i >> 1] += exp2f(acc[nb][i] - mx[i >> 1]);
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                den[r] += __shfl_xor_sync(0xffffffffu, den[r], 1);
+                den[r] += __shfl_xor_sync(0xffffffffu, den[r], 2);
+            }
+        }
+        if ((lane & 3) == 0) {
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int row = rg * 16 + (lane >> 2) + r * 8;
+                s_stat[(t * 64 + row) * 2] = mx[r];
+                s_stat[(t * 64 + row) * 2 + 1] = den[r];
+            }
+        }
+    }
+    cluster.sync();
+    if (tid < groups * 16) {
+        float ms[kSmallCluster * kSmallTiles], ds[kSmallCluster * kSmallTiles];
+#pragma unroll
+        for (int c = 0; c < kSmallCluster; ++c) {
+            const float* remote = cluster.map_shared_rank(s_stat, c);
+#pragma unroll
+            for (int t = 0; t < kSmallTiles; ++t) {
+                const float2 v = *reinterpret_cast<const float2*>(remote + (t * 64 + tid) * 2);
+                ms[c * kSmallTiles + t] = v.x;
+                ds[c * kSmallTiles + t] = v.y;
+            }
+        }
+        float M = -INFINITY, Dn = 0.f;
+#pragma unroll
+        for (int i = 0; i < kSmallCluster * kSmallTiles; ++i) M = fmaxf(M, ms[i]);
+#pragma unroll
+        for (int i = 0; i < kSmallCluster * kSmallTiles; ++i)
+            if (ms[i] != -INFINITY) Dn += ds[i] * exp2f(ms[i] - M);
+        s_max[tid] = M;
+        s_inv[tid] = 1.f / Dn;
+    }
+    __syncthreads();
+
+    // pass 2: column sums of the normalised weights over this CTA's keys, 16 keys of every tile per warp
+    for (int kt = 0; kt < ntiles; ++kt) {
+        uint32_t af[D / 16][4];
+        load_a_frags<D>(af, sK0 + kt * TILE, warp * 16, lane);
+        float acc[8][4];
+        mma_16x64<D>(acc, af, sQ, lane);       // rows = keys, cols = masked queries
+        float colsum[2] = {0.f, 0.f};
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int qrow = nb * 8 + (lane & 3) * 2 + (i & 1);
+                if (qrow < a.m) colsum[i >> 1] += exp2f(acc[nb][i] * scale_log2e - s_max[qrow]) * s_inv[qrow];
+            }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            colsum[r] += __shfl_xor_sync(0xffffffffu, colsum[r], 1);
+            colsum[r] += __shfl_xor_sync(0xffffffffu, colsum[r], 2);
+        }
+        if ((lane & 3) == 0) {
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int j = key0 + kt * 64 + warp * 16 + (lane >> 2) + r * 8;
+                if (j < a.affix_len) a.head_partial[((int64_t)b * a.n_heads + h) * a.affix_len + j] = colsum[r];
+            }
+        }
+    }
+    cluster.sync();        // no CTA leaves while a neighbour may still read its statistics
+}
+
 // ---- pass 3: ordered sum over heads -------------------------------------------------------
 __global__ void __launch_bounds__(256) score_reduce_heads_kernel(const float* __restrict__ head_partial,
                                                                  float* __restrict__ scores, int n_heads, int L,
@@ -276,6 +418,19 @@ static int launch_score_d(const ScoreArgs& a, cudaStream_t stream) {
     // faster with one tile per CTA, L = 8192 with four)
     const int64_t ctas1 = (int64_t)a.n_heads * key_tiles * a.batch;
     const int kt_per_cta = mtiles > 1 ? 1 : ctas1 >= 2400 ? 4 : ctas1 >= 1200 ? 2 : 1;
+    static const bool small_on = [] { const char* e = getenv("ACACHE_SCORE_SMALL"); return !e || atoi(e) != 0; }();
+    if (small_on && a.norm_lo == a.affix_start && a.norm_len == a.affix_len && a.affix_len <= 128 * kSmallCluster && a.m <= 64 &&
+        a.n_heads * a.batch <= 148) {
+        const int tpc = a.affix_len <= 64 * kSmallCluster ? 1 : 2;
+        const size_t smem0 = (size_t)(1 + tpc) * TILE + (tpc * 128 + 128) * sizeof(float);
+        auto kernel = tpc == 1 ? score_small_kernel<D, 1> : score_small_kernel<D, 2>;
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem0);
+        launch_pdl(kernel, dim3(a.n_heads * kSmallCluster, a.batch), 128, smem0, stream, a, scale_log2e);
+        if (a.defer_head_sum) return 1;
+        launch_pdl(score_reduce_heads_kernel, dim3((a.affix_len + 255) / 256, a.batch), 256, 0, stream, a.head_partial,
+                   a.scores, a.n_heads, a.affix_len, a.accumulate);
+        return 2;
+    }
     cudaFuncSetAttribute(score_stats_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
     cudaFuncSetAttribute(score_colsum_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
     launch_pdl(score_stats_kernel<D>, dim3(a.n_heads, n_split, a.batch * mtiles), 128, smem1, stream, a, n_split,

@@ -29,6 +29,11 @@ def dev_i32(a):
     (MID128, 1, 0, 1, 64, 3, False),           # one affix token
     (MID128, 1, 7, 700, 64, 130, True),
     (wl.LLADA_8B, 1, 0, 512, 256, 32, False),
+    # short affixes scored by the one-launch cluster kernel: one or two key tiles per CTA, one to four row groups
+    (wl.TINY, 1, 4, 450, 20, 50, False),
+    (MID128, 2, 3, 1000, 20, 64, False),
+    (MID128, 1, 0, 1024, 8, 17, False),
+    (MID128, 2, 0, 65, 8, 64, False),
 ])
 def test_score_anchors(shape, B, pre, L, post, m, norm_full):
     lay = wl.make_layout(B, pre, L, post, max(m, 1), m)
