@@ -577,7 +577,7 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     int prefilled = 0;
     if (warp == 0 && lane == 0) {
         const CUtensorMap* maps[3] = {&mapB0, &mapB1, &mapB2};
-        const uint64_t pol_w = policy_evict_first();
+        const uint64_t pol_w = g.keep_weights ? policy_evict_last() : policy_evict_first();
         for (int i = 0; i < TC_STAGES + kPrefetchL2 && it0 + i < it1; ++i) {
             const int it = it0 + i, t = it / p.KB, kb = it - t * p.KB, nt = t / p.m_tiles;
             int row0, row1;
@@ -609,7 +609,7 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
         int stage = 0;
         uint32_t phase = 0;
         bool ok = !*abort_flag;
-        const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
+        const uint64_t pol_a = policy_evict_last(), pol_w = g.keep_weights ? pol_a : policy_evict_first();
         for (int it = it0; it < it1 && ok;) {
             const int t = it / p.KB, kb0 = it - t * p.KB;
             const int kb1 = min(p.KB, kb0 + (it1 - it));
@@ -875,7 +875,7 @@ gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __gr
         int stage = 0, issued = 0;
         uint32_t phase = 0;
         bool ok = !*abort_flag;
-        const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
+        const uint64_t pol_a = policy_evict_last(), pol_w = g.keep_weights ? pol_a : policy_evict_first();
         // work list: whole tiles round-robin (pair_u == 0), or this cluster's contiguous range of
         // (tile, K block) iterations, tiles in weight-tile-major order (stream-K)
         const long long it_end = p.pair_u ? min((long long)(cluster_id + 1) * p.pair_u, (long long)tiles * p.KB) : 0;

@@ -120,6 +120,8 @@ struct GemmArgs {
     // out[1] / out[2] (a decode pass refreshing some rows of a larger private slot array) instead of row i
     const int32_t* kv_out_rows;
     int kv_out_stride;
+    // the weights are read again by the next projection (the masked rows' queries before Q/K/V): keep them in L2
+    int keep_weights;
     // --- kEpiResidual ---
     const void* resid;        // bf16 base pointer
     const int64_t* resid_off; // [M] element offset of the residual row, or null => row * N
