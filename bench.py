@@ -282,7 +282,9 @@ def run_ours(args):
     e1.record()
     sync_all()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / args.steps
-    h2d = xh.numel() * 2
+    # page-locked x is read in place: the kernels pull the masked rows, the anchor rows and the anchors' residual rows
+    x_in_place = ctx.host_x_in_place(xh)
+    h2d = B * (lay.n_masked + 2 * n) * shape.hidden * 2 if x_in_place else xh.numel() * 2
     d2h = n * B * shape.hidden * 2 + B * K * 4 + B * L * 4
 
     if rank != 0:
@@ -314,7 +316,9 @@ def run_ours(args):
         "config": workload_config(shape, lay, args, K),
         "clocks": sampler.summary(),
         "e2e": {"value": world * B * K / (ms_e2e * 1e-3), "unit": UNIT, "us_per_layer_step": ms_e2e * 1e3,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "x_transfer": "rows read in place from page-locked host memory by the kernels" if x_in_place
+                else "whole x staged by one copy"},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "layer_step_roofline": {"bound": "hbm" if t_hbm >= t_tc else "tensor", "algorithmic_bytes": step_bytes,

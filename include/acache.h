@@ -417,12 +417,21 @@ acache_status acache_generate_block(acache_ctx *ctx, int32_t n_layers, const aca
  * runs the layer-step with ACACHE_F_SCORE | ACACHE_F_SELECT | flags, and copies y
  * [B, K+e, D], anchor_idx [B, K] and scores [B, L] back to the given HOST buffers.
  * Weights, cache and the request's index arrays stay DEVICE-resident.  All copies are
- * asynchronous on `stream`; the caller synchronises the stream before reading. */
+ * asynchronous on `stream`; the caller synchronises the stream before reading.
+ *   When x_host is page-locked (acache_host_x_in_place returns 1) it is not staged: the kernels read
+ *   the rows the step needs (masked rows, anchor rows and the anchors' residual rows: n_masked + 2 (K+e)
+ *   rows of D bf16 per request) in place over the bus, so x_host must stay valid and unchanged until the
+ *   stream has passed this call. */
 acache_status acache_layer_step_host(acache_ctx *ctx, const acache_layer_weights *w,
                                      const acache_request *req, acache_kv *kv,
                                      const void *x_host, double ratio, uint32_t flags,
                                      float *scores_host, int32_t *anchor_idx_host, void *y_host,
                                      acache_stream_t stream);
+
+/* 1 when acache_layer_step_host reads an x at this HOST address in place (page-locked memory the device
+ * can address), 0 when it stages a copy.  No GPU work; ACACHE_HOST_X_IN_PLACE=0 in the environment
+ * forces 0. */
+int32_t acache_host_x_in_place(const void *x_host);
 
 #ifdef __cplusplus
 }

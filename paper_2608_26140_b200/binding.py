@@ -24,7 +24,8 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_layer_step", "acache_layer_step_host", "acache_stage_timing", "acache_read_stage_times",
            "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step", "acache_probe_select",
            "acache_commit_update", "acache_generate_block", "acache_denoise_step_shared", "acache_recompute_rows_shared",
-           "acache_decode_step_shared", "acache_generate_block_shared", "acache_layer_step_shared"]
+           "acache_decode_step_shared", "acache_generate_block_shared", "acache_layer_step_shared",
+           "acache_host_x_in_place"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -104,6 +105,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_layer_step_host.argtypes = [vp, C.POINTER(LayerWeights), C.POINTER(Request), C.POINTER(KV), vp,
                                            C.c_double, u32, vp, vp, vp, vp]
     lib.acache_layer_step_host.restype = C.c_int
+    lib.acache_host_x_in_place.argtypes = [vp]
+    lib.acache_host_x_in_place.restype = C.c_int32
     lib.acache_score_anchors_static.argtypes = [C.POINTER(ModelDesc), C.POINTER(Request), vp, C.POINTER(KV), vp,
                                                 C.c_int, C.c_int, vp]
     lib.acache_score_anchors_static.restype = C.c_int
@@ -397,6 +400,11 @@ class Context:
         self._check(self.lib.acache_layer_step_host(self.h, C.byref(w), C.byref(req), C.byref(kv), _ptr(x_host),
                                                     float(ratio), int(flags), _ptr(scores_host),
                                                     _ptr(anchor_idx_host), _ptr(y_host), _stream()))
+
+
+    def host_x_in_place(self, x_host) -> bool:
+        """True when layer_step_host reads this x in place (page-locked memory) instead of staging a copy."""
+        return bool(self.lib.acache_host_x_in_place(_ptr(x_host)))
 
 
 # --------------------------------------------------------------------------

@@ -273,6 +273,15 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
 // single-layer entry points read it.  Thread-local: a context is used from one thread at a time.
 static thread_local bool g_reuse_maps = false;
 
+namespace {
+// Device-side address of page-locked host memory (nullptr for pageable or unknown memory).
+const void* mapped_device_pointer(const void* host) {
+    cudaPointerAttributes at{};
+    if (!host || cudaPointerGetAttributes(&at, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+}  // namespace
+
 extern "C" {
 
 acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
@@ -851,6 +860,11 @@ acache_status acache_generate_block(acache_ctx* ctx, int32_t n_layers, const aca
     return ACACHE_OK;
 }
 
+int32_t acache_host_x_in_place(const void* x_host) {
+    static const bool on = [] { const char* e = getenv("ACACHE_HOST_X_IN_PLACE"); return !e || atoi(e) != 0; }();
+    return on && mapped_device_pointer(x_host) != nullptr;
+}
+
 acache_status acache_layer_step_host(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
                                      acache_kv* kv, const void* x_host, double ratio, uint32_t flags,
                                      float* scores_host, int32_t* anchor_idx_host, void* y_host,
@@ -869,8 +883,14 @@ acache_status acache_layer_step_host(acache_ctx* ctx, const acache_layer_weights
     float* ss = wsp<float>(ctx, ctx->o_sstage);
     int32_t* as = wsp<int32_t>(ctx, ctx->o_astage);
     const size_t xb = (size_t)req->batch * req->ctx_len * d.hidden * 2;
-    if (cudaMemcpyAsync(xs, x_host, xb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return check_cuda(ctx, "H2D x");
-    acache_status s = acache_layer_step(ctx, w, req, kv, xs, 0, ratio, flags | ACACHE_F_SCORE | ACACHE_F_SELECT, ss, as,
+    // The step reads x row by row (the masked rows, the anchor rows and their residual), a small part of the
+    // whole: page-locked x is read in place over the bus by the kernels, anything else is staged whole.
+    const void* x_dev = acache_host_x_in_place(x_host) ? mapped_device_pointer(x_host) : nullptr;
+    if (!x_dev) {
+        if (cudaMemcpyAsync(xs, x_host, xb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return check_cuda(ctx, "H2D x");
+        x_dev = xs;
+    }
+    acache_status s = acache_layer_step(ctx, w, req, kv, x_dev, 0, ratio, flags | ACACHE_F_SCORE | ACACHE_F_SELECT, ss, as,
                                         ys, stream);
     if (s != ACACHE_OK) return s;
     const size_t rows = (size_t)req->batch * (k + req->n_extra);

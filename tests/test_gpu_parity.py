@@ -315,6 +315,16 @@ def test_host_buffer_entry_point():
     torch.cuda.synchronize()
     assert np.array_equal(sh.numpy(), s_dev) and np.array_equal(ah.numpy(), a_dev[:, :K])
     assert np.array_equal(ab.to_host_bits(yh), ab.to_host_bits(y_dev[:, :n]))
+    # page-locked x is read in place by the kernels, pageable x is staged by a copy: same results
+    assert dc.ctx.host_x_in_place(xh)
+    xp = torch.from_numpy(case.x.view(np.int16).copy()).view(torch.bfloat16)
+    assert not dc.ctx.host_x_in_place(xp)
+    dc.reset_cache()
+    sh2, ah2, yh2 = torch.zeros_like(sh), torch.zeros_like(ah), torch.zeros_like(yh)
+    dc.ctx.layer_step_host(dc.lw, dc.req, dc.kv(), xp, 0.2, 0, sh2, ah2, yh2)
+    torch.cuda.synchronize()
+    assert np.array_equal(sh2.numpy(), s_dev) and np.array_equal(ah2.numpy(), a_dev[:, :K])
+    assert np.array_equal(ab.to_host_bits(yh2), ab.to_host_bits(y_dev[:, :n]))
 
 
 def test_invalid_arguments_enqueue_nothing():
