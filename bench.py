@@ -283,7 +283,7 @@ def run_ours(args):
     sync_all()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / args.steps
     # page-locked x is read in place: the kernels pull the masked rows, the anchor rows and the anchors' residual rows
-    x_in_place = ctx.host_x_in_place(xh)
+    x_in_place = ctx.host_x_in_place(xh) and (lay.n_masked + 2 * n) * 4 <= T    # the entry point's own rule
     h2d = B * (lay.n_masked + 2 * n) * shape.hidden * 2 if x_in_place else xh.numel() * 2
     d2h = n * B * shape.hidden * 2 + B * K * 4 + B * L * 4
 

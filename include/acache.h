@@ -418,7 +418,8 @@ acache_status acache_generate_block(acache_ctx *ctx, int32_t n_layers, const aca
  * [B, K+e, D], anchor_idx [B, K] and scores [B, L] back to the given HOST buffers.
  * Weights, cache and the request's index arrays stay DEVICE-resident.  All copies are
  * asynchronous on `stream`; the caller synchronises the stream before reading.
- *   When x_host is page-locked (acache_host_x_in_place returns 1) it is not staged: the kernels read
+ *   When x_host is page-locked (acache_host_x_in_place returns 1) and the step needs at most a quarter of
+ *   its rows, it is not staged: the kernels read
  *   the rows the step needs (masked rows, anchor rows and the anchors' residual rows: n_masked + 2 (K+e)
  *   rows of D bf16 per request) in place over the bus, so x_host must stay valid and unchanged until the
  *   stream has passed this call. */

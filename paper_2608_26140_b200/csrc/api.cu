@@ -885,7 +885,10 @@ acache_status acache_layer_step_host(acache_ctx* ctx, const acache_layer_weights
     const size_t xb = (size_t)req->batch * req->ctx_len * d.hidden * 2;
     // The step reads x row by row (the masked rows, the anchor rows and their residual), a small part of the
     // whole: page-locked x is read in place over the bus by the kernels, anything else is staged whole.
-    const void* x_dev = acache_host_x_in_place(x_host) ? mapped_device_pointer(x_host) : nullptr;
+    // (in place only while those rows are at most a quarter of x: reads over the bus from a kernel are slower,
+    // byte for byte, than the copy engine's transfer)
+    const int64_t pulled = (int64_t)req->n_masked + 2 * ((int64_t)k + req->n_extra);
+    const void* x_dev = pulled * 4 <= req->ctx_len && acache_host_x_in_place(x_host) ? mapped_device_pointer(x_host) : nullptr;
     if (!x_dev) {
         if (cudaMemcpyAsync(xs, x_host, xb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return check_cuda(ctx, "H2D x");
         x_dev = xs;

@@ -300,18 +300,20 @@ def test_out_of_range_index_is_flagged_and_skipped():
     assert np.array_equal(ckb[0][keep], case.cache_k[0][keep])
 
 
-def test_host_buffer_entry_point():
-    lay = wl.make_layout(2, 0, 128, 32, 32, 32, "masked")
-    case = make_projected_case(wl.TINY, lay, 0.2, cfg_id=17)
+@pytest.mark.parametrize("extra,ratio", [("masked", 0.2),      # the step needs most of x: staged by one copy
+                                         ("none", 0.05)])      # 46 of 192 rows: page-locked x is read in place
+def test_host_buffer_entry_point(extra, ratio):
+    lay = wl.make_layout(2, 0, 128, 32, 32, 32, extra)
+    case = make_projected_case(wl.TINY, lay, ratio, cfg_id=17)
     dc = DeviceCase(case)
-    K, s_dev, a_dev, y_dev = run_layer_step(dc, 0.2, ab.F_SCORE | ab.F_SELECT)
+    K, s_dev, a_dev, y_dev = run_layer_step(dc, ratio, ab.F_SCORE | ab.F_SELECT)
     n = K + lay.n_extra
     dc.reset_cache()
     xh = torch.from_numpy(case.x.view(np.int16)).view(torch.bfloat16).pin_memory()
     sh = torch.zeros((2, 128), dtype=torch.float32).pin_memory()
     ah = torch.zeros((2, K), dtype=torch.int32).pin_memory()
     yh = torch.zeros((2, n, case.shape.hidden), dtype=torch.bfloat16).pin_memory()
-    dc.ctx.layer_step_host(dc.lw, dc.req, dc.kv(), xh, 0.2, 0, sh, ah, yh)
+    dc.ctx.layer_step_host(dc.lw, dc.req, dc.kv(), xh, ratio, 0, sh, ah, yh)
     torch.cuda.synchronize()
     assert np.array_equal(sh.numpy(), s_dev) and np.array_equal(ah.numpy(), a_dev[:, :K])
     assert np.array_equal(ab.to_host_bits(yh), ab.to_host_bits(y_dev[:, :n]))
@@ -321,7 +323,7 @@ def test_host_buffer_entry_point():
     assert not dc.ctx.host_x_in_place(xp)
     dc.reset_cache()
     sh2, ah2, yh2 = torch.zeros_like(sh), torch.zeros_like(ah), torch.zeros_like(yh)
-    dc.ctx.layer_step_host(dc.lw, dc.req, dc.kv(), xp, 0.2, 0, sh2, ah2, yh2)
+    dc.ctx.layer_step_host(dc.lw, dc.req, dc.kv(), xp, ratio, 0, sh2, ah2, yh2)
     torch.cuda.synchronize()
     assert np.array_equal(sh2.numpy(), s_dev) and np.array_equal(ah2.numpy(), a_dev[:, :K])
     assert np.array_equal(ab.to_host_bits(yh2), ab.to_host_bits(y_dev[:, :n]))
