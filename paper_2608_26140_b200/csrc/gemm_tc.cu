@@ -1184,7 +1184,10 @@ TcPlan make_plan(int M, int K, int units, bool swiglu) {
     p.U = (int)((total + g - 1) / g);
     p.ctas = (int)((total + p.U - 1) / p.U);
     p.smax = 2;   // partial slots per CTA
-    static const int prefetch = [] { const char* e = getenv("ACACHE_GEMM_PREFETCH"); return e ? atoi(e) : 12; }();
+    // K blocks past the ring asked into L2 before the dependency wait.  Off by default: with the neighbouring kernels
+    // as short as they are now the requests compete with the stream that follows (configuration 2: 168.1 us per
+    // layer-step at 0, 170.1 at 12, 175.7 at 28); the ring itself is still filled before the wait.
+    static const int prefetch = [] { const char* e = getenv("ACACHE_GEMM_PREFETCH"); return e ? atoi(e) : 0; }();
     p.prefetch = prefetch;
     return p;
 }
