@@ -52,6 +52,7 @@ constexpr uint32_t GRID_WAIT_LIMIT = 1u << 21;
 struct TcPlan {
     int m_tiles, n_tiles, KB, tiles, U, ctas, smax;
     int prefetch;         // K blocks past the ring whose weight tiles are requested into L2 before the dependency wait
+    int prefill;          // ring stages whose weight halves are loaded before the dependency wait
     int pair_u;           // two-SM kernel, stream-K mode: (pair tile, K block) iterations per cluster (0: whole tiles)
     int m_pairs;          // 256-row tile rows of the two-SM kernel
     int units;            // 128-row B halves over all segments (non-SwiGLU) or ffn/128 (SwiGLU)
@@ -578,11 +579,11 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     if (warp == 0 && lane == 0) {
         const CUtensorMap* maps[3] = {&mapB0, &mapB1, &mapB2};
         const uint64_t pol_w = g.keep_weights ? policy_evict_last() : policy_evict_first();
-        for (int i = 0; i < TC_STAGES + kPrefetchL2 && it0 + i < it1; ++i) {
+        for (int i = 0; i < p.prefill + kPrefetchL2 && it0 + i < it1; ++i) {
             const int it = it0 + i, t = it / p.KB, kb = it - t * p.KB, nt = t / p.m_tiles;
             int row0, row1;
             const int s0 = half_source(g, p, nt, 0, row0), s1 = half_source(g, p, nt, 1, row1);
-            if (i < TC_STAGES) {
+            if (i < p.prefill) {
                 const uint32_t sB = base + i * TC_STAGE_BYTES + TC_A_BYTES;
                 mbar_expect_tx(full_bar(i), TC_A_BYTES + TC_HALF_BYTES * (1 + (s1 >= 0)));
                 tma_load_2d(sB, maps[s0], kb * TC_BK, row0, full_bar(i), pol_w);
@@ -1189,6 +1190,8 @@ TcPlan make_plan(int M, int K, int units, bool swiglu) {
     // layer-step at 0, 170.1 at 12, 175.7 at 28); the ring itself is still filled before the wait.
     static const int prefetch = [] { const char* e = getenv("ACACHE_GEMM_PREFETCH"); return e ? atoi(e) : 0; }();
     p.prefetch = prefetch;
+    static const int prefill = [] { const char* e = getenv("ACACHE_GEMM_PREFILL"); return e ? std::min(std::max(atoi(e), 0), TC_STAGES) : TC_STAGES; }();
+    p.prefill = prefill;
     return p;
 }
 
