@@ -533,7 +533,7 @@ acache_status layer_step_impl(acache_ctx* ctx, const acache_layer_weights* w, co
             // W_q is read again by the Q/K/V projection a few kernels later: leave it in L2 (measured: that
             // projection 43.7 -> 40.8 us at 103 rows)
             static const int keep_wq = [] { const char* e = getenv("ACACHE_KEEP_WQ"); return e ? atoi(e) : 1; }();
-            g.keep_weights = keep_wq;
+            g.keep_weights = keep_wq && do_recompute;      // a scoring-only pass (the probe) never reads W_q again
             g.epilogue = kEpiQKV;
             g.bias[0] = d.qkv_bias ? w->bq : nullptr;
             g.row_pos = mpos; g.rope_cos = req->rope_cos; g.rope_sin = req->rope_sin;
