@@ -1218,7 +1218,8 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
     if (g.M == 0) return 0;
     const bool swiglu = g.epilogue == kEpiSwiGLU;
     const int n_total = swiglu ? g.n[0] : g.n[0] + g.n[1] + g.n[2];
-    const TcPlan p = make_plan(g.M, g.K, n_total / 128, swiglu);
+    TcPlan p = make_plan(g.M, g.K, n_total / 128, swiglu);
+    if (g.prefetch_blocks > 0) p.prefetch = g.prefetch_blocks;
     std::lock_guard<std::mutex> lock(g_map_mutex);
     CUtensorMap map_a, map_b[3];
     {

@@ -122,6 +122,9 @@ struct GemmArgs {
     int kv_out_stride;
     // the weights are read again by the next projection (the masked rows' queries before Q/K/V): keep them in L2
     int keep_weights;
+    // K blocks past the ring asked into L2 before the dependency wait (0: the default; worth it only behind a long
+    // kernel that leaves memory idle)
+    int prefetch_blocks;
     // --- kEpiResidual ---
     const void* resid;        // bf16 base pointer
     const int64_t* resid_off; // [M] element offset of the residual row, or null => row * N
