@@ -195,12 +195,17 @@ acache_status acache_score_anchors(acache_ctx *ctx, const acache_request *req, c
  *   is L (or ctx_len with norm_full); larger problems return ACACHE_ERR_WORKSPACE and
  *   enqueue nothing.  m <= 4096.
  * The first call on each device looks up the array's device address (with that device
- * current); make that first call before any stream capture.  It calls no cudaMalloc,
- * cudaFree or other allocating routine.  All calls share the one array, which keeps the
- * previous call's contents (nothing in it needs clearing: each call overwrites what it
- * reads), so two calls whose kernels may overlap on the GPU (different streams) race;
- * issue them on one stream or order them with events.
- * Inputs, outputs and results are exactly those of acache_score_anchors. */
+ * current) and keeps it for the life of the process; make that first call before any stream
+ * capture, and do not call cudaDeviceReset between calls (the kept address would be stale).
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  All calls share the one
+ * array, which keeps the previous call's contents (nothing in it needs clearing: each call
+ * overwrites what it reads), so two calls whose kernels may overlap on the GPU (different
+ * streams) race; issue them on one stream or order them with events.
+ * Inputs (kv->batch_stride = 0 included), outputs and results are those of
+ * acache_score_anchors up to the order of fp32 additions: with no context there is no status
+ * word for a bounded wait to report to, so this variant always runs the mma.sync scoring
+ * kernels, also at the sizes where acache_score_anchors switches to its tcgen05 kernels
+ * (about twice as fast at 8192 keys). */
 acache_status acache_score_anchors_static(const acache_model_desc *shape, const acache_request *req,
                                           const void *q_mask, const acache_kv *kv, float *scores,
                                           int accumulate, int norm_full, acache_stream_t stream);

@@ -234,9 +234,31 @@ def scatter_kv(cache_k: np.ndarray, cache_v: np.ndarray, rows: np.ndarray,
     return ck, cv
 
 
+def dropna_key_keep(ctx_len: int, affix_start: int, affix_len: int, anchor_idx: Sequence[int]) -> np.ndarray:
+    """Keys that exist under the DropNA layout (Section 5.3, "Is the Non-Anchor Cache Useful?"): every
+    position outside the affix, and of the affix only the anchors; bool [ctx_len]."""
+    keep = np.ones(ctx_len, bool)
+    keep[affix_start:affix_start + affix_len] = False
+    keep[affix_start + np.asarray(anchor_idx, dtype=np.int64)] = True
+    return keep
+
+
+def kv_deviation_scores(k_ref: np.ndarray, v_ref: np.ndarray, k_full: np.ndarray, v_full: np.ndarray) -> np.ndarray:
+    """One layer's term of the KV-deviation selector the paper compares against (appendix
+    "CacheBlend-Style Anchor Selection"): affix token j is ranked by how far its K/V in the affix-only
+    cache lie from its K/V in the full-prompt cache,
+        s_j += sum_{h, c} (K_full[j, h, c] - K_ref[j, h, c])^2 + (V_full[j, h, c] - V_ref[j, h, c])^2.
+    The paper names the quantity ("KV difference") but not the norm; the squared Euclidean distance
+    over K and V together is the reading taken.  Inputs [L, Hkv, d] fp64 (bf16 values); returns fp64 [L].
+    The scores of several layers add, and Eq. 6 then picks the K largest."""
+    dk = np.asarray(k_full, F64) - np.asarray(k_ref, F64)
+    dv = np.asarray(v_full, F64) - np.asarray(v_ref, F64)
+    return (dk * dk).sum(axis=(1, 2)) + (dv * dv).sum(axis=(1, 2))
+
+
 def recompute_rows(weights, shape, x_rows: np.ndarray, rows: np.ndarray,
                    cache_k: np.ndarray, cache_v: np.ndarray, ctx_len: int, cos, sin,
-                   round_storage: bool = True):
+                   round_storage: bool = True, key_keep: Optional[np.ndarray] = None):
     """Recompute the rows R of one request under the current context.
 
     x_rows  [n, D] fp64  layer input at the rows R (bf16 values)
@@ -246,6 +268,9 @@ def recompute_rows(weights, shape, x_rows: np.ndarray, rows: np.ndarray,
     (bf16 bits), y [n, D] fp64 (bf16 values), attention row sums [n, H].
     Queries are formed only for R; keys and values are the whole logical
     context [0, ctx_len) with rows R taken from the fresh k/v (Section 4.3).
+    ``key_keep`` (bool [ctx_len], optional): positions whose key/value exist; the
+    others are removed from every softmax (the DropNA layout of Section 5.3, which
+    discards the non-anchor affix entries).
     """
     H, Hkv, d = shape.n_heads, shape.n_kv_heads, shape.head_dim
     group = H // Hkv
@@ -266,6 +291,8 @@ def recompute_rows(weights, shape, x_rows: np.ndarray, rows: np.ndarray,
     for h in range(H):
         kh = h // group
         z = q[:, h, :] @ Kc[:, kh, :].T / math.sqrt(d)        # [n, T]
+        if key_keep is not None:
+            z = np.where(np.asarray(key_keep, bool)[None, :], z, -np.inf)
         p = softmax_rows(z)
         rowsum[:, h] = p.sum(axis=1)
         o[:, h, :] = p @ Vc[:, kh, :]
@@ -283,13 +310,15 @@ def layer_step(weights, shape, x: np.ndarray, cache_k: np.ndarray, cache_v: np.n
                extra_rows: np.ndarray, cos, sin, ratio: Optional[float] = None,
                K: Optional[int] = None, anchor_idx: Optional[np.ndarray] = None,
                scores_in: Optional[np.ndarray] = None, norm_full: bool = False,
-               round_storage: bool = True):
+               round_storage: bool = True, drop_non_anchor: bool = False):
     """One request, one layer: score -> select -> recompute -> working cache.
 
     x [T, D] bf16 bits (layer input at every position).  If ``anchor_idx`` is
     given the scoring/selection is skipped (the anchor set is fixed per
     request after selection, Section 3.2).  ``scores_in`` is added to this
-    layer's scores (Eq. 5 sums over layers).
+    layer's scores (Eq. 5 sums over layers).  ``drop_non_anchor``: the DropNA
+    ablation of Section 5.3 (same anchors, the non-anchor affix entries are
+    discarded: no query attends them).
     """
     xf = bf16_bits_to_f64(x)
     out = {}
@@ -305,7 +334,8 @@ def layer_step(weights, shape, x: np.ndarray, cache_k: np.ndarray, cache_v: np.n
         anchor_idx, tau, must, may = select_topk(s32, K)
         out.update(scores=s32, scores64=s, tau=tau, must=must, may=may, q_mask=qm)
     rows = recompute_set(anchor_idx, affix_start, extra_rows)
-    r = recompute_rows(weights, shape, xf[rows], rows, cache_k, cache_v, ctx_len, cos, sin, round_storage)
+    keep = dropna_key_keep(ctx_len, affix_start, affix_len, anchor_idx) if drop_non_anchor else None
+    r = recompute_rows(weights, shape, xf[rows], rows, cache_k, cache_v, ctx_len, cos, sin, round_storage, keep)
     out.update(r)
     out.update(anchor_idx=np.asarray(anchor_idx, np.int32), rows=rows)
     return out

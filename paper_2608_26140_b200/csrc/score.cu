@@ -10,6 +10,9 @@
 // Logits run on the tensor cores (bf16 mma.sync, fp32 accumulate) so that the pass stays
 // bound by the K_affix read, not by ALU work.
 #include <cooperative_groups.h>
+
+#include <atomic>
+
 #include "../../include/acache.h"
 #include "common.cuh"
 #include "kernels.h"
@@ -471,7 +474,9 @@ static __device__ __align__(256) float g_static_score_scratch[ACACHE_STATIC_SCRA
 
 namespace {
 constexpr int kMaxDevices = 64;
-float* g_static_scratch_ptr[kMaxDevices] = {};   // device address of the array, per device
+// device address of the array, per device; atomic, so that first calls from two host threads are safe (both
+// look the same address up)
+std::atomic<float*> g_static_scratch_ptr[kMaxDevices];
 }  // namespace
 
 extern "C" acache_status acache_score_anchors_static(const acache_model_desc* shape, const acache_request* req,
@@ -485,8 +490,10 @@ extern "C" acache_status acache_score_anchors_static(const acache_model_desc* sh
     if (req->batch < 0 || req->ctx_len <= 0 || req->affix_len < 0 || req->affix_start < 0 || req->n_masked < 0 ||
         (int64_t)req->affix_start + req->affix_len > req->ctx_len)
         return ACACHE_ERR_INVALID_ARG;
+    // batch_stride 0: one cache shared by every request of the batch (Section 4.1), as in acache_score_anchors
     if (!kv->k || (reinterpret_cast<uintptr_t>(kv->k) & 15u) || kv->ctx_capacity < req->ctx_len ||
-        kv->batch_stride < (int64_t)kv->ctx_capacity * shape->n_kv_heads * shape->head_dim || (kv->batch_stride & 7))
+        (kv->batch_stride != 0 &&
+         (kv->batch_stride < (int64_t)kv->ctx_capacity * shape->n_kv_heads * shape->head_dim || (kv->batch_stride & 7))))
         return ACACHE_ERR_INVALID_ARG;
     if (req->n_masked > 0 && (!q_mask || (reinterpret_cast<uintptr_t>(q_mask) & 15u))) return ACACHE_ERR_INVALID_ARG;
     if (req->n_masked > kMaxMaskedSmem) return ACACHE_ERR_UNSUPPORTED_SHAPE;
@@ -501,15 +508,14 @@ extern "C" acache_status acache_score_anchors_static(const acache_model_desc* sh
     // handle here, so ask the runtime for the address the kernels must be given.
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ACACHE_ERR_CUDA;
-    if (!g_static_scratch_ptr[dev]) {
-        float* p = nullptr;
-        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_score_scratch) != cudaSuccess || !p) {
+    float* scratch = g_static_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&scratch), g_static_score_scratch) != cudaSuccess || !scratch) {
             (void)cudaGetLastError();
             return ACACHE_ERR_CUDA;
         }
-        g_static_scratch_ptr[dev] = p;
+        g_static_scratch_ptr[dev].store(scratch, std::memory_order_release);
     }
-    float* scratch = g_static_scratch_ptr[dev];
 
     ScoreArgs a{};
     a.q_mask = q_mask;

@@ -388,6 +388,81 @@ def test_idempotent_when_cache_is_current():
     assert np.allclose(out["y"], y[out["rows"]], rtol=1e-9, atol=1e-11)
 
 
+# ---------------------------------------------------------------- selector / layout variants (Section 5.3, appendix)
+def test_kv_deviation_scores_brute_force_and_invariants():
+    L, Hkv, d = 9, 2, 6
+    ka, va, kb, vb = (rnd(s_, L, Hkv, d) for s_ in (31, 32, 33, 34))
+    s = orc.kv_deviation_scores(ka, va, kb, vb)
+    brute = []
+    for j in range(L):
+        acc = 0.0
+        for h in range(Hkv):
+            for c in range(d):
+                acc += (kb[j][h][c] - ka[j][h][c]) ** 2 + (vb[j][h][c] - va[j][h][c]) ** 2
+        brute.append(acc)
+    assert np.allclose(s, brute, rtol=1e-13, atol=0)
+    assert np.array_equal(orc.kv_deviation_scores(ka, va, ka, va), np.zeros(L))            # equal caches: nothing deviates
+    assert np.allclose(orc.kv_deviation_scores(kb, vb, ka, va), s, rtol=1e-15)             # symmetric in the two caches
+    perm = np.random.default_rng(3).permutation(L)
+    assert np.allclose(orc.kv_deviation_scores(ka[perm], va[perm], kb[perm], vb[perm]), s[perm], rtol=1e-15)
+    # one changed element of one token: that token's score is the square of the change, all others zero
+    k2 = ka.copy(); k2[4, 1, 3] += 0.75
+    one = orc.kv_deviation_scores(ka, va, k2, va)
+    assert np.isclose(one[4], 0.75 ** 2) and np.count_nonzero(one) == 1
+    # K and V enter with equal weight, and layers add (Eq. 5's sum over layers carries over to this selector)
+    assert np.allclose(orc.kv_deviation_scores(ka, va, kb, va) + orc.kv_deviation_scores(ka, va, ka, vb), s, rtol=1e-13)
+    # the selection on top of it is Eq. 6 unchanged: the K tokens that moved most
+    A, _, _, _ = orc.select_topk(s.astype(np.float32), 3)
+    assert sorted(A.tolist()) == sorted(np.argsort(-np.asarray(brute))[:3].tolist())
+
+
+def test_dropna_keeps_anchors_and_non_affix_keys_only():
+    lay, w, x, xs, cos, sin = small_case(extra="masked")
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    ck, cv = stale_cache(w, SMALL, xs, cos, sin, T)
+    args = (w, SMALL, x, ck, cv, T, l, L, lay.masked_pos[0], lay.extra_rows[0], cos, sin)
+    keepna = orc.layer_step(*args, ratio=0.25)
+    drop = orc.layer_step(*args, anchor_idx=keepna["anchor_idx"], drop_non_anchor=True)
+    A = keepna["anchor_idx"]
+    keep = orc.dropna_key_keep(T, l, L, A)
+    assert keep.sum() == T - L + len(A) and keep[l + A].all() and keep[:l].all() and keep[l + L:].all()
+    # same anchors, same refreshed K/V and working cache; only the attention (and what follows it) differs
+    assert np.array_equal(drop["k_new"], keepna["k_new"]) and np.array_equal(drop["cache_k"], keepna["cache_k"])
+    assert not np.array_equal(drop["y"], keepna["y"])
+    assert np.allclose(drop["rowsum"], 1.0, atol=1e-12)
+    # brute force: attention of every recomputed row over the kept keys, explicit loops
+    H, Hkv, d = SMALL.n_heads, SMALL.n_kv_heads, SMALL.head_dim
+    Kc, Vc = orc.bf16_bits_to_f64(drop["cache_k"]), orc.bf16_bits_to_f64(drop["cache_v"])
+    kept = [t for t in range(T) if keep[t]]
+    for r in (0, len(drop["rows"]) - 1):
+        for h in (0, H - 1):
+            kh = h // (H // Hkv)
+            z = [sum(drop["q"][r, h, c] * Kc[t, kh, c] for c in range(d)) / math.sqrt(d) for t in kept]
+            zmax = max(z)
+            e = [math.exp(v - zmax) for v in z]
+            den = sum(e)
+            o = [sum(e[i] / den * Vc[t, kh, c] for i, t in enumerate(kept)) for c in range(d)]
+            assert np.allclose(orc.bf16_round(np.array(o)), drop["o"][r, h * d:(h + 1) * d], rtol=0, atol=2 ** -8 * max(map(abs, o)))
+    # the dropped entries really are gone: garbage there changes nothing, a change at a kept key does
+    dead = np.setdiff1d(np.arange(l, l + L), l + A)
+    ck2, cv2 = ck.copy(), cv.copy()
+    ck2[dead] = 0x4400; cv2[dead] = 0xC400
+    again = orc.layer_step(w, SMALL, x, ck2, cv2, *args[5:], anchor_idx=A, drop_non_anchor=True)
+    assert np.array_equal(again["y"], drop["y"])
+    ck3 = ck.copy(); ck3[0 if l > 0 else l + L] = 0x4100
+    moved = orc.layer_step(w, SMALL, x, ck3, cv, *args[5:], anchor_idx=A, drop_non_anchor=True)
+    assert not np.array_equal(moved["y"], drop["y"])
+    # ratio 1.0: no non-anchor token remains, both layouts are the full affix recomputation (Section 5.3)
+    full_keep = orc.layer_step(*args, ratio=1.0)
+    full_drop = orc.layer_step(*args, ratio=1.0, drop_non_anchor=True)
+    assert np.array_equal(full_drop["y"], full_keep["y"]) and np.array_equal(full_drop["cache_v"], full_keep["cache_v"])
+    # ratio 0: the rows attend the non-affix keys only, as if the affix had never been cached
+    none = orc.layer_step(*args, ratio=0.0, drop_non_anchor=True)
+    assert np.array_equal(orc.dropna_key_keep(T, l, L, none["anchor_idx"])[l:l + L], np.zeros(L, bool))
+    ck4 = ck.copy(); ck4[l:l + L] = 0x4400
+    assert np.array_equal(orc.layer_step(w, SMALL, x, ck4, cv, *args[5:], ratio=0.0, drop_non_anchor=True, K=0)["y"], none["y"])
+
+
 def test_layer_step_scores_use_stale_keys_and_accumulate():
     lay, w, x, xs, cos, sin = small_case(extra="none")
     T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
