@@ -60,6 +60,8 @@ typedef enum {
 #define ACACHE_F_ACCUMULATE       0x4u /* scores += this layer's scores (Eq. 5 sums over layers)        */
 #define ACACHE_F_SCORE_NORM_FULL  0x8u /* softmax of Eq. 4 over every key of the context, not the affix only */
 #define ACACHE_F_NO_RECOMPUTE    0x10u /* stop after scoring / selection (the selection-time probe)     */
+#define ACACHE_F_DROP_NON_ANCHOR 0x20u /* DropNA layout (Section 5.3): the non-anchor affix entries are discarded, i.e. the
+                                          recomputed rows attend the anchors and the non-affix positions only            */
 
 typedef struct CUstream_st *acache_stream_t;   /* a cudaStream_t */
 typedef struct acache_ctx acache_ctx;           /* opaque */
@@ -219,6 +221,19 @@ int32_t acache_k_from_ratio(int32_t affix_len, double ratio);
 acache_status acache_select_topk(acache_ctx *ctx, const float *scores, int32_t batch, int32_t affix_len,
                                  int32_t k, int32_t *anchor_idx, acache_stream_t stream);
 
+/* The KV-deviation selector the paper compares its own against (appendix "CacheBlend-Style Anchor
+ * Selection"): affix token j is ranked by how far its cached K/V (kv_ref: the affix-only / stale cache)
+ * lie from its K/V under the full prompt (kv_full), without looking at the masked positions:
+ *   scores[b,j] (+)= sum_{h,c} (K_full[b,l+j,h,c] - K_ref[b,l+j,h,c])^2 + (V_full[...] - V_ref[...])^2
+ * (squared Euclidean distance over K and V together; the paper does not fix the norm).  One call is one
+ * layer's term; accumulate != 0 adds to scores, so that the layers sum as in Eq. 5, and
+ * acache_select_topk then picks the anchors exactly as for the attention scores.
+ * kv_ref, kv_full: layout as acache_kv; either may have batch_stride 0 (one copy for the batch).  Only the
+ * affix rows are read.  scores: DEVICE fp32 [B, L].  The sum is evaluated in a fixed order. */
+acache_status acache_score_kv_deviation(acache_ctx *ctx, const acache_request *req, const acache_kv *kv_ref,
+                                        const acache_kv *kv_full, float *scores, int accumulate,
+                                        acache_stream_t stream);
+
 /* Selective recomputation (Section 3.3, Section 4.3) of the rows R = A u E of every
  * request, WITHOUT touching the cache:
  *   xn = RMSNorm(x_r) g1; q,k,v = W{q,k,v} xn (+b); RoPE(q,k; position r)
@@ -251,6 +266,9 @@ acache_status acache_scatter_kv(acache_ctx *ctx, const acache_request *req, acac
  *                            that is not raises ACACHE_FLAG_BAD_INDEX.
  *   flags & ACACHE_F_SELECT: anchor_idx [B, K] is written, K = acache_k_from_ratio(L, ratio);
  *                            otherwise anchor_idx is an input with that K.
+ *   flags & ACACHE_F_DROP_NON_ANCHOR: the DropNA ablation of Section 5.3: K/V of R are refreshed and
+ *                            written as usual, but the attention of the rows of R skips every affix position
+ *                            that is not an anchor (accepted by acache_layer_step_shared as well).
  * scores: DEVICE fp32 [B, L] (may be NULL without F_SCORE/F_SELECT).
  * y: DEVICE bf16 [B, K+e, D]. */
 acache_status acache_layer_step(acache_ctx *ctx, const acache_layer_weights *w,

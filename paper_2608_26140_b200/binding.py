@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libacache.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 FLAG_BAD_INDEX, FLAG_WAIT_EXPIRED = 0x1, 0x2
-F_SCORE, F_SELECT, F_ACCUMULATE, F_SCORE_NORM_FULL, F_NO_RECOMPUTE = 0x1, 0x2, 0x4, 0x8, 0x10
+F_SCORE, F_SELECT, F_ACCUMULATE, F_SCORE_NORM_FULL, F_NO_RECOMPUTE, F_DROP_NON_ANCHOR = 0x1, 0x2, 0x4, 0x8, 0x10, 0x20
 
 EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "acache_destroy",
            "acache_last_error", "acache_poll_status", "acache_launch_count", "acache_score_anchors",
@@ -25,7 +25,7 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step", "acache_probe_select",
            "acache_commit_update", "acache_generate_block", "acache_denoise_step_shared", "acache_recompute_rows_shared",
            "acache_decode_step_shared", "acache_generate_block_shared", "acache_layer_step_shared",
-           "acache_host_x_in_place"]
+           "acache_host_x_in_place", "acache_score_kv_deviation"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -90,6 +90,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_launch_count.restype = C.c_uint64
     lib.acache_score_anchors.argtypes = [vp, C.POINTER(Request), vp, C.POINTER(KV), vp, C.c_int, C.c_int, vp]
     lib.acache_score_anchors.restype = C.c_int
+    lib.acache_score_kv_deviation.argtypes = [vp, C.POINTER(Request), C.POINTER(KV), C.POINTER(KV), vp, C.c_int, vp]
+    lib.acache_score_kv_deviation.restype = C.c_int
     lib.acache_k_from_ratio.argtypes = [i32, C.c_double]
     lib.acache_k_from_ratio.restype = i32
     lib.acache_select_topk.argtypes = [vp, vp, i32, i32, i32, vp, vp]
@@ -265,6 +267,10 @@ class Context:
     def score_anchors(self, req: Request, q_mask, kv: KV, scores, accumulate=False, norm_full=False):
         self._check(self.lib.acache_score_anchors(self.h, C.byref(req), _ptr(q_mask), C.byref(kv), _ptr(scores),
                                                   int(accumulate), int(norm_full), _stream()))
+
+    def score_kv_deviation(self, req: Request, kv_ref: KV, kv_full: KV, scores, accumulate=False):
+        self._check(self.lib.acache_score_kv_deviation(self.h, C.byref(req), C.byref(kv_ref), C.byref(kv_full), _ptr(scores),
+                                                       int(accumulate), _stream()))
 
     def select_topk(self, scores, batch, affix_len, k, anchor_idx):
         self._check(self.lib.acache_select_topk(self.h, _ptr(scores), batch, affix_len, k, _ptr(anchor_idx), _stream()))

@@ -168,7 +168,7 @@ struct MapReuse { bool reuse; };
 acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const acache_request* r,
                             const acache_kv* kv, bool fuse_scatter, const void* x, int x_is_compact,
                             const int32_t* anchor_idx, int k, void* k_new, void* v_new, void* y, cudaStream_t st,
-                            const PrivateRows* priv = nullptr, MapReuse maps = MapReuse{false}) {
+                            const PrivateRows* priv = nullptr, MapReuse maps = MapReuse{false}, bool drop_non_anchor = false) {
     const acache_model_desc& d = c->d;
     const int rows = k + r->n_extra, n = r->batch * rows;
     if (n == 0) {
@@ -245,6 +245,17 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
                              km + (size_t)r->batch * at.excl_words, at.keep_words, st);
             c->launches += 2;
         }
+    }
+    if (drop_non_anchor) {
+        // DropNA layout (Section 5.3): the affix positions that are not anchors do not exist as keys.  The bits
+        // live behind the two masks of the two-source attention; with fresh rows as a second source they are also
+        // OR-ed into the cache-exclusion mask (the anchors then come from the fresh rows).
+        const int words = (r->ctx_len + 31) / 32;
+        uint32_t* km = wsp<uint32_t>(c, c->o_keymask);
+        uint32_t* kd = km + (size_t)r->batch * (words + (d.max_rows + 31) / 32 + 2);
+        launch_drop_mask(anchor_idx, k, r->affix_start, r->affix_len, r->ctx_len, r->batch, kd, fuse_scatter ? nullptr : km, words, st);
+        c->launches += 1;
+        at.key_drop = kd; at.excl_words = words;
     }
     at.batch = r->batch; at.n = rows; at.ctx_len = r->ctx_len;
     at.n_heads = d.n_heads; at.n_kv_heads = d.n_kv_heads; at.head_dim = d.head_dim;
@@ -340,7 +351,7 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
     c->o_stats = take(cur, (size_t)d.max_batch * d.n_heads * score_num_splits(d.max_ctx) * d.max_masked * 8);
     c->o_partial = take(cur, (size_t)d.max_batch * d.n_heads * d.max_affix * 4);
     c->o_slot = take(cur, (size_t)d.max_batch * d.max_ctx * 4);
-    c->o_keymask = take(cur, (size_t)d.max_batch * ((d.max_ctx + 31) / 32 + (d.max_rows + 31) / 32 + 2) * 4);
+    c->o_keymask = take(cur, (size_t)d.max_batch * (2 * ((d.max_ctx + 31) / 32) + (d.max_rows + 31) / 32 + 4) * 4);
     c->o_xstage = take(cur, (size_t)d.max_batch * d.max_ctx * d.hidden * 2);
     c->o_ystage = take(cur, nr * d.hidden * 2);
     c->o_sstage = take(cur, (size_t)d.max_batch * d.max_affix * 4);
@@ -463,6 +474,22 @@ acache_status acache_select_topk(acache_ctx* ctx, const float* scores, int32_t b
     return check_cuda(ctx, "topk");
 }
 
+acache_status acache_score_kv_deviation(acache_ctx* ctx, const acache_request* req, const acache_kv* kv_ref,
+                                        const acache_kv* kv_full, float* scores, int accumulate, acache_stream_t stream) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    if (!kv_ref || !kv_full) return fail(ctx, ACACHE_ERR_INVALID_ARG, "kv_ref / kv_full is NULL");
+    acache_status s = check_request(ctx, req, kv_ref, 0, false, true);
+    if (s != ACACHE_OK) return s;
+    if ((s = check_request(ctx, req, kv_full, 0, false, true)) != ACACHE_OK) return s;
+    if (!scores) return fail(ctx, ACACHE_ERR_INVALID_ARG, "scores is NULL");
+    if (req->batch == 0 || req->affix_len == 0) return ACACHE_OK;
+    launch_kv_deviation(kv_ref->k, kv_ref->v, kv_ref->batch_stride, kv_full->k, kv_full->v, kv_full->batch_stride,
+                        req->affix_start, req->affix_len, ctx->d.n_kv_heads * ctx->d.head_dim, req->batch, scores, accumulate,
+                        stream);
+    ctx->launches += 1;
+    return check_cuda(ctx, "kv deviation");
+}
+
 acache_status acache_recompute_anchors(acache_ctx* ctx, const acache_layer_weights* w, const acache_request* req,
                                        const acache_kv* kv, const void* x, int x_is_compact,
                                        const int32_t* anchor_idx, int32_t k, void* k_new, void* v_new, void* y,
@@ -581,7 +608,8 @@ acache_status layer_step_impl(acache_ctx* ctx, const acache_layer_weights* w, co
         ctx->launches += 1;
     }
     if (do_recompute)
-        return run_recompute(ctx, w, req, kv, !to_slots, x, x_is_compact, anchor_idx, k, k_new, v_new, y, stream);
+        return run_recompute(ctx, w, req, kv, !to_slots, x, x_is_compact, anchor_idx, k, k_new, v_new, y, stream, nullptr,
+                             MapReuse{false}, (flags & ACACHE_F_DROP_NON_ANCHOR) != 0);
     mark(ctx, ACACHE_N_STAGES, stream);
     return check_cuda(ctx, "layer_step");
 }

@@ -126,13 +126,22 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
             }
         }
         const int valid = a.ctx_len - (tile_lo + t) * 64;
+        // keys that do not exist (DropNA layout): two mask words per 64-key tile
+        uint32_t drop[2] = {0u, 0u};
+        if (a.key_drop) {
+            const int w0 = (tile_lo + t) * 2;
+            const uint32_t* kd = a.key_drop + (int64_t)b * a.excl_words;
+            if (w0 < a.excl_words) drop[0] = __ldg(kd + w0);
+            if (w0 + 1 < a.excl_words) drop[1] = __ldg(kd + w0 + 1);
+        }
         float tmax[2] = {-INFINITY, -INFINITY};
 #pragma unroll
         for (int nb = 0; nb < 8; ++nb)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 int col = nb * 8 + (lane & 3) * 2 + (i & 1);
-                float v = col < valid ? s[nb][i] * scale_log2e : -INFINITY;
+                const bool there = col < valid && !((drop[col >> 5] >> (col & 31)) & 1u);
+                float v = there ? s[nb][i] * scale_log2e : -INFINITY;
                 s[nb][i] = v;
                 tmax[i >> 1] = fmaxf(tmax[i >> 1], v);
             }
@@ -142,10 +151,11 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
             tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 1));
             tmax[r] = fmaxf(tmax[r], __shfl_xor_sync(0xffffffffu, tmax[r], 2));
             float nm = fmaxf(mx[r], tmax[r]);
-            corr[r] = exp2f(mx[r] - nm);
+            corr[r] = nm == -INFINITY ? 1.f : exp2f(mx[r] - nm);      // no key seen yet (a tile may be dropped whole)
             mx[r] = nm;
             den[r] *= corr[r];
         }
+        const float mref[2] = {mx[0] == -INFINITY ? 0.f : mx[0], mx[1] == -INFINITY ? 0.f : mx[1]};
 #pragma unroll
         for (int i = 0; i < D / 8; ++i) {
             o[i][0] *= corr[0]; o[i][1] *= corr[0];
@@ -154,8 +164,8 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnArgs a, float 
         uint32_t pf[4][4];
 #pragma unroll
         for (int nb = 0; nb < 8; ++nb) {
-            float p0 = exp2f(s[nb][0] - mx[0]), p1 = exp2f(s[nb][1] - mx[0]);
-            float p2 = exp2f(s[nb][2] - mx[1]), p3 = exp2f(s[nb][3] - mx[1]);
+            float p0 = exp2f(s[nb][0] - mref[0]), p1 = exp2f(s[nb][1] - mref[0]);
+            float p2 = exp2f(s[nb][2] - mref[1]), p3 = exp2f(s[nb][3] - mref[1]);
             den[0] += p0 + p1;
             den[1] += p2 + p3;
             pf[nb >> 1][(nb & 1) * 2] = pack_bf16(p0, p1);
@@ -225,7 +235,8 @@ __global__ void __launch_bounds__(128) attention_combine_kernel(const AttnArgs a
 #pragma unroll
     for (int i = 0; i < D / 32; ++i) acc[i] = 0.f;
     for (int s = 0; s < n_split; ++s) {
-        const float w = exp2f(a.part_ml[(rh * n_split + s) * 2] - m);
+        const float ms = a.part_ml[(rh * n_split + s) * 2];
+        const float w = ms == -INFINITY ? 0.f : exp2f(ms - m);      // a split all of whose keys were dropped
         l += a.part_ml[(rh * n_split + s) * 2 + 1] * w;
         const float* po = a.part_o + (rh * n_split + s) * D;
 #pragma unroll

@@ -113,7 +113,8 @@ struct AttnTcArgs {
     uint32_t* status;
     // two key sources (shared storage + private rows, Section 4.1): after the cache's tiles come the tiles of
     // the fresh rows [B, n, Hkv, d]; pos_excl masks the cache positions those rows serve, row_keep the fresh
-    // rows that do not serve their position (duplicates).  n_fresh_tiles = 0: the cache alone.
+    // rows that do not serve their position (duplicates).  n_fresh_tiles = 0: the cache alone; pos_excl may then
+    // still name cache positions that do not exist as keys (the DropNA layout of Section 5.3).
     int n_fresh_tiles, excl_words, keep_words, cache_shared;
     int kv_prefetch;          // two-query-tile kernel: K/V tiles requested into L2 ahead of the rings
     // one-tile kernel over a shared cache with at most 32 rows per request (decode passes): group = 4 puts the rows
@@ -278,7 +279,7 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
             if (j < n_cache_tiles) {
                 const int valid = a.ctx_len - j * 128 - c4 * 32;
                 keep = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
-                if (a.n_fresh_tiles && j * 4 + c4 < a.excl_words) keep &= ~__ldg(a.pos_excl + (int64_t)bq * a.excl_words + j * 4 + c4);
+                if (a.pos_excl && j * 4 + c4 < a.excl_words) keep &= ~__ldg(a.pos_excl + (int64_t)bq * a.excl_words + j * 4 + c4);
             } else {
                 const int f = j - n_cache_tiles;
                 if (G > 1 && f / a.n_fresh_tiles != q) {
@@ -619,7 +620,7 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
                 if (j < n_cache_tiles) {
                     const int valid = a.ctx_len - j * 128 - w * 32;
                     keep[c] = valid >= 32 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << valid) - 1u);
-                    if (a.n_fresh_tiles && j * 4 + w < a.excl_words) keep[c] &= ~__ldg(a.pos_excl + (int64_t)b * a.excl_words + j * 4 + w);
+                    if (a.pos_excl && j * 4 + w < a.excl_words) keep[c] &= ~__ldg(a.pos_excl + (int64_t)b * a.excl_words + j * 4 + w);
                 } else {
                     const int fw = (j - n_cache_tiles) * 4 + w;
                     keep[c] = fw < a.keep_words ? __ldg(a.row_keep + (int64_t)b * a.keep_words + fw) : 0u;
@@ -866,7 +867,9 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     t.group = group; t.batch = a.batch;
     if (two_src) {
         t.n_fresh_tiles = (n_fresh + 127) / 128; t.excl_words = a.excl_words; t.keep_words = a.keep_words;
-        t.pos_excl = a.pos_excl; t.row_keep = a.row_keep;
+        t.pos_excl = a.pos_excl; t.row_keep = a.row_keep;      // with key_drop the caller has OR-ed it into pos_excl
+    } else if (a.key_drop) {
+        t.excl_words = a.excl_words; t.pos_excl = a.key_drop;
     }
     static const int kv_prefetch = [] { const char* e = getenv("ACACHE_ATTN_KV_PREFETCH"); return e ? atoi(e) : 2; }();
     t.kv_prefetch = kv_prefetch;

@@ -34,6 +34,17 @@ void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, i
 void launch_key_masks(const int32_t* slot, int ctx_len, const int32_t* row_pos, int rows_per_req, int batch,
                       uint32_t* pos_excl, int excl_words, uint32_t* row_keep, int keep_words, cudaStream_t stream);
 
+// scores[b, j] (+)= ||K_full[b, l + j] - K_ref[b, l + j]||^2 + ||V_full[b, l + j] - V_ref[b, l + j]||^2 (batch strides in
+// elements, 0 = one cache shared by the batch).
+void launch_kv_deviation(const void* k_ref, const void* v_ref, int64_t ref_stride, const void* k_full, const void* v_full,
+                         int64_t full_stride, int affix_start, int affix_len, int kv_dim, int batch, float* scores,
+                         int accumulate, cudaStream_t stream);
+
+// key_drop[b, t / 32] bit t % 32 = position t is an affix position that is not an anchor of request b (the DropNA
+// layout: such keys do not exist); or_into (optional, same shape) receives the same bits by OR.
+void launch_drop_mask(const int32_t* anchor_idx, int k, int affix_start, int affix_len, int ctx_len, int batch,
+                      uint32_t* key_drop, uint32_t* or_into, int words, cudaStream_t stream);
+
 // ---- score.cu ---------------------------------------------------------------------------
 struct ScoreArgs {
     const void* q_mask;       // bf16 [B, m, H, d]
@@ -163,6 +174,7 @@ struct AttnArgs {
     const uint32_t* pos_excl; // optional key masks of the same map (launch_key_masks): with them the tensor-core
     const uint32_t* row_keep; //   kernel reads the cache and k_new / v_new as two key sources instead of gathering
     int excl_words, keep_words;
+    const uint32_t* key_drop; // optional [B, excl_words]: bit t = position t does not exist as a key (DropNA, Section 5.3)
     int batch, n, ctx_len, n_heads, n_kv_heads, head_dim;
     void* o;                  // bf16 [B, n, H*d]
     float* part_o;            // scratch for key splits: fp32 [B*n*H, n_split, d]

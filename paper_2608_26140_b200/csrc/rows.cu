@@ -212,4 +212,102 @@ void launch_build_slot_map(int32_t* slot, int ctx_len, const int32_t* row_pos, i
     launch_pdl(slot_map_kernel, batch, 1024, 0, stream, slot, ctx_len, row_pos, rows_per_req);
 }
 
+// ---- KV-deviation selector (the CacheBlend-style variant of the paper's appendix) ------------------
+// scores[b, j] (+)= sum over the KV heads and the head dimension of (K_full - K_ref)^2 + (V_full - V_ref)^2
+// at affix token j.  One CTA per (token, request): the four rows are streamed once with 16-byte loads,
+// squared differences accumulate in fp32, and the block sum runs in a fixed order (bitwise reproducible).
+__global__ void __launch_bounds__(128) kv_deviation_kernel(const __nv_bfloat16* __restrict__ k_ref,
+                                                           const __nv_bfloat16* __restrict__ v_ref, int64_t ref_stride,
+                                                           const __nv_bfloat16* __restrict__ k_full,
+                                                           const __nv_bfloat16* __restrict__ v_full, int64_t full_stride,
+                                                           int affix_start, int affix_len, int kv_dim,
+                                                           float* __restrict__ scores, int accumulate) {
+    __shared__ float red[4];
+    pdl_wait();
+    pdl_launch_dependents();
+    const int j = blockIdx.x, b = blockIdx.y;
+    const int64_t row = (int64_t)(affix_start + j) * kv_dim;
+    const uint4* src[4] = {reinterpret_cast<const uint4*>(k_ref + (int64_t)b * ref_stride + row),
+                           reinterpret_cast<const uint4*>(k_full + (int64_t)b * full_stride + row),
+                           reinterpret_cast<const uint4*>(v_ref + (int64_t)b * ref_stride + row),
+                           reinterpret_cast<const uint4*>(v_full + (int64_t)b * full_stride + row)};
+    const int nchunk = kv_dim >> 3;
+    float acc = 0.f;
+    for (int c0 = threadIdx.x; c0 < nchunk; c0 += 4 * 128) {
+        uint4 u[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = c0 + i * 128;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) u[i][t] = c < nchunk ? __ldcs(src[t] + c) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int t = 0; t < 4; t += 2) {
+                const uint32_t a[4] = {u[i][t].x, u[i][t].y, u[i][t].z, u[i][t].w};
+                const uint32_t f[4] = {u[i][t + 1].x, u[i][t + 1].y, u[i][t + 1].z, u[i][t + 1].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float d0 = bf16_lo(f[e]) - bf16_lo(a[e]), d1 = bf16_hi(f[e]) - bf16_hi(a[e]);
+                    acc = fmaf(d0, d0, acc);
+                    acc = fmaf(d1, d1, acc);
+                }
+            }
+    }
+    const float tot = block_sum(acc, red);
+    if (threadIdx.x == 0) {
+        float* out = scores + (int64_t)b * affix_len + j;
+        *out = accumulate ? *out + tot : tot;
+    }
+}
+
+void launch_kv_deviation(const void* k_ref, const void* v_ref, int64_t ref_stride, const void* k_full, const void* v_full,
+                         int64_t full_stride, int affix_start, int affix_len, int kv_dim, int batch, float* scores,
+                         int accumulate, cudaStream_t stream) {
+    if (batch == 0 || affix_len == 0) return;
+    launch_pdl(kv_deviation_kernel, dim3(affix_len, batch), dim3(128), 0, stream, static_cast<const __nv_bfloat16*>(k_ref),
+               static_cast<const __nv_bfloat16*>(v_ref), ref_stride, static_cast<const __nv_bfloat16*>(k_full),
+               static_cast<const __nv_bfloat16*>(v_full), full_stride, affix_start, affix_len, kv_dim, scores, accumulate);
+}
+
+// ---- DropNA layout (Section 5.3): the non-anchor affix entries do not exist as keys ------------------
+// key_drop[b] bit t = position t lies in the affix and is not one of request b's anchors.  With or_into the same
+// bits are also OR-ed into the cache-exclusion mask of the two-source attention (there the anchors come from
+// the fresh rows, so the whole affix span of the cache is skipped).
+__global__ void __launch_bounds__(256) drop_mask_kernel(const int32_t* __restrict__ anchor_idx, int k, int affix_start,
+                                                        int affix_len, int ctx_len, uint32_t* __restrict__ key_drop,
+                                                        uint32_t* __restrict__ or_into, int words) {
+    extern __shared__ uint32_t bits[];
+    pdl_wait();
+    pdl_launch_dependents();
+    const int b = blockIdx.x;
+    for (int w = threadIdx.x; w < words; w += blockDim.x) {
+        const int lo = max(affix_start - w * 32, 0), hi = min(affix_start + affix_len - w * 32, 32);
+        uint32_t m = 0u;
+        if (hi > lo) m = (hi - lo >= 32 ? 0xffffffffu : ((1u << (hi - lo)) - 1u) << lo);
+        bits[w] = m;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < k; i += blockDim.x) {
+        const int a = anchor_idx[(int64_t)b * k + i];
+        if (a >= 0 && a < affix_len) {
+            const int t = affix_start + a;
+            atomicAnd(&bits[t >> 5], ~(1u << (t & 31)));
+        }
+    }
+    __syncthreads();
+    for (int w = threadIdx.x; w < words; w += blockDim.x) {
+        key_drop[(int64_t)b * words + w] = bits[w];
+        if (or_into) or_into[(int64_t)b * words + w] |= bits[w];
+    }
+}
+
+void launch_drop_mask(const int32_t* anchor_idx, int k, int affix_start, int affix_len, int ctx_len, int batch,
+                      uint32_t* key_drop, uint32_t* or_into, int words, cudaStream_t stream) {
+    if (batch == 0) return;
+    launch_pdl(drop_mask_kernel, dim3(batch), dim3(256), (size_t)words * sizeof(uint32_t), stream, anchor_idx, k, affix_start,
+               affix_len, ctx_len, key_drop, or_into, words);
+}
+
 }  // namespace acache
