@@ -143,6 +143,18 @@ const char *acache_last_error(const acache_ctx *ctx);
  * clears it.  Returns ACACHE_ERR_TIMEOUT if ACACHE_FLAG_WAIT_EXPIRED is set. */
 acache_status acache_poll_status(acache_ctx *ctx, acache_stream_t stream, uint32_t *host_flags);
 
+/* Failure-detection self-test (the paper has no counterpart).  Every wait inside the kernels (mbarrier or
+ * grid-wide barrier) is bounded; when one runs out the kernel stops issuing work, waits for its copies in
+ * flight, frees its tensor memory, raises ACACHE_FLAG_WAIT_EXPIRED and returns, and the context stays usable.
+ * This call makes that happen once, on purpose: the next Q/K/V projection this context launches
+ * (acache_recompute_anchors, acache_layer_step, ...) gives the grid-wide barrier that ends its row-preparation
+ * phase a target one arrival beyond what its grid can deliver and a short poll limit (about a millisecond),
+ * so the wait runs out before any tensor-core work was issued.  The call that contains it still enqueues its
+ * later kernels, whose outputs are then meaningless; acache_poll_status afterwards returns ACACHE_ERR_TIMEOUT
+ * and re-arms the barrier, and the next call on the context runs normally.  Nothing faults, traps or spins
+ * without a bound. */
+acache_status acache_debug_expire_next_wait(acache_ctx *ctx);
+
 /* Number of kernels this context has launched since creation (for accounting). */
 uint64_t acache_launch_count(const acache_ctx *ctx);
 

@@ -25,7 +25,7 @@ EXPORTS = ["acache_create", "acache_workspace_bytes", "acache_set_workspace", "a
            "acache_score_anchors_static", "acache_predict_commit", "acache_denoise_step", "acache_probe_select",
            "acache_commit_update", "acache_generate_block", "acache_denoise_step_shared", "acache_recompute_rows_shared",
            "acache_decode_step_shared", "acache_generate_block_shared", "acache_layer_step_shared",
-           "acache_host_x_in_place", "acache_score_kv_deviation"]
+           "acache_host_x_in_place", "acache_score_kv_deviation", "acache_debug_expire_next_wait"]
 
 STAGES = ["mask_q", "score", "topk", "gather_norm", "qkv", "attention", "oproj", "mlp_norm", "gate_up", "down"]
 
@@ -86,6 +86,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.acache_last_error.restype = C.c_char_p
     lib.acache_poll_status.argtypes = [vp, vp, C.POINTER(u32)]
     lib.acache_poll_status.restype = C.c_int
+    lib.acache_debug_expire_next_wait.argtypes = [vp]
+    lib.acache_debug_expire_next_wait.restype = C.c_int
     lib.acache_launch_count.argtypes = [vp]
     lib.acache_launch_count.restype = C.c_uint64
     lib.acache_score_anchors.argtypes = [vp, C.POINTER(Request), vp, C.POINTER(KV), vp, C.c_int, C.c_int, vp]
@@ -254,6 +256,16 @@ class Context:
         if st not in (OK, ERR_TIMEOUT):
             self._check(st)
         return int(flags.value)
+
+    def poll_status_code(self):
+        """(status code, flags) of acache_poll_status: ERR_TIMEOUT when a bounded device-side wait ran out."""
+        flags = C.c_uint32(0)
+        st = self.lib.acache_poll_status(self.h, _stream(), C.byref(flags))
+        return int(st), int(flags.value)
+
+    def debug_expire_next_wait(self):
+        """Failure-detection self-test: the next Q/K/V projection's grid barrier is made to run out."""
+        self._check(self.lib.acache_debug_expire_next_wait(self.h))
 
     def stage_timing(self, enable: bool):
         self._check(self.lib.acache_stage_timing(self.h, int(enable)))

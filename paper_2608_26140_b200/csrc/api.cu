@@ -26,6 +26,7 @@ struct acache_ctx {
     size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar, o_mcidx, o_lstats, o_lxn, o_keymask;
     std::string err;
     uint64_t launches = 0;
+    int debug_expire_once = 0;      // acache_debug_expire_next_wait: consumed by the next Q/K/V projection
     // optional per-stage timing (acache_stage_timing)
     bool timing = false;
     cudaEvent_t ev[ACACHE_N_STAGES + 1] = {};
@@ -212,6 +213,8 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     if (priv) { g.kv_out_rows = priv->out_rows; g.kv_out_stride = priv->k + priv->e; }
     g.partial = partial; g.status = status; g.grid_bar = grid_bar;
     g.prefetch_blocks = prefetch_by(1);
+    g.debug_expire = c->debug_expire_once;
+    c->debug_expire_once = 0;
     { int nl = launch_gemm(g, st); if (nl < 0) return check_cuda(c, "qkv projection") == ACACHE_OK ? fail(c, ACACHE_ERR_CUDA, "qkv projection launch failed") : ACACHE_ERR_CUDA;
     c->launches += nl; }
 
@@ -441,6 +444,12 @@ acache_status acache_poll_status(acache_ctx* ctx, acache_stream_t stream, uint32
         cudaStreamSynchronize(stream);
         return fail(ctx, ACACHE_ERR_TIMEOUT, "a bounded device-side wait expired");
     }
+    return ACACHE_OK;
+}
+
+acache_status acache_debug_expire_next_wait(acache_ctx* ctx) {
+    if (!ctx) return ACACHE_ERR_INVALID_ARG;
+    ctx->debug_expire_once = 1;
     return ACACHE_OK;
 }
 

@@ -75,14 +75,17 @@ __device__ __forceinline__ int half_source(const GemmArgs& g, const TcPlan& p, i
 // Grid-wide barrier number `k` (1, 2, ...) of this launch on a pair of counters in global
 // memory: arrivals only ever add to bar[0], so barrier k is passed at k * gridDim.x.  Bounded;
 // returns false (and raises the CTA's abort flag) if the others do not arrive.
-__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int k, volatile int* abort_flag) {
+// self_test: the failure-detection self-test (acache_debug_expire_next_wait): the target is one arrival more than
+// the grid can deliver and the poll limit is short, so the wait runs out and the abort path below is taken.
+__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int k, volatile int* abort_flag, bool self_test = false) {
     __syncthreads();
     if (threadIdx.x == 0 && !*abort_flag) {
         __threadfence();
         atomicAdd(&bar[0], 1u);
-        const unsigned int target = k * gridDim.x;
+        const unsigned int target = k * gridDim.x + (self_test ? 1u : 0u);
+        const uint32_t limit = self_test ? (1u << 12) : GRID_WAIT_LIMIT;
         bool ok = false;
-        for (uint32_t i = 0; i < GRID_WAIT_LIMIT; ++i) {
+        for (uint32_t i = 0; i < limit; ++i) {
             unsigned int v;
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
             if (v >= target) { ok = true; break; }
@@ -532,7 +535,7 @@ __device__ __forceinline__ void prep_phase(const GemmArgs& g, float* red, volati
         }
     }
     asm volatile("fence.proxy.async;" ::: "memory");   // the rows are read back through TMA
-    grid_barrier(g.grid_bar, ++nbar, abort_flag);
+    grid_barrier(g.grid_bar, ++nbar, abort_flag, g.debug_expire != 0);
     asm volatile("fence.proxy.async;" ::: "memory");
 }
 
@@ -712,7 +715,16 @@ gemm_tc_kernel(const GemmArgs g, const TcPlan p, const __grid_constant__ CUtenso
     if (*abort_flag) {
         if (threadIdx.x == 0) {
             atomicOr(g.status, kFlagWaitExpired);
-            for (int i = 0; i < 4096; ++i) __nanosleep(64);   // let copies already in flight land
+            // Ring stages whose weight halves were requested before the dependency wait but whose activation tile
+            // never was (the wait that ran out came first): send that tile now, so that the stage's full barrier
+            // completes exactly when all of its copies have landed, and wait for it.  No copy may still be on its
+            // way into this CTA's shared memory when the CTA returns.
+            const uint64_t pol = policy_evict_last();
+            for (int i = 0; i < prefilled; ++i)
+                tma_load_2d(base + i * TC_STAGE_BYTES, &mapA, 0, 0, full_bar(i), pol);
+            for (int i = 0; i < prefilled; ++i)
+                for (uint32_t n = 0; n < TC_WAIT_LIMIT && !mbar_try_wait(full_bar(i), 0); ++n) __nanosleep(40);
+            for (int i = 0; i < 4096; ++i) __nanosleep(64);   // copies of stages that were complete when a role gave up
         }
         __syncthreads();
     } else if (threadIdx.x == 0 && nbar > 0) {

@@ -136,6 +136,8 @@ struct GemmArgs {
     // K blocks past the ring asked into L2 before the dependency wait (0: the default; worth it only behind a long
     // kernel that leaves memory idle)
     int prefetch_blocks;
+    // failure-detection self-test: the grid barrier of the row-preparation phase is given a target it cannot reach
+    int debug_expire;
     // --- kEpiResidual ---
     const void* resid;        // bf16 base pointer
     const int64_t* resid_off; // [M] element offset of the residual row, or null => row * N
