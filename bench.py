@@ -33,10 +33,9 @@ METRIC = "anchor_refresh_affix_tokens_per_s"
 UNIT = "affix tokens/s"
 RATIO = 0.2
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the gate/up GEMM at the default
-# workload (configuration 2, anchors only), from one ncu capture: 202.36 MB read + 5.98 MB written
-# (profiles/layer_step_cfg2_tcgen05.md).  Not captured for other workloads.
-NCU_TRAFFIC_BYTES = {"gate_up": 208334848}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an ncu capture of the kernel as it
+# stands at the commit named here; None until such a capture exists (a figure from an older kernel is not printed).
+NCU_TRAFFIC = {"kernel": None, "bytes": None, "commit": None}
 
 
 def load_peaks():
@@ -67,7 +66,7 @@ def step_work(shape: wl.LayerShape, lay: wl.Layout, K: int):
     params = D * H * d + 2 * D * Hkv * d + H * d * D + 3 * D * Fm
     fl = dict(
         proj=2 * n_r * params + 2 * n_m * D * H * d,
-        score=2 * 2 * n_m * L * H * d,           # logits evaluated twice (statistics + column sums)
+        score=2 * n_m * L * H * d,               # the logits of Eq. 4, counted once
         attn=4 * n_r * T * H * d,
     )
     gate_up_bytes = 2 * Fm * D * 2 + n_r * D * 2 + n_r * Fm * 2
@@ -151,7 +150,8 @@ def run_reference(args):
     dt = (time.perf_counter() - t0) / args.steps
     value = lay.batch * K / dt
     cores = _threads_used()
-    sample = f"{K} of {K_full} anchors per request per step (scoring over all {L} affix keys), {lay.batch} request(s)"
+    sample = (f"{K} of {K_full} anchors per request per step (scoring over all {L} affix keys), {lay.batch} request(s); "
+              f"weights converted bf16 -> fp64 once, outside the timed steps; {cores} BLAS threads")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
@@ -182,11 +182,9 @@ def workload_config(shape, lay, args, K):
 
 
 # ------------------------------------------------------------------------------------------
-def run_ours(args):
+def init_rank():
+    """Device, rank and (for more than one rank) the NCCL process group of this process."""
     import torch
-    from paper_2608_26140_b200 import binding as ab
-    from paper_2608_26140_b200 import build as abuild
-
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -198,6 +196,44 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
+    return rank, world, local, dev, dist
+
+
+def time_blocks(step, steps, n_blocks, sync_all, dist, dev):
+    """Times n_blocks consecutive blocks of exactly `steps` steps each with CUDA events on the launching stream
+    (one event per block boundary, no synchronisation in between); per block the max over ranks.  Returns the
+    per-step times in ms, one per block."""
+    import torch
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_blocks + 1)]
+    sync_all()
+    k = 0
+    ev[0].record()
+    for b in range(n_blocks):
+        for _ in range(steps):
+            step(k)
+            k += 1
+        ev[b + 1].record()
+    sync_all()
+    ms = [ev[b].elapsed_time(ev[b + 1]) / steps for b in range(n_blocks)]
+    if dist is not None:
+        t = torch.tensor(ms, dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = t.tolist()
+    return ms
+
+
+def spread(ms_per_step):
+    v = np.sort(np.asarray(ms_per_step, dtype=np.float64)) * 1e3
+    return {"blocks": int(v.size), "median": float(np.median(v)), "min": float(v[0]), "max": float(v[-1]),
+            "p10": float(v[int(0.1 * (v.size - 1))]), "p90": float(v[int(0.9 * (v.size - 1))]), "unit": "us per step"}
+
+
+def run_ours(args):
+    import torch
+    from paper_2608_26140_b200 import binding as ab
+    from paper_2608_26140_b200 import build as abuild
+
+    rank, world, local, dev, dist = init_rank()
     if rank == 0:
         abuild.build()
     if dist:
@@ -232,24 +268,20 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    def max_over_ranks(ms):
-        return sharding.max_over_ranks(ms, dist, dev)
-
-    for i in range(max(args.warmup, 3)):
+    warmup = max(args.warmup, 3)
+    for i in range(warmup):
         step(i)
     sync_all()
+    # a first block sizes the run: at least 50 blocks of `steps` steps, and enough of them to keep the GPU busy for
+    # about a second, so that the clock sampler sees the load
+    est = time_blocks(step, args.steps, 1, sync_all, dist, dev)[0]
+    n_blocks = int(min(2000, max(50, np.ceil(1000.0 / max(est * args.steps, 1e-3)))))
     sampler = ClockSampler(local)
     sampler.start()
     l0 = ctx.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        step(i)
-    e1.record()
-    sync_all()
-    launches = ctx.launch_count() - l0
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
-    ms_step = ms_total / args.steps
+    blocks = time_blocks(step, args.steps, n_blocks, sync_all, dist, dev)
+    launches_per_step = (ctx.launch_count() - l0) / (n_blocks * args.steps)
+    ms_step = float(np.median(blocks))
 
     # second timed pass over the same steps with an event before every stage
     ctx.stage_timing(True)
@@ -259,8 +291,6 @@ def run_ours(args):
         for s, v in ctx.read_stage_times().items():
             stage[s] += v / args.steps
     ctx.stage_timing(False)
-    sampler.stop_flag = True
-    sampler.join()
     assert ctx.poll_status() == 0, "device status word set during the benchmark"
 
     # end to end: per-step inputs in pinned host memory, results read back to the host
@@ -275,13 +305,10 @@ def run_ours(args):
 
     for i in range(3):
         step_host(i)
-    sync_all()
-    e0.record()
-    for i in range(args.steps):
-        step_host(i)
-    e1.record()
-    sync_all()
-    ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    blocks_e2e = time_blocks(step_host, args.steps, max(50, n_blocks // 4), sync_all, dist, dev)
+    ms_e2e = float(np.median(blocks_e2e))
+    sampler.stop_flag = True
+    sampler.join()
     # page-locked x is read in place: the kernels pull the masked rows, the anchor rows and the anchors' residual rows
     x_in_place = ctx.host_x_in_place(xh) and (lay.n_masked + 2 * n) * 4 <= T    # the entry point's own rule
     h2d = B * (lay.n_masked + 2 * n) * shape.hidden * 2 if x_in_place else xh.numel() * 2
@@ -296,42 +323,225 @@ def run_ours(args):
     step_bytes, step_flops, gu_bytes, gu_flops, n_r = step_work(shape, lay, K)
     t_hbm = step_bytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = step_flops / (peaks["tflops"] * 1e12)
+    floor_s = max(t_hbm, t_tc)
+    hbm_bound = t_hbm >= t_tc
+    s_step = ms_step * 1e-3
     gu_s = stage["gate_up"] * 1e-3
     gu_hbm_bound = gu_bytes / (peaks["hbm_gbs"] * 1e9) >= gu_flops / (peaks["tflops"] * 1e12)
-    if gu_hbm_bound:
-        ach, peak, unit = gu_bytes / gu_s / 1e9, peaks["hbm_gbs"], "GB/s"
-    else:
-        ach, peak, unit = gu_flops / gu_s / 1e12, peaks["tflops"], "TFLOP/s"
-    roofline = {"kernel": "gate/up projection + SwiGLU (stage gate_up)", "bound": "hbm" if gu_hbm_bound else "tensor",
-                "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "peak_source": peaks["source"],
-                "traffic": NCU_TRAFFIC_BYTES["gate_up"] if (args.config == 2 and lay.n_extra == 0 and B == 1) else None,
-                "algorithmic_bytes": gu_bytes, "algorithmic_flops": gu_flops,
-                "us_per_launch": stage["gate_up"] * 1e3}
-    floor_s = max(t_hbm, t_tc)
+    gu_ach, gu_peak, gu_unit = ((gu_bytes / gu_s / 1e9, peaks["hbm_gbs"], "GB/s") if gu_hbm_bound
+                                else (gu_flops / gu_s / 1e12, peaks["tflops"], "TFLOP/s"))
+    # the roofline of the whole fused path: the slower of its bytes at the HBM peak and its flops at the tensor peak,
+    # over the measured time of one layer-step (all its launches)
+    roofline = {"kernel": f"whole layer-step ({launches_per_step:.0f} launches)", "bound": "hbm" if hbm_bound else "tensor",
+                "achieved": (step_bytes / s_step / 1e9) if hbm_bound else (step_flops / s_step / 1e12),
+                "peak": peaks["hbm_gbs"] if hbm_bound else peaks["tflops"], "unit": "GB/s" if hbm_bound else "TFLOP/s",
+                "frac": floor_s / s_step, "peak_source": peaks["source"], "floor_us": floor_s * 1e6,
+                "algorithmic_bytes": step_bytes, "algorithmic_flops": step_flops,
+                "traffic": NCU_TRAFFIC["bytes"], "traffic_of": NCU_TRAFFIC["kernel"], "traffic_commit": NCU_TRAFFIC["commit"],
+                "dominant_kernel": {"kernel": "gate/up projection + SwiGLU (stage gate_up, from the staged pass)",
+                                    "bound": "hbm" if gu_hbm_bound else "tensor", "achieved": gu_ach, "peak": gu_peak,
+                                    "unit": gu_unit, "frac": gu_ach / gu_peak, "algorithmic_bytes": gu_bytes,
+                                    "algorithmic_flops": gu_flops, "us_per_launch": stage["gate_up"] * 1e3}}
     value = sharding.aggregate_throughput(B * K, world, ms_step)
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_step, "us_per_layer_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": workload_config(shape, lay, args, K),
+        "timing": {"protocol": f"{n_blocks} consecutive blocks of {args.steps} layer-steps, one CUDA event per block boundary, "
+                               "max over ranks per block; value and ms_per_step are the median block", **spread(blocks)},
         "clocks": sampler.summary(),
         "e2e": {"value": world * B * K / (ms_e2e * 1e-3), "unit": UNIT, "us_per_layer_step": ms_e2e * 1e3,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "timing": spread(blocks_e2e),
                 "x_transfer": "rows read in place from page-locked host memory by the kernels" if x_in_place
                 else "whole x staged by one copy"},
-        "gpu_launches": int(launches),
+        "gpu_launches": int(round(launches_per_step * args.steps)),
+        "gpu_launches_per_step": launches_per_step,
         "roofline": roofline,
-        "layer_step_roofline": {"bound": "hbm" if t_hbm >= t_tc else "tensor", "algorithmic_bytes": step_bytes,
-                                "algorithmic_flops": step_flops, "floor_us": floor_s * 1e6,
-                                "frac": floor_s / (ms_step * 1e-3), "peak_source": peaks["source"]},
         "stage_us": {s: v * 1e3 for s, v in stage.items()},
         "affix_tokens_covered_per_s": world * B * L / (ms_step * 1e-3),
     }
+    if world == 1 and not args.no_extra:
+        # free the headline workload's buffers, then the other configurations the metric names, each a short run
+        del inst, ctx, xh, yh
+        torch.cuda.empty_cache()
+        out["extra"] = extra_records(args, peaks, dev)
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(case, shape, lay)
     print(json.dumps(out))
     if dist:
         dist.destroy_process_group()
+
+
+def extra_records(args, peaks, dev):
+    """Short measurements of the other workloads the metric names, carried in the same JSON line: one denoising step
+    at benchmark configuration 3 (32 layers, vocabulary 126464, 16 requests), three points of the configuration-5
+    sweep, configuration 2 with every request row recomputed, and the KV-deviation scoring kernel.  All inputs are
+    drawn on the device (timing only; parity at these sizes is in the tests)."""
+    import torch
+    from paper_2608_26140_b200 import binding as ab
+    out = {}
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.SEED_BASE + 77)
+
+    def randn(shape_, std=1.0):
+        t = torch.randn(shape_, generator=gen, device=dev, dtype=torch.bfloat16)
+        return t.mul_(std) if std != 1.0 else t
+
+    def dev_weights(shape, std=0.02):
+        D, F = shape.hidden, shape.ffn
+        dims = dict(wq=(shape.q_dim, D), wk=(shape.kv_dim, D), wv=(shape.kv_dim, D), wo=(D, shape.q_dim),
+                    w_gate=(F, D), w_up=(F, D), w_down=(D, F))
+        w = {k: randn(v, std) for k, v in dims.items()}
+        w["attn_norm_g"] = randn((D,), 0.05).add_(1.0)
+        w["mlp_norm_g"] = randn((D,), 0.05).add_(1.0)
+        w["bq"] = w["bk"] = w["bv"] = None
+        return w
+
+    def timed(fn, steps, warm):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        ev[0].record()
+        for i in range(steps):
+            fn()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        return [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+
+    shape = wl.LLADA_8B
+    kv_std = 0.02 * float(np.sqrt(shape.hidden))
+
+    # ---- configuration 3: acache_denoise_step, 32 layers + LM head + commit
+    n_layers, V, n_blk = 32, 126464, 32
+    lay = wl.config_layout(3, "all", n_masked=32, batch=16)
+    B, T, L, P = lay.batch, lay.ctx_len, lay.affix_len, lay.n_extra
+    K = ab.k_from_ratio(L, RATIO)
+    n = K + P
+    ws = [dev_weights(shape) for _ in range(n_layers)]
+    lws = [ab.Context.weights(w) for w in ws]
+    dk = [randn((B, T, shape.n_kv_heads, shape.head_dim), kv_std) for _ in range(n_layers)]
+    dv = [randn((B, T, shape.n_kv_heads, shape.head_dim), kv_std) for _ in range(n_layers)]
+    kvs = [ab.Context.kv(dk[i], dv[i]) for i in range(n_layers)]
+    embed, w_lm = randn((V, shape.hidden)), randn((V, shape.hidden), 0.02)
+    gain = randn((shape.hidden,), 0.05).add_(1.0)
+    g = np.random.Generator(np.random.Philox(wl.SEED_BASE + 4096 * 3 + 43))
+    ids = g.integers(0, V - 1, size=(B, T)).astype(np.int32)
+    ids[:, lay.affix_start:lay.affix_start + L] = ids[0, lay.affix_start:lay.affix_start + L]
+    ids[:, lay.masked_pos[0]] = V - 1
+    anchors = np.stack([np.sort(g.choice(L, K, replace=False)) for _ in range(B)]).astype(np.int32)
+    where = {int(p): i for i, p in enumerate(lay.extra_rows[0])}
+    block_rows = np.stack([[K + where[int(p)] for p in lay.masked_pos[b][:n_blk]] for b in range(B)]).astype(np.int32)
+    cos_h, sin_h = wl.rope_table(T, shape.head_dim, shape.rope_theta)
+    cos, sin = torch.from_numpy(cos_h).to(dev), torch.from_numpy(sin_h).to(dev)
+    masked = torch.from_numpy(lay.masked_pos.copy()).to(dev)
+    extra = torch.from_numpy(lay.extra_rows.copy()).to(dev)
+    dids = torch.from_numpy(ids).to(dev)
+    req = ab.Context.request(B, T, lay.affix_start, L, masked, extra, cos, sin, token_ids=dids, n_embed=V)
+    ctx = ab.Context.for_shape(shape, B, T, L, n, lay.n_masked, dev, max_vocab=V, max_block=n_blk)
+    ya = torch.zeros((B, n, shape.hidden), dtype=torch.bfloat16, device=dev)
+    yb = torch.zeros_like(ya)
+    da, dbr = torch.from_numpy(anchors).to(dev), torch.from_numpy(block_rows).to(dev)
+    token = torch.zeros((B, n_blk), dtype=torch.int32, device=dev)
+    conf = torch.zeros((B, n_blk), dtype=torch.float32, device=dev)
+    commit = torch.zeros((B, n_blk), dtype=torch.int32, device=dev)
+    sampler = ClockSampler(int(dev.split(":")[1]))
+    sampler.start()
+    l0 = ctx.launch_count()
+    ms = timed(lambda: ctx.denoise_step(lws, kvs, req, embed, da, K, ya, yb, dbr, n_blk, gain, w_lm, V, 0.9, token, conf, commit),
+               steps=4, warm=2)
+    launches = (ctx.launch_count() - l0) / 6
+    sampler.stop_flag = True
+    sampler.join()
+    assert ctx.poll_status() == 0
+    step_bytes, step_flops, _, _, _ = step_work(shape, lay, K)
+    D, H, d = shape.hidden, shape.n_heads, shape.head_dim
+    layer_flops = step_flops - 2 * B * lay.n_masked * D * H * d - 2 * B * lay.n_masked * L * H * d   # a refresh layer scores nothing
+    flops = n_layers * layer_flops + 2 * B * n_blk * D * V
+    bytes_ = n_layers * step_bytes + 2 * V * D
+    floor_s = max(flops / (peaks["tflops"] * 1e12), bytes_ / (peaks["hbm_gbs"] * 1e9))
+    med = float(np.median(ms))
+    out["config3_denoise_step"] = {
+        "workload": f"cfg3: LLaDA-8B shapes, {n_layers} layers (each its own weights and caches), vocab {V}, batch {B} sharing a "
+                    f"{L}-token prefix affix, {P} request rows each, ratio {RATIO} (K={K}), {n} rows recomputed per request "
+                    f"({B * n} per layer), {n_blk}-token block; acache_denoise_step = refresh forward + LM head + commit",
+        "denoise_steps_per_s": 1e3 / med, "ms_per_step": med, "ms_per_step_min": float(min(ms)), "ms_per_step_max": float(max(ms)),
+        "steps": len(ms), "warmup": 2, "gpu_launches_per_step": launches,
+        "roofline": {"bound": "tensor", "achieved": flops / (med * 1e-3) / 1e12, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                     "frac": floor_s / (med * 1e-3), "floor_ms": floor_s * 1e3, "algorithmic_flops": flops,
+                     "algorithmic_bytes": bytes_, "peak_source": peaks["source"]},
+        "affix_tokens_refreshed_per_s": B * K * n_layers / (med * 1e-3), "clocks": sampler.summary(),
+        "data": "synthetic, drawn on the device"}
+    del ws, lws, dk, dv, kvs, embed, w_lm, ctx, ya, yb
+    torch.cuda.empty_cache()
+
+    # ---- layer-steps: configuration 2 with all request rows, three configuration-5 sweep points
+    winst = [dev_weights(shape) for _ in range(3)]
+    wl_inst = [ab.Context.weights(w) for w in winst]
+    points = [("config2_all_request_rows", wl.config_layout(2, "all", n_masked=32, batch=1), RATIO),
+              ("sweep_L8192_B1_r0.2", wl.sweep_layout(8192, 1, "prefix", "none"), 0.2),
+              ("sweep_L2048_B8_r0.2", wl.sweep_layout(2048, 8, "prefix", "none"), 0.2),
+              ("sweep_L512_B64_r0.2", wl.sweep_layout(512, 64, "prefix", "none"), 0.2)]
+    for name, lay, ratio in points:
+        B, T, L = lay.batch, lay.ctx_len, lay.affix_len
+        K = ab.k_from_ratio(L, ratio)
+        n = K + lay.n_extra
+        n_c = 3 if B * T * shape.hidden * 2 < (1 << 28) else 1
+        xs = [randn((B, T, shape.hidden)) for _ in range(n_c)]
+        cks = [randn((B, T, shape.n_kv_heads, shape.head_dim), kv_std) for _ in range(n_c)]
+        cvs = [randn((B, T, shape.n_kv_heads, shape.head_dim), kv_std) for _ in range(n_c)]
+        l = lay.affix_start
+        for t in xs + cks + cvs:
+            t[1:, l:l + L] = t[0:1, l:l + L]
+        cos_h, sin_h = wl.rope_table(T, shape.head_dim, shape.rope_theta)
+        cos, sin = torch.from_numpy(cos_h).to(dev), torch.from_numpy(sin_h).to(dev)
+        masked = torch.from_numpy(lay.masked_pos.copy()).to(dev)
+        extra = torch.from_numpy(lay.extra_rows.copy()).to(dev) if lay.n_extra else None
+        req = ab.Context.request(B, T, l, L, masked, extra, cos, sin)
+        ctx = ab.Context.for_shape(shape, B, T, L, n, lay.n_masked, dev)
+        scores = torch.zeros((B, L), dtype=torch.float32, device=dev)
+        anchors_d = torch.zeros((B, K), dtype=torch.int32, device=dev)
+        y = torch.zeros((B, n, shape.hidden), dtype=torch.bfloat16, device=dev)
+        it = [0]
+
+        def step():
+            i = it[0]
+            it[0] += 1
+            ctx.layer_step(wl_inst[i % 3], req, ab.Context.kv(cks[i % n_c], cvs[i % n_c]), xs[i % n_c], 0, ratio,
+                           ab.F_SCORE | ab.F_SELECT, scores, anchors_d, y)
+
+        ms = timed(step, steps=30, warm=5)
+        ctx.stage_timing(True)
+        stage = {s_: 0.0 for s_ in ab.STAGES}
+        for _ in range(5):
+            step()
+            for s_, v in ctx.read_stage_times().items():
+                stage[s_] += v / 5
+        ctx.stage_timing(False)
+        assert ctx.poll_status() == 0
+        step_bytes, step_flops, _, _, n_r = step_work(shape, lay, K)
+        t_hbm, t_tc = step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (peaks["tflops"] * 1e12)
+        med = float(np.median(ms)) * 1e-3
+        out[name] = {"workload": f"{lay.name}: LLaDA-8B layer, batch {B}, affix {L}, context {T}, {lay.n_masked} masked rows, "
+                                 f"ratio {ratio} (K={K}), {n} rows per request",
+                     "us_per_layer_step": med * 1e6, "us_min": float(min(ms)) * 1e3, "us_max": float(max(ms)) * 1e3, "steps": len(ms),
+                     "affix_tokens_per_s": B * K / med, "rows": n_r,
+                     "roofline": {"bound": "hbm" if t_hbm >= t_tc else "tensor", "floor_us": max(t_hbm, t_tc) * 1e6,
+                                  "frac": max(t_hbm, t_tc) / med, "achieved_gbs": step_bytes / med / 1e9,
+                                  "achieved_tflops": step_flops / med / 1e12, "peak_source": peaks["source"]},
+                     "stage_us": {k_: round(v * 1e3, 1) for k_, v in stage.items() if v}}
+        if name == "sweep_L2048_B8_r0.2":
+            # the KV-deviation selector's scoring kernel on the same caches (HBM-bound: four affix rows per token)
+            ms_d = timed(lambda: ctx.score_kv_deviation(req, ab.Context.kv(cks[0], cvs[0]), ab.Context.kv(cks[-1], cvs[-1]), scores),
+                         steps=20, warm=3)
+            by = 4 * B * L * shape.kv_dim * 2
+            md = float(np.median(ms_d)) * 1e-3
+            out["kv_deviation_scores_L2048_B8"] = {"us": md * 1e6, "algorithmic_bytes": by, "achieved_gbs": by / md / 1e9,
+                                                   "frac_of_hbm_peak": by / md / 1e9 / peaks["hbm_gbs"]}
+        del ctx, xs, cks, cvs, y
+        torch.cuda.empty_cache()
+    return out
 
 
 # ------------------------------------------------------------------------------------------
@@ -841,24 +1051,33 @@ def run_shared(args):
 
 
 def cpu_baseline(case, shape, lay):
-    """The oracle as it stands, timed on this machine's host cores on one step of the workload."""
+    """The oracle as it stands, timed on this machine's host cores on full layer-steps of the workload: the same
+    program and the same protocol as `--impl reference` (weights converted bf16 -> fp64 once, outside the timed
+    steps; numpy's BLAS threads as the box gives them)."""
     from oracle import acache_oracle as orc
     L = lay.affix_len
     K = orc.k_from_ratio(L, RATIO)
+    w64 = {k: (orc.bf16_bits_to_f64(v) if v is not None else None) for k, v in case.weights.items()}
+
+    def one_step():
+        for b in range(lay.batch):
+            orc.layer_step(w64, shape, case.x[b], case.cache_k[b], case.cache_v[b], lay.ctx_len,
+                           lay.affix_start, L, lay.masked_pos[b], lay.extra_rows[b], case.rope_cos, case.rope_sin, K=K)
+
+    one_step()                                   # warm-up (page-in, BLAS thread pool)
     t0 = time.perf_counter()
     reps = 0
     while True:
-        for b in range(lay.batch):
-            orc.layer_step(case.weights, shape, case.x[b], case.cache_k[b], case.cache_v[b], lay.ctx_len,
-                           lay.affix_start, L, lay.masked_pos[b], lay.extra_rows[b], case.rope_cos, case.rope_sin,
-                           ratio=RATIO)
+        one_step()
         reps += 1
-        if time.perf_counter() - t0 > 10.0 or reps >= 3:
+        if time.perf_counter() - t0 > 10.0 or reps >= 20:
             break
     dt = (time.perf_counter() - t0) / reps
-    return {"value": lay.batch * K / dt, "unit": UNIT, "cores": _threads_used(), "kind": "oracle",
+    cores = _threads_used()
+    return {"value": lay.batch * K / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{reps} full layer-step(s) of the same workload ({lay.batch} request(s), {K} anchors each), "
-                      f"{dt:.2f} s per step including the oracle's own bf16->fp64 weight conversion"}
+                      f"{dt:.3f} s per step; weights converted bf16 -> fp64 once, outside the timed steps; "
+                      f"{cores} BLAS threads (numpy matmul, fp64)"}
 
 
 def main():
@@ -873,6 +1092,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--instances", type=int, default=4, help="weight/cache instances rotated between steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="default run only: skip the short configuration-3 / sweep / selector measurements (key `extra`)")
     ap.add_argument("--layers", type=int, default=32, help="layers of the --config 3 denoising step")
     ap.add_argument("--shared", action="store_true",
                     help="--config 3 or 4: one layer with shared affix storage (batch_stride 0) against private caches")
@@ -884,7 +1105,20 @@ def main():
     ap.add_argument("--sweep-affix", default=None, help="--config 5: comma-separated affix lengths (default 512,2048,8192)")
     ap.add_argument("--sweep-batch", default=None, help="--config 5: comma-separated batch sizes (default 1,8,64)")
     ap.add_argument("--sweep-out", default=None, help="--config 5: also write the points as a markdown table to this file")
+    ap.add_argument("--rank-echo", action="store_true", help=argparse.SUPPRESS)   # every rank prints who it is and exits (no GPU)
     args = ap.parse_args()
+    plan, world = sharding.launch_plan(args.gpus, os.environ)
+    if plan == "refuse":
+        raise SystemExit(f"--gpus {args.gpus} but this process is rank of a {world}-rank job: start it with "
+                         f"--nproc-per-node {args.gpus} (or without a launcher: bench.py starts its own ranks)")
+    if plan == "spawn":
+        # no launcher around this process: start the N ranks (one per GPU) and hand them the same arguments
+        import subprocess
+        cmd = sharding.torchrun_command(os.path.abspath(__file__), sys.argv[1:], args.gpus, sharding.free_port())
+        raise SystemExit(subprocess.call(cmd))
+    if args.rank_echo:
+        print(json.dumps({"rank": int(os.environ.get("RANK", "0")), "world": world, "gpus": args.gpus}), flush=True)
+        return
     if args.impl == "reference":
         run_reference(args)
     elif args.shared and args.config in (3, 4) and not args.generate:

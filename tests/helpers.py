@@ -15,6 +15,16 @@ DEV = "cuda:0"
 TOL = 2e-2     # max relative error of refreshed K/V and layer outputs (bf16 storage, fp32 accumulate)
 
 
+def e2e_tol(n_layers: int) -> float:
+    """Gate of an END-TO-END comparison over ``n_layers`` layers (the oracle fed its own layer outputs, not the
+    GPU's).  Every layer adds an error of its own of the single-layer size (at most TOL, the gate of one
+    layer-step) to the one it inherits, and the residual stream hands the inherited error on with gain close to
+    one, so the errors add: n_layers * TOL.  The checks that pin each layer are the teacher-forced ones (oracle
+    layer n fed the GPU's layer-n input), which hold at TOL itself; this looser gate only guards against drift
+    that teacher forcing cannot see."""
+    return n_layers * TOL
+
+
 @functools.lru_cache(maxsize=2)
 def cached_weights(shape, cfg_id):
     """Layer weights of (shape, cfg_id), drawn once per test session (read-only)."""

@@ -9,7 +9,7 @@ from oracle import acache_oracle as orc
 from paper_2608_26140_b200 import binding as ab
 from paper_2608_26140_b200 import workloads as wl
 
-from helpers import DEV, TOL, assert_close_bf16
+from helpers import DEV, TOL, assert_close_bf16, e2e_tol
 
 pytestmark = pytest.mark.gpu
 
@@ -82,25 +82,40 @@ def test_probe_select_refresh(shape, n_layers, norm_full):
     for b in range(B):
         s_ref, probe_caches, probe_ys = orc.probe_forward(layers, shape, x[b], caches[b], T, l, L, lay.masked_pos[b],
                                                          lay.extra_rows[b], cos, sin, norm_full)
+        # scores with teacher forcing: layer n's term (Eq. 4) from the oracle fed the GPU's own layer-n input rows,
+        # summed over the layers (Eq. 5): the single-layer tolerance holds
+        rows_p = np.asarray(lay.extra_rows[b], dtype=np.int64)
+        where = {int(p): i for i, p in enumerate(rows_p)}
+        mask_idx = np.array([where[int(p)] for p in lay.masked_pos[b]])
+        s_tf = np.zeros(L)
+        for n in range(n_layers):
+            x_rows = orc.bf16_bits_to_f64(x[b])[rows_p] if n == 0 else orc.bf16_bits_to_f64(ab.to_host_bits(y[n - 1][b]))
+            r = orc.recompute_rows(layers[n], shape, x_rows, rows_p, caches[b][n][0], caches[b][n][1], T, cos, sin)
+            Kall = orc.bf16_bits_to_f64(caches[b][n][0][:T])
+            s_tf += orc.score_anchors(r["q"][mask_idx], Kall[l:l + L], Kall, l, norm_full)
+        err_tf = np.abs(s_gpu[b] - s_tf) / np.maximum(s_tf, s_tf.mean())
+        assert err_tf.max() < 1e-3, err_tf.max()
+        # end to end the later layers' queries come from hidden rows that already differ by the earlier layers'
+        # rounding, so the scores' gate grows with the layer count like the outputs' (helpers.e2e_tol)
         err = np.abs(s_gpu[b] - s_ref) / np.maximum(s_ref, s_ref.mean())
-        assert err.max() < 2e-3, err.max()            # later layers see the GPU's own (rounded) hidden rows
+        assert err.max() < 1e-3 * n_layers, err.max()
         _, _, must, may = orc.select_topk(s_ref.astype(np.float32), K)
         ok, why = orc.anchor_set_ok(a_gpu[b], K, L, must, may)
         assert ok, why
-        assert_close_bf16(ab.to_host_bits(y[-1][b]), probe_ys[-1], "probe output, end to end", 2 * TOL)
+        assert_close_bf16(ab.to_host_bits(y[-1][b]), probe_ys[-1], "probe output, end to end", e2e_tol(n_layers))
         # end to end with the GPU's anchor set
         rows, ref_caches, ref_ys = orc.refresh_forward(layers, shape, x[b], caches[b], T, l, a_gpu[b],
                                                        lay.extra_rows[b], cos, sin)
-        assert_close_bf16(ab.to_host_bits(yr[-1][b]), ref_ys[-1], "refresh output, end to end", 2 * TOL)
+        assert_close_bf16(ab.to_host_bits(yr[-1][b]), ref_ys[-1], "refresh output, end to end", e2e_tol(n_layers))
         keep = np.setdiff1d(np.arange(T), rows)
         for n in range(n_layers):
             ckb = ab.to_host_bits(dk[n][b])
             assert np.array_equal(ckb[keep], caches[b][n][0][keep]), "non-anchor affix rows changed"
-            assert_close_bf16(ckb[rows], ref_caches[n][0][rows], f"layer {n} K rows", 2 * TOL)
+            assert_close_bf16(ckb[rows], ref_caches[n][0][rows], f"layer {n} K rows", e2e_tol(n_layers))
         # layer-wise teacher forcing: the oracle fed the GPU's layer-n input reproduces its layer-n output
-        for n in range(1, n_layers):
-            xin = ab.to_host_bits(yr[n - 1][b])
-            r = orc.recompute_rows(layers[n], shape, orc.bf16_bits_to_f64(xin), rows, caches[b][n][0], caches[b][n][1],
+        for n in range(n_layers):
+            xin = orc.bf16_bits_to_f64(x[b])[rows] if n == 0 else orc.bf16_bits_to_f64(ab.to_host_bits(yr[n - 1][b]))
+            r = orc.recompute_rows(layers[n], shape, xin, rows, caches[b][n][0], caches[b][n][1],
                                    T, cos, sin)
             assert_close_bf16(ab.to_host_bits(yr[n][b]), r["y"], f"layer {n} output, teacher forced")
             assert_close_bf16(ab.to_host_bits(dv[n][b])[rows], r["v_new"], f"layer {n} V rows, teacher forced")

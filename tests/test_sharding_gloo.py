@@ -72,3 +72,33 @@ def test_two_gloo_ranks_cover_the_batch(tmp_path):
     port = _free_port()
     mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     assert (tmp_path / "ok").exists()
+
+
+def test_launch_plan_and_self_start_command():
+    assert sharding.launch_plan(1, {}) == ("run", 1)
+    assert sharding.launch_plan(8, {}) == ("spawn", 8)
+    assert sharding.launch_plan(8, {"WORLD_SIZE": "8"}) == ("run", 8)
+    assert sharding.launch_plan(8, {"WORLD_SIZE": "1"}) == ("refuse", 1)
+    assert sharding.launch_plan(1, {"WORLD_SIZE": "2"}) == ("refuse", 2)
+    cmd = sharding.torchrun_command("bench.py", ["--gpus", "4", "--steps", "7"], 4, 29511)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29511"
+    assert cmd[-5:] == ["bench.py", "--gpus", "4", "--steps", "7"]
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`python bench.py --gpus 2` with no WORLD_SIZE around it starts two ranks of itself (each prints who it is
+    and leaves: no GPU here); under a launcher with another rank count it refuses."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--rank-echo"], env=env, capture_output=True,
+                       text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    seen = sorted(json.loads(l)["rank"] for l in r.stdout.splitlines() if l.startswith("{"))
+    assert seen == [0, 1]
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--rank-echo"], env={**env, "WORLD_SIZE": "1"},
+                       capture_output=True, text=True, timeout=120)
+    assert r.returncode != 0 and "bench.py starts its own ranks" in r.stderr
