@@ -392,7 +392,9 @@ def probe_forward(layers, shape, x0: np.ndarray, caches, ctx_len: int, affix_sta
 
     layers: list of weight dicts; x0 [T, D] bf16 bits (layer-0 input); caches: list of
     (cache_k, cache_v) bf16 bits per layer; probe_rows: absolute positions P (must contain masked_pos).
-    The scores of layer n use that layer's cache as it is before the probe writes its own rows.
+    The affix keys are the cached (stale) ones.  With ``norm_full`` the softmax of Eq. 4 runs over every key the
+    probe's own attention sees: the affix keys as cached plus the probe rows' fresh keys (Section 3.2: the probe
+    attends with the affix as past KV), i.e. the working cache of this layer.
     Returns (scores fp64 [L], list of working caches, list of per-layer outputs y [|P|, D]).
     """
     rows = np.asarray(probe_rows, dtype=np.int64)
@@ -403,7 +405,7 @@ def probe_forward(layers, shape, x0: np.ndarray, caches, ctx_len: int, affix_sta
     out_caches, ys = [], []
     for W, (ck, cv) in zip(layers, caches):
         r = recompute_rows(W, shape, x_rows, rows, ck, cv, ctx_len, cos, sin, round_storage)
-        Kall = bf16_bits_to_f64(ck[:ctx_len])
+        Kall = bf16_bits_to_f64((r["cache_k"] if norm_full else ck)[:ctx_len])
         s += score_anchors(r["q"][mask_idx], Kall[affix_start:affix_start + affix_len], Kall, affix_start, norm_full)
         x_rows = r["y"]
         out_caches.append((r["cache_k"], r["cache_v"]))

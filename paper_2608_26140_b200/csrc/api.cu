@@ -7,6 +7,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <functional>
 #include <new>
 #include <string>
 
@@ -23,6 +24,7 @@ struct acache_ctx {
     // workspace offsets (bytes)
     size_t o_status, o_row_pos, o_row_pos2, o_row_src, o_xn, o_q, o_o, o_h1, o_xn2, o_act, o_knew, o_vnew;
     size_t o_mrow_pos, o_mrow_src, o_xn_mask, o_qmask, o_stats, o_partial, o_slot;
+    size_t o_rowmask, partial_bytes;
     size_t o_xstage, o_ystage, o_sstage, o_astage, o_gemm, o_attn, o_gridbar, o_mcidx, o_lstats, o_lxn, o_keymask;
     std::string err;
     uint64_t launches = 0;
@@ -155,6 +157,14 @@ static int prefetch_by(int which) {
     }();
     return v[which];
 }
+// Eq. 4-5 taken from the attention of the rows being recomputed (the probe of Section 3.2: the masked rows are among them)
+struct FusedScore {
+    const uint32_t* rowmask;
+    int rm_words;
+    float* scores;
+    int accumulate;
+    int norm_full;          // Eq. 4's softmax over every key (the attention's own denominator) instead of the affix keys
+};
 struct PrivateRows {
     const int32_t* anchor_idx;
     int k;
@@ -169,7 +179,9 @@ struct MapReuse { bool reuse; };
 acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const acache_request* r,
                             const acache_kv* kv, bool fuse_scatter, const void* x, int x_is_compact,
                             const int32_t* anchor_idx, int k, void* k_new, void* v_new, void* y, cudaStream_t st,
-                            const PrivateRows* priv = nullptr, MapReuse maps = MapReuse{false}, bool drop_non_anchor = false) {
+                            const PrivateRows* priv = nullptr, MapReuse maps = MapReuse{false}, bool drop_non_anchor = false,
+                            const FusedScore* fs = nullptr,
+                            const std::function<acache_status()>& after_qkv = std::function<acache_status()>()) {
     const acache_model_desc& d = c->d;
     const int rows = k + r->n_extra, n = r->batch * rows;
     if (n == 0) {
@@ -218,6 +230,10 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     { int nl = launch_gemm(g, st); if (nl < 0) return check_cuda(c, "qkv projection") == ACACHE_OK ? fail(c, ACACHE_ERR_CUDA, "qkv projection launch failed") : ACACHE_ERR_CUDA;
     c->launches += nl; }
 
+    if (after_qkv) {            // work of the caller that wants the fresh K/V in place but precedes the attention
+        const acache_status sq = after_qkv();
+        if (sq != ACACHE_OK) return sq;
+    }
     mark(c, ACACHE_STAGE_ATTENTION, st);
     AttnArgs at{};
     at.q = q; at.cache_k = kv->k; at.cache_v = kv->v; at.kv_batch_stride = kv->batch_stride;
@@ -266,7 +282,16 @@ acache_status run_recompute(acache_ctx* c, const acache_layer_weights* w, const 
     at.status = status;
     at.part_o = wsp<float>(c, c->o_attn);
     at.part_ml = at.part_o + (size_t)2 * 296 * 64 * d.head_dim;
+    if (fs) {
+        at.score_rowmask = fs->rowmask; at.rm_words = fs->rm_words; at.score_partial = wsp<float>(c, c->o_partial);
+        at.affix_start = r->affix_start; at.affix_len = r->affix_len; at.score_norm_full = fs->norm_full;
+    }
     c->launches += launch_attention(at, st);
+    if (fs) {
+        launch_score_reduce_tiles(wsp<float>(c, c->o_partial), fs->rowmask, fs->rm_words, fs->scores, r->batch, d.n_heads,
+                                  (rows + 127) / 128, r->affix_len, fs->accumulate, st);
+        c->launches += 1;
+    }
 
     mark(c, ACACHE_STAGE_OPROJ, st);
     GemmArgs go{};
@@ -352,7 +377,15 @@ acache_status acache_create(const acache_model_desc* desc, acache_ctx** out) {
     c->o_xn_mask = take(cur, nm * d.hidden * 2);
     c->o_qmask = take(cur, nm * qd * 2);
     c->o_stats = take(cur, (size_t)d.max_batch * d.n_heads * score_num_splits(d.max_ctx) * d.max_masked * 8);
-    c->o_partial = take(cur, (size_t)d.max_batch * d.n_heads * d.max_affix * 4);
+    {
+        // per-head column sums [B, H, L]; when the scores come out of the probe's attention, per (head, query tile):
+        // [B, H, ceil(rows / 128), L], as far as that stays within 256 MB (else the separate scoring kernels run)
+        const size_t per_head = (size_t)d.max_batch * d.n_heads * d.max_affix * 4;
+        const size_t tiles = (size_t)(d.max_rows + 127) / 128;
+        c->partial_bytes = d.head_dim == 128 && per_head * tiles <= ((size_t)256 << 20) ? per_head * std::max<size_t>(tiles, 1) : per_head;
+        c->o_partial = take(cur, c->partial_bytes);
+    }
+    c->o_rowmask = take(cur, (size_t)d.max_batch * ((d.max_rows + 31) / 32 + 8) * 4);
     c->o_slot = take(cur, (size_t)d.max_batch * d.max_ctx * 4);
     c->o_keymask = take(cur, (size_t)d.max_batch * (2 * ((d.max_ctx + 31) / 32) + (d.max_rows + 31) / 32 + 4) * 4);
     c->o_xstage = take(cur, (size_t)d.max_batch * d.max_ctx * d.hidden * 2);
@@ -559,56 +592,85 @@ acache_status layer_step_impl(acache_ctx* ctx, const acache_layer_weights* w, co
 
     if (ctx->timing) for (bool& h : ctx->ev_hit) h = false;
     bool fused_head_sum = false;
-    if (do_score && req->batch > 0 && req->affix_len > 0) {
-        void* qmask = wsp<void>(ctx, ctx->o_qmask);
-        mark(ctx, ACACHE_STAGE_MASK_Q, stream);
-        if (req->n_masked > 0) {
-            int32_t* mpos = wsp<int32_t>(ctx, ctx->o_mrow_pos);
-            void* xnm = wsp<void>(ctx, ctx->o_xn_mask);
-            GemmArgs g{};
-            g.a = xnm; g.M = req->batch * req->n_masked; g.K = d.hidden;
-            g.prep.enabled = 1; g.prep.x = x; g.prep.x_is_compact = x_is_compact;
-            if (x_is_compact) {
-                // the masked rows are among the extra rows of the compact input: find where
-                int32_t* cidx = wsp<int32_t>(ctx, ctx->o_mcidx);
-                launch_match_rows(req->masked_pos, req->n_masked, req->extra_rows, req->n_extra, k, req->batch, cidx,
-                                  wsp<uint32_t>(ctx, ctx->o_status), stream);
-                ctx->launches += 1;
-                g.prep.compact_idx = cidx;
-                g.prep.compact_rows = k + req->n_extra;
-            }
-            g.prep.x_batch_stride = (int64_t)req->ctx_len * d.hidden;
-            g.prep.anchor_idx = nullptr; g.prep.k = 0; g.prep.extra_rows = req->masked_pos; g.prep.e = req->n_masked;
-            g.prep.affix_start = req->affix_start; g.prep.affix_len = req->affix_len; g.prep.ctx_len = req->ctx_len;
-            g.prep.gain = w->attn_norm_g; g.prep.eps = d.rms_eps; g.prep.row_pos = mpos;
-            g.prep.row_src = wsp<int64_t>(ctx, ctx->o_mrow_src);
-            if (!x_is_compact && req->token_ids) { g.prep.token_ids = req->token_ids; g.prep.table_rows = req->n_embed; }
-            g.b[0] = w->wq; g.n[0] = d.n_heads * d.head_dim;
-            // W_q is read again by the Q/K/V projection a few kernels later: leave it in L2 (measured: that
-            // projection 43.7 -> 40.8 us at 103 rows)
-            static const int keep_wq = [] { const char* e = getenv("ACACHE_KEEP_WQ"); return e ? atoi(e) : 1; }();
-            g.keep_weights = keep_wq && do_recompute;      // a scoring-only pass (the probe) never reads W_q again
-            g.epilogue = kEpiQKV;
-            g.bias[0] = d.qkv_bias ? w->bq : nullptr;
-            g.row_pos = mpos; g.rope_cos = req->rope_cos; g.rope_sin = req->rope_sin;
-            g.head_dim = d.head_dim; g.rope_segments = 1; g.out[0] = qmask; g.rows_per_req = req->n_masked;
-            g.partial = wsp<float>(ctx, ctx->o_gemm); g.status = wsp<uint32_t>(ctx, ctx->o_status);
-            g.grid_bar = wsp<unsigned int>(ctx, ctx->o_gridbar);
-            g.prefetch_blocks = prefetch_by(0);
-            { int nl = launch_gemm(g, stream); if (nl < 0) return check_cuda(ctx, "masked-row query projection") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "masked-row query projection launch failed") : ACACHE_ERR_CUDA;
-            ctx->launches += nl; }
-        }
-        mark(ctx, ACACHE_STAGE_SCORE, stream);
-        // with a selection to follow, the ordered sum over heads is folded into the selection kernel
-        // (only while one CTA per request can read all heads' partial sums quickly: at L = 8192 the separate,
-        // grid-wide head sum takes 4 us where the folded one took 28)
-        fused_head_sum = do_select && k > 0 && req->n_masked > 0 && (int64_t)req->affix_len * d.n_heads <= 65536;
-        // the masked rows' projection was launched just above: nothing that writes the cache is the scoring kernels'
-        // direct predecessor, so they may request their first key tiles early
-        s = run_score(ctx, req, qmask, kv, scores, (flags & ACACHE_F_ACCUMULATE) ? 1 : 0,
-                      (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, fused_head_sum ? 1 : 0, stream, req->n_masked > 0 ? 1 : 0);
-        if (s != ACACHE_OK) return s;
+    // The probe (Section 3.2): no anchors, no selection in this call, the masked rows among the rows being recomputed, the
+    // softmax of Eq. 4 over the affix keys.  Its scores are the masked-to-affix part of its own attention: no query
+    // projection of the masked rows and no pass over the affix keys of their own.
+    static const bool fuse_on = [] { const char* e = getenv("ACACHE_SCORE_FUSED"); return !e || atoi(e) != 0; }();
+    FusedScore fs{};
+    bool score_in_attention = false;
+    static const bool attn_tc_on = [] { const char* e = getenv("ACACHE_ATTN_TC"); return !(e && e[0] == '0'); }();
+    if (fuse_on && attn_tc_on && !to_slots && do_score && !do_select && do_recompute && k == 0 && d.head_dim == 128 &&
+        req->batch > 0 && req->affix_len > 0 && req->n_masked > 0 && req->n_extra > 0 && (kv->batch_stride & 7) == 0 &&
+        (size_t)req->batch * d.n_heads * ((req->n_extra + 127) / 128) * req->affix_len * 4 <= ctx->partial_bytes) {
+        fs.rm_words = (req->n_extra + 31) / 32;
+        uint32_t* rm = wsp<uint32_t>(ctx, ctx->o_rowmask);
+        launch_row_mask(req->masked_pos, req->n_masked, req->extra_rows, req->n_extra, 0, req->batch, rm, fs.rm_words,
+                        wsp<uint32_t>(ctx, ctx->o_status), stream);
+        ctx->launches += 1;
+        fs.rowmask = rm; fs.scores = scores; fs.accumulate = (flags & ACACHE_F_ACCUMULATE) ? 1 : 0;
+        fs.norm_full = (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0;
+        score_in_attention = true;
     }
+    // Scoring with the separate kernels (the masked rows' query projection, then Eq. 4-5 over the cached keys).  With the
+    // softmax of Eq. 4 over every key of the context, a probe call (no anchors, no selection here, rows written into the
+    // cache) scores after its rows' fresh K are in the cache, as the probe's own attention sees them (Section 3.2);
+    // every other call scores the cache as given, before anything is recomputed.
+    auto score_now = [&]() -> acache_status {
+        if (do_score && !score_in_attention && req->batch > 0 && req->affix_len > 0) {
+            void* qmask = wsp<void>(ctx, ctx->o_qmask);
+            mark(ctx, ACACHE_STAGE_MASK_Q, stream);
+            if (req->n_masked > 0) {
+                int32_t* mpos = wsp<int32_t>(ctx, ctx->o_mrow_pos);
+                void* xnm = wsp<void>(ctx, ctx->o_xn_mask);
+                GemmArgs g{};
+                g.a = xnm; g.M = req->batch * req->n_masked; g.K = d.hidden;
+                g.prep.enabled = 1; g.prep.x = x; g.prep.x_is_compact = x_is_compact;
+                if (x_is_compact) {
+                    // the masked rows are among the extra rows of the compact input: find where
+                    int32_t* cidx = wsp<int32_t>(ctx, ctx->o_mcidx);
+                    launch_match_rows(req->masked_pos, req->n_masked, req->extra_rows, req->n_extra, k, req->batch, cidx,
+                                      wsp<uint32_t>(ctx, ctx->o_status), stream);
+                    ctx->launches += 1;
+                    g.prep.compact_idx = cidx;
+                    g.prep.compact_rows = k + req->n_extra;
+                }
+                g.prep.x_batch_stride = (int64_t)req->ctx_len * d.hidden;
+                g.prep.anchor_idx = nullptr; g.prep.k = 0; g.prep.extra_rows = req->masked_pos; g.prep.e = req->n_masked;
+                g.prep.affix_start = req->affix_start; g.prep.affix_len = req->affix_len; g.prep.ctx_len = req->ctx_len;
+                g.prep.gain = w->attn_norm_g; g.prep.eps = d.rms_eps; g.prep.row_pos = mpos;
+                g.prep.row_src = wsp<int64_t>(ctx, ctx->o_mrow_src);
+                if (!x_is_compact && req->token_ids) { g.prep.token_ids = req->token_ids; g.prep.table_rows = req->n_embed; }
+                g.b[0] = w->wq; g.n[0] = d.n_heads * d.head_dim;
+                // W_q is read again by the Q/K/V projection a few kernels later: leave it in L2 (measured: that
+                // projection 43.7 -> 40.8 us at 103 rows)
+                static const int keep_wq = [] { const char* e = getenv("ACACHE_KEEP_WQ"); return e ? atoi(e) : 1; }();
+                g.keep_weights = keep_wq && do_recompute;      // a scoring-only pass (the probe) never reads W_q again
+                g.epilogue = kEpiQKV;
+                g.bias[0] = d.qkv_bias ? w->bq : nullptr;
+                g.row_pos = mpos; g.rope_cos = req->rope_cos; g.rope_sin = req->rope_sin;
+                g.head_dim = d.head_dim; g.rope_segments = 1; g.out[0] = qmask; g.rows_per_req = req->n_masked;
+                g.partial = wsp<float>(ctx, ctx->o_gemm); g.status = wsp<uint32_t>(ctx, ctx->o_status);
+                g.grid_bar = wsp<unsigned int>(ctx, ctx->o_gridbar);
+                g.prefetch_blocks = prefetch_by(0);
+                { int nl = launch_gemm(g, stream); if (nl < 0) return check_cuda(ctx, "masked-row query projection") == ACACHE_OK ? fail(ctx, ACACHE_ERR_CUDA, "masked-row query projection launch failed") : ACACHE_ERR_CUDA;
+                ctx->launches += nl; }
+            }
+            mark(ctx, ACACHE_STAGE_SCORE, stream);
+            // with a selection to follow, the ordered sum over heads is folded into the selection kernel
+            // (only while one CTA per request can read all heads' partial sums quickly: at L = 8192 the separate,
+            // grid-wide head sum takes 4 us where the folded one took 28)
+            fused_head_sum = do_select && k > 0 && req->n_masked > 0 && (int64_t)req->affix_len * d.n_heads <= 65536;
+            // the masked rows' projection was launched just above: nothing that writes the cache is the scoring kernels'
+            // direct predecessor, so they may request their first key tiles early
+            s = run_score(ctx, req, qmask, kv, scores, (flags & ACACHE_F_ACCUMULATE) ? 1 : 0,
+                          (flags & ACACHE_F_SCORE_NORM_FULL) ? 1 : 0, fused_head_sum ? 1 : 0, stream, req->n_masked > 0 ? 1 : 0);
+            if (s != ACACHE_OK) return s;
+        }
+        return ACACHE_OK;
+    };
+    const bool score_late = do_score && !score_in_attention && !do_select && do_recompute && k == 0 && !to_slots &&
+                            (flags & ACACHE_F_SCORE_NORM_FULL) && req->n_extra > 0;
+    if (!score_late && (s = score_now()) != ACACHE_OK) return s;
     if (do_select && k > 0 && req->batch > 0) {
         mark(ctx, ACACHE_STAGE_TOPK, stream);
         launch_topk(scores, req->batch, req->affix_len, k, anchor_idx,
@@ -618,7 +680,8 @@ acache_status layer_step_impl(acache_ctx* ctx, const acache_layer_weights* w, co
     }
     if (do_recompute)
         return run_recompute(ctx, w, req, kv, !to_slots, x, x_is_compact, anchor_idx, k, k_new, v_new, y, stream, nullptr,
-                             MapReuse{false}, (flags & ACACHE_F_DROP_NON_ANCHOR) != 0);
+                             MapReuse{false}, (flags & ACACHE_F_DROP_NON_ANCHOR) != 0, score_in_attention ? &fs : nullptr,
+                             score_late ? std::function<acache_status()>(score_now) : std::function<acache_status()>());
     mark(ctx, ACACHE_N_STAGES, stream);
     return check_cuda(ctx, "layer_step");
 }

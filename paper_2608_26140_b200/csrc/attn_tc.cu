@@ -123,6 +123,16 @@ struct AttnTcArgs {
     int group, batch;
     const uint32_t* pos_excl;
     const uint32_t* row_keep;
+    // Eq. 4-5 taken from this attention's own logits (two-query-tile kernel; the one-shot probe of Section 3.2): for the
+    // query rows flagged in score_rowmask [B, rm_words] (bit i = compact row i is a masked position) the kernel keeps,
+    // next to the softmax denominator, the same sum restricted to the affix keys, and after the last key tile walks the
+    // affix key tiles once more with the product turned round (D = K Q^T: thread = key, columns = query rows), adding
+    // exp2(s - reference) / denominator over the flagged rows.  score_partial [B, H, q_tiles, L]: per (head, 128-row
+    // query tile) column sums, written only by tiles that hold flagged rows.
+    const uint32_t* score_rowmask;
+    float* score_partial;
+    int rm_words, q_tiles, affix_start, affix_len;
+    int score_norm_full;      // weight = 1 / the full denominator (Eq. 4 over every key) instead of the affix keys' share
 };
 
 __global__ void __launch_bounds__(AT_THREADS, 1)
@@ -434,7 +444,7 @@ attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ
 // and the denominator are rescaled), so the common path is: x = s * scale - reference (two per FFMA2),
 // maximum, exp2 (a quarter of them on the FMA pipe), bf16 pack, store to tensor memory.
 constexpr int AT2_THREADS = 320;                 // warp 0: TMA, warp 1: MMA issuer, warps 2-5 / 6-9: softmax of query tile 0 / 1
-constexpr int AT2_SMEM = 6 * AT_TILE + AT_SLACK + 256;   // Q x2, K x2, V x2
+constexpr int AT2_SMEM = 6 * AT_TILE + AT_SLACK + 256 + 2048;   // Q x2, K x2, V x2, barriers, score tables
 
 __device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, float (&v)[32]) {
     asm volatile(
@@ -496,12 +506,14 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
     const int n_tiles = n_cache_tiles + a.n_fresh_tiles;
     const int kb = a.cache_shared ? 0 : b;
     const int n_sets = (qt * 256 + 128 < a.n) ? 2 : 1;      // the last CTA of an odd tile count has one tile
+    float2* s_tab = reinterpret_cast<float2*>(base_ptr + 6 * AT_TILE + 256);     // [2 query tiles][128 rows] (reference, weight)
 
     if (threadIdx.x == 0) {
         for (int i = 0; i <= 10; ++i) mbar_init(bar(i), 1);
         for (int i = 11; i <= 14; ++i)                         // p_full: the softmax warps of the query tile that have rows
             mbar_init(bar(i), max(1, min(4, (a.n - qt * 256 - (i >= 13 ? 128 : 0) + 31) / 32)));
         for (int i = 15; i <= 18; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(19), 4); mbar_init(bar(20), 4);          // score sweep: the four warps of a query tile are done with D
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -517,6 +529,14 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
     // columns: S of query tile 0 | S of query tile 1 | O of query tile 0 | O of query tile 1, 128 each
     pdl_wait();
     pdl_launch_dependents();
+    // score sweep (Eq. 4-5 from this attention's logits): only CTAs whose 256 query rows hold a flagged row walk the
+    // affix key tiles [sw0, sw0 + n_sw) a second time
+    int n_sw = 0, sw0 = 0;
+    if (a.score_rowmask && a.affix_len > 0) {
+        uint32_t any = 0u;
+        for (int w = qt * 8; w < min(qt * 8 + 8, a.rm_words); ++w) any |= __ldg(a.score_rowmask + (int64_t)b * a.rm_words + w);
+        if (any) { sw0 = a.affix_start >> 7; n_sw = ((a.affix_start + a.affix_len - 1) >> 7) - sw0 + 1; }
+    }
 
     if (warp == 0 && lane == 0) {
         // ---------------- TMA producer ----------------
@@ -555,6 +575,13 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
             mbar_expect_tx(bar(5 + s), AT_TILE);
             tma_load_3d(sV0 + s * AT_TILE, mv, kvh * 128, r0, bz, bar(5 + s), pol_kv);
             tma_load_3d(sV0 + s * AT_TILE + AT_PANEL, mv, kvh * 128 + 64, r0, bz, bar(5 + s), pol_kv);
+        }
+        for (int js = 0; js < n_sw && ok; ++js) {            // the affix key tiles once more (keys only)
+            const int jj = n_tiles + js, s = jj & 1;
+            if (!(ok = mbar_wait(bar(3 + s), ((jj >> 1) & 1) ^ 1, abort_flag))) break;
+            mbar_expect_tx(bar(1 + s), AT_TILE);
+            tma_load_3d(sK0 + s * AT_TILE, &mapK, kvh * 128, (sw0 + js) * 128, kb, bar(1 + s), pol_kv);
+            tma_load_3d(sK0 + s * AT_TILE + AT_PANEL, &mapK, kvh * 128 + 64, (sw0 + js) * 128, kb, bar(1 + s), pol_kv);
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------- MMA issuer ----------------
@@ -599,16 +626,39 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
             tc_commit(bar(7 + s));                           // v_empty
             if (more) tc_commit(bar(3 + (s ^ 1)));           // k_empty of tile j + 1
         }
-    } else if (warp >= 2 && warp < 2 + 4 * n_sets && (warp & 3) * 32 < a.n - qt * 256 - ((warp - 2) >> 2) * 128) {
+        // score sweep: D_t = K Q_t^T into the S buffer of query tile t (its last P V was issued above by this thread, and
+        // the tensor pipe keeps one thread's instructions in order)
+        for (int js = 0; js < n_sw && ok; ++js) {
+            const int jj = n_tiles + js, s = jj & 1;
+            if (!(ok = mbar_wait(bar(1 + s), (jj >> 1) & 1, abort_flag))) break;
+            const uint32_t k = sK0 + s * AT_TILE;
+            for (int t = 0; t < n_sets && ok; ++t) {
+                if (js > 0 && !(ok = mbar_wait(bar(19 + t), (js - 1) & 1, abort_flag))) break;
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t da = smem_desc_sw128(k + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
+                    const uint64_t db = smem_desc_sw128(sQ + t * AT_TILE + (ks >> 2) * AT_PANEL) + (uint64_t)((ks & 3) * 2);
+                    tc_mma(tmem_base + t * 128, da, db, idesc_s, ks > 0 ? 1u : 0u);
+                }
+                tc_commit(bar(9 + t));
+            }
+            if (ok) tc_commit(bar(3 + s));                   // k_empty
+        }
+    } else if (warp >= 2 && warp < 2 + 4 * n_sets) {
+      const int t = (warp - 2) >> 2;
+      const int q = warp & 3;                              // the warp's TMEM lane quarter
+      const int row = q * 32 + lane;
+      const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+      const uint32_t tS = tmem_base + t * 128 + lane_off, tO = tmem_base + 256 + t * 128 + lane_off;
+      const bool has_rows = q * 32 < a.n - qt * 256 - t * 128;
+      // Eq. 4 normalises over the affix keys: the denominator restricted to them is kept next to the full one
+      const bool want_lf = n_sw > 0 && !a.score_norm_full;
+      float m_use = -INFINITY, l = 0.f, lf = 0.f;
+      bool ok = true;
+      if (has_rows) {
         // ---------------- softmax: one thread per query row ----------------
-        const int t = (warp - 2) >> 2;
-        const int q = warp & 3;                              // the warp's TMEM lane quarter
-        const int row = q * 32 + lane;
-        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-        const uint32_t tS = tmem_base + t * 128 + lane_off, tO = tmem_base + 256 + t * 128 + lane_off;
         const float2 sc2 = make_float2(a.scale_log2e, a.scale_log2e);
-        float m_use = -INFINITY, l = 0.f;
-        bool ok = true;
         for (int i = 0; i < 2 * n_tiles && ok; ++i) {
             const int hb = i & 1, j = i >> 1;
             // which of the half's 64 keys count: the cache's positions up to the context end, minus those a
@@ -626,7 +676,18 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
                     keep[c] = fw < a.keep_words ? __ldg(a.row_keep + (int64_t)b * a.keep_words + fw) : 0u;
                 }
             }
-            const bool all = (keep[0] & keep[1]) == 0xffffffffu;
+            // of those keys, the ones inside the affix span (cache tiles only): all, none, or some (then the slow path)
+            uint32_t aff[2] = {0u, 0u};
+            if (want_lf && j < n_cache_tiles) {
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int k0 = j * 128 + (hb * 2 + c) * 32;
+                    const int lo = max(a.affix_start - k0, 0), hi = min(a.affix_start + a.affix_len - k0, 32);
+                    if (hi > lo) aff[c] = (hi - lo >= 32 ? 0xffffffffu : ((1u << (hi - lo)) - 1u) << lo);
+                }
+            }
+            const bool aff_all = (aff[0] & aff[1]) == 0xffffffffu, aff_none = (aff[0] | aff[1]) == 0u;
+            const bool all = (keep[0] & keep[1]) == 0xffffffffu && (aff_all || aff_none);
             // warp-uniform: the tensor-memory accesses below are collective
             if (hb == 0) {
                 if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(9 + t), j & 1, abort_flag)))) break;
@@ -681,6 +742,7 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
                     tc_wait_st();
                 }
                 l *= f;
+                lf *= f;
                 if (raise) {
                     m_use = m_ref + mx;
 #pragma unroll
@@ -691,7 +753,7 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
             }
             // P as packed bf16: the half's 64 keys go to columns 32 hb .. 32 hb + 31 of the S buffer, over S values of
             // keys below 64 that this thread read in the first half
-            float2 l2a = make_float2(0.f, 0.f), l2b = make_float2(0.f, 0.f);
+            float2 l2a = make_float2(0.f, 0.f), l2b = make_float2(0.f, 0.f), lf2 = make_float2(0.f, 0.f);
             uint32_t pk[32];
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -711,13 +773,16 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
                         const float p0 = ((keep[c] >> e) & 1u) ? fast_exp2(sv[c][e]) : 0.f;
                         const float p1 = ((keep[c] >> (e + 1)) & 1u) ? fast_exp2(sv[c][e + 1]) : 0.f;
                         l2a = __fadd2_rn(l2a, make_float2(p0, p1));
+                        lf2 = __fadd2_rn(lf2, make_float2(((aff[c] >> e) & 1u) ? p0 : 0.f, ((aff[c] >> (e + 1)) & 1u) ? p1 : 0.f));
                         pk[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
                     }
                 }
             }
             tc_st32u(tS + hb * 32, pk);
             tc_wait_st();
-            l += (l2a.x + l2a.y) + (l2b.x + l2b.y);
+            const float half_sum = (l2a.x + l2a.y) + (l2b.x + l2b.y);
+            l += half_sum;
+            lf += all ? (aff_all ? half_sum : 0.f) : (lf2.x + lf2.y);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(11 + 2 * t + hb));   // p_full
@@ -744,6 +809,47 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
                 }
             }
         }
+      }
+      if (n_sw > 0) {
+        // ---------------- score sweep: thread = key, columns = the query rows of tile t ----------------
+        // every row's (reference, weight): weight = 1 / (its denominator over the affix keys) for a flagged row, else 0
+        {
+            const int grow = qt * 256 + t * 128 + row;
+            float w = 0.f;
+            const float den = a.score_norm_full ? l : lf;
+            if (has_rows && ok && grow < a.n && den > 0.f &&
+                ((__ldg(a.score_rowmask + (int64_t)b * a.rm_words + (grow >> 5)) >> (grow & 31)) & 1u))
+                w = 1.f / den;
+            s_tab[t * 128 + row] = make_float2(has_rows && m_use > -INFINITY ? m_use : 0.f, w);
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");     // the four warps of query tile t
+        uint32_t nz = 0u;                                              // 32-row column chunks that hold a flagged row
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (__any_sync(0xffffffffu, s_tab[t * 128 + c * 32 + lane].y != 0.f)) nz |= 1u << c;
+        for (int js = 0; js < n_sw; ++js) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(9 + t), (n_tiles + js) & 1, abort_flag))) break;
+            tc_fence_after();
+            float sum = 0.f;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                if (!((nz >> c) & 1u)) continue;
+                float v[32];
+                tc_ld32(tS + c * 32, v);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float2 mw = s_tab[t * 128 + c * 32 + e];
+                    sum += fast_exp2(fmaf(v[e], a.scale_log2e, -mw.x)) * mw.y;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(19 + t));
+            const int key = (sw0 + js) * 128 + row, jrel = key - a.affix_start;
+            if (jrel >= 0 && jrel < a.affix_len)
+                a.score_partial[(((int64_t)b * a.n_heads + h) * a.q_tiles + qt * 2 + t) * a.affix_len + jrel] = sum;
+        }
+      }
     }
     // ---------------- teardown ----------------
     tc_fence_before();
@@ -878,10 +984,16 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     // 1000+ rows, 8-15 % faster; 8192 keys, 5-10 % slower; fewer CTAs than SMs, up to 1.8x slower).
     // ACACHE_ATTN_TC2Q = 0: never, 2: whenever there are two tiles.
     static const int mode_2q = [] { const char* e = getenv("ACACHE_ATTN_TC2Q"); return e ? atoi(e) : 1; }();
-    const bool use_2q = mode_2q == 2 || (mode_2q == 1 && a.ctx_len + (two_src ? n_fresh : 0) <= 4096 &&
-                                         (int64_t)((q_tiles + 1) / 2) * a.n_heads * a.batch >= 148);
+    const bool fused_score = a.score_rowmask && a.score_partial && group == 1;
+    if (fused_score) {
+        t.score_rowmask = a.score_rowmask; t.score_partial = a.score_partial; t.rm_words = a.rm_words; t.q_tiles = q_tiles;
+        t.affix_start = a.affix_start; t.affix_len = a.affix_len; t.score_norm_full = a.score_norm_full;
+    }
+    // the scores are taken from the logits in the two-query-tile kernel only
+    const bool use_2q = fused_score || mode_2q == 2 || (mode_2q == 1 && a.ctx_len + (two_src ? n_fresh : 0) <= 4096 &&
+                                                        (int64_t)((q_tiles + 1) / 2) * a.n_heads * a.batch >= 148);
     cudaError_t err;
-    if (use_2q && q_tiles >= 2)
+    if (use_2q && (q_tiles >= 2 || fused_score))
         err = launch_pdl(attention_tc2q_kernel, dim3((q_tiles + 1) / 2, a.n_heads, a.batch), dim3(AT2_THREADS), AT2_SMEM, stream, t,
                          *mq, *mk, *mv, *mkn, *mvn);
     else

@@ -45,6 +45,15 @@ void launch_kv_deviation(const void* k_ref, const void* v_ref, int64_t ref_strid
 void launch_drop_mask(const int32_t* anchor_idx, int k, int affix_start, int affix_len, int ctx_len, int batch,
                       uint32_t* key_drop, uint32_t* or_into, int words, cudaStream_t stream);
 
+// rowmask[b, i / 32] bit i % 32 = compact row i (k anchors, then the e extra rows) of request b is one of its masked
+// positions; a masked position that is not among the extra rows raises kFlagBadIndex.
+void launch_row_mask(const int32_t* masked_pos, int m, const int32_t* extra_rows, int e, int k, int batch, uint32_t* rowmask,
+                     int words, uint32_t* status, cudaStream_t stream);
+
+// scores[b, j] (+)= sum over heads and over the query tiles that hold a flagged row of partial[b, h, qt, j], in a fixed order.
+void launch_score_reduce_tiles(const float* partial, const uint32_t* rowmask, int rm_words, float* scores, int batch, int n_heads,
+                               int q_tiles, int affix_len, int accumulate, cudaStream_t stream);
+
 // ---- score.cu ---------------------------------------------------------------------------
 struct ScoreArgs {
     const void* q_mask;       // bf16 [B, m, H, d]
@@ -177,6 +186,13 @@ struct AttnArgs {
     const uint32_t* row_keep; //   kernel reads the cache and k_new / v_new as two key sources instead of gathering
     int excl_words, keep_words;
     const uint32_t* key_drop; // optional [B, excl_words]: bit t = position t does not exist as a key (DropNA, Section 5.3)
+    // optional (head dimension 128): Eq. 4-5 from this attention's own logits.  score_rowmask [B, rm_words]: bit i = compact
+    // row i is a masked position; score_partial [B, H, ceil(n / 128), L]: per (head, query tile) column sums over the affix
+    // keys, written by the query tiles that hold a flagged row (launch_score_reduce_tiles adds them up)
+    const uint32_t* score_rowmask;
+    float* score_partial;
+    int rm_words, affix_start, affix_len;
+    int score_norm_full;      // the weights' denominator: this attention's own (all keys) instead of the affix keys only
     int batch, n, ctx_len, n_heads, n_kv_heads, head_dim;
     void* o;                  // bf16 [B, n, H*d]
     float* part_o;            // scratch for key splits: fp32 [B*n*H, n_split, d]

@@ -310,4 +310,64 @@ void launch_drop_mask(const int32_t* anchor_idx, int k, int affix_start, int aff
                affix_len, ctx_len, key_drop, or_into, words);
 }
 
+// ---- Eq. 4-5 from the probe's own attention logits: which compact rows are masked positions, and the final sum --------
+__global__ void __launch_bounds__(256) row_mask_kernel(const int32_t* __restrict__ masked_pos, int m,
+                                                       const int32_t* __restrict__ extra_rows, int e, int k,
+                                                       uint32_t* __restrict__ rowmask, int words, uint32_t* status) {
+    extern __shared__ uint32_t bits[];
+    pdl_wait();
+    pdl_launch_dependents();
+    const int b = blockIdx.x;
+    for (int w = threadIdx.x; w < words; w += blockDim.x) bits[w] = 0u;
+    __syncthreads();
+    for (int i = threadIdx.x; i < m; i += blockDim.x) {
+        const int want = masked_pos[(int64_t)b * m + i];
+        int found = -1;
+        for (int j = 0; j < e; ++j)
+            if (extra_rows[(int64_t)b * e + j] == want) { found = k + j; break; }
+        if (found < 0 || (found >> 5) >= words) atomicOr(status, kFlagBadIndex);
+        else atomicOr(&bits[found >> 5], 1u << (found & 31));
+    }
+    __syncthreads();
+    for (int w = threadIdx.x; w < words; w += blockDim.x) rowmask[(int64_t)b * words + w] = bits[w];
+}
+
+void launch_row_mask(const int32_t* masked_pos, int m, const int32_t* extra_rows, int e, int k, int batch, uint32_t* rowmask,
+                     int words, uint32_t* status, cudaStream_t stream) {
+    if (batch == 0) return;
+    launch_pdl(row_mask_kernel, dim3(batch), dim3(256), (size_t)words * sizeof(uint32_t), stream, masked_pos, m, extra_rows, e, k,
+               rowmask, words, status);
+}
+
+__global__ void __launch_bounds__(256) score_reduce_tiles_kernel(const float* __restrict__ partial,
+                                                                 const uint32_t* __restrict__ rowmask, int rm_words,
+                                                                 float* __restrict__ scores, int n_heads, int q_tiles, int L,
+                                                                 int accumulate) {
+    __shared__ unsigned char live[256];          // query tiles that hold a flagged row (they wrote their partial sums)
+    pdl_wait();
+    pdl_launch_dependents();
+    const int b = blockIdx.y;
+    for (int qt = threadIdx.x; qt < q_tiles; qt += blockDim.x) {
+        uint32_t any = 0u;
+        for (int w = qt * 4; w < min(qt * 4 + 4, rm_words); ++w) any |= rowmask[(int64_t)b * rm_words + w];
+        live[qt] = any != 0u;
+    }
+    __syncthreads();
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= L) return;
+    float s = 0.f;
+    for (int h = 0; h < n_heads; ++h)
+        for (int qt = 0; qt < q_tiles; ++qt)
+            if (live[qt]) s += __ldcg(partial + (((int64_t)b * n_heads + h) * q_tiles + qt) * L + j);
+    float* out = scores + (int64_t)b * L + j;
+    *out = accumulate ? *out + s : s;
+}
+
+void launch_score_reduce_tiles(const float* partial, const uint32_t* rowmask, int rm_words, float* scores, int batch, int n_heads,
+                               int q_tiles, int affix_len, int accumulate, cudaStream_t stream) {
+    if (batch == 0 || affix_len == 0) return;
+    launch_pdl(score_reduce_tiles_kernel, dim3((affix_len + 255) / 256, batch), dim3(256), 0, stream, partial, rowmask, rm_words,
+               scores, n_heads, q_tiles, affix_len, accumulate);
+}
+
 }  // namespace acache

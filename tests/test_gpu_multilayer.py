@@ -27,10 +27,19 @@ def build(shape, n_layers, B, pre, L, post, gen, m):
     return lay, layers, x, caches, cos, sin
 
 
-@pytest.mark.parametrize("shape,n_layers,norm_full", [(wl.TINY, 2, False), (wl.TINY_GQA, 3, True)])
-def test_probe_select_refresh(shape, n_layers, norm_full):
+MID128 = wl.LayerShape(512, 4, 2, 128, 1024, 1e-5, True, 5e5, "mid-d128")
+
+
+@pytest.mark.parametrize("shape,n_layers,norm_full,geom", [
+    (wl.TINY, 2, False, (6, 96, 20, 32, 32)), (wl.TINY_GQA, 3, True, (6, 96, 20, 32, 32)),
+    # head dim 128: the probe's scores come out of its own attention (Eq. 4 over the affix keys); one query tile, then
+    # three with the masked rows straddling two of them and an affix that starts and ends inside key tiles
+    (MID128, 2, False, (6, 96, 20, 32, 32)), (MID128, 3, False, (20, 300, 100, 100, 100)),
+    (MID128, 2, True, (20, 300, 100, 100, 100)),          # normaliser over all keys: the separate scoring kernels
+])
+def test_probe_select_refresh(shape, n_layers, norm_full, geom):
     B, ratio = 2, 0.25
-    lay, layers, x, caches, cos, sin = build(shape, n_layers, B, 6, 96, 20, 32, 32)
+    lay, layers, x, caches, cos, sin = build(shape, n_layers, B, *geom)
     T, l, L, P = lay.ctx_len, lay.affix_start, lay.affix_len, lay.n_extra
     K = orc.k_from_ratio(L, ratio)
     dev_layers = [{k: (ab.to_device_bf16(v, DEV) if v is not None else None) for k, v in w.items()} for w in layers]
@@ -91,7 +100,7 @@ def test_probe_select_refresh(shape, n_layers, norm_full):
         for n in range(n_layers):
             x_rows = orc.bf16_bits_to_f64(x[b])[rows_p] if n == 0 else orc.bf16_bits_to_f64(ab.to_host_bits(y[n - 1][b]))
             r = orc.recompute_rows(layers[n], shape, x_rows, rows_p, caches[b][n][0], caches[b][n][1], T, cos, sin)
-            Kall = orc.bf16_bits_to_f64(caches[b][n][0][:T])
+            Kall = orc.bf16_bits_to_f64((r["cache_k"] if norm_full else caches[b][n][0])[:T])   # as orc.probe_forward
             s_tf += orc.score_anchors(r["q"][mask_idx], Kall[l:l + L], Kall, l, norm_full)
         err_tf = np.abs(s_gpu[b] - s_tf) / np.maximum(s_tf, s_tf.mean())
         assert err_tf.max() < 1e-3, err_tf.max()

@@ -528,6 +528,31 @@ def test_multilayer_probe_scores_and_ratio_zero_refresh():
     assert not np.allclose(s - s1, s1)
 
 
+def test_probe_scores_over_all_keys_are_the_affix_part_of_the_probes_own_attention():
+    """Eq. 4 with the softmax over every key (the reading of Section 3.2's prose): the probe attends the affix as past
+    KV plus its own fresh rows, so the scores are the masked-to-affix columns of exactly that attention."""
+    lay, layers, x, caches, cos, sin = two_layer_case()
+    T, l, L = lay.ctx_len, lay.affix_start, lay.affix_len
+    P, M = lay.extra_rows[0], lay.masked_pos[0]
+    s, pc, _ = orc.probe_forward(layers[:1], SMALL, x, caches[:1], T, l, L, M, P, cos, sin, norm_full=True)
+    r = orc.recompute_rows(layers[0], SMALL, orc.bf16_bits_to_f64(x)[P], np.asarray(P), caches[0][0], caches[0][1], T, cos, sin)
+    where = {int(p): i for i, p in enumerate(P)}
+    q = torch.from_numpy(r["q"][[where[int(p)] for p in M]])                       # [m, H, d]
+    Kw = torch.from_numpy(orc.bf16_bits_to_f64(r["cache_k"][:T]))                  # the working cache: fresh rows P
+    g = SMALL.n_heads // SMALL.n_kv_heads
+    z = torch.einsum("mhd,thd->hmt", q, Kw.repeat_interleave(g, 1)) / math.sqrt(SMALL.head_dim)
+    p = torch.softmax(z, dim=-1)
+    assert np.allclose(s, p[:, :, l:l + L].sum((0, 1)).numpy(), rtol=1e-12)
+    assert abs(s.sum() + p[:, :, :l].sum().item() + p[:, :, l + L:].sum().item() - SMALL.n_heads * len(M)) < 1e-9
+    # what the cache held at the probe's own positions does not matter (its rows are written before they are attended) ...
+    ck2 = caches[0][0].copy(); ck2[P] = 0x4300
+    s2, _, _ = orc.probe_forward(layers[:1], SMALL, x, [(ck2, caches[0][1])], T, l, L, M, P, cos, sin, norm_full=True)
+    assert np.array_equal(s2, s)
+    # ... and the affix-only normaliser of the equation is a different quantity
+    s_eq, _, _ = orc.probe_forward(layers[:1], SMALL, x, caches[:1], T, l, L, M, P, cos, sin)
+    assert not np.allclose(s_eq, s, rtol=1e-3) and np.all(s_eq > s)
+
+
 def test_predict_commit_vs_library_softmax_and_rule():
     g = np.random.default_rng(21)
     n, D, V = 9, 32, 50
