@@ -35,7 +35,8 @@ RATIO = 0.2
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an ncu capture of the kernel as it
 # stands at the commit named here; None until such a capture exists (a figure from an older kernel is not printed).
-NCU_TRAFFIC = {"kernel": None, "bytes": None, "commit": None}
+NCU_TRAFFIC = {"kernel": "gemm_tc_kernel, gate/up projection 103 x 24576 x 4096 (one launch; 204.7 MB algorithmic)",
+               "bytes": 207042048, "commit": "c3e8c66"}
 
 
 def load_peaks():
@@ -275,7 +276,7 @@ def run_ours(args):
     # a first block sizes the run: at least 50 blocks of `steps` steps, and enough of them to keep the GPU busy for
     # about a second, so that the clock sampler sees the load
     est = time_blocks(step, args.steps, 1, sync_all, dist, dev)[0]
-    n_blocks = int(min(2000, max(50, np.ceil(1000.0 / max(est * args.steps, 1e-3)))))
+    n_blocks = args.blocks if args.blocks > 0 else int(min(2000, max(50, np.ceil(1000.0 / max(est * args.steps, 1e-3)))))
     sampler = ClockSampler(local)
     sampler.start()
     l0 = ctx.launch_count()
@@ -305,7 +306,7 @@ def run_ours(args):
 
     for i in range(3):
         step_host(i)
-    blocks_e2e = time_blocks(step_host, args.steps, max(50, n_blocks // 4), sync_all, dist, dev)
+    blocks_e2e = time_blocks(step_host, args.steps, args.blocks if args.blocks > 0 else max(50, n_blocks // 4), sync_all, dist, dev)
     ms_e2e = float(np.median(blocks_e2e))
     sampler.stop_flag = True
     sampler.join()
@@ -337,7 +338,8 @@ def run_ours(args):
                 "peak": peaks["hbm_gbs"] if hbm_bound else peaks["tflops"], "unit": "GB/s" if hbm_bound else "TFLOP/s",
                 "frac": floor_s / s_step, "peak_source": peaks["source"], "floor_us": floor_s * 1e6,
                 "algorithmic_bytes": step_bytes, "algorithmic_flops": step_flops,
-                "traffic": NCU_TRAFFIC["bytes"], "traffic_of": NCU_TRAFFIC["kernel"], "traffic_commit": NCU_TRAFFIC["commit"],
+                "traffic": NCU_TRAFFIC["bytes"] if (args.config == 2 and lay.n_extra == 0 and B == 1) else None,
+                "traffic_of": NCU_TRAFFIC["kernel"], "traffic_commit": NCU_TRAFFIC["commit"],
                 "dominant_kernel": {"kernel": "gate/up projection + SwiGLU (stage gate_up, from the staged pass)",
                                     "bound": "hbm" if gu_hbm_bound else "tensor", "achieved": gu_ach, "peak": gu_peak,
                                     "unit": gu_unit, "frac": gu_ach / gu_peak, "algorithmic_bytes": gu_bytes,
@@ -371,6 +373,80 @@ def run_ours(args):
     print(json.dumps(out))
     if dist:
         dist.destroy_process_group()
+
+
+def probe_layer(cfg, batch, steps, peaks, dev):
+    """One layer of the one-shot probe (Section 3.2) at benchmark configuration 3 or 4: every request's non-affix rows
+    (256 of them masked) through the layer with the affix K/V as cached, the masked-to-affix scores (Eq. 4-5) taken
+    from the layer's own attention.  Device-drawn inputs (timing only)."""
+    import torch
+    from paper_2608_26140_b200 import binding as ab
+    from paper_2608_26140_b200 import build as abuild
+    abuild.build()
+    torch.cuda.set_device(int(dev.split(":")[1]))
+    shape = wl.DREAM_7B if cfg == 4 else wl.LLADA_8B
+    lay = wl.config_layout(cfg, "all", n_masked=256, batch=batch)
+    B, T, L, P = lay.batch, lay.ctx_len, lay.affix_len, lay.n_extra
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.SEED_BASE + 4096 * cfg + 99)
+
+    def randn(shape_, std=1.0):
+        t = torch.randn(shape_, generator=gen, device=dev, dtype=torch.bfloat16)
+        return t.mul_(std) if std != 1.0 else t
+
+    D, F = shape.hidden, shape.ffn
+    w = dict(wq=randn((shape.q_dim, D), 0.02), wk=randn((shape.kv_dim, D), 0.02), wv=randn((shape.kv_dim, D), 0.02),
+             wo=randn((D, shape.q_dim), 0.02), w_gate=randn((F, D), 0.02), w_up=randn((F, D), 0.02), w_down=randn((D, F), 0.02),
+             attn_norm_g=randn((D,), 0.05).add_(1.0), mlp_norm_g=randn((D,), 0.05).add_(1.0))
+    for k_, n_ in (("bq", shape.q_dim), ("bk", shape.kv_dim), ("bv", shape.kv_dim)):
+        w[k_] = randn((n_,), 0.02) if shape.qkv_bias else None
+    kv_std = 0.02 * float(np.sqrt(D))
+    x = randn((B, T, D))
+    ck, cv = randn((B, T, shape.n_kv_heads, shape.head_dim), kv_std), randn((B, T, shape.n_kv_heads, shape.head_dim), kv_std)
+    cos_h, sin_h = wl.rope_table(T, shape.head_dim, shape.rope_theta)
+    cos, sin = torch.from_numpy(cos_h).to(dev), torch.from_numpy(sin_h).to(dev)
+    masked = torch.from_numpy(lay.masked_pos.copy()).to(dev)
+    extra = torch.from_numpy(lay.extra_rows.copy()).to(dev)
+    req = ab.Context.request(B, T, lay.affix_start, L, masked, extra, cos, sin)
+    ctx = ab.Context.for_shape(shape, B, T, L, P, lay.n_masked, dev)
+    scores = torch.zeros((B, L), dtype=torch.float32, device=dev)
+    y = torch.zeros((B, P, D), dtype=torch.bfloat16, device=dev)
+    lw = ab.Context.weights(w)
+
+    def step():
+        ctx.layer_step(lw, req, ab.Context.kv(ck, cv), x, 0, 0.0, ab.F_SCORE, scores, None, y)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    l0 = ctx.launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record()
+    for i in range(steps):
+        step()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    launches = (ctx.launch_count() - l0) / steps
+    ctx.stage_timing(True)
+    step()
+    stage = {k_: round(v * 1e3, 1) for k_, v in ctx.read_stage_times().items() if v}
+    ctx.stage_timing(False)
+    assert ctx.poll_status() == 0
+    mass = float(scores.sum().item()) / (B * shape.n_heads * lay.n_masked)          # Eq. 4: every masked row's weights sum to 1
+    params = D * shape.q_dim + 2 * D * shape.kv_dim + shape.q_dim * D + 3 * D * F
+    flops = 2 * B * P * params + 4 * B * P * T * shape.q_dim
+    med = float(np.median(ms))
+    return {"metric": "probe_layer_ms", "value": med, "unit": "ms per probe layer", "n_gpus": 1, "steps": steps, "warmup": 3,
+            "ms_per_step": med, "ms_min": float(min(ms)), "ms_max": float(max(ms)), "higher_is_better": False, "dtype": "bf16",
+            "data": "synthetic, drawn on the device",
+            "config": {"workload": f"cfg{cfg} probe layer: {shape.name}, batch {B}, affix {L} at {lay.affix_start}, {P} rows per request "
+                                   f"({lay.n_masked} masked), no anchors, scores from the layer's own attention",
+                       "benchmark_config": cfg},
+            "gpu_launches": int(round(launches * steps)), "gpu_launches_per_step": launches, "stage_us": stage,
+            "score_mass_per_masked_row_and_head": mass,
+            "roofline": {"bound": "tensor", "achieved": flops / (med * 1e-3) / 1e12, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                         "frac": flops / (med * 1e-3) / 1e12 / peaks["tflops"], "peak_source": peaks["source"]}}
 
 
 def extra_records(args, peaks, dev):
@@ -541,6 +617,11 @@ def extra_records(args, peaks, dev):
                                                    "frac_of_hbm_peak": by / md / 1e9 / peaks["hbm_gbs"]}
         del ctx, xs, cks, cvs, y
         torch.cuda.empty_cache()
+    del winst, wl_inst
+    torch.cuda.empty_cache()
+    pr = probe_layer(4, None, 5, peaks, dev)
+    out["probe_layer_cfg4"] = {k_: pr[k_] for k_ in ("config", "ms_per_step", "ms_min", "ms_max", "gpu_launches_per_step", "stage_us",
+                                                     "score_mass_per_masked_row_and_head", "roofline")}
     return out
 
 
@@ -1092,6 +1173,12 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--instances", type=int, default=4, help="weight/cache instances rotated between steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="timed blocks of --steps steps (0: at least 50 and about a second of GPU time; a small number keeps a "
+                         "profiler run short)")
+    ap.add_argument("--probe", action="store_true",
+                    help="--config 3 or 4: time one layer of the selection-time probe (all request rows, no anchors, scores "
+                         "accumulated from the layer's own attention)")
     ap.add_argument("--no-extra", action="store_true",
                     help="default run only: skip the short configuration-3 / sweep / selector measurements (key `extra`)")
     ap.add_argument("--layers", type=int, default=32, help="layers of the --config 3 denoising step")
@@ -1121,6 +1208,8 @@ def main():
         return
     if args.impl == "reference":
         run_reference(args)
+    elif args.probe and args.config in (3, 4):
+        print(json.dumps(probe_layer(args.config, args.batch, max(args.steps, 1), load_peaks(), "cuda:0")))
     elif args.shared and args.config in (3, 4) and not args.generate:
         run_shared(args)
     elif args.config == 3:

@@ -314,17 +314,19 @@ void launch_drop_mask(const int32_t* anchor_idx, int k, int affix_start, int aff
 __global__ void __launch_bounds__(256) row_mask_kernel(const int32_t* __restrict__ masked_pos, int m,
                                                        const int32_t* __restrict__ extra_rows, int e, int k,
                                                        uint32_t* __restrict__ rowmask, int words, uint32_t* status) {
-    extern __shared__ uint32_t bits[];
+    extern __shared__ uint32_t bits[];          // [words] the mask, then [e] the request's extra rows
+    int32_t* rows_s = reinterpret_cast<int32_t*>(bits + words);
     pdl_wait();
     pdl_launch_dependents();
     const int b = blockIdx.x;
     for (int w = threadIdx.x; w < words; w += blockDim.x) bits[w] = 0u;
+    for (int j = threadIdx.x; j < e; j += blockDim.x) rows_s[j] = extra_rows[(int64_t)b * e + j];
     __syncthreads();
     for (int i = threadIdx.x; i < m; i += blockDim.x) {
         const int want = masked_pos[(int64_t)b * m + i];
         int found = -1;
         for (int j = 0; j < e; ++j)
-            if (extra_rows[(int64_t)b * e + j] == want) { found = k + j; break; }
+            if (rows_s[j] == want) { found = k + j; break; }
         if (found < 0 || (found >> 5) >= words) atomicOr(status, kFlagBadIndex);
         else atomicOr(&bits[found >> 5], 1u << (found & 31));
     }
@@ -335,30 +337,49 @@ __global__ void __launch_bounds__(256) row_mask_kernel(const int32_t* __restrict
 void launch_row_mask(const int32_t* masked_pos, int m, const int32_t* extra_rows, int e, int k, int batch, uint32_t* rowmask,
                      int words, uint32_t* status, cudaStream_t stream) {
     if (batch == 0) return;
-    launch_pdl(row_mask_kernel, dim3(batch), dim3(256), (size_t)words * sizeof(uint32_t), stream, masked_pos, m, extra_rows, e, k,
-               rowmask, words, status);
+    const size_t smem = (size_t)(words + e) * sizeof(uint32_t);
+    if (smem > 48 * 1024) cudaFuncSetAttribute(row_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    launch_pdl(row_mask_kernel, dim3(batch), dim3(256), smem, stream, masked_pos, m, extra_rows, e, k, rowmask, words, status);
 }
 
 __global__ void __launch_bounds__(256) score_reduce_tiles_kernel(const float* __restrict__ partial,
                                                                  const uint32_t* __restrict__ rowmask, int rm_words,
                                                                  float* __restrict__ scores, int n_heads, int q_tiles, int L,
                                                                  int accumulate) {
-    __shared__ unsigned char live[256];          // query tiles that hold a flagged row (they wrote their partial sums)
+    __shared__ int live[256];                    // the query tiles that hold a flagged row (they wrote their partial sums)
+    __shared__ int n_live;
     pdl_wait();
     pdl_launch_dependents();
     const int b = blockIdx.y;
-    for (int qt = threadIdx.x; qt < q_tiles; qt += blockDim.x) {
-        uint32_t any = 0u;
-        for (int w = qt * 4; w < min(qt * 4 + 4, rm_words); ++w) any |= rowmask[(int64_t)b * rm_words + w];
-        live[qt] = any != 0u;
+    if (threadIdx.x == 0) {
+        int n = 0;
+        for (int qt = 0; qt < q_tiles && qt < 256; ++qt) {
+            uint32_t any = 0u;
+            for (int w = qt * 4; w < min(qt * 4 + 4, rm_words); ++w) any |= rowmask[(int64_t)b * rm_words + w];
+            if (any) live[n++] = qt;
+        }
+        n_live = n;
     }
     __syncthreads();
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= L) return;
+    // (head, live tile) pairs in a fixed order, eight loads in flight at a time
+    const int total = n_heads * n_live;
     float s = 0.f;
-    for (int h = 0; h < n_heads; ++h)
-        for (int qt = 0; qt < q_tiles; ++qt)
-            if (live[qt]) s += __ldcg(partial + (((int64_t)b * n_heads + h) * q_tiles + qt) * L + j);
+    for (int i0 = 0; i0 < total; i0 += 8) {
+        float t[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u;
+            t[u] = 0.f;
+            if (i < total) {
+                const int h = i / n_live, qt = live[i - h * n_live];
+                t[u] = __ldcg(partial + (((int64_t)b * n_heads + h) * q_tiles + qt) * L + j);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += t[u];
+    }
     float* out = scores + (int64_t)b * L + j;
     *out = accumulate ? *out + s : s;
 }
