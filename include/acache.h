@@ -23,6 +23,13 @@
  *  - Asynchrony: every compute entry point only enqueues work on the given stream and
  *    returns; it never synchronises.  Calls that share one context must be issued on
  *    one stream (they share the workspace).
+ *  - Weights are constants of a call: the kernels may start reading them (shared-memory
+ *    ring prefill, L2 requests) before the work enqueued earlier on the stream has
+ *    finished.  They must therefore be complete and visible before the call is enqueued;
+ *    in particular they must not be written by the kernel that immediately precedes the
+ *    call on the same stream (a weight copy or a dequantisation): put an event or any
+ *    other kernel in between, or synchronise.  Every other input (x, the cache, index
+ *    arrays, scores) follows plain stream order.
  *  - Errors: every call returns acache_status.  Argument and shape validation happens
  *    on the host before any launch, so a non-OK status means nothing was enqueued.
  *    Faults that depend on device data (an index outside its range) never trap: the

@@ -33,6 +33,10 @@ the function that takes it):
   * Anchor queries attend the *refreshed* anchor K/V (store-then-attend,
     Appendix C.1), over all T positions with no mask (bidirectional).
 
+Also here: the two ablation variants of the paper that are arithmetic (the KV-deviation
+selector of the appendix, ``kv_deviation_scores``; the DropNA key layout of Section 5.3,
+``dropna_key_keep`` / ``recompute_rows(key_keep=)``), each pinned like the rest.
+
 Pins (tests marked "not gpu"): brute-force nested-loop scoring and selection
 on tiny inputs, closed forms (zero queries -> uniform scores; score mass
 = N*H*m), library special cases (torch scaled_dot_product_attention,

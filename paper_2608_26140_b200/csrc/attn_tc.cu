@@ -977,8 +977,7 @@ int launch_attention_tc(const AttnArgs& a, uint32_t* status, cudaStream_t stream
     } else if (a.key_drop) {
         t.excl_words = a.excl_words; t.pos_excl = a.key_drop;
     }
-    static const int kv_prefetch = [] { const char* e = getenv("ACACHE_ATTN_KV_PREFETCH"); return e ? atoi(e) : 2; }();
-    t.kv_prefetch = kv_prefetch;
+    t.kv_prefetch = 2;        // K/V tiles requested into L2 this many iterations ahead of the two-stage rings
     // Two query tiles per CTA pay off when the halved grid still fills the SMs and the context is short enough
     // for the per-CTA prologue and epilogue to matter (measured, one against the other: 2048-2560 keys with
     // 1000+ rows, 8-15 % faster; 8192 keys, 5-10 % slower; fewer CTAs than SMs, up to 1.8x slower).

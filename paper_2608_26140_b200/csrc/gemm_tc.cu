@@ -1197,13 +1197,12 @@ TcPlan make_plan(int M, int K, int units, bool swiglu) {
     p.U = (int)((total + g - 1) / g);
     p.ctas = (int)((total + p.U - 1) / p.U);
     p.smax = 2;   // partial slots per CTA
-    // K blocks past the ring asked into L2 before the dependency wait.  Off by default: with the neighbouring kernels
-    // as short as they are now the requests compete with the stream that follows (configuration 2: 168.1 us per
-    // layer-step at 0, 170.1 at 12, 175.7 at 28); the ring itself is still filled before the wait.
-    static const int prefetch = [] { const char* e = getenv("ACACHE_GEMM_PREFETCH"); return e ? atoi(e) : 0; }();
-    p.prefetch = prefetch;
-    static const int prefill = [] { const char* e = getenv("ACACHE_GEMM_PREFILL"); return e ? std::min(std::max(atoi(e), 0), TC_STAGES) : TC_STAGES; }();
-    p.prefill = prefill;
+    // K blocks past the ring asked into L2 before the dependency wait: none by default (measured at configuration 2:
+    // 168.1 us per layer-step at 0, 170.1 at 12, 175.7 at 28: with neighbours this short the requests compete with the
+    // stream that follows); GemmArgs::prefetch_blocks sets it per projection.  The ring itself is filled before the
+    // wait (174.9 us per layer-step with no stage prefilled, 169.1 with two, 167.9-168.6 with three or four).
+    p.prefetch = 0;
+    p.prefill = TC_STAGES;
     return p;
 }
 
