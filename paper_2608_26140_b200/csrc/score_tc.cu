@@ -335,6 +335,263 @@ score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_consta
     }
 }
 
+// ---- one pass: the logits stay in tensor memory ------------------------------------------------------
+// With at most 64 masked rows the logits of a whole key range fit in tensor memory in the orientation D = K Q^T
+// (thread = key, one column per masked row: 32 or 64 columns per 128-key tile, up to 512 columns), so the cached keys
+// are read from HBM ONCE: a cluster of eight CTAs covers the normaliser's key range of one (head, request); every CTA
+// streams its eighth through a TMA ring, leaves D of all its tiles in tensor memory and keeps a running column
+// maximum per thread; then (i) the CTA's maximum per masked row (a transposing reduction through shared memory),
+// (ii) e = exp2(s - that maximum) written back over D, its column sums = the CTA's share of the denominator,
+// (iii) the eight CTAs' (maximum, share) meet through distributed shared memory and give each masked row one weight
+// w_r = exp2(m_cta - M) / denominator, (iv) every thread adds e_r w_r over its key's columns: the key's column sum.
+// One exponential per logit, every sum in a fixed order (bitwise reproducible), no float atomics.
+constexpr int S1_CLUSTER = 8;
+constexpr int S1_THREADS = 192;                 // warp 0 TMA, warp 1 MMA, warps 2-5 one thread per key
+constexpr int S1_MAX_TILES = 16;
+// query tile (NP rows x 128: 8 or 16 KB) | key ring, 3 or 2 stages (after the last tile: the transposition buffer [128][65]
+// fp32) | tables | barriers.  About 105 KB / 85 KB: two CTAs per SM, which is also what tensor memory allows at up to 256
+// columns per CTA; a CTA that needs all 512 columns asks for S1_SMEM_WIDE so that no second CTA can be resident beside it
+// (a CTA waiting for tensor memory inside a cluster whose peers wait for it at a cluster barrier would never get it).
+template <int NP> struct S1 {
+    static constexpr int Q_BYTES = 2 * NP * 128;
+    static constexpr int STAGES = NP == 32 ? 3 : 2;
+    static constexpr int TAB_OFF = Q_BYTES + STAGES * ST_K_BYTES;
+    static constexpr int BAR_OFF = TAB_OFF + 2048;
+    static constexpr int SMEM = BAR_OFF + 512 + 1024;
+    static_assert(128 * 65 * 4 <= STAGES * ST_K_BYTES, "the transposition buffer reuses the key ring");
+};
+constexpr int S1_SMEM_WIDE = 120 * 1024;
+
+__device__ __forceinline__ void tc_st32f(uint32_t taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]),
+          "f"(v[9]), "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "f"(v[16]), "f"(v[17]),
+          "f"(v[18]), "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]),
+          "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_sync_s1() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t local_addr, uint32_t rank) {
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(ra) : "memory");
+    return v;
+}
+
+// NP: columns per key tile (the masked rows rounded up to 32 or 64); tpc: 128-key tiles per CTA
+template <int NP>
+__global__ void __cluster_dims__(S1_CLUSTER, 1, 1) __launch_bounds__(S1_THREADS, 2)
+score_onepass_tc_kernel(const ScoreTcArgs a, const int tpc, const uint32_t tmem_cols, const __grid_constant__ CUtensorMap mapQ,
+                        const __grid_constant__ CUtensorMap mapK) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    constexpr int S1_STAGES = S1<NP>::STAGES, S1_BAR_OFF = S1<NP>::BAR_OFF;
+    const uint32_t sQ = base, sK0 = base + S1<NP>::Q_BYTES;
+    float* s_t = reinterpret_cast<float*>(base_ptr + S1<NP>::Q_BYTES);          // [128 keys][65]: per-thread column values
+    float* s_w = reinterpret_cast<float*>(base_ptr + S1<NP>::TAB_OFF);          // [64] per-row scalar handed to the key threads
+    float* s_part = s_w + 64;                                                   // [4 warps][64] partial column reductions
+    float2* s_x = reinterpret_cast<float2*>(s_part + 256);                      // [64] (maximum, denominator share) for the peers
+    const uint32_t bars = base + S1_BAR_OFF;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + S1_BAR_OFF + 448);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + S1_BAR_OFF + 456);
+    // barriers: 0 q_full | 1..3 k_full | 4..6 k_empty | 8..23 d_full of tile t  (S1_STAGES <= 3)
+    auto bar = [&](int i) { return bars + 8 * i; };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rank = blockIdx.x % S1_CLUSTER, h = blockIdx.x / S1_CLUSTER, b = blockIdx.y;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);
+    const int kb = a.cache_shared ? 0 : b;
+    const int key0 = rank * tpc * 128;                                           // first key of this CTA inside the range
+    const int n_keys = max(0, min(tpc * 128, a.norm_len - key0));
+    const int n_tiles = (n_keys + 127) / 128;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 8 + S1_MAX_TILES; ++i) mbar_init(bar(i), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();
+    pdl_launch_dependents();
+
+    if (warp == 0 && lane == 0) {
+        const uint64_t pol = policy_evict_first(), pol_q = policy_evict_last();
+        mbar_expect_tx(bar(0), 2 * NP * 128);                                    // two 64-column panels of NP rows
+        tma3(sQ, &mapQ, h * 128, 0, b, bar(0), pol_q);
+        tma3(sQ + NP * 128, &mapQ, h * 128 + 64, 0, b, bar(0), pol_q);
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int s = t % S1_STAGES;
+            if (!(ok = mbar_wait(bar(4 + s), ((t / S1_STAGES) & 1) ^ 1, abort_flag))) break;
+            mbar_expect_tx(bar(1 + s), ST_K_BYTES);
+            const uint32_t dst = sK0 + s * ST_K_BYTES;
+            const int row = a.norm_lo + key0 + t * 128;
+            tma3(dst, &mapK, kvh * 128, row, kb, bar(1 + s), pol);
+            tma3(dst + ST_PANEL128, &mapK, kvh * 128 + 64, row, kb, bar(1 + s), pol);
+        }
+    } else if (warp == 1 && lane == 0) {
+        const uint32_t idesc = idesc_bf16(NP);
+        bool ok = mbar_wait(bar(0), 0, abort_flag);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int s = t % S1_STAGES;
+            if (!(ok = mbar_wait(bar(1 + s), (t / S1_STAGES) & 1, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t k = sK0 + s * ST_K_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t da = smem_desc_sw128(k + (ks >> 2) * ST_PANEL128) + (uint64_t)((ks & 3) * 2);
+                const uint64_t db = smem_desc_sw128(sQ + (ks >> 2) * (NP * 128)) + (uint64_t)((ks & 3) * 2);
+                tc_mma(tmem_base + t * NP, da, db, idesc, ks > 0 ? 1u : 0u);
+            }
+            tc_commit(bar(8 + t));     // d_full of tile t
+            tc_commit(bar(4 + s));     // k_empty
+        }
+    }
+    // ---------------- key threads: warps 2-5, thread = key lane; everyone meets at the barriers ----------------
+    const bool keyw = warp >= 2;
+    const int q = warp & 3, kl = q * 32 + lane;                                  // this thread's TMEM lane = key inside a tile
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    bool ok = true;
+    // (i) running maximum per column over this thread's keys, as the tiles arrive
+    float cmax[NP];
+#pragma unroll
+    for (int r = 0; r < NP; ++r) cmax[r] = -INFINITY;
+    if (keyw) {
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(8 + t), 0, abort_flag)))) break;
+            tc_fence_after();
+            // the tensor-memory load is collective (.sync.aligned): every lane executes the same one, a lane whose key lies
+            // past the range only leaves the values out of its maximum
+            const bool there = t * 128 + kl < n_keys;
+#pragma unroll
+            for (int c = 0; c < NP / 32; ++c) {
+                float v[32];
+                tc_ld32(tmem_base + lane_off + t * NP + c * 32, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) cmax[c * 32 + i] = there ? fmaxf(cmax[c * 32 + i], v[i]) : cmax[c * 32 + i];
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < NP; ++r) s_t[kl * 65 + r] = cmax[r];
+    }
+    __syncthreads();
+    // transposing reduction: key thread kl takes column kl % NP over 128 * NP / 128 keys, then NP threads combine the parts
+    constexpr int GROUPS = 128 / NP, KPG = NP;                                   // key groups, keys per group
+    if (keyw) {
+        const int r = kl % NP, g = kl / NP;
+        float m = -INFINITY;
+#pragma unroll 8
+        for (int k = 0; k < KPG; ++k) m = fmaxf(m, s_t[(g * KPG + k) * 65 + r]);
+        s_part[g * 64 + r] = m;
+    }
+    __syncthreads();
+    if (threadIdx.x < NP) {
+        float m = -INFINITY;
+#pragma unroll
+        for (int g = 0; g < GROUPS; ++g) m = fmaxf(m, s_part[g * 64 + threadIdx.x]);
+        s_w[threadIdx.x] = m * a.scale_log2e;                                    // the CTA's maximum of row r, in log2 units
+    }
+    __syncthreads();
+    // (ii) e = exp2(s - maximum), written back over D; per-thread column sums
+    if (keyw) {
+        float csum[NP];
+#pragma unroll
+        for (int r = 0; r < NP; ++r) csum[r] = 0.f;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const bool there = t * 128 + kl < n_keys;
+#pragma unroll
+            for (int c = 0; c < NP / 32; ++c) {
+                float v[32];
+                tc_ld32(tmem_base + lane_off + t * NP + c * 32, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float mr = s_w[c * 32 + i];
+                    v[i] = (there && mr > -INFINITY) ? ex2(fmaf(v[i], a.scale_log2e, -mr)) : 0.f;
+                    csum[c * 32 + i] += v[i];
+                }
+                tc_st32f(tmem_base + lane_off + t * NP + c * 32, v);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < NP; ++r) s_t[kl * 65 + r] = csum[r];
+    }
+    __syncthreads();
+    if (keyw) {
+        const int r = kl % NP, g = kl / NP;
+        float d = 0.f;
+#pragma unroll 8
+        for (int k = 0; k < KPG; ++k) d += s_t[(g * KPG + k) * 65 + r];
+        s_part[g * 64 + r] = d;
+    }
+    __syncthreads();
+    if (threadIdx.x < NP) {
+        float d = 0.f;
+#pragma unroll
+        for (int g = 0; g < GROUPS; ++g) d += s_part[g * 64 + threadIdx.x];
+        s_x[threadIdx.x] = make_float2(s_w[threadIdx.x], d);
+    }
+    // (iii) the eight CTAs' statistics meet: one weight per masked row
+    cluster_sync_s1();
+    if (threadIdx.x < NP) {
+        float2 st[S1_CLUSTER];
+#pragma unroll
+        for (int c = 0; c < S1_CLUSTER; ++c) st[c] = ld_cluster_f2(smem_u32(s_x + threadIdx.x), (uint32_t)c);
+        float M = -INFINITY, Dn = 0.f;
+#pragma unroll
+        for (int c = 0; c < S1_CLUSTER; ++c) M = fmaxf(M, st[c].x);
+#pragma unroll
+        for (int c = 0; c < S1_CLUSTER; ++c)
+            if (st[c].x > -INFINITY) Dn += st[c].y * ex2(st[c].x - M);
+        const float mine = s_x[threadIdx.x].x;
+        s_part[threadIdx.x] = ((int)threadIdx.x < a.m && mine > -INFINITY && Dn > 0.f) ? ex2(mine - M) / Dn : 0.f;
+    }
+    __syncthreads();
+    // (iv) the key's column sum
+    if (keyw) {
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < NP / 32; ++c) {
+                float v[32];
+                tc_ld32(tmem_base + lane_off + t * NP + c * 32, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) sum = fmaf(v[i], s_part[c * 32 + i], sum);
+            }
+            const int j = a.norm_lo + key0 + t * 128 + kl - a.affix_start;     // position inside the affix
+            if (t * 128 + kl < n_keys && j >= 0 && j < a.affix_len)
+                a.head_partial[((int64_t)b * a.n_heads + h) * a.affix_len + j] = sum;
+        }
+    }
+    tc_fence_before();
+    cluster_sync_s1();            // no CTA leaves while a peer may still read its statistics
+    if (*abort_flag) {
+        if (threadIdx.x == 0) {
+            atomicOr(a.status, kFlagWaitExpired);
+            for (int i = 0; i < 4096; ++i) __nanosleep(64);
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
 }  // namespace
 
 int score_tc_splits(int norm_len) { return (norm_len + kKeysPerCta1 - 1) / kKeysPerCta1; }
@@ -367,6 +624,39 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
         cudaFuncSetAttribute(score_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              2 * 256 * 128 + CS_STAGES * ST_K_BYTES + CS_TABLES + 1024 + 256);
         attr = true;
+    }
+    static const bool onepass_on = [] { const char* e = getenv("ACACHE_SCORE_ONEPASS"); return !e || atoi(e) != 0; }();
+    if (onepass_on && a.m <= 64) {
+        // the whole key range of a (head, request) over a cluster of eight CTAs, logits kept in tensor memory
+        const int np = a.m <= 32 ? 32 : 64;
+        const int tpc = ((a.norm_len + S1_CLUSTER - 1) / S1_CLUSTER + 127) / 128;
+        if (tpc * np <= 512) {
+            uint32_t cols = 32;
+            while ((int)cols < tpc * np) cols <<= 1;
+            const CUtensorMap* mq1 = get_map3(a.q_mask, a.m, a.n_heads * 128, a.batch, (int64_t)a.m * a.n_heads * 128, np);
+            if (mq1) {
+                const CUtensorMap map_q1 = *mq1;
+                static bool attr1 = false;
+                if (!attr1) {
+                    cudaFuncSetAttribute(score_onepass_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, S1_SMEM_WIDE);
+                    cudaFuncSetAttribute(score_onepass_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, S1_SMEM_WIDE);
+                    attr1 = true;
+                }
+                ScoreTcArgs t1{};
+                t1.row_stats = a.row_stats; t1.head_partial = a.head_partial;
+                t1.m = a.m; t1.n_heads = a.n_heads; t1.n_kv_heads = a.n_kv_heads;
+                t1.norm_lo = a.norm_lo; t1.norm_len = a.norm_len; t1.affix_start = a.affix_start; t1.affix_len = a.affix_len;
+                t1.n_split = 1; t1.cache_shared = shared ? 1 : 0;
+                t1.scale_log2e = 1.4426950408889634f / sqrtf(128.f);
+                t1.status = status;
+                const dim3 grid(a.n_heads * S1_CLUSTER, a.batch);
+                const size_t sm1 = cols > 256 ? (size_t)S1_SMEM_WIDE : (size_t)(np == 32 ? S1<32>::SMEM : S1<64>::SMEM);
+                const cudaError_t e1 = np == 32
+                    ? launch_pdl(score_onepass_tc_kernel<32>, grid, dim3(S1_THREADS), sm1, stream, t1, tpc, cols, map_q1, *mk)
+                    : launch_pdl(score_onepass_tc_kernel<64>, grid, dim3(S1_THREADS), sm1, stream, t1, tpc, cols, map_q1, *mk);
+                return e1 == cudaSuccess ? 1 : -1;
+            }
+        }
     }
     ScoreTcArgs t{};
     t.row_stats = a.row_stats; t.head_partial = a.head_partial;

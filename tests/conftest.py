@@ -19,6 +19,12 @@ def pytest_collection_modifyitems(config, items):
     except Exception:  # pragma: no cover
         has_gpu = False
     if has_gpu:
+        # a kernel that never returns must not hold the whole run: every GPU test gets a generous limit, enforced from a
+        # watchdog thread (a blocked CUDA call never returns to the interpreter, so a signal would not be seen)
+        if config.pluginmanager.hasplugin("timeout"):
+            for it in items:
+                if "gpu" in it.keywords and it.get_closest_marker("timeout") is None:
+                    it.add_marker(pytest.mark.timeout(1500, method="thread"))
         return
     skip = pytest.mark.skip(reason="no CUDA device")
     for it in items:

@@ -34,6 +34,12 @@ def dev_i32(a):
     (MID128, 2, 3, 1000, 20, 64, False),
     (MID128, 1, 0, 1024, 8, 17, False),
     (MID128, 2, 0, 65, 8, 64, False),
+    # from 2048 keys (batch x range) on tcgen05: up to 64 masked rows in one pass with the logits kept in tensor memory
+    # (ragged key ranges, CTAs of the cluster without keys, 32 and 64 columns, both normalisers), more rows in two passes
+    (MID128, 2, 5, 3000, 33, 32, False),
+    (MID128, 1, 0, 2500, 40, 64, True),
+    (MID128, 3, 16, 700, 20, 33, False),
+    (MID128, 1, 7, 2100, 64, 130, True),
 ])
 def test_score_anchors(shape, B, pre, L, post, m, norm_full):
     lay = wl.make_layout(B, pre, L, post, max(m, 1), m)
