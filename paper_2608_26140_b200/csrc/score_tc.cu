@@ -386,10 +386,11 @@ __device__ __forceinline__ float2 ld_cluster_f2(uint32_t local_addr, uint32_t ra
 }
 
 // NP: columns per key tile (the masked rows rounded up to 32 or 64); tpc: 128-key tiles per CTA
+// csize: CTAs per cluster (1, 2, 4 or 8; the launch sets the cluster dimension to the same number)
 template <int NP>
-__global__ void __cluster_dims__(S1_CLUSTER, 1, 1) __launch_bounds__(S1_THREADS, 2)
-score_onepass_tc_kernel(const ScoreTcArgs a, const int tpc, const uint32_t tmem_cols, const __grid_constant__ CUtensorMap mapQ,
-                        const __grid_constant__ CUtensorMap mapK) {
+__global__ void __launch_bounds__(S1_THREADS, 2)
+score_onepass_tc_kernel(const ScoreTcArgs a, const int tpc, const uint32_t tmem_cols, const int csize,
+                        const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -405,7 +406,7 @@ score_onepass_tc_kernel(const ScoreTcArgs a, const int tpc, const uint32_t tmem_
     // barriers: 0 q_full | 1..3 k_full | 4..6 k_empty | 8..23 d_full of tile t  (S1_STAGES <= 3)
     auto bar = [&](int i) { return bars + 8 * i; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rank = blockIdx.x % S1_CLUSTER, h = blockIdx.x / S1_CLUSTER, b = blockIdx.y;
+    const int rank = blockIdx.x % csize, h = blockIdx.x / csize, b = blockIdx.y;
     const int kvh = h / (a.n_heads / a.n_kv_heads);
     const int kb = a.cache_shared ? 0 : b;
     const int key0 = rank * tpc * 128;                                           // first key of this CTA inside the range
@@ -550,7 +551,8 @@ score_onepass_tc_kernel(const ScoreTcArgs a, const int tpc, const uint32_t tmem_
     if (threadIdx.x < NP) {
         float2 st[S1_CLUSTER];
 #pragma unroll
-        for (int c = 0; c < S1_CLUSTER; ++c) st[c] = ld_cluster_f2(smem_u32(s_x + threadIdx.x), (uint32_t)c);
+        for (int c = 0; c < S1_CLUSTER; ++c)
+            st[c] = c < csize ? ld_cluster_f2(smem_u32(s_x + threadIdx.x), (uint32_t)c) : make_float2(-INFINITY, 0.f);
         float M = -INFINITY, Dn = 0.f;
 #pragma unroll
         for (int c = 0; c < S1_CLUSTER; ++c) M = fmaxf(M, st[c].x);
@@ -627,10 +629,17 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
     }
     static const bool onepass_on = [] { const char* e = getenv("ACACHE_SCORE_ONEPASS"); return !e || atoi(e) != 0; }();
     if (onepass_on && a.m <= 64) {
-        // the whole key range of a (head, request) over a cluster of eight CTAs, logits kept in tensor memory
+        // One pass, logits kept in tensor memory.  A (head, request) pair's key range is cut over a cluster of csize CTAs:
+        // as few as tensor memory allows (256 columns per CTA keep two CTAs on an SM) once the pairs alone fill the
+        // machine, more when there are few pairs (measured: at L = 512, B = 8 eight CTAs of half a tile each took 51 us
+        // where the two-pass kernels take 24).
         const int np = a.m <= 32 ? 32 : 64;
-        const int tpc = ((a.norm_len + S1_CLUSTER - 1) / S1_CLUSTER + 127) / 128;
-        if (tpc * np <= 512) {
+        const int tiles = (a.norm_len + 127) / 128;
+        int csize = 1;
+        while (csize < S1_CLUSTER && ((tiles + csize - 1) / csize) * np > 256) csize <<= 1;        // tensor memory
+        while (csize < S1_CLUSTER && csize * 2 <= tiles && (int64_t)a.n_heads * a.batch * csize < 2 * 148) csize <<= 1;   // fill
+        const int tpc = (tiles + csize - 1) / csize;
+        if (tpc * np <= 512 && tpc >= 2) {
             uint32_t cols = 32;
             while ((int)cols < tpc * np) cols <<= 1;
             const CUtensorMap* mq1 = get_map3(a.q_mask, a.m, a.n_heads * 128, a.batch, (int64_t)a.m * a.n_heads * 128, np);
@@ -649,11 +658,21 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
                 t1.n_split = 1; t1.cache_shared = shared ? 1 : 0;
                 t1.scale_log2e = 1.4426950408889634f / sqrtf(128.f);
                 t1.status = status;
-                const dim3 grid(a.n_heads * S1_CLUSTER, a.batch);
-                const size_t sm1 = cols > 256 ? (size_t)S1_SMEM_WIDE : (size_t)(np == 32 ? S1<32>::SMEM : S1<64>::SMEM);
+                cudaLaunchConfig_t cfg{};
+                cfg.gridDim = dim3(a.n_heads * csize, a.batch);
+                cfg.blockDim = dim3(S1_THREADS);
+                cfg.dynamicSmemBytes = cols > 256 ? (size_t)S1_SMEM_WIDE : (size_t)(np == 32 ? S1<32>::SMEM : S1<64>::SMEM);
+                cfg.stream = stream;
+                cudaLaunchAttribute at[2];
+                at[0].id = cudaLaunchAttributeClusterDimension;
+                at[0].val.clusterDim.x = csize; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                at[1].val.programmaticStreamSerializationAllowed = 1;
+                cfg.attrs = at;
+                cfg.numAttrs = 2;
                 const cudaError_t e1 = np == 32
-                    ? launch_pdl(score_onepass_tc_kernel<32>, grid, dim3(S1_THREADS), sm1, stream, t1, tpc, cols, map_q1, *mk)
-                    : launch_pdl(score_onepass_tc_kernel<64>, grid, dim3(S1_THREADS), sm1, stream, t1, tpc, cols, map_q1, *mk);
+                    ? cudaLaunchKernelEx(&cfg, score_onepass_tc_kernel<32>, t1, tpc, cols, csize, map_q1, *mk)
+                    : cudaLaunchKernelEx(&cfg, score_onepass_tc_kernel<64>, t1, tpc, cols, csize, map_q1, *mk);
                 return e1 == cudaSuccess ? 1 : -1;
             }
         }
