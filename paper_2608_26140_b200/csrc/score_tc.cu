@@ -638,8 +638,12 @@ int launch_score_tc(const ScoreArgs& a, uint32_t* status, cudaStream_t stream) {
         int csize = 1;
         while (csize < S1_CLUSTER && ((tiles + csize - 1) / csize) * np > 256) csize <<= 1;        // tensor memory
         while (csize < S1_CLUSTER && csize * 2 <= tiles && (int64_t)a.n_heads * a.batch * csize < 2 * 148) csize <<= 1;   // fill
+        // ACACHE_SCORE_CLUSTER = 1, 2, 4 or 8 forces the cluster size wherever tensor memory allows it (the tests run
+        // every size over the same cases, ragged and empty key ranges included)
+        static const int forced = [] { const char* e = getenv("ACACHE_SCORE_CLUSTER"); return e ? atoi(e) : 0; }();
+        if ((forced == 1 || forced == 2 || forced == 4 || forced == 8) && ((tiles + forced - 1) / forced) * np <= 512) csize = forced;
         const int tpc = (tiles + csize - 1) / csize;
-        if (tpc * np <= 512 && tpc >= 2) {
+        if (tpc * np <= 512 && (tpc >= 2 || forced)) {
             uint32_t cols = 32;
             while ((int)cols < tpc * np) cols <<= 1;
             const CUtensorMap* mq1 = get_map3(a.q_mask, a.m, a.n_heads * 128, a.batch, (int64_t)a.m * a.n_heads * 128, np);
