@@ -310,9 +310,9 @@ def run_ours(args):
     ms_e2e = float(np.median(blocks_e2e))
     sampler.stop_flag = True
     sampler.join()
-    # page-locked x is read in place: the kernels pull the masked rows, the anchor rows and the anchors' residual rows
-    x_in_place = ctx.host_x_in_place(xh) and (lay.n_masked + 2 * n) * 4 <= T    # the entry point's own rule
-    h2d = B * (lay.n_masked + 2 * n) * shape.hidden * 2 if x_in_place else xh.numel() * 2
+    # page-locked x is read in place: the kernels pull the masked rows and the recomputed rows, each once
+    x_in_place = ctx.host_x_in_place(xh) and (lay.n_masked + n) * 4 <= T    # the entry point's own rule
+    h2d = B * (lay.n_masked + n) * shape.hidden * 2 if x_in_place else xh.numel() * 2
     d2h = n * B * shape.hidden * 2 + B * K * 4 + B * L * 4
 
     if rank != 0:

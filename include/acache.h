@@ -462,9 +462,9 @@ acache_status acache_generate_block(acache_ctx *ctx, int32_t n_layers, const aca
  * asynchronous on `stream`; the caller synchronises the stream before reading.
  *   When x_host is page-locked (acache_host_x_in_place returns 1) and the step needs at most a quarter of
  *   its rows, it is not staged: the kernels read
- *   the rows the step needs (masked rows, anchor rows and the anchors' residual rows: n_masked + 2 (K+e)
- *   rows of D bf16 per request) in place over the bus, so x_host must stay valid and unchanged until the
- *   stream has passed this call. */
+ *   the rows the step needs (the masked rows and the K+e recomputed rows: n_masked + K + e rows of D bf16 per
+ *   request, each once) in place over the bus, so x_host must stay valid and unchanged until the
+ *   stream has passed this call.  Page-locked scores_host / anchor_idx_host are written by a copy kernel. */
 acache_status acache_layer_step_host(acache_ctx *ctx, const acache_layer_weights *w,
                                      const acache_request *req, acache_kv *kv,
                                      const void *x_host, double ratio, uint32_t flags,

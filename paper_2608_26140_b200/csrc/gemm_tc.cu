@@ -468,7 +468,8 @@ __device__ __forceinline__ int64_t prep_row_source(const GemmArgs& g, int row, b
 // out = bf16(x * rsqrt(mean(x^2) + eps) * g) for one row, by one warp: two passes over the row with
 // eight independent 16-byte loads in flight per lane (the second pass hits L1 / L2).
 __device__ __forceinline__ void rmsnorm_row_warp(const uint4* __restrict__ xr, const uint4* __restrict__ gn,
-                                                 uint4* __restrict__ out, int hidden, float eps, int lane) {
+                                                 uint4* __restrict__ out, int hidden, float eps, int lane,
+                                                 uint4* __restrict__ raw) {
     const int nchunk = hidden >> 3;
     float ss = 0.f;
     for (int c0 = 0; c0 < nchunk; c0 += 256) {
@@ -477,6 +478,7 @@ __device__ __forceinline__ void rmsnorm_row_warp(const uint4* __restrict__ xr, c
         for (int i = 0; i < 8; ++i) {
             const int c = c0 + i * 32 + lane;
             u[i] = c < nchunk ? __ldcg(xr + c) : make_uint4(0, 0, 0, 0);
+            if (raw && c < nchunk) raw[c] = u[i];
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -520,18 +522,21 @@ __device__ __forceinline__ void prep_phase(const GemmArgs& g, float* red, volati
     const RowPrep& rp = g.prep;
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(rp.x);
     __nv_bfloat16* a_out = static_cast<__nv_bfloat16*>(const_cast<void*>(g.a));
+    __nv_bfloat16* raw = static_cast<__nv_bfloat16*>(rp.raw_out);
     if (g.M <= (int)gridDim.x) {
         for (int row = blockIdx.x; row < g.M; row += gridDim.x) {
             const int64_t src = prep_row_source(g, row, threadIdx.x == 0);
             rmsnorm_row(reinterpret_cast<const uint4*>(x + src), reinterpret_cast<const uint4*>(rp.gain),
-                        reinterpret_cast<uint4*>(a_out + (int64_t)row * g.K), g.K, rp.eps, red);
+                        reinterpret_cast<uint4*>(a_out + (int64_t)row * g.K), g.K, rp.eps, red,
+                        raw ? reinterpret_cast<uint4*>(raw + (int64_t)row * g.K) : nullptr);
         }
     } else {
         const int nw = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
         for (int row = blockIdx.x * nw + warp; row < g.M; row += gridDim.x * nw) {
             const int64_t src = prep_row_source(g, row, lane == 0);
             rmsnorm_row_warp(reinterpret_cast<const uint4*>(x + src), reinterpret_cast<const uint4*>(rp.gain),
-                             reinterpret_cast<uint4*>(a_out + (int64_t)row * g.K), g.K, rp.eps, lane);
+                             reinterpret_cast<uint4*>(a_out + (int64_t)row * g.K), g.K, rp.eps, lane,
+                             raw ? reinterpret_cast<uint4*>(raw + (int64_t)row * g.K) : nullptr);
         }
     }
     asm volatile("fence.proxy.async;" ::: "memory");   // the rows are read back through TMA

@@ -54,6 +54,9 @@ void launch_row_mask(const int32_t* masked_pos, int m, const int32_t* extra_rows
 void launch_score_reduce_tiles(const float* partial, const uint32_t* rowmask, int rm_words, float* scores, int batch, int n_heads,
                                int q_tiles, int affix_len, int accumulate, cudaStream_t stream);
 
+// a_out[0, n_a) = a, b_out[0, n_b) = b (4-byte words); the outputs may be page-locked host memory seen from the device.
+void launch_copy_out_words(const void* a, void* a_out, int n_a, const void* b, void* b_out, int n_b, cudaStream_t stream);
+
 // ---- score.cu ---------------------------------------------------------------------------
 struct ScoreArgs {
     const void* q_mask;       // bf16 [B, m, H, d]
@@ -114,6 +117,7 @@ struct RowPrep {
     int affix_start, affix_len, ctx_len;
     const void* gain;
     float eps;
+    void* raw_out;            // optional bf16 [M, K]: the gathered rows as read (x far away, e.g. in host memory: read it once)
     int32_t* row_pos;
     int64_t* row_src;
 };

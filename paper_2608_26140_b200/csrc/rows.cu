@@ -342,6 +342,25 @@ void launch_row_mask(const int32_t* masked_pos, int m, const int32_t* extra_rows
     launch_pdl(row_mask_kernel, dim3(batch), dim3(256), smem, stream, masked_pos, m, extra_rows, e, k, rowmask, words, status);
 }
 
+// Two small results of a step (scores, anchor indices: 4-byte words) copied to page-locked host memory by plain
+// stores over the bus, one launch instead of two copy-engine transfers.
+__global__ void __launch_bounds__(256) copy_out_words_kernel(const uint32_t* __restrict__ a, uint32_t* __restrict__ a_out, int n_a,
+                                                             const uint32_t* __restrict__ b, uint32_t* __restrict__ b_out, int n_b) {
+    pdl_wait();
+    pdl_launch_dependents();
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_a + n_b; i += gridDim.x * blockDim.x) {
+        if (i < n_a) a_out[i] = a[i];
+        else b_out[i - n_a] = b[i - n_a];
+    }
+}
+
+void launch_copy_out_words(const void* a, void* a_out, int n_a, const void* b, void* b_out, int n_b, cudaStream_t stream) {
+    if (n_a + n_b <= 0) return;
+    const int blocks = (n_a + n_b + 255) / 256;
+    launch_pdl(copy_out_words_kernel, dim3(blocks < 148 ? blocks : 148), dim3(256), 0, stream, static_cast<const uint32_t*>(a),
+               static_cast<uint32_t*>(a_out), n_a, static_cast<const uint32_t*>(b), static_cast<uint32_t*>(b_out), n_b);
+}
+
 __global__ void __launch_bounds__(256) score_reduce_tiles_kernel(const float* __restrict__ partial,
                                                                  const uint32_t* __restrict__ rowmask, int rm_words,
                                                                  float* __restrict__ scores, int n_heads, int q_tiles, int L,

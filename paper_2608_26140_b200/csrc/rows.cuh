@@ -33,9 +33,10 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 // out = bf16(x * rsqrt(mean(x^2) + eps) * g) for one row of `hidden` bf16 values; all threads
-// of the block take part.
+// of the block take part.  raw (optional): the row as it was read is stored there too.
 __device__ __forceinline__ void rmsnorm_row(const uint4* __restrict__ xr, const uint4* __restrict__ g,
-                                            uint4* __restrict__ out, int hidden, float eps, float* red) {
+                                            uint4* __restrict__ out, int hidden, float eps, float* red,
+                                            uint4* __restrict__ raw = nullptr) {
     const int nchunk = hidden >> 3;
     if (nchunk <= 3 * (int)blockDim.x) {
         // the row fits in three 16-byte pieces per thread: one pass, the row stays in registers, and the gain is
@@ -51,6 +52,13 @@ __device__ __forceinline__ void rmsnorm_row(const uint4* __restrict__ xr, const 
         for (int i = 0; i < 3; ++i) {
             const int c = threadIdx.x + i * blockDim.x;
             gg[i] = c < nchunk ? g[c] : make_uint4(0u, 0u, 0u, 0u);
+        }
+        if (raw) {
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+                const int c = threadIdx.x + i * blockDim.x;
+                if (c < nchunk) raw[c] = u[i];
+            }
         }
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
@@ -77,6 +85,7 @@ __device__ __forceinline__ void rmsnorm_row(const uint4* __restrict__ xr, const 
     float ss = 0.f;
     for (int c = threadIdx.x; c < nchunk; c += blockDim.x) {
         uint4 u = __ldcg(xr + c);
+        if (raw) raw[c] = u;
         const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

@@ -306,29 +306,32 @@ def test_out_of_range_index_is_flagged_and_skipped():
     assert np.array_equal(ckb[0][keep], case.cache_k[0][keep])
 
 
-@pytest.mark.parametrize("extra,ratio", [("masked", 0.2),      # the step needs most of x: staged by one copy
-                                         ("none", 0.05)])      # 46 of 192 rows: page-locked x is read in place
-def test_host_buffer_entry_point(extra, ratio):
-    lay = wl.make_layout(2, 0, 128, 32, 32, 32, extra)
-    case = make_projected_case(wl.TINY, lay, ratio, cfg_id=17)
+@pytest.mark.parametrize("shape,L,extra,ratio", [
+    (wl.TINY, 128, "masked", 0.2),       # the step needs most of x: staged by one copy
+    (wl.TINY, 128, "none", 0.05),        # 38 of 192 rows: page-locked x is read in place, each row once
+    (MID128, 600, "all", 0.05),          # in place with request rows among the recomputed ones (their residual comes
+])                                       # from the device copy the row preparation leaves), head dimension 128
+def test_host_buffer_entry_point(shape, L, extra, ratio):
+    lay = wl.make_layout(2, 0, L, 32, 32, 32, extra)
+    case = make_projected_case(shape, lay, ratio, cfg_id=17)
     dc = DeviceCase(case)
     K, s_dev, a_dev, y_dev = run_layer_step(dc, ratio, ab.F_SCORE | ab.F_SELECT)
     n = K + lay.n_extra
     dc.reset_cache()
     xh = torch.from_numpy(case.x.view(np.int16)).view(torch.bfloat16).pin_memory()
-    sh = torch.zeros((2, 128), dtype=torch.float32).pin_memory()
+    sh = torch.zeros((2, L), dtype=torch.float32).pin_memory()
     ah = torch.zeros((2, K), dtype=torch.int32).pin_memory()
     yh = torch.zeros((2, n, case.shape.hidden), dtype=torch.bfloat16).pin_memory()
     dc.ctx.layer_step_host(dc.lw, dc.req, dc.kv(), xh, ratio, 0, sh, ah, yh)
     torch.cuda.synchronize()
     assert np.array_equal(sh.numpy(), s_dev) and np.array_equal(ah.numpy(), a_dev[:, :K])
     assert np.array_equal(ab.to_host_bits(yh), ab.to_host_bits(y_dev[:, :n]))
-    # page-locked x is read in place by the kernels, pageable x is staged by a copy: same results
+    # page-locked x is read in place by the kernels, pageable x is staged by a copy: same results; so are pageable outputs
     assert dc.ctx.host_x_in_place(xh)
     xp = torch.from_numpy(case.x.view(np.int16).copy()).view(torch.bfloat16)
     assert not dc.ctx.host_x_in_place(xp)
     dc.reset_cache()
-    sh2, ah2, yh2 = torch.zeros_like(sh), torch.zeros_like(ah), torch.zeros_like(yh)
+    sh2, ah2, yh2 = (torch.zeros(t.shape, dtype=t.dtype) for t in (sh, ah, yh))
     dc.ctx.layer_step_host(dc.lw, dc.req, dc.kv(), xp, ratio, 0, sh2, ah2, yh2)
     torch.cuda.synchronize()
     assert np.array_equal(sh2.numpy(), s_dev) and np.array_equal(ah2.numpy(), a_dev[:, :K])
