@@ -465,12 +465,55 @@ __device__ __forceinline__ int64_t prep_row_source(const GemmArgs& g, int row, b
     return src;
 }
 
-// out = bf16(x * rsqrt(mean(x^2) + eps) * g) for one row, by one warp: two passes over the row with
-// eight independent 16-byte loads in flight per lane (the second pass hits L1 / L2).
+// out = bf16(x * rsqrt(mean(x^2) + eps) * g) for one row, by one warp: rows of up to 4096 values in one pass from
+// registers; longer ones in two passes with eight independent 16-byte loads in flight per lane (the second pass hits
+// L1 / L2).
 __device__ __forceinline__ void rmsnorm_row_warp(const uint4* __restrict__ xr, const uint4* __restrict__ gn,
                                                  uint4* __restrict__ out, int hidden, float eps, int lane,
                                                  uint4* __restrict__ raw) {
     const int nchunk = hidden >> 3;
+    if (nchunk <= 512) {
+        // rows of up to 4096 values: one pass, the row stays in registers (sixteen 16-byte loads in flight per lane,
+        // one trip to memory per row instead of two), the gain is requested before the warp-wide sum
+        uint4 u[16];
+        float s1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int c = i * 32 + lane;
+            u[i] = c < nchunk ? __ldcg(xr + c) : make_uint4(0, 0, 0, 0);
+        }
+        if (raw) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int c = i * 32 + lane;
+                if (c < nchunk) raw[c] = u[i];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { const float a = bf16_lo(w[e]), b = bf16_hi(w[e]); s1 += a * a + b * b; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+        const float rstd1 = rsqrtf(s1 / (float)hidden + eps);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int c = i * 32 + lane;
+            if (c < nchunk) {
+                const uint4 gg = __ldg(gn + c);
+                const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+                const uint32_t gw[4] = {gg.x, gg.y, gg.z, gg.w};
+                uint32_t r[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    r[e] = pack_bf16(bf16_lo(w[e]) * rstd1 * bf16_lo(gw[e]), bf16_hi(w[e]) * rstd1 * bf16_hi(gw[e]));
+                out[c] = make_uint4(r[0], r[1], r[2], r[3]);
+            }
+        }
+        return;
+    }
     float ss = 0.f;
     for (int c0 = 0; c0 < nchunk; c0 += 256) {
         uint4 u[8];
@@ -532,11 +575,17 @@ __device__ __forceinline__ void prep_phase(const GemmArgs& g, float* red, volati
         }
     } else {
         const int nw = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-        for (int row = blockIdx.x * nw + warp; row < g.M; row += gridDim.x * nw) {
-            const int64_t src = prep_row_source(g, row, lane == 0);
+        // the source of the next row (index lookups: a dependent trip to memory) is asked for before this row is read
+        int row = blockIdx.x * nw + warp;
+        int64_t src = row < g.M ? prep_row_source(g, row, lane == 0) : 0;
+        while (row < g.M) {
+            const int next = row + gridDim.x * nw;
+            const int64_t src_next = next < g.M ? prep_row_source(g, next, lane == 0) : 0;
             rmsnorm_row_warp(reinterpret_cast<const uint4*>(x + src), reinterpret_cast<const uint4*>(rp.gain),
                              reinterpret_cast<uint4*>(a_out + (int64_t)row * g.K), g.K, rp.eps, lane,
                              raw ? reinterpret_cast<uint4*>(raw + (int64_t)row * g.K) : nullptr);
+            row = next;
+            src = src_next;
         }
     }
     asm volatile("fence.proxy.async;" ::: "memory");   // the rows are read back through TMA
