@@ -67,6 +67,33 @@ def test_score_anchors(shape, B, pre, L, post, m, norm_full):
     assert ctx.poll_status() == 0
 
 
+@pytest.mark.parametrize("L,m,norm_full", [(2300, 32, False),     # the one-pass tcgen05 kernel (ragged last tile)
+                                           (2300, 64, True),      # 64 columns per tile, all keys in the denominator
+                                           (2300, 130, False)])   # more than 64 masked rows: the two tcgen05 passes
+def test_score_anchors_over_a_cache_shared_by_the_batch(L, m, norm_full):
+    """batch_stride = 0 (Section 4.1: one copy of the affix K/V for every request) on the long-affix scoring kernels: every
+    request reads the same keys with its own masked rows."""
+    shape, B = MID128, 3
+    lay = wl.make_layout(B, 4, L, 30, max(m, 1), m)
+    T = lay.ctx_len
+    ck, _ = wl.random_kv_cache(shape, lay, 91)
+    q = wl.random_q_mask(shape, lay, 92)
+    ctx = ab.Context.for_shape(shape, B, T, L, 1, m, DEV)
+    dk = ab.to_device_bf16(ck[:1], DEV)                                   # one [T, Hkv, d] copy
+    dq = ab.to_device_bf16(q, DEV)
+    req = ab.Context.request(B, T, lay.affix_start, L, dev_i32(lay.masked_pos), None, None, None)
+    scores = torch.full((B, L), -1.0, dtype=torch.float32, device=DEV)
+    ctx.score_anchors(req, dq, ab.KV(dk.data_ptr(), dk.data_ptr(), 0, T), scores, accumulate=False, norm_full=norm_full)
+    torch.cuda.synchronize()
+    s_gpu = scores.cpu().numpy().astype(np.float64)
+    kf = orc.bf16_bits_to_f64(ck[0, :T])
+    for b in range(B):
+        ref = orc.score_anchors(orc.bf16_bits_to_f64(q[b]), kf[lay.affix_start:lay.affix_start + L], kf, lay.affix_start, norm_full)
+        err = np.abs(s_gpu[b] - ref) / np.maximum(ref, ref.mean())
+        assert err.max() < 1e-3, (b, err.max())
+    assert ctx.poll_status() == 0
+
+
 def test_score_is_bitwise_reproducible():
     shape, B, L, m = MID128, 2, 1000, 64
     lay = wl.make_layout(B, 0, L, 8, m, m)
