@@ -56,6 +56,8 @@ struct TcPlan {
     int pair_u;           // two-SM kernel, stream-K mode: (pair tile, K block) iterations per cluster (0: whole tiles)
     int m_pairs;          // 256-row tile rows of the two-SM kernel
     int units;            // 128-row B halves over all segments (non-SwiGLU) or ffn/128 (SwiGLU)
+    int group_n;          // two-SM kernel, whole tiles: weight tiles per group of the tile order
+    int w_keep;           // weights loaded with the evict-last policy (every row tile re-reads them from L2) instead of evict-first
 };
 
 // Which weight matrix and row the 128-row half `h` of N tile `nt` starts at; -1 if past the end.
@@ -811,19 +813,26 @@ constexpr int TC2_SMEM = TC2_STAGES * TC2_STAGE_BYTES + 1024 + 256;
 
 // Tile order of the two-SM kernel: groups of kTileGroupN weight tiles; inside a group the row
 // pairs are walked with the group's weight tiles innermost.  The ~74 clusters running at any
-// moment then cover about 9 row pairs x 8 weight tiles, whose A and B blocks (tens of MB) stay in
+// moment then cover a few row pairs x the group's weight tiles, whose A and B blocks (tens of MB) stay in
 // L2 while they are reused, instead of streaming the whole A matrix from HBM once per weight tile.
-constexpr int kTileGroupN = 8;
-__device__ __forceinline__ void tile_coords(int t, int m_pairs, int n_tiles, int& nt, int& mp) {
-    const int full = n_tiles / kTileGroupN, per_group = kTileGroupN * m_pairs;
+// With three or more row pairs the weight tiles are loaded with the evict-last policy like the rows: every row
+// pair re-reads them, and with evict-first (right for the few-row launches, whose weights pass through once) they
+// left L2 between two uses.  Measured on the 32-layer step of 14 752 rows per layer under the power cap: 209-216 ms
+// -> 191-197 ms at a 100-150 MHz higher SM clock (gate/up moved 8.6 GB through HBM per launch for 0.5 GB of
+// operands; the saved traffic is power the tensor cores get); groups of 16 weight tiles then beat 8 by 1-2 %
+// (4, 24, 32, 48 are slower), and cutting the row pairs into L2-sized blocks as well changes nothing more.
+constexpr int kTileGroupN = 16;
+constexpr int kKeepWeightsFromPairs = 3;
+__device__ __forceinline__ void tile_coords(int t, int m_pairs, int n_tiles, int group_n, int& nt, int& mp) {
+    const int full = n_tiles / group_n, per_group = group_n * m_pairs;
     if (t < full * per_group) {
         const int grp = t / per_group, r = t - grp * per_group;
-        mp = r / kTileGroupN;
-        nt = grp * kTileGroupN + (r - mp * kTileGroupN);
+        mp = r / group_n;
+        nt = grp * group_n + (r - mp * group_n);
     } else {
-        const int r = t - full * per_group, gn = n_tiles - full * kTileGroupN;
+        const int r = t - full * per_group, gn = n_tiles - full * group_n;
         mp = r / gn;
-        nt = full * kTileGroupN + (r - mp * gn);
+        nt = full * group_n + (r - mp * gn);
     }
 }
 
@@ -886,14 +895,15 @@ gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __gr
         int stage = 0, issued = 0;
         uint32_t phase = 0;
         bool ok = !*abort_flag;
-        const uint64_t pol_a = policy_evict_last(), pol_w = g.keep_weights ? pol_a : policy_evict_first();
+        const uint64_t pol_a = policy_evict_last();
+        const uint64_t pol_w = (g.keep_weights || p.w_keep) ? pol_a : policy_evict_first();
         // work list: whole tiles round-robin (pair_u == 0), or this cluster's contiguous range of
         // (tile, K block) iterations, tiles in weight-tile-major order (stream-K)
         const long long it_end = p.pair_u ? min((long long)(cluster_id + 1) * p.pair_u, (long long)tiles * p.KB) : 0;
         long long it = p.pair_u ? (long long)cluster_id * p.pair_u : 0;
         for (int t = p.pair_u ? (int)(it / p.KB) : cluster_id; ok && (p.pair_u ? it < it_end : t < tiles);) {
             int nt, mp;
-            if (p.pair_u) { nt = t / m_pairs; mp = t - nt * m_pairs; } else tile_coords(t, m_pairs, p.n_tiles, nt, mp);
+            if (p.pair_u) { nt = t / m_pairs; mp = t - nt * m_pairs; } else tile_coords(t, m_pairs, p.n_tiles, p.group_n, nt, mp);
             const int kb0 = p.pair_u ? (int)(it - (long long)t * p.KB) : 0;
             const int kb1 = p.pair_u ? (int)min((long long)p.KB, (long long)(kb0 + (it_end - it))) : p.KB;
             int brow;
@@ -961,7 +971,7 @@ gemm_tc2_kernel(const GemmArgs g, const TcPlan p, const int clusters, const __gr
         const uint64_t pol_p = policy_evict_last();
         for (int t = p.pair_u ? (int)(it / p.KB) : cluster_id; ok && (p.pair_u ? it < it_end : t < tiles);) {
             int nt, mp;
-            if (p.pair_u) { nt = t / m_pairs; mp = t - nt * m_pairs; } else tile_coords(t, m_pairs, p.n_tiles, nt, mp);
+            if (p.pair_u) { nt = t / m_pairs; mp = t - nt * m_pairs; } else tile_coords(t, m_pairs, p.n_tiles, p.group_n, nt, mp);
             const int kb0 = p.pair_u ? (int)(it - (long long)t * p.KB) : 0;
             const int kb1 = p.pair_u ? (int)min((long long)p.KB, (long long)(kb0 + (it_end - it))) : p.KB;
             const int grow = (mp * 2 + (int)rank) * TC_BM + row;
@@ -1283,6 +1293,9 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
         if (max_clusters < 1) goto single_cta;
         TcPlan pp = p;
         pp.m_pairs = m_pairs;
+        static const int group_n = [] { const char* e = getenv("ACACHE_GEMM_GROUP_N"); return e && atoi(e) > 0 ? atoi(e) : kTileGroupN; }();
+        pp.group_n = group_n;
+        static const int w_keep_from = [] { const char* e = getenv("ACACHE_GEMM_WKEEP_PAIRS"); return e ? atoi(e) : kKeepWeightsFromPairs; }();
         int clusters = std::min(std::min(max_clusters, sm_count() / 2), tiles);
         // measured: cutting tiles pays (partial tiles + finish kernel included) up to about two thirds of a wave
         static const int stream_k_pct = [] { const char* e = getenv("ACACHE_GEMM_PAIR_STREAMK_PCT"); return e ? atoi(e) : 66; }();
@@ -1306,6 +1319,7 @@ int launch_gemm(const GemmArgs& g, cudaStream_t stream) {
             }
             if (split.n >= 159) { pp.pair_u = 0; split.n = 0; clusters = std::min(std::min(max_clusters, sm_count() / 2), tiles); }
         }
+        pp.w_keep = (m_pairs >= w_keep_from && pp.pair_u == 0) ? 1 : 0;      // whole tiles, walked by three or more row pairs
         cfg.gridDim = dim3(clusters * 2);
         if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, g, pp, clusters, *mA, *mB[0], *mB[1], *mB[2]) != cudaSuccess) return -1;
         if (split.n == 0) return 1;
