@@ -263,7 +263,8 @@ score_colsum_tc_kernel(const ScoreTcArgs a, const int n_pad, const __grid_consta
     }
 
     if (warp == 0 && lane == 0) {
-        const uint64_t pol = policy_evict_first();
+        // the last read of the keys by this head; with grouped-query attention the other query heads of the KV head still want them
+        const uint64_t pol = a.n_heads == a.n_kv_heads ? policy_evict_first() : policy_evict_last();
         const uint64_t pol_q = policy_evict_last();
         mbar_expect_tx(bar(0), q_bytes);               // whole boxes of 128 rows, zero fill included
         for (int p = 0; p < 2; ++p)
@@ -431,7 +432,8 @@ score_onepass_tc_kernel(const ScoreTcArgs a, const int tpc, const uint32_t tmem_
     pdl_launch_dependents();
 
     if (warp == 0 && lane == 0) {
-        const uint64_t pol = policy_evict_first(), pol_q = policy_evict_last();
+        // the keys are read once per query head: with grouped-query attention the other heads of the KV head still want them
+        const uint64_t pol = a.n_heads == a.n_kv_heads ? policy_evict_first() : policy_evict_last(), pol_q = policy_evict_last();
         mbar_expect_tx(bar(0), 2 * NP * 128);                                    // two 64-column panels of NP rows
         tma3(sQ, &mapQ, h * 128, 0, b, bar(0), pol_q);
         tma3(sQ + NP * 128, &mapQ, h * 128 + 64, 0, b, bar(0), pol_q);
