@@ -135,6 +135,18 @@ struct AttnTcArgs {
     int score_norm_full;      // weight = 1 / the full denominator (Eq. 4 over every key) instead of the affix keys' share
 };
 
+// Wait for the two-query-tile kernel's threads whose hand-overs sit on the critical path of every key tile (the thread that
+// issues the tensor-core instructions, the softmax threads waiting for S): no sleep between polls (the many-row attention
+// went from 785 to 748 us on a 14 752-row layer; the one-tile kernel did not change); bounded like every wait.
+__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < (TC_WAIT_LIMIT << 4); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 4095u) == 4095u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
 __global__ void __launch_bounds__(AT_THREADS, 1)
 attention_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                     const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapKn,
@@ -597,8 +609,8 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
             }
             tc_commit(bar(9 + t));
         };
-        bool ok = mbar_wait(bar(0), 0, abort_flag);
-        if (ok && n_tiles > 0 && (ok = mbar_wait(bar(1), 0, abort_flag))) {
+        bool ok = mbar_spin(bar(0), 0, abort_flag);
+        if (ok && n_tiles > 0 && (ok = mbar_spin(bar(1), 0, abort_flag))) {
             tc_fence_after();
             for (int t = 0; t < n_sets; ++t) issue_s(t, 0);
             tc_commit(bar(3));                               // k_empty of stage 0
@@ -606,12 +618,12 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
         for (int j = 0; j < n_tiles && ok; ++j) {
             const int s = j & 1;
             const bool more = j + 1 < n_tiles;
-            if (!(ok = mbar_wait(bar(5 + s), (j >> 1) & 1, abort_flag))) break;                       // V of tile j landed
-            if (more && !(ok = mbar_wait(bar(1 + (s ^ 1)), ((j + 1) >> 1) & 1, abort_flag))) break;   // K of tile j + 1 landed
+            if (!(ok = mbar_spin(bar(5 + s), (j >> 1) & 1, abort_flag))) break;                       // V of tile j landed
+            if (more && !(ok = mbar_spin(bar(1 + (s ^ 1)), ((j + 1) >> 1) & 1, abort_flag))) break;   // K of tile j + 1 landed
             const uint32_t v = sV0 + s * AT_TILE;
             for (int t = 0; t < n_sets && ok; ++t) {
                 for (int hb = 0; hb < 2 && ok; ++hb) {
-                    if (!(ok = mbar_wait(bar(11 + 2 * t + hb), j & 1, abort_flag))) break;  // P of this half written, O rescaled
+                    if (!(ok = mbar_spin(bar(11 + 2 * t + hb), j & 1, abort_flag))) break;  // P of this half written, O rescaled
                     tc_fence_after();
 #pragma unroll
                     for (int k4 = 0; k4 < 4; ++k4) {
@@ -630,10 +642,10 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
         // the tensor pipe keeps one thread's instructions in order)
         for (int js = 0; js < n_sw && ok; ++js) {
             const int jj = n_tiles + js, s = jj & 1;
-            if (!(ok = mbar_wait(bar(1 + s), (jj >> 1) & 1, abort_flag))) break;
+            if (!(ok = mbar_spin(bar(1 + s), (jj >> 1) & 1, abort_flag))) break;
             const uint32_t k = sK0 + s * AT_TILE;
             for (int t = 0; t < n_sets && ok; ++t) {
-                if (js > 0 && !(ok = mbar_wait(bar(19 + t), (js - 1) & 1, abort_flag))) break;
+                if (js > 0 && !(ok = mbar_spin(bar(19 + t), (js - 1) & 1, abort_flag))) break;
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -690,7 +702,7 @@ attention_tc2q_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap ma
             const bool all = (keep[0] & keep[1]) == 0xffffffffu && (aff_all || aff_none);
             // warp-uniform: the tensor-memory accesses below are collective
             if (hb == 0) {
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar(9 + t), j & 1, abort_flag)))) break;
+                if (!(ok = __all_sync(0xffffffffu, mbar_spin(bar(9 + t), j & 1, abort_flag)))) break;
                 tc_fence_after();
             }
             float sv[2][32];
